@@ -1,0 +1,213 @@
+"""Pins for the oracle's scoring functions, losses and gradients: special cases the
+scoring-function table and the loss equations fix, numpy library routines, closed forms,
+and central finite differences in fp64."""
+import itertools
+
+import numpy as np
+import pytest
+
+from oracle.kge_oracle import make_config
+
+MODELS = [("transe", 1), ("transe", 2), ("transh", 1), ("transh", 2), ("rotate", 1), ("rotate", 2),
+          ("distmult", 1), ("complex", 1)]
+
+
+def _rows(rng, d, score):
+    h, t = rng.standard_normal(d), rng.standard_normal(d)
+    r = rng.uniform(-np.pi, np.pi, d // 2) if score == "rotate" else rng.standard_normal(d)
+    w = rng.standard_normal(d) if score == "transh" else None
+    return h, r, w, t
+
+
+def test_transe_zero_at_h_eq_t_r_zero_and_numpy_norms(oracle64):
+    rng = np.random.default_rng(0)
+    h = rng.standard_normal(16)
+    for p in (1, 2):
+        assert oracle64.score("transe", p, h, np.zeros(16), h) == 0.0
+        r, t = rng.standard_normal(16), rng.standard_normal(16)
+        assert oracle64.score("transe", p, h, r, t) == pytest.approx(-np.linalg.norm(h + r - t, ord=p), rel=1e-13)
+    # antisymmetric: swapping h and t changes the score when r != 0
+    assert oracle64.score("transe", 1, h, r, t) != pytest.approx(oracle64.score("transe", 1, t, r, h))
+
+
+def test_distmult_symmetry_and_einsum(oracle64):
+    rng = np.random.default_rng(1)
+    h, r, t = rng.standard_normal((3, 12))
+    f = oracle64.score("distmult", 1, h, r, t)
+    assert f == pytest.approx(oracle64.score("distmult", 1, t, r, h), rel=1e-13)
+    assert f == pytest.approx(np.einsum("k,k,k->", r, h, t), rel=1e-12)
+
+
+def test_complex_reduces_to_distmult_and_matches_numpy_complex(oracle64):
+    rng = np.random.default_rng(2)
+    d = 10
+    hr, rr, tr = rng.standard_normal((3, d // 2))
+    inter = lambda re, im: np.stack([re, im], 1).reshape(-1)
+    z = np.zeros(d // 2)
+    f = oracle64.score("complex", 1, inter(hr, z), inter(rr, z), inter(tr, z))
+    assert f == pytest.approx(oracle64.score("distmult", 1, hr, rr, tr), rel=1e-13)
+    hi, ri, ti = rng.standard_normal((3, d // 2))
+    hc, rc, tc = hr + 1j * hi, rr + 1j * ri, tr + 1j * ti
+    f = oracle64.score("complex", 1, inter(hr, hi), inter(rr, ri), inter(tr, ti))
+    assert f == pytest.approx(np.real(np.sum(rc * hc * np.conj(tc))), rel=1e-12)
+    # f(t, r, h) = f(h, conj r, t)
+    assert oracle64.score("complex", 1, inter(tr, ti), inter(rr, ri), inter(hr, hi)) == pytest.approx(
+        oracle64.score("complex", 1, inter(hr, hi), inter(rr, -ri), inter(tr, ti)), rel=1e-12)
+
+
+def test_rotate_special_phases_and_numpy_complex(oracle64):
+    rng = np.random.default_rng(3)
+    d = 12
+    h, t = rng.standard_normal(d), rng.standard_normal(d)
+    hc, tc = h[0::2] + 1j * h[1::2], t[0::2] + 1j * t[1::2]
+    zero = np.zeros(d // 2)
+    assert oracle64.score("rotate", 1, h, zero, t) == pytest.approx(-np.abs(hc - tc).sum(), rel=1e-13)
+    assert oracle64.score("rotate", 2, h, zero, t) == pytest.approx(-np.linalg.norm(h - t), rel=1e-13)
+    assert oracle64.score("rotate", 1, h, np.full(d // 2, np.pi), t) == pytest.approx(-np.abs(-hc - tc).sum(), rel=1e-12)
+    th = rng.uniform(-np.pi, np.pi, d // 2)
+    assert oracle64.score("rotate", 1, h, th, t) == pytest.approx(-np.abs(hc * np.exp(1j * th) - tc).sum(), rel=1e-12)
+    # L1 over moduli differs from the literal real L1 (|Re| + |Im|)
+    assert oracle64.score("rotate", 1, h, zero, t) != pytest.approx(-np.abs(h - t).sum())
+
+
+def test_transh_special_cases(oracle64):
+    rng = np.random.default_rng(4)
+    d = 9
+    h, r, w, t = rng.standard_normal((4, d))
+    what = w / np.linalg.norm(w)
+    for p in (1, 2):
+        # the definition, with numpy
+        x = (h - what @ h * what) + r - (t - what @ t * what)
+        assert oracle64.score("transh", p, h, r, t, w=w) == pytest.approx(-np.linalg.norm(x, ord=p), rel=1e-12)
+        # r = 0 and t = h + lambda w: both project to the same point
+        assert oracle64.score("transh", p, h, np.zeros(d), h + 2.5 * what, w=w) == pytest.approx(0.0, abs=1e-13)
+        # normal orthogonal to h, t: TransE
+        w2 = np.zeros(d); w2[0] = 3.0
+        h2, t2 = h.copy(), t.copy(); h2[0] = t2[0] = 0.0
+        assert oracle64.score("transh", p, h2, r, t2, w=w2) == pytest.approx(oracle64.score("transe", p, h2, r, t2), rel=1e-13)
+        # the scale of w does not matter
+        assert oracle64.score("transh", p, h, r, t, w=7 * w) == pytest.approx(oracle64.score("transh", p, h, r, t, w=w), rel=1e-12)
+
+
+def test_bf16_operand_variant_is_close_and_exact_on_bf16_inputs(oracle64):
+    rng = np.random.default_rng(5)
+    d = 64
+    for score in ("distmult", "complex"):
+        h, r, t = rng.standard_normal((3, d)) / np.sqrt(d)
+        f, fb = oracle64.score(score, 1, h, r, t), oracle64.score(score, 1, h, r, t, bf16=1)
+        assert fb != f and abs(fb - f) < 2e-2 * np.abs(np.stack([h * r, t])).max() * d ** 0.5
+    # inputs already representable in bf16 (small integers): both variants agree exactly
+    h, t = rng.integers(-8, 8, d).astype(float), rng.integers(-8, 8, d).astype(float)
+    r = np.ones(d)
+    assert oracle64.score("distmult", 1, h, r, t, bf16=1) == oracle64.score("distmult", 1, h, r, t)
+    assert oracle64.score("transe", 2, h, np.zeros(d), t, bf16=1) == pytest.approx(-np.linalg.norm(h - t), rel=1e-13)
+
+
+# ----------------------------------------------------------------------------- losses
+def test_sampled_softmax_uniform_scores_closed_forms(oracle64):
+    N, E = 37, 1000
+    base = dict(num_entities=E, num_relations=1, dim=4, score="distmult", loss="softmax", num_neg=N)
+    L, gpos, G = oracle64.row_loss(make_config(**base), 0.3, np.full(N, 0.3))
+    assert L == pytest.approx(np.log(N + 1), rel=1e-13)                      # c = 0
+    assert gpos + G.sum() == pytest.approx(0.0, abs=1e-14) and G == pytest.approx(1 / (N + 1))
+    L, _, _ = oracle64.row_loss(make_config(**base, ce_correction=np.log((E - 1) / N)), 0.3, np.full(N, 0.3))
+    assert L == pytest.approx(np.log(E), rel=1e-13)                          # the paper's c
+    # general scores against scipy-free numpy logsumexp, including large magnitudes
+    rng = np.random.default_rng(6)
+    F = rng.standard_normal(N) * 50
+    c = 1.7
+    L, gpos, G = oracle64.row_loss(make_config(**base, ce_correction=c), 2.0, F)
+    z = np.concatenate([[2.0], F + c])
+    lse = z.max() + np.log(np.exp(z - z.max()).sum())
+    assert L == pytest.approx(-2.0 + lse, rel=1e-12)
+    assert gpos + 1 + G.sum() == pytest.approx(1.0, rel=1e-12)
+
+
+def test_logsigmoid_closed_forms(oracle64):
+    N = 8
+    base = dict(num_entities=10, num_relations=1, dim=4, score="transe", loss="logsigmoid", num_neg=N)
+    L, gpos, G = oracle64.row_loss(make_config(**base, gamma=0.0, adv_temp=0.0), 0.0, np.zeros(N))
+    assert L == pytest.approx(2 * np.log(2), rel=1e-13)
+    assert gpos == pytest.approx(-0.5) and G == pytest.approx(np.full(N, 0.5 / N))
+    # definition with numpy, gamma and self-adversarial temperature on
+    rng = np.random.default_rng(7)
+    F = -np.abs(rng.standard_normal(N)) * 6
+    fpos, gamma, a = -3.0, 5.0, 0.7
+    L, gpos, G = oracle64.row_loss(make_config(**base, gamma=gamma, adv_temp=a), fpos, F)
+    sig = lambda z: 1 / (1 + np.exp(-z))
+    w = np.exp(a * F) / np.exp(a * F).sum()
+    assert L == pytest.approx(-np.log(sig(gamma + fpos)) - (w * np.log(sig(-gamma - F))).sum(), rel=1e-12)
+    assert G == pytest.approx(w * sig(gamma + F), rel=1e-12)
+    # a = 0: uniform weights; very negative argument stays finite
+    L, _, G = oracle64.row_loss(make_config(**base, gamma=0.0, adv_temp=0.0), -800.0, np.full(N, 800.0))
+    assert L == pytest.approx(1600.0, rel=1e-13) and np.isfinite(G).all()
+
+
+# ----------------------------------------------------------------------------- gradients
+def _tiny_problem(rng, score, E=7, R=3, d=4, B=3, N=5):
+    ent = rng.standard_normal((E, d)) * 0.7
+    rel = rng.uniform(-np.pi, np.pi, (R, d // 2)) if score == "rotate" else rng.standard_normal((R, d)) * 0.7
+    relw = rng.standard_normal((R, d)) if score == "transh" else None
+    # repeated rows on purpose: entity 2 is a head, a tail and a negative; relation 1 twice
+    heads = np.array([2, 0, 5], np.int32); rels = np.array([1, 1, 0], np.int32)
+    tails = np.array([3, 2, 6], np.int32); negs = np.array([2, 4, 4, 1, 6], np.int32)
+    return ent, rel, relw, heads, rels, tails, negs
+
+
+@pytest.mark.parametrize("score,p", MODELS)
+@pytest.mark.parametrize("loss", ["logsigmoid", "softmax"])
+def test_batch_grads_match_central_finite_differences(oracle64, score, p, loss):
+    rng = np.random.default_rng(100 * MODELS.index((score, p)) + len(loss))
+    ent, rel, relw, heads, rels, tails, negs = _tiny_problem(rng, score)
+    E, d = ent.shape
+    cfg = make_config(num_entities=E, num_relations=len(rel), dim=d, score=score, p_norm=p, loss=loss,
+                      batch=3, num_neg=5, gamma=1.5 if loss == "logsigmoid" else 0.0, adv_temp=0.8,
+                      ce_correction=0.4, loss_scale=0.5)
+    out = oracle64.batch_grads(cfg, ent, rel, relw, heads, rels, tails, negs)
+    base = oracle64.batch_loss(cfg, ent, rel, relw, heads, rels, tails, negs)
+    assert out["loss"] == pytest.approx(base["loss"], rel=1e-14)
+    # StopGrad: the self-adversarial weights are constants of the differentiation
+    w_fixed = None
+    if loss == "logsigmoid":
+        aF = cfg.adv_temp * base["F"]
+        w_fixed = np.exp(aF - aF.max(1, keepdims=True)); w_fixed /= w_fixed.sum(1, keepdims=True)
+    # analytic table gradients = scatter-add of the per-slot gradient rows
+    g_ent = np.zeros_like(ent); g_rel = np.zeros_like(rel)
+    np.add.at(g_ent, heads, out["dh"]); np.add.at(g_ent, tails, out["dtpos"]); np.add.at(g_ent, negs, out["dtneg"])
+    np.add.at(g_rel, rels, out["dr"])
+    g_w = None
+    if relw is not None:
+        g_w = np.zeros_like(relw); np.add.at(g_w, rels, out["dw"])
+
+    def loss_at(e, r, w):
+        return oracle64.batch_loss(cfg, e, r, w, heads, rels, tails, negs, w_fixed=w_fixed)["loss"]
+
+    eps = 1e-6
+    for name, tab, grad in (("ent", ent, g_ent), ("rel", rel, g_rel), ("relw", relw, g_w)):
+        if tab is None:
+            continue
+        for idx in itertools.product(range(tab.shape[0]), range(tab.shape[1])):
+            args = dict(ent=ent, rel=rel, relw=relw)
+            plus, minus = tab.copy(), tab.copy()
+            plus[idx] += eps; minus[idx] -= eps
+            args[name] = plus; lp = loss_at(args["ent"], args["rel"], args["relw"])
+            args[name] = minus; lm = loss_at(args["ent"], args["rel"], args["relw"])
+            fd = (lp - lm) / (2 * eps)
+            assert grad[idx] == pytest.approx(fd, rel=2e-6, abs=2e-8), (name, idx)
+    # untouched rows have zero gradient, touched tables do not vanish
+    assert np.abs(g_ent).sum() > 0 and np.abs(g_rel).sum() > 0
+    assert (g_rel[2] == 0).all()
+
+
+def test_subgradient_conventions_at_kinks(oracle64):
+    d = 4
+    h = np.array([1.0, -2.0, 0.5, 0.0]); r = np.zeros(d)
+    # L1: coordinates with zero residual get zero gradient
+    dh, dr, _, dt = oracle64.score_grad("transe", 1, 1.0, h, r, np.array([1.0, 0.0, 0.5, 3.0]))
+    assert (dh == np.array([0.0, 1.0, 0.0, 1.0])).all() and (dt == -dh).all() and (dr == dh).all()
+    # L2 / modulus at zero distance: zero gradient, no NaN
+    for score in ("transe", "rotate"):
+        rr = np.zeros(d // 2) if score == "rotate" else r
+        for p in (1, 2):
+            dh, _, _, dt = oracle64.score_grad(score, p, 1.0, h, rr, h)
+            assert (dh == 0).all() and (dt == 0).all()
