@@ -1,0 +1,224 @@
+/*
+ * kge.h -- C ABI of the B200 (sm_100a) library for the shared-negative scoring block of
+ * BESS-style knowledge-graph-embedding training and inference.
+ *
+ * Conventions for every entry point
+ * ---------------------------------
+ * - Memory: the caller owns ALL device memory (tables, optimiser state, workspace, every
+ *   id / output array).  The library owns only the host-side handle.  Unless a parameter
+ *   is marked [host], a pointer is a DEVICE pointer.
+ * - Streams: `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *   stream).  Calls enqueue work and return; only the entry points documented as
+ *   synchronising wait for the stream.
+ * - Errors: the return value is 0 (KGE_OK) or a negative kge_status.  Argument errors are
+ *   detected on the host before anything is launched.  Problems found on the device (an
+ *   id outside its table, a top-k candidate list that filled up) never trap: the kernel
+ *   records a code in a sticky status word inside the workspace, substitutes row 0 for the
+ *   offending id, and carries on; kge_get_status() reports and clears it.
+ * - Layouts: tables are row-major fp32 [rows, dim] with dim % 4 == 0 and 16-byte aligned
+ *   bases.  Complex rows (RotatE, ComplEx) are interleaved (re0, im0, re1, im1, ...), the
+ *   identification of C^(d/2) with R^d of the scoring-function table.  A RotatE relation
+ *   row holds dim/2 phases.  TransH keeps translations in `rel` and hyperplane normals in
+ *   `relw`, both [R, dim].  Adam state is [rows, 2*width] (first moment, then second
+ *   moment); row-wise Adagrad state is [rows]; SGD has none.
+ * - Determinism: every result is a pure function of the inputs; no floating-point atomics
+ *   are used anywhere.
+ */
+#ifndef KGE_H_
+#define KGE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kge_handle kge_handle; /* host-side object */
+
+/* Scoring functions: the table "Scoring functions" (Section 3.1). */
+typedef enum { KGE_TRANSE = 0, KGE_TRANSH = 1, KGE_ROTATE = 2, KGE_DISTMULT = 3, KGE_COMPLEX = 4 } kge_score_t;
+/* Loss functions: Section 3.1 "Loss Functions". */
+typedef enum { KGE_LOSS_LOGSIGMOID = 0, KGE_LOSS_SAMPLED_SOFTMAX = 1 } kge_loss_t;
+/* The paper names no optimiser; these are the textbook rules applied to touched rows only. */
+typedef enum { KGE_OPT_SGD = 0, KGE_OPT_ADAM = 1, KGE_OPT_ROWWISE_ADAGRAD = 2 } kge_opt_t;
+/* Arithmetic of the B x N score block (and of full-entity scoring). */
+typedef enum { KGE_PREC_FP32 = 0, KGE_PREC_BF16_TC = 1 } kge_prec_t;
+
+typedef enum {
+    KGE_OK = 0,
+    KGE_ERR_BAD_ARG = -1,        /* NULL / out-of-range argument, misaligned pointer */
+    KGE_ERR_DIVISIBILITY = -2,   /* B % P^2 (or B % P with head_part >= 0) or N % P != 0 */
+    KGE_ERR_EMPTY_BUCKET = -3,   /* a triple bucket T_{i,j} or entity partition E_j that must be sampled is empty */
+    KGE_ERR_WORKSPACE = -4,      /* workspace missing or smaller than kge_workspace_bytes() */
+    KGE_ERR_UNSUPPORTED = -5,    /* combination not implemented */
+    KGE_ERR_NOT_READY = -6,      /* tables not bound / graph not loaded */
+    KGE_ERR_CUDA = -7,           /* a CUDA runtime call failed (see kge_last_cuda_error) */
+    KGE_ERR_ID_RANGE = -8,       /* device: an entity / relation id was outside its table */
+    KGE_ERR_TOPK_OVERFLOW = -9,  /* device: a candidate list overflowed and could not be recovered */
+    KGE_ERR_NO_EXTENSION = -10   /* used by the Python binding when the shared library is missing */
+} kge_status;
+
+typedef struct {
+    int64_t num_entities;   /* |E| */
+    int64_t num_relations;  /* |R| */
+    int32_t dim;            /* d: floats per entity row; % 4 == 0, <= 512; even for RotatE / ComplEx */
+    int32_t score;          /* kge_score_t */
+    int32_t p_norm;         /* 1 or 2 (distance models; RotatE L1 = sum of complex moduli) */
+    int32_t loss;           /* kge_loss_t */
+    int32_t opt;            /* kge_opt_t */
+    int32_t prec;           /* kge_prec_t */
+    int32_t batch;          /* B positives per step */
+    int32_t num_neg;        /* N negatives shared by the whole batch (Eq. 4) */
+    int32_t num_parts;      /* P logical entity partitions, shard size S = ceil(|E| / P) */
+    int32_t head_part;      /* -1: slots spread evenly over all P*P buckets, bucket-major;
+                               i >= 0: the micro-batch B_i of Eq. 3 (all heads in partition i) */
+    int32_t sample_mode;    /* 0: cube-root relation law of Section 4 "Training"; 1: uniform over the bucket */
+    int32_t _reserved;
+    float gamma;            /* margin of the log-sigmoid loss */
+    float adv_temp;         /* a >= 0, self-adversarial temperature (0 = uniform weights 1/N) */
+    float ce_correction;    /* c of the sampled-softmax loss; the paper's value is log((|E|-1)/N) */
+    float loss_scale;       /* batch loss = loss_scale * sum_b L_b */
+    float lr;               /* default learning rate (kge_train_step takes one per call) */
+    float beta1, beta2;     /* Adam */
+    float eps;              /* Adam / Adagrad denominator epsilon */
+    uint64_t seed;          /* sampler seed (Philox key) */
+} kge_config;
+
+/* Validate the configuration and create the handle.  Allocates nothing on the device. */
+int kge_create(const kge_config* cfg /*[host]*/, kge_handle** out /*[host]*/);
+void kge_destroy(kge_handle* h);
+
+/* Bytes of device workspace needed for a graph of `num_triples` triples, inference batches
+ * of up to `max_queries` queries and top-`topk` lists.  Zero for either means "not used". */
+size_t kge_workspace_bytes(const kge_handle* h, int64_t num_triples, int32_t max_queries, int32_t topk);
+
+/*
+ * Attach caller-owned device memory.  ent [E, d]; rel [R, d] (RotatE [R, d/2]); relw [R, d]
+ * for TransH, else NULL; *_state as described above or NULL for SGD; workspace of at
+ * least kge_workspace_bytes() bytes, 256-byte aligned.  The workspace must be the one sized
+ * with the same (num_triples, max_queries, topk).  Zero-fills the workspace header
+ * asynchronously on `stream`.
+ */
+int kge_bind(kge_handle* h, float* ent, float* rel, float* relw,
+             float* ent_state, float* rel_state, float* relw_state,
+             void* workspace, size_t workspace_bytes,
+             int64_t num_triples, int32_t max_queries, int32_t topk, void* stream);
+
+/*
+ * Graph preprocessing (Section 4 "Partitioning"): logical partition part(e) = e div S,
+ * buckets T_{i,j} = {(h,r,t): part(h) = i, part(t) = j}; the triples are put in the
+ * canonical order "stable sort by (i, j, r)", with per-bucket relation offsets and the
+ * running sums of the integer cube-root weights w_r = floor((n_r * 2^60)^(1/3)), n_r counted
+ * inside the bucket.  h, r, t: [host] int32 arrays of length n.  The sorted copy lives in the
+ * workspace.  Synchronises `stream`.  KGE_ERR_EMPTY_BUCKET if a bucket or partition the
+ * sampler would need is empty; KGE_ERR_BAD_ARG if an id is out of range.
+ */
+int kge_graph_load(kge_handle* h, const int32_t* heads /*[host]*/, const int32_t* rels /*[host]*/,
+                   const int32_t* tails /*[host]*/, int64_t n, void* stream);
+
+/*
+ * Draw the batch of step `step` (Section 4 "Training", Eq. 3 and Eq. 4): B positives, with
+ * replacement, B/P^2 from every bucket (or B/P from each T_{i,j} of head_part i), the
+ * relation by p(r) ~ n_r^(1/3) and the triple uniform within (bucket, r); N negatives,
+ * N/P uniform entities from each partition E_j, shared by all positives.  Random words come
+ * from Philox4x32-10 with key = seed and counter = (slot, step lo, step hi, stream) where
+ * stream 0 draws positives and 1 negatives; a 64-bit word x maps to [0, n) as floor(x n / 2^64).
+ * Outputs: heads, rels, tails [B], negs [N] int32.
+ */
+int kge_sample_batch(kge_handle* h, uint64_t step, int32_t* heads, int32_t* rels, int32_t* tails,
+                     int32_t* negs, void* stream);
+
+/*
+ * One training step on one batch: gather rows, per-query vectors, positive scores, the
+ * B x N shared-negative score block (scoring-function table), the loss (log-sigmoid with
+ * self-adversarial weights under StopGrad, or sampled softmax with correction c), the
+ * backward pass, de-duplication of touched rows and the sparse row update.  All gradients
+ * are taken at the pre-step tables.  If heads/rels/tails/negs are all NULL the batch of
+ * `step` is sampled internally exactly as kge_sample_batch would.  `step` also drives Adam's
+ * bias correction (t = step + 1).  loss_out: one float, loss_scale * sum_b L_b (may be NULL).
+ */
+int kge_train_step(kge_handle* h, uint64_t step, float lr,
+                   const int32_t* heads, const int32_t* rels, const int32_t* tails, const int32_t* negs,
+                   float* loss_out, void* stream);
+
+/*
+ * The same step for callers that keep the batch on the host: ids are [host] arrays (pinned
+ * memory makes the copies asynchronous), copied in on `stream`; the loss is copied back to
+ * *loss_out [host] and the stream is synchronised before returning.
+ */
+int kge_train_step_host(kge_handle* h, uint64_t step, float lr,
+                        const int32_t* heads, const int32_t* rels, const int32_t* tails, const int32_t* negs,
+                        float* loss_out /*[host]*/, void* stream);
+
+/*
+ * Full-entity inference (Section 3.1 "Inference"): every query (h, r, ?) is scored against
+ * all |E| entities; out_ids / out_scores [nq, k] receive the k best tails ordered by
+ * (score descending, entity id ascending) -- unused places (k > |E|) hold id -1 and -inf.
+ * If true_tails is given, out_ranks[q] (int32) = 1 + number of entities ordered before the
+ * true tail under the same order; neither the head nor the true tail is filtered.  nq must
+ * not exceed the max_queries the workspace was sized for, k not its topk.
+ * Synchronises `stream` (candidate-list occupancy is checked between entity chunks).
+ */
+int kge_score_all_topk(kge_handle* h, const int32_t* q_heads, const int32_t* q_rels, int32_t nq, int32_t k,
+                       const int32_t* true_tails, int32_t* out_ids, float* out_scores, int32_t* out_ranks,
+                       void* stream);
+
+/*
+ * Mean reciprocal rank of the true tails (task metric of Section 2): mean over queries of
+ * 1/rank if rank <= k_cutoff else 0; k_cutoff = 10 is the paper's metric, 0 = no cut-off.
+ * mrr_out: [host] double.  Synchronises `stream`.
+ */
+int kge_eval_mrr(kge_handle* h, const int32_t* q_heads, const int32_t* q_rels, const int32_t* true_tails,
+                 int32_t nq, int32_t k_cutoff, double* mrr_out /*[host]*/, void* stream);
+
+/* Synchronise `stream`, return the sticky device status word (0 or a negative code), clear it. */
+int kge_get_status(kge_handle* h, void* stream);
+
+/* Kernels launched by this handle since creation (the library's own launches only). */
+int64_t kge_launch_count(const kge_handle* h);
+
+/*
+ * Per-stage device timing for the benchmark's roofline report (not part of the method).
+ * While enabled, kge_train_step brackets each of its launches with CUDA events on `stream`
+ * and synchronises the stream at the end of the step to accumulate the elapsed times.
+ * kge_profile_read copies the totals: ms[KGE_NUM_STAGES] and launches[KGE_NUM_STAGES]
+ * ([host] arrays), stages in the order of kge_stage_t; reset != 0 clears them.
+ */
+typedef enum {
+    KGE_STAGE_SAMPLE = 0, KGE_STAGE_BUILD, KGE_STAGE_BLOCK, KGE_STAGE_LOSS, KGE_STAGE_TH_CPASS,
+    KGE_STAGE_ACCUM_Q, KGE_STAGE_ACCUM_T, KGE_STAGE_CHAIN, KGE_STAGE_RANK, KGE_STAGE_SEGMENT,
+    KGE_STAGE_UPDATE, KGE_NUM_STAGES
+} kge_stage_t;
+int kge_profile(kge_handle* h, int enable);
+int kge_profile_read(kge_handle* h, double* ms /*[host]*/, int64_t* launches /*[host]*/, int reset);
+
+const char* kge_error_string(int code);
+const char* kge_last_cuda_error(const kge_handle* h);
+
+/*
+ * Parity taps (never on a timed path): copy an intermediate of the most recent
+ * kge_train_step to host memory.  Synchronises `stream`.  `bytes` must match exactly;
+ * kge_debug_bytes returns the size (0 if the tap does not exist for this configuration).
+ */
+typedef enum {
+    KGE_TAP_Q = 0,         /* [B, d] per-query vectors */
+    KGE_TAP_FPOS = 1,      /* [B] positive scores */
+    KGE_TAP_G = 2,         /* [B, N] dL/dF (for p = 2 distance models: dL/dF divided by the distance) */
+    KGE_TAP_GRAD_ENT = 3,  /* [2B+N, d] gradient rows of [heads | tails | negs] */
+    KGE_TAP_GRAD_REL = 4,  /* [B, k] relation gradient rows */
+    KGE_TAP_GRAD_RELW = 5, /* [B, d] TransH normal gradient rows */
+    KGE_TAP_ENT_UNIQ = 6,  /* [U] int32 distinct touched entity ids, ascending */
+    KGE_TAP_ENT_SEG = 7,   /* [U+1] int32 segment offsets into the permutation */
+    KGE_TAP_ENT_PERM = 8,  /* [2B+N] int32 source positions, stably sorted by id */
+    KGE_TAP_REL_UNIQ = 9, KGE_TAP_REL_SEG = 10, KGE_TAP_REL_PERM = 11,
+    KGE_TAP_LROW = 12,     /* [B] per-positive loss */
+    KGE_TAP_BATCH = 13     /* [3B+N] int32 heads | rels | tails | negs used by the step */
+} kge_tap_t;
+size_t kge_debug_bytes(kge_handle* h, int tap, void* stream);
+int kge_debug_export(kge_handle* h, int tap, void* dst /*[host]*/, size_t bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KGE_H_ */

@@ -1,0 +1,434 @@
+// Host side of the C ABI: handle, workspace layout, graph preprocessing, entry points.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "kge_common.cuh"
+
+using namespace kge;
+
+namespace {
+
+// Walks the caller's workspace in 256-byte steps; with base == nullptr it only measures.
+struct Carver {
+    char* base;
+    size_t used = 0;
+    explicit Carver(char* b) : base(b) {}
+    template <typename T>
+    T* take(size_t count) {
+        size_t bytes = (count * sizeof(T) + 255) / 256 * 256;
+        T* p = base ? reinterpret_cast<T*>(base + used) : nullptr;
+        used += bytes;
+        return p;
+    }
+};
+
+int pick_split(int rows, int cols, int num_sms) {
+    // One CTA covers 32 owner rows; aim for about two CTAs per SM, never splitting the
+    // reduced dimension into pieces shorter than 32.
+    int row_ctas = (rows + 31) / 32;
+    int want = (2 * num_sms + row_ctas - 1) / row_ctas;
+    int max_split = std::max(1, cols / 32);
+    return std::max(1, std::min(std::min(want, max_split), 16));
+}
+
+size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t topk, Workspace* out) {
+    const kge_config& c = h->cfg;
+    const size_t B = c.batch, N = c.num_neg, d = c.dim, kw = h->kw;
+    const size_t P = c.num_parts, R = c.num_relations;
+    const bool th = c.score == KGE_TRANSH;
+    Carver cv(base);
+    Workspace w{};
+    w.status = cv.take<int32_t>(64);
+    w.loss = reinterpret_cast<float*>(w.status ? w.status + 8 : nullptr);
+    w.counts = w.status ? w.status + 16 : nullptr;
+    w.gh = cv.take<int32_t>(T); w.gr = cv.take<int32_t>(T); w.gt = cv.take<int32_t>(T);
+    w.off = cv.take<int64_t>(P * P * (R + 1));
+    w.wcum = cv.take<uint64_t>(P * P * (R + 1));
+    w.heads = cv.take<int32_t>(3 * B + N);
+    if (w.heads) { w.rels = w.heads + B; w.tails = w.rels + B; w.negs = w.tails + B; }
+    w.Q = cv.take<float>(B * d);
+    w.What = th ? cv.take<float>(B * d) : nullptr;
+    w.Tneg = cv.take<float>(N * d);
+    w.fpos = cv.take<float>(B); w.gpos = cv.take<float>(B); w.Lrow = cv.take<float>(B);
+    w.F = cv.take<float>(B * N);
+    w.U = th ? cv.take<float>(B * N) : nullptr;
+    w.Cc = th ? cv.take<float>(B * N) : nullptr;
+    w.dQpart = cv.take<float>((size_t)h->split_q * B * d);
+    w.dWpart = th ? cv.take<float>((size_t)h->split_q * B * d) : nullptr;
+    w.dTpart = cv.take<float>((size_t)h->split_t * N * d);
+    w.grad_ent = cv.take<float>((2 * B + N) * d);
+    w.grad_rel = cv.take<float>(B * kw);
+    w.grad_relw = th ? cv.take<float>(B * d) : nullptr;
+    const size_t ne = 2 * B + N;
+    w.ent_perm = cv.take<int32_t>(ne); w.ent_sorted = cv.take<int32_t>(ne);
+    w.ent_uniq = cv.take<int32_t>(ne); w.ent_seg = cv.take<int32_t>(ne + 1);
+    w.rel_perm = cv.take<int32_t>(B); w.rel_sorted = cv.take<int32_t>(B);
+    w.rel_uniq = cv.take<int32_t>(B); w.rel_seg = cv.take<int32_t>(B + 1);
+    if (maxq > 0) {
+        const size_t q = maxq, k = std::max(topk, 1);
+        w.iq = cv.take<float>(q * d);
+        w.iwhat = th ? cv.take<float>(q * d) : nullptr;
+        w.iftrue = cv.take<float>(q);
+        w.thr = cv.take<float>(q); w.thr_id = cv.take<int32_t>(q);
+        w.cand_cnt = cv.take<int32_t>(q); w.beat_tmp = cv.take<int32_t>(q); w.beat = cv.take<int32_t>(q);
+        w.cand_score = cv.take<float>(q * kCandCap); w.cand_id = cv.take<int32_t>(q * kCandCap);
+        w.top_score = cv.take<float>(q * k); w.top_id = cv.take<int32_t>(q * k);
+    }
+    if (out) *out = w;
+    return cv.used;
+}
+
+// Largest w with w^3 <= n * 2^60 (0 for n = 0): integer cube-root sampling weight.
+uint64_t icbrt_weight(uint64_t n) {
+    if (n == 0) return 0;
+    const unsigned __int128 target = (unsigned __int128)n << 60;
+    uint64_t lo = 0, hi = (uint64_t)1 << 42;
+    while (lo < hi) {
+        uint64_t mid = lo + (hi - lo + 1) / 2;
+        if ((unsigned __int128)mid * mid * mid <= target) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+}  // namespace
+
+extern "C" {
+
+int kge_create(const kge_config* cfg, kge_handle** out) {
+    if (!cfg || !out) return KGE_ERR_BAD_ARG;
+    const kge_config& c = *cfg;
+    if (c.num_entities <= 0 || c.num_entities > INT32_MAX || c.num_relations <= 0 || c.num_relations > INT32_MAX)
+        return KGE_ERR_BAD_ARG;
+    if (c.dim <= 0 || c.dim % 4 != 0 || c.dim > kMaxDim) return KGE_ERR_BAD_ARG;
+    if (c.score < KGE_TRANSE || c.score > KGE_COMPLEX) return KGE_ERR_BAD_ARG;
+    if (c.p_norm != 1 && c.p_norm != 2) return KGE_ERR_BAD_ARG;
+    if (c.loss != KGE_LOSS_LOGSIGMOID && c.loss != KGE_LOSS_SAMPLED_SOFTMAX) return KGE_ERR_BAD_ARG;
+    if (c.opt < KGE_OPT_SGD || c.opt > KGE_OPT_ROWWISE_ADAGRAD) return KGE_ERR_BAD_ARG;
+    if (c.prec != KGE_PREC_FP32 && c.prec != KGE_PREC_BF16_TC) return KGE_ERR_BAD_ARG;
+    if (c.batch <= 0 || c.num_neg <= 0 || c.num_parts <= 0) return KGE_ERR_BAD_ARG;
+    if (c.head_part >= c.num_parts || c.head_part < -1) return KGE_ERR_BAD_ARG;
+    if (c.sample_mode != 0 && c.sample_mode != 1) return KGE_ERR_BAD_ARG;
+    if (!(c.adv_temp >= 0.f)) return KGE_ERR_BAD_ARG;
+    if ((int64_t)c.batch * c.num_neg > ((int64_t)1 << 31)) return KGE_ERR_BAD_ARG;
+    const int64_t P = c.num_parts;
+    if (c.num_neg % P != 0) return KGE_ERR_DIVISIBILITY;
+    if (c.head_part < 0 ? (c.batch % (P * P) != 0) : (c.batch % P != 0)) return KGE_ERR_DIVISIBILITY;
+    const int64_t S = (c.num_entities + P - 1) / P;
+    if (c.num_entities - (P - 1) * S <= 0) return KGE_ERR_EMPTY_BUCKET;  // last partition E_P would be empty
+    if (c.prec == KGE_PREC_BF16_TC) return KGE_ERR_UNSUPPORTED;
+    kge_handle* h = new (std::nothrow) kge_handle();
+    if (!h) return KGE_ERR_BAD_ARG;
+    h->cfg = c;
+    h->kw = c.score == KGE_ROTATE ? c.dim / 2 : c.dim;
+    h->kind = kind_of(c);
+    h->bound = h->graph_loaded = false;
+    h->launches = 0;
+    h->num_sms = 148;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+        h->num_sms = sms;
+    else
+        (void)cudaGetLastError();
+    h->split_q = pick_split(c.batch, c.num_neg, h->num_sms);
+    h->split_t = pick_split(c.num_neg, c.batch, h->num_sms);
+    *out = h;
+    return KGE_OK;
+}
+
+void kge_destroy(kge_handle* h) {
+    if (!h) return;
+    if (h->prof.created)
+        for (int i = 0; i < ST_COUNT; ++i) { cudaEventDestroy(h->prof.a[i]); cudaEventDestroy(h->prof.b[i]); }
+    delete h;
+}
+
+int kge_profile(kge_handle* h, int enable) {
+    if (!h) return KGE_ERR_BAD_ARG;
+    if (enable && !h->prof.created) {
+        for (int i = 0; i < ST_COUNT; ++i) {
+            KGE_CUDA_CHECK(h, cudaEventCreate(&h->prof.a[i]));
+            KGE_CUDA_CHECK(h, cudaEventCreate(&h->prof.b[i]));
+        }
+        h->prof.created = true;
+    }
+    h->prof.on = enable != 0;
+    return KGE_OK;
+}
+
+int kge_profile_read(kge_handle* h, double* ms, int64_t* launches, int reset) {
+    if (!h || !ms || !launches) return KGE_ERR_BAD_ARG;
+    for (int i = 0; i < ST_COUNT; ++i) {
+        ms[i] = h->prof.ms[i]; launches[i] = h->prof.n[i];
+        if (reset) { h->prof.ms[i] = 0.0; h->prof.n[i] = 0; }
+    }
+    return KGE_OK;
+}
+
+size_t kge_workspace_bytes(const kge_handle* h, int64_t num_triples, int32_t max_queries, int32_t topk) {
+    if (!h || num_triples < 0 || max_queries < 0 || topk < 0) return 0;
+    return layout(h, nullptr, num_triples, max_queries, topk, nullptr);
+}
+
+int kge_bind(kge_handle* h, float* ent, float* rel, float* relw, float* ent_state, float* rel_state,
+             float* relw_state, void* workspace, size_t workspace_bytes, int64_t num_triples,
+             int32_t max_queries, int32_t topk, void* stream) {
+    if (!h || !ent || !rel) return KGE_ERR_BAD_ARG;
+    if (h->cfg.score == KGE_TRANSH && !relw) return KGE_ERR_BAD_ARG;
+    if (h->cfg.opt != KGE_OPT_SGD && (!ent_state || !rel_state || (h->cfg.score == KGE_TRANSH && !relw_state)))
+        return KGE_ERR_BAD_ARG;
+    if (num_triples < 0 || max_queries < 0 || topk < 0 || topk > kCandCap) return KGE_ERR_BAD_ARG;
+    auto misaligned = [](const void* p, size_t a) { return p && (reinterpret_cast<uintptr_t>(p) % a) != 0; };
+    if (misaligned(ent, 16) || misaligned(rel, 16) || misaligned(relw, 16) || misaligned(ent_state, 16) ||
+        misaligned(rel_state, 16) || misaligned(relw_state, 16) || misaligned(workspace, 256))
+        return KGE_ERR_BAD_ARG;
+    if (!workspace || workspace_bytes < layout(h, nullptr, num_triples, max_queries, topk, nullptr))
+        return KGE_ERR_WORKSPACE;
+    h->ent = ent; h->rel = rel; h->relw = relw;
+    h->ent_state = ent_state; h->rel_state = rel_state; h->relw_state = relw_state;
+    h->ws_base = static_cast<char*>(workspace);
+    h->ws_bytes = workspace_bytes;
+    h->num_triples = num_triples; h->max_queries = max_queries; h->topk = topk;
+    layout(h, h->ws_base, num_triples, max_queries, topk, &h->ws);
+    KGE_CUDA_CHECK(h, cudaMemsetAsync(h->ws.status, 0, 256, static_cast<cudaStream_t>(stream)));
+    h->bound = true;
+    h->graph_loaded = false;
+    return KGE_OK;
+}
+
+int kge_graph_load(kge_handle* h, const int32_t* heads, const int32_t* rels, const int32_t* tails, int64_t n,
+                   void* stream) {
+    if (!h || !heads || !rels || !tails || n < 0) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    if (n != h->num_triples) return KGE_ERR_WORKSPACE;
+    const kge_config& c = h->cfg;
+    const int64_t E = c.num_entities, R = c.num_relations, P = c.num_parts;
+    const int64_t S = (E + P - 1) / P;
+    const int64_t nkeys = P * P * R;
+    std::vector<int64_t> start(nkeys + 1, 0);
+    for (int64_t e = 0; e < n; ++e) {
+        if (heads[e] < 0 || heads[e] >= E || tails[e] < 0 || tails[e] >= E || rels[e] < 0 || rels[e] >= R)
+            return KGE_ERR_BAD_ARG;
+        start[((heads[e] / S) * P + tails[e] / S) * R + rels[e] + 1] += 1;
+    }
+    for (int64_t k = 0; k < nkeys; ++k) start[k + 1] += start[k];
+    std::vector<int64_t> off(P * P * (R + 1));
+    std::vector<uint64_t> wcum(P * P * (R + 1));
+    for (int64_t b = 0; b < P * P; ++b) {
+        uint64_t acc = 0;
+        for (int64_t r = 0; r <= R; ++r) {
+            off[b * (R + 1) + r] = start[b * R + r];
+            wcum[b * (R + 1) + r] = acc;
+            if (r < R) acc += icbrt_weight((uint64_t)(start[b * R + r + 1] - start[b * R + r]));
+        }
+        const bool needed = c.head_part < 0 || b / P == c.head_part;
+        const bool empty = c.sample_mode == 0 ? acc == 0 : start[b * R + R] == start[b * R];
+        if (needed && empty) return KGE_ERR_EMPTY_BUCKET;
+    }
+    std::vector<int32_t> sh(n), sr(n), st(n);
+    std::vector<int64_t> cursor(start.begin(), start.end() - 1);
+    for (int64_t e = 0; e < n; ++e) {  // input order inside a key is kept: stable
+        int64_t dst = cursor[((heads[e] / S) * P + tails[e] / S) * R + rels[e]]++;
+        sh[dst] = heads[e]; sr[dst] = rels[e]; st[dst] = tails[e];
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    Workspace& w = h->ws;
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.gh, sh.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.gr, sr.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.gt, st.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.off, off.data(), off.size() * sizeof(int64_t), cudaMemcpyHostToDevice, s));
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.wcum, wcum.data(), wcum.size() * sizeof(uint64_t), cudaMemcpyHostToDevice, s));
+    KGE_CUDA_CHECK(h, cudaStreamSynchronize(s));
+    h->graph_loaded = true;
+    return KGE_OK;
+}
+
+int kge_sample_batch(kge_handle* h, uint64_t step, int32_t* heads, int32_t* rels, int32_t* tails, int32_t* negs,
+                     void* stream) {
+    if (!h || !heads || !rels || !tails || !negs) return KGE_ERR_BAD_ARG;
+    if (!h->bound || !h->graph_loaded) return KGE_ERR_NOT_READY;
+    return launch_sample(h, step, heads, rels, tails, negs, static_cast<cudaStream_t>(stream));
+}
+
+int kge_train_step(kge_handle* h, uint64_t step, float lr, const int32_t* heads, const int32_t* rels,
+                   const int32_t* tails, const int32_t* negs, float* loss_out, void* stream) {
+    if (!h) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    const int given = (heads != nullptr) + (rels != nullptr) + (tails != nullptr) + (negs != nullptr);
+    if (given != 0 && given != 4) return KGE_ERR_BAD_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    Workspace& w = h->ws;
+    if (given == 0) {
+        if (!h->graph_loaded) return KGE_ERR_NOT_READY;
+        int rc = launch_sample(h, step, w.heads, w.rels, w.tails, w.negs, s);
+        if (rc != KGE_OK) return rc;
+        heads = w.heads; rels = w.rels; tails = w.tails; negs = w.negs;
+    }
+    int rc = launch_forward_backward(h, heads, rels, tails, negs, s);
+    if (rc != KGE_OK) return rc;
+    rc = launch_dedup_update(h, step, lr, heads, rels, tails, negs, loss_out, s);
+    if (rc != KGE_OK) return rc;
+    return h->prof.on ? stage_collect(h, s) : KGE_OK;
+}
+
+int kge_train_step_host(kge_handle* h, uint64_t step, float lr, const int32_t* heads, const int32_t* rels,
+                        const int32_t* tails, const int32_t* negs, float* loss_out, void* stream) {
+    if (!h || !heads || !rels || !tails || !negs) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    Workspace& w = h->ws;
+    const size_t B = h->cfg.batch, N = h->cfg.num_neg;
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.heads, heads, B * 4, cudaMemcpyHostToDevice, s));
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.rels, rels, B * 4, cudaMemcpyHostToDevice, s));
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.tails, tails, B * 4, cudaMemcpyHostToDevice, s));
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.negs, negs, N * 4, cudaMemcpyHostToDevice, s));
+    int rc = kge_train_step(h, step, lr, w.heads, w.rels, w.tails, w.negs, w.loss, stream);
+    if (rc != KGE_OK) return rc;
+    if (loss_out) KGE_CUDA_CHECK(h, cudaMemcpyAsync(loss_out, w.loss, 4, cudaMemcpyDeviceToHost, s));
+    KGE_CUDA_CHECK(h, cudaStreamSynchronize(s));
+    return KGE_OK;
+}
+
+int kge_score_all_topk(kge_handle* h, const int32_t* q_heads, const int32_t* q_rels, int32_t nq, int32_t k,
+                       const int32_t* true_tails, int32_t* out_ids, float* out_scores, int32_t* out_ranks,
+                       void* stream) {
+    if (!h || !q_heads || !q_rels || !out_ids || !out_scores || nq < 0 || k <= 0) return KGE_ERR_BAD_ARG;
+    if (out_ranks && !true_tails) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    if (nq > h->max_queries || k > h->topk) return KGE_ERR_WORKSPACE;
+    if (nq == 0) return KGE_OK;
+    return run_score_all_topk(h, q_heads, q_rels, nq, k, true_tails, out_ids, out_scores, out_ranks,
+                              static_cast<cudaStream_t>(stream));
+}
+
+int kge_eval_mrr(kge_handle* h, const int32_t* q_heads, const int32_t* q_rels, const int32_t* true_tails,
+                 int32_t nq, int32_t k_cutoff, double* mrr_out, void* stream) {
+    if (!h || !q_heads || !q_rels || !true_tails || !mrr_out || nq <= 0 || k_cutoff < 0) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    if (nq > h->max_queries || h->topk < 1) return KGE_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    Workspace& w = h->ws;
+    // a k = 1 search whose lists are discarded; only the ranks are used
+    int rc = run_score_all_topk(h, q_heads, q_rels, nq, 1, true_tails, nullptr, nullptr, w.beat_tmp, s);
+    if (rc != KGE_OK) return rc;
+    std::vector<int32_t> ranks(nq);
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(ranks.data(), w.beat_tmp, nq * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    KGE_CUDA_CHECK(h, cudaStreamSynchronize(s));
+    double acc = 0.0;
+    for (int32_t q = 0; q < nq; ++q)
+        if (k_cutoff == 0 || ranks[q] <= k_cutoff) acc += 1.0 / (double)ranks[q];
+    *mrr_out = acc / nq;
+    return KGE_OK;
+}
+
+int kge_get_status(kge_handle* h, void* stream) {
+    if (!h) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int32_t word = 0;
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(&word, h->ws.status, 4, cudaMemcpyDeviceToHost, s));
+    KGE_CUDA_CHECK(h, cudaMemsetAsync(h->ws.status, 0, 4, s));
+    KGE_CUDA_CHECK(h, cudaStreamSynchronize(s));
+    return word;
+}
+
+}  // extern "C"
+
+namespace kge {
+int stage_collect(kge_handle* h, cudaStream_t s) {
+    KGE_CUDA_CHECK(h, cudaStreamSynchronize(s));
+    for (int i = 0; i < ST_COUNT; ++i) {
+        if (!h->prof.used[i]) continue;
+        float ms = 0.f;
+        KGE_CUDA_CHECK(h, cudaEventElapsedTime(&ms, h->prof.a[i], h->prof.b[i]));
+        h->prof.ms[i] += ms; h->prof.n[i] += 1; h->prof.used[i] = false;
+    }
+    return KGE_OK;
+}
+}  // namespace kge
+
+extern "C" {
+
+int64_t kge_launch_count(const kge_handle* h) { return h ? h->launches : 0; }
+
+const char* kge_error_string(int code) {
+    switch (code) {
+        case KGE_OK: return "ok";
+        case KGE_ERR_BAD_ARG: return "bad argument";
+        case KGE_ERR_DIVISIBILITY: return "batch / negatives not divisible by the partition count";
+        case KGE_ERR_EMPTY_BUCKET: return "a triple bucket or entity partition that must be sampled is empty";
+        case KGE_ERR_WORKSPACE: return "workspace missing, too small, or sized for other limits";
+        case KGE_ERR_UNSUPPORTED: return "combination not implemented";
+        case KGE_ERR_NOT_READY: return "tables not bound or graph not loaded";
+        case KGE_ERR_CUDA: return "CUDA runtime error";
+        case KGE_ERR_ID_RANGE: return "an entity or relation id was outside its table";
+        case KGE_ERR_TOPK_OVERFLOW: return "top-k candidate list overflow";
+        case KGE_ERR_NO_EXTENSION: return "CUDA extension not built";
+        default: return "unknown error";
+    }
+}
+
+const char* kge_last_cuda_error(const kge_handle* h) { return h ? h->cuda_err.c_str() : ""; }
+
+size_t kge_debug_bytes(kge_handle* h, int tap, void* stream) {
+    if (!h || !h->bound) return 0;
+    const kge_config& c = h->cfg;
+    const size_t B = c.batch, N = c.num_neg, d = c.dim;
+    int32_t counts[2] = {0, 0};
+    if (tap == KGE_TAP_ENT_UNIQ || tap == KGE_TAP_ENT_SEG || tap == KGE_TAP_REL_UNIQ || tap == KGE_TAP_REL_SEG) {
+        cudaStream_t s = static_cast<cudaStream_t>(stream);
+        if (cudaMemcpyAsync(counts, h->ws.counts, 8, cudaMemcpyDeviceToHost, s) != cudaSuccess) return 0;
+        if (cudaStreamSynchronize(s) != cudaSuccess) return 0;
+    }
+    switch (tap) {
+        case KGE_TAP_Q: return B * d * 4;
+        case KGE_TAP_FPOS: case KGE_TAP_LROW: return B * 4;
+        case KGE_TAP_G: return B * N * 4;
+        case KGE_TAP_GRAD_ENT: return (2 * B + N) * d * 4;
+        case KGE_TAP_GRAD_REL: return B * h->kw * 4;
+        case KGE_TAP_GRAD_RELW: return c.score == KGE_TRANSH ? B * d * 4 : 0;
+        case KGE_TAP_ENT_UNIQ: return (size_t)counts[0] * 4;
+        case KGE_TAP_ENT_SEG: return ((size_t)counts[0] + 1) * 4;
+        case KGE_TAP_ENT_PERM: return (2 * B + N) * 4;
+        case KGE_TAP_REL_UNIQ: return (size_t)counts[1] * 4;
+        case KGE_TAP_REL_SEG: return ((size_t)counts[1] + 1) * 4;
+        case KGE_TAP_REL_PERM: return B * 4;
+        case KGE_TAP_BATCH: return (3 * B + N) * 4;
+        default: return 0;
+    }
+}
+
+int kge_debug_export(kge_handle* h, int tap, void* dst, size_t bytes, void* stream) {
+    if (!h || !dst) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    const size_t want = kge_debug_bytes(h, tap, stream);
+    if (want == 0 || want != bytes) return KGE_ERR_BAD_ARG;
+    const Workspace& w = h->ws;
+    const void* src = nullptr;
+    switch (tap) {
+        case KGE_TAP_Q: src = w.Q; break;
+        case KGE_TAP_FPOS: src = w.fpos; break;
+        case KGE_TAP_LROW: src = w.Lrow; break;
+        case KGE_TAP_G: src = w.F; break;
+        case KGE_TAP_GRAD_ENT: src = w.grad_ent; break;
+        case KGE_TAP_GRAD_REL: src = w.grad_rel; break;
+        case KGE_TAP_GRAD_RELW: src = w.grad_relw; break;
+        case KGE_TAP_ENT_UNIQ: src = w.ent_uniq; break;
+        case KGE_TAP_ENT_SEG: src = w.ent_seg; break;
+        case KGE_TAP_ENT_PERM: src = w.ent_perm; break;
+        case KGE_TAP_REL_UNIQ: src = w.rel_uniq; break;
+        case KGE_TAP_REL_SEG: src = w.rel_seg; break;
+        case KGE_TAP_REL_PERM: src = w.rel_perm; break;
+        case KGE_TAP_BATCH: src = w.heads; break;
+        default: return KGE_ERR_BAD_ARG;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, s));
+    KGE_CUDA_CHECK(h, cudaStreamSynchronize(s));
+    return KGE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,174 @@
+// Shared declarations of the sm_100a KGE library: host handle, workspace layout, small
+// device helpers.  Internal to the library (the public surface is include/kge.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+
+#include "../../include/kge.h"
+
+namespace kge {
+
+constexpr int kMaxDim = 512;     // floats per entity row
+constexpr int kCandCap = 1024;   // top-k candidate slots per query between two selections
+
+// Arithmetic shape of a pair (query b, tail n) once the per-query vector q_b is built.
+enum Kind : int {
+    KIND_L1 = 0,     // TransE p=1:            -sum_k |q_k - t_k|
+    KIND_L2 = 1,     // TransE / RotatE p=2:   -sqrt(sum_k (q_k - t_k)^2)
+    KIND_CL1 = 2,    // RotatE p=1:            -sum_k |q_k - t_k| over complex moduli
+    KIND_DOT = 3,    // DistMult / ComplEx:    sum_k q_k t_k
+    KIND_TH_L1 = 4,  // TransH p=1:            x = (q - t) + (w.t) w per pair
+    KIND_TH_L2 = 5   // TransH p=2
+};
+
+inline Kind kind_of(const kge_config& c) {
+    switch (c.score) {
+        case KGE_TRANSE: return c.p_norm == 1 ? KIND_L1 : KIND_L2;
+        case KGE_ROTATE: return c.p_norm == 1 ? KIND_CL1 : KIND_L2;
+        case KGE_TRANSH: return c.p_norm == 1 ? KIND_TH_L1 : KIND_TH_L2;
+        default: return KIND_DOT;
+    }
+}
+
+// Device workspace, carved out of the caller's buffer by kge_bind.
+struct Workspace {
+    int32_t* status;       // [4] sticky status word + scratch flags
+    float* loss;           // [1]
+    int32_t* counts;       // [8]  U_ent, U_rel, ...
+    // graph (canonical order)
+    int32_t *gh, *gr, *gt; // [T]
+    int64_t* off;          // [P*P*(R+1)]
+    uint64_t* wcum;        // [P*P*(R+1)]
+    // batch
+    int32_t *heads, *rels, *tails, *negs;  // contiguous [3B+N]
+    float *Q, *What, *Tneg;                // [B,d], [B,d] (TransH), [N,d]
+    float *fpos, *gpos, *Lrow;             // [B]
+    float *F;                              // [B,N] scores, overwritten by dL/dF
+    float *U, *Cc;                         // [B,N] TransH: w.t and the S.w contraction
+    float *dQpart, *dWpart, *dTpart;       // [Sq,B,d], [Sq,B,d] (TransH), [St,N,d]
+    float *grad_ent, *grad_rel, *grad_relw;  // [2B+N,d], [B,kw], [B,d]
+    // dedup
+    int32_t *ent_perm, *ent_sorted, *ent_uniq, *ent_seg;  // [2B+N], [2B+N], [2B+N], [2B+N+1]
+    int32_t *rel_perm, *rel_sorted, *rel_uniq, *rel_seg;  // [B] ...
+    // inference
+    float *iq, *iwhat, *iftrue;            // [maxq,d], [maxq,d], [maxq]
+    float *thr;                            // [maxq] current k-th best score (-inf until the list is full)
+    int32_t *thr_id;                       // [maxq] its id
+    int32_t *cand_cnt, *beat_tmp, *beat;   // [maxq]
+    float *cand_score; int32_t *cand_id;   // [maxq, kCandCap]
+    float *top_score; int32_t *top_id;     // [maxq, topk] running lists
+};
+
+}  // namespace kge
+
+namespace kge {
+// Optional per-stage device timing (kge_profile): CUDA events around each launch.
+enum Stage : int {
+    ST_SAMPLE = 0, ST_BUILD, ST_BLOCK, ST_LOSS, ST_TH_CPASS, ST_ACCUM_Q, ST_ACCUM_T, ST_CHAIN,
+    ST_RANK, ST_SEGMENT, ST_UPDATE, ST_COUNT
+};
+struct StageTimer {
+    bool on = false, created = false;
+    cudaEvent_t a[ST_COUNT], b[ST_COUNT];
+    bool used[ST_COUNT] = {};
+    double ms[ST_COUNT] = {};
+    int64_t n[ST_COUNT] = {};
+};
+}  // namespace kge
+
+struct kge_handle {
+    kge_config cfg;
+    kge::StageTimer prof;
+    int kw;                 // floats per relation row
+    kge::Kind kind;
+    float *ent, *rel, *relw, *ent_state, *rel_state, *relw_state;
+    char* ws_base;
+    size_t ws_bytes;
+    kge::Workspace ws;
+    int64_t num_triples;
+    int32_t max_queries, topk;
+    int split_q, split_t;   // column splits of the two backward accumulations
+    bool bound, graph_loaded;
+    int64_t launches;
+    int num_sms;
+    std::string cuda_err;
+};
+
+namespace kge {
+
+#define KGE_CUDA_CHECK(h, expr)                                   \
+    do {                                                          \
+        cudaError_t e_ = (expr);                                  \
+        if (e_ != cudaSuccess) {                                  \
+            (h)->cuda_err = std::string(#expr) + ": " + cudaGetErrorString(e_); \
+            return KGE_ERR_CUDA;                                  \
+        }                                                         \
+    } while (0)
+
+#define KGE_LAUNCH_CHECK(h)                                       \
+    do {                                                          \
+        (h)->launches += 1;                                       \
+        cudaError_t e_ = cudaGetLastError();                      \
+        if (e_ != cudaSuccess) {                                  \
+            (h)->cuda_err = std::string("kernel launch: ") + cudaGetErrorString(e_); \
+            return KGE_ERR_CUDA;                                  \
+        }                                                         \
+    } while (0)
+
+inline void stage_begin(kge_handle* h, int id, cudaStream_t s) {
+    if (h->prof.on) { cudaEventRecord(h->prof.a[id], s); }
+}
+inline void stage_end(kge_handle* h, int id, cudaStream_t s) {
+    if (h->prof.on) { cudaEventRecord(h->prof.b[id], s); h->prof.used[id] = true; }
+}
+// Synchronises the stream and folds the recorded stage times into the running totals.
+int stage_collect(kge_handle* h, cudaStream_t s);
+
+// ---- launch wrappers implemented in the other translation units ----
+int launch_sample(kge_handle* h, uint64_t step, int32_t* heads, int32_t* rels, int32_t* tails, int32_t* negs,
+                  cudaStream_t s);
+int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* rels, const int32_t* tails,
+                            const int32_t* negs, cudaStream_t s);
+int launch_dedup_update(kge_handle* h, uint64_t step, float lr, const int32_t* heads, const int32_t* rels,
+                        const int32_t* tails, const int32_t* negs, float* loss_out, cudaStream_t s);
+int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int32_t nq, int32_t k,
+                       const int32_t* true_tails, int32_t* out_ids, float* out_scores, int32_t* out_ranks,
+                       cudaStream_t s);
+
+#ifdef __CUDACC__
+// ---- device helpers ----
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// Records `code` in the sticky status word unless one is already there.
+__device__ __forceinline__ void set_status(int32_t* status, int code) { atomicCAS(status, 0, code); }
+
+// Bounds-checked id: an id outside [0, rows) is reported and replaced by row 0.
+__device__ __forceinline__ int64_t checked_id(int32_t id, int64_t rows, int32_t* status) {
+    if (id < 0 || (int64_t)id >= rows) {
+        set_status(status, KGE_ERR_ID_RANGE);
+        return 0;
+    }
+    return id;
+}
+
+__device__ __forceinline__ float softplusf(float z) { return fmaxf(z, 0.f) + log1pf(expf(-fabsf(z))); }
+__device__ __forceinline__ float sigmoidf(float z) {
+    if (z >= 0.f) return 1.f / (1.f + expf(-z));
+    float e = expf(z);
+    return e / (1.f + e);
+}
+#endif
+
+}  // namespace kge

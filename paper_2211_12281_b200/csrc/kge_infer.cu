@@ -1,0 +1,388 @@
+// Full-entity inference (Section 3.1 "Inference"): every query is scored against every
+// entity; per query the k best tails under (score descending, id ascending) and the rank
+// of the true tail.  The entity table is streamed once, in chunks that grow geometrically;
+// inside a chunk a pair survives only if it beats the query's current k-th best, survivors
+// are appended to a per-query candidate list, and a selection step between chunks merges
+// them into the running top-k and tightens the threshold (the single-device analogue of the
+// per-worker top-K followed by a final top-K over the gathered candidates).
+//
+// fp32 arithmetic here is "canonical": per pair one accumulator, embedding index ascending,
+// rounding exactly where written (intrinsics keep the compiler from fusing anything else),
+// so that ties and near-ties order the same way on any implementation of the same recipe.
+#include <algorithm>
+#include <climits>
+#include <cmath>
+#include <vector>
+
+#include "kge_common.cuh"
+
+namespace kge {
+
+namespace {
+
+struct InferParams {
+    int nq, k, d, d4, score, kind;
+    int64_t E, R;
+    const float *ent, *rel, *relw;
+    const int32_t *qh, *qr, *tt;   // tt may be NULL
+    int64_t e_lo, e_hi;            // entity range of this launch
+    int q_tiles;
+    Workspace w;
+};
+
+// One canonical accumulation step over the 4 floats of a slice.
+template <int KIND>
+__device__ __forceinline__ void canon_update(float& acc, float4 q, float4 t) {
+    if (KIND == KIND_DOT) {
+        acc = __fmaf_rn(q.x, t.x, acc); acc = __fmaf_rn(q.y, t.y, acc);
+        acc = __fmaf_rn(q.z, t.z, acc); acc = __fmaf_rn(q.w, t.w, acc);
+    } else if (KIND == KIND_L1) {
+        acc = __fadd_rn(acc, fabsf(__fsub_rn(q.x, t.x))); acc = __fadd_rn(acc, fabsf(__fsub_rn(q.y, t.y)));
+        acc = __fadd_rn(acc, fabsf(__fsub_rn(q.z, t.z))); acc = __fadd_rn(acc, fabsf(__fsub_rn(q.w, t.w)));
+    } else if (KIND == KIND_L2) {
+        float x;
+        x = __fsub_rn(q.x, t.x); acc = __fmaf_rn(x, x, acc); x = __fsub_rn(q.y, t.y); acc = __fmaf_rn(x, x, acc);
+        x = __fsub_rn(q.z, t.z); acc = __fmaf_rn(x, x, acc); x = __fsub_rn(q.w, t.w); acc = __fmaf_rn(x, x, acc);
+    } else {  // KIND_CL1
+        float xr = __fsub_rn(q.x, t.x), xi = __fsub_rn(q.y, t.y);
+        acc = __fadd_rn(acc, __fsqrt_rn(__fmaf_rn(xr, xr, __fmul_rn(xi, xi))));
+        xr = __fsub_rn(q.z, t.z); xi = __fsub_rn(q.w, t.w);
+        acc = __fadd_rn(acc, __fsqrt_rn(__fmaf_rn(xr, xr, __fmul_rn(xi, xi))));
+    }
+}
+
+__device__ __forceinline__ float4 canon_th_x(float u, float4 w, float4 q, float4 t) {
+    return make_float4(__fmaf_rn(u, w.x, __fsub_rn(q.x, t.x)), __fmaf_rn(u, w.y, __fsub_rn(q.y, t.y)),
+                       __fmaf_rn(u, w.z, __fsub_rn(q.z, t.z)), __fmaf_rn(u, w.w, __fsub_rn(q.w, t.w)));
+}
+__device__ __forceinline__ void canon_th_acc(int kind, float& acc, float4 x) {
+    if (kind == KIND_TH_L1) {
+        acc = __fadd_rn(acc, fabsf(x.x)); acc = __fadd_rn(acc, fabsf(x.y));
+        acc = __fadd_rn(acc, fabsf(x.z)); acc = __fadd_rn(acc, fabsf(x.w));
+    } else {
+        acc = __fmaf_rn(x.x, x.x, acc); acc = __fmaf_rn(x.y, x.y, acc);
+        acc = __fmaf_rn(x.z, x.z, acc); acc = __fmaf_rn(x.w, x.w, acc);
+    }
+}
+__device__ __forceinline__ float canon_finish(int kind, float acc) {
+    if (kind == KIND_DOT) return acc;
+    if (kind == KIND_L2 || kind == KIND_TH_L2) return -__fsqrt_rn(acc);
+    return -acc;
+}
+
+__device__ __forceinline__ bool ordered_before(float fa, int32_t ia, float fb, int32_t ib) {
+    return fa > fb || (fa == fb && ia < ib);
+}
+
+// ------------------------------------------------------------------------------------------
+// query set-up: one thread per query builds q (and the TransH unit normal) sequentially,
+// scores the true tail, and resets the query's running state.
+// ------------------------------------------------------------------------------------------
+__global__ void query_setup_kernel(InferParams p) {
+    const int q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.nq) return;
+    const int d = p.d;
+    const float* h = p.ent + checked_id(p.qh[q], p.E, p.w.status) * d;
+    const int64_t rid = checked_id(p.qr[q], p.R, p.w.status);
+    float* qv = p.w.iq + (int64_t)q * d;
+    float* wh = p.score == KGE_TRANSH ? p.w.iwhat + (int64_t)q * d : nullptr;
+    if (p.score == KGE_TRANSE) {
+        const float* r = p.rel + rid * d;
+        for (int k = 0; k < d; ++k) qv[k] = __fadd_rn(h[k], r[k]);
+    } else if (p.score == KGE_DISTMULT) {
+        const float* r = p.rel + rid * d;
+        for (int k = 0; k < d; ++k) qv[k] = __fmul_rn(r[k], h[k]);
+    } else if (p.score == KGE_COMPLEX) {
+        const float* r = p.rel + rid * d;
+        for (int k = 0; k < d; k += 2) {
+            qv[k] = __fmaf_rn(r[k], h[k], -__fmul_rn(r[k + 1], h[k + 1]));
+            qv[k + 1] = __fmaf_rn(r[k], h[k + 1], __fmul_rn(r[k + 1], h[k]));
+        }
+    } else if (p.score == KGE_ROTATE) {
+        const float* th = p.rel + rid * (d / 2);
+        for (int k = 0; k < d; k += 2) {
+            const float cs = cosf(th[k / 2]), sn = sinf(th[k / 2]);
+            qv[k] = __fmaf_rn(h[k], cs, -__fmul_rn(h[k + 1], sn));
+            qv[k + 1] = __fmaf_rn(h[k], sn, __fmul_rn(h[k + 1], cs));
+        }
+    } else {  // TransH
+        const float* r = p.rel + rid * d;
+        const float* w = p.relw + rid * d;
+        float s = 0.f;
+        for (int k = 0; k < d; ++k) s = __fmaf_rn(w[k], w[k], s);
+        const float den = fmaxf(__fsqrt_rn(s), 1e-12f);
+        float a = 0.f;
+        for (int k = 0; k < d; ++k) { wh[k] = __fdiv_rn(w[k], den); a = __fmaf_rn(wh[k], h[k], a); }
+        for (int k = 0; k < d; ++k) qv[k] = __fadd_rn(__fmaf_rn(-a, wh[k], h[k]), r[k]);
+    }
+    if (p.tt) {
+        const float* t = p.ent + checked_id(p.tt[q], p.E, p.w.status) * d;
+        float acc = 0.f;
+        if (p.score == KGE_TRANSH) {
+            float u = 0.f;
+            for (int k = 0; k < d; ++k) u = __fmaf_rn(wh[k], t[k], u);
+            for (int k = 0; k < d; k += 4)
+                canon_th_acc(p.kind, acc, canon_th_x(u, *reinterpret_cast<const float4*>(wh + k),
+                                                     *reinterpret_cast<const float4*>(qv + k),
+                                                     *reinterpret_cast<const float4*>(t + k)));
+        } else {
+            for (int k = 0; k < d; k += 4) {
+                const float4 q4 = *reinterpret_cast<const float4*>(qv + k);
+                const float4 t4 = *reinterpret_cast<const float4*>(t + k);
+                if (p.kind == KIND_DOT) canon_update<KIND_DOT>(acc, q4, t4);
+                else if (p.kind == KIND_L1) canon_update<KIND_L1>(acc, q4, t4);
+                else if (p.kind == KIND_L2) canon_update<KIND_L2>(acc, q4, t4);
+                else canon_update<KIND_CL1>(acc, q4, t4);
+            }
+        }
+        p.w.iftrue[q] = canon_finish(p.kind, acc);
+    }
+    for (int j = 0; j < p.k; ++j) {
+        p.w.top_score[(int64_t)q * p.k + j] = -INFINITY;
+        p.w.top_id[(int64_t)q * p.k + j] = INT_MAX;
+    }
+    p.w.thr[q] = -INFINITY; p.w.thr_id[q] = INT_MAX;
+    p.w.cand_cnt[q] = 0; p.w.beat_tmp[q] = 0; p.w.beat[q] = 0;
+}
+
+// ------------------------------------------------------------------------------------------
+// score tile: 64 queries x 64 entities per CTA, 4 x 4 pairs per thread.  Consecutive CTAs
+// walk the query tiles of one entity tile, so an entity tile is fetched from HBM once and
+// served to the other query tiles by L2.
+// ------------------------------------------------------------------------------------------
+constexpr int IQ = 64, IE = 64, IKC = 32, ILD = IKC + 4;
+
+template <int KIND>
+__global__ void __launch_bounds__(256) score_tile_kernel(InferParams p) {
+    constexpr bool TH = KIND == KIND_TH_L1 || KIND == KIND_TH_L2;
+    __shared__ __align__(16) float Qs[IQ * ILD];
+    __shared__ __align__(16) float Ts[IE * ILD];
+    __shared__ __align__(16) float Ws[TH ? IQ * ILD : 4];
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int qt = blockIdx.x % p.q_tiles;
+    const int64_t et = blockIdx.x / p.q_tiles;
+    const int q0 = qt * IQ;
+    const int64_t e0 = p.e_lo + et * IE;
+    const int d4 = p.d4;
+    const float4* Qg = reinterpret_cast<const float4*>(p.w.iq);
+    const float4* Wg = reinterpret_cast<const float4*>(p.w.iwhat);
+    const float4* Tg = reinterpret_cast<const float4*>(p.ent);
+
+    float acc[4][4], u[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { acc[i][j] = 0.f; u[i][j] = 0.f; }
+    const int npass = TH ? 2 : 1;
+    for (int pass = 0; pass < npass; ++pass) {
+        const bool upass = TH && pass == 0;
+        for (int k0 = 0; k0 < p.d; k0 += IKC) {
+#pragma unroll
+            for (int it = 0; it < 2; ++it) {
+                const int idx = tid + 256 * it, row = idx >> 3, c4 = idx & 7;
+                const int gc = (k0 >> 2) + c4;
+                const bool kin = gc < d4;
+                float4 qv = make_float4(0.f, 0.f, 0.f, 0.f), tv = qv, wv = qv;
+                if (kin && q0 + row < p.nq) {
+                    qv = Qg[(int64_t)(q0 + row) * d4 + gc];
+                    if (TH) wv = Wg[(int64_t)(q0 + row) * d4 + gc];
+                }
+                if (kin && e0 + row < p.e_hi) tv = Tg[(e0 + row) * d4 + gc];
+                *reinterpret_cast<float4*>(&Qs[row * ILD + c4 * 4]) = qv;
+                *reinterpret_cast<float4*>(&Ts[row * ILD + c4 * 4]) = tv;
+                if (TH) *reinterpret_cast<float4*>(&Ws[row * ILD + c4 * 4]) = wv;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int kk = 0; kk < IKC; kk += 4) {
+                float4 qv[4], tv[4], wv[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    qv[i] = *reinterpret_cast<const float4*>(&Qs[(ty + 16 * i) * ILD + kk]);
+                    tv[i] = *reinterpret_cast<const float4*>(&Ts[(tx + 16 * i) * ILD + kk]);
+                    if (TH) wv[i] = *reinterpret_cast<const float4*>(&Ws[(ty + 16 * i) * ILD + kk]);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (!TH) {
+                            canon_update<TH ? KIND_L1 : KIND>(acc[i][j], qv[i], tv[j]);
+                        } else if (upass) {
+                            u[i][j] = __fmaf_rn(wv[i].x, tv[j].x, u[i][j]); u[i][j] = __fmaf_rn(wv[i].y, tv[j].y, u[i][j]);
+                            u[i][j] = __fmaf_rn(wv[i].z, tv[j].z, u[i][j]); u[i][j] = __fmaf_rn(wv[i].w, tv[j].w, u[i][j]);
+                        } else {
+                            canon_th_acc(KIND, acc[i][j], canon_th_x(u[i][j], wv[i], qv[i], tv[j]));
+                        }
+                    }
+            }
+            __syncthreads();
+        }
+    }
+    // epilogue: rank counting against the true tail, threshold filter into the candidate lists
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int q = q0 + ty + 16 * i;
+        const bool qin = q < p.nq;
+        float thr = 0.f, ft = 0.f; int32_t thr_id = 0, tt = 0;
+        if (qin) {
+            thr = p.w.thr[q]; thr_id = p.w.thr_id[q];
+            if (p.tt) { ft = p.w.iftrue[q]; tt = p.tt[q]; }
+        }
+        int beat = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t e = e0 + tx + 16 * j;
+            if (!qin || e >= p.e_hi) continue;
+            const float f = canon_finish(KIND, acc[i][j]);
+            if (p.tt && ordered_before(f, (int32_t)e, ft, tt)) ++beat;
+            if (ordered_before(f, (int32_t)e, thr, thr_id)) {
+                const int slot = atomicAdd(&p.w.cand_cnt[q], 1);
+                if (slot < kCandCap) {
+                    p.w.cand_score[(int64_t)q * kCandCap + slot] = f;
+                    p.w.cand_id[(int64_t)q * kCandCap + slot] = (int32_t)e;
+                } else {
+                    p.w.status[1] = 1;   // this chunk overflowed a list: the host redoes it in small pieces
+                }
+            }
+        }
+        // the 16 lanes sharing a query row are contiguous: one atomic per row and tile
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) beat += __shfl_xor_sync(0xffffffffu, beat, o);
+        if (tx == 0 && beat > 0) atomicAdd(&p.w.beat_tmp[q], beat);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// select: one CTA per query merges the running top-k with this chunk's candidates by a
+// bitonic sort in shared memory under (score descending, id ascending), commits the chunk's
+// rank count and resets the candidate list.
+// ------------------------------------------------------------------------------------------
+constexpr int SEL_THREADS = 128;
+constexpr int SEL_MAX = 2 * kCandCap;   // k <= kCandCap plus at most kCandCap candidates
+
+__global__ void __launch_bounds__(SEL_THREADS) select_kernel(InferParams p) {
+    __shared__ float ss[SEL_MAX];
+    __shared__ int32_t si[SEL_MAX];
+    const int q = blockIdx.x, tid = threadIdx.x;
+    const int cnt = min(p.w.cand_cnt[q], kCandCap);
+    const int total = p.k + cnt;
+    int n2 = 1;
+    while (n2 < total) n2 <<= 1;
+    for (int i = tid; i < n2; i += SEL_THREADS) {
+        float s = -INFINITY; int32_t id = INT_MAX;
+        if (i < p.k) { s = p.w.top_score[(int64_t)q * p.k + i]; id = p.w.top_id[(int64_t)q * p.k + i]; }
+        else if (i < total) { s = p.w.cand_score[(int64_t)q * kCandCap + i - p.k]; id = p.w.cand_id[(int64_t)q * kCandCap + i - p.k]; }
+        ss[i] = s; si[i] = id;
+    }
+    __syncthreads();
+    for (int size = 2; size <= n2; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            for (int t = tid; t < n2 / 2; t += SEL_THREADS) {
+                const int lo = 2 * t - (t & (stride - 1)), hi = lo + stride;
+                const bool up = (lo & size) == 0;   // "up" blocks end with the best element first
+                const float a = ss[lo], b = ss[hi]; const int32_t ia = si[lo], ib = si[hi];
+                const bool b_first = ordered_before(b, ib, a, ia);
+                if (b_first == up) { ss[lo] = b; si[lo] = ib; ss[hi] = a; si[hi] = ia; }
+            }
+            __syncthreads();
+        }
+    }
+    for (int i = tid; i < p.k; i += SEL_THREADS) {
+        p.w.top_score[(int64_t)q * p.k + i] = ss[i];
+        p.w.top_id[(int64_t)q * p.k + i] = si[i];
+    }
+    if (tid == 0) {
+        p.w.thr[q] = ss[p.k - 1]; p.w.thr_id[q] = si[p.k - 1];
+        p.w.beat[q] += p.w.beat_tmp[q];
+        p.w.beat_tmp[q] = 0; p.w.cand_cnt[q] = 0;
+    }
+}
+
+__global__ void reset_chunk_kernel(InferParams p) {
+    const int q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q < p.nq) { p.w.cand_cnt[q] = 0; p.w.beat_tmp[q] = 0; }
+    if (q == 0) p.w.status[1] = 0;
+}
+
+__global__ void finish_kernel(InferParams p, int32_t* out_ids, float* out_scores, int32_t* out_ranks) {
+    const int q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.nq) return;
+    if (out_ids)
+        for (int j = 0; j < p.k; ++j) {
+            const int32_t id = p.w.top_id[(int64_t)q * p.k + j];
+            out_ids[(int64_t)q * p.k + j] = id == INT_MAX ? -1 : id;
+            out_scores[(int64_t)q * p.k + j] = p.w.top_score[(int64_t)q * p.k + j];
+        }
+    if (out_ranks) out_ranks[q] = 1 + p.w.beat[q];
+}
+
+void launch_score_tiles(const InferParams& p, cudaStream_t s) {
+    const int64_t e_tiles = (p.e_hi - p.e_lo + IE - 1) / IE;
+    const unsigned grid = (unsigned)(e_tiles * p.q_tiles);
+    switch (p.kind) {
+        case KIND_L1: score_tile_kernel<KIND_L1><<<grid, 256, 0, s>>>(p); break;
+        case KIND_L2: score_tile_kernel<KIND_L2><<<grid, 256, 0, s>>>(p); break;
+        case KIND_CL1: score_tile_kernel<KIND_CL1><<<grid, 256, 0, s>>>(p); break;
+        case KIND_DOT: score_tile_kernel<KIND_DOT><<<grid, 256, 0, s>>>(p); break;
+        case KIND_TH_L1: score_tile_kernel<KIND_TH_L1><<<grid, 256, 0, s>>>(p); break;
+        default: score_tile_kernel<KIND_TH_L2><<<grid, 256, 0, s>>>(p); break;
+    }
+}
+
+}  // namespace
+
+int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int32_t nq, int32_t k,
+                       const int32_t* true_tails, int32_t* out_ids, float* out_scores, int32_t* out_ranks,
+                       cudaStream_t s) {
+    const kge_config& c = h->cfg;
+    InferParams p;
+    p.nq = nq; p.k = k; p.d = c.dim; p.d4 = c.dim / 4; p.score = c.score; p.kind = h->kind;
+    p.E = c.num_entities; p.R = c.num_relations;
+    p.ent = h->ent; p.rel = h->rel; p.relw = h->relw;
+    p.qh = qh; p.qr = qr; p.tt = true_tails;
+    p.q_tiles = (nq + IQ - 1) / IQ;
+    p.w = h->ws;
+    p.e_lo = 0; p.e_hi = 0;
+    const int qblocks = (nq + 127) / 128;
+    query_setup_kernel<<<qblocks, 128, 0, s>>>(p);
+    KGE_LAUNCH_CHECK(h);
+    KGE_CUDA_CHECK(h, cudaMemsetAsync(h->ws.status + 1, 0, 4, s));
+
+    // Chunk i covers as many entities as all chunks before it (the first: one candidate
+    // list's worth, since nothing is filtered yet), capped so a launch stays bounded.
+    const int64_t max_chunk = std::max<int64_t>(kCandCap, std::min<int64_t>((int64_t)1 << 22, (int64_t)0x7fffffff / p.q_tiles * IE / 2));
+    int64_t lo = 0;
+    while (lo < p.E) {
+        const int64_t len = std::min<int64_t>(std::min<int64_t>(std::max<int64_t>(lo, kCandCap), max_chunk), p.E - lo);
+        p.e_lo = lo; p.e_hi = lo + len;
+        launch_score_tiles(p, s);
+        KGE_LAUNCH_CHECK(h);
+        int32_t overflow = 0;
+        KGE_CUDA_CHECK(h, cudaMemcpyAsync(&overflow, h->ws.status + 1, 4, cudaMemcpyDeviceToHost, s));
+        KGE_CUDA_CHECK(h, cudaStreamSynchronize(s));
+        if (!overflow) {
+            select_kernel<<<nq, SEL_THREADS, 0, s>>>(p);
+            KGE_LAUNCH_CHECK(h);
+        } else {
+            // A list filled up (scores rising along the table): redo the chunk in pieces that
+            // cannot overflow, selecting after each.
+            reset_chunk_kernel<<<qblocks, 128, 0, s>>>(p);
+            KGE_LAUNCH_CHECK(h);
+            for (int64_t sub = lo; sub < lo + len; sub += kCandCap) {
+                p.e_lo = sub; p.e_hi = std::min<int64_t>(sub + kCandCap, lo + len);
+                launch_score_tiles(p, s);
+                KGE_LAUNCH_CHECK(h);
+                select_kernel<<<nq, SEL_THREADS, 0, s>>>(p);
+                KGE_LAUNCH_CHECK(h);
+            }
+        }
+        lo += len;
+    }
+    finish_kernel<<<qblocks, 128, 0, s>>>(p, out_ids, out_scores, out_ranks);
+    KGE_LAUNCH_CHECK(h);
+    KGE_CUDA_CHECK(h, cudaStreamSynchronize(s));
+    return KGE_OK;
+}
+
+}  // namespace kge

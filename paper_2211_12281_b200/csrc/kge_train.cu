@@ -1,0 +1,781 @@
+// Forward and backward of one shared-negative batch on CUDA cores (fp32):
+//   build    : gather rows, per-query vectors q_b, positive scores, staged negative rows
+//   block    : F[b,n] = f(q_b, t_n) for the whole B x N block (scoring-function table)
+//   loss     : per-positive loss and dL/dF (Section 3.1 "Loss Functions"), in place
+//   accum    : dQ_b = sum_n G_bn df/dq,  dT_n = sum_b G_bn df/dt  (owner computes, no atomics)
+//   chain    : positive pair, chain rule q -> (h, r, w), reduction of the column splits
+#include "kge_common.cuh"
+
+namespace kge {
+
+namespace {
+
+struct TrainParams {
+    int B, N, d, d4, kw;
+    int score, kind, loss;
+    float gamma, adv_temp, ce_c, loss_scale;
+    int64_t E, R;
+    const float *ent, *rel, *relw;
+    const int32_t *heads, *rels, *tails, *negs;
+    int split_q, split_t;
+    Workspace w;
+};
+
+__device__ __forceinline__ float4 f4zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+__device__ __forceinline__ float4 f4add(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
+__device__ __forceinline__ float4 f4sub(float4 a, float4 b) { return make_float4(a.x - b.x, a.y - b.y, a.z - b.z, a.w - b.w); }
+__device__ __forceinline__ float4 f4mul(float4 a, float4 b) { return make_float4(a.x * b.x, a.y * b.y, a.z * b.z, a.w * b.w); }
+__device__ __forceinline__ float4 f4scale(float s, float4 a) { return make_float4(s * a.x, s * a.y, s * a.z, s * a.w); }
+__device__ __forceinline__ float4 f4fma(float s, float4 a, float4 c) {
+    return make_float4(fmaf(s, a.x, c.x), fmaf(s, a.y, c.y), fmaf(s, a.z, c.z), fmaf(s, a.w, c.w));
+}
+__device__ __forceinline__ float f4dot(float4 a, float4 b) { return a.x * b.x + a.y * b.y + a.z * b.z + a.w * b.w; }
+__device__ __forceinline__ float sgnf(float x) { return (x > 0.f ? 1.f : 0.f) - (x < 0.f ? 1.f : 0.f); }
+__device__ __forceinline__ float4 f4sgn(float4 a) { return make_float4(sgnf(a.x), sgnf(a.y), sgnf(a.z), sgnf(a.w)); }
+
+constexpr int kMaxChunks = kMaxDim / 128;  // float4 chunks per lane when one warp owns a row
+
+// ------------------------------------------------------------------------------------------
+// build: one warp per row.  Warps [0, B) build q_b and f+_b; warps [B, B+N) stage t-_n.
+// ------------------------------------------------------------------------------------------
+
+// Per-lane contribution to the "distance accumulator" of a pair, for non-TransH kinds.
+__device__ __forceinline__ float pair_partial(int kind, float4 q, float4 t) {
+    if (kind == KIND_DOT) return f4dot(q, t);
+    const float4 x = f4sub(q, t);
+    if (kind == KIND_L1) return fabsf(x.x) + fabsf(x.y) + fabsf(x.z) + fabsf(x.w);
+    if (kind == KIND_CL1) return sqrtf(fmaf(x.x, x.x, x.y * x.y)) + sqrtf(fmaf(x.z, x.z, x.w * x.w));
+    return f4dot(x, x);
+}
+
+__global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (warp >= p.B + p.N) return;
+    const int d4 = p.d4;
+    if (warp >= p.B) {
+        const int n = warp - p.B;
+        const int64_t id = checked_id(p.negs[n], p.E, p.w.status);
+        const float4* src = reinterpret_cast<const float4*>(p.ent) + id * d4;
+        float4* dst = reinterpret_cast<float4*>(p.w.Tneg) + (int64_t)n * d4;
+        for (int c = lane; c < d4; c += 32) dst[c] = src[c];
+        return;
+    }
+    const int b = warp;
+    const int64_t hid = checked_id(p.heads[b], p.E, p.w.status);
+    const int64_t rid = checked_id(p.rels[b], p.R, p.w.status);
+    const int64_t tid = checked_id(p.tails[b], p.E, p.w.status);
+    const float4* hrow = reinterpret_cast<const float4*>(p.ent) + hid * d4;
+    const float4* trow = reinterpret_cast<const float4*>(p.ent) + tid * d4;
+    float4 h[kMaxChunks], t[kMaxChunks], q[kMaxChunks], wh[kMaxChunks];
+#pragma unroll
+    for (int i = 0; i < kMaxChunks; ++i) {
+        const int c = lane + 32 * i;
+        h[i] = c < d4 ? hrow[c] : f4zero();
+        t[i] = c < d4 ? trow[c] : f4zero();
+        q[i] = f4zero(); wh[i] = f4zero();
+    }
+    if (p.score == KGE_ROTATE) {
+        const float2* th = reinterpret_cast<const float2*>(p.rel) + rid * d4;  // d/2 phases = d4 float2
+#pragma unroll
+        for (int i = 0; i < kMaxChunks; ++i) {
+            const int c = lane + 32 * i;
+            if (c < d4) {
+                const float2 ph = th[c];
+                float s0, c0, s1, c1;
+                sincosf(ph.x, &s0, &c0); sincosf(ph.y, &s1, &c1);
+                q[i] = make_float4(h[i].x * c0 - h[i].y * s0, h[i].x * s0 + h[i].y * c0,
+                                   h[i].z * c1 - h[i].w * s1, h[i].z * s1 + h[i].w * c1);
+            }
+        }
+    } else {
+        const float4* rrow = reinterpret_cast<const float4*>(p.rel) + rid * d4;
+        float4 r[kMaxChunks];
+#pragma unroll
+        for (int i = 0; i < kMaxChunks; ++i) { const int c = lane + 32 * i; r[i] = c < d4 ? rrow[c] : f4zero(); }
+        if (p.score == KGE_TRANSE) {
+#pragma unroll
+            for (int i = 0; i < kMaxChunks; ++i) q[i] = f4add(h[i], r[i]);
+        } else if (p.score == KGE_DISTMULT) {
+#pragma unroll
+            for (int i = 0; i < kMaxChunks; ++i) q[i] = f4mul(r[i], h[i]);
+        } else if (p.score == KGE_COMPLEX) {
+#pragma unroll
+            for (int i = 0; i < kMaxChunks; ++i)
+                q[i] = make_float4(r[i].x * h[i].x - r[i].y * h[i].y, r[i].x * h[i].y + r[i].y * h[i].x,
+                                   r[i].z * h[i].z - r[i].w * h[i].w, r[i].z * h[i].w + r[i].w * h[i].z);
+        } else {  // TransH: unit normal, projected head plus translation
+            const float4* wrow = reinterpret_cast<const float4*>(p.relw) + rid * d4;
+            float nrm2 = 0.f;
+#pragma unroll
+            for (int i = 0; i < kMaxChunks; ++i) {
+                const int c = lane + 32 * i;
+                wh[i] = c < d4 ? wrow[c] : f4zero();
+                nrm2 += f4dot(wh[i], wh[i]);
+            }
+            const float inv = 1.f / fmaxf(sqrtf(warp_sum(nrm2)), 1e-12f);
+            float a = 0.f;
+#pragma unroll
+            for (int i = 0; i < kMaxChunks; ++i) { wh[i] = f4scale(inv, wh[i]); a += f4dot(wh[i], h[i]); }
+            a = warp_sum(a);
+#pragma unroll
+            for (int i = 0; i < kMaxChunks; ++i) q[i] = f4add(f4fma(-a, wh[i], h[i]), r[i]);
+        }
+    }
+    float4* qdst = reinterpret_cast<float4*>(p.w.Q) + (int64_t)b * d4;
+#pragma unroll
+    for (int i = 0; i < kMaxChunks; ++i) { const int c = lane + 32 * i; if (c < d4) qdst[c] = q[i]; }
+    float acc = 0.f;
+    if (p.score == KGE_TRANSH) {
+        float4* wdst = reinterpret_cast<float4*>(p.w.What) + (int64_t)b * d4;
+        float u = 0.f;
+#pragma unroll
+        for (int i = 0; i < kMaxChunks; ++i) {
+            const int c = lane + 32 * i;
+            if (c < d4) wdst[c] = wh[i];
+            u += f4dot(wh[i], t[i]);
+        }
+        u = warp_sum(u);
+#pragma unroll
+        for (int i = 0; i < kMaxChunks; ++i) {
+            const float4 x = f4fma(u, wh[i], f4sub(q[i], t[i]));
+            acc += p.kind == KIND_TH_L1 ? fabsf(x.x) + fabsf(x.y) + fabsf(x.z) + fabsf(x.w) : f4dot(x, x);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < kMaxChunks; ++i) acc += pair_partial(p.kind, q[i], t[i]);
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) {
+        float f = acc;
+        if (p.kind == KIND_L1 || p.kind == KIND_CL1 || p.kind == KIND_TH_L1) f = -acc;
+        else if (p.kind == KIND_L2 || p.kind == KIND_TH_L2) f = -sqrtf(acc);
+        p.w.fpos[b] = f;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// block: 64 x 64 pairs per CTA, 256 threads, 4 x 4 pairs per thread, the embedding axis
+// streamed through shared memory in slices of 32.  MODE 0 writes F (and U = w.t for TransH);
+// MODE 1 (TransH only) writes the contraction c_bn = sum_k S_bnk w_bk needed by the backward.
+// ------------------------------------------------------------------------------------------
+constexpr int TB = 64, TN = 64, KC = 32, LDS = KC + 4;
+
+template <int KIND>
+__device__ __forceinline__ void pair_update(float& acc, float4 q, float4 t) {
+    if (KIND == KIND_DOT) {
+        acc = fmaf(q.x, t.x, acc); acc = fmaf(q.y, t.y, acc); acc = fmaf(q.z, t.z, acc); acc = fmaf(q.w, t.w, acc);
+    } else if (KIND == KIND_L1) {
+        acc += fabsf(q.x - t.x); acc += fabsf(q.y - t.y); acc += fabsf(q.z - t.z); acc += fabsf(q.w - t.w);
+    } else if (KIND == KIND_L2) {
+        float x;
+        x = q.x - t.x; acc = fmaf(x, x, acc); x = q.y - t.y; acc = fmaf(x, x, acc);
+        x = q.z - t.z; acc = fmaf(x, x, acc); x = q.w - t.w; acc = fmaf(x, x, acc);
+    } else {  // KIND_CL1
+        float xr = q.x - t.x, xi = q.y - t.y;
+        acc += sqrtf(fmaf(xr, xr, xi * xi));
+        xr = q.z - t.z; xi = q.w - t.w;
+        acc += sqrtf(fmaf(xr, xr, xi * xi));
+    }
+}
+
+template <int KIND, int MODE>
+__global__ void __launch_bounds__(256) block_kernel(TrainParams p) {
+    constexpr bool TH = KIND == KIND_TH_L1 || KIND == KIND_TH_L2;
+    __shared__ __align__(16) float Qs[TB * LDS];
+    __shared__ __align__(16) float Ts[TN * LDS];
+    __shared__ __align__(16) float Ws[TH ? TB * LDS : 4];
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int b0 = blockIdx.y * TB, n0 = blockIdx.x * TN;
+    const int d4 = p.d4;
+    const float4* Qg = reinterpret_cast<const float4*>(p.w.Q);
+    const float4* Tg = reinterpret_cast<const float4*>(p.w.Tneg);
+    const float4* Wg = reinterpret_cast<const float4*>(p.w.What);
+
+    float acc[4][4], u[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { acc[i][j] = 0.f; u[i][j] = 0.f; }
+    if (TH && MODE == 1) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int b = b0 + ty + 16 * i, n = n0 + tx + 16 * j;
+                u[i][j] = (b < p.B && n < p.N) ? p.w.U[(int64_t)b * p.N + n] : 0.f;
+            }
+    }
+    const int npass = (TH && MODE == 0) ? 2 : 1;
+    for (int pass = 0; pass < npass; ++pass) {
+        const bool upass = TH && MODE == 0 && pass == 0;
+        for (int k0 = 0; k0 < p.d; k0 += KC) {
+#pragma unroll
+            for (int it = 0; it < 2; ++it) {
+                const int idx = tid + 256 * it, row = idx >> 3, c4 = idx & 7;
+                const int gc = (k0 >> 2) + c4;
+                const bool kin = gc < d4;
+                float4 qv = f4zero(), tv = f4zero(), wv = f4zero();
+                if (kin && b0 + row < p.B) {
+                    qv = Qg[(int64_t)(b0 + row) * d4 + gc];
+                    if (TH) wv = Wg[(int64_t)(b0 + row) * d4 + gc];
+                }
+                if (kin && n0 + row < p.N) tv = Tg[(int64_t)(n0 + row) * d4 + gc];
+                *reinterpret_cast<float4*>(&Qs[row * LDS + c4 * 4]) = qv;
+                *reinterpret_cast<float4*>(&Ts[row * LDS + c4 * 4]) = tv;
+                if (TH) *reinterpret_cast<float4*>(&Ws[row * LDS + c4 * 4]) = wv;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int kk = 0; kk < KC; kk += 4) {
+                float4 qv[4], tv[4], wv[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    qv[i] = *reinterpret_cast<const float4*>(&Qs[(ty + 16 * i) * LDS + kk]);
+                    tv[i] = *reinterpret_cast<const float4*>(&Ts[(tx + 16 * i) * LDS + kk]);
+                    if (TH) wv[i] = *reinterpret_cast<const float4*>(&Ws[(ty + 16 * i) * LDS + kk]);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (!TH) {
+                            pair_update<TH ? KIND_L1 : KIND>(acc[i][j], qv[i], tv[j]);
+                        } else if (upass) {
+                            u[i][j] = fmaf(wv[i].x, tv[j].x, u[i][j]); u[i][j] = fmaf(wv[i].y, tv[j].y, u[i][j]);
+                            u[i][j] = fmaf(wv[i].z, tv[j].z, u[i][j]); u[i][j] = fmaf(wv[i].w, tv[j].w, u[i][j]);
+                        } else {
+                            const float4 x = f4fma(u[i][j], wv[i], f4sub(qv[i], tv[j]));
+                            if (MODE == 0) {
+                                if (KIND == KIND_TH_L1) acc[i][j] += fabsf(x.x) + fabsf(x.y) + fabsf(x.z) + fabsf(x.w);
+                                else acc[i][j] += f4dot(x, x);
+                            } else {
+                                if (KIND == KIND_TH_L1) acc[i][j] += f4dot(f4sgn(x), wv[i]);
+                                else acc[i][j] += f4dot(x, wv[i]);
+                            }
+                        }
+                    }
+            }
+            __syncthreads();
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int b = b0 + ty + 16 * i, n = n0 + tx + 16 * j;
+            if (b >= p.B || n >= p.N) continue;
+            const int64_t o = (int64_t)b * p.N + n;
+            if (MODE == 1) {
+                p.w.Cc[o] = -p.w.F[o] * acc[i][j];   // F holds G (p=1) or G / distance (p=2) by now
+            } else {
+                float f = acc[i][j];
+                if (KIND == KIND_L1 || KIND == KIND_CL1 || KIND == KIND_TH_L1) f = -f;
+                else if (KIND == KIND_L2 || KIND == KIND_TH_L2) f = -sqrtf(f);
+                p.w.F[o] = f;
+                if (TH) p.w.U[o] = u[i][j];
+            }
+        }
+}
+
+// ------------------------------------------------------------------------------------------
+// loss: one CTA per positive.  Overwrites F[b,:] with loss_scale * dL_b/dF_bn (divided by the
+// distance for p = 2 kinds, which is the factor every later use needs).
+// ------------------------------------------------------------------------------------------
+constexpr int LOSS_THREADS = 128;
+
+__device__ __forceinline__ float block_sum(float v, float* sm) {
+    v = warp_sum(v);
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    __syncthreads();
+    if (lane == 0) sm[w] = v;
+    __syncthreads();
+    float t = 0.f;
+    for (int i = 0; i < LOSS_THREADS / 32; ++i) t += sm[i];
+    return t;
+}
+__device__ __forceinline__ float block_max(float v, float* sm) {
+    v = warp_max(v);
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    __syncthreads();
+    if (lane == 0) sm[w] = v;
+    __syncthreads();
+    float t = sm[0];
+    for (int i = 1; i < LOSS_THREADS / 32; ++i) t = fmaxf(t, sm[i]);
+    return t;
+}
+
+__global__ void __launch_bounds__(LOSS_THREADS) loss_kernel(TrainParams p) {
+    __shared__ float sm[LOSS_THREADS / 32];
+    const int b = blockIdx.x, tid = threadIdx.x;
+    float* Frow = p.w.F + (int64_t)b * p.N;
+    const float fp = p.w.fpos[b];
+    const bool l2 = p.kind == KIND_L2 || p.kind == KIND_TH_L2;
+    const float ls = p.loss_scale;
+    if (p.loss == KGE_LOSS_LOGSIGMOID) {
+        const float a = p.adv_temp, gamma = p.gamma;
+        float m = 0.f, z = (float)p.N;
+        if (a > 0.f) {
+            float lm = -INFINITY;
+            for (int n = tid; n < p.N; n += LOSS_THREADS) lm = fmaxf(lm, a * Frow[n]);
+            m = block_max(lm, sm);
+            float lz = 0.f;
+            for (int n = tid; n < p.N; n += LOSS_THREADS) lz += expf(a * Frow[n] - m);
+            z = block_sum(lz, sm);
+        }
+        float lacc = 0.f;
+        for (int n = tid; n < p.N; n += LOSS_THREADS) {
+            const float f = Frow[n];
+            const float w = a > 0.f ? expf(a * f - m) / z : 1.f / z;
+            lacc += w * softplusf(gamma + f);
+            float g = ls * w * sigmoidf(gamma + f);
+            if (l2) g = f < 0.f ? g / -f : 0.f;
+            Frow[n] = g;
+        }
+        const float lsum = block_sum(lacc, sm);
+        if (tid == 0) {
+            p.w.Lrow[b] = softplusf(-(gamma + fp)) + lsum;
+            p.w.gpos[b] = -ls * sigmoidf(-(gamma + fp));
+        }
+    } else {
+        const float c = p.ce_c;
+        float lm = -INFINITY;
+        for (int n = tid; n < p.N; n += LOSS_THREADS) lm = fmaxf(lm, Frow[n] + c);
+        const float m = fmaxf(block_max(lm, sm), fp);
+        float lz = 0.f;
+        for (int n = tid; n < p.N; n += LOSS_THREADS) lz += expf(Frow[n] + c - m);
+        const float epos = expf(fp - m);
+        const float z = block_sum(lz, sm) + epos;
+        for (int n = tid; n < p.N; n += LOSS_THREADS) {
+            const float f = Frow[n];
+            float g = ls * expf(f + c - m) / z;
+            if (l2) g = f < 0.f ? g / -f : 0.f;
+            Frow[n] = g;
+        }
+        if (tid == 0) {
+            p.w.Lrow[b] = -fp + (m + logf(z));
+            p.w.gpos[b] = ls * (epos / z - 1.f);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// accum: out[r, :] = sum over the other side c of weight(r, c) * d f / d(owner row), for 32
+// owner rows per CTA (4 per warp, a lane owns NCH float4 slices of the row) and one column
+// split per blockIdx.y.  OWNER_Q: owner = queries (weights G[r, c]); else owner = negative
+// tails (weights G[c, r]).  The sum runs over c ascending inside a split; the splits are
+// added in ascending order by the chain kernel, so the result does not depend on timing.
+// ------------------------------------------------------------------------------------------
+struct AccArgs {
+    const float *own, *oth;     // [own_rows, d], [oth_rows, d]
+    const float *what;          // TransH: unit normals of the queries [B, d]
+    const float *G, *U, *Cc;    // [B, N]
+    int own_rows, oth_rows, N, d4, split;
+    float *out, *out2;          // [split, own_rows, d]; out2: TransH normal gradient (OWNER_Q)
+};
+
+constexpr int ACC_ROWS = 32, ACC_CC = 32, ACC_LDW = 36;
+
+template <int KIND>
+__device__ __forceinline__ void acc_update(float4& acc, float4 a, float4 b, float w) {
+    if (KIND == KIND_DOT) {
+        acc = f4fma(w, b, acc);
+    } else if (KIND == KIND_L1) {  // acc -= w * sign(a - b)
+        acc.x += (a.x < b.x ? w : 0.f) - (a.x > b.x ? w : 0.f);
+        acc.y += (a.y < b.y ? w : 0.f) - (a.y > b.y ? w : 0.f);
+        acc.z += (a.z < b.z ? w : 0.f) - (a.z > b.z ? w : 0.f);
+        acc.w += (a.w < b.w ? w : 0.f) - (a.w > b.w ? w : 0.f);
+    } else if (KIND == KIND_L2) {  // w already holds G / distance
+        acc = f4fma(w, f4sub(b, a), acc);
+    } else {                       // KIND_CL1: acc -= w * (a - b) / |a - b| per complex component
+        float xr = a.x - b.x, xi = a.y - b.y, m2 = fmaf(xr, xr, xi * xi);
+        float s = m2 > 0.f ? w * rsqrtf(m2) : 0.f;
+        acc.x = fmaf(-s, xr, acc.x); acc.y = fmaf(-s, xi, acc.y);
+        xr = a.z - b.z; xi = a.w - b.w; m2 = fmaf(xr, xr, xi * xi);
+        s = m2 > 0.f ? w * rsqrtf(m2) : 0.f;
+        acc.z = fmaf(-s, xr, acc.z); acc.w = fmaf(-s, xi, acc.w);
+    }
+}
+
+template <int KIND, int NCH, bool OWNER_Q>
+__global__ void __launch_bounds__(256) accum_kernel(AccArgs a) {
+    constexpr bool TH = KIND == KIND_TH_L1 || KIND == KIND_TH_L2;
+    extern __shared__ __align__(16) float smem[];
+    const int d4 = a.d4;
+    float4* Bs = reinterpret_cast<float4*>(smem);                        // [32][d4]
+    float4* W2s = Bs + (TH && !OWNER_Q ? ACC_CC * d4 : 0);               // TransH dT: normals of the queries
+    float* Gs = reinterpret_cast<float*>(W2s + ACC_CC * d4);             // [32][36] weights, [c][r]
+    float* Us = Gs + ACC_CC * ACC_LDW;
+    float* Cs = Us + (TH ? ACC_CC * ACC_LDW : 0);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int r0 = blockIdx.x * ACC_ROWS;
+    const int per = ((a.oth_rows + a.split - 1) / a.split + ACC_CC - 1) / ACC_CC * ACC_CC;
+    const int c_begin = blockIdx.y * per;
+    const int c_end = min(a.oth_rows, c_begin + per);
+
+    float4 A[4][NCH], Wn[TH && OWNER_Q ? 4 : 1][NCH], acc[4][NCH], acc2[TH && OWNER_Q ? 4 : 1][NCH];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < NCH; ++j) {
+            const int r = r0 + warp * 4 + i, c = lane + 32 * j;
+            const bool in = r < a.own_rows && c < d4;
+            A[i][j] = in ? reinterpret_cast<const float4*>(a.own)[(int64_t)r * d4 + c] : f4zero();
+            acc[i][j] = f4zero();
+            if (TH && OWNER_Q) {
+                Wn[i][j] = in ? reinterpret_cast<const float4*>(a.what)[(int64_t)r * d4 + c] : f4zero();
+                acc2[i][j] = f4zero();
+            }
+        }
+
+    for (int c0 = c_begin; c0 < c_end; c0 += ACC_CC) {
+        for (int idx = tid; idx < ACC_CC * d4; idx += 256) {
+            const int rr = idx / d4, cc = idx - rr * d4, row = c0 + rr;
+            Bs[idx] = row < c_end ? reinterpret_cast<const float4*>(a.oth)[(int64_t)row * d4 + cc] : f4zero();
+            if (TH && !OWNER_Q)
+                W2s[idx] = row < c_end ? reinterpret_cast<const float4*>(a.what)[(int64_t)row * d4 + cc] : f4zero();
+        }
+        for (int idx = tid; idx < ACC_CC * ACC_ROWS; idx += 256) {
+            int rr, cc;
+            int64_t g;
+            if (OWNER_Q) { cc = idx & 31; rr = idx >> 5; g = (int64_t)(r0 + rr) * a.N + (c0 + cc); }
+            else         { rr = idx & 31; cc = idx >> 5; g = (int64_t)(c0 + cc) * a.N + (r0 + rr); }
+            const bool in = (r0 + rr) < a.own_rows && (c0 + cc) < c_end;
+            Gs[cc * ACC_LDW + rr] = in ? a.G[g] : 0.f;
+            if (TH) { Us[cc * ACC_LDW + rr] = in ? a.U[g] : 0.f; Cs[cc * ACC_LDW + rr] = in ? a.Cc[g] : 0.f; }
+        }
+        __syncthreads();
+#pragma unroll 4
+        for (int cc = 0; cc < ACC_CC; ++cc) {
+            const float4 g4 = *reinterpret_cast<const float4*>(&Gs[cc * ACC_LDW + warp * 4]);
+            const float gw[4] = {g4.x, g4.y, g4.z, g4.w};
+            float uw[4] = {0.f, 0.f, 0.f, 0.f}, cw[4] = {0.f, 0.f, 0.f, 0.f};
+            if (TH) {
+                const float4 u4 = *reinterpret_cast<const float4*>(&Us[cc * ACC_LDW + warp * 4]);
+                const float4 c4 = *reinterpret_cast<const float4*>(&Cs[cc * ACC_LDW + warp * 4]);
+                uw[0] = u4.x; uw[1] = u4.y; uw[2] = u4.z; uw[3] = u4.w;
+                cw[0] = c4.x; cw[1] = c4.y; cw[2] = c4.z; cw[3] = c4.w;
+            }
+#pragma unroll
+            for (int j = 0; j < NCH; ++j) {
+                const int c = lane + 32 * j;
+                if (c >= d4) continue;
+                const float4 bv = Bs[cc * d4 + c];
+                if (!TH) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc_update<TH ? KIND_L1 : KIND>(acc[i][j], A[i][j], bv, gw[i]);
+                } else if (OWNER_Q) {   // own = q_b (A), normal Wn; other = t_n (bv)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float4 x = f4fma(uw[i], Wn[i][j], f4sub(A[i][j], bv));
+                        const float4 S = KIND == KIND_TH_L1 ? f4scale(-gw[i], f4sgn(x)) : f4scale(-gw[i], x);
+                        acc[i][j] = f4add(acc[i][j], S);
+                        acc2[i][j] = f4fma(cw[i], bv, f4fma(uw[i], S, acc2[i][j]));
+                    }
+                } else {                // own = t_n (A); other = q_b (bv) with its normal wv
+                    const float4 wv = W2s[cc * d4 + c];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float4 x = f4fma(uw[i], wv, f4sub(bv, A[i][j]));
+                        const float4 S = KIND == KIND_TH_L1 ? f4scale(-gw[i], f4sgn(x)) : f4scale(-gw[i], x);
+                        acc[i][j] = f4fma(cw[i], wv, f4sub(acc[i][j], S));
+                    }
+                }
+            }
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < NCH; ++j) {
+            const int r = r0 + warp * 4 + i, c = lane + 32 * j;
+            if (r >= a.own_rows || c >= d4) continue;
+            const int64_t o = ((int64_t)blockIdx.y * a.own_rows + r) * d4 + c;
+            reinterpret_cast<float4*>(a.out)[o] = acc[i][j];
+            if (TH && OWNER_Q) reinterpret_cast<float4*>(a.out2)[o] = acc2[i][j];
+        }
+}
+
+// ------------------------------------------------------------------------------------------
+// chain: one warp per row.  Warps [0, B): add the column splits of dQ (and of the TransH
+// normal gradient), add the positive pair, apply the chain rule q -> (h, r, w) and write
+// the gradient rows of the head, the positive tail and the relation.  Warps [B, B+N): add
+// the row splits of dT and write the gradient row of the negative tail.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (warp >= p.B + p.N) return;
+    const int d4 = p.d4;
+    float4* gent = reinterpret_cast<float4*>(p.w.grad_ent);
+    if (warp >= p.B) {
+        const int n = warp - p.B;
+        const float4* part = reinterpret_cast<const float4*>(p.w.dTpart);
+        for (int c = lane; c < d4; c += 32) {
+            float4 s = f4zero();
+            for (int sp = 0; sp < p.split_t; ++sp) s = f4add(s, part[((int64_t)sp * p.N + n) * d4 + c]);
+            gent[(int64_t)(2 * p.B + n) * d4 + c] = s;
+        }
+        return;
+    }
+    const int b = warp;
+    const int64_t hid = checked_id(p.heads[b], p.E, p.w.status);
+    const int64_t rid = checked_id(p.rels[b], p.R, p.w.status);
+    const int64_t tid = checked_id(p.tails[b], p.E, p.w.status);
+    const float4* hrow = reinterpret_cast<const float4*>(p.ent) + hid * d4;
+    const float4* trow = reinterpret_cast<const float4*>(p.ent) + tid * d4;
+    const float4* qrow = reinterpret_cast<const float4*>(p.w.Q) + (int64_t)b * d4;
+    const float gp = p.w.gpos[b], fp = p.w.fpos[b];
+
+    float4 h[kMaxChunks], t[kMaxChunks], q[kMaxChunks], dq[kMaxChunks], dt[kMaxChunks];
+#pragma unroll
+    for (int i = 0; i < kMaxChunks; ++i) {
+        const int c = lane + 32 * i;
+        const bool in = c < d4;
+        h[i] = in ? hrow[c] : f4zero(); t[i] = in ? trow[c] : f4zero(); q[i] = in ? qrow[c] : f4zero();
+        float4 s = f4zero();
+        if (in)
+            for (int sp = 0; sp < p.split_q; ++sp)
+                s = f4add(s, reinterpret_cast<const float4*>(p.w.dQpart)[((int64_t)sp * p.B + b) * d4 + c]);
+        dq[i] = s; dt[i] = f4zero();
+    }
+    float4* gh = gent + (int64_t)b * d4;
+    float4* gt = gent + (int64_t)(p.B + b) * d4;
+
+    if (p.score == KGE_TRANSH) {
+        const float4* whrow = reinterpret_cast<const float4*>(p.w.What) + (int64_t)b * d4;
+        const float4* wrow = reinterpret_cast<const float4*>(p.relw) + rid * d4;
+        float4 wh[kMaxChunks], dwh[kMaxChunks];
+        float u = 0.f, a = 0.f, nrm2 = 0.f;
+#pragma unroll
+        for (int i = 0; i < kMaxChunks; ++i) {
+            const int c = lane + 32 * i;
+            const bool in = c < d4;
+            wh[i] = in ? whrow[c] : f4zero();
+            const float4 wraw = in ? wrow[c] : f4zero();
+            nrm2 += f4dot(wraw, wraw);
+            float4 s = f4zero();
+            if (in)
+                for (int sp = 0; sp < p.split_q; ++sp)
+                    s = f4add(s, reinterpret_cast<const float4*>(p.w.dWpart)[((int64_t)sp * p.B + b) * d4 + c]);
+            dwh[i] = s;
+            u += f4dot(wh[i], t[i]); a += f4dot(wh[i], h[i]);
+        }
+        u = warp_sum(u); a = warp_sum(a); nrm2 = warp_sum(nrm2);
+        // positive pair
+        const float scale = p.kind == KIND_TH_L1 ? gp : (fp < 0.f ? gp / -fp : 0.f);
+        float4 S[kMaxChunks];
+        float cpos = 0.f;
+#pragma unroll
+        for (int i = 0; i < kMaxChunks; ++i) {
+            const float4 x = f4fma(u, wh[i], f4sub(q[i], t[i]));
+            S[i] = p.kind == KIND_TH_L1 ? f4scale(-scale, f4sgn(x)) : f4scale(-scale, x);
+            cpos += f4dot(S[i], wh[i]);
+        }
+        cpos = warp_sum(cpos);
+        float wdq = 0.f;
+#pragma unroll
+        for (int i = 0; i < kMaxChunks; ++i) {
+            dq[i] = f4add(dq[i], S[i]);
+            dt[i] = f4fma(cpos, wh[i], f4scale(-1.f, S[i]));
+            dwh[i] = f4fma(cpos, t[i], f4fma(u, S[i], dwh[i]));
+            wdq += f4dot(wh[i], dq[i]);
+        }
+        wdq = warp_sum(wdq);
+        // q = h - (w.h) w + r
+        float wdw = 0.f;
+#pragma unroll
+        for (int i = 0; i < kMaxChunks; ++i) {
+            dwh[i] = f4fma(-a, dq[i], f4fma(-wdq, h[i], dwh[i]));
+            wdw += f4dot(wh[i], dwh[i]);
+        }
+        wdw = warp_sum(wdw);
+        const float nrm = sqrtf(nrm2);
+        const bool clamped = !(nrm > 1e-12f);
+        const float inv = 1.f / fmaxf(nrm, 1e-12f);
+        float4* gr = reinterpret_cast<float4*>(p.w.grad_rel) + (int64_t)b * d4;
+        float4* gw = reinterpret_cast<float4*>(p.w.grad_relw) + (int64_t)b * d4;
+#pragma unroll
+        for (int i = 0; i < kMaxChunks; ++i) {
+            const int c = lane + 32 * i;
+            if (c >= d4) continue;
+            gh[c] = f4fma(-wdq, wh[i], dq[i]);
+            gt[c] = dt[i];
+            gr[c] = dq[i];
+            gw[c] = clamped ? f4scale(inv, dwh[i]) : f4scale(inv, f4fma(-wdw, wh[i], dwh[i]));
+        }
+        return;
+    }
+
+    // positive pair for the kinds whose pair is a function of (q, t) alone
+#pragma unroll
+    for (int i = 0; i < kMaxChunks; ++i) {
+        if (p.kind == KIND_DOT) {
+            dq[i] = f4fma(gp, t[i], dq[i]);
+            dt[i] = f4scale(gp, q[i]);
+        } else if (p.kind == KIND_L1) {
+            const float4 s = f4sgn(f4sub(q[i], t[i]));
+            dq[i] = f4fma(-gp, s, dq[i]);
+            dt[i] = f4scale(gp, s);
+        } else if (p.kind == KIND_L2) {
+            const float cpos = fp < 0.f ? gp / -fp : 0.f;
+            const float4 x = f4sub(q[i], t[i]);
+            dq[i] = f4fma(-cpos, x, dq[i]);
+            dt[i] = f4scale(cpos, x);
+        } else {  // KIND_CL1
+            const float4 x = f4sub(q[i], t[i]);
+            const float m0 = fmaf(x.x, x.x, x.y * x.y), m1 = fmaf(x.z, x.z, x.w * x.w);
+            const float s0 = m0 > 0.f ? gp * rsqrtf(m0) : 0.f, s1 = m1 > 0.f ? gp * rsqrtf(m1) : 0.f;
+            const float4 g = make_float4(s0 * x.x, s0 * x.y, s1 * x.z, s1 * x.w);
+            dq[i] = f4sub(dq[i], g);
+            dt[i] = g;
+        }
+    }
+    if (p.score == KGE_ROTATE) {
+        const float2* th = reinterpret_cast<const float2*>(p.rel) + rid * d4;
+        float2* gr = reinterpret_cast<float2*>(p.w.grad_rel) + (int64_t)b * d4;
+#pragma unroll
+        for (int i = 0; i < kMaxChunks; ++i) {
+            const int c = lane + 32 * i;
+            if (c >= d4) continue;
+            const float2 ph = th[c];
+            float s0, c0, s1, c1;
+            sincosf(ph.x, &s0, &c0); sincosf(ph.y, &s1, &c1);
+            gh[c] = make_float4(dq[i].x * c0 + dq[i].y * s0, -dq[i].x * s0 + dq[i].y * c0,
+                                dq[i].z * c1 + dq[i].w * s1, -dq[i].z * s1 + dq[i].w * c1);
+            gt[c] = dt[i];
+            gr[c] = make_float2(-dq[i].x * q[i].y + dq[i].y * q[i].x, -dq[i].z * q[i].w + dq[i].w * q[i].z);
+        }
+        return;
+    }
+    const float4* rrow = reinterpret_cast<const float4*>(p.rel) + rid * d4;
+    float4* gr = reinterpret_cast<float4*>(p.w.grad_rel) + (int64_t)b * d4;
+#pragma unroll
+    for (int i = 0; i < kMaxChunks; ++i) {
+        const int c = lane + 32 * i;
+        if (c >= d4) continue;
+        gt[c] = dt[i];
+        if (p.score == KGE_TRANSE) {
+            gh[c] = dq[i]; gr[c] = dq[i];
+        } else if (p.score == KGE_DISTMULT) {
+            const float4 r = rrow[c];
+            gh[c] = f4mul(dq[i], r); gr[c] = f4mul(dq[i], h[i]);
+        } else {  // ComplEx: q = r * h
+            const float4 r = rrow[c];
+            gh[c] = make_float4(dq[i].x * r.x + dq[i].y * r.y, -dq[i].x * r.y + dq[i].y * r.x,
+                                dq[i].z * r.z + dq[i].w * r.w, -dq[i].z * r.w + dq[i].w * r.z);
+            gr[c] = make_float4(dq[i].x * h[i].x + dq[i].y * h[i].y, -dq[i].x * h[i].y + dq[i].y * h[i].x,
+                                dq[i].z * h[i].z + dq[i].w * h[i].w, -dq[i].z * h[i].w + dq[i].w * h[i].z);
+        }
+    }
+}
+
+// ---- host-side dispatch ----
+template <int KIND, int MODE>
+void launch_block(const TrainParams& p, cudaStream_t s) {
+    dim3 grid((p.N + TN - 1) / TN, (p.B + TB - 1) / TB);
+    block_kernel<KIND, MODE><<<grid, 256, 0, s>>>(p);
+}
+
+template <int KIND, int NCH, bool OWNER_Q>
+cudaError_t launch_accum_inst(const AccArgs& a, cudaStream_t s) {
+    constexpr bool TH = KIND == KIND_TH_L1 || KIND == KIND_TH_L2;
+    size_t smem = (size_t)ACC_CC * a.d4 * 16 * ((TH && !OWNER_Q) ? 2 : 1) + (size_t)ACC_CC * ACC_LDW * 4 * (TH ? 3 : 1);
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(accum_kernel<KIND, NCH, OWNER_Q>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    dim3 grid((a.own_rows + ACC_ROWS - 1) / ACC_ROWS, a.split);
+    accum_kernel<KIND, NCH, OWNER_Q><<<grid, 256, smem, s>>>(a);
+    return cudaSuccess;
+}
+
+template <int KIND, bool OWNER_Q>
+cudaError_t launch_accum_kind(const AccArgs& a, cudaStream_t s) {
+    if (a.d4 <= 32) return launch_accum_inst<KIND, 1, OWNER_Q>(a, s);
+    if (a.d4 <= 64) return launch_accum_inst<KIND, 2, OWNER_Q>(a, s);
+    return launch_accum_inst<KIND, 4, OWNER_Q>(a, s);
+}
+
+template <bool OWNER_Q>
+cudaError_t launch_accum(int kind, const AccArgs& a, cudaStream_t s) {
+    switch (kind) {
+        case KIND_L1: return launch_accum_kind<KIND_L1, OWNER_Q>(a, s);
+        case KIND_L2: return launch_accum_kind<KIND_L2, OWNER_Q>(a, s);
+        case KIND_CL1: return launch_accum_kind<KIND_CL1, OWNER_Q>(a, s);
+        case KIND_DOT: return launch_accum_kind<KIND_DOT, OWNER_Q>(a, s);
+        case KIND_TH_L1: return launch_accum_kind<KIND_TH_L1, OWNER_Q>(a, s);
+        default: return launch_accum_kind<KIND_TH_L2, OWNER_Q>(a, s);
+    }
+}
+
+}  // namespace
+
+int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* rels, const int32_t* tails,
+                            const int32_t* negs, cudaStream_t s) {
+    const kge_config& c = h->cfg;
+    TrainParams p;
+    p.B = c.batch; p.N = c.num_neg; p.d = c.dim; p.d4 = c.dim / 4; p.kw = h->kw;
+    p.score = c.score; p.kind = h->kind; p.loss = c.loss;
+    p.gamma = c.gamma; p.adv_temp = c.adv_temp; p.ce_c = c.ce_correction; p.loss_scale = c.loss_scale;
+    p.E = c.num_entities; p.R = c.num_relations;
+    p.ent = h->ent; p.rel = h->rel; p.relw = h->relw;
+    p.heads = heads; p.rels = rels; p.tails = tails; p.negs = negs;
+    p.split_q = h->split_q; p.split_t = h->split_t;
+    p.w = h->ws;
+
+    const int row_warps = p.B + p.N;
+    stage_begin(h, ST_BUILD, s);
+    build_kernel<<<(row_warps * 32 + 255) / 256, 256, 0, s>>>(p);
+    stage_end(h, ST_BUILD, s);
+    KGE_LAUNCH_CHECK(h);
+    stage_begin(h, ST_BLOCK, s);
+    switch (p.kind) {
+        case KIND_L1: launch_block<KIND_L1, 0>(p, s); break;
+        case KIND_L2: launch_block<KIND_L2, 0>(p, s); break;
+        case KIND_CL1: launch_block<KIND_CL1, 0>(p, s); break;
+        case KIND_DOT: launch_block<KIND_DOT, 0>(p, s); break;
+        case KIND_TH_L1: launch_block<KIND_TH_L1, 0>(p, s); break;
+        default: launch_block<KIND_TH_L2, 0>(p, s); break;
+    }
+    stage_end(h, ST_BLOCK, s);
+    KGE_LAUNCH_CHECK(h);
+    stage_begin(h, ST_LOSS, s);
+    loss_kernel<<<p.B, LOSS_THREADS, 0, s>>>(p);
+    stage_end(h, ST_LOSS, s);
+    KGE_LAUNCH_CHECK(h);
+    if (p.kind == KIND_TH_L1 || p.kind == KIND_TH_L2) {
+        stage_begin(h, ST_TH_CPASS, s);
+        if (p.kind == KIND_TH_L1) launch_block<KIND_TH_L1, 1>(p, s); else launch_block<KIND_TH_L2, 1>(p, s);
+        stage_end(h, ST_TH_CPASS, s);
+        KGE_LAUNCH_CHECK(h);
+    }
+
+    AccArgs aq;
+    aq.own = p.w.Q; aq.oth = p.w.Tneg; aq.what = p.w.What; aq.G = p.w.F; aq.U = p.w.U; aq.Cc = p.w.Cc;
+    aq.own_rows = p.B; aq.oth_rows = p.N; aq.N = p.N; aq.d4 = p.d4; aq.split = p.split_q;
+    aq.out = p.w.dQpart; aq.out2 = p.w.dWpart;
+    stage_begin(h, ST_ACCUM_Q, s);
+    KGE_CUDA_CHECK(h, launch_accum<true>(p.kind, aq, s));
+    stage_end(h, ST_ACCUM_Q, s);
+    KGE_LAUNCH_CHECK(h);
+    AccArgs at = aq;
+    at.own = p.w.Tneg; at.oth = p.w.Q; at.own_rows = p.N; at.oth_rows = p.B; at.split = p.split_t;
+    at.out = p.w.dTpart; at.out2 = nullptr;
+    stage_begin(h, ST_ACCUM_T, s);
+    KGE_CUDA_CHECK(h, launch_accum<false>(p.kind, at, s));
+    stage_end(h, ST_ACCUM_T, s);
+    KGE_LAUNCH_CHECK(h);
+    stage_begin(h, ST_CHAIN, s);
+    chain_kernel<<<(row_warps * 32 + 255) / 256, 256, 0, s>>>(p);
+    stage_end(h, ST_CHAIN, s);
+    KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
+}
+
+}  // namespace kge

@@ -1,0 +1,73 @@
+"""CPU-only checks of the C-ABI boundary: the shared library builds, loads, exports every
+symbol the header declares, and rejects bad configurations on the host (no GPU needed)."""
+import ctypes as C
+import re
+from pathlib import Path
+
+import pytest
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module")
+def K():
+    from paper_2211_12281_b200 import build
+    build.build()
+    import paper_2211_12281_b200 as K
+    return K
+
+
+def test_library_exports_every_declared_symbol(K):
+    header = (ROOT / "include" / "kge.h").read_text()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(kge_[a-z_0-9]+)\s*\(", header))
+    assert {"kge_sample_batch", "kge_train_step", "kge_score_all_topk", "kge_eval_mrr"} <= declared
+    lib = K.lib()
+    for name in sorted(declared):
+        assert hasattr(lib, name), name
+    from paper_2211_12281_b200.binding import SIGNATURES
+    assert set(SIGNATURES) == declared
+
+
+def test_config_struct_matches_header_layout(K):
+    # 2 x int64 + 12 x int32 + 8 x float + uint64 = 104 bytes, seed 8-byte aligned
+    assert C.sizeof(K.KgeConfig) == 104 and K.KgeConfig.seed.offset == 96 and K.KgeConfig.gamma.offset == 64
+
+
+def _create(K, **over):
+    kw = dict(num_entities=1000, num_relations=10, dim=32, score="distmult", batch=64, num_neg=128, num_parts=2)
+    kw.update(over)
+    return K.Kge(K.KgeConfig.make(**kw))
+
+
+def test_create_validates_arguments_on_the_host(K):
+    h = _create(K)
+    assert h.workspace_bytes(20000, 100, 10) > h.workspace_bytes(20000, 0, 0) > h.workspace_bytes(0, 0, 0) > 0
+    for bad, code in ((dict(dim=30), -1), (dict(dim=1024), -1), (dict(p_norm=3), -1), (dict(score=7), -1),
+                      (dict(batch=66), -2), (dict(num_neg=127), -2), (dict(batch=66, head_part=0), None),
+                      (dict(head_part=2), -1), (dict(adv_temp=-1.0), -1), (dict(num_entities=0), -1),
+                      (dict(num_entities=9, num_parts=4, batch=16, num_neg=4), -3)):
+        if code is None:
+            _create(K, **bad)           # B % P suffices when the head partition is fixed
+            continue
+        with pytest.raises(K.KgeError) as e:
+            _create(K, **bad)
+        assert e.value.code == code, bad
+
+
+def test_calls_before_bind_are_refused(K):
+    h = _create(K)
+    lib = K.lib()
+    assert lib.kge_train_step(h._h, 0, 0.1, None, None, None, None, None, None) == -6
+    assert lib.kge_get_status(h._h, None) == -6
+    assert lib.kge_train_step(None, 0, 0.1, None, None, None, None, None, None) == -1
+    assert lib.kge_error_string(-6) == b"tables not bound or graph not loaded"
+
+
+def test_missing_library_fails_loudly(K, monkeypatch, tmp_path):
+    from paper_2211_12281_b200 import binding
+    monkeypatch.setattr(binding, "_LIB", None)
+    monkeypatch.setattr(binding, "_PKG", tmp_path)
+    with pytest.raises(K.KgeError) as e:
+        binding.lib()
+    assert e.value.code == binding.KGE_ERR_NO_EXTENSION

@@ -1,0 +1,95 @@
+"""GPU parity of full-entity scoring: top-k ids bit-exact against the fp32 oracle (both
+sides decide the order in fp32 with the same per-pair operation order), scores at 1e-4,
+ranks exact, MRR within 1e-3; exact ties, k > |E|, the list-overflow path."""
+import numpy as np
+import pytest
+
+from parity_util import GpuSide, Problem, assert_close
+
+pytestmark = pytest.mark.gpu
+
+
+def _infer(gpu, qh, qr, tt, K):
+    t = gpu.torch
+    dev = gpu.ent.device
+    nq = len(qh)
+    ids = t.empty((nq, K), dtype=t.int32, device=dev); sc = t.empty((nq, K), dtype=t.float32, device=dev)
+    ranks = t.empty(nq, dtype=t.int32, device=dev)
+    gpu.kge.score_all_topk(gpu.dev_i32(qh), gpu.dev_i32(qr), K, gpu.dev_i32(tt), ids, sc, ranks)
+    assert gpu.kge.get_status() == 0
+    return ids.cpu().numpy(), sc.cpu().numpy(), ranks.cpu().numpy()
+
+
+@pytest.mark.parametrize("score,p", [("transe", 1), ("transe", 2), ("distmult", 1), ("complex", 1),
+                                     ("transh", 1), ("transh", 2), ("rotate", 2), ("rotate", 1)])
+def test_topk_rank_mrr_against_fp32_oracle(oracle32, oracle64, score, p):
+    import kge_synth
+    E, R, d, K, nq = 5000, 9, 40, 10, 70          # chunks 1024, 1024, 2048, 904; ragged tiles
+    prob = Problem(E=E, R=R, T=100, d=d, score=score, p_norm=p, B=4, N=4, P=1, graph_seed=11)
+    prob.ent[3000] = prob.ent[17]; prob.ent[4999] = prob.ent[17]; prob.ent[1] = prob.ent[0]   # exact ties
+    qh, qr, tt = kge_synth.make_queries(E, R, nq, seed=11)
+    tt[0] = qh[0]; tt[1] = 4999; tt[2] = 17
+    gpu = GpuSide(prob, max_queries=nq, topk=K, load_graph=False)
+    ids, sc, ranks = _infer(gpu, qh, qr, tt, K)
+    cfg = prob.oracle_cfg()
+    o_ids, o_sc, o_ranks = oracle32.score_all_topk(cfg, prob.ent, prob.rel, prob.relw, qh, qr, K, true_tails=tt)
+    if score == "rotate":
+        # sin / cos come from different math libraries: compare as sets, audit near-ties
+        r_ids, r_sc, r_ranks = oracle64.score_all_topk(cfg, prob.ent, prob.rel, prob.relw, qh, qr, K + 5, true_tails=tt)
+        for q in range(nq):
+            extra = set(ids[q]) - set(r_ids[q, :K])
+            for e in extra:
+                assert e in set(r_ids[q]), "id outside the oracle's top (k+5)"
+                f = r_sc[q][list(r_ids[q]).index(e)]
+                assert abs(f - r_sc[q, K - 1]) <= 1e-4 * abs(f)
+        assert_close(sc, r_sc[:, :K], what="scores")
+        assert np.abs(ranks - r_ranks).max() <= 2
+    else:
+        assert (ids == o_ids).all()
+        assert (sc == o_sc).all() or np.allclose(sc, o_sc, rtol=1e-6)
+        assert (ranks == o_ranks).all()
+    mrr = gpu.kge.eval_mrr(gpu.dev_i32(qh), gpu.dev_i32(qr), gpu.dev_i32(tt), 10)
+    assert abs(mrr - oracle64.mrr(o_ranks, 10)) <= 1e-3
+    mrr0 = gpu.kge.eval_mrr(gpu.dev_i32(qh), gpu.dev_i32(qr), gpu.dev_i32(tt), 0)
+    assert abs(mrr0 - oracle64.mrr(o_ranks, 0)) <= 1e-3
+
+
+def test_config1_mrr_after_training(oracle32, oracle64):
+    """BASELINE configs[0]: 10 SGD steps, then MRR of the first 100 triples ranked against
+    all 1,000 entities.  Inference parity is taken on the GPU's own trained tables."""
+    prob = Problem(E=1000, R=10, T=20000, d=32, score="distmult", loss="logsigmoid", B=64, N=128, P=2,
+                   lr=0.1, seed=0, graph_seed=0)
+    gpu = GpuSide(prob, max_queries=100, topk=10)
+    for step in range(10):
+        gpu.kge.train_step(step, prob.lr)
+    qh, qr, tt = prob.h[:100], prob.r[:100], prob.t[:100]
+    ids, sc, ranks = _infer(gpu, qh, qr, tt, 10)
+    ent, rel, _ = gpu.tables()
+    o_ids, o_sc, o_ranks = oracle32.score_all_topk(prob.oracle_cfg(), ent, rel, None, qh, qr, 10, true_tails=tt)
+    assert (ids == o_ids).all() and (ranks == o_ranks).all()
+    assert abs(gpu.kge.eval_mrr(gpu.dev_i32(qh), gpu.dev_i32(qr), gpu.dev_i32(tt), 0) - oracle64.mrr(o_ranks, 0)) <= 1e-3
+
+
+def test_k_larger_than_entities_and_single_query(oracle32):
+    prob = Problem(E=9, R=2, T=50, d=16, score="transe", p_norm=1, B=4, N=4, P=1, graph_seed=12)
+    gpu = GpuSide(prob, max_queries=4, topk=12, load_graph=False)
+    ids, sc, ranks = _infer(gpu, np.array([3]), np.array([1]), np.array([4]), 12)
+    o_ids, o_sc, o_ranks = oracle32.score_all_topk(prob.oracle_cfg(), prob.ent, prob.rel, None, [3], [1], 12, true_tails=[4])
+    assert (ids == o_ids).all() and (ranks == o_ranks).all()
+    assert (ids[0, 9:] == -1).all() and np.isneginf(sc[0, 9:]).all()
+
+
+def test_rising_scores_take_the_overflow_path(oracle32):
+    """Scores that grow with the entity id make every entity of a chunk beat the current
+    k-th best, which fills the candidate list; the library must redo the chunk in pieces."""
+    E, d, K = 6000, 16, 5
+    prob = Problem(E=E, R=2, T=50, d=d, score="distmult", B=4, N=4, P=1, graph_seed=13)
+    prob.ent[:] = 0.0
+    prob.ent[:, 0] = np.arange(E, dtype=np.float32) / E + 0.5
+    prob.rel[:] = 1.0
+    gpu = GpuSide(prob, max_queries=8, topk=K, load_graph=False)
+    qh, qr, tt = np.array([10, 4000, 5999]), np.array([0, 1, 0]), np.array([0, 5999, 3000])
+    ids, sc, ranks = _infer(gpu, qh, qr, tt, K)
+    o_ids, _, o_ranks = oracle32.score_all_topk(prob.oracle_cfg(), prob.ent, prob.rel, None, qh, qr, K, true_tails=tt)
+    assert (ids == o_ids).all() and (ranks == o_ranks).all()
+    assert (ids[0] == np.arange(E - 1, E - 1 - K, -1)).all()

@@ -1,0 +1,177 @@
+"""GPU parity of the training step against the fp64 oracle: per-stage taps (positive
+scores, dL/dF, gradient rows, dedup segments) and updated tables, for all five scoring
+functions, both norms, both losses and the three optimisers; sizes span several tiles with
+ragged tails.  Tolerance: |a-b| <= 1e-4 max(|a|,|b|) + atol, atol a small multiple of fp32
+epsilon times the magnitude of the summed terms."""
+import numpy as np
+import pytest
+
+from parity_util import GpuSide, OracleSide, Problem, assert_close
+
+pytestmark = pytest.mark.gpu
+
+MODELS = [("transe", 1), ("transe", 2), ("transh", 1), ("transh", 2), ("rotate", 1), ("rotate", 2),
+          ("distmult", 1), ("complex", 1)]
+
+
+def _check_step(gpu, orc, step, batch, *, taps=True, rows_atol=2e-6):
+    prob = gpu.prob
+    B, N, d = prob.B, prob.N, prob.d
+    dev = [gpu.dev_i32(a) for a in batch]
+    loss_dev = gpu.torch.zeros(1, dtype=gpu.torch.float32, device=gpu.ent.device)
+    want = orc.grads(batch) if taps else None
+    gpu.kge.train_step(step, prob.lr, *dev, loss_out=loss_dev)
+    assert gpu.kge.get_status() == 0
+    loss_o = orc.step(step, batch)
+    assert_close(loss_dev.item(), loss_o, atol=1e-5, what="loss")
+    if taps:
+        kge = gpu.kge
+        l2 = prob.kw["p_norm"] == 2 and prob.score in ("transe", "transh", "rotate")
+        G = kge.debug_export("G").reshape(B, N)
+        if l2:   # the tap holds dL/dF divided by the distance; undo with the oracle's distances
+            F = orc.o.batch_loss(orc.cfg, *orc._pre, *batch)["F"]
+            G = G * -F
+        assert_close(G, want["G"], atol=1e-7, what="G")
+        ge = kge.debug_export("GRAD_ENT").reshape(2 * B + N, d)
+        scale = max(np.abs(want["dh"]).max(), np.abs(want["dtneg"]).max(), 1e-30)
+        assert_close(ge[:B], want["dh"], atol=2e-5 * scale, what="dh")
+        assert_close(ge[B:2 * B], want["dtpos"], atol=2e-5 * scale, what="dtpos")
+        assert_close(ge[2 * B:], want["dtneg"], atol=2e-5 * scale, what="dtneg")
+        assert_close(kge.debug_export("GRAD_REL").reshape(B, -1), want["dr"],
+                     atol=2e-5 * max(np.abs(want["dr"]).max(), 1e-30), what="dr")
+        if prob.score == "transh":
+            assert_close(kge.debug_export("GRAD_RELW").reshape(B, d), want["dw"],
+                         atol=2e-5 * max(np.abs(want["dw"]).max(), 1e-30), what="dw")
+        # dedup: bit-exact
+        ids = np.concatenate([batch[0], batch[2], batch[3]])
+        for pre, lst in (("ENT", ids), ("REL", batch[1])):
+            uniq, seg, perm = orc.o.dedup(lst)
+            assert (kge.debug_export(pre + "_UNIQ") == uniq).all()
+            assert (kge.debug_export(pre + "_SEG") == seg).all()
+            assert (kge.debug_export(pre + "_PERM") == perm).all()
+    ent, rel, relw = gpu.tables()
+    assert_close(ent, orc.ent, atol=rows_atol, what="entity table")
+    assert_close(rel, orc.rel, atol=rows_atol, what="relation table")
+    if relw is not None:
+        assert_close(relw, orc.relw, atol=rows_atol, what="normal table")
+    for got, want_s, name in zip(gpu.states, orc.states, ("ent_state", "rel_state", "relw_state")):
+        if got is not None:
+            assert_close(got.cpu().numpy(), want_s, atol=1e-9, what=name)
+
+
+def _run(oracle64, prob, steps=2, taps=True, external_batch=None):
+    gpu, orc = GpuSide(prob), OracleSide(prob, oracle64)
+    for step in range(steps):
+        batch = external_batch if external_batch is not None else orc.sample(step)
+        # each step is compared from identical tables: the oracle restarts from the GPU's rows
+        orc.set_tables(*gpu.tables(), states=[None if s is None else s.cpu().numpy() for s in gpu.states])
+        orc._pre = (orc.ent.copy(), orc.rel.copy(), None if orc.relw is None else orc.relw.copy())
+        _check_step(gpu, orc, step, batch, taps=taps)
+    return gpu, orc
+
+
+@pytest.mark.parametrize("score,p", MODELS)
+@pytest.mark.parametrize("loss", ["logsigmoid", "softmax"])
+def test_step_taps_and_tables_all_models(oracle64, score, p, loss):
+    # B = 72 and N = 70 leave ragged 64-wide tiles; d = 40 leaves a ragged 32-wide slice
+    prob = Problem(E=500, R=7, T=20000, d=40, score=score, p_norm=p, loss=loss, B=72, N=70, P=2,
+                   gamma=6.0 if loss == "logsigmoid" and score in ("transe", "transh", "rotate") else 0.0,
+                   adv_temp=1.0 if loss == "logsigmoid" else 0.0, ce_correction=0.5, loss_scale=0.25,
+                   lr=0.05, graph_seed=3, relation_zipf=1.0)
+    _run(oracle64, prob)
+
+
+@pytest.mark.parametrize("opt", ["adam", "adagrad"])
+@pytest.mark.parametrize("score,p", [("transe", 1), ("complex", 1), ("transh", 2), ("rotate", 1)])
+def test_optimisers_with_state(oracle64, opt, score, p):
+    prob = Problem(E=300, R=5, T=10000, d=32, score=score, p_norm=p, loss="softmax", opt=opt, B=64, N=96, P=2,
+                   ce_correction=0.1, lr=0.01, graph_seed=4, relation_zipf=1.0)
+    _run(oracle64, prob, steps=3, taps=False)
+
+
+def test_wide_rows_and_many_splits(oracle64):
+    # d = 256 (two slices per lane), B << N so the dQ accumulation is split over columns
+    prob = Problem(E=2000, R=11, T=40000, d=256, score="distmult", loss="softmax", B=32, N=640, P=4,
+                   ce_correction=1.0, lr=0.1, graph_seed=5)
+    _run(oracle64, prob, steps=1)
+    prob = Problem(E=2000, R=11, T=40000, d=384, score="transe", p_norm=1, loss="logsigmoid", B=256, N=32, P=4,
+                   gamma=12.0, adv_temp=0.5, lr=0.1, graph_seed=6)
+    _run(oracle64, prob, steps=1)
+
+
+def test_repeated_rows_one_entity_everywhere(oracle64):
+    """One entity is head, tail and negative several times; one relation for the whole batch."""
+    prob = Problem(E=64, R=2, T=2000, d=32, score="distmult", loss="logsigmoid", B=16, N=16, P=1, lr=0.1)
+    rng = np.random.default_rng(0)
+    heads, tails, negs = rng.integers(0, 64, 16), rng.integers(0, 64, 16), rng.integers(0, 64, 16)
+    heads[[0, 5, 9]] = 7; tails[[1, 5]] = 7; negs[[0, 3, 15]] = 7
+    rels = np.zeros(16, np.int64)
+    batch = [a.astype(np.int32) for a in (heads, rels, tails, negs)]
+    _run(oracle64, prob, steps=2, external_batch=batch)
+
+
+def test_config1_ten_sgd_steps_free_running(oracle64):
+    """BASELINE configs[0]: 10 SGD steps of DistMult with internal sampling, both sides
+    running freely from the same initial tables."""
+    prob = Problem(E=1000, R=10, T=20000, d=32, score="distmult", loss="logsigmoid", B=64, N=128, P=2,
+                   lr=0.1, seed=0, graph_seed=0)
+    gpu, orc = GpuSide(prob), OracleSide(prob, oracle64)
+    loss_dev = gpu.torch.zeros(1, dtype=gpu.torch.float32, device=gpu.ent.device)
+    for step in range(10):
+        gpu.kge.train_step(step, prob.lr, loss_out=loss_dev)
+        assert (gpu.kge.debug_export("BATCH") == np.concatenate(orc.sample(step))).all()
+        loss_o = orc.step(step, orc.sample(step))
+        assert_close(loss_dev.item(), loss_o, atol=1e-5, what=f"loss step {step}")
+    ent, rel, _ = gpu.tables()
+    assert_close(ent, orc.ent, atol=2e-6, what="entity table after 10 steps")
+    assert_close(rel, orc.rel, atol=2e-6, what="relation table after 10 steps")
+    assert gpu.kge.get_status() == 0
+    # run twice: bit-identical (no atomics on floats anywhere)
+    gpu2 = GpuSide(prob)
+    for step in range(10):
+        gpu2.kge.train_step(step, prob.lr)
+    assert (gpu2.tables()[0] == ent).all() and (gpu2.tables()[1] == rel).all()
+
+
+@pytest.mark.parametrize("score,p", [("transe", 1), ("rotate", 1)])
+def test_config2_full_size_step(oracle64, score, p):
+    """BASELINE configs[1] at full size, in the launch configuration the benchmark times:
+    100,000 entities, d = 128, B = N = 1,024, P = 4, log-sigmoid with margin 12, SGD 0.05."""
+    prob = Problem(E=100000, R=500, T=2000000, d=128, score=score, p_norm=p, loss="logsigmoid",
+                   B=1024, N=1024, P=4, gamma=12.0, adv_temp=1.0, lr=0.05, seed=0, graph_seed=1,
+                   relation_zipf=1.0)
+    gpu, orc = GpuSide(prob), OracleSide(prob, oracle64)
+    batch = orc.sample(0)
+    orc._pre = (orc.ent.copy(), orc.rel.copy(), None)
+    touched = np.unique(np.concatenate([batch[0], batch[2], batch[3]]))
+    before = orc.ent[touched].copy()
+    _check_step(gpu, orc, 0, batch, taps=True)
+    assert np.abs(orc.ent[touched] - before).max() > 1e-4      # the step moved the touched rows
+
+
+def test_host_entry_point_matches_device_entry_point(oracle64):
+    prob = Problem(E=500, R=7, T=20000, d=32, score="transe", p_norm=1, B=64, N=64, P=2, gamma=6.0, lr=0.05)
+    a, b = GpuSide(prob), GpuSide(prob)
+    t = a.torch
+    orc = OracleSide(prob, oracle64)
+    for step in range(3):
+        batch = orc.sample(step)
+        loss_a = t.zeros(1, dtype=t.float32, device=a.ent.device)
+        a.kge.train_step(step, prob.lr, *[a.dev_i32(x) for x in batch], loss_out=loss_a)
+        pinned = [t.from_numpy(x).pin_memory() for x in batch]
+        loss_b = t.zeros(1, dtype=t.float32).pin_memory()
+        b.kge.train_step_host(step, prob.lr, *pinned, loss_b)
+        assert loss_a.item() == loss_b.item()
+    assert (a.tables()[0] == b.tables()[0]).all() and (a.tables()[1] == b.tables()[1]).all()
+
+
+def test_out_of_range_id_sets_status_and_does_not_fault(oracle64):
+    prob = Problem(E=100, R=3, T=3000, d=16, score="transe", B=16, N=16, P=1, gamma=1.0)
+    gpu = GpuSide(prob)
+    orc = OracleSide(prob, oracle64)
+    batch = [x.copy() for x in orc.sample(0)]
+    batch[3][5] = 100                      # one past the table
+    gpu.kge.train_step(0, 0.1, *[gpu.dev_i32(x) for x in batch])
+    assert gpu.kge.get_status() == -8      # KGE_ERR_ID_RANGE, reported once, then cleared
+    assert gpu.kge.get_status() == 0
+    assert np.isfinite(gpu.tables()[0]).all()
