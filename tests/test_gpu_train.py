@@ -20,6 +20,7 @@ def _check_step(gpu, orc, step, batch, *, taps=True, rows_atol=2e-6):
     dev = [gpu.dev_i32(a) for a in batch]
     loss_dev = gpu.torch.zeros(1, dtype=gpu.torch.float32, device=gpu.ent.device)
     want = orc.grads(batch) if taps else None
+    grads_for_adam = (want or orc.grads(batch)) if prob.opt == "adam" else None
     gpu.kge.train_step(step, prob.lr, *dev, loss_out=loss_dev)
     assert gpu.kge.get_status() == 0
     loss_o = orc.step(step, batch)
@@ -50,13 +51,40 @@ def _check_step(gpu, orc, step, batch, *, taps=True, rows_atol=2e-6):
             assert (kge.debug_export(pre + "_SEG") == seg).all()
             assert (kge.debug_export(pre + "_PERM") == perm).all()
     ent, rel, relw = gpu.tables()
-    assert_close(ent, orc.ent, atol=rows_atol, what="entity table")
-    assert_close(rel, orc.rel, atol=rows_atol, what="relation table")
-    if relw is not None:
-        assert_close(relw, orc.relw, atol=rows_atol, what="normal table")
+    if prob.opt == "adam":
+        _check_adam_tables(prob, batch, grads_for_adam, (ent, rel, relw), (orc.ent, orc.rel, orc.relw), rows_atol)
+    else:
+        assert_close(ent, orc.ent, atol=rows_atol, what="entity table")
+        assert_close(rel, orc.rel, atol=rows_atol, what="relation table")
+        if relw is not None:
+            assert_close(relw, orc.relw, atol=rows_atol, what="normal table")
     for got, want_s, name in zip(gpu.states, orc.states, ("ent_state", "rel_state", "relw_state")):
         if got is not None:
             assert_close(got.cpu().numpy(), want_s, atol=1e-9, what=name)
+
+
+def _check_adam_tables(prob, batch, g, got, want, rows_atol):
+    """Adam divides by sqrt(v) + eps, so its step is discontinuous where a gradient
+    coordinate is zero: there fp32 rounding noise (1e-9) against the exact zero (the softmax
+    probabilities of a row sum to one, so e.g. a TransE-L1 coordinate with every tail on the
+    same side of q cancels exactly) decides a step of order lr.  Coordinates whose exact
+    gradient is below 1e-4 of the table's largest are only required to move by a bounded
+    amount (10 lr); all others meet the normal tolerance."""
+    heads, rels, tails, negs = batch
+    tabs = [np.zeros_like(want[0]), np.zeros_like(want[1]), None if want[2] is None else np.zeros_like(want[2])]
+    np.add.at(tabs[0], heads, g["dh"]); np.add.at(tabs[0], tails, g["dtpos"]); np.add.at(tabs[0], negs, g["dtneg"])
+    np.add.at(tabs[1], rels, g["dr"])
+    if tabs[2] is not None:
+        np.add.at(tabs[2], rels, g["dw"])
+    for name, gt, a, b in zip(("entity", "relation", "normal"), tabs, got, want):
+        if gt is None:
+            continue
+        ill = np.abs(gt) < 1e-4 * np.abs(gt).max()
+        a, b = np.asarray(a, np.float64), np.asarray(b, np.float64)
+        assert_close(np.where(ill, b, a), b, atol=rows_atol, what=name + " table (well-conditioned coordinates)")
+        assert (np.abs(a - b)[ill] <= 10 * prob.lr).all(), name
+        touched = np.abs(gt).max(axis=1) > 0
+        assert ill[touched].mean() < 0.25
 
 
 def _run(oracle64, prob, steps=2, taps=True, external_batch=None):
