@@ -1,0 +1,314 @@
+#!/usr/bin/env python
+"""Benchmark of the shared-negative scoring block: one "step" = one pass of the whole
+training hot path (sample, gather, score block, loss, backward, dedup, sparse update) over
+one synthetic batch.
+
+    python bench.py --gpus N --steps K --warmup W            # the CUDA library
+    python bench.py --impl reference --steps K --warmup W    # the CPU oracle, as it stands
+
+Prints ONE JSON line.  At N > 1 (launched by torch.distributed.run) every rank trains an
+independent replica on its own GPU -- the method's hot path exchanges nothing between
+devices -- and `value` is the sum over replicas divided by the slowest replica's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+import numpy as np
+
+import kge_synth
+
+METRIC = "positive triples/sec (fwd+bwd+update, N shared negs)"
+UNIT = "triples/s"
+
+# BASELINE configs[1]: 100,000 entities, 500 relations (Zipf 1.0), 2,000,000 triples with
+# Zipf(1.1) degrees, d = 128 fp32, log-sigmoid loss with margin 12 (self-adversarial
+# temperature 1), B = N = 1,024, P = 4, SGD lr 0.05.
+WORKLOADS = {
+    "c2_transe_l1": dict(E=100_000, R=500, T=2_000_000, d=128, score="transe", p_norm=1, loss="logsigmoid",
+                         opt="sgd", B=1024, N=1024, P=4, gamma=12.0, adv_temp=1.0, lr=0.05,
+                         entity_zipf=1.1, relation_zipf=1.0, graph_seed=1),
+    "c2_rotate_l1": dict(E=100_000, R=500, T=2_000_000, d=128, score="rotate", p_norm=1, loss="logsigmoid",
+                         opt="sgd", B=1024, N=1024, P=4, gamma=12.0, adv_temp=1.0, lr=0.05,
+                         entity_zipf=1.1, relation_zipf=1.0, graph_seed=1),
+    "c1_distmult": dict(E=1000, R=10, T=20_000, d=32, score="distmult", p_norm=1, loss="logsigmoid",
+                        opt="sgd", B=64, N=128, P=2, gamma=0.0, adv_temp=0.0, lr=0.1,
+                        entity_zipf=1.1, relation_zipf=0.0, graph_seed=0),
+}
+
+# fp32 CUDA-core peak used for "bound": "alu": 148 SMs x 128 fp32 lanes x 1.965 GHz, one
+# instruction per lane per clock (an FMA counts as one).
+ALU_PEAK_TOPS = 148 * 128 * 1.965e9 / 1e12
+
+# Algorithmic fp32 lane-operations per (query, negative, embedding coordinate) of each stage,
+# by pair kind: the minimum a CUDA-core evaluation of the definition needs.
+STAGE_OPS = {
+    "transe1": dict(block=2, accum_q=3, accum_t=3),     # sub, |.|+add  /  compare, sign-select, add
+    "rotate1": dict(block=3.5, accum_q=5, accum_t=5),   # per real coordinate; one sqrt / rsqrt per complex pair
+    "distmult1": dict(block=1, accum_q=1, accum_t=1),   # one FMA
+}
+
+
+def cfg_kwargs(w, seed):
+    return dict(num_entities=w["E"], num_relations=w["R"], dim=w["d"], score=w["score"], p_norm=w["p_norm"],
+                loss=w["loss"], opt=w["opt"], batch=w["B"], num_neg=w["N"], num_parts=w["P"], gamma=w["gamma"],
+                adv_temp=w["adv_temp"], lr=w["lr"], seed=seed)
+
+
+class ClockSampler:
+    """nvidia-smi samples (SM clock, throttle reasons) taken while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.rows, self.proc = [], None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for row in self.rows:
+            try:
+                sm.append(float(row[0])); mx.append(float(row[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, val in zip(names, row[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def measured_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return {"hbm_gbs": d.get("hbm_gbs"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "source": "fallback"}
+
+
+def oracle_step_time(w, batch_size, steps, warmup, seed=0):
+    """Seconds per oracle training step on a batch of `batch_size` positives x all N negatives."""
+    from oracle.kge_oracle import Oracle, make_config, num_threads
+    o = Oracle("f64")
+    kw = cfg_kwargs(w, seed)
+    kw["batch"] = batch_size
+    cfg = make_config(**kw)
+    h, r, t = kge_synth.make_graph(w["E"], w["R"], w["T"], seed=w["graph_seed"], entity_zipf=w["entity_zipf"],
+                                   relation_zipf=w["relation_zipf"])
+    ent, rel, relw = kge_synth.make_tables(w["E"], w["R"], w["d"], w["score"], seed=w["graph_seed"])
+    graph = o.graph_build(w["E"], w["R"], w["P"], h, r, t)
+    ent, rel = o.arr(ent), o.arr(rel)
+    relw = None if relw is None else o.arr(relw)
+    times = []
+    for step in range(warmup + steps):
+        batch = o.sample_batch(cfg, step, graph)
+        t0 = time.perf_counter()
+        o.train_step(cfg, w["lr"], step, ent, rel, relw, None, None, None, *batch)
+        dt = time.perf_counter() - t0
+        if step >= warmup:
+            times.append(dt)
+    return float(np.mean(times)), num_threads()
+
+
+def run_reference(args, w, name):
+    """The reference arm: the CPU oracle, untouched, on the machine's host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    P2 = w["P"] * w["P"]
+    # calibrate the per-step sample so that warmup + steps stay within about two minutes
+    t_cal, cores = oracle_step_time(w, 4 * P2, 1, 0)
+    per_pos = t_cal / (4 * P2)
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    b_ref = int(min(w["B"], max(P2, (budget / per_pos) // P2 * P2)))
+    t_step, cores = oracle_step_time(w, b_ref, args.steps, args.warmup)
+    value = b_ref / t_step
+    sample = (f"{args.steps} steps, each a full training step (sample, forward, backward, dedup, update) on "
+              f"{b_ref} of the workload's {w['B']} positives against all {w['N']} shared negatives")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_step * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": name, "entities": w["E"], "relations": w["R"], "triples": w["T"], "dim": w["d"],
+                       "batch": b_ref, "num_neg": w["N"], "parts": w["P"]},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, w, name):
+    import torch
+    import torch.distributed as dist
+    import paper_2211_12281_b200 as K
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    B, N = w["B"], w["N"]
+    h, r, t = kge_synth.make_graph(w["E"], w["R"], w["T"], seed=w["graph_seed"], entity_zipf=w["entity_zipf"],
+                                   relation_zipf=w["relation_zipf"])
+    ent, rel, relw = kge_synth.make_tables(w["E"], w["R"], w["d"], w["score"], seed=w["graph_seed"])
+    ent_d, rel_d = torch.from_numpy(ent).to(dev), torch.from_numpy(rel).to(dev)
+    relw_d = None if relw is None else torch.from_numpy(relw).to(dev)
+    kge = K.Kge(K.KgeConfig.make(**cfg_kwargs(w, seed=rank)))       # each replica draws its own batches
+    kge.bind(ent_d, rel_d, relw_d, num_triples=w["T"])
+    kge.graph_load(h, r, t)
+    loss = torch.zeros(1, dtype=torch.float32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # 2 x L2: evicts the tables between steps
+
+    def timed_steps(first_step, count, fn):
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(count)]
+        for i, (a, b) in enumerate(evs):
+            flush.zero_()
+            a.record()
+            fn(first_step + i)
+            b.record()
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in evs]
+
+    step_fn = lambda s: kge.train_step(s, w["lr"], loss_out=loss)
+    warm = max(args.warmup, 3)
+    timed_steps(0, warm, step_fn)
+    assert kge.get_status() == 0
+
+    # ---- device-resident timing: K steps, CUDA events on the launching stream ----
+    barrier()
+    clocks = ClockSampler(local)
+    launches0 = kge.launch_count()
+    ms = timed_steps(warm, args.steps, step_fn)
+    barrier()
+    clock_info = clocks.stop()
+    launches = kge.launch_count() - launches0
+    total_ms = float(np.sum(ms))
+    if world > 1:
+        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = tt.item()
+    ms_per_step = total_ms / args.steps
+    value = world * B / (ms_per_step * 1e-3)
+    assert np.isfinite(loss.item()) and kge.get_status() == 0
+
+    # ---- end to end: ids in pinned host memory -> H2D, step, loss -> D2H, every step ----
+    nxt = warm + args.steps
+    ids_dev = [torch.empty(n, dtype=torch.int32, device=dev) for n in (B, B, B, N)]
+    pinned = []
+    for i in range(args.steps):
+        kge.sample_batch(nxt + i, *ids_dev)
+        pinned.append([x.cpu().pin_memory() for x in ids_dev])
+    loss_host = torch.zeros(1, dtype=torch.float32).pin_memory()
+    host_fn = lambda s: kge.train_step_host(s, w["lr"], *pinned[s - nxt], loss_host)
+    barrier()
+    e2e_ms = float(np.sum(timed_steps(nxt, args.steps, host_fn)))
+    barrier()
+    if world > 1:
+        tt = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = tt.item()
+    e2e_value = world * B / (e2e_ms / args.steps * 1e-3)
+    nxt += args.steps
+
+    # ---- per-kernel times (CUDA events around every launch, same stream) for the roofline ----
+    kge.profile(True)
+    prof_steps = min(args.steps, 100)
+    timed_steps(nxt, prof_steps, step_fn)
+    stages = kge.profile_read()
+    kge.profile(False)
+    per_stage_us = {k: 1e3 * v[0] / v[1] for k, v in stages.items() if v[1] > 0}
+    kind = f"{w['score']}{w['p_norm']}"
+    ops = STAGE_OPS.get(kind, {})
+    compute_stages = [s for s in ("block", "accum_q", "accum_t") if s in per_stage_us]
+    dominant = max(compute_stages, key=lambda s: per_stage_us[s])
+    roofline = None
+    if dominant in ops:
+        alg_ops = ops[dominant] * B * N * w["d"]
+        achieved = alg_ops / (per_stage_us[dominant] * 1e-6) / 1e12
+        roofline = {"bound": "alu", "kernel": dominant, "achieved": achieved, "peak": ALU_PEAK_TOPS,
+                    "unit": "TFLOP/s", "frac": achieved / ALU_PEAK_TOPS, "traffic": None,
+                    "op": "one fp32 CUDA-core instruction per lane (FMA = 1)",
+                    "peak_source": "148 SMs x 128 lanes x 1.965 GHz", "us_per_launch": per_stage_us[dominant]}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": name, "entities": w["E"], "relations": w["R"], "triples": w["T"], "dim": w["d"],
+                       "batch": B, "num_neg": N, "parts": w["P"], "score": w["score"], "p_norm": w["p_norm"],
+                       "loss": w["loss"], "opt": w["opt"], "replicas": world,
+                       "l2": "flushed between steps (256 MiB write), untimed"},
+            "scored_pairs_per_s": world * B * (N + 1) / (ms_per_step * 1e-3),
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": (3 * B + N) * 4, "d2h_bytes_per_step": 4},
+            "gpu_launches": int(launches), "clocks": clock_info, "roofline": roofline,
+            "stage_us": per_stage_us, "loss": loss.item()}
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        b_cpu = min(B, 256)
+        t_step, cores = oracle_step_time(w, b_cpu, 2, 1)
+        line["cpu_baseline"] = {"value": b_cpu / t_step, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"2 full training steps on {b_cpu} of the {B} positives against all {N} "
+                                          f"shared negatives (fp64 oracle, OpenMP)"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="c2_transe_l1")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w, args.workload)
+    else:
+        run_ours(args, w, args.workload)
+
+
+if __name__ == "__main__":
+    main()
