@@ -60,7 +60,8 @@ def _check_step(gpu, orc, step, batch, *, taps=True, rows_atol=2e-6):
             assert_close(relw, orc.relw, atol=rows_atol, what="normal table")
     for got, want_s, name in zip(gpu.states, orc.states, ("ent_state", "rel_state", "relw_state")):
         if got is not None:
-            assert_close(got.cpu().numpy(), want_s, atol=1e-9, what=name)
+            # moments are linear / quadratic in a gradient that is itself a cancelling sum
+            assert_close(got.cpu().numpy(), want_s, atol=2e-5 * float(np.abs(want_s).max()) + 1e-12, what=name)
 
 
 def _check_adam_tables(prob, batch, g, got, want, rows_atol):
