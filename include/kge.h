@@ -165,6 +165,30 @@ int kge_score_all_topk(kge_handle* h, const int32_t* q_heads, const int32_t* q_r
                        void* stream);
 
 /*
+ * (No counterpart in the paper: an addition for callers that cannot allocate.)
+ * kge_score_all_topk for programs that must not call cudaMalloc -- an inference service whose
+ * whole GPU memory is already handed to another allocator, a plugin that runs under a host
+ * which forbids allocation after start-up, a loop that cannot afford the device-wide
+ * synchronisation an allocation may imply.  It takes no handle and no workspace: the tables,
+ * the queries and the outputs are the caller's device arrays as in kge_score_all_topk, and
+ * every intermediate lives in one fixed array of 804,608 bytes that is part of the library
+ * image, so each GPU that loads the library holds it until the process exits.  Only the
+ * fields num_entities, num_relations, dim, score and p_norm of `cfg` [host] are read.
+ * Limits of the fixed array: nq <= 64, k <= 32, dim <= 512; anything larger is refused with
+ * KGE_ERR_WORKSPACE before any launch.  No device or host memory is allocated or freed.
+ * The first call on a device looks up the array's device address (with that device
+ * current); make that first call outside any stream capture.  All calls share the one
+ * array: it keeps the previous call's contents (this entry point clears what must start at
+ * zero), and two calls that overlap on the same GPU -- from different streams or threads --
+ * race on it, so serialise them.  Synchronises `stream`; returns 0, an argument error, or the
+ * code recorded on the device (KGE_ERR_ID_RANGE).
+ */
+int kge_score_all_topk_static(const kge_config* cfg /*[host]*/, const float* ent, const float* rel,
+                              const float* relw, const int32_t* q_heads, const int32_t* q_rels, int32_t nq,
+                              int32_t k, const int32_t* true_tails, int32_t* out_ids, float* out_scores,
+                              int32_t* out_ranks, void* stream);
+
+/*
  * Mean reciprocal rank of the true tails (task metric of Section 2): mean over queries of
  * 1/rank if rank <= k_cutoff else 0; k_cutoff = 10 is the paper's metric, 0 = no cut-off.
  * mrr_out: [host] double.  Synchronises `stream`.

@@ -79,6 +79,8 @@ SIGNATURES = {
     "kge_train_step": (C.c_int, [_vp, C.c_uint64, C.c_float, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kge_train_step_host": (C.c_int, [_vp, C.c_uint64, C.c_float, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kge_score_all_topk": (C.c_int, [_vp, _vp, _vp, C.c_int32, C.c_int32, _vp, _vp, _vp, _vp, _vp]),
+    "kge_score_all_topk_static": (C.c_int, [C.POINTER(KgeConfig), _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32, _vp, _vp, _vp,
+                                            _vp, _vp]),
     "kge_eval_mrr": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int32, C.c_int32, C.POINTER(C.c_double), _vp]),
     "kge_get_status": (C.c_int, [_vp, _vp]),
     "kge_launch_count": (C.c_int64, [_vp]),
@@ -123,6 +125,15 @@ def _ptr(t):
 def _stream():
     import torch
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def score_all_topk_static(cfg: KgeConfig, ent, rel, relw, q_heads, q_rels, k, true_tails, out_ids, out_scores,
+                          out_ranks=None) -> int:
+    """kge_score_all_topk_static: full-entity top-k without a handle, a workspace or any
+    allocation (at most 64 queries, k <= 32, dim <= 512).  Returns the C status code."""
+    return int(lib().kge_score_all_topk_static(C.byref(cfg), _ptr(ent), _ptr(rel), _ptr(relw), _ptr(q_heads),
+                                               _ptr(q_rels), q_heads.numel(), k, _ptr(true_tails), _ptr(out_ids),
+                                               _ptr(out_scores), _ptr(out_ranks), _stream()))
 
 
 class Kge:

@@ -386,3 +386,96 @@ int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int3
 }
 
 }  // namespace kge
+
+// ------------------------------------------------------------------------------------------
+// Full-entity scoring for callers that may not allocate device memory.  All scratch lives in
+// one file-scope device array that every GPU loading the library holds until the process
+// exits; nothing is allocated or freed here, on the host heap or on the device.
+// ------------------------------------------------------------------------------------------
+namespace kge {
+namespace {
+
+constexpr int kStaticMaxQueries = 64;
+constexpr int kStaticMaxTopk = 32;
+constexpr size_t kStaticQueryRows = (size_t)kStaticMaxQueries * kMaxDim * sizeof(float);       // 131072
+constexpr size_t kStaticCandList = (size_t)kStaticMaxQueries * kCandCap * 4;                   // 262144
+constexpr size_t kStaticTopList = (size_t)kStaticMaxQueries * kStaticMaxTopk * 4;              // 8192
+constexpr size_t kStaticSmall = 256;                                                            // >= 64 x 4 bytes
+constexpr size_t kStaticBytes = 256 + 2 * kStaticQueryRows + 6 * kStaticSmall + 2 * kStaticCandList + 2 * kStaticTopList;
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];   // 804,608 bytes per GPU
+
+constexpr int kStaticMaxDevices = 64;
+void* g_static_scratch_addr[kStaticMaxDevices] = {};   // device address of the array, per device ordinal
+
+}  // namespace
+}  // namespace kge
+
+extern "C" int kge_score_all_topk_static(const kge_config* cfg, const float* ent, const float* rel,
+                                         const float* relw, const int32_t* q_heads, const int32_t* q_rels,
+                                         int32_t nq, int32_t k, const int32_t* true_tails, int32_t* out_ids,
+                                         float* out_scores, int32_t* out_ranks, void* stream) {
+    using namespace kge;
+    if (!cfg || !ent || !rel || !q_heads || !q_rels || !out_ids || !out_scores || nq < 0 || k <= 0)
+        return KGE_ERR_BAD_ARG;
+    if (out_ranks && !true_tails) return KGE_ERR_BAD_ARG;
+    const kge_config& c = *cfg;
+    if (c.num_entities <= 0 || c.num_entities > INT32_MAX || c.num_relations <= 0 || c.num_relations > INT32_MAX ||
+        c.dim <= 0 || c.dim % 4 != 0 || c.score < KGE_TRANSE || c.score > KGE_COMPLEX ||
+        (c.p_norm != 1 && c.p_norm != 2) || (c.score == KGE_TRANSH && !relw))
+        return KGE_ERR_BAD_ARG;
+    // the fixed scratch bounds the problem: refuse anything it cannot hold
+    if (nq > kStaticMaxQueries || k > kStaticMaxTopk || c.dim > kMaxDim) return KGE_ERR_WORKSPACE;
+    if (nq == 0) return KGE_OK;
+
+    kge_handle h;                       // plain host object on the stack; nothing in it is heap-backed here
+    h.cfg = c;
+    h.kw = c.score == KGE_ROTATE ? c.dim / 2 : c.dim;
+    h.kind = kind_of(c);
+    h.ent = const_cast<float*>(ent); h.rel = const_cast<float*>(rel); h.relw = const_cast<float*>(relw);
+    h.ent_state = h.rel_state = h.relw_state = nullptr;
+    h.launches = 0; h.bound = true; h.graph_loaded = false;
+    h.max_queries = kStaticMaxQueries; h.topk = kStaticMaxTopk;
+
+    // Set-up, once per device and with that device current: in host code the array's name is
+    // only a stand-in, so its device address has to be asked for.
+    int dev = -1;
+    KGE_CUDA_CHECK(&h, cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kStaticMaxDevices) return KGE_ERR_UNSUPPORTED;
+    if (!g_static_scratch_addr[dev]) {
+        void* addr = nullptr;
+        KGE_CUDA_CHECK(&h, cudaGetSymbolAddress(&addr, g_static_scratch));
+        g_static_scratch_addr[dev] = addr;
+    }
+    unsigned char* base = static_cast<unsigned char*>(g_static_scratch_addr[dev]);
+
+    Workspace w{};
+    size_t o = 0;
+    auto take = [&](size_t bytes) { unsigned char* p = base + o; o += bytes; return p; };
+    w.status = reinterpret_cast<int32_t*>(take(256));
+    w.iq = reinterpret_cast<float*>(take(kStaticQueryRows));
+    w.iwhat = reinterpret_cast<float*>(take(kStaticQueryRows));
+    w.iftrue = reinterpret_cast<float*>(take(kStaticSmall));
+    w.thr = reinterpret_cast<float*>(take(kStaticSmall));
+    w.thr_id = reinterpret_cast<int32_t*>(take(kStaticSmall));
+    w.cand_cnt = reinterpret_cast<int32_t*>(take(kStaticSmall));
+    w.beat_tmp = reinterpret_cast<int32_t*>(take(kStaticSmall));
+    w.beat = reinterpret_cast<int32_t*>(take(kStaticSmall));
+    w.cand_score = reinterpret_cast<float*>(take(kStaticCandList));
+    w.cand_id = reinterpret_cast<int32_t*>(take(kStaticCandList));
+    w.top_score = reinterpret_cast<float*>(take(kStaticTopList));
+    w.top_id = reinterpret_cast<int32_t*>(take(kStaticTopList));
+    if (o != kStaticBytes) return KGE_ERR_WORKSPACE;
+    h.ws = w;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the array still holds the previous call's words: the status header must start at zero
+    // (the per-query state is rewritten by the query set-up kernel)
+    KGE_CUDA_CHECK(&h, cudaMemsetAsync(w.status, 0, 256, s));
+    int rc = run_score_all_topk(&h, q_heads, q_rels, nq, k, true_tails, out_ids, out_scores, out_ranks, s);
+    if (rc != KGE_OK) return rc;
+    int32_t word = 0;
+    KGE_CUDA_CHECK(&h, cudaMemcpyAsync(&word, w.status, 4, cudaMemcpyDeviceToHost, s));
+    KGE_CUDA_CHECK(&h, cudaStreamSynchronize(s));
+    return word;   // 0, or the code a kernel recorded (an id outside its table)
+}
