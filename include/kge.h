@@ -14,7 +14,9 @@
  *   detected on the host before anything is launched.  Problems found on the device (an
  *   id outside its table, a top-k candidate list that filled up) never trap: the kernel
  *   records a code in a sticky status word inside the workspace, substitutes row 0 for the
- *   offending id, and carries on; kge_get_status() reports and clears it.
+ *   offending id, and carries on; kge_get_status() reports and clears it.  Every wait of a
+ *   kernel on an asynchronous copy is bounded; if one runs out the kernel records
+ *   KGE_ERR_TIMEOUT and returns.
  * - Layouts: tables are row-major fp32 [rows, dim] with dim % 4 == 0 and 16-byte aligned
  *   bases.  Complex rows (RotatE, ComplEx) are interleaved (re0, im0, re1, im1, ...), the
  *   identification of C^(d/2) with R^d of the scoring-function table.  A RotatE relation
@@ -56,7 +58,8 @@ typedef enum {
     KGE_ERR_CUDA = -7,           /* a CUDA runtime call failed (see kge_last_cuda_error) */
     KGE_ERR_ID_RANGE = -8,       /* device: an entity / relation id was outside its table */
     KGE_ERR_TOPK_OVERFLOW = -9,  /* device: a candidate list overflowed and could not be recovered */
-    KGE_ERR_NO_EXTENSION = -10   /* used by the Python binding when the shared library is missing */
+    KGE_ERR_NO_EXTENSION = -10,  /* used by the Python binding when the shared library is missing */
+    KGE_ERR_TIMEOUT = -11        /* device: a bounded wait on an asynchronous copy ran out; the step's results are invalid */
 } kge_status;
 
 typedef struct {

@@ -26,12 +26,12 @@ struct Carver {
 };
 
 int pick_split(int rows, int cols, int num_sms) {
-    // One CTA covers 32 owner rows; aim for about two CTAs per SM, never splitting the
-    // reduced dimension into pieces shorter than 32.
-    int row_ctas = (rows + 31) / 32;
-    int want = (2 * num_sms + row_ctas - 1) / row_ctas;
-    int max_split = std::max(1, cols / 32);
-    return std::max(1, std::min(std::min(want, max_split), 16));
+    // One CTA covers 32 owner rows and walks its share of the reduced dimension in chunks of
+    // 32; aim for about four CTAs per SM, at most 16 splits, and no empty split.
+    const int row_ctas = (rows + 31) / 32;
+    const int want = std::max(1, std::min((4 * num_sms + row_ctas / 2) / row_ctas, 16));
+    const int per = ((cols + want - 1) / want + 31) / 32 * 32;
+    return std::max(1, (cols + per - 1) / per);
 }
 
 size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t topk, Workspace* out) {
@@ -53,6 +53,8 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
     w.What = th ? cv.take<float>(B * d) : nullptr;
     w.Tneg = cv.take<float>(N * d);
     w.fpos = cv.take<float>(B); w.gpos = cv.take<float>(B); w.Lrow = cv.take<float>(B);
+    w.Grow = cv.take<float>(B);
+    w.Cpart = cv.take<float>((size_t)h->split_t * N);
     w.F = cv.take<float>(B * N);
     w.U = th ? cv.take<float>(B * N) : nullptr;
     w.Cc = th ? cv.take<float>(B * N) : nullptr;
@@ -67,6 +69,12 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
     w.ent_uniq = cv.take<int32_t>(ne); w.ent_seg = cv.take<int32_t>(ne + 1);
     w.rel_perm = cv.take<int32_t>(B); w.rel_sorted = cv.take<int32_t>(B);
     w.rel_uniq = cv.take<int32_t>(B); w.rel_seg = cv.take<int32_t>(B + 1);
+    w.ent_segof = cv.take<int32_t>(ne); w.rel_segof = cv.take<int32_t>(B);
+    w.ent_tkeys = cv.take<uint64_t>((size_t)dedup_tiles((int)ne) * 1024);
+    w.rel_tkeys = cv.take<uint64_t>((size_t)dedup_tiles((int)B) * 1024);
+    w.part_ent = cv.take<float>(ne * d);
+    w.part_rel = cv.take<float>(B * kw);
+    w.part_relw = th ? cv.take<float>(B * d) : nullptr;
     if (maxq > 0) {
         const size_t q = maxq, k = std::max(topk, 1);
         w.iq = cv.take<float>(q * d);
@@ -125,6 +133,7 @@ int kge_create(const kge_config* cfg, kge_handle** out) {
     h->kw = c.score == KGE_ROTATE ? c.dim / 2 : c.dim;
     h->kind = kind_of(c);
     h->bound = h->graph_loaded = false;
+    h->streams_ready = false;
     h->launches = 0;
     h->num_sms = 148;
     int dev = 0, sms = 0;
@@ -143,6 +152,10 @@ void kge_destroy(kge_handle* h) {
     if (!h) return;
     if (h->prof.created)
         for (int i = 0; i < ST_COUNT; ++i) { cudaEventDestroy(h->prof.a[i]); cudaEventDestroy(h->prof.b[i]); }
+    if (h->streams_ready) {
+        cudaStreamDestroy(h->side[0]); cudaStreamDestroy(h->side[1]);
+        cudaEventDestroy(h->ev_ids); cudaEventDestroy(h->ev_loss); cudaEventDestroy(h->ev_seg); cudaEventDestroy(h->ev_t);
+    }
     delete h;
 }
 
@@ -194,6 +207,13 @@ int kge_bind(kge_handle* h, float* ent, float* rel, float* relw, float* ent_stat
     h->num_triples = num_triples; h->max_queries = max_queries; h->topk = topk;
     layout(h, h->ws_base, num_triples, max_queries, topk, &h->ws);
     KGE_CUDA_CHECK(h, cudaMemsetAsync(h->ws.status, 0, 256, static_cast<cudaStream_t>(stream)));
+    if (!h->streams_ready) {
+        KGE_CUDA_CHECK(h, cudaStreamCreateWithFlags(&h->side[0], cudaStreamNonBlocking));
+        KGE_CUDA_CHECK(h, cudaStreamCreateWithFlags(&h->side[1], cudaStreamNonBlocking));
+        cudaEvent_t* evs[4] = {&h->ev_ids, &h->ev_loss, &h->ev_seg, &h->ev_t};
+        for (cudaEvent_t* e : evs) KGE_CUDA_CHECK(h, cudaEventCreateWithFlags(e, cudaEventDisableTiming));
+        h->streams_ready = true;
+    }
     h->bound = true;
     h->graph_loaded = false;
     return KGE_OK;
@@ -267,9 +287,23 @@ int kge_train_step(kge_handle* h, uint64_t step, float lr, const int32_t* heads,
         if (rc != KGE_OK) return rc;
         heads = w.heads; rels = w.rels; tails = w.tails; negs = w.negs;
     }
-    int rc = launch_forward_backward(h, heads, rels, tails, negs, s);
+    // With per-stage timing on, everything runs in order on the caller's stream.  Otherwise
+    // the sort of the touched ids (which needs only the ids) runs on a side stream beside
+    // the forward and backward kernels, and joins before the update.
+    const bool fork = !h->prof.on;
+    int rc;
+    if (fork) {
+        KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_ids, s));
+        KGE_CUDA_CHECK(h, cudaStreamWaitEvent(h->side[0], h->ev_ids, 0));
+        rc = launch_dedup(h, heads, rels, tails, negs, h->side[0]);
+        if (rc != KGE_OK) return rc;
+        KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_seg, h->side[0]));
+    }
+    rc = launch_forward_backward(h, heads, rels, tails, negs, loss_out, s, fork ? h->side[1] : nullptr);
     if (rc != KGE_OK) return rc;
-    rc = launch_dedup_update(h, step, lr, heads, rels, tails, negs, loss_out, s);
+    if (fork) KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_seg, 0));
+    else if ((rc = launch_dedup(h, heads, rels, tails, negs, s)) != KGE_OK) return rc;
+    rc = launch_update(h, step, lr, s);
     if (rc != KGE_OK) return rc;
     return h->prof.on ? stage_collect(h, s) : KGE_OK;
 }
@@ -367,6 +401,7 @@ const char* kge_error_string(int code) {
         case KGE_ERR_ID_RANGE: return "an entity or relation id was outside its table";
         case KGE_ERR_TOPK_OVERFLOW: return "top-k candidate list overflow";
         case KGE_ERR_NO_EXTENSION: return "CUDA extension not built";
+        case KGE_ERR_TIMEOUT: return "a bounded wait on an asynchronous copy ran out";
         default: return "unknown error";
     }
 }

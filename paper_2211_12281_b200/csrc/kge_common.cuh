@@ -46,6 +46,8 @@ struct Workspace {
     int32_t *heads, *rels, *tails, *negs;  // contiguous [3B+N]
     float *Q, *What, *Tneg;                // [B,d], [B,d] (TransH), [N,d]
     float *fpos, *gpos, *Lrow;             // [B]
+    float *Grow;                           // [B] row sums of dL/dF (TransE p=1 backward)
+    float *Cpart;                          // [St, N] column sums of dL/dF per row split (TransE p=1 backward)
     float *F;                              // [B,N] scores, overwritten by dL/dF
     float *U, *Cc;                         // [B,N] TransH: w.t and the S.w contraction
     float *dQpart, *dWpart, *dTpart;       // [Sq,B,d], [Sq,B,d] (TransH), [St,N,d]
@@ -53,6 +55,9 @@ struct Workspace {
     // dedup
     int32_t *ent_perm, *ent_sorted, *ent_uniq, *ent_seg;  // [2B+N], [2B+N], [2B+N], [2B+N+1]
     int32_t *rel_perm, *rel_sorted, *rel_uniq, *rel_seg;  // [B] ...
+    int32_t *ent_segof, *rel_segof;        // [2B+N], [B] segment index of every sorted position
+    uint64_t *ent_tkeys, *rel_tkeys;       // tile-sorted (id, position) keys, padded to whole tiles
+    float *part_ent, *part_rel, *part_relw;  // [list length, width] partial sums of long segments
     // inference
     float *iq, *iwhat, *iftrue;            // [maxq,d], [maxq,d], [maxq]
     float *thr;                            // [maxq] current k-th best score (-inf until the list is full)
@@ -94,6 +99,11 @@ struct kge_handle {
     bool bound, graph_loaded;
     int64_t launches;
     int num_sms;
+    // Side streams and events of the training step: the sort of the touched ids and one of the
+    // two backward accumulations run beside the main stream's kernels (created by kge_bind).
+    bool streams_ready;
+    cudaStream_t side[2];
+    cudaEvent_t ev_ids, ev_loss, ev_seg, ev_t;
     std::string cuda_err;
 };
 
@@ -130,10 +140,15 @@ int stage_collect(kge_handle* h, cudaStream_t s);
 // ---- launch wrappers implemented in the other translation units ----
 int launch_sample(kge_handle* h, uint64_t step, int32_t* heads, int32_t* rels, int32_t* tails, int32_t* negs,
                   cudaStream_t s);
+// Forward and backward; `side` (or NULL) runs the accumulation over the queries concurrently.
 int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* rels, const int32_t* tails,
-                            const int32_t* negs, cudaStream_t s);
-int launch_dedup_update(kge_handle* h, uint64_t step, float lr, const int32_t* heads, const int32_t* rels,
-                        const int32_t* tails, const int32_t* negs, float* loss_out, cudaStream_t s);
+                            const int32_t* negs, float* loss_out, cudaStream_t s, cudaStream_t side);
+// Stable sort of the touched ids, distinct ids and segments (needs only the batch ids).
+int launch_dedup(kge_handle* h, const int32_t* heads, const int32_t* rels, const int32_t* tails,
+                 const int32_t* negs, cudaStream_t s);
+// Segment sums of the gradient rows and the optimiser step (needs both of the above).
+int launch_update(kge_handle* h, uint64_t step, float lr, cudaStream_t s);
+int dedup_tiles(int n);     // sort tiles of a list of n ids
 int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int32_t nq, int32_t k,
                        const int32_t* true_tails, int32_t* out_ids, float* out_scores, int32_t* out_ranks,
                        cudaStream_t s);
@@ -161,6 +176,40 @@ __device__ __forceinline__ int64_t checked_id(int32_t id, int64_t rows, int32_t*
         return 0;
     }
     return id;
+}
+
+// ---- asynchronous bulk copies (TMA engine, untiled form) completing on a shared-memory barrier ----
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t arrivals) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(arrivals) : "memory");
+}
+// Makes freshly initialised barriers visible to the asynchronous proxy; follow with __syncthreads().
+__device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Polls the barrier phase `parity` a bounded number of times; false = gave up.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+    for (int i = 0; i < (1 << 20); ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 128) __nanosleep(64);
+    }
+    return false;
+}
+// dst (shared) and src (global) 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
 __device__ __forceinline__ float softplusf(float z) { return fmaxf(z, 0.f) + log1pf(expf(-fabsf(z))); }

@@ -18,6 +18,7 @@ struct TrainParams {
     const float *ent, *rel, *relw;
     const int32_t *heads, *rels, *tails, *negs;
     int split_q, split_t;
+    float* loss_out;    // caller's device scalar for the batch loss, or NULL
     Workspace w;
 };
 
@@ -33,7 +34,6 @@ __device__ __forceinline__ float f4dot(float4 a, float4 b) { return a.x * b.x + 
 __device__ __forceinline__ float sgnf(float x) { return (x > 0.f ? 1.f : 0.f) - (x < 0.f ? 1.f : 0.f); }
 __device__ __forceinline__ float4 f4sgn(float4 a) { return make_float4(sgnf(a.x), sgnf(a.y), sgnf(a.z), sgnf(a.w)); }
 
-constexpr int kMaxChunks = kMaxDim / 128;  // float4 chunks per lane when one warp owns a row
 
 // ------------------------------------------------------------------------------------------
 // build: one warp per row.  Warps [0, B) build q_b and f+_b; warps [B, B+N) stage t-_n.
@@ -48,6 +48,7 @@ __device__ __forceinline__ float pair_partial(int kind, float4 q, float4 t) {
     return f4dot(x, x);
 }
 
+template <int kMaxChunks>   // float4 slices per lane: a warp owns a row
 __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
@@ -279,10 +280,112 @@ __global__ void __launch_bounds__(256) block_kernel(TrainParams p) {
 }
 
 // ------------------------------------------------------------------------------------------
-// loss: one CTA per positive.  Overwrites F[b,:] with loss_scale * dL_b/dF_bn (divided by the
-// distance for p = 2 kinds, which is the factor every later use needs).
+// block, kinds that are a function of (q, t) alone: 64 x 64 pairs per CTA, 4 x 4 per thread.
+// The 64 query rows and 64 negative rows of the tile are brought into shared memory by one
+// asynchronous bulk copy per row (padded rows, so the 128-bit reads below are conflict-free),
+// up to 128 floats of the embedding axis per stage, two stages when the rows are longer.
 // ------------------------------------------------------------------------------------------
-constexpr int LOSS_THREADS = 128;
+constexpr int FKC = 128;
+
+__host__ __device__ inline int block_tma_kc(int d) { return d < FKC ? d : FKC; }
+__host__ __device__ inline int block_tma_stages(int d) { return d > FKC ? 2 : 1; }
+inline size_t block_tma_smem(int d) {
+    return (size_t)block_tma_stages(d) * 2 * TB * (block_tma_kc(d) + 4) * sizeof(float) + 2 * sizeof(uint64_t);
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(256) block_tma_kernel(TrainParams p) {
+    extern __shared__ __align__(128) unsigned char smraw[];
+    const int kc = block_tma_kc(p.d), ld = kc + 4, nstage = block_tma_stages(p.d);
+    const int nchunk = (p.d + kc - 1) / kc;
+    float* base = reinterpret_cast<float*>(smraw);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smraw + (size_t)nstage * 2 * TB * ld * sizeof(float));
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int b0 = blockIdx.y * TB, n0 = blockIdx.x * TN;
+
+    if (tid == 0) {
+        for (int st = 0; st < nstage; ++st) mbar_init(&bars[st], 2 * TB);
+        mbar_init_fence();
+    }
+    __syncthreads();
+
+    // rows [0, 64) of a stage hold queries, rows [64, 128) negatives; thread r < 128 owns row r
+    auto issue = [&](int chunk, int stage) {
+        if (tid >= 2 * TB) return;
+        const bool isq = tid < TB;
+        const int g = isq ? b0 + tid : n0 + tid - TB;
+        float* dst = base + ((size_t)stage * 2 * TB + tid) * ld;
+        const int k0 = chunk * kc, len = min(kc, p.d - k0);
+        if (g < (isq ? p.B : p.N)) {
+            const float* src = (isq ? p.w.Q : p.w.Tneg) + (int64_t)g * p.d + k0;
+            mbar_arrive_expect_tx(&bars[stage], (uint32_t)len * 4u);
+            bulk_g2s(dst, src, (uint32_t)len * 4u, &bars[stage]);
+        } else {
+            if (chunk < nstage)   // rows outside the problem stay zero for the whole kernel
+                for (int k = 0; k < kc; k += 4) *reinterpret_cast<float4*>(dst + k) = f4zero();
+            mbar_arrive(&bars[stage]);
+        }
+    };
+    issue(0, 0);
+    if (nstage > 1 && nchunk > 1) issue(1, 1);
+
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int chunk = 0; chunk < nchunk; ++chunk) {
+        const int stage = chunk % nstage;
+        const bool ok = mbar_wait_bounded(&bars[stage], (uint32_t)(chunk / nstage) & 1u);
+        if (!__syncthreads_and(ok)) {
+            if (tid == 0) set_status(p.w.status, KGE_ERR_TIMEOUT);
+            // give copies still in flight a bounded chance to land before shared memory is released
+            for (int st = 0; st < nstage; ++st) (void)mbar_wait_bounded(&bars[st], (uint32_t)(chunk / nstage) & 1u);
+            return;
+        }
+        const float* Qs = base + (size_t)stage * 2 * TB * ld;
+        const float* Ts = Qs + TB * ld;
+        const int len = min(kc, p.d - chunk * kc);
+#pragma unroll 2
+        for (int kk = 0; kk < len; kk += 4) {
+            float4 qv[4], tv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                qv[i] = *reinterpret_cast<const float4*>(&Qs[(ty + 16 * i) * ld + kk]);
+                tv[i] = *reinterpret_cast<const float4*>(&Ts[(tx + 16 * i) * ld + kk]);
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) pair_update<KIND>(acc[i][j], qv[i], tv[j]);
+        }
+        if (chunk + nstage < nchunk) {
+            __syncthreads();             // every thread is done reading this stage
+            issue(chunk + nstage, stage);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int b = b0 + ty + 16 * i, n = n0 + tx + 16 * j;
+            if (b >= p.B || n >= p.N) continue;
+            float f = acc[i][j];
+            if (KIND == KIND_L1 || KIND == KIND_CL1) f = -f;
+            else if (KIND == KIND_L2) f = -sqrtf(f);
+            p.w.F[(int64_t)b * p.N + n] = f;
+        }
+}
+
+// ------------------------------------------------------------------------------------------
+// loss: one CTA per positive.  The row of scores is read once into shared memory (rows too
+// long for it are re-read from global memory), then overwritten with loss_scale * dL_b/dF_bn
+// (divided by the distance for p = 2 kinds, which is the factor every later use needs).
+// Also leaves the row sum of what it wrote, used by the TransE p = 1 backward.
+// ------------------------------------------------------------------------------------------
+constexpr int LOSS_THREADS = 256;
+constexpr int LOSS_SMEM_FLOATS = 24 * 1024;   // rows up to 24,576 scores are staged in shared memory
 
 __device__ __forceinline__ float block_sum(float v, float* sm) {
     v = warp_sum(v);
@@ -305,58 +408,127 @@ __device__ __forceinline__ float block_max(float v, float* sm) {
     return t;
 }
 
-__global__ void __launch_bounds__(LOSS_THREADS) loss_kernel(TrainParams p) {
-    __shared__ float sm[LOSS_THREADS / 32];
-    const int b = blockIdx.x, tid = threadIdx.x;
-    float* Frow = p.w.F + (int64_t)b * p.N;
+// softplus(z) and sigmoid(z) from one exponential.
+__device__ __forceinline__ void softplus_sigmoid(float z, float& sp, float& sg) {
+    const float e = expf(-fabsf(z));
+    sp = fmaxf(z, 0.f) + log1pf(e);
+    const float r = 1.f / (1.f + e);
+    sg = z >= 0.f ? r : e * r;
+}
+
+struct BlockReduce {   // all LOSS_THREADS threads of the CTA work on one row
+    float* sm;
+    __device__ __forceinline__ float sum(float v) const { return block_sum(v, sm); }
+    __device__ __forceinline__ float max(float v) const { return block_max(v, sm); }
+};
+struct WarpReduce {    // one warp works on one row
+    __device__ __forceinline__ float sum(float v) const { return warp_sum(v); }
+    __device__ __forceinline__ float max(float v) const { return warp_max(v); }
+};
+
+// Loss and dL/dF of positive b.  `row` holds the scores (shared or global memory), the
+// calling threads cover it as t0, t0 + stride, ...; `lead` marks the one thread that writes
+// the per-row scalars.
+template <class Reduce>
+__device__ __forceinline__ void loss_row(const TrainParams& p, int b, const float* row, float* Frow, int t0, int stride,
+                                         bool lead, Reduce red) {
+    const int N = p.N;
     const float fp = p.w.fpos[b];
     const bool l2 = p.kind == KIND_L2 || p.kind == KIND_TH_L2;
     const float ls = p.loss_scale;
+    float gsum = 0.f;
     if (p.loss == KGE_LOSS_LOGSIGMOID) {
         const float a = p.adv_temp, gamma = p.gamma;
-        float m = 0.f, z = (float)p.N;
+        float m = 0.f, z = (float)N;
         if (a > 0.f) {
             float lm = -INFINITY;
-            for (int n = tid; n < p.N; n += LOSS_THREADS) lm = fmaxf(lm, a * Frow[n]);
-            m = block_max(lm, sm);
+            for (int n = t0; n < N; n += stride) lm = fmaxf(lm, a * row[n]);
+            m = red.max(lm);
             float lz = 0.f;
-            for (int n = tid; n < p.N; n += LOSS_THREADS) lz += expf(a * Frow[n] - m);
-            z = block_sum(lz, sm);
+            for (int n = t0; n < N; n += stride) lz += expf(a * row[n] - m);
+            z = red.sum(lz);
         }
+        const float invz = 1.f / z;
         float lacc = 0.f;
-        for (int n = tid; n < p.N; n += LOSS_THREADS) {
-            const float f = Frow[n];
-            const float w = a > 0.f ? expf(a * f - m) / z : 1.f / z;
-            lacc += w * softplusf(gamma + f);
-            float g = ls * w * sigmoidf(gamma + f);
+        for (int n = t0; n < N; n += stride) {
+            const float f = row[n];
+            const float w = a > 0.f ? expf(a * f - m) * invz : invz;
+            float sp, sg;
+            softplus_sigmoid(gamma + f, sp, sg);
+            lacc += w * sp;
+            float g = ls * w * sg;
             if (l2) g = f < 0.f ? g / -f : 0.f;
             Frow[n] = g;
+            gsum += g;
         }
-        const float lsum = block_sum(lacc, sm);
-        if (tid == 0) {
-            p.w.Lrow[b] = softplusf(-(gamma + fp)) + lsum;
-            p.w.gpos[b] = -ls * sigmoidf(-(gamma + fp));
+        const float lsum = red.sum(lacc);
+        if (lead) {
+            float sp, sg;
+            softplus_sigmoid(-(gamma + fp), sp, sg);
+            p.w.Lrow[b] = sp + lsum;
+            p.w.gpos[b] = -ls * sg;
         }
     } else {
         const float c = p.ce_c;
         float lm = -INFINITY;
-        for (int n = tid; n < p.N; n += LOSS_THREADS) lm = fmaxf(lm, Frow[n] + c);
-        const float m = fmaxf(block_max(lm, sm), fp);
+        for (int n = t0; n < N; n += stride) lm = fmaxf(lm, row[n] + c);
+        const float m = fmaxf(red.max(lm), fp);
         float lz = 0.f;
-        for (int n = tid; n < p.N; n += LOSS_THREADS) lz += expf(Frow[n] + c - m);
+        for (int n = t0; n < N; n += stride) lz += expf(row[n] + c - m);
         const float epos = expf(fp - m);
-        const float z = block_sum(lz, sm) + epos;
-        for (int n = tid; n < p.N; n += LOSS_THREADS) {
-            const float f = Frow[n];
-            float g = ls * expf(f + c - m) / z;
+        const float z = red.sum(lz) + epos;
+        const float invz = 1.f / z;
+        for (int n = t0; n < N; n += stride) {
+            const float f = row[n];
+            float g = ls * expf(f + c - m) * invz;
             if (l2) g = f < 0.f ? g / -f : 0.f;
             Frow[n] = g;
+            gsum += g;
         }
-        if (tid == 0) {
+        if (lead) {
             p.w.Lrow[b] = -fp + (m + logf(z));
-            p.w.gpos[b] = ls * (epos / z - 1.f);
+            p.w.gpos[b] = ls * (epos * invz - 1.f);
         }
     }
+    gsum = red.sum(gsum);
+    if (lead) p.w.Grow[b] = gsum;
+}
+
+__device__ __forceinline__ void stage_row(float* dst, const float* src, int N, int t0, int stride) {
+    if ((N & 3) == 0) {
+        for (int n = t0; n < (N >> 2); n += stride) reinterpret_cast<float4*>(dst)[n] = reinterpret_cast<const float4*>(src)[n];
+    } else {
+        for (int n = t0; n < N; n += stride) dst[n] = src[n];
+    }
+}
+
+// One CTA per positive: long rows.
+__global__ void __launch_bounds__(LOSS_THREADS) loss_kernel(TrainParams p) {
+    extern __shared__ __align__(16) float rowbuf[];
+    __shared__ float sm[LOSS_THREADS / 32];
+    const int b = blockIdx.x, tid = threadIdx.x;
+    float* Frow = p.w.F + (int64_t)b * p.N;
+    const float* row = Frow;
+    if (p.N <= LOSS_SMEM_FLOATS) {
+        stage_row(rowbuf, Frow, p.N, tid, LOSS_THREADS);
+        __syncthreads();
+        row = rowbuf;
+    }
+    loss_row(p, b, row, Frow, tid, LOSS_THREADS, tid == 0, BlockReduce{sm});
+}
+
+// One warp per positive: rows of up to LOSS_WARP_MAX_N scores (N % 4 == 0), no CTA-wide barriers.
+constexpr int LOSS_WARP_MAX_N = 2048;
+__global__ void __launch_bounds__(LOSS_THREADS) loss_warp_kernel(TrainParams p) {
+    extern __shared__ __align__(16) float rowbuf[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.x * (LOSS_THREADS / 32) + warp;
+    if (b >= p.B) return;
+    float* Frow = p.w.F + (int64_t)b * p.N;
+    float* row = rowbuf + (size_t)warp * p.N;
+    stage_row(row, Frow, p.N, lane, 32);
+    __syncwarp();
+    loss_row(p, b, row, Frow, lane, 32, lane == 0, WarpReduce{});
 }
 
 // ------------------------------------------------------------------------------------------
@@ -372,6 +544,8 @@ struct AccArgs {
     const float *G, *U, *Cc;    // [B, N]
     int own_rows, oth_rows, N, d4, split;
     float *out, *out2;          // [split, own_rows, d]; out2: TransH normal gradient (OWNER_Q)
+    float *csum;                // [split, own_rows] weight sums per owner row (TransE p = 1, owner = negatives)
+    int32_t* status;
 };
 
 constexpr int ACC_ROWS = 32, ACC_CC = 32, ACC_LDW = 36;
@@ -499,23 +673,198 @@ __global__ void __launch_bounds__(256) accum_kernel(AccArgs a) {
 }
 
 // ------------------------------------------------------------------------------------------
-// chain: one warp per row.  Warps [0, B): add the column splits of dQ (and of the TransH
+// accum, kinds that are a function of (q, t) alone.  Same ownership as above (32 owner rows
+// per CTA, 4 per warp, one column split per blockIdx.y), but the rows of the other side arrive
+// 32 at a time by one asynchronous bulk copy into a double buffer, and the 32 x 32 weight tile
+// of the next chunk is prefetched through registers while the current chunk is consumed.
+//
+// TransE p = 1: the term is w * sign(q - t).  Writing sign = 2 [q > t] - 1 (the value at an
+// exact tie is a free choice of sub-gradient of |x| at 0; this kernel takes -1, the positive
+// pair in the chain kernel takes 0), the sum becomes 2 P - (sum of the weights) with
+// P = sum of w over the pairs with q > t: one compare and one predicated add per element.
+// The kernel accumulates P; the weight sums come from the loss kernel (rows) and from this
+// kernel's own pass over the weight tiles (columns, OWNER_Q = false).
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void add_if_gt(float& acc, float a, float b, float w) {
+    asm("{\n .reg .pred p;\n setp.gt.f32 p, %1, %2;\n @p add.f32 %0, %0, %3;\n}\n" : "+f"(acc) : "f"(a), "f"(b), "f"(w));
+}
+
+template <int KIND, bool OWNER_Q>
+__device__ __forceinline__ void acc_update2(float4& acc, float4 own, float4 oth, float w) {
+    if (KIND == KIND_L1) {
+        if (OWNER_Q) {   // own = q, oth = t
+            add_if_gt(acc.x, own.x, oth.x, w); add_if_gt(acc.y, own.y, oth.y, w);
+            add_if_gt(acc.z, own.z, oth.z, w); add_if_gt(acc.w, own.w, oth.w, w);
+        } else {         // own = t, oth = q
+            add_if_gt(acc.x, oth.x, own.x, w); add_if_gt(acc.y, oth.y, own.y, w);
+            add_if_gt(acc.z, oth.z, own.z, w); add_if_gt(acc.w, oth.w, own.w, w);
+        }
+    } else {
+        acc_update<KIND>(acc, own, oth, w);
+    }
+}
+
+inline size_t accum_tma_smem(int d4) {
+    return (size_t)2 * ACC_CC * d4 * 16 + (size_t)2 * ACC_CC * ACC_LDW * 4 + 8 * 32 * 4 + 2 * sizeof(uint64_t);
+}
+
+template <int KIND, int NCH, bool OWNER_Q>
+__global__ void __launch_bounds__(256) accum_tma_kernel(AccArgs a) {
+    extern __shared__ __align__(128) unsigned char smraw[];
+    const int d4 = a.d4;
+    float4* Bs = reinterpret_cast<float4*>(smraw);                                  // [2][32][d4]
+    float* Gs = reinterpret_cast<float*>(Bs + 2 * ACC_CC * d4);                     // [2][32][36], [c][r]
+    float* Csum = Gs + 2 * ACC_CC * ACC_LDW;                                        // [8][32]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(Csum + 8 * 32);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int r0 = blockIdx.x * ACC_ROWS;
+    const int per = ((a.oth_rows + a.split - 1) / a.split + ACC_CC - 1) / ACC_CC * ACC_CC;
+    const int c_begin = blockIdx.y * per;
+    const int c_end = min(a.oth_rows, c_begin + per);
+    const int nchunk = c_end > c_begin ? (c_end - c_begin + ACC_CC - 1) / ACC_CC : 0;
+
+    if (tid == 0) { mbar_init(&bars[0], 1); mbar_init(&bars[1], 1); mbar_init_fence(); }
+    __syncthreads();
+
+    auto issue_rows = [&](int chunk, int buf) {      // thread 0 only
+        const int c0 = c_begin + chunk * ACC_CC;
+        const uint32_t bytes = (uint32_t)min(ACC_CC, c_end - c0) * (uint32_t)d4 * 16u;
+        mbar_arrive_expect_tx(&bars[buf], bytes);
+        bulk_g2s(Bs + (size_t)buf * ACC_CC * d4, reinterpret_cast<const float4*>(a.oth) + (int64_t)c0 * d4, bytes, &bars[buf]);
+    };
+    float greg[4];
+    auto load_weights = [&](int chunk) {
+        const int c0 = c_begin + chunk * ACC_CC;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int idx = tid + 256 * e;
+            int rr, cc; int64_t g;
+            if (OWNER_Q) { cc = idx & 31; rr = idx >> 5; g = (int64_t)(r0 + rr) * a.N + (c0 + cc); }
+            else         { rr = idx & 31; cc = idx >> 5; g = (int64_t)(c0 + cc) * a.N + (r0 + rr); }
+            greg[e] = ((r0 + rr) < a.own_rows && (c0 + cc) < c_end) ? a.G[g] : 0.f;
+        }
+    };
+    auto store_weights = [&](int buf) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int idx = tid + 256 * e;
+            const int rr = OWNER_Q ? idx >> 5 : idx & 31, cc = OWNER_Q ? idx & 31 : idx >> 5;
+            Gs[(buf * ACC_CC + cc) * ACC_LDW + rr] = greg[e];
+        }
+    };
+
+    float4 A[4][NCH], acc[4][NCH];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < NCH; ++j) {
+            const int r = r0 + warp * 4 + i, c = lane + 32 * j;
+            A[i][j] = (r < a.own_rows && c < d4) ? reinterpret_cast<const float4*>(a.own)[(int64_t)r * d4 + c] : f4zero();
+            acc[i][j] = f4zero();
+        }
+    float csum = 0.f;   // KIND_L1, owner = negatives: column (lane) sum of the weights this warp has seen
+
+    if (nchunk > 0) {
+        if (tid == 0) issue_rows(0, 0);
+        load_weights(0);
+        store_weights(0);
+    }
+    __syncthreads();
+    for (int chunk = 0; chunk < nchunk; ++chunk) {
+        const int cur = chunk & 1;
+        const bool more = chunk + 1 < nchunk;
+        if (more) {
+            if (tid == 0) issue_rows(chunk + 1, cur ^ 1);
+            load_weights(chunk + 1);
+        }
+        const bool ok = mbar_wait_bounded(&bars[cur], (uint32_t)(chunk >> 1) & 1u);
+        if (!__syncthreads_and(ok)) {
+            if (tid == 0) set_status(a.status, KGE_ERR_TIMEOUT);
+            (void)mbar_wait_bounded(&bars[cur ^ 1], (uint32_t)((chunk + 1) >> 1) & 1u);
+            return;
+        }
+        const int ccmax = min(ACC_CC, c_end - (c_begin + chunk * ACC_CC));
+        const float4* Bc = Bs + (size_t)cur * ACC_CC * d4;
+        const float* Gc = Gs + cur * ACC_CC * ACC_LDW;
+        if (KIND == KIND_L1 && !OWNER_Q) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { const int cc = warp + 8 * e; if (cc < ccmax) csum += Gc[cc * ACC_LDW + lane]; }
+        }
+#pragma unroll 4
+        for (int cc = 0; cc < ccmax; ++cc) {
+            const float4 g4 = *reinterpret_cast<const float4*>(&Gc[cc * ACC_LDW + warp * 4]);
+            const float gw[4] = {g4.x, g4.y, g4.z, g4.w};
+#pragma unroll
+            for (int j = 0; j < NCH; ++j) {
+                const int c = lane + 32 * j;
+                if (c >= d4) continue;
+                const float4 bv = Bc[cc * d4 + c];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc_update2<KIND, OWNER_Q>(acc[i][j], A[i][j], bv, gw[i]);
+            }
+        }
+        if (more) store_weights(cur ^ 1);
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < NCH; ++j) {
+            const int r = r0 + warp * 4 + i, c = lane + 32 * j;
+            if (r >= a.own_rows || c >= d4) continue;
+            reinterpret_cast<float4*>(a.out)[((int64_t)blockIdx.y * a.own_rows + r) * d4 + c] = acc[i][j];
+        }
+    if (KIND == KIND_L1 && !OWNER_Q) {
+        Csum[warp * 32 + lane] = csum;
+        __syncthreads();
+        if (warp == 0 && r0 + lane < a.own_rows) {
+            float t = 0.f;
+            for (int w = 0; w < 8; ++w) t += Csum[w * 32 + lane];
+            a.csum[(int64_t)blockIdx.y * a.own_rows + r0 + lane] = t;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// chain: one warp per row (plus one CTA for the batch loss).  Warps [0, B): add the column splits of dQ (and of the TransH
 // normal gradient), add the positive pair, apply the chain rule q -> (h, r, w) and write
 // the gradient rows of the head, the positive tail and the relation.  Warps [B, B+N): add
 // the row splits of dT and write the gradient row of the negative tail.
 // ------------------------------------------------------------------------------------------
+template <int kMaxChunks>
 __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
+    if (blockIdx.x == gridDim.x - 1) {   // the extra last CTA adds up the batch loss
+        __shared__ float lsum[8];
+        float v = 0.f;
+        for (int b = threadIdx.x; b < p.B; b += 256) v += p.w.Lrow[b];
+        v = warp_sum(v);
+        if (lane == 0) lsum[threadIdx.x >> 5] = v;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            float t = 0.f;
+            for (int i = 0; i < 8; ++i) t += lsum[i];
+            t *= p.loss_scale;
+            *p.w.loss = t;
+            if (p.loss_out) *p.loss_out = t;
+        }
+        return;
+    }
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (warp >= p.B + p.N) return;
     const int d4 = p.d4;
     float4* gent = reinterpret_cast<float4*>(p.w.grad_ent);
     if (warp >= p.B) {
         const int n = warp - p.B;
         const float4* part = reinterpret_cast<const float4*>(p.w.dTpart);
+        float wsum = 0.f;   // TransE p = 1: the splits hold P, the gradient is 2 P - (column sum of dL/dF)
+        if (p.kind == KIND_L1)
+            for (int sp = 0; sp < p.split_t; ++sp) wsum += p.w.Cpart[(int64_t)sp * p.N + n];
         for (int c = lane; c < d4; c += 32) {
             float4 s = f4zero();
             for (int sp = 0; sp < p.split_t; ++sp) s = f4add(s, part[((int64_t)sp * p.N + n) * d4 + c]);
+            if (p.kind == KIND_L1) s = make_float4(2.f * s.x - wsum, 2.f * s.y - wsum, 2.f * s.z - wsum, 2.f * s.w - wsum);
             gent[(int64_t)(2 * p.B + n) * d4 + c] = s;
         }
         return;
@@ -539,6 +888,10 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
         if (in)
             for (int sp = 0; sp < p.split_q; ++sp)
                 s = f4add(s, reinterpret_cast<const float4*>(p.w.dQpart)[((int64_t)sp * p.B + b) * d4 + c]);
+        if (p.kind == KIND_L1 && in) {   // the splits hold P; dQ = (row sum of dL/dF) - 2 P
+            const float rs = p.w.Grow[b];
+            s = make_float4(rs - 2.f * s.x, rs - 2.f * s.y, rs - 2.f * s.z, rs - 2.f * s.w);
+        }
         dq[i] = s; dt[i] = f4zero();
     }
     float4* gh = gent + (int64_t)b * d4;
@@ -679,9 +1032,40 @@ void launch_block(const TrainParams& p, cudaStream_t s) {
     block_kernel<KIND, MODE><<<grid, 256, 0, s>>>(p);
 }
 
+template <int KIND>
+cudaError_t launch_block_tma(const TrainParams& p, cudaStream_t s) {
+    const size_t smem = block_tma_smem(p.d);
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(block_tma_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)block_tma_smem(kMaxDim));
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    dim3 grid((p.N + TN - 1) / TN, (p.B + TB - 1) / TB);
+    block_tma_kernel<KIND><<<grid, 256, smem, s>>>(p);
+    return cudaSuccess;
+}
+
+template <int KIND, int NCH, bool OWNER_Q>
+cudaError_t launch_accum_tma_inst(const AccArgs& a, cudaStream_t s) {
+    const size_t smem = accum_tma_smem(a.d4);
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(accum_tma_kernel<KIND, NCH, OWNER_Q>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)accum_tma_smem(kMaxDim / 4));
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    dim3 grid((a.own_rows + ACC_ROWS - 1) / ACC_ROWS, a.split);
+    accum_tma_kernel<KIND, NCH, OWNER_Q><<<grid, 256, smem, s>>>(a);
+    return cudaSuccess;
+}
+
 template <int KIND, int NCH, bool OWNER_Q>
 cudaError_t launch_accum_inst(const AccArgs& a, cudaStream_t s) {
     constexpr bool TH = KIND == KIND_TH_L1 || KIND == KIND_TH_L2;
+    if (!TH) return launch_accum_tma_inst<TH ? KIND_L1 : KIND, NCH, OWNER_Q>(a, s);
     size_t smem = (size_t)ACC_CC * a.d4 * 16 * ((TH && !OWNER_Q) ? 2 : 1) + (size_t)ACC_CC * ACC_LDW * 4 * (TH ? 3 : 1);
     static bool configured = false;
     if (!configured) {
@@ -717,7 +1101,7 @@ cudaError_t launch_accum(int kind, const AccArgs& a, cudaStream_t s) {
 }  // namespace
 
 int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* rels, const int32_t* tails,
-                            const int32_t* negs, cudaStream_t s) {
+                            const int32_t* negs, float* loss_out, cudaStream_t s, cudaStream_t side) {
     const kge_config& c = h->cfg;
     TrainParams p;
     p.B = c.batch; p.N = c.num_neg; p.d = c.dim; p.d4 = c.dim / 4; p.kw = h->kw;
@@ -727,26 +1111,48 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     p.ent = h->ent; p.rel = h->rel; p.relw = h->relw;
     p.heads = heads; p.rels = rels; p.tails = tails; p.negs = negs;
     p.split_q = h->split_q; p.split_t = h->split_t;
+    p.loss_out = loss_out;
     p.w = h->ws;
+    const int nch = p.d4 <= 32 ? 1 : (p.d4 <= 64 ? 2 : 4);
 
     const int row_warps = p.B + p.N;
     stage_begin(h, ST_BUILD, s);
-    build_kernel<<<(row_warps * 32 + 255) / 256, 256, 0, s>>>(p);
+    {
+        const int grid = (row_warps * 32 + 255) / 256;
+        if (nch == 1) build_kernel<1><<<grid, 256, 0, s>>>(p);
+        else if (nch == 2) build_kernel<2><<<grid, 256, 0, s>>>(p);
+        else build_kernel<4><<<grid, 256, 0, s>>>(p);
+    }
     stage_end(h, ST_BUILD, s);
     KGE_LAUNCH_CHECK(h);
     stage_begin(h, ST_BLOCK, s);
     switch (p.kind) {
-        case KIND_L1: launch_block<KIND_L1, 0>(p, s); break;
-        case KIND_L2: launch_block<KIND_L2, 0>(p, s); break;
-        case KIND_CL1: launch_block<KIND_CL1, 0>(p, s); break;
-        case KIND_DOT: launch_block<KIND_DOT, 0>(p, s); break;
+        case KIND_L1: KGE_CUDA_CHECK(h, launch_block_tma<KIND_L1>(p, s)); break;
+        case KIND_L2: KGE_CUDA_CHECK(h, launch_block_tma<KIND_L2>(p, s)); break;
+        case KIND_CL1: KGE_CUDA_CHECK(h, launch_block_tma<KIND_CL1>(p, s)); break;
+        case KIND_DOT: KGE_CUDA_CHECK(h, launch_block_tma<KIND_DOT>(p, s)); break;
         case KIND_TH_L1: launch_block<KIND_TH_L1, 0>(p, s); break;
         default: launch_block<KIND_TH_L2, 0>(p, s); break;
     }
     stage_end(h, ST_BLOCK, s);
     KGE_LAUNCH_CHECK(h);
     stage_begin(h, ST_LOSS, s);
-    loss_kernel<<<p.B, LOSS_THREADS, 0, s>>>(p);
+    {
+        static bool configured = false;
+        if (!configured) {
+            KGE_CUDA_CHECK(h, cudaFuncSetAttribute(loss_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   LOSS_SMEM_FLOATS * 4));
+            KGE_CUDA_CHECK(h, cudaFuncSetAttribute(loss_warp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   LOSS_THREADS / 32 * LOSS_WARP_MAX_N * 4));
+            configured = true;
+        }
+    }
+    if (p.N <= LOSS_WARP_MAX_N && (p.N & 3) == 0) {
+        constexpr int rows = LOSS_THREADS / 32;
+        loss_warp_kernel<<<(p.B + rows - 1) / rows, LOSS_THREADS, (size_t)rows * p.N * 4, s>>>(p);
+    } else {
+        loss_kernel<<<p.B, LOSS_THREADS, p.N <= LOSS_SMEM_FLOATS ? (size_t)p.N * 4 : 0, s>>>(p);
+    }
     stage_end(h, ST_LOSS, s);
     KGE_LAUNCH_CHECK(h);
     if (p.kind == KIND_TH_L1 || p.kind == KIND_TH_L2) {
@@ -759,20 +1165,33 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     AccArgs aq;
     aq.own = p.w.Q; aq.oth = p.w.Tneg; aq.what = p.w.What; aq.G = p.w.F; aq.U = p.w.U; aq.Cc = p.w.Cc;
     aq.own_rows = p.B; aq.oth_rows = p.N; aq.N = p.N; aq.d4 = p.d4; aq.split = p.split_q;
-    aq.out = p.w.dQpart; aq.out2 = p.w.dWpart;
-    stage_begin(h, ST_ACCUM_Q, s);
-    KGE_CUDA_CHECK(h, launch_accum<true>(p.kind, aq, s));
-    stage_end(h, ST_ACCUM_Q, s);
+    aq.out = p.w.dQpart; aq.out2 = p.w.dWpart; aq.csum = nullptr; aq.status = p.w.status;
+    // the two accumulations are independent: with a side stream they run concurrently
+    if (side) {
+        KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_loss, s));
+        KGE_CUDA_CHECK(h, cudaStreamWaitEvent(side, h->ev_loss, 0));
+    }
+    cudaStream_t sq = side ? side : s;
+    stage_begin(h, ST_ACCUM_Q, sq);
+    KGE_CUDA_CHECK(h, launch_accum<true>(p.kind, aq, sq));
+    stage_end(h, ST_ACCUM_Q, sq);
     KGE_LAUNCH_CHECK(h);
+    if (side) KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_t, side));
     AccArgs at = aq;
     at.own = p.w.Tneg; at.oth = p.w.Q; at.own_rows = p.N; at.oth_rows = p.B; at.split = p.split_t;
-    at.out = p.w.dTpart; at.out2 = nullptr;
+    at.out = p.w.dTpart; at.out2 = nullptr; at.csum = p.w.Cpart;
     stage_begin(h, ST_ACCUM_T, s);
     KGE_CUDA_CHECK(h, launch_accum<false>(p.kind, at, s));
     stage_end(h, ST_ACCUM_T, s);
     KGE_LAUNCH_CHECK(h);
+    if (side) KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_t, 0));
     stage_begin(h, ST_CHAIN, s);
-    chain_kernel<<<(row_warps * 32 + 255) / 256, 256, 0, s>>>(p);
+    {
+        const int grid = (row_warps * 32 + 255) / 256 + 1;
+        if (nch == 1) chain_kernel<1><<<grid, 256, 0, s>>>(p);
+        else if (nch == 2) chain_kernel<2><<<grid, 256, 0, s>>>(p);
+        else chain_kernel<4><<<grid, 256, 0, s>>>(p);
+    }
     stage_end(h, ST_CHAIN, s);
     KGE_LAUNCH_CHECK(h);
     return KGE_OK;

@@ -1,8 +1,18 @@
 // Deterministic de-duplication of touched rows and the sparse row update.
-//   rank    : stable sort of the id lists by counting, rank(i) = #{j : (id_j, j) < (id_i, i)}
-//   segment : distinct ids, segment offsets (single-CTA scan), batch loss reduction
-//   update  : one warp per distinct row: sum the segment's gradient rows in ascending source
-//             position, then SGD / Adam / row-wise Adagrad on the table row
+//   tile_sort : every 1024 ids of a list, tagged with their source position, sorted in shared memory
+//   rank      : global stable rank of each id = sum over tiles of (keys below it); scatter to
+//               the permutation and the sorted id list
+//   segment   : distinct ids, segment offsets, segment index of every sorted position
+//               (single-CTA scan), batch loss reduction
+//   piece sum : one warp per sorted position; a segment of at most 16 rows is summed in
+//               ascending source position by the warp at its first position and the row is
+//               updated at once (SGD / Adam / row-wise Adagrad); a longer segment is cut
+//               into pieces of 16 rows, each summed by its own warp into a partial row
+//   piece join: the first position of a long segment adds its pieces in ascending order and
+//               updates the row
+// The summation order of a segment is therefore fixed by the batch alone: results are
+// bit-reproducible, and a row that occurs hundreds of times in a batch does not serialise
+// behind a single warp.
 #include <cmath>
 
 #include "kge_common.cuh"
@@ -11,13 +21,20 @@ namespace kge {
 
 namespace {
 
+constexpr int SORT_TILE = 1024;      // keys per shared-memory sort
+constexpr int SORT_THREADS = 512;
+constexpr int RANK_THREADS = 256;
+constexpr int SEG_THREADS = 1024;
+constexpr int PIECE = 16;            // gradient rows summed by one warp in one go
+
 struct IdList {
     const int32_t *a, *b, *c;   // the list is the concatenation a[0..na) | b[0..nb) | c[0..nc)
     int na, nb, nc;
     int64_t rows;               // table rows (ids outside [0, rows) are reported and read as 0)
-    int32_t *perm, *sorted, *uniq, *seg;
+    int32_t *perm, *sorted, *uniq, *seg, *seg_of;
+    uint64_t* tkeys;            // [tiles * SORT_TILE] tile-sorted (id << 32 | position), padded with ~0
     int32_t* count;             // number of distinct ids
-    __device__ __forceinline__ int n() const { return na + nb + nc; }
+    __host__ __device__ __forceinline__ int n() const { return na + nb + nc; }
     __device__ __forceinline__ int32_t raw(int i) const {
         return i < na ? a[i] : (i < na + nb ? b[i - na] : c[i - na - nb]);
     }
@@ -25,257 +42,330 @@ struct IdList {
 
 struct DedupParams {
     IdList ent, rel;
-    int ent_blocks;             // rank kernel: blocks [0, ent_blocks) serve the entity list
+    int ent_tiles;              // sort / rank kernels: tiles [0, ent_tiles) serve the entity list
     int32_t* status;
-    const float* Lrow; int B; float loss_scale; float* loss; float* loss_out;
 };
 
-constexpr int RANK_THREADS = 256;
-
-__global__ void __launch_bounds__(RANK_THREADS) rank_kernel(DedupParams p) {
-    __shared__ int32_t keys[RANK_THREADS];
-    const bool is_ent = (int)blockIdx.x < p.ent_blocks;
+__global__ void __launch_bounds__(SORT_THREADS) tile_sort_kernel(DedupParams p) {
+    __shared__ uint64_t k[SORT_TILE];
+    const bool is_ent = (int)blockIdx.x < p.ent_tiles;
     const IdList& L = is_ent ? p.ent : p.rel;
-    const int n = L.n();
-    const int i = (is_ent ? blockIdx.x : blockIdx.x - p.ent_blocks) * RANK_THREADS + threadIdx.x;
-    int32_t mine = 0;
-    if (i < n) mine = (int32_t)checked_id(L.raw(i), L.rows, p.status);
-    int rank = 0;
-    for (int j0 = 0; j0 < n; j0 += RANK_THREADS) {
-        const int j = j0 + threadIdx.x;
-        __syncthreads();
-        if (j < n) {
-            const int32_t v = L.raw(j);
-            keys[threadIdx.x] = (v < 0 || (int64_t)v >= L.rows) ? 0 : v;
-        }
-        __syncthreads();
-        const int m = min(RANK_THREADS, n - j0);
-        if (i < n) {
-            // positions before i count when id <= mine, positions after i when id < mine
-            for (int jj = 0; jj < m; ++jj) {
-                const int32_t kj = keys[jj];
-                rank += (kj < mine) || (kj == mine && (j0 + jj) < i);
-            }
+    const int tile = is_ent ? blockIdx.x : blockIdx.x - p.ent_tiles;
+    const int n = L.n(), tid = threadIdx.x;
+    for (int j = tid; j < SORT_TILE; j += SORT_THREADS) {
+        const int i = tile * SORT_TILE + j;
+        uint64_t key = ~0ull;
+        if (i < n) key = ((uint64_t)(uint32_t)checked_id(L.raw(i), L.rows, p.status) << 32) | (uint32_t)i;
+        k[j] = key;
+    }
+    __syncthreads();
+    for (int size = 2; size <= SORT_TILE; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            const int lo = 2 * tid - (tid & (stride - 1)), hi = lo + stride;
+            const bool up = (lo & size) == 0;
+            const uint64_t x = k[lo], y = k[hi];
+            if ((x > y) == up) { k[lo] = y; k[hi] = x; }
+            __syncthreads();
         }
     }
-    if (i < n) { L.perm[rank] = i; L.sorted[rank] = mine; }
+    for (int j = tid; j < SORT_TILE; j += SORT_THREADS) L.tkeys[(int64_t)tile * SORT_TILE + j] = k[j];
 }
 
-constexpr int SEG_THREADS = 1024;
+// Keys are distinct (the position is part of the key), so "number of keys below mine" summed
+// over all tiles is the position of the key in the stable sort by id.
+__global__ void __launch_bounds__(RANK_THREADS) rank_kernel(DedupParams p) {
+    __shared__ uint64_t sk[SORT_TILE];
+    constexpr int PER_TILE = SORT_TILE / RANK_THREADS;
+    int blk = blockIdx.x;
+    const bool is_ent = blk < p.ent_tiles * PER_TILE;
+    const IdList& L = is_ent ? p.ent : p.rel;
+    if (!is_ent) blk -= p.ent_tiles * PER_TILE;
+    const int tile = blk / PER_TILE, j = (blk % PER_TILE) * RANK_THREADS + threadIdx.x;
+    const int n = L.n(), tiles = (n + SORT_TILE - 1) / SORT_TILE;
+    const uint64_t key = L.tkeys[(int64_t)tile * SORT_TILE + j];
+    int rank = j;
+    for (int t = 0; t < tiles; ++t) {
+        if (t == tile) continue;
+        __syncthreads();
+        for (int x = threadIdx.x; x < SORT_TILE; x += RANK_THREADS) sk[x] = L.tkeys[(int64_t)t * SORT_TILE + x];
+        __syncthreads();
+        int lo = 0;
+#pragma unroll
+        for (int step = SORT_TILE >> 1; step >= 1; step >>= 1) lo += (sk[lo + step - 1] < key) ? step : 0;
+        lo += (sk[lo] < key) ? 1 : 0;
+        rank += lo;
+    }
+    if (key != ~0ull) { L.perm[rank] = (int32_t)(uint32_t)key; L.sorted[rank] = (int32_t)(key >> 32); }
+}
 
-// blockIdx.x = 0: entity list, 1: relation list, 2: batch loss.
+// blockIdx.x = 0: entity list, 1: relation list.
 __global__ void __launch_bounds__(SEG_THREADS) segment_kernel(DedupParams p) {
     __shared__ int32_t warp_tot[SEG_THREADS / 32];
-    __shared__ int32_t carry;
-    __shared__ float lsum[SEG_THREADS / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (blockIdx.x == 2) {
-        float v = 0.f;
-        for (int b = tid; b < p.B; b += SEG_THREADS) v += p.Lrow[b];
-        v = warp_sum(v);
-        if (lane == 0) lsum[warp] = v;
-        __syncthreads();
-        if (tid == 0) {
-            float t = 0.f;
-            for (int i = 0; i < SEG_THREADS / 32; ++i) t += lsum[i];
-            t *= p.loss_scale;
-            *p.loss = t;
-            if (p.loss_out) *p.loss_out = t;
-        }
-        return;
-    }
     const IdList& L = blockIdx.x == 0 ? p.ent : p.rel;
     const int n = L.n();
-    if (tid == 0) carry = 0;
-    __syncthreads();
-    for (int base = 0; base < n; base += SEG_THREADS) {
-        const int r = base + tid;
-        const int32_t id = r < n ? L.sorted[r] : 0;
-        const int flag = r < n && (r == 0 || L.sorted[r - 1] != id);
-        int incl = flag;   // inclusive scan of the head flags
+    const int per = (n + SEG_THREADS - 1) / SEG_THREADS;
+    const int r0 = min(n, tid * per), r1 = min(n, r0 + per);
+    int cnt = 0;
+    int32_t prev = r0 > 0 && r0 < n ? L.sorted[r0 - 1] : -1;
+    for (int r = r0; r < r1; ++r) { const int32_t id = L.sorted[r]; cnt += id != prev; prev = id; }
+    int incl = cnt;   // inclusive scan of the per-thread segment-head counts
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        if (lane == 31) warp_tot[warp] = incl;
-        __syncthreads();
-        int before = carry;
-        for (int w = 0; w < warp; ++w) before += warp_tot[w];
-        if (flag) { const int u = before + incl - 1; L.uniq[u] = id; L.seg[u] = r; }
-        __syncthreads();
-        if (tid == SEG_THREADS - 1) carry = before + incl;
-        __syncthreads();
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
     }
-    if (tid == 0) { L.seg[carry] = n; *L.count = carry; }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    int before = 0, total = 0;
+    for (int w = 0; w < SEG_THREADS / 32; ++w) { if (w < warp) before += warp_tot[w]; total += warp_tot[w]; }
+    int u = before + incl - cnt;
+    prev = r0 > 0 && r0 < n ? L.sorted[r0 - 1] : -1;
+    for (int r = r0; r < r1; ++r) {
+        const int32_t id = L.sorted[r];
+        if (id != prev) { L.uniq[u] = id; L.seg[u] = r; ++u; }
+        L.seg_of[r] = u - 1;
+        prev = id;
+    }
+    if (tid == 0) { L.seg[total] = n; *L.count = total; }
 }
 
 struct UpdateJob {
     float* table; float* state;        // [rows, width], optimiser state
     const float* grads;                // [n, width] gradient rows by source position
-    const int32_t *uniq, *seg, *perm;
-    const int32_t* count;              // distinct rows (device scalar)
-    int width, max_rows;               // max_rows = list length (upper bound of *count)
+    float* part;                       // [n, width] partial sums of long segments, row = first sorted position of the piece
+    const int32_t *uniq, *seg, *perm, *sorted, *seg_of;
+    int width, n;                      // n = list length
 };
 
 struct UpdateParams {
     UpdateJob job[3];
     int njobs;
-    int warp_begin[4];                 // job j serves warps [warp_begin[j], warp_begin[j+1])
+    int warp_begin[4];                 // job j serves warps [warp_begin[j], warp_begin[j+1]): one per sorted position
     int opt;
     float lr, beta1, beta2, eps, corr1, corr2;   // corr = 1 - beta^t
 };
 
-__global__ void __launch_bounds__(256) update_kernel(UpdateParams p) {
-    const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-    int j = 0;
-    while (j + 1 < p.njobs && gw >= p.warp_begin[j + 1]) ++j;
-    if (gw >= p.warp_begin[p.njobs]) return;
-    const UpdateJob& J = p.job[j];
-    const int u = gw - p.warp_begin[j];
-    if (u >= *J.count) return;
-    const int w4 = J.width >> 2;       // width % 4 == 0 except RotatE relation rows (width % 2 == 0)
-    const int64_t row = J.uniq[u];
-    const int s0 = J.seg[u], s1 = J.seg[u + 1];
-    if ((J.width & 3) == 0) {
-        constexpr int MAXC = kMaxDim / 128;
-        float4 g[MAXC];
+template <typename V> struct VecOps;
+template <> struct VecOps<float> {
+    static constexpr int LEN = 1;
+    static __device__ __forceinline__ float zero() { return 0.f; }
+    static __device__ __forceinline__ void add(float& a, float b) { a += b; }
+};
+template <> struct VecOps<float4> {
+    static constexpr int LEN = 4;
+    static __device__ __forceinline__ float4 zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+    static __device__ __forceinline__ void add(float4& a, float4 b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
+};
+
+// One optimiser step on table row `row` with the summed gradient g (lane l holds elements
+// l, l + 32, ... of the row in units of V).
+template <typename V, int NCH>
+__device__ __forceinline__ void apply_row(const UpdateJob& J, const UpdateParams& p, int64_t row, V (&g)[NCH], int lane) {
+    constexpr int LEN = VecOps<V>::LEN;
+    const int wv = J.width / LEN;
+    V* prow = reinterpret_cast<V*>(J.table) + row * wv;
+    if (p.opt == KGE_OPT_SGD) {
 #pragma unroll
-        for (int i = 0; i < MAXC; ++i) g[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s = s0; s < s1; ++s) {
-            const float4* gr = reinterpret_cast<const float4*>(J.grads) + (int64_t)J.perm[s] * w4;
+        for (int i = 0; i < NCH; ++i) {
+            const int c = lane + 32 * i;
+            if (c < wv) {
+                V v = prow[c];
+                float* vv = reinterpret_cast<float*>(&v); const float* gg = reinterpret_cast<const float*>(&g[i]);
 #pragma unroll
-            for (int i = 0; i < MAXC; ++i) {
-                const int c = lane + 32 * i;
-                if (c < w4) { const float4 v = gr[c]; g[i].x += v.x; g[i].y += v.y; g[i].z += v.z; g[i].w += v.w; }
+                for (int e = 0; e < LEN; ++e) vv[e] -= p.lr * gg[e];
+                prow[c] = v;
             }
         }
-        float4* prow = reinterpret_cast<float4*>(J.table) + row * w4;
-        if (p.opt == KGE_OPT_SGD) {
+    } else if (p.opt == KGE_OPT_ADAM) {
+        V* mrow = reinterpret_cast<V*>(J.state) + row * 2 * wv;
+        V* vrow = mrow + wv;
 #pragma unroll
-            for (int i = 0; i < MAXC; ++i) {
-                const int c = lane + 32 * i;
-                if (c < w4) {
-                    float4 v = prow[c];
-                    v.x -= p.lr * g[i].x; v.y -= p.lr * g[i].y; v.z -= p.lr * g[i].z; v.w -= p.lr * g[i].w;
-                    prow[c] = v;
+        for (int i = 0; i < NCH; ++i) {
+            const int c = lane + 32 * i;
+            if (c < wv) {
+                V m = mrow[c], v = vrow[c], x = prow[c];
+                float* mm = reinterpret_cast<float*>(&m); float* vv = reinterpret_cast<float*>(&v);
+                float* xx = reinterpret_cast<float*>(&x); const float* gg = reinterpret_cast<const float*>(&g[i]);
+#pragma unroll
+                for (int e = 0; e < LEN; ++e) {
+                    mm[e] = p.beta1 * mm[e] + (1.f - p.beta1) * gg[e];
+                    vv[e] = p.beta2 * vv[e] + (1.f - p.beta2) * gg[e] * gg[e];
+                    xx[e] -= p.lr * (mm[e] / p.corr1) / (sqrtf(vv[e] / p.corr2) + p.eps);
                 }
-            }
-        } else if (p.opt == KGE_OPT_ADAM) {
-            float4* mrow = reinterpret_cast<float4*>(J.state) + row * 2 * w4;
-            float4* vrow = mrow + w4;
-#pragma unroll
-            for (int i = 0; i < MAXC; ++i) {
-                const int c = lane + 32 * i;
-                if (c < w4) {
-                    float4 m = mrow[c], v = vrow[c], x = prow[c];
-                    const float gg[4] = {g[i].x, g[i].y, g[i].z, g[i].w};
-                    float* mm = &m.x; float* vv = &v.x; float* xx = &x.x;
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        mm[e] = p.beta1 * mm[e] + (1.f - p.beta1) * gg[e];
-                        vv[e] = p.beta2 * vv[e] + (1.f - p.beta2) * gg[e] * gg[e];
-                        xx[e] -= p.lr * (mm[e] / p.corr1) / (sqrtf(vv[e] / p.corr2) + p.eps);
-                    }
-                    mrow[c] = m; vrow[c] = v; prow[c] = x;
-                }
-            }
-        } else {
-            float ss = 0.f;
-#pragma unroll
-            for (int i = 0; i < MAXC; ++i) ss += g[i].x * g[i].x + g[i].y * g[i].y + g[i].z * g[i].z + g[i].w * g[i].w;
-            ss = warp_sum(ss) / (float)J.width;
-            const float acc = J.state[row] + ss;
-            __syncwarp();
-            if (lane == 0) J.state[row] = acc;
-            const float step = p.lr / (sqrtf(acc) + p.eps);
-#pragma unroll
-            for (int i = 0; i < MAXC; ++i) {
-                const int c = lane + 32 * i;
-                if (c < w4) {
-                    float4 v = prow[c];
-                    v.x -= step * g[i].x; v.y -= step * g[i].y; v.z -= step * g[i].z; v.w -= step * g[i].w;
-                    prow[c] = v;
-                }
+                mrow[c] = m; vrow[c] = v; prow[c] = x;
             }
         }
     } else {
-        // narrow rows whose width is only even (RotatE phases with d % 8 != 0): scalar lanes
-        constexpr int MAXS = kMaxDim / 2 / 32;
-        float g[MAXS];
-#pragma unroll
-        for (int i = 0; i < MAXS; ++i) g[i] = 0.f;
-        for (int s = s0; s < s1; ++s) {
-            const float* gr = J.grads + (int64_t)J.perm[s] * J.width;
-#pragma unroll
-            for (int i = 0; i < MAXS; ++i) { const int c = lane + 32 * i; if (c < J.width) g[i] += gr[c]; }
-        }
-        float* prow = J.table + row * J.width;
         float ss = 0.f;
 #pragma unroll
-        for (int i = 0; i < MAXS; ++i) ss += g[i] * g[i];
-        ss = warp_sum(ss) / (float)J.width;
-        float step = p.lr;
-        if (p.opt == KGE_OPT_ROWWISE_ADAGRAD) {
-            const float acc = J.state[row] + ss;
-            __syncwarp();
-            if (lane == 0) J.state[row] = acc;
-            step = p.lr / (sqrtf(acc) + p.eps);
-        }
+        for (int i = 0; i < NCH; ++i) {
+            const float* gg = reinterpret_cast<const float*>(&g[i]);
 #pragma unroll
-        for (int i = 0; i < MAXS; ++i) {
+            for (int e = 0; e < LEN; ++e) ss += gg[e] * gg[e];   // lanes beyond the row hold zeros
+        }
+        ss = warp_sum(ss) / (float)J.width;
+        const float acc = J.state[row] + ss;
+        __syncwarp();
+        if (lane == 0) J.state[row] = acc;
+        const float step = p.lr / (sqrtf(acc) + p.eps);
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
             const int c = lane + 32 * i;
-            if (c >= J.width) continue;
-            if (p.opt == KGE_OPT_ADAM) {
-                float* m = J.state + row * 2 * J.width + c; float* v = m + J.width;
-                const float mm = p.beta1 * *m + (1.f - p.beta1) * g[i];
-                const float vv = p.beta2 * *v + (1.f - p.beta2) * g[i] * g[i];
-                *m = mm; *v = vv;
-                prow[c] -= p.lr * (mm / p.corr1) / (sqrtf(vv / p.corr2) + p.eps);
-            } else {
-                prow[c] -= step * g[i];
+            if (c < wv) {
+                V v = prow[c];
+                float* vv = reinterpret_cast<float*>(&v); const float* gg = reinterpret_cast<const float*>(&g[i]);
+#pragma unroll
+                for (int e = 0; e < LEN; ++e) vv[e] -= step * gg[e];
+                prow[c] = v;
             }
         }
     }
 }
 
+// g += rows[idx[0]], rows[idx[1]], ... in that order, four loads in flight at a time.
+template <typename V, int NCH, typename IndexOf>
+__device__ __forceinline__ void ordered_sum(const V* rows, int wv, int count, IndexOf index_of, V (&g)[NCH], int lane) {
+    for (int s = 0; s < count; s += 4) {
+        V v[4][NCH];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const V* src = rows + (s + r < count ? index_of(s + r) : 0) * wv;
+#pragma unroll
+            for (int i = 0; i < NCH; ++i) {
+                const int c = lane + 32 * i;
+                v[r][i] = (s + r < count && c < wv) ? src[c] : VecOps<V>::zero();
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int i = 0; i < NCH; ++i) VecOps<V>::add(g[i], v[r][i]);
+    }
+}
+
+// One warp per sorted position.  A warp whose position opens a segment of at most PIECE rows
+// sums it and updates the row.  In a longer segment every PIECE-th position sums its piece
+// into the partial buffer (row index = the piece's first sorted position).
+template <typename V, int NCH>
+__device__ __forceinline__ void piece_sum(const UpdateJob& J, const UpdateParams& p, int r, int lane) {
+    const int wv = J.width / VecOps<V>::LEN;
+    const int u = J.seg_of[r];
+    const int s0 = J.seg[u], s1 = J.seg[u + 1];
+    const int len = s1 - s0;
+    const bool whole = len <= PIECE;
+    if (whole ? r != s0 : ((r - s0) % PIECE) != 0) return;
+    const int count = whole ? len : min(PIECE, s1 - r);
+    const int32_t src = lane < count ? J.perm[r + lane] : 0;
+    V g[NCH];
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) g[i] = VecOps<V>::zero();
+    ordered_sum<V, NCH>(reinterpret_cast<const V*>(J.grads), wv, count,
+                        [&](int s) { return (int64_t)__shfl_sync(0xffffffffu, src, s); }, g, lane);
+    if (whole) {
+        apply_row<V, NCH>(J, p, J.uniq[u], g, lane);
+    } else {
+        V* dst = reinterpret_cast<V*>(J.part) + (int64_t)r * wv;
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) { const int c = lane + 32 * i; if (c < wv) dst[c] = g[i]; }
+    }
+}
+
+// One warp per sorted position; only the first position of a segment longer than PIECE rows
+// works: it adds the segment's pieces in ascending order and updates the row.
+template <typename V, int NCH>
+__device__ __forceinline__ void piece_join(const UpdateJob& J, const UpdateParams& p, int r, int lane) {
+    const int wv = J.width / VecOps<V>::LEN;
+    if (r > 0 && J.sorted[r - 1] == J.sorted[r]) return;
+    const int u = J.seg_of[r];
+    const int s1 = J.seg[u + 1];
+    if (s1 - r <= PIECE) return;
+    V g[NCH];
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) g[i] = VecOps<V>::zero();
+    ordered_sum<V, NCH>(reinterpret_cast<const V*>(J.part), wv, (s1 - r + PIECE - 1) / PIECE,
+                        [&](int s) { return (int64_t)r + (int64_t)s * PIECE; }, g, lane);
+    apply_row<V, NCH>(J, p, J.uniq[u], g, lane);
+}
+
+template <bool JOIN, typename V, int NCH>
+__device__ __forceinline__ void piece_do(const UpdateJob& J, const UpdateParams& p, int r, int lane) {
+    if (JOIN) piece_join<V, NCH>(J, p, r, lane); else piece_sum<V, NCH>(J, p, r, lane);
+}
+
+template <bool JOIN>
+__global__ void __launch_bounds__(256) piece_kernel(UpdateParams p) {
+    const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (gw >= p.warp_begin[p.njobs]) return;
+    int j = 0;
+    while (j + 1 < p.njobs && gw >= p.warp_begin[j + 1]) ++j;
+    const UpdateJob& J = p.job[j];
+    const int r = gw - p.warp_begin[j];
+    if ((J.width & 3) == 0) {
+        const int wv = J.width >> 2;
+        if (wv <= 32) piece_do<JOIN, float4, 1>(J, p, r, lane);
+        else if (wv <= 64) piece_do<JOIN, float4, 2>(J, p, r, lane);
+        else piece_do<JOIN, float4, 4>(J, p, r, lane);
+    } else {
+        // narrow rows whose width is only even (RotatE phases with d % 8 != 0): scalar lanes
+        if (J.width <= 64) piece_do<JOIN, float, 2>(J, p, r, lane);
+        else piece_do<JOIN, float, kMaxDim / 2 / 32>(J, p, r, lane);
+    }
+}
+
 }  // namespace
 
-int launch_dedup_update(kge_handle* h, uint64_t step, float lr, const int32_t* heads, const int32_t* rels,
-                        const int32_t* tails, const int32_t* negs, float* loss_out, cudaStream_t s) {
+int dedup_tiles(int n) { return (n + SORT_TILE - 1) / SORT_TILE; }
+
+int launch_dedup(kge_handle* h, const int32_t* heads, const int32_t* rels, const int32_t* tails,
+                 const int32_t* negs, cudaStream_t s) {
     const kge_config& c = h->cfg;
     Workspace& w = h->ws;
     const int B = c.batch, N = c.num_neg;
     DedupParams dp;
-    dp.ent = IdList{heads, tails, negs, B, B, N, c.num_entities, w.ent_perm, w.ent_sorted, w.ent_uniq, w.ent_seg, w.counts};
-    dp.rel = IdList{rels, rels, rels, B, 0, 0, c.num_relations, w.rel_perm, w.rel_sorted, w.rel_uniq, w.rel_seg, w.counts + 1};
-    dp.ent_blocks = (2 * B + N + RANK_THREADS - 1) / RANK_THREADS;
+    dp.ent = IdList{heads, tails, negs, B, B, N, c.num_entities,
+                    w.ent_perm, w.ent_sorted, w.ent_uniq, w.ent_seg, w.ent_segof, w.ent_tkeys, w.counts};
+    dp.rel = IdList{rels, rels, rels, B, 0, 0, c.num_relations,
+                    w.rel_perm, w.rel_sorted, w.rel_uniq, w.rel_seg, w.rel_segof, w.rel_tkeys, w.counts + 1};
+    dp.ent_tiles = dedup_tiles(2 * B + N);
     dp.status = w.status;
-    dp.Lrow = w.Lrow; dp.B = B; dp.loss_scale = c.loss_scale; dp.loss = w.loss; dp.loss_out = loss_out;
-    const int rel_blocks = (B + RANK_THREADS - 1) / RANK_THREADS;
+    const int tiles = dp.ent_tiles + dedup_tiles(B);
     stage_begin(h, ST_RANK, s);
-    rank_kernel<<<dp.ent_blocks + rel_blocks, RANK_THREADS, 0, s>>>(dp);
+    tile_sort_kernel<<<tiles, SORT_THREADS, 0, s>>>(dp);
+    KGE_LAUNCH_CHECK(h);
+    rank_kernel<<<tiles * (SORT_TILE / RANK_THREADS), RANK_THREADS, 0, s>>>(dp);
     stage_end(h, ST_RANK, s);
     KGE_LAUNCH_CHECK(h);
     stage_begin(h, ST_SEGMENT, s);
-    segment_kernel<<<3, SEG_THREADS, 0, s>>>(dp);
+    segment_kernel<<<2, SEG_THREADS, 0, s>>>(dp);
     stage_end(h, ST_SEGMENT, s);
     KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
+}
 
+int launch_update(kge_handle* h, uint64_t step, float lr, cudaStream_t s) {
+    const kge_config& c = h->cfg;
+    Workspace& w = h->ws;
+    const int B = c.batch, N = c.num_neg;
     UpdateParams up;
     up.njobs = c.score == KGE_TRANSH ? 3 : 2;
-    up.job[0] = UpdateJob{h->ent, h->ent_state, w.grad_ent, w.ent_uniq, w.ent_seg, w.ent_perm, w.counts, c.dim, 2 * B + N};
-    up.job[1] = UpdateJob{h->rel, h->rel_state, w.grad_rel, w.rel_uniq, w.rel_seg, w.rel_perm, w.counts + 1, h->kw, B};
-    up.job[2] = UpdateJob{h->relw, h->relw_state, w.grad_relw, w.rel_uniq, w.rel_seg, w.rel_perm, w.counts + 1, c.dim, B};
+    up.job[0] = UpdateJob{h->ent, h->ent_state, w.grad_ent, w.part_ent, w.ent_uniq, w.ent_seg, w.ent_perm,
+                          w.ent_sorted, w.ent_segof, c.dim, 2 * B + N};
+    up.job[1] = UpdateJob{h->rel, h->rel_state, w.grad_rel, w.part_rel, w.rel_uniq, w.rel_seg, w.rel_perm,
+                          w.rel_sorted, w.rel_segof, h->kw, B};
+    up.job[2] = UpdateJob{h->relw, h->relw_state, w.grad_relw, w.part_relw, w.rel_uniq, w.rel_seg, w.rel_perm,
+                          w.rel_sorted, w.rel_segof, c.dim, B};
     up.warp_begin[0] = 0;
-    for (int j = 0; j < 3; ++j) up.warp_begin[j + 1] = up.warp_begin[j] + (j < up.njobs ? up.job[j].max_rows : 0);
+    for (int j = 0; j < 3; ++j) up.warp_begin[j + 1] = up.warp_begin[j] + (j < up.njobs ? up.job[j].n : 0);
     up.opt = c.opt;
     up.lr = lr; up.beta1 = c.beta1; up.beta2 = c.beta2; up.eps = c.eps;
     up.corr1 = (float)(1.0 - std::pow((double)c.beta1, (double)(step + 1)));
     up.corr2 = (float)(1.0 - std::pow((double)c.beta2, (double)(step + 1)));
     const int warps = up.warp_begin[up.njobs];
     stage_begin(h, ST_UPDATE, s);
-    update_kernel<<<(warps * 32 + 255) / 256, 256, 0, s>>>(up);
+    piece_kernel<false><<<(warps * 32 + 255) / 256, 256, 0, s>>>(up);
+    KGE_LAUNCH_CHECK(h);
+    piece_kernel<true><<<(warps * 32 + 255) / 256, 256, 0, s>>>(up);
     stage_end(h, ST_UPDATE, s);
     KGE_LAUNCH_CHECK(h);
     return KGE_OK;
