@@ -54,7 +54,7 @@ ALU_PEAK_TOPS = 148 * 128 * 1.965e9 / 1e12
 # Algorithmic fp32 lane-operations per (query, negative, embedding coordinate) of each stage,
 # by pair kind: the minimum a CUDA-core evaluation of the definition needs.
 STAGE_OPS = {
-    "transe1": dict(block=2, accum_q=3, accum_t=3),     # sub, |.|+add  /  compare, sign-select, add
+    "transe1": dict(block=2, accum_q=2, accum_t=2),     # sub, |.|+add  /  compare, predicated add
     "rotate1": dict(block=3.5, accum_q=5, accum_t=5),   # per real coordinate; one sqrt / rsqrt per complex pair
     "distmult1": dict(block=1, accum_q=1, accum_t=1),   # one FMA
 }
@@ -297,7 +297,7 @@ def run_ours(args, w, name):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=5000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=sorted(WORKLOADS), default="c2_transe_l1")

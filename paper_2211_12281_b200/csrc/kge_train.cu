@@ -280,41 +280,43 @@ __global__ void __launch_bounds__(256) block_kernel(TrainParams p) {
 }
 
 // ------------------------------------------------------------------------------------------
-// block, kinds that are a function of (q, t) alone: 64 x 64 pairs per CTA, 4 x 4 per thread.
-// The 64 query rows and 64 negative rows of the tile are brought into shared memory by one
+// block, kinds that are a function of (q, t) alone: 32 x 64 pairs per CTA, 4 x 4 per thread.
+// The 32 query rows and 64 negative rows of the tile are brought into shared memory by one
 // asynchronous bulk copy per row (padded rows, so the 128-bit reads below are conflict-free),
 // up to 128 floats of the embedding axis per stage, two stages when the rows are longer.
 // ------------------------------------------------------------------------------------------
 constexpr int FKC = 128;
+constexpr int FTQ = 32;                  // query rows per tile
+constexpr int FTHREADS = FTQ * 4;        // 4 x 4 pairs per thread, 64 negative columns per tile
 
 __host__ __device__ inline int block_tma_kc(int d) { return d < FKC ? d : FKC; }
 __host__ __device__ inline int block_tma_stages(int d) { return d > FKC ? 2 : 1; }
 inline size_t block_tma_smem(int d) {
-    return (size_t)block_tma_stages(d) * 2 * TB * (block_tma_kc(d) + 4) * sizeof(float) + 2 * sizeof(uint64_t);
+    return (size_t)block_tma_stages(d) * (FTQ + TN) * (block_tma_kc(d) + 4) * sizeof(float) + 2 * sizeof(uint64_t);
 }
 
 template <int KIND>
-__global__ void __launch_bounds__(256) block_tma_kernel(TrainParams p) {
+__global__ void __launch_bounds__(FTHREADS) block_tma_kernel(TrainParams p) {
     extern __shared__ __align__(128) unsigned char smraw[];
+    constexpr int ROWS = FTQ + TN;       // rows [0, FTQ) of a stage hold queries, the rest negatives
     const int kc = block_tma_kc(p.d), ld = kc + 4, nstage = block_tma_stages(p.d);
     const int nchunk = (p.d + kc - 1) / kc;
     float* base = reinterpret_cast<float*>(smraw);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smraw + (size_t)nstage * 2 * TB * ld * sizeof(float));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smraw + (size_t)nstage * ROWS * ld * sizeof(float));
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-    const int b0 = blockIdx.y * TB, n0 = blockIdx.x * TN;
+    const int b0 = blockIdx.y * FTQ, n0 = blockIdx.x * TN;
 
     if (tid == 0) {
-        for (int st = 0; st < nstage; ++st) mbar_init(&bars[st], 2 * TB);
+        for (int st = 0; st < nstage; ++st) mbar_init(&bars[st], ROWS);
         mbar_init_fence();
     }
     __syncthreads();
 
-    // rows [0, 64) of a stage hold queries, rows [64, 128) negatives; thread r < 128 owns row r
-    auto issue = [&](int chunk, int stage) {
-        if (tid >= 2 * TB) return;
-        const bool isq = tid < TB;
-        const int g = isq ? b0 + tid : n0 + tid - TB;
-        float* dst = base + ((size_t)stage * 2 * TB + tid) * ld;
+    auto issue = [&](int chunk, int stage) {     // thread r < ROWS owns row r of the stage
+        if (tid >= ROWS) return;
+        const bool isq = tid < FTQ;
+        const int g = isq ? b0 + tid : n0 + tid - FTQ;
+        float* dst = base + ((size_t)stage * ROWS + tid) * ld;
         const int k0 = chunk * kc, len = min(kc, p.d - k0);
         if (g < (isq ? p.B : p.N)) {
             const float* src = (isq ? p.w.Q : p.w.Tneg) + (int64_t)g * p.d + k0;
@@ -344,15 +346,15 @@ __global__ void __launch_bounds__(256) block_tma_kernel(TrainParams p) {
             for (int st = 0; st < nstage; ++st) (void)mbar_wait_bounded(&bars[st], (uint32_t)(chunk / nstage) & 1u);
             return;
         }
-        const float* Qs = base + (size_t)stage * 2 * TB * ld;
-        const float* Ts = Qs + TB * ld;
+        const float* Qs = base + (size_t)stage * ROWS * ld;
+        const float* Ts = Qs + FTQ * ld;
         const int len = min(kc, p.d - chunk * kc);
 #pragma unroll 2
         for (int kk = 0; kk < len; kk += 4) {
             float4 qv[4], tv[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                qv[i] = *reinterpret_cast<const float4*>(&Qs[(ty + 16 * i) * ld + kk]);
+                qv[i] = *reinterpret_cast<const float4*>(&Qs[(ty + (FTQ / 4) * i) * ld + kk]);
                 tv[i] = *reinterpret_cast<const float4*>(&Ts[(tx + 16 * i) * ld + kk]);
             }
 #pragma unroll
@@ -369,7 +371,7 @@ __global__ void __launch_bounds__(256) block_tma_kernel(TrainParams p) {
     for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int b = b0 + ty + 16 * i, n = n0 + tx + 16 * j;
+            const int b = b0 + ty + (FTQ / 4) * i, n = n0 + tx + 16 * j;
             if (b >= p.B || n >= p.N) continue;
             float f = acc[i][j];
             if (KIND == KIND_L1 || KIND == KIND_CL1) f = -f;
@@ -674,7 +676,7 @@ __global__ void __launch_bounds__(256) accum_kernel(AccArgs a) {
 
 // ------------------------------------------------------------------------------------------
 // accum, kinds that are a function of (q, t) alone.  Same ownership as above (32 owner rows
-// per CTA, 4 per warp, one column split per blockIdx.y), but the rows of the other side arrive
+// per CTA, here 8 per warp, one column split per blockIdx.y), but the rows of the other side arrive
 // 32 at a time by one asynchronous bulk copy into a double buffer, and the 32 x 32 weight tile
 // of the next chunk is prefetched through registers while the current chunk is consumed.
 //
@@ -708,13 +710,17 @@ inline size_t accum_tma_smem(int d4) {
     return (size_t)2 * ACC_CC * d4 * 16 + (size_t)2 * ACC_CC * ACC_LDW * 4 + 8 * 32 * 4 + 2 * sizeof(uint64_t);
 }
 
-template <int KIND, int NCH, bool OWNER_Q>
-__global__ void __launch_bounds__(256) accum_tma_kernel(AccArgs a) {
+// ACC_WARPS warps per CTA, 32 / ACC_WARPS owner rows per warp (8 rows while the registers last).
+template <int KIND, int NCH, bool OWNER_Q, int ACC_WARPS>
+__global__ void __launch_bounds__(32 * ACC_WARPS) accum_tma_kernel(AccArgs a) {
+    constexpr int ACC_RPW = ACC_ROWS / ACC_WARPS;
+    constexpr int ACC_THREADS = 32 * ACC_WARPS;
+    constexpr int ACC_WPT = ACC_ROWS * ACC_CC / ACC_THREADS;   // weights of a tile handled per thread
     extern __shared__ __align__(128) unsigned char smraw[];
     const int d4 = a.d4;
     float4* Bs = reinterpret_cast<float4*>(smraw);                                  // [2][32][d4]
     float* Gs = reinterpret_cast<float*>(Bs + 2 * ACC_CC * d4);                     // [2][32][36], [c][r]
-    float* Csum = Gs + 2 * ACC_CC * ACC_LDW;                                        // [8][32]
+    float* Csum = Gs + 2 * ACC_CC * ACC_LDW;                                        // [warps][32]
     uint64_t* bars = reinterpret_cast<uint64_t*>(Csum + 8 * 32);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -733,12 +739,12 @@ __global__ void __launch_bounds__(256) accum_tma_kernel(AccArgs a) {
         mbar_arrive_expect_tx(&bars[buf], bytes);
         bulk_g2s(Bs + (size_t)buf * ACC_CC * d4, reinterpret_cast<const float4*>(a.oth) + (int64_t)c0 * d4, bytes, &bars[buf]);
     };
-    float greg[4];
+    float greg[ACC_WPT];
     auto load_weights = [&](int chunk) {
         const int c0 = c_begin + chunk * ACC_CC;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int idx = tid + 256 * e;
+        for (int e = 0; e < ACC_WPT; ++e) {
+            const int idx = tid + ACC_THREADS * e;
             int rr, cc; int64_t g;
             if (OWNER_Q) { cc = idx & 31; rr = idx >> 5; g = (int64_t)(r0 + rr) * a.N + (c0 + cc); }
             else         { rr = idx & 31; cc = idx >> 5; g = (int64_t)(c0 + cc) * a.N + (r0 + rr); }
@@ -747,19 +753,19 @@ __global__ void __launch_bounds__(256) accum_tma_kernel(AccArgs a) {
     };
     auto store_weights = [&](int buf) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int idx = tid + 256 * e;
+        for (int e = 0; e < ACC_WPT; ++e) {
+            const int idx = tid + ACC_THREADS * e;
             const int rr = OWNER_Q ? idx >> 5 : idx & 31, cc = OWNER_Q ? idx & 31 : idx >> 5;
             Gs[(buf * ACC_CC + cc) * ACC_LDW + rr] = greg[e];
         }
     };
 
-    float4 A[4][NCH], acc[4][NCH];
+    float4 A[ACC_RPW][NCH], acc[ACC_RPW][NCH];
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < ACC_RPW; ++i)
 #pragma unroll
         for (int j = 0; j < NCH; ++j) {
-            const int r = r0 + warp * 4 + i, c = lane + 32 * j;
+            const int r = r0 + warp * ACC_RPW + i, c = lane + 32 * j;
             A[i][j] = (r < a.own_rows && c < d4) ? reinterpret_cast<const float4*>(a.own)[(int64_t)r * d4 + c] : f4zero();
             acc[i][j] = f4zero();
         }
@@ -789,29 +795,36 @@ __global__ void __launch_bounds__(256) accum_tma_kernel(AccArgs a) {
         const float* Gc = Gs + cur * ACC_CC * ACC_LDW;
         if (KIND == KIND_L1 && !OWNER_Q) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) { const int cc = warp + 8 * e; if (cc < ccmax) csum += Gc[cc * ACC_LDW + lane]; }
+            for (int e = 0; e < ACC_CC / ACC_WARPS; ++e) {
+                const int cc = warp + ACC_WARPS * e;
+                if (cc < ccmax) csum += Gc[cc * ACC_LDW + lane];
+            }
         }
-#pragma unroll 4
+#pragma unroll 2
         for (int cc = 0; cc < ccmax; ++cc) {
-            const float4 g4 = *reinterpret_cast<const float4*>(&Gc[cc * ACC_LDW + warp * 4]);
-            const float gw[4] = {g4.x, g4.y, g4.z, g4.w};
+            float gw[ACC_RPW];
+#pragma unroll
+            for (int i = 0; i < ACC_RPW; i += 4) {
+                const float4 g4 = *reinterpret_cast<const float4*>(&Gc[cc * ACC_LDW + warp * ACC_RPW + i]);
+                gw[i] = g4.x; gw[i + 1] = g4.y; gw[i + 2] = g4.z; gw[i + 3] = g4.w;
+            }
 #pragma unroll
             for (int j = 0; j < NCH; ++j) {
                 const int c = lane + 32 * j;
                 if (c >= d4) continue;
                 const float4 bv = Bc[cc * d4 + c];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) acc_update2<KIND, OWNER_Q>(acc[i][j], A[i][j], bv, gw[i]);
+                for (int i = 0; i < ACC_RPW; ++i) acc_update2<KIND, OWNER_Q>(acc[i][j], A[i][j], bv, gw[i]);
             }
         }
         if (more) store_weights(cur ^ 1);
         __syncthreads();
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < ACC_RPW; ++i)
 #pragma unroll
         for (int j = 0; j < NCH; ++j) {
-            const int r = r0 + warp * 4 + i, c = lane + 32 * j;
+            const int r = r0 + warp * ACC_RPW + i, c = lane + 32 * j;
             if (r >= a.own_rows || c >= d4) continue;
             reinterpret_cast<float4*>(a.out)[((int64_t)blockIdx.y * a.own_rows + r) * d4 + c] = acc[i][j];
         }
@@ -820,7 +833,7 @@ __global__ void __launch_bounds__(256) accum_tma_kernel(AccArgs a) {
         __syncthreads();
         if (warp == 0 && r0 + lane < a.own_rows) {
             float t = 0.f;
-            for (int w = 0; w < 8; ++w) t += Csum[w * 32 + lane];
+            for (int w = 0; w < ACC_WARPS; ++w) t += Csum[w * 32 + lane];
             a.csum[(int64_t)blockIdx.y * a.own_rows + r0 + lane] = t;
         }
     }
@@ -1042,23 +1055,24 @@ cudaError_t launch_block_tma(const TrainParams& p, cudaStream_t s) {
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    dim3 grid((p.N + TN - 1) / TN, (p.B + TB - 1) / TB);
-    block_tma_kernel<KIND><<<grid, 256, smem, s>>>(p);
+    dim3 grid((p.N + TN - 1) / TN, (p.B + FTQ - 1) / FTQ);
+    block_tma_kernel<KIND><<<grid, FTHREADS, smem, s>>>(p);
     return cudaSuccess;
 }
 
 template <int KIND, int NCH, bool OWNER_Q>
 cudaError_t launch_accum_tma_inst(const AccArgs& a, cudaStream_t s) {
+    constexpr int WARPS = NCH == 4 ? 8 : 4;
     const size_t smem = accum_tma_smem(a.d4);
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(accum_tma_kernel<KIND, NCH, OWNER_Q>,
+        cudaError_t e = cudaFuncSetAttribute(accum_tma_kernel<KIND, NCH, OWNER_Q, WARPS>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)accum_tma_smem(kMaxDim / 4));
         if (e != cudaSuccess) return e;
         configured = true;
     }
     dim3 grid((a.own_rows + ACC_ROWS - 1) / ACC_ROWS, a.split);
-    accum_tma_kernel<KIND, NCH, OWNER_Q><<<grid, 256, smem, s>>>(a);
+    accum_tma_kernel<KIND, NCH, OWNER_Q, WARPS><<<grid, 32 * WARPS, smem, s>>>(a);
     return cudaSuccess;
 }
 
