@@ -10,7 +10,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libkge.so"
-SOURCES = ["kge_api.cu", "kge_sample.cu", "kge_train.cu", "kge_update.cu", "kge_infer.cu"]
+SOURCES = ["kge_api.cu", "kge_sample.cu", "kge_train.cu", "kge_tc.cu", "kge_update.cu", "kge_infer.cu"]
 
 
 def nvcc_path() -> str:

@@ -53,6 +53,11 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
     w.What = th ? cv.take<float>(B * d) : nullptr;
     w.Tneg = cv.take<float>(N * d);
     w.fpos = cv.take<float>(B); w.gpos = cv.take<float>(B); w.Lrow = cv.take<float>(B);
+    const bool tc = c.prec == KGE_PREC_BF16_TC;
+    w.Qb = tc ? cv.take<uint16_t>(B * d) : nullptr;
+    w.Tb = tc ? cv.take<uint16_t>(N * d) : nullptr;
+    w.qn2 = tc ? cv.take<float>(B) : nullptr;
+    w.tn2 = tc ? cv.take<float>(N) : nullptr;
     w.Grow = cv.take<float>(B);
     w.Cpart = cv.take<float>((size_t)h->split_t * N);
     w.F = cv.take<float>(B * N);
@@ -126,7 +131,12 @@ int kge_create(const kge_config* cfg, kge_handle** out) {
     if (c.head_part < 0 ? (c.batch % (P * P) != 0) : (c.batch % P != 0)) return KGE_ERR_DIVISIBILITY;
     const int64_t S = (c.num_entities + P - 1) / P;
     if (c.num_entities - (P - 1) * S <= 0) return KGE_ERR_EMPTY_BUCKET;  // last partition E_P would be empty
-    if (c.prec == KGE_PREC_BF16_TC) return KGE_ERR_UNSUPPORTED;
+    if (c.prec == KGE_PREC_BF16_TC) {
+        // tensor cores serve the scoring functions that are dense contractions: DistMult, ComplEx,
+        // and TransE with p = 2 through the norm expansion; rows are cut into 64-element slices
+        const bool contraction = c.score == KGE_DISTMULT || c.score == KGE_COMPLEX || (c.score == KGE_TRANSE && c.p_norm == 2);
+        if (!contraction || c.dim % 64 != 0) return KGE_ERR_UNSUPPORTED;
+    }
     kge_handle* h = new (std::nothrow) kge_handle();
     if (!h) return KGE_ERR_BAD_ARG;
     h->cfg = c;
@@ -207,6 +217,11 @@ int kge_bind(kge_handle* h, float* ent, float* rel, float* relw, float* ent_stat
     h->num_triples = num_triples; h->max_queries = max_queries; h->topk = topk;
     layout(h, h->ws_base, num_triples, max_queries, topk, &h->ws);
     KGE_CUDA_CHECK(h, cudaMemsetAsync(h->ws.status, 0, 256, static_cast<cudaStream_t>(stream)));
+    if (h->cfg.prec == KGE_PREC_BF16_TC) {
+        int rc = tc_make_operand_map(h, h->tm_q, h->ws.Qb, h->cfg.batch, h->cfg.dim);
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_t, h->ws.Tb, h->cfg.num_neg, h->cfg.dim);
+        if (rc != KGE_OK) return rc;
+    }
     if (!h->streams_ready) {
         KGE_CUDA_CHECK(h, cudaStreamCreateWithFlags(&h->side[0], cudaStreamNonBlocking));
         KGE_CUDA_CHECK(h, cudaStreamCreateWithFlags(&h->side[1], cudaStreamNonBlocking));

@@ -1,0 +1,250 @@
+// Tensor-core score block (5th-generation tensor cores: tcgen05.mma with the accumulator in
+// tensor memory, operands staged in shared memory by TMA tensor copies).
+//
+//   C[M, N] = A[M, K] . B[N, K]^T      A, B bf16, K contiguous; fp32 accumulation
+//
+// One CTA computes one 128 x 128 tile of C.  Warp 0 feeds a ring of shared-memory stages with
+// TMA (one elected lane), warp 1 issues the MMAs (one elected lane) and owns the tensor-memory
+// allocation, warps 2-5 read the finished accumulator out of tensor memory (each warp may
+// only touch the 32 lanes of its own quarter) and apply the epilogue:
+//   EPI_STORE   F = acc                                   DistMult / ComplEx (scoring-function table)
+//   EPI_L2DIST  F = -sqrt(max(|q|^2 + |t|^2 - 2 acc, 0))  TransE with p = 2 by the norm expansion
+// Every wait on a barrier is bounded; a wait that runs out records KGE_ERR_TIMEOUT, tells the
+// other warps to stop, and the CTA still releases its tensor memory before it returns.
+#include <cuda.h>
+
+#include "kge_common.cuh"
+
+namespace kge {
+
+namespace {
+
+constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 64;      // BK bf16 = one 128-byte swizzle row
+constexpr int TC_STAGES = 3;
+constexpr int TC_THREADS = 192;
+constexpr uint32_t TC_A_BYTES = TC_BM * TC_BK * 2, TC_B_BYTES = TC_BN * TC_BK * 2;
+constexpr uint32_t TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
+constexpr size_t TC_SMEM_BYTES = 1024 + (size_t)TC_STAGES * TC_STAGE_BYTES + 128;
+constexpr uint32_t TC_TMEM_COLS = 128;                    // fp32 accumulator: one column per element of a row
+
+enum { EPI_STORE = 0, EPI_L2DIST = 1 };
+
+struct TcGemmParams {
+    int M, N, K;
+    float* C; int64_t ldc;
+    const float *row_norm2, *col_norm2;   // EPI_L2DIST: |q_b|^2 [M], |t_n|^2 [N]
+    int32_t* status;
+};
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major operand tile written by TMA with the 128-byte
+// swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart, tile base 1024-byte aligned.
+__device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);   // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                          // leading byte offset (not used by swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                          // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                          // layout type: 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M x N tile.
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives on the barrier once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 32 consecutive fp32 columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                             const __grid_constant__ CUtensorMap tmB, TcGemmParams p) {
+    extern __shared__ unsigned char tc_smem_raw[];
+    unsigned char* base = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
+    uint64_t* full = reinterpret_cast<uint64_t*>(base + (size_t)TC_STAGES * TC_STAGE_BYTES);
+    uint64_t* empty = full + TC_STAGES;
+    uint64_t* accum_full = empty + TC_STAGES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum_full + 1);
+    volatile uint32_t* stop = tmem_slot + 1;    // set by a warp whose wait ran out
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.y * TC_BM, n0 = blockIdx.x * TC_BN;
+    const int nkb = (p.K + TC_BK - 1) / TC_BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        mbar_init(accum_full, 1);
+        *stop = 0;
+        mbar_init_fence();
+    }
+    if (warp == 1) {   // one warp allocates the accumulator columns and gives up the right to allocate more
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TC_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_acc = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kb = 0; kb < nkb && !*stop; ++kb) {
+                const int s = kb % TC_STAGES;
+                if (!mbar_wait_bounded(&empty[s], ((kb / TC_STAGES) & 1) ^ 1)) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); break; }
+                unsigned char* sa = base + (size_t)s * TC_STAGE_BYTES;
+                mbar_arrive_expect_tx(&full[s], TC_STAGE_BYTES);
+                tma_load_2d(sa, &tmA, kb * TC_BK, m0, &full[s]);
+                tma_load_2d(sa + TC_A_BYTES, &tmB, kb * TC_BK, n0, &full[s]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(TC_BM, TC_BN);
+            bool ok = true;
+            for (int kb = 0; kb < nkb && !*stop; ++kb) {
+                const int s = kb % TC_STAGES;
+                if (!mbar_wait_bounded(&full[s], (kb / TC_STAGES) & 1)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t sa = smem_u32(base + (size_t)s * TC_STAGE_BYTES);
+#pragma unroll
+                for (int k = 0; k < TC_BK / 16; ++k) {   // one MMA covers 16 bf16 = 32 bytes of K
+                    umma_bf16(tmem_acc, umma_desc_k_sw128(sa + k * 32), umma_desc_k_sw128(sa + TC_A_BYTES + k * 32),
+                              idesc, (kb | k) != 0);
+                }
+                umma_commit(&empty[s]);            // the stage is free once these MMAs have read it
+            }
+            if (!ok) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); }
+            umma_commit(accum_full);               // also on failure, so the epilogue warps do not wait in vain
+        }
+    } else {
+        const bool ok = mbar_wait_bounded(accum_full, 0);
+        tc_fence_after();
+        if (ok && !*stop) {
+            const int quarter = warp & 3;          // tensor-memory lanes this warp may read
+            const int row = m0 + quarter * 32 + lane;
+            float rn = 0.f;
+            if (EPI == EPI_L2DIST && row < p.M) rn = p.row_norm2[row];
+#pragma unroll 1
+            for (int c0 = 0; c0 < TC_BN; c0 += 32) {
+                float v[32];
+                tmem_ld32(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
+                if (row < p.M) {
+                    float* dst = p.C + (int64_t)row * p.ldc + n0 + c0;
+                    if (EPI == EPI_L2DIST) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const int col = n0 + c0 + i;
+                            const float d2 = rn + (col < p.N ? p.col_norm2[col] : 0.f) - 2.f * v[i];
+                            v[i] = -sqrtf(fmaxf(d2, 0.f));
+                        }
+                    }
+                    if (n0 + c0 + 32 <= p.N && (p.ldc & 3) == 0) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4)
+                            *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) if (n0 + c0 + i < p.N) dst[i] = v[i];
+                    }
+                }
+            }
+        } else if (!ok && lane == 0) {
+            *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(TC_TMEM_COLS) : "memory");
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+}  // namespace
+
+// Tensor map of a row-major bf16 matrix [rows, cols] (cols contiguous, cols % 8 == 0, base
+// 16-byte aligned) read in boxes of 128 rows x 64 columns with the 128-byte swizzle.
+int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) { h->cuda_err = "cuTensorMapEncodeTiled is not available from this driver"; return KGE_ERR_CUDA; }
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)TC_BM};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(static_cast<CUtensorMap*>(map_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
+                          dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { h->cuda_err = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r); return KGE_ERR_CUDA; }
+    return KGE_OK;
+}
+
+// F[B, N] from the bf16 copies of the query vectors and the staged negatives.
+int launch_tc_scores(kge_handle* h, cudaStream_t s) {
+    const kge_config& c = h->cfg;
+    TcGemmParams p;
+    p.M = c.batch; p.N = c.num_neg; p.K = c.dim;
+    p.C = h->ws.F; p.ldc = c.num_neg;
+    p.row_norm2 = h->ws.qn2; p.col_norm2 = h->ws.tn2;
+    p.status = h->ws.status;
+    static bool configured = false;
+    if (!configured) {
+        KGE_CUDA_CHECK(h, cudaFuncSetAttribute(tc_gemm_kernel<EPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES));
+        KGE_CUDA_CHECK(h, cudaFuncSetAttribute(tc_gemm_kernel<EPI_L2DIST>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES));
+        configured = true;
+    }
+    const dim3 grid((p.N + TC_BN - 1) / TC_BN, (p.M + TC_BM - 1) / TC_BM);
+    const CUtensorMap& tq = *reinterpret_cast<const CUtensorMap*>(h->tm_q);
+    const CUtensorMap& tt = *reinterpret_cast<const CUtensorMap*>(h->tm_t);
+    if (h->kind == KIND_L2) tc_gemm_kernel<EPI_L2DIST><<<grid, TC_THREADS, TC_SMEM_BYTES, s>>>(tq, tt, p);
+    else tc_gemm_kernel<EPI_STORE><<<grid, TC_THREADS, TC_SMEM_BYTES, s>>>(tq, tt, p);
+    KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
+}
+
+}  // namespace kge

@@ -4,6 +4,8 @@
 //   loss     : per-positive loss and dL/dF (Section 3.1 "Loss Functions"), in place
 //   accum    : dQ_b = sum_n G_bn df/dq,  dT_n = sum_b G_bn df/dt  (owner computes, no atomics)
 //   chain    : positive pair, chain rule q -> (h, r, w), reduction of the column splits
+#include <cuda_bf16.h>
+
 #include "kge_common.cuh"
 
 namespace kge {
@@ -33,6 +35,11 @@ __device__ __forceinline__ float4 f4fma(float s, float4 a, float4 c) {
 __device__ __forceinline__ float f4dot(float4 a, float4 b) { return a.x * b.x + a.y * b.y + a.z * b.z + a.w * b.w; }
 __device__ __forceinline__ float sgnf(float x) { return (x > 0.f ? 1.f : 0.f) - (x < 0.f ? 1.f : 0.f); }
 __device__ __forceinline__ float4 f4sgn(float4 a) { return make_float4(sgnf(a.x), sgnf(a.y), sgnf(a.z), sgnf(a.w)); }
+// Four floats rounded to bf16 (nearest even), packed in memory order.
+__device__ __forceinline__ uint2 pack_bf16x4(float4 v) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    return make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+}
 
 
 // ------------------------------------------------------------------------------------------
@@ -59,7 +66,16 @@ __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
         const int64_t id = checked_id(p.negs[n], p.E, p.w.status);
         const float4* src = reinterpret_cast<const float4*>(p.ent) + id * d4;
         float4* dst = reinterpret_cast<float4*>(p.w.Tneg) + (int64_t)n * d4;
-        for (int c = lane; c < d4; c += 32) dst[c] = src[c];
+        float nrm2 = 0.f;
+        for (int c = lane; c < d4; c += 32) {
+            const float4 v = src[c];
+            dst[c] = v;
+            if (p.w.Tb) {   // tensor-core scoring: bf16 copy and the squared norm of the unrounded row
+                reinterpret_cast<uint2*>(p.w.Tb)[(int64_t)n * d4 + c] = pack_bf16x4(v);
+                nrm2 += f4dot(v, v);
+            }
+        }
+        if (p.w.Tb) { nrm2 = warp_sum(nrm2); if (lane == 0) p.w.tn2[n] = nrm2; }
         return;
     }
     const int b = warp;
@@ -126,6 +142,16 @@ __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
     float4* qdst = reinterpret_cast<float4*>(p.w.Q) + (int64_t)b * d4;
 #pragma unroll
     for (int i = 0; i < kMaxChunks; ++i) { const int c = lane + 32 * i; if (c < d4) qdst[c] = q[i]; }
+    if (p.w.Qb) {
+        float nrm2 = 0.f;
+#pragma unroll
+        for (int i = 0; i < kMaxChunks; ++i) {
+            const int c = lane + 32 * i;
+            if (c < d4) { reinterpret_cast<uint2*>(p.w.Qb)[(int64_t)b * d4 + c] = pack_bf16x4(q[i]); nrm2 += f4dot(q[i], q[i]); }
+        }
+        nrm2 = warp_sum(nrm2);
+        if (lane == 0) p.w.qn2[b] = nrm2;
+    }
     float acc = 0.f;
     if (p.score == KGE_TRANSH) {
         float4* wdst = reinterpret_cast<float4*>(p.w.What) + (int64_t)b * d4;
@@ -1140,6 +1166,11 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     stage_end(h, ST_BUILD, s);
     KGE_LAUNCH_CHECK(h);
     stage_begin(h, ST_BLOCK, s);
+    if (c.prec == KGE_PREC_BF16_TC) {
+        const int rc = launch_tc_scores(h, s);
+        if (rc != KGE_OK) return rc;
+        h->launches -= 1;   // counted again below
+    } else
     switch (p.kind) {
         case KIND_L1: KGE_CUDA_CHECK(h, launch_block_tma<KIND_L1>(p, s)); break;
         case KIND_L2: KGE_CUDA_CHECK(h, launch_block_tma<KIND_L2>(p, s)); break;

@@ -28,13 +28,14 @@ class Problem:
 
     def __init__(self, *, E, R, T, d, score, p_norm=1, loss="logsigmoid", opt="sgd", B, N, P,
                  gamma=0.0, adv_temp=0.0, ce_correction=0.0, loss_scale=1.0, lr=0.1, head_part=-1,
-                 sample_mode=0, seed=0, graph_seed=0, relation_zipf=0.0, eps=None):
+                 sample_mode=0, seed=0, graph_seed=0, relation_zipf=0.0, eps=None, tc=False):
         self.kw = dict(num_entities=E, num_relations=R, dim=d, score=score, p_norm=p_norm, loss=loss, opt=opt,
                        batch=B, num_neg=N, num_parts=P, gamma=gamma, adv_temp=adv_temp,
                        ce_correction=ce_correction, loss_scale=loss_scale, lr=lr, head_part=head_part,
                        sample_mode=sample_mode, seed=seed, eps=eps)
         self.E, self.R, self.T, self.d, self.B, self.N, self.P = E, R, T, d, B, N, P
         self.score, self.opt, self.lr = score, opt, lr
+        self.tc = tc      # bf16 tensor-core score block on the GPU, bf16-rounded operands in the oracle
         self.h, self.r, self.t = kge_synth.make_graph(E, R, T, seed=graph_seed, relation_zipf=relation_zipf)
         self.ent, self.rel, self.relw = kge_synth.make_tables(E, R, d, score, seed=graph_seed)
 
@@ -43,7 +44,7 @@ class Problem:
         return self.d // 2 if self.score == "rotate" else self.d
 
     def oracle_cfg(self):
-        return oracle_config(**self.kw)
+        return oracle_config(**self.kw, bf16_operands=1 if self.tc else 0)
 
     def state_shapes(self):
         if self.opt == "sgd":
@@ -69,7 +70,7 @@ class GpuSide:
         self.relw = None if prob.relw is None else torch.from_numpy(prob.relw).to(dev)
         shapes = prob.state_shapes()
         self.states = [None if s is None else torch.zeros(s, dtype=torch.float32, device=dev) for s in shapes]
-        self.kge = K.Kge(K.KgeConfig.make(**prob.kw))
+        self.kge = K.Kge(K.KgeConfig.make(**prob.kw, prec=K.PREC_BF16_TC if prob.tc else K.PREC_FP32))
         self.kge.bind(self.ent, self.rel, self.relw, *self.states, num_triples=prob.T if load_graph else 0,
                       max_queries=max_queries, topk=topk)
         if load_graph:
