@@ -34,6 +34,16 @@ int pick_split(int rows, int cols, int num_sms) {
     return std::max(1, (cols + per - 1) / per);
 }
 
+// Tensor-core contraction [rows, cols] over `depth`: enough K splits to give every SM a tile,
+// each split at least four 64-wide slices deep, at most 16, none empty.
+int pick_split_tc(int rows, int cols, int depth, int num_sms) {
+    const int tiles = ((rows + 127) / 128) * ((cols + 127) / 128);
+    const int kb = (depth + 63) / 64;
+    const int want = std::max(1, std::min(std::min((num_sms + tiles - 1) / tiles, std::max(1, kb / 4)), 16));
+    const int per = (kb + want - 1) / want;
+    return (kb + per - 1) / per;
+}
+
 size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t topk, Workspace* out) {
     const kge_config& c = h->cfg;
     const size_t B = c.batch, N = c.num_neg, d = c.dim, kw = h->kw;
@@ -58,6 +68,12 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
     w.Tb = tc ? cv.take<uint16_t>(N * d) : nullptr;
     w.qn2 = tc ? cv.take<float>(B) : nullptr;
     w.tn2 = tc ? cv.take<float>(N) : nullptr;
+    const size_t ldN = (N + 7) / 8 * 8, ldB = (B + 7) / 8 * 8;
+    w.Gb = tc ? cv.take<uint16_t>(B * ldN) : nullptr;
+    w.GbT = tc ? cv.take<uint16_t>(N * ldB) : nullptr;
+    w.TbT = tc ? cv.take<uint16_t>(d * ldN) : nullptr;
+    w.QbT = tc ? cv.take<uint16_t>(d * ldB) : nullptr;
+    w.Gcol = tc ? cv.take<float>(N) : nullptr;
     w.Grow = cv.take<float>(B);
     w.Cpart = cv.take<float>((size_t)h->split_t * N);
     w.F = cv.take<float>(B * N);
@@ -154,6 +170,10 @@ int kge_create(const kge_config* cfg, kge_handle** out) {
         (void)cudaGetLastError();
     h->split_q = pick_split(c.batch, c.num_neg, h->num_sms);
     h->split_t = pick_split(c.num_neg, c.batch, h->num_sms);
+    if (c.prec == KGE_PREC_BF16_TC) {   // the backward contractions run as 128 x 128 tensor-core tiles split over K
+        h->split_q = pick_split_tc(c.batch, c.dim, c.num_neg, h->num_sms);
+        h->split_t = pick_split_tc(c.num_neg, c.dim, c.batch, h->num_sms);
+    }
     *out = h;
     return KGE_OK;
 }
@@ -218,8 +238,14 @@ int kge_bind(kge_handle* h, float* ent, float* rel, float* relw, float* ent_stat
     layout(h, h->ws_base, num_triples, max_queries, topk, &h->ws);
     KGE_CUDA_CHECK(h, cudaMemsetAsync(h->ws.status, 0, 256, static_cast<cudaStream_t>(stream)));
     if (h->cfg.prec == KGE_PREC_BF16_TC) {
-        int rc = tc_make_operand_map(h, h->tm_q, h->ws.Qb, h->cfg.batch, h->cfg.dim);
-        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_t, h->ws.Tb, h->cfg.num_neg, h->cfg.dim);
+        const int64_t B = h->cfg.batch, N = h->cfg.num_neg, d = h->cfg.dim;
+        const int64_t ldN = (N + 7) / 8 * 8, ldB = (B + 7) / 8 * 8;
+        int rc = tc_make_operand_map(h, h->tm_q, h->ws.Qb, B, d, d);
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_t, h->ws.Tb, N, d, d);
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_g, h->ws.Gb, B, N, ldN);
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_gt, h->ws.GbT, N, B, ldB);
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_tt, h->ws.TbT, d, N, ldN);
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_qt, h->ws.QbT, d, B, ldB);
         if (rc != KGE_OK) return rc;
     }
     if (!h->streams_ready) {

@@ -47,6 +47,8 @@ struct Workspace {
     float *Q, *What, *Tneg;                // [B,d], [B,d] (TransH), [N,d]
     float *fpos, *gpos, *Lrow;             // [B]
     uint16_t *Qb, *Tb;                     // [B,d], [N,d] bf16 copies of Q and Tneg (tensor-core scoring)
+    uint16_t *Gb, *GbT, *TbT, *QbT;        // bf16 [B,ldN], [N,ldB], [d,ldN], [d,ldB]: dL/dF and transposes (ld = size rounded up to 8)
+    float *Gcol;                           // [N] column sums of dL/dF (TransE p=2 on tensor cores)
     float *qn2, *tn2;                      // [B], [N] squared norms of the fp32 rows (TransE p=2 by norm expansion)
     float *Grow;                           // [B] row sums of dL/dF (TransE p=1 backward)
     float *Cpart;                          // [St, N] column sums of dL/dF per row split (TransE p=1 backward)
@@ -103,7 +105,8 @@ struct kge_handle {
     int num_sms;
     // Side streams and events of the training step: the sort of the touched ids and one of the
     // two backward accumulations run beside the main stream's kernels (created by kge_bind).
-    alignas(64) unsigned char tm_q[128], tm_t[128];   // TMA tensor maps of Qb and Tb (tensor-core scoring)
+    // TMA tensor maps (tensor-core path): Qb, Tb for the scores; Gb, Tb^T for dQ; Gb^T, Qb^T for dT
+    alignas(64) unsigned char tm_q[128], tm_t[128], tm_g[128], tm_gt[128], tm_tt[128], tm_qt[128];
     bool streams_ready;
     cudaStream_t side[2];
     cudaEvent_t ev_ids, ev_loss, ev_seg, ev_t;
@@ -152,7 +155,8 @@ int launch_dedup(kge_handle* h, const int32_t* heads, const int32_t* rels, const
 // Segment sums of the gradient rows and the optimiser step (needs both of the above).
 int launch_update(kge_handle* h, uint64_t step, float lr, cudaStream_t s);
 // Tensor-core score block: F from the bf16 operand copies; tensor maps are made at bind time.
-int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols);
+int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols, int64_t ld);
+int launch_tc_backward(kge_handle* h, cudaStream_t s, cudaStream_t side);
 int launch_tc_scores(kge_handle* h, cudaStream_t s);
 int dedup_tiles(int n);     // sort tiles of a list of n ids
 int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int32_t nq, int32_t k,

@@ -12,6 +12,9 @@
 // Every wait on a barrier is bounded; a wait that runs out records KGE_ERR_TIMEOUT, tells the
 // other warps to stop, and the CTA still releases its tensor memory before it returns.
 #include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <algorithm>
 
 #include "kge_common.cuh"
 
@@ -31,7 +34,9 @@ enum { EPI_STORE = 0, EPI_L2DIST = 1 };
 
 struct TcGemmParams {
     int M, N, K;
+    int kb_per_split;                     // 64-wide slices of K per blockIdx.z
     float* C; int64_t ldc;
+    int64_t split_stride;                 // floats between the output slabs of consecutive K splits
     const float *row_norm2, *col_norm2;   // EPI_L2DIST: |q_b|^2 [M], |t_n|^2 [N]
     int32_t* status;
 };
@@ -101,7 +106,9 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.y * TC_BM, n0 = blockIdx.x * TC_BN;
-    const int nkb = (p.K + TC_BK - 1) / TC_BK;
+    const int kb_begin = blockIdx.z * p.kb_per_split;
+    const int nkb = min(p.kb_per_split, (p.K + TC_BK - 1) / TC_BK - kb_begin);   // >= 1 by the launch geometry
+    float* const Cout = p.C + (int64_t)blockIdx.z * p.split_stride;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < TC_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -125,8 +132,8 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
                 if (!mbar_wait_bounded(&empty[s], ((kb / TC_STAGES) & 1) ^ 1)) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); break; }
                 unsigned char* sa = base + (size_t)s * TC_STAGE_BYTES;
                 mbar_arrive_expect_tx(&full[s], TC_STAGE_BYTES);
-                tma_load_2d(sa, &tmA, kb * TC_BK, m0, &full[s]);
-                tma_load_2d(sa + TC_A_BYTES, &tmB, kb * TC_BK, n0, &full[s]);
+                tma_load_2d(sa, &tmA, (kb_begin + kb) * TC_BK, m0, &full[s]);
+                tma_load_2d(sa + TC_A_BYTES, &tmB, (kb_begin + kb) * TC_BK, n0, &full[s]);
             }
         }
     } else if (warp == 1) {
@@ -161,7 +168,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
                 float v[32];
                 tmem_ld32(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
                 if (row < p.M) {
-                    float* dst = p.C + (int64_t)row * p.ldc + n0 + c0;
+                    float* dst = Cout + (int64_t)row * p.ldc + n0 + c0;
                     if (EPI == EPI_L2DIST) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
@@ -190,6 +197,61 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(TC_TMEM_COLS) : "memory");
 }
 
+// src fp32 [R, C] (leading dimension lds) -> bf16 copies for the backward contractions:
+// dst_rm [R, ld_rm] as it is (optional) and dst_t [C, ld_t] transposed; colsum[C] (optional)
+// = column sums of src, added in ascending row order.  A CTA owns 32 columns and walks the
+// rows of its blockIdx.y share in tiles of 32.
+struct CastParams {
+    const float* src; int64_t lds;
+    int R, C, rows_per_cta;
+    uint16_t* dst_rm; int64_t ld_rm;
+    uint16_t* dst_t; int64_t ld_t;
+    float* colsum;
+};
+
+__device__ __forceinline__ uint16_t bf16_bits(float v) {
+    const __nv_bfloat16 b = __float2bfloat16_rn(v);
+    return *reinterpret_cast<const uint16_t*>(&b);
+}
+
+__global__ void __launch_bounds__(256) cast_transpose_kernel(CastParams p) {
+    __shared__ float tile[32][33];
+    __shared__ float csm[8][32];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int c0 = blockIdx.x * 32;
+    const int r_begin = blockIdx.y * p.rows_per_cta, r_end = min(p.R, r_begin + p.rows_per_cta);
+    float cs = 0.f;
+    for (int r0 = r_begin; r0 < r_end; r0 += 32) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = r0 + ty + 8 * i, c = c0 + tx;
+            float v = 0.f;
+            if (r < r_end && c < p.C) {
+                v = p.src[(int64_t)r * p.lds + c];
+                if (p.dst_rm) p.dst_rm[(int64_t)r * p.ld_rm + c] = bf16_bits(v);
+            }
+            tile[ty + 8 * i][tx] = v;
+            cs += v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int c = c0 + ty + 8 * i, r = r0 + tx;
+            if (c < p.C && r < r_end) p.dst_t[(int64_t)c * p.ld_t + r] = bf16_bits(tile[tx][ty + 8 * i]);
+        }
+        __syncthreads();
+    }
+    if (p.colsum) {   // thread (tx, ty) has summed rows ty, ty + 8, ... of column tx: add the 8 partial sums in order
+        csm[ty][tx] = cs;
+        __syncthreads();
+        if (ty == 0 && c0 + tx < p.C) {
+            float t = 0.f;
+            for (int w = 0; w < 8; ++w) t += csm[w][tx];
+            p.colsum[c0 + tx] = t;
+        }
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -208,13 +270,14 @@ EncodeTiledFn encode_tiled_fn() {
 
 }  // namespace
 
-// Tensor map of a row-major bf16 matrix [rows, cols] (cols contiguous, cols % 8 == 0, base
-// 16-byte aligned) read in boxes of 128 rows x 64 columns with the 128-byte swizzle.
-int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols) {
+// Tensor map of a row-major bf16 matrix [rows, cols] with leading dimension ld (ld % 8 == 0,
+// base 16-byte aligned) read in boxes of 128 rows x 64 columns with the 128-byte swizzle;
+// what a box covers beyond the matrix reads as zero.
+int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols, int64_t ld) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) { h->cuda_err = "cuTensorMapEncodeTiled is not available from this driver"; return KGE_ERR_CUDA; }
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
     const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)TC_BM};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = fn(static_cast<CUtensorMap*>(map_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
@@ -229,6 +292,7 @@ int launch_tc_scores(kge_handle* h, cudaStream_t s) {
     const kge_config& c = h->cfg;
     TcGemmParams p;
     p.M = c.batch; p.N = c.num_neg; p.K = c.dim;
+    p.kb_per_split = (p.K + TC_BK - 1) / TC_BK; p.split_stride = 0;
     p.C = h->ws.F; p.ldc = c.num_neg;
     p.row_norm2 = h->ws.qn2; p.col_norm2 = h->ws.tn2;
     p.status = h->ws.status;
@@ -244,6 +308,74 @@ int launch_tc_scores(kge_handle* h, cudaStream_t s) {
     if (h->kind == KIND_L2) tc_gemm_kernel<EPI_L2DIST><<<grid, TC_THREADS, TC_SMEM_BYTES, s>>>(tq, tt, p);
     else tc_gemm_kernel<EPI_STORE><<<grid, TC_THREADS, TC_SMEM_BYTES, s>>>(tq, tt, p);
     KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
+}
+
+
+namespace {
+int launch_cast(kge_handle* h, const float* src, int64_t lds, int R, int C, uint16_t* dst_rm, int64_t ld_rm,
+                uint16_t* dst_t, int64_t ld_t, float* colsum, cudaStream_t s) {
+    CastParams cp{src, lds, R, C, R, dst_rm, ld_rm, dst_t, ld_t, colsum};
+    int row_ctas = 1;
+    if (!colsum) {   // no column sums: the rows may be shared out to fill the device
+        const int col_ctas = (C + 31) / 32;
+        row_ctas = std::max(1, std::min((R + 31) / 32, (2 * h->num_sms + col_ctas - 1) / col_ctas));
+        cp.rows_per_cta = ((R + row_ctas - 1) / row_ctas + 31) / 32 * 32;
+        row_ctas = (R + cp.rows_per_cta - 1) / cp.rows_per_cta;
+    }
+    cast_transpose_kernel<<<dim3((C + 31) / 32, row_ctas), 256, 0, s>>>(cp);
+    KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
+}
+
+int launch_tc_gemm(kge_handle* h, const unsigned char* tmA, const unsigned char* tmB, int M, int N, int K, int split,
+                   float* C, int64_t ldc, cudaStream_t s) {
+    TcGemmParams p;
+    p.M = M; p.N = N; p.K = K;
+    const int kb = (K + TC_BK - 1) / TC_BK;
+    p.kb_per_split = (kb + split - 1) / split;
+    p.C = C; p.ldc = ldc; p.split_stride = (int64_t)M * ldc;
+    p.row_norm2 = p.col_norm2 = nullptr;
+    p.status = h->ws.status;
+    const dim3 grid((N + TC_BN - 1) / TC_BN, (M + TC_BM - 1) / TC_BM, (kb + p.kb_per_split - 1) / p.kb_per_split);
+    tc_gemm_kernel<EPI_STORE><<<grid, TC_THREADS, TC_SMEM_BYTES, s>>>(*reinterpret_cast<const CUtensorMap*>(tmA),
+                                                                       *reinterpret_cast<const CUtensorMap*>(tmB), p);
+    KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
+}
+}  // namespace
+
+// The two backward contractions on tensor cores, from bf16 copies of dL/dF (held in F):
+//   dQ partial[split] = G . T      (A = Gb [B, N],   B operand = Tb^T [d, N])
+//   dT partial[split] = G^T . Q    (A = Gb^T [N, B], B operand = Qb^T [d, B])
+// The K splits land in the same partial buffers the CUDA-core path uses and are added in
+// ascending order by the chain kernel.  With a side stream the dQ contraction runs beside dT.
+int launch_tc_backward(kge_handle* h, cudaStream_t s, cudaStream_t side) {
+    const kge_config& c = h->cfg;
+    Workspace& w = h->ws;
+    const int B = c.batch, N = c.num_neg, d = c.dim;
+    const int64_t ldN = (N + 7) / 8 * 8, ldB = (B + 7) / 8 * 8;
+    int rc;
+    stage_begin(h, ST_TH_CPASS, s);   // stage slot shared with the TransH pass: operand casts
+    if ((rc = launch_cast(h, w.F, N, B, N, w.Gb, ldN, w.GbT, ldB, w.Gcol, s)) != KGE_OK) return rc;
+    if ((rc = launch_cast(h, w.Tneg, d, N, d, nullptr, 0, w.TbT, ldN, nullptr, s)) != KGE_OK) return rc;
+    if ((rc = launch_cast(h, w.Q, d, B, d, nullptr, 0, w.QbT, ldB, nullptr, s)) != KGE_OK) return rc;
+    stage_end(h, ST_TH_CPASS, s);
+    if (side) {
+        KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_loss, s));
+        KGE_CUDA_CHECK(h, cudaStreamWaitEvent(side, h->ev_loss, 0));
+    }
+    cudaStream_t sq = side ? side : s;
+    stage_begin(h, ST_ACCUM_Q, sq);
+    rc = launch_tc_gemm(h, h->tm_g, h->tm_tt, B, d, N, h->split_q, w.dQpart, d, sq);
+    stage_end(h, ST_ACCUM_Q, sq);
+    if (rc != KGE_OK) return rc;
+    if (side) KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_t, side));
+    stage_begin(h, ST_ACCUM_T, s);
+    rc = launch_tc_gemm(h, h->tm_gt, h->tm_qt, N, d, B, h->split_t, w.dTpart, d, s);
+    stage_end(h, ST_ACCUM_T, s);
+    if (rc != KGE_OK) return rc;
+    if (side) KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_t, 0));
     return KGE_OK;
 }
 

@@ -21,6 +21,7 @@ struct TrainParams {
     const int32_t *heads, *rels, *tails, *negs;
     int split_q, split_t;
     float* loss_out;    // caller's device scalar for the batch loss, or NULL
+    int tc_l2;          // TransE p = 2 with tensor-core backward: the splits hold C.T and C^T.Q, C = dL/dF / distance
     Workspace w;
 };
 
@@ -904,6 +905,11 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
             float4 s = f4zero();
             for (int sp = 0; sp < p.split_t; ++sp) s = f4add(s, part[((int64_t)sp * p.N + n) * d4 + c]);
             if (p.kind == KIND_L1) s = make_float4(2.f * s.x - wsum, 2.f * s.y - wsum, 2.f * s.z - wsum, 2.f * s.w - wsum);
+            if (p.tc_l2) {   // dT_n = sum_b C_bn (q_b - t_n) = (C^T Q)_n - (column sum of C) t_n
+                const float cs = p.w.Gcol[n];
+                const float4 t = reinterpret_cast<const float4*>(p.w.Tneg)[(int64_t)n * d4 + c];
+                s = make_float4(s.x - cs * t.x, s.y - cs * t.y, s.z - cs * t.z, s.w - cs * t.w);
+            }
             gent[(int64_t)(2 * p.B + n) * d4 + c] = s;
         }
         return;
@@ -930,6 +936,10 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
         if (p.kind == KIND_L1 && in) {   // the splits hold P; dQ = (row sum of dL/dF) - 2 P
             const float rs = p.w.Grow[b];
             s = make_float4(rs - 2.f * s.x, rs - 2.f * s.y, rs - 2.f * s.z, rs - 2.f * s.w);
+        }
+        if (p.tc_l2 && in) {             // dQ_b = sum_n C_bn (t_n - q_b) = (C T)_b - (row sum of C) q_b
+            const float rs = p.w.Grow[b];
+            s = make_float4(s.x - rs * q[i].x, s.y - rs * q[i].y, s.z - rs * q[i].z, s.w - rs * q[i].w);
         }
         dq[i] = s; dt[i] = f4zero();
     }
@@ -1152,6 +1162,7 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     p.heads = heads; p.rels = rels; p.tails = tails; p.negs = negs;
     p.split_q = h->split_q; p.split_t = h->split_t;
     p.loss_out = loss_out;
+    p.tc_l2 = c.prec == KGE_PREC_BF16_TC && p.kind == KIND_L2;
     p.w = h->ws;
     const int nch = p.d4 <= 32 ? 1 : (p.d4 <= 64 ? 2 : 4);
 
@@ -1207,6 +1218,10 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
         KGE_LAUNCH_CHECK(h);
     }
 
+    if (c.prec == KGE_PREC_BF16_TC) {
+        const int rc = launch_tc_backward(h, s, side);
+        if (rc != KGE_OK) return rc;
+    } else {
     AccArgs aq;
     aq.own = p.w.Q; aq.oth = p.w.Tneg; aq.what = p.w.What; aq.G = p.w.F; aq.U = p.w.U; aq.Cc = p.w.Cc;
     aq.own_rows = p.B; aq.oth_rows = p.N; aq.N = p.N; aq.d4 = p.d4; aq.split = p.split_q;
@@ -1230,6 +1245,7 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     stage_end(h, ST_ACCUM_T, s);
     KGE_LAUNCH_CHECK(h);
     if (side) KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_t, 0));
+    }
     stage_begin(h, ST_CHAIN, s);
     {
         const int grid = (row_warps * 32 + 255) / 256 + 1;

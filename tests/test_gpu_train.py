@@ -17,12 +17,20 @@ MODELS = [("transe", 1), ("transe", 2), ("transh", 1), ("transh", 2), ("rotate",
 def _check_step(gpu, orc, step, batch, *, taps=True, rows_atol=2e-6):
     prob = gpu.prob
     B, N, d = prob.B, prob.N, prob.d
-    # tensor-core path: the norm expansion |q|^2 + |t|^2 - 2 q.t cancels in fp32, so distances (and
-    # everything downstream) carry an absolute error of a few 1e-7 / distance; its stated bound is
-    # 2e-2 relative on scores.  The gradient taps get ten times the fp32 path's absolute slack.
-    ga = 2e-4 if prob.tc else 2e-5
+    # tensor-core path: the scores come from bf16-rounded operands (matched by the oracle, so dL/dF
+    # is still compared tightly), and the two backward contractions take dL/dF, q and t rounded
+    # to bf16 (relative error 2^-9 per factor) with fp32 accumulation.  A gradient coordinate is a
+    # sum of signed terms, so its error is bounded relative to the largest gradient, not to itself:
+    # 1e-2 of the largest coordinate for the taps, and lr times 1e-2 of the largest summed
+    # magnitude for the updated rows.  The stated bound of this path is 2e-2 relative on scores.
+    ga = 1e-2 if prob.tc else 2e-5
     if prob.tc:
-        rows_atol = max(rows_atol, 2e-5)
+        g = orc.grads(batch)
+        mag = np.zeros((prob.E, d))
+        np.add.at(mag, batch[0], np.abs(g["dh"])); np.add.at(mag, batch[2], np.abs(g["dtpos"]))
+        np.add.at(mag, batch[3], np.abs(g["dtneg"]))
+        rmag = np.zeros((prob.R, g["dr"].shape[1])); np.add.at(rmag, batch[1], np.abs(g["dr"]))
+        rows_atol = 1e-2 * prob.lr * max(mag.max(), rmag.max())
     dev = [gpu.dev_i32(a) for a in batch]
     loss_dev = gpu.torch.zeros(1, dtype=gpu.torch.float32, device=gpu.ent.device)
     want = orc.grads(batch) if taps else None
