@@ -42,6 +42,19 @@ WORKLOADS = {
     "c2_rotate_l1": dict(E=100_000, R=500, T=2_000_000, d=128, score="rotate", p_norm=1, loss="logsigmoid",
                          opt="sgd", B=1024, N=1024, P=4, gamma=12.0, adv_temp=1.0, lr=0.05,
                          entity_zipf=1.1, relation_zipf=1.0, graph_seed=1),
+    # BASELINE configs[2]: 10,000,000 entities, 1,000 relations (Zipf 1.0), 100,000,000 Zipf(1.1) triples,
+    # d = 256, sampled-softmax loss with the paper's correction, B = 4,096 x N = 16,384, P = 8, Adam on
+    # touched rows, bf16 tensor-core score block.  Tables are drawn on the device (10 GB + 20 GB of state).
+    "c3_distmult": dict(E=10_000_000, R=1000, T=100_000_000, d=256, score="distmult", p_norm=1, loss="softmax",
+                        opt="adam", B=4096, N=16384, P=8, gamma=0.0, adv_temp=0.0, lr=0.001, tc=True,
+                        ce_correction="paper", entity_zipf=1.1, relation_zipf=1.0, graph_seed=2, device_tables=True),
+    "c3_complex": dict(E=10_000_000, R=1000, T=100_000_000, d=256, score="complex", p_norm=1, loss="softmax",
+                       opt="adam", B=4096, N=16384, P=8, gamma=0.0, adv_temp=0.0, lr=0.001, tc=True,
+                       ce_correction="paper", entity_zipf=1.1, relation_zipf=1.0, graph_seed=2, device_tables=True),
+    # a tenth of configs[2]'s graph and table with the same batch shape: quick runs of the tensor-core step
+    "c3s_distmult": dict(E=1_000_000, R=1000, T=10_000_000, d=256, score="distmult", p_norm=1, loss="softmax",
+                         opt="adam", B=4096, N=16384, P=8, gamma=0.0, adv_temp=0.0, lr=0.001, tc=True,
+                         ce_correction="paper", entity_zipf=1.1, relation_zipf=1.0, graph_seed=2, device_tables=True),
     "c1_distmult": dict(E=1000, R=10, T=20_000, d=32, score="distmult", p_norm=1, loss="logsigmoid",
                         opt="sgd", B=64, N=128, P=2, gamma=0.0, adv_temp=0.0, lr=0.1,
                         entity_zipf=1.1, relation_zipf=0.0, graph_seed=0),
@@ -61,9 +74,12 @@ STAGE_OPS = {
 
 
 def cfg_kwargs(w, seed):
+    c = w.get("ce_correction", 0.0)
+    if c == "paper":                       # c = log((|E| - 1) / N), Section 3.1 "Loss Functions"
+        c = float(np.log((w["E"] - 1) / w["N"]))
     return dict(num_entities=w["E"], num_relations=w["R"], dim=w["d"], score=w["score"], p_norm=w["p_norm"],
                 loss=w["loss"], opt=w["opt"], batch=w["B"], num_neg=w["N"], num_parts=w["P"], gamma=w["gamma"],
-                adv_temp=w["adv_temp"], lr=w["lr"], seed=seed)
+                adv_temp=w["adv_temp"], ce_correction=c, lr=w["lr"], seed=seed)
 
 
 class ClockSampler:
@@ -190,11 +206,30 @@ def run_ours(args, w, name):
     B, N = w["B"], w["N"]
     h, r, t = kge_synth.make_graph(w["E"], w["R"], w["T"], seed=w["graph_seed"], entity_zipf=w["entity_zipf"],
                                    relation_zipf=w["relation_zipf"])
-    ent, rel, relw = kge_synth.make_tables(w["E"], w["R"], w["d"], w["score"], seed=w["graph_seed"])
-    ent_d, rel_d = torch.from_numpy(ent).to(dev), torch.from_numpy(rel).to(dev)
-    relw_d = None if relw is None else torch.from_numpy(relw).to(dev)
-    kge = K.Kge(K.KgeConfig.make(**cfg_kwargs(w, seed=rank)))       # each replica draws its own batches
-    kge.bind(ent_d, rel_d, relw_d, num_triples=w["T"])
+    kw_rel = w["d"] // 2 if w["score"] == "rotate" else w["d"]
+    if w.get("device_tables"):
+        # large tables are drawn on the device with the same law (N(0, 1/sqrt(d)) rows)
+        gen = torch.Generator(device=dev); gen.manual_seed(w["graph_seed"] + 1_000_003)
+        ent_d = torch.empty((w["E"], w["d"]), dtype=torch.float32, device=dev).normal_(0.0, w["d"] ** -0.5, generator=gen)
+        rel_d = torch.empty((w["R"], kw_rel), dtype=torch.float32, device=dev).normal_(0.0, w["d"] ** -0.5, generator=gen)
+        relw_d = None
+        if w["score"] == "transh":
+            relw_d = torch.empty((w["R"], w["d"]), dtype=torch.float32, device=dev).normal_(0.0, w["d"] ** -0.5, generator=gen)
+    else:
+        ent, rel, relw = kge_synth.make_tables(w["E"], w["R"], w["d"], w["score"], seed=w["graph_seed"])
+        ent_d, rel_d = torch.from_numpy(ent).to(dev), torch.from_numpy(rel).to(dev)
+        relw_d = None if relw is None else torch.from_numpy(relw).to(dev)
+    states = [None, None, None]
+    if w["opt"] == "adam":
+        states = [torch.zeros((w["E"], 2 * w["d"]), dtype=torch.float32, device=dev),
+                  torch.zeros((w["R"], 2 * kw_rel), dtype=torch.float32, device=dev),
+                  None if relw_d is None else torch.zeros((w["R"], 2 * w["d"]), dtype=torch.float32, device=dev)]
+    elif w["opt"] == "adagrad":
+        states = [torch.zeros(w["E"], dtype=torch.float32, device=dev), torch.zeros(w["R"], dtype=torch.float32, device=dev),
+                  None if relw_d is None else torch.zeros(w["R"], dtype=torch.float32, device=dev)]
+    prec = K.PREC_BF16_TC if w.get("tc") else K.PREC_FP32
+    kge = K.Kge(K.KgeConfig.make(**cfg_kwargs(w, seed=rank), prec=prec))       # each replica draws its own batches
+    kge.bind(ent_d, rel_d, relw_d, *states, num_triples=w["T"])
     kge.graph_load(h, r, t)
     loss = torch.zeros(1, dtype=torch.float32, device=dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # 2 x L2: evicts the tables between steps
@@ -262,7 +297,16 @@ def run_ours(args, w, name):
     compute_stages = [s for s in ("block", "accum_q", "accum_t") if s in per_stage_us]
     dominant = max(compute_stages, key=lambda s: per_stage_us[s])
     roofline = None
-    if dominant in ops:
+    if w.get("tc"):
+        # each of the three contractions is 2 B N d flops; bf16 operands, fp32 accumulation
+        peaks = json.loads((ROOT / "MEASURED_PEAKS.json").read_text()) if (ROOT / "MEASURED_PEAKS.json").exists() else {}
+        peak = peaks.get("bf16_tflops_sustained", 1400.0)
+        achieved = 2.0 * B * N * w["d"] / (per_stage_us[dominant] * 1e-6) / 1e12
+        roofline = {"bound": "tensor", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                    "frac": achieved / peak, "traffic": None,
+                    "peak_source": "measured (sustained cuBLAS bf16)" if peaks else "fallback",
+                    "us_per_launch": per_stage_us[dominant]}
+    elif dominant in ops:
         alg_ops = ops[dominant] * B * N * w["d"]
         achieved = alg_ops / (per_stage_us[dominant] * 1e-6) / 1e12
         roofline = {"bound": "alu", "kernel": dominant, "achieved": achieved, "peak": ALU_PEAK_TOPS,
@@ -272,7 +316,7 @@ def run_ours(args, w, name):
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "vs_baseline": None, "dtype": "bf16" if w.get("tc") else "f32", "data": "synthetic",
             "config": {"workload": name, "entities": w["E"], "relations": w["R"], "triples": w["T"], "dim": w["d"],
                        "batch": B, "num_neg": N, "parts": w["P"], "score": w["score"], "p_norm": w["p_norm"],
                        "loss": w["loss"], "opt": w["opt"], "replicas": world,
