@@ -34,12 +34,13 @@ int pick_split(int rows, int cols, int num_sms) {
     return std::max(1, (cols + per - 1) / per);
 }
 
-// Tensor-core contraction [rows, cols] over `depth`: enough K splits to give every SM a tile,
-// each split at least four 64-wide slices deep, at most 16, none empty.
+// Tensor-core contraction [rows, cols] over `depth` on persistent CTAs (one per SM): as many K
+// splits as still give every SM at most one tile (or one split when there are more tiles than
+// SMs), each at least four 64-wide slices deep, at most 16, none empty.
 int pick_split_tc(int rows, int cols, int depth, int num_sms) {
     const int tiles = ((rows + 127) / 128) * ((cols + 127) / 128);
     const int kb = (depth + 63) / 64;
-    const int want = std::max(1, std::min(std::min((num_sms + tiles - 1) / tiles, std::max(1, kb / 4)), 16));
+    const int want = std::max(1, std::min(std::min(num_sms / tiles, std::max(1, kb / 4)), 16));
     const int per = (kb + want - 1) / want;
     return (kb + per - 1) / per;
 }

@@ -3,10 +3,11 @@
 //
 //   C[M, N] = A[M, K] . B[N, K]^T      A, B bf16, K contiguous; fp32 accumulation
 //
-// One CTA computes one 128 x 128 tile of C.  Warp 0 feeds a ring of shared-memory stages with
-// TMA (one elected lane), warp 1 issues the MMAs (one elected lane) and owns the tensor-memory
-// allocation, warps 2-5 read the finished accumulator out of tensor memory (each warp may
-// only touch the 32 lanes of its own quarter) and apply the epilogue:
+// Persistent CTAs (one per SM) each walk a run of 128 x 128 output tiles.  Warp 0 feeds a ring of
+// shared-memory stages with TMA (one elected lane), warp 1 issues the MMAs (one elected lane)
+// into one of two accumulators in tensor memory and owns the allocation, warps 2-9 drain the
+// other accumulator meanwhile (a warp may only touch the 32 lanes of its own quarter; two warps
+// share a quarter, 64 columns each) and apply the epilogue:
 //   EPI_STORE   F = acc                                   DistMult / ComplEx (scoring-function table)
 //   EPI_L2DIST  F = -sqrt(max(|q|^2 + |t|^2 - 2 acc, 0))  TransE with p = 2 by the norm expansion
 // Every wait on a barrier is bounded; a wait that runs out records KGE_ERR_TIMEOUT, tells the
@@ -23,18 +24,20 @@ namespace kge {
 namespace {
 
 constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 64;      // BK bf16 = one 128-byte swizzle row
-constexpr int TC_STAGES = 3;
-constexpr int TC_THREADS = 192;
+constexpr int TC_STAGES = 4;
+constexpr int TC_EPI_WARPS = 8;                           // two per tensor-memory lane quarter, 64 columns each
+constexpr int TC_THREADS = 32 * (2 + TC_EPI_WARPS);
 constexpr uint32_t TC_A_BYTES = TC_BM * TC_BK * 2, TC_B_BYTES = TC_BN * TC_BK * 2;
 constexpr uint32_t TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
 constexpr size_t TC_SMEM_BYTES = 1024 + (size_t)TC_STAGES * TC_STAGE_BYTES + 128;
-constexpr uint32_t TC_TMEM_COLS = 128;                    // fp32 accumulator: one column per element of a row
+constexpr uint32_t TC_TMEM_COLS = 256;                    // two fp32 accumulators of 128 columns, used in turn
 
 enum { EPI_STORE = 0, EPI_L2DIST = 1 };
 
 struct TcGemmParams {
     int M, N, K;
-    int kb_per_split;                     // 64-wide slices of K per blockIdx.z
+    int kb_per_split;                     // 64-wide slices of K per split
+    int tiles_m, tiles_n, items;          // items = splits * tiles_m * tiles_n
     float* C; int64_t ldc;
     int64_t split_stride;                 // floats between the output slabs of consecutive K splits
     const float *row_norm2, *col_norm2;   // EPI_L2DIST: |q_b|^2 [M], |t_n|^2 [N]
@@ -93,6 +96,47 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+struct TcItem { int z, m0, n0; };   // K split, first row, first column
+
+// Epilogue of one warp on one item: 64 columns [col_off, col_off + 64) of the tile row held by
+// this thread's tensor-memory lane (taddr points at the first of them).
+template <int EPI>
+__device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr) {
+    float* const Cout = p.C + (int64_t)it.z * p.split_stride;
+    float rn = 0.f;
+    if (EPI == EPI_L2DIST && row < p.M) rn = p.row_norm2[row];
+#pragma unroll 1
+    for (int c0 = col_off; c0 < col_off + 64; c0 += 32) {
+        float v[32];
+        tmem_ld32(taddr + (uint32_t)(c0 - col_off), v);
+        if (row >= p.M) continue;
+        const int ncol = it.n0 + c0;
+        float* dst = Cout + (int64_t)row * p.ldc + ncol;
+        if (EPI == EPI_L2DIST) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float d2 = rn + (ncol + i < p.N ? p.col_norm2[ncol + i] : 0.f) - 2.f * v[i];
+                v[i] = -sqrtf(fmaxf(d2, 0.f));
+            }
+        }
+        if (ncol + 32 <= p.N && (p.ldc & 3) == 0) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+                *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) if (ncol + i < p.N) dst[i] = v[i];
+        }
+    }
+}
+
+// Work item = (K split, row tile, column tile), column tile fastest.  A CTA takes a contiguous
+// run of items, so consecutive items mostly share their A rows (kept warm in L2).
+__device__ __forceinline__ TcItem tc_item(const TcGemmParams& p, int item) {
+    const int tn = item % p.tiles_n, r = item / p.tiles_n;
+    return TcItem{r / p.tiles_m, (r % p.tiles_m) * TC_BM, tn * TC_BN};
+}
+
 template <int EPI>
 __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
                                                              const __grid_constant__ CUtensorMap tmB, TcGemmParams p) {
@@ -100,101 +144,95 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
     unsigned char* base = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
     uint64_t* full = reinterpret_cast<uint64_t*>(base + (size_t)TC_STAGES * TC_STAGE_BYTES);
     uint64_t* empty = full + TC_STAGES;
-    uint64_t* accum_full = empty + TC_STAGES;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum_full + 1);
-    volatile uint32_t* stop = tmem_slot + 1;    // set by a warp whose wait ran out
+    uint64_t* acc_full = empty + TC_STAGES;      // [2] accumulator buffer written
+    uint64_t* acc_empty = acc_full + 2;          // [2] accumulator buffer drained by all epilogue warps
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    volatile uint32_t* stop = tmem_slot + 1;     // set by a warp whose wait ran out
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.y * TC_BM, n0 = blockIdx.x * TC_BN;
-    const int kb_begin = blockIdx.z * p.kb_per_split;
-    const int nkb = min(p.kb_per_split, (p.K + TC_BK - 1) / TC_BK - kb_begin);   // >= 1 by the launch geometry
-    float* const Cout = p.C + (int64_t)blockIdx.z * p.split_stride;
+    const int per_cta = (p.items + gridDim.x - 1) / gridDim.x;
+    const int item_begin = blockIdx.x * per_cta, item_end = min(p.items, item_begin + per_cta);
+    const int kb_total = (p.K + TC_BK - 1) / TC_BK;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < TC_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        mbar_init(accum_full, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], TC_EPI_WARPS); }
         *stop = 0;
         mbar_init_fence();
     }
-    if (warp == 1) {   // one warp allocates the accumulator columns and gives up the right to allocate more
+    if (warp == 1) {   // one warp allocates both accumulator buffers and gives up the right to allocate more
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TC_TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_acc = *tmem_slot;
+    const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int kb = 0; kb < nkb && !*stop; ++kb) {
-                const int s = kb % TC_STAGES;
-                if (!mbar_wait_bounded(&empty[s], ((kb / TC_STAGES) & 1) ^ 1)) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); break; }
-                unsigned char* sa = base + (size_t)s * TC_STAGE_BYTES;
-                mbar_arrive_expect_tx(&full[s], TC_STAGE_BYTES);
-                tma_load_2d(sa, &tmA, (kb_begin + kb) * TC_BK, m0, &full[s]);
-                tma_load_2d(sa + TC_A_BYTES, &tmB, (kb_begin + kb) * TC_BK, n0, &full[s]);
+            int ring = 0;    // slices issued so far: stage = ring % STAGES, phase = ring / STAGES
+            for (int item = item_begin; item < item_end && !*stop; ++item) {
+                const TcItem it = tc_item(p, item);
+                const int kb0 = it.z * p.kb_per_split, nkb = min(p.kb_per_split, kb_total - kb0);
+                for (int kb = 0; kb < nkb; ++kb, ++ring) {
+                    const int s = ring % TC_STAGES;
+                    if (!mbar_wait_bounded(&empty[s], ((ring / TC_STAGES) & 1) ^ 1)) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); break; }
+                    unsigned char* sa = base + (size_t)s * TC_STAGE_BYTES;
+                    mbar_arrive_expect_tx(&full[s], TC_STAGE_BYTES);
+                    tma_load_2d(sa, &tmA, (kb0 + kb) * TC_BK, it.m0, &full[s]);
+                    tma_load_2d(sa + TC_A_BYTES, &tmB, (kb0 + kb) * TC_BK, it.n0, &full[s]);
+                }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(TC_BM, TC_BN);
+            int ring = 0;
             bool ok = true;
-            for (int kb = 0; kb < nkb && !*stop; ++kb) {
-                const int s = kb % TC_STAGES;
-                if (!mbar_wait_bounded(&full[s], (kb / TC_STAGES) & 1)) { ok = false; break; }
+            for (int item = item_begin, local = 0; item < item_end && ok && !*stop; ++item, ++local) {
+                const TcItem it = tc_item(p, item);
+                const int nkb = min(p.kb_per_split, kb_total - it.z * p.kb_per_split);
+                const int buf = local & 1;
+                // the epilogue warps must have drained this buffer (two items ago)
+                if (!mbar_wait_bounded(&acc_empty[buf], ((local >> 1) & 1) ^ 1)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t sa = smem_u32(base + (size_t)s * TC_STAGE_BYTES);
+                const uint32_t tmem_acc = tmem_base + (uint32_t)buf * TC_BN;
+                for (int kb = 0; kb < nkb; ++kb, ++ring) {
+                    const int s = ring % TC_STAGES;
+                    if (!mbar_wait_bounded(&full[s], (ring / TC_STAGES) & 1)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(base + (size_t)s * TC_STAGE_BYTES);
 #pragma unroll
-                for (int k = 0; k < TC_BK / 16; ++k) {   // one MMA covers 16 bf16 = 32 bytes of K
-                    umma_bf16(tmem_acc, umma_desc_k_sw128(sa + k * 32), umma_desc_k_sw128(sa + TC_A_BYTES + k * 32),
-                              idesc, (kb | k) != 0);
+                    for (int k = 0; k < TC_BK / 16; ++k)   // one MMA covers 16 bf16 = 32 bytes of K
+                        umma_bf16(tmem_acc, umma_desc_k_sw128(sa + k * 32), umma_desc_k_sw128(sa + TC_A_BYTES + k * 32),
+                                  idesc, (kb | k) != 0);
+                    umma_commit(&empty[s]);            // the stage is free once these MMAs have read it
                 }
-                umma_commit(&empty[s]);            // the stage is free once these MMAs have read it
+                umma_commit(&acc_full[buf]);           // also after a failed wait, so the epilogue warps wake up
             }
             if (!ok) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); }
-            umma_commit(accum_full);               // also on failure, so the epilogue warps do not wait in vain
         }
     } else {
-        const bool ok = mbar_wait_bounded(accum_full, 0);
-        tc_fence_after();
-        if (ok && !*stop) {
-            const int quarter = warp & 3;          // tensor-memory lanes this warp may read
-            const int row = m0 + quarter * 32 + lane;
-            float rn = 0.f;
-            if (EPI == EPI_L2DIST && row < p.M) rn = p.row_norm2[row];
-#pragma unroll 1
-            for (int c0 = 0; c0 < TC_BN; c0 += 32) {
-                float v[32];
-                tmem_ld32(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
-                if (row < p.M) {
-                    float* dst = Cout + (int64_t)row * p.ldc + n0 + c0;
-                    if (EPI == EPI_L2DIST) {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const int col = n0 + c0 + i;
-                            const float d2 = rn + (col < p.N ? p.col_norm2[col] : 0.f) - 2.f * v[i];
-                            v[i] = -sqrtf(fmaxf(d2, 0.f));
-                        }
-                    }
-                    if (n0 + c0 + 32 <= p.N && (p.ldc & 3) == 0) {
-#pragma unroll
-                        for (int i = 0; i < 32; i += 4)
-                            *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) if (n0 + c0 + i < p.N) dst[i] = v[i];
-                    }
-                }
-            }
-        } else if (!ok && lane == 0) {
-            *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT);
+        const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
+        const int chalf = (warp - 2) >> 2;             // which 64 of the 128 columns
+        for (int item = item_begin, local = 0; item < item_end; ++item, ++local) {
+            const int buf = local & 1;
+            const bool ok = mbar_wait_bounded(&acc_full[buf], (local >> 1) & 1);
+            tc_fence_after();
+            if (!ok || *stop) { if (lane == 0) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); } break; }
+            const TcItem it = tc_item(p, item);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * TC_BN + chalf * 64);
+            tc_epilogue<EPI>(p, it, it.m0 + quarter * 32 + lane, chalf * 64, taddr);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);
         }
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 1)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(TC_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
 }
 
 // src fp32 [R, C] (leading dimension lds) -> bf16 copies for the backward contractions:
@@ -293,6 +331,7 @@ int launch_tc_scores(kge_handle* h, cudaStream_t s) {
     TcGemmParams p;
     p.M = c.batch; p.N = c.num_neg; p.K = c.dim;
     p.kb_per_split = (p.K + TC_BK - 1) / TC_BK; p.split_stride = 0;
+    p.tiles_m = (p.M + TC_BM - 1) / TC_BM; p.tiles_n = (p.N + TC_BN - 1) / TC_BN; p.items = p.tiles_m * p.tiles_n;
     p.C = h->ws.F; p.ldc = c.num_neg;
     p.row_norm2 = h->ws.qn2; p.col_norm2 = h->ws.tn2;
     p.status = h->ws.status;
@@ -302,7 +341,7 @@ int launch_tc_scores(kge_handle* h, cudaStream_t s) {
         KGE_CUDA_CHECK(h, cudaFuncSetAttribute(tc_gemm_kernel<EPI_L2DIST>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES));
         configured = true;
     }
-    const dim3 grid((p.N + TC_BN - 1) / TC_BN, (p.M + TC_BM - 1) / TC_BM);
+    const dim3 grid(std::min(p.items, h->num_sms));
     const CUtensorMap& tq = *reinterpret_cast<const CUtensorMap*>(h->tm_q);
     const CUtensorMap& tt = *reinterpret_cast<const CUtensorMap*>(h->tm_t);
     if (h->kind == KIND_L2) tc_gemm_kernel<EPI_L2DIST><<<grid, TC_THREADS, TC_SMEM_BYTES, s>>>(tq, tt, p);
@@ -337,7 +376,9 @@ int launch_tc_gemm(kge_handle* h, const unsigned char* tmA, const unsigned char*
     p.C = C; p.ldc = ldc; p.split_stride = (int64_t)M * ldc;
     p.row_norm2 = p.col_norm2 = nullptr;
     p.status = h->ws.status;
-    const dim3 grid((N + TC_BN - 1) / TC_BN, (M + TC_BM - 1) / TC_BM, (kb + p.kb_per_split - 1) / p.kb_per_split);
+    p.tiles_m = (M + TC_BM - 1) / TC_BM; p.tiles_n = (N + TC_BN - 1) / TC_BN;
+    p.items = p.tiles_m * p.tiles_n * ((kb + p.kb_per_split - 1) / p.kb_per_split);
+    const dim3 grid(std::min(p.items, h->num_sms));
     tc_gemm_kernel<EPI_STORE><<<grid, TC_THREADS, TC_SMEM_BYTES, s>>>(*reinterpret_cast<const CUtensorMap*>(tmA),
                                                                        *reinterpret_cast<const CUtensorMap*>(tmB), p);
     KGE_LAUNCH_CHECK(h);
