@@ -10,6 +10,10 @@
 // share a quarter, 64 columns each) and apply the epilogue:
 //   EPI_STORE   F = acc                                   DistMult / ComplEx (scoring-function table)
 //   EPI_L2DIST  F = -sqrt(max(|q|^2 + |t|^2 - 2 acc, 0))  TransE with p = 2 by the norm expansion
+//   EPI_STATS   no score leaves the chip: per row and 64-column piece the running maximum, the sum
+//               of exponentials and the weighted loss sum of Section 3.1 "Loss Functions"
+//   EPI_GRAD    scores recomputed, dL/dF formed from the finished row statistics and written as
+//               bf16 in both orientations for the two backward contractions
 // Every wait on a barrier is bounded; a wait that runs out records KGE_ERR_TIMEOUT, tells the
 // other warps to stop, and the CTA still releases its tensor memory before it returns.
 #include <cuda.h>
@@ -32,7 +36,7 @@ constexpr uint32_t TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
 constexpr size_t TC_SMEM_BYTES = 1024 + (size_t)TC_STAGES * TC_STAGE_BYTES + 128;
 constexpr uint32_t TC_TMEM_COLS = 256;                    // two fp32 accumulators of 128 columns, used in turn
 
-enum { EPI_STORE = 0, EPI_L2DIST = 1 };
+enum { EPI_STORE = 0, EPI_L2DIST = 1, EPI_STATS = 2, EPI_GRAD = 3 };
 
 struct TcGemmParams {
     int M, N, K;
@@ -40,8 +44,17 @@ struct TcGemmParams {
     int tiles_m, tiles_n, items;          // items = splits * tiles_m * tiles_n
     float* C; int64_t ldc;
     int64_t split_stride;                 // floats between the output slabs of consecutive K splits
-    const float *row_norm2, *col_norm2;   // EPI_L2DIST: |q_b|^2 [M], |t_n|^2 [N]
+    const float *row_norm2, *col_norm2;   // norm expansion: |q_b|^2 [M], |t_n|^2 [N]
     int32_t* status;
+    // fused loss epilogues (EPI_STATS, EPI_GRAD): the score is acc, or for l2 != 0 the distance score above
+    int l2, loss;
+    float gamma, adv_temp, ce_c, loss_scale;
+    float4* stat_part;                    // [M, 2 * tiles_n] per 64-column piece: (max, sum exp, weighted loss sum, -)
+    const float2* row_stat;               // [M] (max, 1 / normaliser) of the whole row
+    uint16_t* Gb; int64_t ldg;            // [M, ldg] bf16 dL/dF (divided by the distance for l2)
+    uint16_t* GbT; int64_t ldgt;          // [N, ldgt] its transpose
+    float* grow_part;                     // [M, 2 * tiles_n] sums of the written values per 64-column piece
+    float* gcol_part;                     // [4 * tiles_m, N] sums per 32-row piece (l2 only)
 };
 
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
@@ -98,10 +111,128 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 
 struct TcItem { int z, m0, n0; };   // K split, first row, first column
 
+// softplus(z) and sigmoid(z) from one exponential.
+__device__ __forceinline__ void tc_softplus_sigmoid(float z, float& sp, float& sg) {
+    const float e = expf(-fabsf(z));
+    sp = fmaxf(z, 0.f) + log1pf(e);
+    const float r = 1.f / (1.f + e);
+    sg = z >= 0.f ? r : e * r;
+}
+
+// Score of a pair from the accumulator: the contraction itself, or the distance score of the
+// norm expansion.
+__device__ __forceinline__ float tc_score(const TcGemmParams& p, float acc, float rn, int col) {
+    if (!p.l2) return acc;
+    return -sqrtf(fmaxf(rn + p.col_norm2[col] - 2.f * acc, 0.f));
+}
+
+// First pass of the fused loss: running (max, sum of exponentials, exponentially weighted loss
+// sum) over this thread's 64 columns of one row, rescaled whenever the maximum moves.
+// x = a f for the self-adversarial weights, x = f + c for the sampled softmax.
+__device__ __forceinline__ void tc_epilogue_stats(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr) {
+    const bool ce = p.loss == KGE_LOSS_SAMPLED_SOFTMAX;
+    const float rn = (p.l2 && row < p.M) ? p.row_norm2[row] : 0.f;
+    float m = -INFINITY, z = 0.f, l = 0.f;
+#pragma unroll 1
+    for (int c0 = col_off; c0 < col_off + 64; c0 += 32) {
+        float v[32];
+        tmem_ld32(taddr + (uint32_t)(c0 - col_off), v);
+        if (row >= p.M) continue;
+        const int ncol = it.n0 + c0;
+        float cm = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            if (ncol + i < p.N) {
+                v[i] = tc_score(p, v[i], rn, ncol + i);
+                cm = fmaxf(cm, ce ? v[i] + p.ce_c : p.adv_temp * v[i]);
+            }
+        }
+        if (cm > m) { const float r = expf(m - cm); z *= r; l *= r; m = cm; }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            if (ncol + i < p.N) {
+                const float e = expf((ce ? v[i] + p.ce_c : p.adv_temp * v[i]) - m);
+                z += e;
+                if (!ce) { float sp, sg; tc_softplus_sigmoid(p.gamma + v[i], sp, sg); l += e * sp; }
+            }
+        }
+    }
+    if (row < p.M)
+        p.stat_part[(int64_t)row * (2 * p.tiles_n) + (it.n0 / TC_BN) * 2 + col_off / 64] = make_float4(m, z, l, 0.f);
+}
+
+__device__ __forceinline__ uint16_t bf16_bits(float v) {
+    const __nv_bfloat16 b = __float2bfloat16_rn(v);
+    return *reinterpret_cast<const uint16_t*>(&b);
+}
+__device__ __forceinline__ float bf16_value(uint16_t bits) { return __uint_as_float((uint32_t)bits << 16); }
+
+// Second pass: dL/dF from the recomputed score and the row's final (max, 1 / normaliser),
+// written as bf16 in both orientations for the two backward contractions.
+__device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr) {
+    const bool ce = p.loss == KGE_LOSS_SAMPLED_SOFTMAX;
+    const bool rin = row < p.M;
+    const float rn = (p.l2 && rin) ? p.row_norm2[row] : 0.f;
+    const float2 st = rin ? p.row_stat[row] : make_float2(0.f, 0.f);
+    const int lane = threadIdx.x & 31;
+    float rsum = 0.f;
+#pragma unroll 1
+    for (int c0 = col_off; c0 < col_off + 64; c0 += 32) {
+        float v[32];
+        tmem_ld32(taddr + (uint32_t)(c0 - col_off), v);
+        const int ncol = it.n0 + c0;
+        uint32_t g2[16];     // bf16 pairs in memory order
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            float g = 0.f;
+            if (rin && ncol + i < p.N) {
+                const float f = tc_score(p, v[i], rn, ncol + i);
+                if (ce) {
+                    g = p.loss_scale * expf(f + p.ce_c - st.x) * st.y;
+                } else {
+                    float sp, sg;
+                    tc_softplus_sigmoid(p.gamma + f, sp, sg);
+                    g = p.loss_scale * expf(p.adv_temp * f - st.x) * st.y * sg;
+                }
+                if (p.l2) g = f < 0.f ? g / -f : 0.f;
+            }
+            const uint16_t gb = bf16_bits(g);
+            v[i] = bf16_value(gb);          // the value the contractions will see
+            rsum += v[i];
+            if (i & 1) g2[i >> 1] |= (uint32_t)gb << 16; else g2[i >> 1] = gb;
+        }
+        if (rin) {
+            uint16_t* dst = p.Gb + (int64_t)row * p.ldg + ncol;
+            if (ncol + 32 <= p.N) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    reinterpret_cast<uint4*>(dst)[i] = make_uint4(g2[4 * i], g2[4 * i + 1], g2[4 * i + 2], g2[4 * i + 3]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) if (ncol + i < p.N) dst[i] = (uint16_t)(g2[i >> 1] >> ((i & 1) * 16));
+            }
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (ncol + i < p.N) p.GbT[(int64_t)(ncol + i) * p.ldgt + row] = (uint16_t)(g2[i >> 1] >> ((i & 1) * 16));
+        }
+        if (p.l2) {   // column sums over this warp's 32 rows (rows outside the problem hold zeros)
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float cs = warp_sum(v[i]);
+                if (lane == 0 && ncol + i < p.N)
+                    p.gcol_part[(int64_t)((it.m0 / TC_BM) * 4 + ((row - it.m0) >> 5)) * p.N + ncol + i] = cs;
+            }
+        }
+    }
+    if (rin) p.grow_part[(int64_t)row * (2 * p.tiles_n) + (it.n0 / TC_BN) * 2 + col_off / 64] = rsum;
+}
+
 // Epilogue of one warp on one item: 64 columns [col_off, col_off + 64) of the tile row held by
 // this thread's tensor-memory lane (taddr points at the first of them).
 template <int EPI>
 __device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr) {
+    if (EPI == EPI_STATS) { tc_epilogue_stats(p, it, row, col_off, taddr); return; }
+    if (EPI == EPI_GRAD) { tc_epilogue_grad(p, it, row, col_off, taddr); return; }
     float* const Cout = p.C + (int64_t)it.z * p.split_stride;
     float rn = 0.f;
     if (EPI == EPI_L2DIST && row < p.M) rn = p.row_norm2[row];
@@ -246,11 +377,6 @@ struct CastParams {
     uint16_t* dst_t; int64_t ld_t;
     float* colsum;
 };
-
-__device__ __forceinline__ uint16_t bf16_bits(float v) {
-    const __nv_bfloat16 b = __float2bfloat16_rn(v);
-    return *reinterpret_cast<const uint16_t*>(&b);
-}
 
 __global__ void __launch_bounds__(256) cast_transpose_kernel(CastParams p) {
     __shared__ float tile[32][33];
