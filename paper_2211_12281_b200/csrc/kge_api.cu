@@ -75,6 +75,11 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
     w.TbT = tc ? cv.take<uint16_t>(d * ldN) : nullptr;
     w.QbT = tc ? cv.take<uint16_t>(d * ldB) : nullptr;
     w.Gcol = tc ? cv.take<float>(N) : nullptr;
+    const size_t tiles_n = (N + 127) / 128, tiles_m = (B + 127) / 128;
+    w.stat_part = tc ? cv.take<float>(B * 2 * tiles_n * 4) : nullptr;
+    w.row_stat = tc ? cv.take<float>(B * 2) : nullptr;
+    w.grow_part = tc ? cv.take<float>(B * 2 * tiles_n) : nullptr;
+    w.gcol_part = tc ? cv.take<float>(4 * tiles_m * N) : nullptr;
     w.Grow = cv.take<float>(B);
     w.Cpart = cv.take<float>((size_t)h->split_t * N);
     w.F = cv.take<float>(B * N);
@@ -503,6 +508,20 @@ int kge_debug_export(kge_handle* h, int tap, void* dst, size_t bytes, void* stre
         default: return KGE_ERR_BAD_ARG;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (tap == KGE_TAP_G && h->cfg.prec == KGE_PREC_BF16_TC) {
+        // the tensor-core path keeps dL/dF only as bf16 [B, ldN]: widen it on the host
+        const size_t B = h->cfg.batch, N = h->cfg.num_neg, ldN = (N + 7) / 8 * 8;
+        std::vector<uint16_t> tmp(B * ldN);
+        KGE_CUDA_CHECK(h, cudaMemcpyAsync(tmp.data(), w.Gb, tmp.size() * 2, cudaMemcpyDeviceToHost, s));
+        KGE_CUDA_CHECK(h, cudaStreamSynchronize(s));
+        float* out = static_cast<float*>(dst);
+        for (size_t b = 0; b < B; ++b)
+            for (size_t n = 0; n < N; ++n) {
+                const uint32_t bits = (uint32_t)tmp[b * ldN + n] << 16;
+                std::memcpy(&out[b * N + n], &bits, 4);
+            }
+        return KGE_OK;
+    }
     KGE_CUDA_CHECK(h, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, s));
     KGE_CUDA_CHECK(h, cudaStreamSynchronize(s));
     return KGE_OK;

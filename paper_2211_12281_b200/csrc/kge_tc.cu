@@ -8,10 +8,11 @@
 // into one of two accumulators in tensor memory and owns the allocation, warps 2-9 drain the
 // other accumulator meanwhile (a warp may only touch the 32 lanes of its own quarter; two warps
 // share a quarter, 64 columns each) and apply the epilogue:
-//   EPI_STORE   F = acc                                   DistMult / ComplEx (scoring-function table)
-//   EPI_L2DIST  F = -sqrt(max(|q|^2 + |t|^2 - 2 acc, 0))  TransE with p = 2 by the norm expansion
+//   EPI_STORE   C = acc (the backward contractions)
 //   EPI_STATS   no score leaves the chip: per row and 64-column piece the running maximum, the sum
-//               of exponentials and the weighted loss sum of Section 3.1 "Loss Functions"
+//               of exponentials and the weighted loss sum of Section 3.1 "Loss Functions"; the
+//               score is the contraction (DistMult, ComplEx) or, for TransE with p = 2, the
+//               norm expansion -sqrt(max(|q|^2 + |t|^2 - 2 acc, 0))
 //   EPI_GRAD    scores recomputed, dL/dF formed from the finished row statistics and written as
 //               bf16 in both orientations for the two backward contractions
 // Every wait on a barrier is bounded; a wait that runs out records KGE_ERR_TIMEOUT, tells the
@@ -36,7 +37,7 @@ constexpr uint32_t TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
 constexpr size_t TC_SMEM_BYTES = 1024 + (size_t)TC_STAGES * TC_STAGE_BYTES + 128;
 constexpr uint32_t TC_TMEM_COLS = 256;                    // two fp32 accumulators of 128 columns, used in turn
 
-enum { EPI_STORE = 0, EPI_L2DIST = 1, EPI_STATS = 2, EPI_GRAD = 3 };
+enum { EPI_STORE = 0, EPI_STATS = 1, EPI_GRAD = 2, EPI_L2 = 4, EPI_CE = 8 };   // L2 / CE: flags of the fused epilogues
 
 struct TcGemmParams {
     int M, N, K;
@@ -119,19 +120,25 @@ __device__ __forceinline__ void tc_softplus_sigmoid(float z, float& sp, float& s
     sg = z >= 0.f ? r : e * r;
 }
 
-// Score of a pair from the accumulator: the contraction itself, or the distance score of the
-// norm expansion.
+// Score of a pair from the accumulator: the contraction itself, or (L2) the distance score of
+// the norm expansion.
+template <bool L2>
 __device__ __forceinline__ float tc_score(const TcGemmParams& p, float acc, float rn, int col) {
-    if (!p.l2) return acc;
+    if (!L2) return acc;
     return -sqrtf(fmaxf(rn + p.col_norm2[col] - 2.f * acc, 0.f));
 }
 
+constexpr float kLog2e = 1.4426950408889634f;
+__device__ __forceinline__ float fast_exp2(float y) { float r; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(y)); return r; }
+
 // First pass of the fused loss: running (max, sum of exponentials, exponentially weighted loss
-// sum) over this thread's 64 columns of one row, rescaled whenever the maximum moves.
-// x = a f for the self-adversarial weights, x = f + c for the sampled softmax.
+// sum) over this thread's 64 columns of one row, rescaled whenever the maximum moves.  The
+// exponent is x = a f for the self-adversarial weights and x = f + c for the sampled softmax;
+// it is carried in base 2 (y = x log2 e), so an exponential is one ex2 of a difference.
+template <bool L2, bool CE>
 __device__ __forceinline__ void tc_epilogue_stats(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr) {
-    const bool ce = p.loss == KGE_LOSS_SAMPLED_SOFTMAX;
-    const float rn = (p.l2 && row < p.M) ? p.row_norm2[row] : 0.f;
+    const float rn = (L2 && row < p.M) ? p.row_norm2[row] : 0.f;
+    const float k1 = CE ? kLog2e : p.adv_temp * kLog2e, k0 = CE ? p.ce_c * kLog2e : 0.f;
     float m = -INFINITY, z = 0.f, l = 0.f;
 #pragma unroll 1
     for (int c0 = col_off; c0 < col_off + 64; c0 += 32) {
@@ -139,22 +146,21 @@ __device__ __forceinline__ void tc_epilogue_stats(const TcGemmParams& p, const T
         tmem_ld32(taddr + (uint32_t)(c0 - col_off), v);
         if (row >= p.M) continue;
         const int ncol = it.n0 + c0;
+        const int valid = min(32, p.N - ncol);     // columns of this chunk inside the problem (may be <= 0)
         float cm = -INFINITY;
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-            if (ncol + i < p.N) {
-                v[i] = tc_score(p, v[i], rn, ncol + i);
-                cm = fmaxf(cm, ce ? v[i] + p.ce_c : p.adv_temp * v[i]);
-            }
+            if (L2 || !CE) v[i] = (valid == 32 || i < valid) ? tc_score<L2>(p, v[i], rn, ncol + i) : 0.f;
+            const float y = fmaf(v[i], k1, k0);
+            cm = fmaxf(cm, (valid == 32 || i < valid) ? y : -INFINITY);
         }
-        if (cm > m) { const float r = expf(m - cm); z *= r; l *= r; m = cm; }
+        if (cm > m) { const float r = fast_exp2(m - cm); z *= r; l *= r; m = cm; }
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-            if (ncol + i < p.N) {
-                const float e = expf((ce ? v[i] + p.ce_c : p.adv_temp * v[i]) - m);
-                z += e;
-                if (!ce) { float sp, sg; tc_softplus_sigmoid(p.gamma + v[i], sp, sg); l += e * sp; }
-            }
+            float e = fast_exp2(fmaf(v[i], k1, k0) - m);
+            if (valid != 32 && i >= valid) e = 0.f;
+            z += e;
+            if (!CE) { float sp, sg; tc_softplus_sigmoid(p.gamma + v[i], sp, sg); l = fmaf(e, sp, l); }
         }
     }
     if (row < p.M)
@@ -167,13 +173,15 @@ __device__ __forceinline__ uint16_t bf16_bits(float v) {
 }
 __device__ __forceinline__ float bf16_value(uint16_t bits) { return __uint_as_float((uint32_t)bits << 16); }
 
-// Second pass: dL/dF from the recomputed score and the row's final (max, 1 / normaliser),
+// Second pass: dL/dF from the recomputed score and the row's final (base-2 max, 1 / normaliser),
 // written as bf16 in both orientations for the two backward contractions.
+template <bool L2, bool CE>
 __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr) {
-    const bool ce = p.loss == KGE_LOSS_SAMPLED_SOFTMAX;
     const bool rin = row < p.M;
-    const float rn = (p.l2 && rin) ? p.row_norm2[row] : 0.f;
+    const float rn = (L2 && rin) ? p.row_norm2[row] : 0.f;
     const float2 st = rin ? p.row_stat[row] : make_float2(0.f, 0.f);
+    const float k1 = CE ? kLog2e : p.adv_temp * kLog2e, k0 = (CE ? p.ce_c * kLog2e : 0.f) - st.x;
+    const float scale = p.loss_scale * st.y;
     const int lane = threadIdx.x & 31;
     float rsum = 0.f;
 #pragma unroll 1
@@ -181,61 +189,60 @@ __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const Tc
         float v[32];
         tmem_ld32(taddr + (uint32_t)(c0 - col_off), v);
         const int ncol = it.n0 + c0;
+        const int valid = rin ? min(32, p.N - ncol) : 0;
         uint32_t g2[16];     // bf16 pairs in memory order
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
             float g = 0.f;
-            if (rin && ncol + i < p.N) {
-                const float f = tc_score(p, v[i], rn, ncol + i);
-                if (ce) {
-                    g = p.loss_scale * expf(f + p.ce_c - st.x) * st.y;
-                } else {
-                    float sp, sg;
-                    tc_softplus_sigmoid(p.gamma + f, sp, sg);
-                    g = p.loss_scale * expf(p.adv_temp * f - st.x) * st.y * sg;
-                }
-                if (p.l2) g = f < 0.f ? g / -f : 0.f;
+            if (valid == 32 || i < valid) {
+                const float f = tc_score<L2>(p, v[i], rn, ncol + i);
+                g = scale * fast_exp2(fmaf(f, k1, k0));
+                if (!CE) { float sp, sg; tc_softplus_sigmoid(p.gamma + f, sp, sg); g *= sg; }
+                if (L2) g = f < 0.f ? g / -f : 0.f;
             }
-            const uint16_t gb = bf16_bits(g);
-            v[i] = bf16_value(gb);          // the value the contractions will see
-            rsum += v[i];
-            if (i & 1) g2[i >> 1] |= (uint32_t)gb << 16; else g2[i >> 1] = gb;
+            v[i] = g;
         }
-        if (rin) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const __nv_bfloat162 pr = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+            g2[i] = *reinterpret_cast<const uint32_t*>(&pr);
+        }
+        if (valid > 0) {
             uint16_t* dst = p.Gb + (int64_t)row * p.ldg + ncol;
-            if (ncol + 32 <= p.N) {
+            if (valid == 32) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
                     reinterpret_cast<uint4*>(dst)[i] = make_uint4(g2[4 * i], g2[4 * i + 1], g2[4 * i + 2], g2[4 * i + 3]);
             } else {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) if (ncol + i < p.N) dst[i] = (uint16_t)(g2[i >> 1] >> ((i & 1) * 16));
+                for (int i = 0; i < 32; ++i) if (i < valid) dst[i] = (uint16_t)(g2[i >> 1] >> ((i & 1) * 16));
             }
+            uint16_t* dt = p.GbT + (int64_t)ncol * p.ldgt + row;
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-                if (ncol + i < p.N) p.GbT[(int64_t)(ncol + i) * p.ldgt + row] = (uint16_t)(g2[i >> 1] >> ((i & 1) * 16));
+                if (valid == 32 || i < valid) dt[(int64_t)i * p.ldgt] = (uint16_t)(g2[i >> 1] >> ((i & 1) * 16));
         }
-        if (p.l2) {   // column sums over this warp's 32 rows (rows outside the problem hold zeros)
+        if (L2) {   // the norm expansion also needs the sums of what the contractions will see
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
-                const float cs = warp_sum(v[i]);
+                const float gv = bf16_value((uint16_t)(g2[i >> 1] >> ((i & 1) * 16)));
+                rsum += gv;
+                const float cs = warp_sum(gv);   // over this warp's 32 rows (rows outside the problem hold zeros)
                 if (lane == 0 && ncol + i < p.N)
                     p.gcol_part[(int64_t)((it.m0 / TC_BM) * 4 + ((row - it.m0) >> 5)) * p.N + ncol + i] = cs;
             }
         }
     }
-    if (rin) p.grow_part[(int64_t)row * (2 * p.tiles_n) + (it.n0 / TC_BN) * 2 + col_off / 64] = rsum;
+    if (L2 && rin) p.grow_part[(int64_t)row * (2 * p.tiles_n) + (it.n0 / TC_BN) * 2 + col_off / 64] = rsum;
 }
 
 // Epilogue of one warp on one item: 64 columns [col_off, col_off + 64) of the tile row held by
 // this thread's tensor-memory lane (taddr points at the first of them).
 template <int EPI>
 __device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr) {
-    if (EPI == EPI_STATS) { tc_epilogue_stats(p, it, row, col_off, taddr); return; }
-    if (EPI == EPI_GRAD) { tc_epilogue_grad(p, it, row, col_off, taddr); return; }
+    if ((EPI & 3) == EPI_STATS) { tc_epilogue_stats<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, col_off, taddr); return; }
+    if ((EPI & 3) == EPI_GRAD) { tc_epilogue_grad<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, col_off, taddr); return; }
     float* const Cout = p.C + (int64_t)it.z * p.split_stride;
-    float rn = 0.f;
-    if (EPI == EPI_L2DIST && row < p.M) rn = p.row_norm2[row];
 #pragma unroll 1
     for (int c0 = col_off; c0 < col_off + 64; c0 += 32) {
         float v[32];
@@ -243,13 +250,6 @@ __device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem&
         if (row >= p.M) continue;
         const int ncol = it.n0 + c0;
         float* dst = Cout + (int64_t)row * p.ldc + ncol;
-        if (EPI == EPI_L2DIST) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const float d2 = rn + (ncol + i < p.N ? p.col_norm2[ncol + i] : 0.f) - 2.f * v[i];
-                v[i] = -sqrtf(fmaxf(d2, 0.f));
-            }
-        }
         if (ncol + 32 <= p.N && (p.ldc & 3) == 0) {
 #pragma unroll
             for (int i = 0; i < 32; i += 4)
@@ -451,31 +451,139 @@ int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t 
     return KGE_OK;
 }
 
-// F[B, N] from the bf16 copies of the query vectors and the staged negatives.
-int launch_tc_scores(kge_handle* h, cudaStream_t s) {
+namespace {
+
+// One warp per positive merges the per-piece statistics of its row (and the positive score,
+// which the sampled softmax normalises over too) into the row's final (max, 1 / normaliser),
+// the per-positive loss and dL/df+.
+struct CombineParams {
+    const float4* stat_part; int pieces; int B;
+    const float* fpos;
+    int loss; float gamma, ce_c, loss_scale;
+    float2* row_stat; float *Lrow, *gpos;
+};
+
+__global__ void __launch_bounds__(256) stats_combine_kernel(CombineParams p) {
+    const int b = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (b >= p.B) return;
+    const float4* row = p.stat_part + (int64_t)b * p.pieces;
+    const float fp = p.fpos[b];
+    const bool ce = p.loss == KGE_LOSS_SAMPLED_SOFTMAX;
+    // the pieces carry their maxima and exponent sums in base 2 (exponent times log2 e)
+    float m = -INFINITY;
+    for (int j = lane; j < p.pieces; j += 32) m = fmaxf(m, row[j].x);
+    m = warp_max(m);
+    if (ce) m = fmaxf(m, fp * kLog2e);
+    float z = 0.f, l = 0.f;
+    for (int j = lane; j < p.pieces; j += 32) {
+        const float4 s = row[j];
+        const float r = exp2f(s.x - m);    // a piece without valid columns has max = -inf: weight 0
+        z += s.y * r; l += s.z * r;
+    }
+    z = warp_sum(z); l = warp_sum(l);
+    if (lane != 0) return;
+    if (ce) {
+        const float epos = exp2f(fp * kLog2e - m);
+        z += epos;
+        p.Lrow[b] = -fp + (m + log2f(z)) * 0.6931471805599453f;
+        p.gpos[b] = p.loss_scale * (epos / z - 1.f);
+    } else {
+        float sp, sg;
+        tc_softplus_sigmoid(-(p.gamma + fp), sp, sg);
+        p.Lrow[b] = sp + l / z;
+        p.gpos[b] = -p.loss_scale * sg;
+    }
+    p.row_stat[b] = make_float2(m, 1.f / z);
+}
+
+// Norm expansion only: row sums and column sums of the written dL/dF from their pieces,
+// added in ascending piece order.
+__global__ void __launch_bounds__(256) grad_sums_kernel(const float* grow_part, int row_pieces, float* Grow, int B,
+                                                        const float* gcol_part, int col_pieces, float* Gcol, int N) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < B) {
+        float t = 0.f;
+        for (int j = 0; j < row_pieces; ++j) t += grow_part[(int64_t)i * row_pieces + j];
+        Grow[i] = t;
+    } else if (i - B < N) {
+        const int n = i - B;
+        float t = 0.f;
+        for (int j = 0; j < col_pieces; ++j) t += gcol_part[(int64_t)j * N + n];
+        Gcol[n] = t;
+    }
+}
+
+}  // namespace
+
+namespace {
+template <int EPI>
+cudaError_t launch_gemm_inst(const unsigned char* tmA, const unsigned char* tmB, const TcGemmParams& p, int num_sms, cudaStream_t s) {
+    static bool configured = false;
+    if (!configured) {
+        const cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    tc_gemm_kernel<EPI><<<std::min(p.items, num_sms), TC_THREADS, TC_SMEM_BYTES, s>>>(
+        *reinterpret_cast<const CUtensorMap*>(tmA), *reinterpret_cast<const CUtensorMap*>(tmB), p);
+    return cudaSuccess;
+}
+
+// Scores Q . T^T with one of the fused loss epilogues.
+cudaError_t launch_fused(int pass, bool l2, bool ce, kge_handle* h, const TcGemmParams& p, cudaStream_t s) {
+    const int key = (pass == EPI_GRAD ? 4 : 0) | (l2 ? 2 : 0) | (ce ? 1 : 0);
+    switch (key) {
+        case 0: return launch_gemm_inst<EPI_STATS>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        case 1: return launch_gemm_inst<EPI_STATS | EPI_CE>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        case 2: return launch_gemm_inst<EPI_STATS | EPI_L2>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        case 3: return launch_gemm_inst<EPI_STATS | EPI_L2 | EPI_CE>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        case 4: return launch_gemm_inst<EPI_GRAD>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        case 5: return launch_gemm_inst<EPI_GRAD | EPI_CE>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        case 6: return launch_gemm_inst<EPI_GRAD | EPI_L2>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        default: return launch_gemm_inst<EPI_GRAD | EPI_L2 | EPI_CE>(h->tm_q, h->tm_t, p, h->num_sms, s);
+    }
+}
+}  // namespace
+
+// Forward of the tensor-core path without the B x N score block ever leaving the chip:
+//   pass 1  scores -> per-piece statistics;  merge per row -> loss, dL/df+, (max, 1 / normaliser)
+//   pass 2  scores again -> dL/dF as bf16, as it is and transposed, for the backward contractions
+int launch_tc_forward(kge_handle* h, cudaStream_t s) {
     const kge_config& c = h->cfg;
-    TcGemmParams p;
+    Workspace& w = h->ws;
+    TcGemmParams p{};
     p.M = c.batch; p.N = c.num_neg; p.K = c.dim;
     p.kb_per_split = (p.K + TC_BK - 1) / TC_BK; p.split_stride = 0;
     p.tiles_m = (p.M + TC_BM - 1) / TC_BM; p.tiles_n = (p.N + TC_BN - 1) / TC_BN; p.items = p.tiles_m * p.tiles_n;
-    p.C = h->ws.F; p.ldc = c.num_neg;
-    p.row_norm2 = h->ws.qn2; p.col_norm2 = h->ws.tn2;
-    p.status = h->ws.status;
-    static bool configured = false;
-    if (!configured) {
-        KGE_CUDA_CHECK(h, cudaFuncSetAttribute(tc_gemm_kernel<EPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES));
-        KGE_CUDA_CHECK(h, cudaFuncSetAttribute(tc_gemm_kernel<EPI_L2DIST>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES));
-        configured = true;
-    }
-    const dim3 grid(std::min(p.items, h->num_sms));
-    const CUtensorMap& tq = *reinterpret_cast<const CUtensorMap*>(h->tm_q);
-    const CUtensorMap& tt = *reinterpret_cast<const CUtensorMap*>(h->tm_t);
-    if (h->kind == KIND_L2) tc_gemm_kernel<EPI_L2DIST><<<grid, TC_THREADS, TC_SMEM_BYTES, s>>>(tq, tt, p);
-    else tc_gemm_kernel<EPI_STORE><<<grid, TC_THREADS, TC_SMEM_BYTES, s>>>(tq, tt, p);
+    p.C = nullptr; p.ldc = 0;
+    p.row_norm2 = w.qn2; p.col_norm2 = w.tn2;
+    p.status = w.status;
+    p.l2 = h->kind == KIND_L2; p.loss = c.loss;
+    p.gamma = c.gamma; p.adv_temp = c.adv_temp; p.ce_c = c.ce_correction; p.loss_scale = c.loss_scale;
+    p.stat_part = reinterpret_cast<float4*>(w.stat_part); p.row_stat = reinterpret_cast<const float2*>(w.row_stat);
+    p.Gb = w.Gb; p.ldg = (c.num_neg + 7) / 8 * 8;
+    p.GbT = w.GbT; p.ldgt = (c.batch + 7) / 8 * 8;
+    p.grow_part = w.grow_part; p.gcol_part = w.gcol_part;
+    const bool ce = c.loss == KGE_LOSS_SAMPLED_SOFTMAX;
+    stage_begin(h, ST_BLOCK, s);
+    KGE_CUDA_CHECK(h, launch_fused(EPI_STATS, p.l2 != 0, ce, h, p, s));
+    stage_end(h, ST_BLOCK, s);
     KGE_LAUNCH_CHECK(h);
+    stage_begin(h, ST_LOSS, s);
+    CombineParams cp{p.stat_part, 2 * p.tiles_n, p.M, w.fpos, c.loss, c.gamma, c.ce_correction, c.loss_scale,
+                     reinterpret_cast<float2*>(w.row_stat), w.Lrow, w.gpos};
+    stats_combine_kernel<<<(p.M * 32 + 255) / 256, 256, 0, s>>>(cp);
+    KGE_LAUNCH_CHECK(h);
+    KGE_CUDA_CHECK(h, launch_fused(EPI_GRAD, p.l2 != 0, ce, h, p, s));
+    KGE_LAUNCH_CHECK(h);
+    if (p.l2) {
+        grad_sums_kernel<<<(p.M + p.N + 255) / 256, 256, 0, s>>>(w.grow_part, 2 * p.tiles_n, w.Grow, p.M,
+                                                                 w.gcol_part, 4 * p.tiles_m, w.Gcol, p.N);
+        KGE_LAUNCH_CHECK(h);
+    }
+    stage_end(h, ST_LOSS, s);
     return KGE_OK;
 }
-
 
 namespace {
 int launch_cast(kge_handle* h, const float* src, int64_t lds, int R, int C, uint16_t* dst_rm, int64_t ld_rm,
@@ -504,15 +612,13 @@ int launch_tc_gemm(kge_handle* h, const unsigned char* tmA, const unsigned char*
     p.status = h->ws.status;
     p.tiles_m = (M + TC_BM - 1) / TC_BM; p.tiles_n = (N + TC_BN - 1) / TC_BN;
     p.items = p.tiles_m * p.tiles_n * ((kb + p.kb_per_split - 1) / p.kb_per_split);
-    const dim3 grid(std::min(p.items, h->num_sms));
-    tc_gemm_kernel<EPI_STORE><<<grid, TC_THREADS, TC_SMEM_BYTES, s>>>(*reinterpret_cast<const CUtensorMap*>(tmA),
-                                                                       *reinterpret_cast<const CUtensorMap*>(tmB), p);
+    KGE_CUDA_CHECK(h, launch_gemm_inst<EPI_STORE>(tmA, tmB, p, h->num_sms, s));
     KGE_LAUNCH_CHECK(h);
     return KGE_OK;
 }
 }  // namespace
 
-// The two backward contractions on tensor cores, from bf16 copies of dL/dF (held in F):
+// The two backward contractions on tensor cores, from the bf16 dL/dF the forward left behind:
 //   dQ partial[split] = G . T      (A = Gb [B, N],   B operand = Tb^T [d, N])
 //   dT partial[split] = G^T . Q    (A = Gb^T [N, B], B operand = Qb^T [d, B])
 // The K splits land in the same partial buffers the CUDA-core path uses and are added in
@@ -524,7 +630,6 @@ int launch_tc_backward(kge_handle* h, cudaStream_t s, cudaStream_t side) {
     const int64_t ldN = (N + 7) / 8 * 8, ldB = (B + 7) / 8 * 8;
     int rc;
     stage_begin(h, ST_TH_CPASS, s);   // stage slot shared with the TransH pass: operand casts
-    if ((rc = launch_cast(h, w.F, N, B, N, w.Gb, ldN, w.GbT, ldB, w.Gcol, s)) != KGE_OK) return rc;
     if ((rc = launch_cast(h, w.Tneg, d, N, d, nullptr, 0, w.TbT, ldN, nullptr, s)) != KGE_OK) return rc;
     if ((rc = launch_cast(h, w.Q, d, B, d, nullptr, 0, w.QbT, ldB, nullptr, s)) != KGE_OK) return rc;
     stage_end(h, ST_TH_CPASS, s);

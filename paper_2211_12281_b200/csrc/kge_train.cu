@@ -1176,12 +1176,12 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     }
     stage_end(h, ST_BUILD, s);
     KGE_LAUNCH_CHECK(h);
-    stage_begin(h, ST_BLOCK, s);
     if (c.prec == KGE_PREC_BF16_TC) {
-        const int rc = launch_tc_scores(h, s);
+        // tensor cores: scores, loss and dL/dF in two fused passes, the score block never stored
+        const int rc = launch_tc_forward(h, s);
         if (rc != KGE_OK) return rc;
-        h->launches -= 1;   // counted again below
-    } else
+    } else {
+    stage_begin(h, ST_BLOCK, s);
     switch (p.kind) {
         case KIND_L1: KGE_CUDA_CHECK(h, launch_block_tma<KIND_L1>(p, s)); break;
         case KIND_L2: KGE_CUDA_CHECK(h, launch_block_tma<KIND_L2>(p, s)); break;
@@ -1211,6 +1211,7 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     }
     stage_end(h, ST_LOSS, s);
     KGE_LAUNCH_CHECK(h);
+    }
     if (p.kind == KIND_TH_L1 || p.kind == KIND_TH_L2) {
         stage_begin(h, ST_TH_CPASS, s);
         if (p.kind == KIND_TH_L1) launch_block<KIND_TH_L1, 1>(p, s); else launch_block<KIND_TH_L2, 1>(p, s);
