@@ -223,13 +223,15 @@ __device__ __forceinline__ void apply_row(const UpdateJob& J, const UpdateParams
     }
 }
 
-// g += rows[idx[0]], rows[idx[1]], ... in that order, four loads in flight at a time.
+// g += rows[idx[0]], rows[idx[1]], ... in that order, a few rows' loads in flight at a time
+// (four for narrow rows, two for wide ones, to keep the register count down).
 template <typename V, int NCH, typename IndexOf>
 __device__ __forceinline__ void ordered_sum(const V* rows, int wv, int count, IndexOf index_of, V (&g)[NCH], int lane) {
-    for (int s = 0; s < count; s += 4) {
-        V v[4][NCH];
+    constexpr int BATCH = NCH == 1 ? 4 : 2;
+    for (int s = 0; s < count; s += BATCH) {
+        V v[BATCH][NCH];
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
+        for (int r = 0; r < BATCH; ++r) {
             const V* src = rows + (s + r < count ? index_of(s + r) : 0) * wv;
 #pragma unroll
             for (int i = 0; i < NCH; ++i) {
@@ -238,7 +240,7 @@ __device__ __forceinline__ void ordered_sum(const V* rows, int wv, int count, In
             }
         }
 #pragma unroll
-        for (int r = 0; r < 4; ++r)
+        for (int r = 0; r < BATCH; ++r)
 #pragma unroll
             for (int i = 0; i < NCH; ++i) VecOps<V>::add(g[i], v[r][i]);
     }
@@ -257,6 +259,16 @@ __device__ __forceinline__ void piece_sum(const UpdateJob& J, const UpdateParams
     if (whole ? r != s0 : ((r - s0) % PIECE) != 0) return;
     const int count = whole ? len : min(PIECE, s1 - r);
     const int32_t src = lane < count ? J.perm[r + lane] : 0;
+    if (whole) {   // start fetching the table row (and its optimiser state) while the gradients are summed
+        const int64_t row = J.uniq[u];
+        const int row_lines = (J.width * 4 + 127) / 128;
+        const char* base = reinterpret_cast<const char*>(J.table + row * J.width);
+        if (lane < row_lines) asm volatile("prefetch.global.L2 [%0];" ::"l"(base + lane * 128));
+        if (p.opt == KGE_OPT_ADAM) {
+            const char* sb = reinterpret_cast<const char*>(J.state + row * 2 * J.width);
+            for (int ln = lane; ln < 2 * row_lines; ln += 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(sb + ln * 128));
+        }
+    }
     V g[NCH];
 #pragma unroll
     for (int i = 0; i < NCH; ++i) g[i] = VecOps<V>::zero();
@@ -294,7 +306,7 @@ __device__ __forceinline__ void piece_do(const UpdateJob& J, const UpdateParams&
 }
 
 template <bool JOIN>
-__global__ void __launch_bounds__(256) piece_kernel(UpdateParams p) {
+__global__ void __launch_bounds__(256, 3) piece_kernel(UpdateParams p) {
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (gw >= p.warp_begin[p.njobs]) return;
     int j = 0;
