@@ -60,6 +60,17 @@ WORKLOADS = {
                         entity_zipf=1.1, relation_zipf=0.0, graph_seed=0),
 }
 
+# BASELINE configs[4]: 15,000 (h, r) queries against all 91,000,000 entities of d = 128, top-10 and the
+# rank of a designated true tail.  The "s" variants keep the query batch and shrink the table.
+INFER_WORKLOADS = {
+    "c5_transe_l1": dict(E=91_000_000, R=1400, d=128, Q=15000, K=10, score="transe", p_norm=1),
+    "c5_distmult": dict(E=91_000_000, R=1400, d=128, Q=15000, K=10, score="distmult", p_norm=1),
+    "c5_distmult_tc": dict(E=91_000_000, R=1400, d=128, Q=15000, K=10, score="distmult", p_norm=1, tc=True),
+    "c5s_distmult_tc": dict(E=4_000_000, R=1400, d=128, Q=15000, K=10, score="distmult", p_norm=1, tc=True),
+    "c5s_transe_l1": dict(E=4_000_000, R=1400, d=128, Q=15000, K=10, score="transe", p_norm=1),
+    "c5s_distmult": dict(E=4_000_000, R=1400, d=128, Q=15000, K=10, score="distmult", p_norm=1),
+}
+
 # fp32 CUDA-core peak used for "bound": "alu": 148 SMs x 128 fp32 lanes x 1.965 GHz, one
 # instruction per lane per clock (an FMA counts as one).
 ALU_PEAK_TOPS = 148 * 128 * 1.965e9 / 1e12
@@ -338,15 +349,80 @@ def run_ours(args, w, name):
         dist.destroy_process_group()
 
 
+def run_infer(args, w, name):
+    """Full-entity scoring with top-k and rank: one step = one pass of all queries over the table."""
+    import torch
+    import paper_2211_12281_b200 as K
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    E, R, d, Q, k = w["E"], w["R"], w["d"], w["Q"], w["K"]
+    gen = torch.Generator(device=dev); gen.manual_seed(5)
+    ent = torch.empty((E, d), dtype=torch.float32, device=dev).normal_(0.0, d ** -0.5, generator=gen)
+    rel = torch.empty((R, d), dtype=torch.float32, device=dev).normal_(0.0, d ** -0.5, generator=gen)
+    qh, qr, tt = kge_synth.make_queries(E, R, Q, seed=5)
+    qh_d, qr_d, tt_d = (torch.from_numpy(a).to(dev) for a in (qh, qr, tt))
+    kge = K.Kge(K.KgeConfig.make(num_entities=E, num_relations=R, dim=d, score=w["score"], p_norm=w["p_norm"],
+                                 prec=K.PREC_BF16_TC if w.get("tc") else K.PREC_FP32))
+    kge.bind(ent, rel, max_queries=Q, topk=k)
+    ids = torch.empty((Q, k), dtype=torch.int32, device=dev)
+    sc = torch.empty((Q, k), dtype=torch.float32, device=dev)
+    ranks = torch.empty(Q, dtype=torch.int32, device=dev)
+    steps, warm = max(1, min(args.steps, 5)), max(1, min(args.warmup, 2))
+    for _ in range(warm):
+        kge.score_all_topk(qh_d, qr_d, k, tt_d, ids, sc, ranks)
+    clocks = ClockSampler(0)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = kge.launch_count()
+    a.record()
+    for _ in range(steps):
+        kge.score_all_topk(qh_d, qr_d, k, tt_d, ids, sc, ranks)
+    b.record(); torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / steps
+    clock_info = clocks.stop()
+    assert kge.get_status() == 0
+    pairs = float(Q) * E
+    t_hbm = E * d * 4 / (measured_peaks()["hbm_gbs"] * 1e9)
+    ops = {"transe": 2.0, "distmult": 1.0}[w["score"]]
+    t_alu = ops * pairs * d / (ALU_PEAK_TOPS * 1e12)
+    bound = "alu" if t_alu > t_hbm else "hbm"
+    if w.get("tc"):
+        peaks = json.loads((ROOT / "MEASURED_PEAKS.json").read_text()) if (ROOT / "MEASURED_PEAKS.json").exists() else {}
+        peak = peaks.get("bf16_tflops_sustained", 1400.0)
+        t_tc = 2.0 * pairs * d / (peak * 1e12)
+        bound = "tensor" if t_tc > t_hbm else "hbm"
+    roof = {"bound": bound, "kernel": "tc_gemm<topk>" if w.get("tc") else "score_tile", "frac": max(t_alu, t_hbm) / (ms * 1e-3), "traffic": None,
+            "t_alu_ms": t_alu * 1e3, "t_hbm_ms": t_hbm * 1e3}
+    if bound == "tensor":
+        roof.update(achieved=2.0 * pairs * d / (ms * 1e-3) / 1e12, peak=peak, unit="TFLOP/s", frac=t_tc / (ms * 1e-3))
+    elif bound == "alu":
+        roof.update(achieved=ops * pairs * d / (ms * 1e-3) / 1e12, peak=ALU_PEAK_TOPS, unit="TFLOP/s")
+    else:
+        roof.update(achieved=E * d * 4 / (ms * 1e-3) / 1e9, peak=measured_peaks()["hbm_gbs"], unit="GB/s")
+    line = {"metric": "scored pairs/sec (full-entity top-k + rank)", "value": pairs / (ms * 1e-3), "unit": "pairs/s",
+            "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if w.get("tc") else "f32", "data": "synthetic",
+            "config": {"workload": name, "entities": E, "relations": R, "dim": d, "queries": Q, "topk": k,
+                       "score": w["score"], "p_norm": w["p_norm"], "l2": "table larger than L2" if E * d * 4 > 126e6 else "table fits L2"},
+            "queries_per_s": Q / (ms * 1e-3), "gpu_launches": int((kge.launch_count() - l0) / steps),
+            "clocks": clock_info, "roofline": roof, "mean_rank": float(ranks.float().mean().item())}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="c2_transe_l1")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS) + sorted(INFER_WORKLOADS), default="c2_transe_l1")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.workload in INFER_WORKLOADS:
+        if args.impl == "reference":
+            raise SystemExit("--impl reference covers the training workloads")
+        return run_infer(args, INFER_WORKLOADS[args.workload], args.workload)
     w = WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, w, args.workload)

@@ -111,6 +111,10 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
         w.cand_cnt = cv.take<int32_t>(q); w.beat_tmp = cv.take<int32_t>(q); w.beat = cv.take<int32_t>(q);
         w.cand_score = cv.take<float>(q * kCandCap); w.cand_id = cv.take<int32_t>(q * kCandCap);
         w.top_score = cv.take<float>(q * k); w.top_id = cv.take<int32_t>(q * k);
+        // tensor-core inference (dot-product models): bf16 query vectors and a bf16 copy of the whole table
+        const bool tci = c.prec == KGE_PREC_BF16_TC && (c.score == KGE_DISTMULT || c.score == KGE_COMPLEX);
+        w.iqb = tci ? cv.take<uint16_t>(q * d) : nullptr;
+        w.Eb = tci ? cv.take<uint16_t>((size_t)c.num_entities * d) : nullptr;
     }
     if (out) *out = w;
     return cv.used;
@@ -252,6 +256,10 @@ int kge_bind(kge_handle* h, float* ent, float* rel, float* relw, float* ent_stat
         if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_gt, h->ws.GbT, N, B, ldB);
         if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_tt, h->ws.TbT, d, N, ldN);
         if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_qt, h->ws.QbT, d, B, ldB);
+        if (rc == KGE_OK && h->ws.Eb) {
+            rc = tc_make_operand_map(h, h->tm_iq, h->ws.iqb, max_queries, d, d);
+            if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_eb, h->ws.Eb, h->cfg.num_entities, d, d);
+        }
         if (rc != KGE_OK) return rc;
     }
     if (!h->streams_ready) {

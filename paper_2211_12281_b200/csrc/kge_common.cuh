@@ -66,6 +66,7 @@ struct Workspace {
     float *part_ent, *part_rel, *part_relw;  // [list length, width] partial sums of long segments
     // inference
     float *iq, *iwhat, *iftrue;            // [maxq,d], [maxq,d], [maxq]
+    uint16_t *iqb, *Eb;                    // [maxq,d], [E,d] bf16 query vectors and entity table (tensor-core inference)
     float *thr;                            // [maxq] current k-th best score (-inf until the list is full)
     int32_t *thr_id;                       // [maxq] its id
     int32_t *cand_cnt, *beat_tmp, *beat;   // [maxq]
@@ -109,6 +110,7 @@ struct kge_handle {
     // two backward accumulations run beside the main stream's kernels (created by kge_bind).
     // TMA tensor maps (tensor-core path): Qb, Tb for the scores; Gb, Tb^T for dQ; Gb^T, Qb^T for dT
     alignas(64) unsigned char tm_q[128], tm_t[128], tm_g[128], tm_gt[128], tm_tt[128], tm_qt[128];
+    alignas(64) unsigned char tm_iq[128], tm_eb[128];   // inference: bf16 query vectors and bf16 entity table
     bool streams_ready;
     cudaStream_t side[2];
     cudaEvent_t ev_ids, ev_loss, ev_seg, ev_t;
@@ -160,6 +162,8 @@ int launch_update(kge_handle* h, uint64_t step, float lr, cudaStream_t s);
 int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols, int64_t ld);
 int launch_tc_backward(kge_handle* h, cudaStream_t s, cudaStream_t side);
 int launch_tc_forward(kge_handle* h, cudaStream_t s);
+int launch_cast_bf16(kge_handle* h, const float* src, uint16_t* dst, int64_t count, cudaStream_t s);
+int launch_tc_infer_chunk(kge_handle* h, int nq, int64_t e_lo, int64_t e_hi, const int32_t* true_tails, cudaStream_t s);
 int dedup_tiles(int n);     // sort tiles of a list of n ids
 int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int32_t nq, int32_t k,
                        const int32_t* true_tails, int32_t* out_ids, float* out_scores, int32_t* out_ranks,

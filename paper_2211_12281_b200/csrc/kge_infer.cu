@@ -299,6 +299,19 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(InferParams p) {
     }
 }
 
+// Tensor-core inference: the true tail's score in the arithmetic of that path (operands rounded
+// to bf16, fp32 accumulation), one thread per query.
+__global__ void ftrue_bf16_kernel(InferParams p) {
+    const int q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.nq || !p.tt) return;
+    const uint16_t* qb = p.w.iqb + (int64_t)q * p.d;
+    const uint16_t* tb = p.w.Eb + checked_id(p.tt[q], p.E, p.w.status) * p.d;
+    float acc = 0.f;
+    for (int k = 0; k < p.d; ++k)
+        acc = __fmaf_rn(__uint_as_float((uint32_t)qb[k] << 16), __uint_as_float((uint32_t)tb[k] << 16), acc);
+    p.w.iftrue[q] = acc;
+}
+
 __global__ void reset_chunk_kernel(InferParams p) {
     const int q = blockIdx.x * blockDim.x + threadIdx.x;
     if (q < p.nq) { p.w.cand_cnt[q] = 0; p.w.beat_tmp[q] = 0; }
@@ -348,6 +361,20 @@ int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int3
     query_setup_kernel<<<qblocks, 128, 0, s>>>(p);
     KGE_LAUNCH_CHECK(h);
     KGE_CUDA_CHECK(h, cudaMemsetAsync(h->ws.status + 1, 0, 4, s));
+    const bool tc = h->ws.Eb != nullptr;    // dot-product model with the tensor-core score block
+    if (tc) {
+        int rc = launch_cast_bf16(h, h->ws.iq, h->ws.iqb, (int64_t)nq * c.dim, s);
+        if (rc == KGE_OK) rc = launch_cast_bf16(h, h->ent, h->ws.Eb, c.num_entities * c.dim, s);
+        if (rc != KGE_OK) return rc;
+        ftrue_bf16_kernel<<<qblocks, 128, 0, s>>>(p);
+        KGE_LAUNCH_CHECK(h);
+    }
+    auto score_chunk = [&](const InferParams& ip) -> int {
+        if (tc) return launch_tc_infer_chunk(h, nq, ip.e_lo, ip.e_hi, true_tails, s);
+        launch_score_tiles(ip, s);
+        KGE_LAUNCH_CHECK(h);
+        return KGE_OK;
+    };
 
     // Chunk i covers as many entities as all chunks before it (the first: one candidate
     // list's worth, since nothing is filtered yet), capped so a launch stays bounded.
@@ -356,8 +383,7 @@ int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int3
     while (lo < p.E) {
         const int64_t len = std::min<int64_t>(std::min<int64_t>(std::max<int64_t>(lo, kCandCap), max_chunk), p.E - lo);
         p.e_lo = lo; p.e_hi = lo + len;
-        launch_score_tiles(p, s);
-        KGE_LAUNCH_CHECK(h);
+        { const int rc = score_chunk(p); if (rc != KGE_OK) return rc; }
         int32_t overflow = 0;
         KGE_CUDA_CHECK(h, cudaMemcpyAsync(&overflow, h->ws.status + 1, 4, cudaMemcpyDeviceToHost, s));
         KGE_CUDA_CHECK(h, cudaStreamSynchronize(s));
@@ -371,8 +397,7 @@ int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int3
             KGE_LAUNCH_CHECK(h);
             for (int64_t sub = lo; sub < lo + len; sub += kCandCap) {
                 p.e_lo = sub; p.e_hi = std::min<int64_t>(sub + kCandCap, lo + len);
-                launch_score_tiles(p, s);
-                KGE_LAUNCH_CHECK(h);
+                { const int rc = score_chunk(p); if (rc != KGE_OK) return rc; }
                 select_kernel<<<nq, SEL_THREADS, 0, s>>>(p);
                 KGE_LAUNCH_CHECK(h);
             }

@@ -35,9 +35,10 @@ constexpr int TC_THREADS = 32 * (2 + TC_EPI_WARPS);
 constexpr uint32_t TC_A_BYTES = TC_BM * TC_BK * 2, TC_B_BYTES = TC_BN * TC_BK * 2;
 constexpr uint32_t TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
 constexpr size_t TC_SMEM_BYTES = 1024 + (size_t)TC_STAGES * TC_STAGE_BYTES + 128;
+constexpr int TC_BEAT_ROWS_MAX = 20 * 1024;                // queries whose rank counts fit in shared memory beside the stages
 constexpr uint32_t TC_TMEM_COLS = 256;                    // two fp32 accumulators of 128 columns, used in turn
 
-enum { EPI_STORE = 0, EPI_STATS = 1, EPI_GRAD = 2, EPI_L2 = 4, EPI_CE = 8 };   // L2 / CE: flags of the fused epilogues
+enum { EPI_STORE = 0, EPI_STATS = 1, EPI_GRAD = 2, EPI_TOPK = 3, EPI_L2 = 4, EPI_CE = 8 };   // L2 / CE: flags of the fused loss epilogues
 
 struct TcGemmParams {
     int M, N, K;
@@ -56,6 +57,16 @@ struct TcGemmParams {
     uint16_t* GbT; int64_t ldgt;          // [N, ldgt] its transpose
     float* grow_part;                     // [M, 2 * tiles_n] sums of the written values per 64-column piece
     float* gcol_part;                     // [4 * tiles_m, N] sums per 32-row piece (l2 only)
+    // full-entity scoring (EPI_TOPK): rows are queries, columns the entities [n_base, n_base + N)
+    int m_fastest;                        // walk the row tiles of one column tile first (the column tile stays in L2)
+    int64_t n_base;
+    const float *thr, *ftrue;             // [M] current k-th best score; score of the true tail
+    const int32_t *thr_id, *tt;           // [M] its id; true tail ids (or NULL)
+    int32_t *cand_cnt, *beat_tmp;         // [M] candidates appended in this chunk; entities ordered before the true tail
+    float* cand_score; int32_t* cand_id;  // [M, cand_cap]
+    int cand_cap;
+    int32_t* overflow;                    // set when a candidate list is full
+    int beat_rows;                        // rows whose rank counts are gathered in shared memory first (0: global atomics)
 };
 
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
@@ -236,11 +247,53 @@ __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const Tc
     if (L2 && rin) p.grow_part[(int64_t)row * (2 * p.tiles_n) + (it.n0 / TC_BN) * 2 + col_off / 64] = rsum;
 }
 
+// Full-entity scoring (Section 3.1 "Inference"): a score survives into the query's candidate
+// list if it is ordered before the query's current k-th best under (score descending, entity
+// id ascending); entities ordered before the true tail are counted for its rank.
+__device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr, int32_t* beat_sm) {
+    const bool rin = row < p.M;
+    float thr = 0.f, ft = 0.f; int32_t thr_id = 0, tt = -1;
+    if (rin) {
+        thr = p.thr[row]; thr_id = p.thr_id[row];
+        if (p.tt) { ft = p.ftrue[row]; tt = p.tt[row]; }
+    }
+    int beat = 0;
+#pragma unroll 1
+    for (int c0 = col_off; c0 < col_off + 64; c0 += 32) {
+        float v[32];
+        tmem_ld32(taddr + (uint32_t)(c0 - col_off), v);
+        if (!rin) continue;
+        const int ncol = it.n0 + c0;
+        const int valid = min(32, p.N - ncol);
+        const int32_t e0 = (int32_t)(p.n_base + ncol);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            if (valid != 32 && i >= valid) continue;
+            const float f = v[i];
+            const int32_t e = e0 + i;
+            if (tt >= 0 && e != tt && (f > ft || (f == ft && e < tt))) ++beat;
+            if (f > thr || (f == thr && e < thr_id)) {
+                const int slot = atomicAdd(&p.cand_cnt[row], 1);
+                if (slot < p.cand_cap) {
+                    p.cand_score[(int64_t)row * p.cand_cap + slot] = f;
+                    p.cand_id[(int64_t)row * p.cand_cap + slot] = e;
+                } else {
+                    *p.overflow = 1;   // the host redoes this chunk in pieces that cannot overflow
+                }
+            }
+        }
+    }
+    if (rin && beat > 0) {
+        if (row < p.beat_rows) atomicAdd(&beat_sm[row], beat); else atomicAdd(&p.beat_tmp[row], beat);
+    }
+}
+
 // Epilogue of one warp on one item: 64 columns [col_off, col_off + 64) of the tile row held by
 // this thread's tensor-memory lane (taddr points at the first of them).
 template <int EPI>
-__device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr) {
+__device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr, int32_t* beat_sm) {
     if ((EPI & 3) == EPI_STATS) { tc_epilogue_stats<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, col_off, taddr); return; }
+    if ((EPI & 3) == EPI_TOPK) { tc_epilogue_topk(p, it, row, col_off, taddr, beat_sm); return; }
     if ((EPI & 3) == EPI_GRAD) { tc_epilogue_grad<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, col_off, taddr); return; }
     float* const Cout = p.C + (int64_t)it.z * p.split_stride;
 #pragma unroll 1
@@ -263,8 +316,9 @@ __device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem&
 
 // Work item = (K split, row tile, column tile), column tile fastest.  A CTA takes a contiguous
 // run of items, so consecutive items mostly share their A rows (kept warm in L2).
-__device__ __forceinline__ TcItem tc_item(const TcGemmParams& p, int item) {
-    const int tn = item % p.tiles_n, r = item / p.tiles_n;
+__device__ __forceinline__ TcItem tc_item(const TcGemmParams& p, int64_t item) {
+    if (p.m_fastest) return TcItem{0, (int)(item % p.tiles_m) * TC_BM, (int)(item / p.tiles_m) * TC_BN};
+    const int tn = (int)(item % p.tiles_n), r = (int)(item / p.tiles_n);
     return TcItem{r / p.tiles_m, (r % p.tiles_m) * TC_BM, tn * TC_BN};
 }
 
@@ -279,6 +333,9 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
     uint64_t* acc_empty = acc_full + 2;          // [2] accumulator buffer drained by all epilogue warps
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     volatile uint32_t* stop = tmem_slot + 1;     // set by a warp whose wait ran out
+    int32_t* beat_sm = reinterpret_cast<int32_t*>(base + (size_t)TC_STAGES * TC_STAGE_BYTES + 128);   // [beat_rows], EPI_TOPK
+    if ((EPI & 3) == EPI_TOPK)
+        for (int i = threadIdx.x; i < p.beat_rows; i += TC_THREADS) beat_sm[i] = 0;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int per_cta = (p.items + gridDim.x - 1) / gridDim.x;
@@ -312,7 +369,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
                     unsigned char* sa = base + (size_t)s * TC_STAGE_BYTES;
                     mbar_arrive_expect_tx(&full[s], TC_STAGE_BYTES);
                     tma_load_2d(sa, &tmA, (kb0 + kb) * TC_BK, it.m0, &full[s]);
-                    tma_load_2d(sa + TC_A_BYTES, &tmB, (kb0 + kb) * TC_BK, it.n0, &full[s]);
+                    tma_load_2d(sa + TC_A_BYTES, &tmB, (kb0 + kb) * TC_BK, (int)p.n_base + it.n0, &full[s]);
                 }
             }
         }
@@ -354,7 +411,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
             if (!ok || *stop) { if (lane == 0) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); } break; }
             const TcItem it = tc_item(p, item);
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * TC_BN + chalf * 64);
-            tc_epilogue<EPI>(p, it, it.m0 + quarter * 32 + lane, chalf * 64, taddr);
+            tc_epilogue<EPI>(p, it, it.m0 + quarter * 32 + lane, chalf * 64, taddr, beat_sm);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
@@ -364,6 +421,8 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
     __syncthreads();
     if (warp == 1)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
+    if ((EPI & 3) == EPI_TOPK)     // hand this CTA's rank counts over (integer adds: the result does not depend on the order)
+        for (int i = threadIdx.x; i < p.beat_rows; i += TC_THREADS) { const int32_t b = beat_sm[i]; if (b) atomicAdd(&p.beat_tmp[i], b); }
 }
 
 // src fp32 [R, C] (leading dimension lds) -> bf16 copies for the backward contractions:
@@ -517,14 +576,16 @@ __global__ void __launch_bounds__(256) grad_sums_kernel(const float* grow_part, 
 
 namespace {
 template <int EPI>
-cudaError_t launch_gemm_inst(const unsigned char* tmA, const unsigned char* tmB, const TcGemmParams& p, int num_sms, cudaStream_t s) {
+cudaError_t launch_gemm_inst(const unsigned char* tmA, const unsigned char* tmB, const TcGemmParams& p, int num_sms, cudaStream_t s,
+                             size_t extra_smem = 0) {
     static bool configured = false;
     if (!configured) {
-        const cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES);
+        const cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)(TC_SMEM_BYTES + TC_BEAT_ROWS_MAX * 4));
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    tc_gemm_kernel<EPI><<<std::min(p.items, num_sms), TC_THREADS, TC_SMEM_BYTES, s>>>(
+    tc_gemm_kernel<EPI><<<std::min(p.items, num_sms), TC_THREADS, TC_SMEM_BYTES + extra_smem, s>>>(
         *reinterpret_cast<const CUtensorMap*>(tmA), *reinterpret_cast<const CUtensorMap*>(tmB), p);
     return cudaSuccess;
 }
@@ -603,7 +664,7 @@ int launch_cast(kge_handle* h, const float* src, int64_t lds, int R, int C, uint
 
 int launch_tc_gemm(kge_handle* h, const unsigned char* tmA, const unsigned char* tmB, int M, int N, int K, int split,
                    float* C, int64_t ldc, cudaStream_t s) {
-    TcGemmParams p;
+    TcGemmParams p{};
     p.M = M; p.N = N; p.K = K;
     const int kb = (K + TC_BK - 1) / TC_BK;
     p.kb_per_split = (kb + split - 1) / split;
@@ -648,6 +709,48 @@ int launch_tc_backward(kge_handle* h, cudaStream_t s, cudaStream_t side) {
     stage_end(h, ST_ACCUM_T, s);
     if (rc != KGE_OK) return rc;
     if (side) KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_t, 0));
+    return KGE_OK;
+}
+
+
+namespace {
+__global__ void __launch_bounds__(256) cast_bf16_kernel(const float4* src, uint2* dst, int64_t n4) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+        const float4 v = src[i];
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+        dst[i] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+    }
+}
+}  // namespace
+
+// bf16 copy of `count` floats (count % 4 == 0, both 16-byte aligned).
+int launch_cast_bf16(kge_handle* h, const float* src, uint16_t* dst, int64_t count, cudaStream_t s) {
+    const int64_t n4 = count / 4;
+    const int grid = (int)std::min<int64_t>((n4 + 255) / 256, (int64_t)h->num_sms * 16);
+    cast_bf16_kernel<<<std::max(grid, 1), 256, 0, s>>>(reinterpret_cast<const float4*>(src), reinterpret_cast<uint2*>(dst), n4);
+    KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
+}
+
+// One chunk of full-entity scoring on tensor cores: the bf16 query vectors against the bf16
+// rows [e_lo, e_hi) of the entity table, survivors appended to the candidate lists.
+int launch_tc_infer_chunk(kge_handle* h, int nq, int64_t e_lo, int64_t e_hi, const int32_t* true_tails, cudaStream_t s) {
+    const Workspace& w = h->ws;
+    TcGemmParams p{};
+    p.M = nq; p.N = (int)(e_hi - e_lo); p.K = h->cfg.dim;
+    p.kb_per_split = (p.K + TC_BK - 1) / TC_BK;
+    p.tiles_m = (p.M + TC_BM - 1) / TC_BM; p.tiles_n = (p.N + TC_BN - 1) / TC_BN;
+    if ((int64_t)p.tiles_m * p.tiles_n > 0x7fffffff) return KGE_ERR_BAD_ARG;
+    p.items = p.tiles_m * p.tiles_n;
+    p.status = w.status;
+    p.m_fastest = 1; p.n_base = e_lo;
+    p.thr = w.thr; p.thr_id = w.thr_id; p.ftrue = w.iftrue; p.tt = true_tails;
+    p.cand_cnt = w.cand_cnt; p.beat_tmp = w.beat_tmp; p.cand_score = w.cand_score; p.cand_id = w.cand_id;
+    p.cand_cap = kCandCap; p.overflow = w.status + 1;
+    p.beat_rows = std::min(nq, TC_BEAT_ROWS_MAX);
+    // (the table's tensor map covers all rows; the kernel offsets its row coordinate by n_base)
+    KGE_CUDA_CHECK(h, launch_gemm_inst<EPI_TOPK>(h->tm_iq, h->tm_eb, p, h->num_sms, s, (size_t)p.beat_rows * 4));
+    KGE_LAUNCH_CHECK(h);
     return KGE_OK;
 }
 

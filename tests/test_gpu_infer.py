@@ -54,6 +54,33 @@ def test_topk_rank_mrr_against_fp32_oracle(oracle32, oracle64, score, p):
     assert abs(mrr0 - oracle64.mrr(o_ranks, 0)) <= 1e-3
 
 
+@pytest.mark.parametrize("score", ["distmult", "complex"])
+def test_tensor_core_topk_against_bf16_operand_oracle(oracle64, score):
+    """Full-entity scoring on tensor cores (bf16 operands, fp32 accumulation) against the oracle
+    with bf16-rounded operands.  The accumulation order differs, so the lists are compared as
+    sets with a near-tie audit (2e-2 relative is the stated bound of this path; 1e-4 is used),
+    ranks within 2, MRR within 1e-3.  E = 5000 leaves ragged 128-wide tiles, nq = 200 two row tiles."""
+    import kge_synth
+    E, R, d, K, nq = 5000, 9, 64, 10, 200
+    prob = Problem(E=E, R=R, T=100, d=d, score=score, p_norm=1, B=8, N=8, P=1, graph_seed=12, tc=True)
+    qh, qr, tt = kge_synth.make_queries(E, R, nq, seed=12)
+    tt[0] = qh[0]
+    gpu = GpuSide(prob, max_queries=nq, topk=K, load_graph=False)
+    ids, sc, ranks = _infer(gpu, qh, qr, tt, K)
+    cfg = prob.oracle_cfg()
+    r_ids, r_sc, r_ranks = oracle64.score_all_topk(cfg, prob.ent, prob.rel, prob.relw, qh, qr, K + 5, true_tails=tt)
+    for q in range(nq):
+        assert len(set(ids[q])) == K
+        for e in set(ids[q]) - set(r_ids[q, :K]):
+            assert e in set(r_ids[q]), "id outside the oracle's top (k+5)"
+            f = r_sc[q][list(r_ids[q]).index(e)]
+            assert abs(f - r_sc[q, K - 1]) <= 1e-4 * abs(f) + 1e-6
+    assert_close(sc, r_sc[:, :K], atol=1e-5, what="scores")
+    assert np.abs(ranks - r_ranks).max() <= 2
+    mrr = gpu.kge.eval_mrr(gpu.dev_i32(qh), gpu.dev_i32(qr), gpu.dev_i32(tt), 0)
+    assert abs(mrr - oracle64.mrr(r_ranks, 0)) <= 1e-3
+
+
 def test_config1_mrr_after_training(oracle32, oracle64):
     """BASELINE configs[0]: 10 SGD steps, then MRR of the first 100 triples ranked against
     all 1,000 entities.  Inference parity is taken on the GPU's own trained tables."""
