@@ -247,9 +247,22 @@ __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const Tc
     if (L2 && rin) p.grow_part[(int64_t)row * (2 * p.tiles_n) + (it.n0 / TC_BN) * 2 + col_off / 64] = rsum;
 }
 
+// Largest float below x (x finite or -inf; -inf maps to itself).
+__device__ __forceinline__ float float_below(float x) {
+    if (x == 0.f) return __uint_as_float(0x80000001u);
+    if (x == -INFINITY) return x;
+    const uint32_t b = __float_as_uint(x);
+    return __uint_as_float(x > 0.f ? b - 1u : b + 1u);
+}
+
 // Full-entity scoring (Section 3.1 "Inference"): a score survives into the query's candidate
 // list if it is ordered before the query's current k-th best under (score descending, entity
 // id ascending); entities ordered before the true tail are counted for its rank.
+// Within a run of 32 consecutive entity ids that does not contain the reference id, "ordered
+// before (f0, id0)" is a plain comparison: f >= f0 if the run lies below id0, f > f0 if above;
+// f >= f0 is written f > (largest float below f0).  Only the run that contains the reference
+// id takes the element-by-element form, so the common case costs a compare-and-count per score
+// for the rank and one maximum per score for the candidate test.
 __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr, int32_t* beat_sm) {
     const bool rin = row < p.M;
     float thr = 0.f, ft = 0.f; int32_t thr_id = 0, tt = -1;
@@ -257,6 +270,7 @@ __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const Tc
         thr = p.thr[row]; thr_id = p.thr_id[row];
         if (p.tt) { ft = p.ftrue[row]; tt = p.tt[row]; }
     }
+    const float thr_lo = float_below(thr), ft_lo = float_below(ft);
     int beat = 0;
 #pragma unroll 1
     for (int c0 = col_off; c0 < col_off + 64; c0 += 32) {
@@ -265,20 +279,43 @@ __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const Tc
         if (!rin) continue;
         const int ncol = it.n0 + c0;
         const int valid = min(32, p.N - ncol);
+        if (valid <= 0) continue;
         const int32_t e0 = (int32_t)(p.n_base + ncol);
+        if (valid != 32) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            if (valid != 32 && i >= valid) continue;
-            const float f = v[i];
-            const int32_t e = e0 + i;
-            if (tt >= 0 && e != tt && (f > ft || (f == ft && e < tt))) ++beat;
-            if (f > thr || (f == thr && e < thr_id)) {
-                const int slot = atomicAdd(&p.cand_cnt[row], 1);
-                if (slot < p.cand_cap) {
-                    p.cand_score[(int64_t)row * p.cand_cap + slot] = f;
-                    p.cand_id[(int64_t)row * p.cand_cap + slot] = e;
-                } else {
-                    *p.overflow = 1;   // the host redoes this chunk in pieces that cannot overflow
+            for (int i = 0; i < 32; ++i) if (i >= valid) v[i] = -INFINITY;   // never counted, never a candidate
+        }
+        // rank of the true tail
+        if (tt >= 0) {
+            if (tt < e0 || tt >= e0 + 32) {
+                const float c = tt >= e0 + 32 ? ft_lo : ft;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) beat += v[i] > c ? 1 : 0;
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int32_t e = e0 + i;
+                    if (e != tt && (v[i] > ft || (v[i] == ft && e < tt))) ++beat;
+                }
+            }
+        }
+        // candidates: anything ordered before the current k-th best
+        float vmax = v[0];
+#pragma unroll
+        for (int i = 1; i < 32; ++i) vmax = fmaxf(vmax, v[i]);
+        if (vmax > thr_lo) {   // rare once the threshold has tightened
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {     // (padded columns hold -inf and never pass)
+                const float f = v[i];
+                const int32_t e = e0 + i;
+                if (f > thr || (f == thr && e < thr_id && f != -INFINITY)) {
+                    const int slot = atomicAdd(&p.cand_cnt[row], 1);
+                    if (slot < p.cand_cap) {
+                        p.cand_score[(int64_t)row * p.cand_cap + slot] = f;
+                        p.cand_id[(int64_t)row * p.cand_cap + slot] = e;
+                    } else {
+                        *p.overflow = 1;   // the host redoes this chunk in pieces that cannot overflow
+                    }
                 }
             }
         }
