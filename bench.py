@@ -137,6 +137,27 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(value, device=None):
+    """The slowest rank's time: all-reduce MAX over the process group (identity on one rank)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_seed(rank):
+    """Sampler seed of a replica: every rank trains its own copy on its own batches."""
+    return int(rank)
+
+
+def whole_job_value(world, units_per_rank_step, ms_per_step):
+    """Throughput of all replicas together: units of all ranks over the slowest rank's step time."""
+    return world * units_per_rank_step / (ms_per_step * 1e-3)
+
+
 def measured_peaks():
     p = ROOT / "MEASURED_PEAKS.json"
     if p.exists():
@@ -239,7 +260,7 @@ def run_ours(args, w, name):
         states = [torch.zeros(w["E"], dtype=torch.float32, device=dev), torch.zeros(w["R"], dtype=torch.float32, device=dev),
                   None if relw_d is None else torch.zeros(w["R"], dtype=torch.float32, device=dev)]
     prec = K.PREC_BF16_TC if w.get("tc") else K.PREC_FP32
-    kge = K.Kge(K.KgeConfig.make(**cfg_kwargs(w, seed=rank), prec=prec))       # each replica draws its own batches
+    kge = K.Kge(K.KgeConfig.make(**cfg_kwargs(w, seed=replica_seed(rank)), prec=prec))       # each replica draws its own batches
     kge.bind(ent_d, rel_d, relw_d, *states, num_triples=w["T"])
     kge.graph_load(h, r, t)
     loss = torch.zeros(1, dtype=torch.float32, device=dev)
@@ -268,13 +289,9 @@ def run_ours(args, w, name):
     barrier()
     clock_info = clocks.stop()
     launches = kge.launch_count() - launches0
-    total_ms = float(np.sum(ms))
-    if world > 1:
-        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = tt.item()
+    total_ms = max_over_ranks(float(np.sum(ms)), dev)
     ms_per_step = total_ms / args.steps
-    value = world * B / (ms_per_step * 1e-3)
+    value = whole_job_value(world, B, ms_per_step)
     assert np.isfinite(loss.item()) and kge.get_status() == 0
 
     # ---- end to end: ids in pinned host memory -> H2D, step, loss -> D2H, every step ----
@@ -289,11 +306,8 @@ def run_ours(args, w, name):
     barrier()
     e2e_ms = float(np.sum(timed_steps(nxt, args.steps, host_fn)))
     barrier()
-    if world > 1:
-        tt = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = tt.item()
-    e2e_value = world * B / (e2e_ms / args.steps * 1e-3)
+    e2e_ms = max_over_ranks(e2e_ms, dev)
+    e2e_value = whole_job_value(world, B, e2e_ms / args.steps)
     nxt += args.steps
 
     # ---- per-kernel times (CUDA events around every launch, same stream) for the roofline ----
