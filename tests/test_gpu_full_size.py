@@ -1,0 +1,87 @@
+"""Parity at the benchmark's full table sizes, on what the oracle can afford: the rows one step
+touches.  The GPU runs the step on the whole table (10 M x 256 fp32 plus Adam state for
+configs[2]); the rows of the batch are pulled out before and after, the ids are renumbered
+densely, and the fp64 oracle runs the same step on that compact problem -- every quantity of
+the step depends on the tables only through the rows the batch names, and the sampled-softmax
+correction c is passed as a number, so the compact problem has the same answer."""
+import numpy as np
+import pytest
+
+import kge_synth
+from oracle.kge_oracle import make_config
+from parity_util import assert_close
+
+pytestmark = pytest.mark.gpu
+
+
+def _compact(ids_list, touched):
+    return [np.searchsorted(touched, ids).astype(np.int32) for ids in ids_list]
+
+
+@pytest.mark.parametrize("score", ["distmult", "complex"])
+def test_config3_full_table_step_on_touched_rows(oracle64, score):
+    import torch
+    import paper_2211_12281_b200 as K
+    dev = torch.device("cuda:0")
+    free, _ = torch.cuda.mem_get_info()
+    if free < 45e9:
+        pytest.skip("needs 45 GB of free device memory")
+    # configs[2] with a graph of 20 M triples instead of 100 M (the step never sees the graph's size)
+    E, R, T, d, B, N, P = 10_000_000, 1000, 20_000_000, 256, 4096, 16384, 8
+    lr, c = 1e-3, float(np.log((E - 1) / N))
+    kw = dict(num_entities=E, num_relations=R, dim=d, score=score, loss="softmax", opt="adam", batch=B, num_neg=N,
+              num_parts=P, ce_correction=c, lr=lr, seed=0)
+    h, r, t = kge_synth.make_graph(E, R, T, seed=2, relation_zipf=1.0)
+    gen = torch.Generator(device=dev); gen.manual_seed(7)
+    ent = torch.empty((E, d), dtype=torch.float32, device=dev).normal_(0.0, d ** -0.5, generator=gen)
+    rel = torch.empty((R, d), dtype=torch.float32, device=dev).normal_(0.0, d ** -0.5, generator=gen)
+    ent_state = torch.zeros((E, 2 * d), dtype=torch.float32, device=dev)
+    rel_state = torch.zeros((R, 2 * d), dtype=torch.float32, device=dev)
+    kge = K.Kge(K.KgeConfig.make(**kw, prec=K.PREC_BF16_TC))
+    kge.bind(ent, rel, None, ent_state, rel_state, num_triples=T)
+    kge.graph_load(h, r, t)
+
+    # the batch of step 0: sampled on the device, bit-exact against the oracle's sampler
+    bufs = [torch.empty(n, dtype=torch.int32, device=dev) for n in (B, B, B, N)]
+    kge.sample_batch(0, *bufs)
+    heads, rels, tails, negs = (b.cpu().numpy() for b in bufs)
+    graph = oracle64.graph_build(E, R, P, h, r, t)
+    want = oracle64.sample_batch(make_config(**kw), 0, graph)
+    for got, exp in zip((heads, rels, tails, negs), want):
+        assert (got == exp).all()
+    S = (E + P - 1) // P
+    assert (np.bincount(negs // S, minlength=P) == N // P).all()                       # Eq. 4
+    assert (np.bincount((heads // S) * P + tails // S, minlength=P * P) == B // (P * P)).all()   # Eq. 3
+
+    touched = np.unique(np.concatenate([heads, tails, negs]))
+    tidx = torch.from_numpy(touched.astype(np.int64)).to(dev)
+    before = ent[tidx].cpu().numpy()
+    rel_before = rel.cpu().numpy()
+    loss = torch.zeros(1, dtype=torch.float32, device=dev)
+    kge.train_step(0, lr, *bufs, loss_out=loss)
+    assert kge.get_status() == 0
+    after, m_after = ent[tidx].cpu().numpy(), ent_state[tidx].cpu().numpy()
+
+    # the same step on the compact problem, fp64, scores from bf16-rounded operands
+    ch, ct, cn = _compact([heads, tails, negs], touched)
+    ckw = dict(kw, num_entities=len(touched), num_parts=1)
+    cfg = make_config(**ckw, bf16_operands=1)
+    g = oracle64.batch_grads(cfg, before, rel_before, None, ch, rels, ct, cn)
+    e64, r64 = oracle64.arr(before).copy(), oracle64.arr(rel_before).copy()
+    es, rs = np.zeros((len(touched), 2 * d)), np.zeros((R, 2 * d))
+    loss_o = oracle64.train_step(cfg, lr, 0, e64, r64, None, es, rs, None, ch, rels, ct, cn)
+    assert_close(loss.item(), loss_o, rtol=1e-4, atol=1e-3, what="loss")
+
+    # Adam's first moment is (1 - beta1) x gradient: linear, so it carries the gradient's error
+    # bound of this path (bf16 factors in the backward contractions: 1e-2 of the largest summed
+    # magnitude); the table rows are compared where the step is well conditioned.
+    mag = np.zeros((len(touched), d))
+    np.add.at(mag, ch, np.abs(g["dh"])); np.add.at(mag, ct, np.abs(g["dtpos"])); np.add.at(mag, cn, np.abs(g["dtneg"]))
+    assert_close(m_after[:, :d], es[:, :d], rtol=1e-2, atol=0.1 * 1e-2 * mag.max(), what="first moments of the touched rows")
+    gsum = es[:, :d] / 0.1
+    well = np.abs(gsum) > 0.05 * np.abs(gsum).max()
+    assert well.sum() > 1000
+    assert_close(np.where(well, after, e64), e64, rtol=1e-4, atol=0.05 * lr, what="touched rows (well-conditioned coordinates)")
+    assert (np.abs(after - e64) <= 2.5 * lr).all()                  # an Adam step never exceeds about lr
+    untouched = torch.from_numpy(np.setdiff1d(np.arange(0, E, 997), touched)).to(dev)
+    assert (ent_state[untouched] == 0).all()                          # rows outside the batch are not written
