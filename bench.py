@@ -84,6 +84,11 @@ STAGE_OPS = {
 }
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
+# summarised in profiles/train_step_c2_transe_l1_launches.md (None once the kernel has changed since).
+NCU_TRAFFIC_BYTES = {("c2_transe_l1", "accum_q"): 5.27e6, ("c2_transe_l1", "accum_t"): 5.27e6, ("c2_transe_l1", "block"): 1.07e6}
+
+
 def cfg_kwargs(w, seed):
     c = w.get("ce_correction", 0.0)
     if c == "paper":                       # c = log((|E| - 1) / N), Section 3.1 "Loss Functions"
@@ -335,7 +340,7 @@ def run_ours(args, w, name):
         alg_ops = ops[dominant] * B * N * w["d"]
         achieved = alg_ops / (per_stage_us[dominant] * 1e-6) / 1e12
         roofline = {"bound": "alu", "kernel": dominant, "achieved": achieved, "peak": ALU_PEAK_TOPS,
-                    "unit": "TFLOP/s", "frac": achieved / ALU_PEAK_TOPS, "traffic": None,
+                    "unit": "TFLOP/s", "frac": achieved / ALU_PEAK_TOPS, "traffic": NCU_TRAFFIC_BYTES.get((name, dominant)),
                     "op": "one fp32 CUDA-core instruction per lane (FMA = 1)",
                     "peak_source": "148 SMs x 128 lanes x 1.965 GHz", "us_per_launch": per_stage_us[dominant]}
 

@@ -189,6 +189,8 @@ __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
 // ------------------------------------------------------------------------------------------
 constexpr int TB = 64, TN = 64, KC = 32, LDS = KC + 4;
 
+__device__ __forceinline__ float approx_sqrt(float x) { float r; asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+
 template <int KIND>
 __device__ __forceinline__ void pair_update(float& acc, float4 q, float4 t) {
     if (KIND == KIND_DOT) {
@@ -199,11 +201,11 @@ __device__ __forceinline__ void pair_update(float& acc, float4 q, float4 t) {
         float x;
         x = q.x - t.x; acc = fmaf(x, x, acc); x = q.y - t.y; acc = fmaf(x, x, acc);
         x = q.z - t.z; acc = fmaf(x, x, acc); x = q.w - t.w; acc = fmaf(x, x, acc);
-    } else {  // KIND_CL1
+    } else {  // KIND_CL1: one special-function square root per complex component (relative error 2^-22)
         float xr = q.x - t.x, xi = q.y - t.y;
-        acc += sqrtf(fmaf(xr, xr, xi * xi));
+        acc += approx_sqrt(fmaf(xr, xr, xi * xi));
         xr = q.z - t.z; xi = q.w - t.w;
-        acc += sqrtf(fmaf(xr, xr, xi * xi));
+        acc += approx_sqrt(fmaf(xr, xr, xi * xi));
     }
 }
 
