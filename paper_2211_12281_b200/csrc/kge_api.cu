@@ -38,7 +38,8 @@ int pick_split(int rows, int cols, int num_sms) {
 // splits as still give every SM at most one tile (or one split when there are more tiles than
 // SMs), each at least four 64-wide slices deep, at most 16, none empty.
 int pick_split_tc(int rows, int cols, int depth, int num_sms) {
-    const int tiles = ((rows + 127) / 128) * ((cols + 127) / 128);
+    const int bn = tc_backward_tile_cols(cols);
+    const int tiles = ((rows + 127) / 128) * ((cols + bn - 1) / bn);
     const int kb = (depth + 63) / 64;
     const int want = std::max(1, std::min(std::min(num_sms / tiles, std::max(1, kb / 4)), 16));
     const int per = (kb + want - 1) / want;
@@ -69,11 +70,8 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
     w.Tb = tc ? cv.take<uint16_t>(N * d) : nullptr;
     w.qn2 = tc ? cv.take<float>(B) : nullptr;
     w.tn2 = tc ? cv.take<float>(N) : nullptr;
-    const size_t ldN = (N + 7) / 8 * 8, ldB = (B + 7) / 8 * 8;
+    const size_t ldN = (N + 7) / 8 * 8;
     w.Gb = tc ? cv.take<uint16_t>(B * ldN) : nullptr;
-    w.GbT = tc ? cv.take<uint16_t>(N * ldB) : nullptr;
-    w.TbT = tc ? cv.take<uint16_t>(d * ldN) : nullptr;
-    w.QbT = tc ? cv.take<uint16_t>(d * ldB) : nullptr;
     w.Gcol = tc ? cv.take<float>(N) : nullptr;
     const size_t tiles_n = (N + 127) / 128, tiles_m = (B + 127) / 128;
     w.stat_part = tc ? cv.take<float>(B * 2 * tiles_n * 4) : nullptr;
@@ -249,16 +247,16 @@ int kge_bind(kge_handle* h, float* ent, float* rel, float* relw, float* ent_stat
     KGE_CUDA_CHECK(h, cudaMemsetAsync(h->ws.status, 0, 256, static_cast<cudaStream_t>(stream)));
     if (h->cfg.prec == KGE_PREC_BF16_TC) {
         const int64_t B = h->cfg.batch, N = h->cfg.num_neg, d = h->cfg.dim;
-        const int64_t ldN = (N + 7) / 8 * 8, ldB = (B + 7) / 8 * 8;
-        int rc = tc_make_operand_map(h, h->tm_q, h->ws.Qb, B, d, d);
-        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_t, h->ws.Tb, N, d, d);
-        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_g, h->ws.Gb, B, N, ldN);
-        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_gt, h->ws.GbT, N, B, ldB);
-        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_tt, h->ws.TbT, d, N, ldN);
-        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_qt, h->ws.QbT, d, B, ldB);
+        const int64_t ldN = (N + 7) / 8 * 8;
+        int rc = tc_make_operand_map(h, h->tm_q, h->ws.Qb, B, d, d, 128);
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_t, h->ws.Tb, N, d, d, 128);
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_g, h->ws.Gb, B, N, ldN, 128);
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_g64, h->ws.Gb, B, N, ldN, 64);
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_t64, h->ws.Tb, N, d, d, 64);
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_q64, h->ws.Qb, B, d, d, 64);
         if (rc == KGE_OK && h->ws.Eb) {
-            rc = tc_make_operand_map(h, h->tm_iq, h->ws.iqb, max_queries, d, d);
-            if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_eb, h->ws.Eb, h->cfg.num_entities, d, d);
+            rc = tc_make_operand_map(h, h->tm_iq, h->ws.iqb, max_queries, d, d, 128);
+            if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_eb, h->ws.Eb, h->cfg.num_entities, d, d, 128);
         }
         if (rc != KGE_OK) return rc;
     }

@@ -47,7 +47,7 @@ struct Workspace {
     float *Q, *What, *Tneg;                // [B,d], [B,d] (TransH), [N,d]
     float *fpos, *gpos, *Lrow;             // [B]
     uint16_t *Qb, *Tb;                     // [B,d], [N,d] bf16 copies of Q and Tneg (tensor-core scoring)
-    uint16_t *Gb, *GbT, *TbT, *QbT;        // bf16 [B,ldN], [N,ldB], [d,ldN], [d,ldB]: dL/dF and transposes (ld = size rounded up to 8)
+    uint16_t *Gb;                          // bf16 [B,ldN] dL/dF (ldN = N rounded up to 8)
     float *Gcol;                           // [N] column sums of dL/dF (TransE p=2 on tensor cores)
     float *stat_part, *row_stat;           // [B, 2*tiles_n, 4], [B, 2] loss statistics of the fused tensor-core forward
     float *grow_part, *gcol_part;          // [B, 2*tiles_n], [4*tiles_m, N] partial sums of dL/dF
@@ -108,8 +108,9 @@ struct kge_handle {
     int num_sms;
     // Side streams and events of the training step: the sort of the touched ids and one of the
     // two backward accumulations run beside the main stream's kernels (created by kge_bind).
-    // TMA tensor maps (tensor-core path): Qb, Tb for the scores; Gb, Tb^T for dQ; Gb^T, Qb^T for dT
-    alignas(64) unsigned char tm_q[128], tm_t[128], tm_g[128], tm_gt[128], tm_tt[128], tm_qt[128];
+    // TMA tensor maps (tensor-core path): Qb, Tb (128-row boxes) for the scores; Gb (128-row boxes) and Tb (64-row boxes,
+    // read MN-major) for dQ; Gb and Qb (64-row boxes, read MN-major) for dT
+    alignas(64) unsigned char tm_q[128], tm_t[128], tm_g[128], tm_g64[128], tm_t64[128], tm_q64[128];
     alignas(64) unsigned char tm_iq[128], tm_eb[128];   // inference: bf16 query vectors and bf16 entity table
     bool streams_ready;
     cudaStream_t side[2];
@@ -159,7 +160,8 @@ int launch_dedup(kge_handle* h, const int32_t* heads, const int32_t* rels, const
 // Segment sums of the gradient rows and the optimiser step (needs both of the above).
 int launch_update(kge_handle* h, uint64_t step, float lr, cudaStream_t s);
 // Tensor-core score block: F from the bf16 operand copies; tensor maps are made at bind time.
-int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols, int64_t ld);
+int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows);
+int tc_backward_tile_cols(int cols);
 int launch_tc_backward(kge_handle* h, cudaStream_t s, cudaStream_t side);
 int launch_tc_forward(kge_handle* h, cudaStream_t s);
 int launch_cast_bf16(kge_handle* h, const float* src, uint16_t* dst, int64_t count, cudaStream_t s);

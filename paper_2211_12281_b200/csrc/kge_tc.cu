@@ -32,11 +32,11 @@ constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 64;      // BK bf16 = one 128-by
 constexpr int TC_STAGES = 4;
 constexpr int TC_EPI_WARPS = 8;                           // two per tensor-memory lane quarter, 64 columns each
 constexpr int TC_THREADS = 32 * (2 + TC_EPI_WARPS);
-constexpr uint32_t TC_A_BYTES = TC_BM * TC_BK * 2, TC_B_BYTES = TC_BN * TC_BK * 2;
-constexpr uint32_t TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
-constexpr size_t TC_SMEM_BYTES = 1024 + (size_t)TC_STAGES * TC_STAGE_BYTES + 128;
+constexpr uint32_t TC_A_BYTES = TC_BM * TC_BK * 2;
+constexpr uint32_t TC_MN_GROUP_BYTES = 64 * TC_BK * 2;    // MN-major operand: 64 contiguous elements x 64 K rows per TMA box
+__host__ __device__ constexpr uint32_t tc_stage_bytes(int bn) { return TC_A_BYTES + (uint32_t)bn * TC_BK * 2; }
+__host__ __device__ constexpr size_t tc_smem_bytes(int bn) { return 1024 + (size_t)TC_STAGES * tc_stage_bytes(bn) + 128; }
 constexpr int TC_BEAT_ROWS_MAX = 20 * 1024;                // queries whose rank counts fit in shared memory beside the stages
-constexpr uint32_t TC_TMEM_COLS = 256;                    // two fp32 accumulators of 128 columns, used in turn
 
 enum { EPI_STORE = 0, EPI_STATS = 1, EPI_GRAD = 2, EPI_TOPK = 3, EPI_L2 = 4, EPI_CE = 8 };   // L2 / CE: flags of the fused loss epilogues
 
@@ -44,6 +44,7 @@ struct TcGemmParams {
     int M, N, K;
     int kb_per_split;                     // 64-wide slices of K per split
     int tiles_m, tiles_n, items;          // items = splits * tiles_m * tiles_n
+    int bn;                               // columns per tile (128 or 256)
     float* C; int64_t ldc;
     int64_t split_stride;                 // floats between the output slabs of consecutive K splits
     const float *row_norm2, *col_norm2;   // norm expansion: |q_b|^2 [M], |t_n|^2 [N]
@@ -54,7 +55,6 @@ struct TcGemmParams {
     float4* stat_part;                    // [M, 2 * tiles_n] per 64-column piece: (max, sum exp, weighted loss sum, -)
     const float2* row_stat;               // [M] (max, 1 / normaliser) of the whole row
     uint16_t* Gb; int64_t ldg;            // [M, ldg] bf16 dL/dF (divided by the distance for l2)
-    uint16_t* GbT; int64_t ldgt;          // [N, ldgt] its transpose
     float* grow_part;                     // [M, 2 * tiles_n] sums of the written values per 64-column piece
     float* gcol_part;                     // [4 * tiles_m, N] sums per 32-row piece (l2 only)
     // full-entity scoring (EPI_TOPK): rows are queries, columns the entities [n_base, n_base + N)
@@ -87,9 +87,24 @@ __device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t smem_addr) {
     return d;
 }
 
-// Instruction descriptor: D fp32, A and B bf16, both K-major, M x N tile.
-__host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+// The same for an operand whose M (or N) index is the contiguous one ("MN-major"), as TMA leaves
+// it from boxes of 64 contiguous elements x 64 K rows: inside a box a K row is 128 bytes, groups
+// of 8 K rows are 1024 bytes apart (stride offset), the next 64 elements of M / N are one box
+// (8192 bytes) further (leading offset).
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(TC_MN_GROUP_BYTES >> 4) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// Instruction descriptor: D fp32, A and B bf16, M x N tile; a_mn / b_mn: that operand is MN-major.
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n, bool a_mn = false, bool b_mn = false) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
@@ -185,7 +200,7 @@ __device__ __forceinline__ uint16_t bf16_bits(float v) {
 __device__ __forceinline__ float bf16_value(uint16_t bits) { return __uint_as_float((uint32_t)bits << 16); }
 
 // Second pass: dL/dF from the recomputed score and the row's final (base-2 max, 1 / normaliser),
-// written as bf16 in both orientations for the two backward contractions.
+// written as bf16 for the two backward contractions (which read it K-major and MN-major).
 template <bool L2, bool CE>
 __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr) {
     const bool rin = row < p.M;
@@ -228,10 +243,6 @@ __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const Tc
 #pragma unroll
                 for (int i = 0; i < 32; ++i) if (i < valid) dst[i] = (uint16_t)(g2[i >> 1] >> ((i & 1) * 16));
             }
-            uint16_t* dt = p.GbT + (int64_t)ncol * p.ldgt + row;
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-                if (valid == 32 || i < valid) dt[(int64_t)i * p.ldgt] = (uint16_t)(g2[i >> 1] >> ((i & 1) * 16));
         }
         if (L2) {   // the norm expansion also needs the sums of what the contractions will see
 #pragma unroll
@@ -325,16 +336,17 @@ __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const Tc
     }
 }
 
-// Epilogue of one warp on one item: 64 columns [col_off, col_off + 64) of the tile row held by
+// Epilogue of one warp on one item: WIDTH columns [col_off, col_off + WIDTH) of the tile row held by
 // this thread's tensor-memory lane (taddr points at the first of them).
-template <int EPI>
+template <int EPI, int WIDTH>
 __device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr, int32_t* beat_sm) {
+    static_assert((EPI & 3) == EPI_STORE || WIDTH == 64, "the fused epilogues work on 64-column pieces");
     if ((EPI & 3) == EPI_STATS) { tc_epilogue_stats<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, col_off, taddr); return; }
     if ((EPI & 3) == EPI_TOPK) { tc_epilogue_topk(p, it, row, col_off, taddr, beat_sm); return; }
     if ((EPI & 3) == EPI_GRAD) { tc_epilogue_grad<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, col_off, taddr); return; }
     float* const Cout = p.C + (int64_t)it.z * p.split_stride;
 #pragma unroll 1
-    for (int c0 = col_off; c0 < col_off + 64; c0 += 32) {
+    for (int c0 = col_off; c0 < col_off + WIDTH; c0 += 32) {
         float v[32];
         tmem_ld32(taddr + (uint32_t)(c0 - col_off), v);
         if (row >= p.M) continue;
@@ -354,14 +366,19 @@ __device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem&
 // Work item = (K split, row tile, column tile), column tile fastest.  A CTA takes a contiguous
 // run of items, so consecutive items mostly share their A rows (kept warm in L2).
 __device__ __forceinline__ TcItem tc_item(const TcGemmParams& p, int64_t item) {
-    if (p.m_fastest) return TcItem{0, (int)(item % p.tiles_m) * TC_BM, (int)(item / p.tiles_m) * TC_BN};
+    if (p.m_fastest) return TcItem{0, (int)(item % p.tiles_m) * TC_BM, (int)(item / p.tiles_m) * p.bn};
     const int tn = (int)(item % p.tiles_n), r = (int)(item / p.tiles_n);
-    return TcItem{r / p.tiles_m, (r % p.tiles_m) * TC_BM, tn * TC_BN};
+    return TcItem{r / p.tiles_m, (r % p.tiles_m) * TC_BM, tn * p.bn};
 }
 
-template <int EPI>
+// BN: columns per tile (128, or 256 for the backward contractions of wide rows); A_MN / B_MN:
+// the operand is read MN-major (its tensor map has the contraction index as rows), which is how
+// dL/dF, Q and T serve as transposed operands without a transposed copy.
+template <int EPI, int BN = 128, bool A_MN = false, bool B_MN = false>
 __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
                                                              const __grid_constant__ CUtensorMap tmB, TcGemmParams p) {
+    constexpr uint32_t TC_STAGE_BYTES = tc_stage_bytes(BN);
+    constexpr uint32_t TC_TMEM_COLS = 2 * BN;          // two fp32 accumulators, used in turn
     extern __shared__ unsigned char tc_smem_raw[];
     unsigned char* base = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
     uint64_t* full = reinterpret_cast<uint64_t*>(base + (size_t)TC_STAGES * TC_STAGE_BYTES);
@@ -405,14 +422,28 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
                     if (!mbar_wait_bounded(&empty[s], ((ring / TC_STAGES) & 1) ^ 1)) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); break; }
                     unsigned char* sa = base + (size_t)s * TC_STAGE_BYTES;
                     mbar_arrive_expect_tx(&full[s], TC_STAGE_BYTES);
-                    tma_load_2d(sa, &tmA, (kb0 + kb) * TC_BK, it.m0, &full[s]);
-                    tma_load_2d(sa + TC_A_BYTES, &tmB, (kb0 + kb) * TC_BK, (int)p.n_base + it.n0, &full[s]);
+                    const int k0 = (kb0 + kb) * TC_BK;
+                    if (A_MN) {
+#pragma unroll
+                        for (int g = 0; g < TC_BM / 64; ++g) tma_load_2d(sa + g * TC_MN_GROUP_BYTES, &tmA, it.m0 + 64 * g, k0, &full[s]);
+                    } else {
+                        tma_load_2d(sa, &tmA, k0, it.m0, &full[s]);
+                    }
+                    unsigned char* sb = sa + TC_A_BYTES;
+                    if (B_MN) {
+#pragma unroll
+                        for (int g = 0; g < BN / 64; ++g) tma_load_2d(sb + g * TC_MN_GROUP_BYTES, &tmB, it.n0 + 64 * g, k0, &full[s]);
+                    } else {
+#pragma unroll
+                        for (int g = 0; g < BN / 128; ++g)   // boxes of 128 rows, one after the other
+                            tma_load_2d(sb + g * (128 * TC_BK * 2), &tmB, k0, (int)p.n_base + it.n0 + 128 * g, &full[s]);
+                    }
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(TC_BM, TC_BN);
+            constexpr uint32_t idesc = umma_idesc_bf16(TC_BM, BN, A_MN, B_MN);
             int ring = 0;
             bool ok = true;
             for (int item = item_begin, local = 0; item < item_end && ok && !*stop; ++item, ++local) {
@@ -422,16 +453,18 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
                 // the epilogue warps must have drained this buffer (two items ago)
                 if (!mbar_wait_bounded(&acc_empty[buf], ((local >> 1) & 1) ^ 1)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t tmem_acc = tmem_base + (uint32_t)buf * TC_BN;
+                const uint32_t tmem_acc = tmem_base + (uint32_t)buf * BN;
                 for (int kb = 0; kb < nkb; ++kb, ++ring) {
                     const int s = ring % TC_STAGES;
                     if (!mbar_wait_bounded(&full[s], (ring / TC_STAGES) & 1)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = smem_u32(base + (size_t)s * TC_STAGE_BYTES);
 #pragma unroll
-                    for (int k = 0; k < TC_BK / 16; ++k)   // one MMA covers 16 bf16 = 32 bytes of K
-                        umma_bf16(tmem_acc, umma_desc_k_sw128(sa + k * 32), umma_desc_k_sw128(sa + TC_A_BYTES + k * 32),
-                                  idesc, (kb | k) != 0);
+                    for (int k = 0; k < TC_BK / 16; ++k) {   // one MMA covers 16 of K: 32 bytes of a K-major row, 16 rows MN-major
+                        const uint64_t ad = A_MN ? umma_desc_mn_sw128(sa + k * 2048) : umma_desc_k_sw128(sa + k * 32);
+                        const uint64_t bd = B_MN ? umma_desc_mn_sw128(sa + TC_A_BYTES + k * 2048) : umma_desc_k_sw128(sa + TC_A_BYTES + k * 32);
+                        umma_bf16(tmem_acc, ad, bd, idesc, (kb | k) != 0);
+                    }
                     umma_commit(&empty[s]);            // the stage is free once these MMAs have read it
                 }
                 umma_commit(&acc_full[buf]);           // also after a failed wait, so the epilogue warps wake up
@@ -440,15 +473,15 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
         }
     } else {
         const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
-        const int chalf = (warp - 2) >> 2;             // which 64 of the 128 columns
+        const int chalf = (warp - 2) >> 2;             // which half of the tile's columns
         for (int item = item_begin, local = 0; item < item_end; ++item, ++local) {
             const int buf = local & 1;
             const bool ok = mbar_wait_bounded(&acc_full[buf], (local >> 1) & 1);
             tc_fence_after();
             if (!ok || *stop) { if (lane == 0) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); } break; }
             const TcItem it = tc_item(p, item);
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * TC_BN + chalf * 64);
-            tc_epilogue<EPI>(p, it, it.m0 + quarter * 32 + lane, chalf * 64, taddr, beat_sm);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + chalf * (BN / 2));
+            tc_epilogue<EPI, BN / 2>(p, it, it.m0 + quarter * 32 + lane, chalf * (BN / 2), taddr, beat_sm);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
@@ -460,56 +493,6 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
     if ((EPI & 3) == EPI_TOPK)     // hand this CTA's rank counts over (integer adds: the result does not depend on the order)
         for (int i = threadIdx.x; i < p.beat_rows; i += TC_THREADS) { const int32_t b = beat_sm[i]; if (b) atomicAdd(&p.beat_tmp[i], b); }
-}
-
-// src fp32 [R, C] (leading dimension lds) -> bf16 copies for the backward contractions:
-// dst_rm [R, ld_rm] as it is (optional) and dst_t [C, ld_t] transposed; colsum[C] (optional)
-// = column sums of src, added in ascending row order.  A CTA owns 32 columns and walks the
-// rows of its blockIdx.y share in tiles of 32.
-struct CastParams {
-    const float* src; int64_t lds;
-    int R, C, rows_per_cta;
-    uint16_t* dst_rm; int64_t ld_rm;
-    uint16_t* dst_t; int64_t ld_t;
-    float* colsum;
-};
-
-__global__ void __launch_bounds__(256) cast_transpose_kernel(CastParams p) {
-    __shared__ float tile[32][33];
-    __shared__ float csm[8][32];
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    const int c0 = blockIdx.x * 32;
-    const int r_begin = blockIdx.y * p.rows_per_cta, r_end = min(p.R, r_begin + p.rows_per_cta);
-    float cs = 0.f;
-    for (int r0 = r_begin; r0 < r_end; r0 += 32) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int r = r0 + ty + 8 * i, c = c0 + tx;
-            float v = 0.f;
-            if (r < r_end && c < p.C) {
-                v = p.src[(int64_t)r * p.lds + c];
-                if (p.dst_rm) p.dst_rm[(int64_t)r * p.ld_rm + c] = bf16_bits(v);
-            }
-            tile[ty + 8 * i][tx] = v;
-            cs += v;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int c = c0 + ty + 8 * i, r = r0 + tx;
-            if (c < p.C && r < r_end) p.dst_t[(int64_t)c * p.ld_t + r] = bf16_bits(tile[tx][ty + 8 * i]);
-        }
-        __syncthreads();
-    }
-    if (p.colsum) {   // thread (tx, ty) has summed rows ty, ty + 8, ... of column tx: add the 8 partial sums in order
-        csm[ty][tx] = cs;
-        __syncthreads();
-        if (ty == 0 && c0 + tx < p.C) {
-            float t = 0.f;
-            for (int w = 0; w < 8; ++w) t += csm[w][tx];
-            p.colsum[c0 + tx] = t;
-        }
-    }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -531,14 +514,15 @@ EncodeTiledFn encode_tiled_fn() {
 }  // namespace
 
 // Tensor map of a row-major bf16 matrix [rows, cols] with leading dimension ld (ld % 8 == 0,
-// base 16-byte aligned) read in boxes of 128 rows x 64 columns with the 128-byte swizzle;
-// what a box covers beyond the matrix reads as zero.
-int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols, int64_t ld) {
+// base 16-byte aligned) read in boxes of box_rows rows x 64 columns with the 128-byte swizzle
+// (128 rows for a K-major operand tile, 64 for an MN-major one); what a box covers beyond the
+// matrix reads as zero.
+int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) { h->cuda_err = "cuTensorMapEncodeTiled is not available from this driver"; return KGE_ERR_CUDA; }
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)TC_BM};
+    const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = fn(static_cast<CUtensorMap*>(map_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
                           dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -612,17 +596,19 @@ __global__ void __launch_bounds__(256) grad_sums_kernel(const float* grow_part, 
 }  // namespace
 
 namespace {
-template <int EPI>
+template <int EPI, int BN = 128, bool A_MN = false, bool B_MN = false>
 cudaError_t launch_gemm_inst(const unsigned char* tmA, const unsigned char* tmB, const TcGemmParams& p, int num_sms, cudaStream_t s,
                              size_t extra_smem = 0) {
+    constexpr size_t smem = tc_smem_bytes(BN);
+    constexpr size_t extra_max = (EPI & 3) == EPI_TOPK ? (size_t)TC_BEAT_ROWS_MAX * 4 : 0;
     static bool configured = false;
     if (!configured) {
-        const cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)(TC_SMEM_BYTES + TC_BEAT_ROWS_MAX * 4));
+        const cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<EPI, BN, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)(smem + extra_max));
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    tc_gemm_kernel<EPI><<<std::min(p.items, num_sms), TC_THREADS, TC_SMEM_BYTES + extra_smem, s>>>(
+    tc_gemm_kernel<EPI, BN, A_MN, B_MN><<<std::min(p.items, num_sms), TC_THREADS, smem + extra_smem, s>>>(
         *reinterpret_cast<const CUtensorMap*>(tmA), *reinterpret_cast<const CUtensorMap*>(tmB), p);
     return cudaSuccess;
 }
@@ -652,6 +638,7 @@ int launch_tc_forward(kge_handle* h, cudaStream_t s) {
     TcGemmParams p{};
     p.M = c.batch; p.N = c.num_neg; p.K = c.dim;
     p.kb_per_split = (p.K + TC_BK - 1) / TC_BK; p.split_stride = 0;
+    p.bn = TC_BN;
     p.tiles_m = (p.M + TC_BM - 1) / TC_BM; p.tiles_n = (p.N + TC_BN - 1) / TC_BN; p.items = p.tiles_m * p.tiles_n;
     p.C = nullptr; p.ldc = 0;
     p.row_norm2 = w.qn2; p.col_norm2 = w.tn2;
@@ -660,7 +647,6 @@ int launch_tc_forward(kge_handle* h, cudaStream_t s) {
     p.gamma = c.gamma; p.adv_temp = c.adv_temp; p.ce_c = c.ce_correction; p.loss_scale = c.loss_scale;
     p.stat_part = reinterpret_cast<float4*>(w.stat_part); p.row_stat = reinterpret_cast<const float2*>(w.row_stat);
     p.Gb = w.Gb; p.ldg = (c.num_neg + 7) / 8 * 8;
-    p.GbT = w.GbT; p.ldgt = (c.batch + 7) / 8 * 8;
     p.grow_part = w.grow_part; p.gcol_part = w.gcol_part;
     const bool ce = c.loss == KGE_LOSS_SAMPLED_SOFTMAX;
     stage_begin(h, ST_BLOCK, s);
@@ -684,69 +670,49 @@ int launch_tc_forward(kge_handle* h, cudaStream_t s) {
 }
 
 namespace {
-int launch_cast(kge_handle* h, const float* src, int64_t lds, int R, int C, uint16_t* dst_rm, int64_t ld_rm,
-                uint16_t* dst_t, int64_t ld_t, float* colsum, cudaStream_t s) {
-    CastParams cp{src, lds, R, C, R, dst_rm, ld_rm, dst_t, ld_t, colsum};
-    int row_ctas = 1;
-    if (!colsum) {   // no column sums: the rows may be shared out to fill the device
-        const int col_ctas = (C + 31) / 32;
-        row_ctas = std::max(1, std::min((R + 31) / 32, (2 * h->num_sms + col_ctas - 1) / col_ctas));
-        cp.rows_per_cta = ((R + row_ctas - 1) / row_ctas + 31) / 32 * 32;
-        row_ctas = (R + cp.rows_per_cta - 1) / cp.rows_per_cta;
-    }
-    cast_transpose_kernel<<<dim3((C + 31) / 32, row_ctas), 256, 0, s>>>(cp);
-    KGE_LAUNCH_CHECK(h);
-    return KGE_OK;
-}
-
-int launch_tc_gemm(kge_handle* h, const unsigned char* tmA, const unsigned char* tmB, int M, int N, int K, int split,
-                   float* C, int64_t ldc, cudaStream_t s) {
+// One backward contraction C[M, N] (+ K splits) with the tile width that fits the row width.
+template <bool A_MN>
+int launch_tc_bwd_gemm(kge_handle* h, const unsigned char* tmA, const unsigned char* tmB, int M, int N, int K, int split,
+                       float* C, int64_t ldc, cudaStream_t s) {
     TcGemmParams p{};
     p.M = M; p.N = N; p.K = K;
     const int kb = (K + TC_BK - 1) / TC_BK;
     p.kb_per_split = (kb + split - 1) / split;
     p.C = C; p.ldc = ldc; p.split_stride = (int64_t)M * ldc;
-    p.row_norm2 = p.col_norm2 = nullptr;
     p.status = h->ws.status;
-    p.tiles_m = (M + TC_BM - 1) / TC_BM; p.tiles_n = (N + TC_BN - 1) / TC_BN;
+    p.bn = tc_backward_tile_cols(N);
+    p.tiles_m = (M + TC_BM - 1) / TC_BM; p.tiles_n = (N + p.bn - 1) / p.bn;
     p.items = p.tiles_m * p.tiles_n * ((kb + p.kb_per_split - 1) / p.kb_per_split);
-    KGE_CUDA_CHECK(h, launch_gemm_inst<EPI_STORE>(tmA, tmB, p, h->num_sms, s));
+    if (p.bn == 256) KGE_CUDA_CHECK(h, (launch_gemm_inst<EPI_STORE, 256, A_MN, true>(tmA, tmB, p, h->num_sms, s)));
+    else KGE_CUDA_CHECK(h, (launch_gemm_inst<EPI_STORE, 128, A_MN, true>(tmA, tmB, p, h->num_sms, s)));
     KGE_LAUNCH_CHECK(h);
     return KGE_OK;
 }
 }  // namespace
 
-// The two backward contractions on tensor cores, from the bf16 dL/dF the forward left behind:
-//   dQ partial[split] = G . T      (A = Gb [B, N],   B operand = Tb^T [d, N])
-//   dT partial[split] = G^T . Q    (A = Gb^T [N, B], B operand = Qb^T [d, B])
+// Columns per tile of a backward contraction whose output rows are `cols` wide.
+int tc_backward_tile_cols(int cols) { return cols > 128 ? 256 : 128; }
+
+// The two backward contractions on tensor cores, from the bf16 dL/dF the forward left behind.
+// No operand is transposed in memory: an operand whose contraction index is its row index is
+// read MN-major.
+//   dQ partial[split] = G . T      A = Gb [B, N] (K-major),          B operand = Tb [N, d] (MN-major)
+//   dT partial[split] = G^T . Q    A = Gb [B, N] read MN-major,      B operand = Qb [B, d] (MN-major)
 // The K splits land in the same partial buffers the CUDA-core path uses and are added in
-// ascending order by the chain kernel.  With a side stream the dQ contraction runs beside dT.
+// ascending order by the chain kernel.
 int launch_tc_backward(kge_handle* h, cudaStream_t s, cudaStream_t side) {
     const kge_config& c = h->cfg;
     Workspace& w = h->ws;
     const int B = c.batch, N = c.num_neg, d = c.dim;
-    const int64_t ldN = (N + 7) / 8 * 8, ldB = (B + 7) / 8 * 8;
-    int rc;
-    stage_begin(h, ST_TH_CPASS, s);   // stage slot shared with the TransH pass: operand casts
-    if ((rc = launch_cast(h, w.Tneg, d, N, d, nullptr, 0, w.TbT, ldN, nullptr, s)) != KGE_OK) return rc;
-    if ((rc = launch_cast(h, w.Q, d, B, d, nullptr, 0, w.QbT, ldB, nullptr, s)) != KGE_OK) return rc;
-    stage_end(h, ST_TH_CPASS, s);
-    if (side) {
-        KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_loss, s));
-        KGE_CUDA_CHECK(h, cudaStreamWaitEvent(side, h->ev_loss, 0));
-    }
-    cudaStream_t sq = side ? side : s;
-    stage_begin(h, ST_ACCUM_Q, sq);
-    rc = launch_tc_gemm(h, h->tm_g, h->tm_tt, B, d, N, h->split_q, w.dQpart, d, sq);
-    stage_end(h, ST_ACCUM_Q, sq);
+    (void)side;   // both contractions are persistent kernels that fill the device: run them in order
+    stage_begin(h, ST_ACCUM_Q, s);
+    int rc = launch_tc_bwd_gemm<false>(h, h->tm_g, h->tm_t64, B, d, N, h->split_q, w.dQpart, d, s);
+    stage_end(h, ST_ACCUM_Q, s);
     if (rc != KGE_OK) return rc;
-    if (side) KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_t, side));
     stage_begin(h, ST_ACCUM_T, s);
-    rc = launch_tc_gemm(h, h->tm_gt, h->tm_qt, N, d, B, h->split_t, w.dTpart, d, s);
+    rc = launch_tc_bwd_gemm<true>(h, h->tm_g64, h->tm_q64, N, d, B, h->split_t, w.dTpart, d, s);
     stage_end(h, ST_ACCUM_T, s);
-    if (rc != KGE_OK) return rc;
-    if (side) KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_t, 0));
-    return KGE_OK;
+    return rc;
 }
 
 
@@ -776,6 +742,7 @@ int launch_tc_infer_chunk(kge_handle* h, int nq, int64_t e_lo, int64_t e_hi, con
     TcGemmParams p{};
     p.M = nq; p.N = (int)(e_hi - e_lo); p.K = h->cfg.dim;
     p.kb_per_split = (p.K + TC_BK - 1) / TC_BK;
+    p.bn = TC_BN;
     p.tiles_m = (p.M + TC_BM - 1) / TC_BM; p.tiles_n = (p.N + TC_BN - 1) / TC_BN;
     if ((int64_t)p.tiles_m * p.tiles_n > 0x7fffffff) return KGE_ERR_BAD_ARG;
     p.items = p.tiles_m * p.tiles_n;
