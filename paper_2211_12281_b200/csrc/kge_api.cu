@@ -74,9 +74,9 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
     w.Gb = tc ? cv.take<uint16_t>(B * ldN) : nullptr;
     w.Gcol = tc ? cv.take<float>(N) : nullptr;
     const size_t tiles_n = (N + 127) / 128, tiles_m = (B + 127) / 128;
-    w.stat_part = tc ? cv.take<float>(B * 2 * tiles_n * 4) : nullptr;
+    w.stat_part = tc ? cv.take<float>(B * tc_pieces_per_tile() * tiles_n * 4) : nullptr;
     w.row_stat = tc ? cv.take<float>(B * 2) : nullptr;
-    w.grow_part = tc ? cv.take<float>(B * 2 * tiles_n) : nullptr;
+    w.grow_part = tc ? cv.take<float>(B * tc_pieces_per_tile() * tiles_n) : nullptr;
     w.gcol_part = tc ? cv.take<float>(4 * tiles_m * N) : nullptr;
     w.Grow = cv.take<float>(B);
     w.Cpart = cv.take<float>((size_t)h->split_t * N);

@@ -49,8 +49,8 @@ struct Workspace {
     uint16_t *Qb, *Tb;                     // [B,d], [N,d] bf16 copies of Q and Tneg (tensor-core scoring)
     uint16_t *Gb;                          // bf16 [B,ldN] dL/dF (ldN = N rounded up to 8)
     float *Gcol;                           // [N] column sums of dL/dF (TransE p=2 on tensor cores)
-    float *stat_part, *row_stat;           // [B, 2*tiles_n, 4], [B, 2] loss statistics of the fused tensor-core forward
-    float *grow_part, *gcol_part;          // [B, 2*tiles_n], [4*tiles_m, N] partial sums of dL/dF
+    float *stat_part, *row_stat;           // [B, pieces, 4], [B, 2] loss statistics of the fused tensor-core forward
+    float *grow_part, *gcol_part;          // [B, pieces], [4*tiles_m, N] partial sums of dL/dF
     float *qn2, *tn2;                      // [B], [N] squared norms of the fp32 rows (TransE p=2 by norm expansion)
     float *Grow;                           // [B] row sums of dL/dF (TransE p=1 backward)
     float *Cpart;                          // [St, N] column sums of dL/dF per row split (TransE p=1 backward)
@@ -162,6 +162,7 @@ int launch_update(kge_handle* h, uint64_t step, float lr, cudaStream_t s);
 // Tensor-core score block: F from the bf16 operand copies; tensor maps are made at bind time.
 int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows);
 int tc_backward_tile_cols(int cols);
+int tc_pieces_per_tile();
 int launch_tc_backward(kge_handle* h, cudaStream_t s, cudaStream_t side);
 int launch_tc_forward(kge_handle* h, cudaStream_t s);
 int launch_cast_bf16(kge_handle* h, const float* src, uint16_t* dst, int64_t count, cudaStream_t s);

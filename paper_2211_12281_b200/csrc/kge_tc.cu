@@ -5,9 +5,9 @@
 //
 // Persistent CTAs (one per SM) each walk a run of 128 x 128 output tiles.  Warp 0 feeds a ring of
 // shared-memory stages with TMA (one elected lane), warp 1 issues the MMAs (one elected lane)
-// into one of two accumulators in tensor memory and owns the allocation, warps 2-9 drain the
-// other accumulator meanwhile (a warp may only touch the 32 lanes of its own quarter; two warps
-// share a quarter, 64 columns each) and apply the epilogue:
+// into one of two accumulators in tensor memory and owns the allocation, warps 2-17 drain the
+// other accumulator meanwhile (a warp may only touch the 32 lanes of its own quarter; four warps
+// share a quarter, a quarter of the columns each) and apply the epilogue:
 //   EPI_STORE   C = acc (the backward contractions)
 //   EPI_STATS   no score leaves the chip: per row and 64-column piece the running maximum, the sum
 //               of exponentials and the weighted loss sum of Section 3.1 "Loss Functions"; the
@@ -30,8 +30,12 @@ namespace {
 
 constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 64;      // BK bf16 = one 128-byte swizzle row
 constexpr int TC_STAGES = 4;
-constexpr int TC_EPI_WARPS = 8;                           // two per tensor-memory lane quarter, 64 columns each
-constexpr int TC_THREADS = 32 * (2 + TC_EPI_WARPS);
+constexpr int TC_EPI_WARPS = 8;                           // epilogue warps of the training kernels: TC_EPI_GROUPS per tensor-memory lane quarter
+constexpr int TC_EPI_WARPS_TOPK = 16;                     // the filter epilogue of full-entity scoring profits from more
+constexpr int TC_EPI_GROUPS = TC_EPI_WARPS / 4;
+constexpr int TC_PIECE = TC_BN / TC_EPI_GROUPS;           // columns of a 128-wide tile per piece of loss statistics
+__host__ __device__ constexpr int tc_epi_warps(int epi) { return (epi & 3) == 3 ? TC_EPI_WARPS_TOPK : TC_EPI_WARPS; }   // 3 = EPI_TOPK
+__host__ __device__ constexpr int tc_threads(int epi) { return 32 * (2 + tc_epi_warps(epi)); }
 constexpr uint32_t TC_A_BYTES = TC_BM * TC_BK * 2;
 constexpr uint32_t TC_MN_GROUP_BYTES = 64 * TC_BK * 2;    // MN-major operand: 64 contiguous elements x 64 K rows per TMA box
 __host__ __device__ constexpr uint32_t tc_stage_bytes(int bn) { return TC_A_BYTES + (uint32_t)bn * TC_BK * 2; }
@@ -52,10 +56,10 @@ struct TcGemmParams {
     // fused loss epilogues (EPI_STATS, EPI_GRAD): the score is acc, or for l2 != 0 the distance score above
     int l2, loss;
     float gamma, adv_temp, ce_c, loss_scale;
-    float4* stat_part;                    // [M, 2 * tiles_n] per 64-column piece: (max, sum exp, weighted loss sum, -)
+    float4* stat_part;                    // [M, pieces] per column piece of a tile: (max, sum exp, weighted loss sum, -)
     const float2* row_stat;               // [M] (max, 1 / normaliser) of the whole row
     uint16_t* Gb; int64_t ldg;            // [M, ldg] bf16 dL/dF (divided by the distance for l2)
-    float* grow_part;                     // [M, 2 * tiles_n] sums of the written values per 64-column piece
+    float* grow_part;                     // [M, pieces] sums of the written values per column piece
     float* gcol_part;                     // [4 * tiles_m, N] sums per 32-row piece (l2 only)
     // full-entity scoring (EPI_TOPK): rows are queries, columns the entities [n_base, n_base + N)
     int m_fastest;                        // walk the row tiles of one column tile first (the column tile stays in L2)
@@ -167,7 +171,7 @@ __device__ __forceinline__ void tc_epilogue_stats(const TcGemmParams& p, const T
     const float k1 = CE ? kLog2e : p.adv_temp * kLog2e, k0 = CE ? p.ce_c * kLog2e : 0.f;
     float m = -INFINITY, z = 0.f, l = 0.f;
 #pragma unroll 1
-    for (int c0 = col_off; c0 < col_off + 64; c0 += 32) {
+    for (int c0 = col_off; c0 < col_off + TC_PIECE; c0 += 32) {
         float v[32];
         tmem_ld32(taddr + (uint32_t)(c0 - col_off), v);
         if (row >= p.M) continue;
@@ -190,7 +194,7 @@ __device__ __forceinline__ void tc_epilogue_stats(const TcGemmParams& p, const T
         }
     }
     if (row < p.M)
-        p.stat_part[(int64_t)row * (2 * p.tiles_n) + (it.n0 / TC_BN) * 2 + col_off / 64] = make_float4(m, z, l, 0.f);
+        p.stat_part[(int64_t)row * (TC_EPI_GROUPS * p.tiles_n) + (it.n0 / TC_BN) * TC_EPI_GROUPS + col_off / TC_PIECE] = make_float4(m, z, l, 0.f);
 }
 
 __device__ __forceinline__ uint16_t bf16_bits(float v) {
@@ -211,7 +215,7 @@ __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const Tc
     const int lane = threadIdx.x & 31;
     float rsum = 0.f;
 #pragma unroll 1
-    for (int c0 = col_off; c0 < col_off + 64; c0 += 32) {
+    for (int c0 = col_off; c0 < col_off + TC_PIECE; c0 += 32) {
         float v[32];
         tmem_ld32(taddr + (uint32_t)(c0 - col_off), v);
         const int ncol = it.n0 + c0;
@@ -255,7 +259,7 @@ __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const Tc
             }
         }
     }
-    if (L2 && rin) p.grow_part[(int64_t)row * (2 * p.tiles_n) + (it.n0 / TC_BN) * 2 + col_off / 64] = rsum;
+    if (L2 && rin) p.grow_part[(int64_t)row * (TC_EPI_GROUPS * p.tiles_n) + (it.n0 / TC_BN) * TC_EPI_GROUPS + col_off / TC_PIECE] = rsum;
 }
 
 // Largest float below x (x finite or -inf; -inf maps to itself).
@@ -274,6 +278,7 @@ __device__ __forceinline__ float float_below(float x) {
 // f >= f0 is written f > (largest float below f0).  Only the run that contains the reference
 // id takes the element-by-element form, so the common case costs a compare-and-count per score
 // for the rank and one maximum per score for the candidate test.
+template <int WIDTH>
 __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr, int32_t* beat_sm) {
     const bool rin = row < p.M;
     float thr = 0.f, ft = 0.f; int32_t thr_id = 0, tt = -1;
@@ -284,7 +289,7 @@ __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const Tc
     const float thr_lo = float_below(thr), ft_lo = float_below(ft);
     int beat = 0;
 #pragma unroll 1
-    for (int c0 = col_off; c0 < col_off + 64; c0 += 32) {
+    for (int c0 = col_off; c0 < col_off + WIDTH; c0 += 32) {
         float v[32];
         tmem_ld32(taddr + (uint32_t)(c0 - col_off), v);
         if (!rin) continue;
@@ -340,9 +345,9 @@ __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const Tc
 // this thread's tensor-memory lane (taddr points at the first of them).
 template <int EPI, int WIDTH>
 __device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr, int32_t* beat_sm) {
-    static_assert((EPI & 3) == EPI_STORE || WIDTH == 64, "the fused epilogues work on 64-column pieces");
+    static_assert((EPI & 3) == EPI_STORE || (EPI & 3) == EPI_TOPK || WIDTH == TC_PIECE, "the fused loss epilogues work on fixed pieces of a 128-column tile");
     if ((EPI & 3) == EPI_STATS) { tc_epilogue_stats<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, col_off, taddr); return; }
-    if ((EPI & 3) == EPI_TOPK) { tc_epilogue_topk(p, it, row, col_off, taddr, beat_sm); return; }
+    if ((EPI & 3) == EPI_TOPK) { tc_epilogue_topk<WIDTH>(p, it, row, col_off, taddr, beat_sm); return; }
     if ((EPI & 3) == EPI_GRAD) { tc_epilogue_grad<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, col_off, taddr); return; }
     float* const Cout = p.C + (int64_t)it.z * p.split_stride;
 #pragma unroll 1
@@ -375,10 +380,11 @@ __device__ __forceinline__ TcItem tc_item(const TcGemmParams& p, int64_t item) {
 // the operand is read MN-major (its tensor map has the contraction index as rows), which is how
 // dL/dF, Q and T serve as transposed operands without a transposed copy.
 template <int EPI, int BN = 128, bool A_MN = false, bool B_MN = false>
-__global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
+__global__ void __launch_bounds__(tc_threads(EPI)) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
                                                              const __grid_constant__ CUtensorMap tmB, TcGemmParams p) {
     constexpr uint32_t TC_STAGE_BYTES = tc_stage_bytes(BN);
     constexpr uint32_t TC_TMEM_COLS = 2 * BN;          // two fp32 accumulators, used in turn
+    constexpr int EW = tc_epi_warps(EPI), EG = EW / 4, TC_THREADS = tc_threads(EPI);
     extern __shared__ unsigned char tc_smem_raw[];
     unsigned char* base = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
     uint64_t* full = reinterpret_cast<uint64_t*>(base + (size_t)TC_STAGES * TC_STAGE_BYTES);
@@ -398,7 +404,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < TC_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], TC_EPI_WARPS); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EW); }
         *stop = 0;
         mbar_init_fence();
     }
@@ -473,15 +479,15 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
         }
     } else {
         const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
-        const int chalf = (warp - 2) >> 2;             // which half of the tile's columns
+        const int cgrp = (warp - 2) >> 2;              // which group of the tile's columns
         for (int item = item_begin, local = 0; item < item_end; ++item, ++local) {
             const int buf = local & 1;
             const bool ok = mbar_wait_bounded(&acc_full[buf], (local >> 1) & 1);
             tc_fence_after();
             if (!ok || *stop) { if (lane == 0) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); } break; }
             const TcItem it = tc_item(p, item);
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + chalf * (BN / 2));
-            tc_epilogue<EPI, BN / 2>(p, it, it.m0 + quarter * 32 + lane, chalf * (BN / 2), taddr, beat_sm);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cgrp * (BN / EG));
+            tc_epilogue<EPI, BN / EG>(p, it, it.m0 + quarter * 32 + lane, cgrp * (BN / EG), taddr, beat_sm);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
@@ -608,7 +614,7 @@ cudaError_t launch_gemm_inst(const unsigned char* tmA, const unsigned char* tmB,
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    tc_gemm_kernel<EPI, BN, A_MN, B_MN><<<std::min(p.items, num_sms), TC_THREADS, smem + extra_smem, s>>>(
+    tc_gemm_kernel<EPI, BN, A_MN, B_MN><<<std::min(p.items, num_sms), tc_threads(EPI), smem + extra_smem, s>>>(
         *reinterpret_cast<const CUtensorMap*>(tmA), *reinterpret_cast<const CUtensorMap*>(tmB), p);
     return cudaSuccess;
 }
@@ -654,14 +660,14 @@ int launch_tc_forward(kge_handle* h, cudaStream_t s) {
     stage_end(h, ST_BLOCK, s);
     KGE_LAUNCH_CHECK(h);
     stage_begin(h, ST_LOSS, s);
-    CombineParams cp{p.stat_part, 2 * p.tiles_n, p.M, w.fpos, c.loss, c.gamma, c.ce_correction, c.loss_scale,
+    CombineParams cp{p.stat_part, TC_EPI_GROUPS * p.tiles_n, p.M, w.fpos, c.loss, c.gamma, c.ce_correction, c.loss_scale,
                      reinterpret_cast<float2*>(w.row_stat), w.Lrow, w.gpos};
     stats_combine_kernel<<<(p.M * 32 + 255) / 256, 256, 0, s>>>(cp);
     KGE_LAUNCH_CHECK(h);
     KGE_CUDA_CHECK(h, launch_fused(EPI_GRAD, p.l2 != 0, ce, h, p, s));
     KGE_LAUNCH_CHECK(h);
     if (p.l2) {
-        grad_sums_kernel<<<(p.M + p.N + 255) / 256, 256, 0, s>>>(w.grow_part, 2 * p.tiles_n, w.Grow, p.M,
+        grad_sums_kernel<<<(p.M + p.N + 255) / 256, 256, 0, s>>>(w.grow_part, TC_EPI_GROUPS * p.tiles_n, w.Grow, p.M,
                                                                  w.gcol_part, 4 * p.tiles_m, w.Gcol, p.N);
         KGE_LAUNCH_CHECK(h);
     }
@@ -692,6 +698,9 @@ int launch_tc_bwd_gemm(kge_handle* h, const unsigned char* tmA, const unsigned c
 
 // Columns per tile of a backward contraction whose output rows are `cols` wide.
 int tc_backward_tile_cols(int cols) { return cols > 128 ? 256 : 128; }
+
+// Column pieces per 128-wide tile for which the fused forward keeps separate statistics.
+int tc_pieces_per_tile() { return TC_EPI_GROUPS; }
 
 // The two backward contractions on tensor cores, from the bf16 dL/dF the forward left behind.
 // No operand is transposed in memory: an operand whose contraction index is its row index is
