@@ -95,6 +95,7 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
     w.rel_perm = cv.take<int32_t>(B); w.rel_sorted = cv.take<int32_t>(B);
     w.rel_uniq = cv.take<int32_t>(B); w.rel_seg = cv.take<int32_t>(B + 1);
     w.ent_segof = cv.take<int32_t>(ne); w.rel_segof = cv.take<int32_t>(B);
+    w.ent_done = cv.take<int32_t>(ne); w.rel_done = cv.take<int32_t>(B); w.relw_done = th ? cv.take<int32_t>(B) : nullptr;
     w.ent_tkeys = cv.take<uint64_t>((size_t)dedup_tiles((int)ne) * 1024);
     w.rel_tkeys = cv.take<uint64_t>((size_t)dedup_tiles((int)B) * 1024);
     w.part_ent = cv.take<float>(ne * d);

@@ -62,6 +62,7 @@ struct Workspace {
     int32_t *ent_perm, *ent_sorted, *ent_uniq, *ent_seg;  // [2B+N], [2B+N], [2B+N], [2B+N+1]
     int32_t *rel_perm, *rel_sorted, *rel_uniq, *rel_seg;  // [B] ...
     int32_t *ent_segof, *rel_segof;        // [2B+N], [B] segment index of every sorted position
+    int32_t *ent_done, *rel_done, *relw_done;   // [2B+N], [B], [B] finished pieces per long segment
     uint64_t *ent_tkeys, *rel_tkeys;       // tile-sorted (id, position) keys, padded to whole tiles
     float *part_ent, *part_rel, *part_relw;  // [list length, width] partial sums of long segments
     // inference

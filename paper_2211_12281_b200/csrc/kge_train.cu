@@ -439,11 +439,13 @@ __device__ __forceinline__ float block_max(float v, float* sm) {
     return t;
 }
 
-// softplus(z) and sigmoid(z) from one exponential.
+// softplus(z) and sigmoid(z) from one exponential.  The special-function forms used here are good
+// to a few 1e-7 absolute on softplus and a few 1e-6 relative on the exponentials, two orders below
+// the tolerance of this path.
 __device__ __forceinline__ void softplus_sigmoid(float z, float& sp, float& sg) {
-    const float e = expf(-fabsf(z));
-    sp = fmaxf(z, 0.f) + log1pf(e);
-    const float r = 1.f / (1.f + e);
+    const float e = __expf(-fabsf(z));
+    sp = fmaxf(z, 0.f) + __logf(1.f + e);
+    const float r = __frcp_rn(1.f + e);
     sg = z >= 0.f ? r : e * r;
 }
 
@@ -457,13 +459,28 @@ struct WarpReduce {    // one warp works on one row
     __device__ __forceinline__ float max(float v) const { return warp_max(v); }
 };
 
-// Loss and dL/dF of positive b.  `row` holds the scores (shared or global memory), the
-// calling threads cover it as t0, t0 + stride, ...; `lead` marks the one thread that writes
-// the per-row scalars.
-template <class Reduce>
-__device__ __forceinline__ void loss_row(const TrainParams& p, int b, const float* row, float* Frow, int t0, int stride,
-                                         bool lead, Reduce red) {
+// How a thread reaches its share of a row of scores: element i of count(), read with get(i),
+// dL/dF written back with put(i, g).
+struct StridedRow {    // scores in shared or global memory, covered as t0, t0 + stride, ...
+    const float* row; float* out; int t0, stride, n;
+    __device__ __forceinline__ int count() const { return n > t0 ? (n - t0 + stride - 1) / stride : 0; }
+    __device__ __forceinline__ float get(int i) const { return row[t0 + i * stride]; }
+    __device__ __forceinline__ void put(int i, float g) { out[t0 + i * stride] = g; }
+};
+template <int V4>      // scores in registers: V4 float4 per lane, the row is 128 * V4 long
+struct RegisterRow {
+    float4 f[V4], g[V4];
+    __device__ __forceinline__ constexpr int count() const { return 4 * V4; }
+    __device__ __forceinline__ float get(int i) const { return reinterpret_cast<const float*>(&f[i >> 2])[i & 3]; }
+    __device__ __forceinline__ void put(int i, float v) { reinterpret_cast<float*>(&g[i >> 2])[i & 3] = v; }
+};
+
+// Loss and dL/dF of positive b over the calling threads' shares of the row; `lead` marks the
+// one thread that writes the per-row scalars.
+template <class Reduce, class Row>
+__device__ __forceinline__ void loss_row(const TrainParams& p, int b, Row& row, bool lead, Reduce red) {
     const int N = p.N;
+    const int cnt = row.count();
     const float fp = p.w.fpos[b];
     const bool l2 = p.kind == KIND_L2 || p.kind == KIND_TH_L2;
     const float ls = p.loss_scale;
@@ -473,23 +490,26 @@ __device__ __forceinline__ void loss_row(const TrainParams& p, int b, const floa
         float m = 0.f, z = (float)N;
         if (a > 0.f) {
             float lm = -INFINITY;
-            for (int n = t0; n < N; n += stride) lm = fmaxf(lm, a * row[n]);
+#pragma unroll
+            for (int i = 0; i < cnt; ++i) lm = fmaxf(lm, a * row.get(i));
             m = red.max(lm);
             float lz = 0.f;
-            for (int n = t0; n < N; n += stride) lz += expf(a * row[n] - m);
+#pragma unroll
+            for (int i = 0; i < cnt; ++i) lz += __expf(a * row.get(i) - m);
             z = red.sum(lz);
         }
         const float invz = 1.f / z;
         float lacc = 0.f;
-        for (int n = t0; n < N; n += stride) {
-            const float f = row[n];
-            const float w = a > 0.f ? expf(a * f - m) * invz : invz;
+#pragma unroll
+        for (int i = 0; i < cnt; ++i) {
+            const float f = row.get(i);
+            const float w = a > 0.f ? __expf(a * f - m) * invz : invz;
             float sp, sg;
             softplus_sigmoid(gamma + f, sp, sg);
             lacc += w * sp;
             float g = ls * w * sg;
             if (l2) g = f < 0.f ? g / -f : 0.f;
-            Frow[n] = g;
+            row.put(i, g);
             gsum += g;
         }
         const float lsum = red.sum(lacc);
@@ -502,18 +522,21 @@ __device__ __forceinline__ void loss_row(const TrainParams& p, int b, const floa
     } else {
         const float c = p.ce_c;
         float lm = -INFINITY;
-        for (int n = t0; n < N; n += stride) lm = fmaxf(lm, row[n] + c);
+#pragma unroll
+        for (int i = 0; i < cnt; ++i) lm = fmaxf(lm, row.get(i) + c);
         const float m = fmaxf(red.max(lm), fp);
         float lz = 0.f;
-        for (int n = t0; n < N; n += stride) lz += expf(row[n] + c - m);
-        const float epos = expf(fp - m);
+#pragma unroll
+        for (int i = 0; i < cnt; ++i) lz += __expf(row.get(i) + c - m);
+        const float epos = __expf(fp - m);
         const float z = red.sum(lz) + epos;
         const float invz = 1.f / z;
-        for (int n = t0; n < N; n += stride) {
-            const float f = row[n];
-            float g = ls * expf(f + c - m) * invz;
+#pragma unroll
+        for (int i = 0; i < cnt; ++i) {
+            const float f = row.get(i);
+            float g = ls * __expf(f + c - m) * invz;
             if (l2) g = f < 0.f ? g / -f : 0.f;
-            Frow[n] = g;
+            row.put(i, g);
             gsum += g;
         }
         if (lead) {
@@ -545,7 +568,8 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_kernel(TrainParams p) {
         __syncthreads();
         row = rowbuf;
     }
-    loss_row(p, b, row, Frow, tid, LOSS_THREADS, tid == 0, BlockReduce{sm});
+    StridedRow sr{row, Frow, tid, LOSS_THREADS, p.N};
+    loss_row(p, b, sr, tid == 0, BlockReduce{sm});
 }
 
 // One warp per positive: rows of up to LOSS_WARP_MAX_N scores (N % 4 == 0), no CTA-wide barriers.
@@ -559,7 +583,24 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_warp_kernel(TrainParams p) 
     float* row = rowbuf + (size_t)warp * p.N;
     stage_row(row, Frow, p.N, lane, 32);
     __syncwarp();
-    loss_row(p, b, row, Frow, lane, 32, lane == 0, WarpReduce{});
+    StridedRow sr{row, Frow, lane, 32, p.N};
+    loss_row(p, b, sr, lane == 0, WarpReduce{});
+}
+
+// One warp per positive with the whole row in registers (N = 128 * V4): every pass over the row
+// is unrolled, so the exponentials of a lane's 4 * V4 scores are independent instructions.
+template <int V4>
+__global__ void __launch_bounds__(LOSS_THREADS) loss_reg_kernel(TrainParams p) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.x * (LOSS_THREADS / 32) + warp;
+    if (b >= p.B) return;
+    float4* Frow = reinterpret_cast<float4*>(p.w.F + (int64_t)b * p.N);
+    RegisterRow<V4> rr;
+#pragma unroll
+    for (int j = 0; j < V4; ++j) rr.f[j] = Frow[j * 32 + lane];
+    loss_row(p, b, rr, lane == 0, WarpReduce{});
+#pragma unroll
+    for (int j = 0; j < V4; ++j) Frow[j * 32 + lane] = rr.g[j];
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1205,7 +1246,12 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
             configured = true;
         }
     }
-    if (p.N <= LOSS_WARP_MAX_N && (p.N & 3) == 0) {
+    constexpr int loss_rows = LOSS_THREADS / 32;
+    const int loss_grid = (p.B + loss_rows - 1) / loss_rows;
+    if (p.N == 256) loss_reg_kernel<2><<<loss_grid, LOSS_THREADS, 0, s>>>(p);
+    else if (p.N == 512) loss_reg_kernel<4><<<loss_grid, LOSS_THREADS, 0, s>>>(p);
+    else if (p.N == 1024) loss_reg_kernel<8><<<loss_grid, LOSS_THREADS, 0, s>>>(p);
+    else if (p.N <= LOSS_WARP_MAX_N && (p.N & 3) == 0) {
         constexpr int rows = LOSS_THREADS / 32;
         loss_warp_kernel<<<(p.B + rows - 1) / rows, LOSS_THREADS, (size_t)rows * p.N * 4, s>>>(p);
     } else {

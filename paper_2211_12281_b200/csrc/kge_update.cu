@@ -4,12 +4,12 @@
 //               the permutation and the sorted id list
 //   segment   : distinct ids, segment offsets, segment index of every sorted position
 //               (single-CTA scan), batch loss reduction
-//   piece sum : one warp per sorted position; a segment of at most 16 rows is summed in
+//   piece     : one warp per sorted position; a segment of at most 16 rows is summed in
 //               ascending source position by the warp at its first position and the row is
 //               updated at once (SGD / Adam / row-wise Adagrad); a longer segment is cut
-//               into pieces of 16 rows, each summed by its own warp into a partial row
-//   piece join: the first position of a long segment adds its pieces in ascending order and
-//               updates the row
+//               into pieces of 16 rows, each summed by its own warp into a partial row, and
+//               the warp that finishes the last outstanding piece adds the pieces in
+//               ascending order and updates the row
 // The summation order of a segment is therefore fixed by the batch alone: results are
 // bit-reproducible, and a row that occurs hundreds of times in a batch does not serialise
 // behind a single warp.
@@ -32,6 +32,7 @@ struct IdList {
     int na, nb, nc;
     int64_t rows;               // table rows (ids outside [0, rows) are reported and read as 0)
     int32_t *perm, *sorted, *uniq, *seg, *seg_of;
+    int32_t *seg_done, *seg_done2;   // [n] pieces finished per long segment (zeroed here for the update kernel); second table on the same list, or NULL
     uint64_t* tkeys;            // [tiles * SORT_TILE] tile-sorted (id << 32 | position), padded with ~0
     int32_t* count;             // number of distinct ids
     __host__ __device__ __forceinline__ int n() const { return na + nb + nc; }
@@ -125,6 +126,8 @@ __global__ void __launch_bounds__(SEG_THREADS) segment_kernel(DedupParams p) {
         const int32_t id = L.sorted[r];
         if (id != prev) { L.uniq[u] = id; L.seg[u] = r; ++u; }
         L.seg_of[r] = u - 1;
+        L.seg_done[r] = 0;
+        if (L.seg_done2) L.seg_done2[r] = 0;
         prev = id;
     }
     if (tid == 0) { L.seg[total] = n; *L.count = total; }
@@ -135,6 +138,7 @@ struct UpdateJob {
     const float* grads;                // [n, width] gradient rows by source position
     float* part;                       // [n, width] partial sums of long segments, row = first sorted position of the piece
     const int32_t *uniq, *seg, *perm, *sorted, *seg_of;
+    int32_t* seg_done;                 // [n] per segment: pieces of a long segment that have been written
     int width, n;                      // n = list length
 };
 
@@ -225,7 +229,8 @@ __device__ __forceinline__ void apply_row(const UpdateJob& J, const UpdateParams
 
 // g += rows[idx[0]], rows[idx[1]], ... in that order, a few rows' loads in flight at a time
 // (four for narrow rows, two for wide ones, to keep the register count down).
-template <typename V, int NCH, typename IndexOf>
+// FRESH: the rows were written by other warps of this launch; read them past the L1 cache.
+template <typename V, int NCH, bool FRESH = false, typename IndexOf>
 __device__ __forceinline__ void ordered_sum(const V* rows, int wv, int count, IndexOf index_of, V (&g)[NCH], int lane) {
     constexpr int BATCH = NCH == 1 ? 4 : 2;
     for (int s = 0; s < count; s += BATCH) {
@@ -236,7 +241,7 @@ __device__ __forceinline__ void ordered_sum(const V* rows, int wv, int count, In
 #pragma unroll
             for (int i = 0; i < NCH; ++i) {
                 const int c = lane + 32 * i;
-                v[r][i] = (s + r < count && c < wv) ? src[c] : VecOps<V>::zero();
+                v[r][i] = (s + r < count && c < wv) ? (FRESH ? __ldcg(src + c) : src[c]) : VecOps<V>::zero();
             }
         }
 #pragma unroll
@@ -276,36 +281,27 @@ __device__ __forceinline__ void piece_sum(const UpdateJob& J, const UpdateParams
                         [&](int s) { return (int64_t)__shfl_sync(0xffffffffu, src, s); }, g, lane);
     if (whole) {
         apply_row<V, NCH>(J, p, J.uniq[u], g, lane);
-    } else {
-        V* dst = reinterpret_cast<V*>(J.part) + (int64_t)r * wv;
-#pragma unroll
-        for (int i = 0; i < NCH; ++i) { const int c = lane + 32 * i; if (c < wv) dst[c] = g[i]; }
+        return;
     }
-}
-
-// One warp per sorted position; only the first position of a segment longer than PIECE rows
-// works: it adds the segment's pieces in ascending order and updates the row.
-template <typename V, int NCH>
-__device__ __forceinline__ void piece_join(const UpdateJob& J, const UpdateParams& p, int r, int lane) {
-    const int wv = J.width / VecOps<V>::LEN;
-    if (r > 0 && J.sorted[r - 1] == J.sorted[r]) return;
-    const int u = J.seg_of[r];
-    const int s1 = J.seg[u + 1];
-    if (s1 - r <= PIECE) return;
-    V g[NCH];
+    V* dst = reinterpret_cast<V*>(J.part) + (int64_t)r * wv;
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) { const int c = lane + 32 * i; if (c < wv) dst[c] = g[i]; }
+    // The warp that finishes the segment's last outstanding piece adds all pieces, in ascending
+    // order whoever that warp is, and updates the row.
+    const int npieces = (len + PIECE - 1) / PIECE;
+    __threadfence();
+    int done = 0;
+    if (lane == 0) done = atomicAdd(&J.seg_done[u], 1);
+    done = __shfl_sync(0xffffffffu, done, 0);
+    if (done != npieces - 1) return;
+    __threadfence();
 #pragma unroll
     for (int i = 0; i < NCH; ++i) g[i] = VecOps<V>::zero();
-    ordered_sum<V, NCH>(reinterpret_cast<const V*>(J.part), wv, (s1 - r + PIECE - 1) / PIECE,
-                        [&](int s) { return (int64_t)r + (int64_t)s * PIECE; }, g, lane);
+    ordered_sum<V, NCH, true>(reinterpret_cast<const V*>(J.part), wv, npieces,
+                              [&](int s) { return (int64_t)s0 + (int64_t)s * PIECE; }, g, lane);
     apply_row<V, NCH>(J, p, J.uniq[u], g, lane);
 }
 
-template <bool JOIN, typename V, int NCH>
-__device__ __forceinline__ void piece_do(const UpdateJob& J, const UpdateParams& p, int r, int lane) {
-    if (JOIN) piece_join<V, NCH>(J, p, r, lane); else piece_sum<V, NCH>(J, p, r, lane);
-}
-
-template <bool JOIN>
 __global__ void __launch_bounds__(256, 3) piece_kernel(UpdateParams p) {
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (gw >= p.warp_begin[p.njobs]) return;
@@ -315,13 +311,13 @@ __global__ void __launch_bounds__(256, 3) piece_kernel(UpdateParams p) {
     const int r = gw - p.warp_begin[j];
     if ((J.width & 3) == 0) {
         const int wv = J.width >> 2;
-        if (wv <= 32) piece_do<JOIN, float4, 1>(J, p, r, lane);
-        else if (wv <= 64) piece_do<JOIN, float4, 2>(J, p, r, lane);
-        else piece_do<JOIN, float4, 4>(J, p, r, lane);
+        if (wv <= 32) piece_sum<float4, 1>(J, p, r, lane);
+        else if (wv <= 64) piece_sum<float4, 2>(J, p, r, lane);
+        else piece_sum<float4, 4>(J, p, r, lane);
     } else {
         // narrow rows whose width is only even (RotatE phases with d % 8 != 0): scalar lanes
-        if (J.width <= 64) piece_do<JOIN, float, 2>(J, p, r, lane);
-        else piece_do<JOIN, float, kMaxDim / 2 / 32>(J, p, r, lane);
+        if (J.width <= 64) piece_sum<float, 2>(J, p, r, lane);
+        else piece_sum<float, kMaxDim / 2 / 32>(J, p, r, lane);
     }
 }
 
@@ -336,9 +332,9 @@ int launch_dedup(kge_handle* h, const int32_t* heads, const int32_t* rels, const
     const int B = c.batch, N = c.num_neg;
     DedupParams dp;
     dp.ent = IdList{heads, tails, negs, B, B, N, c.num_entities,
-                    w.ent_perm, w.ent_sorted, w.ent_uniq, w.ent_seg, w.ent_segof, w.ent_tkeys, w.counts};
+                    w.ent_perm, w.ent_sorted, w.ent_uniq, w.ent_seg, w.ent_segof, w.ent_done, nullptr, w.ent_tkeys, w.counts};
     dp.rel = IdList{rels, rels, rels, B, 0, 0, c.num_relations,
-                    w.rel_perm, w.rel_sorted, w.rel_uniq, w.rel_seg, w.rel_segof, w.rel_tkeys, w.counts + 1};
+                    w.rel_perm, w.rel_sorted, w.rel_uniq, w.rel_seg, w.rel_segof, w.rel_done, w.relw_done, w.rel_tkeys, w.counts + 1};
     dp.ent_tiles = dedup_tiles(2 * B + N);
     dp.status = w.status;
     const int tiles = dp.ent_tiles + dedup_tiles(B);
@@ -362,11 +358,11 @@ int launch_update(kge_handle* h, uint64_t step, float lr, cudaStream_t s) {
     UpdateParams up;
     up.njobs = c.score == KGE_TRANSH ? 3 : 2;
     up.job[0] = UpdateJob{h->ent, h->ent_state, w.grad_ent, w.part_ent, w.ent_uniq, w.ent_seg, w.ent_perm,
-                          w.ent_sorted, w.ent_segof, c.dim, 2 * B + N};
+                          w.ent_sorted, w.ent_segof, w.ent_done, c.dim, 2 * B + N};
     up.job[1] = UpdateJob{h->rel, h->rel_state, w.grad_rel, w.part_rel, w.rel_uniq, w.rel_seg, w.rel_perm,
-                          w.rel_sorted, w.rel_segof, h->kw, B};
+                          w.rel_sorted, w.rel_segof, w.rel_done, h->kw, B};
     up.job[2] = UpdateJob{h->relw, h->relw_state, w.grad_relw, w.part_relw, w.rel_uniq, w.rel_seg, w.rel_perm,
-                          w.rel_sorted, w.rel_segof, c.dim, B};
+                          w.rel_sorted, w.rel_segof, w.relw_done, c.dim, B};
     up.warp_begin[0] = 0;
     for (int j = 0; j < 3; ++j) up.warp_begin[j + 1] = up.warp_begin[j] + (j < up.njobs ? up.job[j].n : 0);
     up.opt = c.opt;
@@ -375,9 +371,7 @@ int launch_update(kge_handle* h, uint64_t step, float lr, cudaStream_t s) {
     up.corr2 = (float)(1.0 - std::pow((double)c.beta2, (double)(step + 1)));
     const int warps = up.warp_begin[up.njobs];
     stage_begin(h, ST_UPDATE, s);
-    piece_kernel<false><<<(warps * 32 + 255) / 256, 256, 0, s>>>(up);
-    KGE_LAUNCH_CHECK(h);
-    piece_kernel<true><<<(warps * 32 + 255) / 256, 256, 0, s>>>(up);
+    piece_kernel<<<(warps * 32 + 255) / 256, 256, 0, s>>>(up);
     stage_end(h, ST_UPDATE, s);
     KGE_LAUNCH_CHECK(h);
     return KGE_OK;
