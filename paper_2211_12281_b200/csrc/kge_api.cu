@@ -335,25 +335,27 @@ int kge_train_step(kge_handle* h, uint64_t step, float lr, const int32_t* heads,
     if (given != 0 && given != 4) return KGE_ERR_BAD_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     Workspace& w = h->ws;
-    if (given == 0) {
-        if (!h->graph_loaded) return KGE_ERR_NOT_READY;
-        int rc = launch_sample(h, step, w.heads, w.rels, w.tails, w.negs, s);
-        if (rc != KGE_OK) return rc;
-        heads = w.heads; rels = w.rels; tails = w.tails; negs = w.negs;
-    }
     // With per-stage timing on, everything runs in order on the caller's stream.  Otherwise
     // the sort of the touched ids (which needs only the ids) runs on a side stream beside
     // the forward and backward kernels, and joins before the update.
     const bool fork = !h->prof.on;
+    bool fused = false;
     int rc;
-    if (fork) {
-        KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_ids, s));
-        KGE_CUDA_CHECK(h, cudaStreamWaitEvent(h->side[0], h->ev_ids, 0));
-        rc = launch_dedup(h, heads, rels, tails, negs, h->side[0]);
-        if (rc != KGE_OK) return rc;
-        KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_seg, h->side[0]));
+    if (given == 0) {
+        if (!h->graph_loaded) return KGE_ERR_NOT_READY;
+        // The gather kernel can draw the batch itself when the 8 query warps of a CTA share a
+        // triple bucket and the bucket's cumulative weights fit its shared memory.
+        const kge_config& c = h->cfg;
+        const int buckets = c.head_part < 0 ? c.num_parts * c.num_parts : c.num_parts;
+        fused = fork && (c.batch / buckets) % 8 == 0 && c.num_relations + 1 <= 4096;
+        if (!fused) {
+            rc = launch_sample(h, step, w.heads, w.rels, w.tails, w.negs, s);
+            if (rc != KGE_OK) return rc;
+        }
+        heads = w.heads; rels = w.rels; tails = w.tails; negs = w.negs;
     }
-    rc = launch_forward_backward(h, heads, rels, tails, negs, loss_out, s, fork ? h->side[1] : nullptr);
+    rc = launch_forward_backward(h, heads, rels, tails, negs, loss_out, s, fork ? h->side[1] : nullptr,
+                                 fork ? h->side[0] : nullptr, fused, step);
     if (rc != KGE_OK) return rc;
     if (fork) KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_seg, 0));
     else if ((rc = launch_dedup(h, heads, rels, tails, negs, s)) != KGE_OK) return rc;

@@ -152,9 +152,13 @@ int stage_collect(kge_handle* h, cudaStream_t s);
 // ---- launch wrappers implemented in the other translation units ----
 int launch_sample(kge_handle* h, uint64_t step, int32_t* heads, int32_t* rels, int32_t* tails, int32_t* negs,
                   cudaStream_t s);
-// Forward and backward; `side` (or NULL) runs the accumulation over the queries concurrently.
+// Forward and backward; `side` (or NULL) runs the accumulation over the queries concurrently;
+// `dedup_side` (or NULL) gets the sort of the touched ids as soon as the ids are final (the
+// caller waits for ev_seg before the update); with `fused_sample` the gather kernel draws the
+// batch of `step` itself and leaves the ids in the workspace (heads ... negs must point there).
 int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* rels, const int32_t* tails,
-                            const int32_t* negs, float* loss_out, cudaStream_t s, cudaStream_t side);
+                            const int32_t* negs, float* loss_out, cudaStream_t s, cudaStream_t side, cudaStream_t dedup_side,
+                            bool fused_sample, uint64_t step);
 // Stable sort of the touched ids, distinct ids and segments (needs only the batch ids).
 int launch_dedup(kge_handle* h, const int32_t* heads, const int32_t* rels, const int32_t* tails,
                  const int32_t* negs, cudaStream_t s);

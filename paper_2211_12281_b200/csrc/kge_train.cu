@@ -6,7 +6,7 @@
 //   chain    : positive pair, chain rule q -> (h, r, w), reduction of the column splits
 #include <cuda_bf16.h>
 
-#include "kge_common.cuh"
+#include "kge_sample.cuh"
 
 namespace kge {
 
@@ -21,6 +21,9 @@ struct TrainParams {
     const int32_t *heads, *rels, *tails, *negs;
     int split_q, split_t;
     float* loss_out;    // caller's device scalar for the batch loss, or NULL
+    int fused_sample;   // the gather kernel draws the batch itself (ids land in sp.heads ...) instead of reading it
+    int slots_per_bucket;
+    SampleParams sp;
     int tc_l2;          // TransE p = 2 with tensor-core backward: the splits hold C.T and C^T.Q, C = dL/dF / distance
     Workspace w;
 };
@@ -58,13 +61,29 @@ __device__ __forceinline__ float pair_partial(int kind, float4 q, float4 t) {
 
 template <int kMaxChunks>   // float4 slices per lane: a warp owns a row
 __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
+    extern __shared__ uint64_t bucket_wcum[];   // fused sampling: cumulative weights of this CTA's bucket
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
+    int64_t bucket_base = 0;
+    if (p.fused_sample) {
+        // The 8 query warps of a CTA draw from one triple bucket (the host checks that the slots
+        // of a bucket are a multiple of 8): its cumulative weights are fetched side by side.
+        const int w0 = blockIdx.x * (blockDim.x >> 5);
+        if (w0 < p.B) {
+            bucket_base = sample_bucket_base(p.sp, w0 / p.slots_per_bucket);
+            if (p.sp.sample_mode == 0)
+                for (int r = threadIdx.x; r <= (int)p.sp.R; r += blockDim.x) bucket_wcum[r] = p.sp.wcum[bucket_base + r];
+        }
+        __syncthreads();
+    }
     if (warp >= p.B + p.N) return;
     const int d4 = p.d4;
     if (warp >= p.B) {
         const int n = warp - p.B;
-        const int64_t id = checked_id(p.negs[n], p.E, p.w.status);
+        int32_t neg;
+        if (p.fused_sample) { neg = sample_negative(p.sp, n); if (lane == 0) p.sp.negs[n] = neg; }
+        else neg = p.negs[n];
+        const int64_t id = checked_id(neg, p.E, p.w.status);
         const float4* src = reinterpret_cast<const float4*>(p.ent) + id * d4;
         float4* dst = reinterpret_cast<float4*>(p.w.Tneg) + (int64_t)n * d4;
         float nrm2 = 0.f;
@@ -80,9 +99,19 @@ __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
         return;
     }
     const int b = warp;
-    const int64_t hid = checked_id(p.heads[b], p.E, p.w.status);
-    const int64_t rid = checked_id(p.rels[b], p.R, p.w.status);
-    const int64_t tid = checked_id(p.tails[b], p.E, p.w.status);
+    int32_t ih, ir, it;
+    if (p.fused_sample) {
+        if (lane == 0) {
+            sample_positive(p.sp, b, bucket_base, bucket_wcum, ih, ir, it);
+            p.sp.heads[b] = ih; p.sp.rels[b] = ir; p.sp.tails[b] = it;
+        }
+        ih = __shfl_sync(0xffffffffu, ih, 0); ir = __shfl_sync(0xffffffffu, ir, 0); it = __shfl_sync(0xffffffffu, it, 0);
+    } else {
+        ih = p.heads[b]; ir = p.rels[b]; it = p.tails[b];
+    }
+    const int64_t hid = checked_id(ih, p.E, p.w.status);
+    const int64_t rid = checked_id(ir, p.R, p.w.status);
+    const int64_t tid = checked_id(it, p.E, p.w.status);
     const float4* hrow = reinterpret_cast<const float4*>(p.ent) + hid * d4;
     const float4* trow = reinterpret_cast<const float4*>(p.ent) + tid * d4;
     float4 h[kMaxChunks], t[kMaxChunks], q[kMaxChunks], wh[kMaxChunks];
@@ -1194,7 +1223,8 @@ cudaError_t launch_accum(int kind, const AccArgs& a, cudaStream_t s) {
 }  // namespace
 
 int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* rels, const int32_t* tails,
-                            const int32_t* negs, float* loss_out, cudaStream_t s, cudaStream_t side) {
+                            const int32_t* negs, float* loss_out, cudaStream_t s, cudaStream_t side, cudaStream_t dedup_side,
+                            bool fused_sample, uint64_t step) {
     const kge_config& c = h->cfg;
     TrainParams p;
     p.B = c.batch; p.N = c.num_neg; p.d = c.dim; p.d4 = c.dim / 4; p.kw = h->kw;
@@ -1205,6 +1235,10 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     p.heads = heads; p.rels = rels; p.tails = tails; p.negs = negs;
     p.split_q = h->split_q; p.split_t = h->split_t;
     p.loss_out = loss_out;
+    p.fused_sample = fused_sample ? 1 : 0;
+    p.sp = make_sample_params(h, step);
+    p.sp.heads = h->ws.heads; p.sp.rels = h->ws.rels; p.sp.tails = h->ws.tails; p.sp.negs = h->ws.negs;
+    p.slots_per_bucket = c.batch / (c.head_part < 0 ? c.num_parts * c.num_parts : c.num_parts);
     p.tc_l2 = c.prec == KGE_PREC_BF16_TC && p.kind == KIND_L2;
     p.w = h->ws;
     const int nch = p.d4 <= 32 ? 1 : (p.d4 <= 64 ? 2 : 4);
@@ -1213,12 +1247,21 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     stage_begin(h, ST_BUILD, s);
     {
         const int grid = (row_warps * 32 + 255) / 256;
-        if (nch == 1) build_kernel<1><<<grid, 256, 0, s>>>(p);
-        else if (nch == 2) build_kernel<2><<<grid, 256, 0, s>>>(p);
-        else build_kernel<4><<<grid, 256, 0, s>>>(p);
+        const size_t smem = fused_sample ? (size_t)(c.num_relations + 1) * 8 : 0;
+        if (nch == 1) build_kernel<1><<<grid, 256, smem, s>>>(p);
+        else if (nch == 2) build_kernel<2><<<grid, 256, smem, s>>>(p);
+        else build_kernel<4><<<grid, 256, smem, s>>>(p);
     }
     stage_end(h, ST_BUILD, s);
     KGE_LAUNCH_CHECK(h);
+    if (dedup_side) {
+        // the batch ids are final: the sort of the touched ids runs beside everything up to the update
+        KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_ids, s));
+        KGE_CUDA_CHECK(h, cudaStreamWaitEvent(dedup_side, h->ev_ids, 0));
+        const int rc = launch_dedup(h, heads, rels, tails, negs, dedup_side);
+        if (rc != KGE_OK) return rc;
+        KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_seg, dedup_side));
+    }
     if (c.prec == KGE_PREC_BF16_TC) {
         // tensor cores: scores, loss and dL/dF in two fused passes, the score block never stored
         const int rc = launch_tc_forward(h, s);
