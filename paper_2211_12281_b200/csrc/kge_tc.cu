@@ -177,21 +177,27 @@ __device__ __forceinline__ void tc_epilogue_stats(const TcGemmParams& p, const T
         if (row >= p.M) continue;
         const int ncol = it.n0 + c0;
         const int valid = min(32, p.N - ncol);     // columns of this chunk inside the problem (may be <= 0)
-        float cm = -INFINITY;
+        // four independent chains each for the maximum and the sums: a single chain of 32 dependent
+        // operations would leave the few epilogue warps waiting on their own results
+        float cmv[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
             if (L2 || !CE) v[i] = (valid == 32 || i < valid) ? tc_score<L2>(p, v[i], rn, ncol + i) : 0.f;
             const float y = fmaf(v[i], k1, k0);
-            cm = fmaxf(cm, (valid == 32 || i < valid) ? y : -INFINITY);
+            cmv[i & 3] = fmaxf(cmv[i & 3], (valid == 32 || i < valid) ? y : -INFINITY);
         }
+        const float cm = fmaxf(fmaxf(cmv[0], cmv[1]), fmaxf(cmv[2], cmv[3]));
         if (cm > m) { const float r = fast_exp2(m - cm); z *= r; l *= r; m = cm; }
+        float zv[4] = {0.f, 0.f, 0.f, 0.f}, lv[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
             float e = fast_exp2(fmaf(v[i], k1, k0) - m);
             if (valid != 32 && i >= valid) e = 0.f;
-            z += e;
-            if (!CE) { float sp, sg; tc_softplus_sigmoid(p.gamma + v[i], sp, sg); l = fmaf(e, sp, l); }
+            zv[i & 3] += e;
+            if (!CE) { float sp, sg; tc_softplus_sigmoid(p.gamma + v[i], sp, sg); lv[i & 3] = fmaf(e, sp, lv[i & 3]); }
         }
+        z += (zv[0] + zv[1]) + (zv[2] + zv[3]);
+        if (!CE) l += (lv[0] + lv[1]) + (lv[2] + lv[3]);
     }
     if (row < p.M)
         p.stat_part[(int64_t)row * (TC_EPI_GROUPS * p.tiles_n) + (it.n0 / TC_BN) * TC_EPI_GROUPS + col_off / TC_PIECE] = make_float4(m, z, l, 0.f);
