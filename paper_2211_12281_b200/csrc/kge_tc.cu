@@ -161,6 +161,35 @@ __device__ __forceinline__ float tc_score(const TcGemmParams& p, float acc, floa
 constexpr float kLog2e = 1.4426950408889634f;
 __device__ __forceinline__ float fast_exp2(float y) { float r; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(y)); return r; }
 
+// One chunk of 32 scores of the first pass.  FULL: all 32 columns lie inside the problem (no
+// per-element masking); otherwise the first `valid` do.
+template <bool L2, bool CE, bool FULL>
+__device__ __forceinline__ void tc_stats_chunk(const TcGemmParams& p, float (&v)[32], float rn, int ncol, int valid,
+                                               float k1, float k0, float& m, float& z, float& l) {
+    // four independent chains each for the maximum and the sums: a single chain of 32 dependent
+    // operations would leave the few epilogue warps waiting on their own results
+    float cmv[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        if (L2) v[i] = (FULL || i < valid) ? tc_score<true>(p, v[i], rn, ncol + i) : 0.f;
+        const float y = fmaf(v[i], k1, k0);        // exponent in base 2
+        if (CE) v[i] = y;                          // the sampled softmax does not need the score itself again
+        cmv[i & 3] = fmaxf(cmv[i & 3], (FULL || i < valid) ? y : -INFINITY);
+    }
+    const float cm = fmaxf(fmaxf(cmv[0], cmv[1]), fmaxf(cmv[2], cmv[3]));
+    if (cm > m) { const float r = fast_exp2(m - cm); z *= r; l *= r; m = cm; }
+    float zv[4] = {0.f, 0.f, 0.f, 0.f}, lv[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        float e = fast_exp2((CE ? v[i] : fmaf(v[i], k1, k0)) - m);
+        if (!FULL && i >= valid) e = 0.f;
+        zv[i & 3] += e;
+        if (!CE) { float sp, sg; tc_softplus_sigmoid(p.gamma + v[i], sp, sg); lv[i & 3] = fmaf(e, sp, lv[i & 3]); }
+    }
+    z += (zv[0] + zv[1]) + (zv[2] + zv[3]);
+    if (!CE) l += (lv[0] + lv[1]) + (lv[2] + lv[3]);
+}
+
 // First pass of the fused loss: running (max, sum of exponentials, exponentially weighted loss
 // sum) over this thread's 64 columns of one row, rescaled whenever the maximum moves.  The
 // exponent is x = a f for the self-adversarial weights and x = f + c for the sampled softmax;
@@ -177,27 +206,8 @@ __device__ __forceinline__ void tc_epilogue_stats(const TcGemmParams& p, const T
         if (row >= p.M) continue;
         const int ncol = it.n0 + c0;
         const int valid = min(32, p.N - ncol);     // columns of this chunk inside the problem (may be <= 0)
-        // four independent chains each for the maximum and the sums: a single chain of 32 dependent
-        // operations would leave the few epilogue warps waiting on their own results
-        float cmv[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            if (L2 || !CE) v[i] = (valid == 32 || i < valid) ? tc_score<L2>(p, v[i], rn, ncol + i) : 0.f;
-            const float y = fmaf(v[i], k1, k0);
-            cmv[i & 3] = fmaxf(cmv[i & 3], (valid == 32 || i < valid) ? y : -INFINITY);
-        }
-        const float cm = fmaxf(fmaxf(cmv[0], cmv[1]), fmaxf(cmv[2], cmv[3]));
-        if (cm > m) { const float r = fast_exp2(m - cm); z *= r; l *= r; m = cm; }
-        float zv[4] = {0.f, 0.f, 0.f, 0.f}, lv[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            float e = fast_exp2(fmaf(v[i], k1, k0) - m);
-            if (valid != 32 && i >= valid) e = 0.f;
-            zv[i & 3] += e;
-            if (!CE) { float sp, sg; tc_softplus_sigmoid(p.gamma + v[i], sp, sg); lv[i & 3] = fmaf(e, sp, lv[i & 3]); }
-        }
-        z += (zv[0] + zv[1]) + (zv[2] + zv[3]);
-        if (!CE) l += (lv[0] + lv[1]) + (lv[2] + lv[3]);
+        if (valid == 32) tc_stats_chunk<L2, CE, true>(p, v, rn, ncol, valid, k1, k0, m, z, l);
+        else if (valid > 0) tc_stats_chunk<L2, CE, false>(p, v, rn, ncol, valid, k1, k0, m, z, l);
     }
     if (row < p.M)
         p.stat_part[(int64_t)row * (TC_EPI_GROUPS * p.tiles_n) + (it.n0 / TC_BN) * TC_EPI_GROUPS + col_off / TC_PIECE] = make_float4(m, z, l, 0.f);
@@ -208,6 +218,17 @@ __device__ __forceinline__ uint16_t bf16_bits(float v) {
     return *reinterpret_cast<const uint16_t*>(&b);
 }
 __device__ __forceinline__ float bf16_value(uint16_t bits) { return __uint_as_float((uint32_t)bits << 16); }
+
+// dL/dF of one pair from its accumulator: scale = loss_scale / normaliser, k0 already holds minus
+// the row's base-2 maximum.
+template <bool L2, bool CE>
+__device__ __forceinline__ float tc_grad_one(const TcGemmParams& p, float acc, float rn, int col, float k1, float k0, float scale) {
+    const float f = tc_score<L2>(p, acc, rn, col);
+    float g = scale * fast_exp2(fmaf(f, k1, k0));
+    if (!CE) { float sp, sg; tc_softplus_sigmoid(p.gamma + f, sp, sg); g *= sg; }
+    if (L2) g = f < 0.f ? g / -f : 0.f;
+    return g;
+}
 
 // Second pass: dL/dF from the recomputed score and the row's final (base-2 max, 1 / normaliser),
 // written as bf16 for the two backward contractions (which read it K-major and MN-major).
@@ -227,16 +248,12 @@ __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const Tc
         const int ncol = it.n0 + c0;
         const int valid = rin ? min(32, p.N - ncol) : 0;
         uint32_t g2[16];     // bf16 pairs in memory order
+        if (valid == 32) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            float g = 0.f;
-            if (valid == 32 || i < valid) {
-                const float f = tc_score<L2>(p, v[i], rn, ncol + i);
-                g = scale * fast_exp2(fmaf(f, k1, k0));
-                if (!CE) { float sp, sg; tc_softplus_sigmoid(p.gamma + f, sp, sg); g *= sg; }
-                if (L2) g = f < 0.f ? g / -f : 0.f;
-            }
-            v[i] = g;
+            for (int i = 0; i < 32; ++i) v[i] = tc_grad_one<L2, CE>(p, v[i], rn, ncol + i, k1, k0, scale);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = i < valid ? tc_grad_one<L2, CE>(p, v[i], rn, ncol + i, k1, k0, scale) : 0.f;
         }
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
