@@ -124,7 +124,8 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 // 32 consecutive fp32 columns of this thread's tensor-memory lane.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+// (the registers are valid after tmem_ld_wait)
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, float (&v)[32]) {
     uint32_t r[32];
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -135,10 +136,11 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) { tmem_ld32_issue(taddr, v); tmem_ld_wait(); }
 
 struct TcItem { int z, m0, n0; };   // K split, first row, first column
 
@@ -199,15 +201,18 @@ __device__ __forceinline__ void tc_epilogue_stats(const TcGemmParams& p, const T
     const float rn = (L2 && row < p.M) ? p.row_norm2[row] : 0.f;
     const float k1 = CE ? kLog2e : p.adv_temp * kLog2e, k0 = CE ? p.ce_c * kLog2e : 0.f;
     float m = -INFINITY, z = 0.f, l = 0.f;
-#pragma unroll 1
-    for (int c0 = col_off; c0 < col_off + TC_PIECE; c0 += 32) {
-        float v[32];
-        tmem_ld32(taddr + (uint32_t)(c0 - col_off), v);
-        if (row >= p.M) continue;
-        const int ncol = it.n0 + c0;
-        const int valid = min(32, p.N - ncol);     // columns of this chunk inside the problem (may be <= 0)
-        if (valid == 32) tc_stats_chunk<L2, CE, true>(p, v, rn, ncol, valid, k1, k0, m, z, l);
-        else if (valid > 0) tc_stats_chunk<L2, CE, false>(p, v, rn, ncol, valid, k1, k0, m, z, l);
+    static_assert(TC_PIECE == 64, "two chunks of 32 columns per piece");
+    float v0[32], v1[32];
+    tmem_ld32_issue(taddr, v0);                // both chunks are requested before the first is used
+    tmem_ld32_issue(taddr + 32u, v1);
+    tmem_ld_wait();
+    if (row < p.M) {
+        const int ncol = it.n0 + col_off;
+        const int valid0 = min(32, p.N - ncol), valid1 = min(32, p.N - ncol - 32);   // columns inside the problem (may be <= 0)
+        if (valid0 == 32) tc_stats_chunk<L2, CE, true>(p, v0, rn, ncol, valid0, k1, k0, m, z, l);
+        else if (valid0 > 0) tc_stats_chunk<L2, CE, false>(p, v0, rn, ncol, valid0, k1, k0, m, z, l);
+        if (valid1 == 32) tc_stats_chunk<L2, CE, true>(p, v1, rn, ncol + 32, valid1, k1, k0, m, z, l);
+        else if (valid1 > 0) tc_stats_chunk<L2, CE, false>(p, v1, rn, ncol + 32, valid1, k1, k0, m, z, l);
     }
     if (row < p.M)
         p.stat_part[(int64_t)row * (TC_EPI_GROUPS * p.tiles_n) + (it.n0 / TC_BN) * TC_EPI_GROUPS + col_off / TC_PIECE] = make_float4(m, z, l, 0.f);
