@@ -55,6 +55,15 @@ WORKLOADS = {
     "c3s_distmult": dict(E=1_000_000, R=1000, T=10_000_000, d=256, score="distmult", p_norm=1, loss="softmax",
                          opt="adam", B=4096, N=16384, P=8, gamma=0.0, adv_temp=0.0, lr=0.001, tc=True,
                          ce_correction="paper", entity_zipf=1.1, relation_zipf=1.0, graph_seed=2, device_tables=True),
+    # BASELINE configs[3]: 91,000,000 entities (46.6 GB table), 1,400 relations, d = 128, B = N = 8,192, P = 16, row-wise
+    # Adagrad, log-sigmoid loss with margin 12.  The graph is cut to 60 M of the 600 M triples (host-side preprocessing;
+    # the step does not depend on the graph's size).  TransE-L2 on tensor cores, TransH on CUDA cores.
+    "c4_transe_l2": dict(E=91_000_000, R=1400, T=60_000_000, d=128, score="transe", p_norm=2, loss="logsigmoid",
+                         opt="adagrad", B=8192, N=8192, P=16, gamma=12.0, adv_temp=1.0, lr=0.05, tc=True,
+                         entity_zipf=1.1, relation_zipf=1.0, graph_seed=3, device_tables=True),
+    "c4_transh_l1": dict(E=91_000_000, R=1400, T=60_000_000, d=128, score="transh", p_norm=1, loss="logsigmoid",
+                         opt="adagrad", B=8192, N=8192, P=16, gamma=12.0, adv_temp=1.0, lr=0.05,
+                         entity_zipf=1.1, relation_zipf=1.0, graph_seed=3, device_tables=True),
     "c1_distmult": dict(E=1000, R=10, T=20_000, d=32, score="distmult", p_norm=1, loss="logsigmoid",
                         opt="sgd", B=64, N=128, P=2, gamma=0.0, adv_temp=0.0, lr=0.1,
                         entity_zipf=1.1, relation_zipf=0.0, graph_seed=0),
@@ -81,6 +90,7 @@ STAGE_OPS = {
     "transe1": dict(block=2, accum_q=2, accum_t=2),     # sub, |.|+add  /  compare, predicated add
     "rotate1": dict(block=3.5, accum_q=5, accum_t=5),   # per real coordinate; one sqrt / rsqrt per complex pair
     "distmult1": dict(block=1, accum_q=1, accum_t=1),   # one FMA
+    "transh1": dict(block=4, accum_q=11, accum_t=8),     # w.t dot, residual, |.| / residual again, sign, two or three accumulations
 }
 
 
