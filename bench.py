@@ -327,13 +327,15 @@ def run_ours(args, w, name):
 
     # ---- end to end: ids in pinned host memory -> H2D, step, loss -> D2H, every step ----
     nxt = warm + args.steps
-    ids_dev = [torch.empty(n, dtype=torch.int32, device=dev) for n in (B, B, B, N)]
+    ids_all = torch.empty(3 * B + N, dtype=torch.int32, device=dev)          # heads | rels | tails | negs, back to back
+    ids_dev = [ids_all[0:B], ids_all[B:2 * B], ids_all[2 * B:3 * B], ids_all[3 * B:]]
     pinned = []
-    for i in range(args.steps):
+    for i in range(min(args.steps, 256)):                                   # a ring of pinned host batches
         kge.sample_batch(nxt + i, *ids_dev)
-        pinned.append([x.cpu().pin_memory() for x in ids_dev])
+        host = ids_all.cpu().pin_memory()
+        pinned.append([host[0:B], host[B:2 * B], host[2 * B:3 * B], host[3 * B:]])
     loss_host = torch.zeros(1, dtype=torch.float32).pin_memory()
-    host_fn = lambda s: kge.train_step_host(s, w["lr"], *pinned[s - nxt], loss_host)
+    host_fn = lambda s: kge.train_step_host(s, w["lr"], *pinned[(s - nxt) % len(pinned)], loss_host)
     barrier()
     e2e_ms = float(np.sum(timed_steps(nxt, args.steps, host_fn)))
     barrier()

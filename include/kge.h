@@ -147,7 +147,8 @@ int kge_train_step(kge_handle* h, uint64_t step, float lr,
 
 /*
  * The same step for callers that keep the batch on the host: ids are [host] arrays (pinned
- * memory makes the copies asynchronous), copied in on `stream`; the loss is copied back to
+ * memory makes the copies asynchronous), copied in on `stream` (as one copy when the four
+ * lists lie back to back in the order heads, rels, tails, negs); the loss is copied back to
  * *loss_out [host] and the stream is synchronised before returning.
  */
 int kge_train_step_host(kge_handle* h, uint64_t step, float lr,

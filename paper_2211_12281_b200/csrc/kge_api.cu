@@ -357,8 +357,8 @@ int kge_train_step(kge_handle* h, uint64_t step, float lr, const int32_t* heads,
     rc = launch_forward_backward(h, heads, rels, tails, negs, loss_out, s, fork ? h->side[1] : nullptr,
                                  fork ? h->side[0] : nullptr, fused, step);
     if (rc != KGE_OK) return rc;
-    if (fork) KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_seg, 0));
-    else if ((rc = launch_dedup(h, heads, rels, tails, negs, s)) != KGE_OK) return rc;
+    // with side streams the id sort has been joined before the chain kernel
+    if (!fork && (rc = launch_dedup(h, heads, rels, tails, negs, s)) != KGE_OK) return rc;
     rc = launch_update(h, step, lr, s);
     if (rc != KGE_OK) return rc;
     return h->prof.on ? stage_collect(h, s) : KGE_OK;
@@ -371,10 +371,15 @@ int kge_train_step_host(kge_handle* h, uint64_t step, float lr, const int32_t* h
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     Workspace& w = h->ws;
     const size_t B = h->cfg.batch, N = h->cfg.num_neg;
-    KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.heads, heads, B * 4, cudaMemcpyHostToDevice, s));
-    KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.rels, rels, B * 4, cudaMemcpyHostToDevice, s));
-    KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.tails, tails, B * 4, cudaMemcpyHostToDevice, s));
-    KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.negs, negs, N * 4, cudaMemcpyHostToDevice, s));
+    if (rels == heads + B && tails == rels + B && negs == tails + B) {
+        // the four lists lie back to back on the host, as they do in the workspace: one copy
+        KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.heads, heads, (3 * B + N) * 4, cudaMemcpyHostToDevice, s));
+    } else {
+        KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.heads, heads, B * 4, cudaMemcpyHostToDevice, s));
+        KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.rels, rels, B * 4, cudaMemcpyHostToDevice, s));
+        KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.tails, tails, B * 4, cudaMemcpyHostToDevice, s));
+        KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.negs, negs, N * 4, cudaMemcpyHostToDevice, s));
+    }
     int rc = kge_train_step(h, step, lr, w.heads, w.rels, w.tails, w.negs, w.loss, stream);
     if (rc != KGE_OK) return rc;
     if (loss_out) KGE_CUDA_CHECK(h, cudaMemcpyAsync(loss_out, w.loss, 4, cudaMemcpyDeviceToHost, s));

@@ -236,6 +236,15 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
+// Programmatic dependent launch.  A kernel started with launch_dependent() may become resident
+// while the kernel before it in the stream still runs; it must call grid_dependency_wait()
+// before it touches anything that kernel (or an earlier one) writes or reads, and everything
+// before that call may only set up its own shared memory.  The wait returns once the preceding
+// kernels have finished and their writes are visible; with no programmatic edge it returns at
+// once.  allow_dependents() lets the next kernel become resident from now on.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void allow_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float softplusf(float z) { return fmaxf(z, 0.f) + log1pf(expf(-fabsf(z))); }
 __device__ __forceinline__ float sigmoidf(float z) {
     if (z >= 0.f) return 1.f / (1.f + expf(-z));
@@ -243,5 +252,17 @@ __device__ __forceinline__ float sigmoidf(float z) {
     return e / (1.f + e);
 }
 #endif
+
+// Launch with a programmatic edge to the kernel before it in the stream (see grid_dependency_wait).
+template <class... P, class... A>
+inline cudaError_t launch_dependent(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, A&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+}
 
 }  // namespace kge

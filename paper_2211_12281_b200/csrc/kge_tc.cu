@@ -144,24 +144,43 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) { tmem
 
 struct TcItem { int z, m0, n0; };   // K split, first row, first column
 
-// softplus(z) and sigmoid(z) from one exponential.
-__device__ __forceinline__ void tc_softplus_sigmoid(float z, float& sp, float& sg) {
-    const float e = expf(-fabsf(z));
-    sp = fmaxf(z, 0.f) + log1pf(e);
-    const float r = 1.f / (1.f + e);
-    sg = z >= 0.f ? r : e * r;
+constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
+__device__ __forceinline__ float fast_exp2(float y) { float r; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(y)); return r; }
+__device__ __forceinline__ float fast_log2(float y) { float r; asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(y)); return r; }
+__device__ __forceinline__ float fast_rcp(float y) { float r; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(y)); return r; }
+__device__ __forceinline__ float fast_rsqrt(float y) { float r; asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(y)); return r; }
+
+// The fused epilogues evaluate one transcendental per special-function instruction: their
+// inputs come from bf16 operands, so the approximate forms (relative error about 2^-22) are
+// far inside the error of the scores, and an epilogue of a d = 128 contraction is bound by
+// exactly these instructions.
+// softplus(z) = max(z, 0) + log(1 + exp(-|z|))
+__device__ __forceinline__ float tc_softplus(float z) {
+    const float e = fast_exp2(-fabsf(z) * kLog2e);
+    return fmaf(fast_log2(1.f + e), kLn2, fmaxf(z, 0.f));
+}
+// sigmoid(z) from the same exponential
+__device__ __forceinline__ float tc_sigmoid(float z) {
+    const float e = fast_exp2(-fabsf(z) * kLog2e);
+    const float r = fast_rcp(1.f + e);
+    return z >= 0.f ? r : e * r;
 }
 
 // Score of a pair from the accumulator: the contraction itself, or (L2) the distance score of
-// the norm expansion.
+// the norm expansion, with the reciprocal distance the gradient needs (0 at distance 0).
+template <bool L2>
+__device__ __forceinline__ float tc_score_inv(const TcGemmParams& p, float acc, float rn, int col, float& inv) {
+    if (!L2) { inv = 0.f; return acc; }
+    const float s2 = fmaxf(rn + p.col_norm2[col] - 2.f * acc, 0.f);
+    inv = s2 > 0.f ? fast_rsqrt(s2) : 0.f;
+    return -s2 * inv;
+}
 template <bool L2>
 __device__ __forceinline__ float tc_score(const TcGemmParams& p, float acc, float rn, int col) {
-    if (!L2) return acc;
-    return -sqrtf(fmaxf(rn + p.col_norm2[col] - 2.f * acc, 0.f));
+    float inv;
+    return tc_score_inv<L2>(p, acc, rn, col, inv);
 }
 
-constexpr float kLog2e = 1.4426950408889634f;
-__device__ __forceinline__ float fast_exp2(float y) { float r; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(y)); return r; }
 
 // One chunk of 32 scores of the first pass.  FULL: all 32 columns lie inside the problem (no
 // per-element masking); otherwise the first `valid` do.
@@ -186,7 +205,7 @@ __device__ __forceinline__ void tc_stats_chunk(const TcGemmParams& p, float (&v)
         float e = fast_exp2((CE ? v[i] : fmaf(v[i], k1, k0)) - m);
         if (!FULL && i >= valid) e = 0.f;
         zv[i & 3] += e;
-        if (!CE) { float sp, sg; tc_softplus_sigmoid(p.gamma + v[i], sp, sg); lv[i & 3] = fmaf(e, sp, lv[i & 3]); }
+        if (!CE) lv[i & 3] = fmaf(e, tc_softplus(p.gamma + v[i]), lv[i & 3]);
     }
     z += (zv[0] + zv[1]) + (zv[2] + zv[3]);
     if (!CE) l += (lv[0] + lv[1]) + (lv[2] + lv[3]);
@@ -228,10 +247,11 @@ __device__ __forceinline__ float bf16_value(uint16_t bits) { return __uint_as_fl
 // the row's base-2 maximum.
 template <bool L2, bool CE>
 __device__ __forceinline__ float tc_grad_one(const TcGemmParams& p, float acc, float rn, int col, float k1, float k0, float scale) {
-    const float f = tc_score<L2>(p, acc, rn, col);
+    float inv;
+    const float f = tc_score_inv<L2>(p, acc, rn, col, inv);
     float g = scale * fast_exp2(fmaf(f, k1, k0));
-    if (!CE) { float sp, sg; tc_softplus_sigmoid(p.gamma + f, sp, sg); g *= sg; }
-    if (L2) g = f < 0.f ? g / -f : 0.f;
+    if (!CE) g *= tc_sigmoid(p.gamma + f);
+    if (L2) g *= inv;
     return g;
 }
 
@@ -279,12 +299,23 @@ __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const Tc
         if (L2) {   // the norm expansion also needs the sums of what the contractions will see
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
-                const float gv = bf16_value((uint16_t)(g2[i >> 1] >> ((i & 1) * 16)));
-                rsum += gv;
-                const float cs = warp_sum(gv);   // over this warp's 32 rows (rows outside the problem hold zeros)
-                if (lane == 0 && ncol + i < p.N)
-                    p.gcol_part[(int64_t)((it.m0 / TC_BM) * 4 + ((row - it.m0) >> 5)) * p.N + ncol + i] = cs;
+                v[i] = bf16_value((uint16_t)(g2[i >> 1] >> ((i & 1) * 16)));
+                rsum += v[i];
             }
+            // Sums over this warp's 32 rows (rows outside the problem hold zeros) of all 32 columns
+            // at once: each exchange halves the columns a lane still carries, so 31 shuffles do
+            // what 32 separate warp sums need 160 for; lane c ends with the sum of column c.
+#pragma unroll
+            for (int half = 16; half >= 1; half >>= 1) {
+                const bool upper = (lane & half) != 0;
+#pragma unroll
+                for (int j = 0; j < half; ++j) {
+                    const float send = upper ? v[j] : v[j + half], keep = upper ? v[j + half] : v[j];
+                    v[j] = keep + __shfl_xor_sync(0xffffffffu, send, half);
+                }
+            }
+            if (ncol + lane < p.N)
+                p.gcol_part[(int64_t)((it.m0 / TC_BM) * 4 + ((row - it.m0) >> 5)) * p.N + ncol + lane] = v[0];
         }
     }
     if (L2 && rin) p.grow_part[(int64_t)row * (TC_EPI_GROUPS * p.tiles_n) + (it.n0 / TC_BN) * TC_EPI_GROUPS + col_off / TC_PIECE] = rsum;
@@ -602,8 +633,8 @@ __global__ void __launch_bounds__(256) stats_combine_kernel(CombineParams p) {
         p.Lrow[b] = -fp + (m + log2f(z)) * 0.6931471805599453f;
         p.gpos[b] = p.loss_scale * (epos / z - 1.f);
     } else {
-        float sp, sg;
-        tc_softplus_sigmoid(-(p.gamma + fp), sp, sg);
+        const float zp = -(p.gamma + fp), ep = expf(-fabsf(zp)), rp = 1.f / (1.f + ep);   // once per row: the exact forms
+        const float sp = fmaxf(zp, 0.f) + log1pf(ep), sg = zp >= 0.f ? rp : ep * rp;
         p.Lrow[b] = sp + l / z;
         p.gpos[b] = -p.loss_scale * sg;
     }

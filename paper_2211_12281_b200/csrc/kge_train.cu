@@ -64,6 +64,7 @@ __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
     extern __shared__ uint64_t bucket_wcum[];   // fused sampling: cumulative weights of this CTA's bucket
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
+    allow_dependents();   // the score kernel may set up its shared memory while this one runs
     int64_t bucket_base = 0;
     if (p.fused_sample) {
         // The 8 query warps of a CTA draw from one triple bucket (the host checks that the slots
@@ -369,6 +370,8 @@ __global__ void __launch_bounds__(FTHREADS) block_tma_kernel(TrainParams p) {
         mbar_init_fence();
     }
     __syncthreads();
+    grid_dependency_wait();
+    allow_dependents();
 
     auto issue = [&](int chunk, int stage) {     // thread r < ROWS owns row r of the stage
         if (tid >= ROWS) return;
@@ -590,6 +593,8 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_kernel(TrainParams p) {
     extern __shared__ __align__(16) float rowbuf[];
     __shared__ float sm[LOSS_THREADS / 32];
     const int b = blockIdx.x, tid = threadIdx.x;
+    grid_dependency_wait();
+    allow_dependents();
     float* Frow = p.w.F + (int64_t)b * p.N;
     const float* row = Frow;
     if (p.N <= LOSS_SMEM_FLOATS) {
@@ -607,6 +612,8 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_warp_kernel(TrainParams p) 
     extern __shared__ __align__(16) float rowbuf[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = blockIdx.x * (LOSS_THREADS / 32) + warp;
+    grid_dependency_wait();
+    allow_dependents();
     if (b >= p.B) return;
     float* Frow = p.w.F + (int64_t)b * p.N;
     float* row = rowbuf + (size_t)warp * p.N;
@@ -622,6 +629,8 @@ template <int V4>
 __global__ void __launch_bounds__(LOSS_THREADS) loss_reg_kernel(TrainParams p) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = blockIdx.x * (LOSS_THREADS / 32) + warp;
+    grid_dependency_wait();
+    allow_dependents();
     if (b >= p.B) return;
     float4* Frow = reinterpret_cast<float4*>(p.w.F + (int64_t)b * p.N);
     RegisterRow<V4> rr;
@@ -831,6 +840,8 @@ __global__ void __launch_bounds__(32 * ACC_WARPS) accum_tma_kernel(AccArgs a) {
 
     if (tid == 0) { mbar_init(&bars[0], 1); mbar_init(&bars[1], 1); mbar_init_fence(); }
     __syncthreads();
+    grid_dependency_wait();
+    allow_dependents();
 
     auto issue_rows = [&](int chunk, int buf) {      // thread 0 only
         const int c0 = c_begin + chunk * ACC_CC;
@@ -947,6 +958,8 @@ __global__ void __launch_bounds__(32 * ACC_WARPS) accum_tma_kernel(AccArgs a) {
 template <int kMaxChunks>
 __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
     const int lane = threadIdx.x & 31;
+    grid_dependency_wait();
+    allow_dependents();
     if (blockIdx.x == gridDim.x - 1) {   // the extra last CTA adds up the batch loss
         __shared__ float lsum[8];
         float v = 0.f;
@@ -1164,8 +1177,7 @@ cudaError_t launch_block_tma(const TrainParams& p, cudaStream_t s) {
         configured = true;
     }
     dim3 grid((p.N + TN - 1) / TN, (p.B + FTQ - 1) / FTQ);
-    block_tma_kernel<KIND><<<grid, FTHREADS, smem, s>>>(p);
-    return cudaSuccess;
+    return launch_dependent(block_tma_kernel<KIND>, grid, dim3(FTHREADS), smem, s, p);
 }
 
 template <int KIND, int NCH, bool OWNER_Q>
@@ -1180,8 +1192,7 @@ cudaError_t launch_accum_tma_inst(const AccArgs& a, cudaStream_t s) {
         configured = true;
     }
     dim3 grid((a.own_rows + ACC_ROWS - 1) / ACC_ROWS, a.split);
-    accum_tma_kernel<KIND, NCH, OWNER_Q, WARPS><<<grid, 32 * WARPS, smem, s>>>(a);
-    return cudaSuccess;
+    return launch_dependent(accum_tma_kernel<KIND, NCH, OWNER_Q, WARPS>, grid, dim3(32 * WARPS), smem, s, a);
 }
 
 template <int KIND, int NCH, bool OWNER_Q>
@@ -1291,14 +1302,14 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     }
     constexpr int loss_rows = LOSS_THREADS / 32;
     const int loss_grid = (p.B + loss_rows - 1) / loss_rows;
-    if (p.N == 256) loss_reg_kernel<2><<<loss_grid, LOSS_THREADS, 0, s>>>(p);
-    else if (p.N == 512) loss_reg_kernel<4><<<loss_grid, LOSS_THREADS, 0, s>>>(p);
-    else if (p.N == 1024) loss_reg_kernel<8><<<loss_grid, LOSS_THREADS, 0, s>>>(p);
+    if (p.N == 256) KGE_CUDA_CHECK(h, launch_dependent(loss_reg_kernel<2>, dim3(loss_grid), dim3(LOSS_THREADS), 0, s, p));
+    else if (p.N == 512) KGE_CUDA_CHECK(h, launch_dependent(loss_reg_kernel<4>, dim3(loss_grid), dim3(LOSS_THREADS), 0, s, p));
+    else if (p.N == 1024) KGE_CUDA_CHECK(h, launch_dependent(loss_reg_kernel<8>, dim3(loss_grid), dim3(LOSS_THREADS), 0, s, p));
     else if (p.N <= LOSS_WARP_MAX_N && (p.N & 3) == 0) {
         constexpr int rows = LOSS_THREADS / 32;
-        loss_warp_kernel<<<(p.B + rows - 1) / rows, LOSS_THREADS, (size_t)rows * p.N * 4, s>>>(p);
+        KGE_CUDA_CHECK(h, launch_dependent(loss_warp_kernel, dim3((p.B + rows - 1) / rows), dim3(LOSS_THREADS), (size_t)rows * p.N * 4, s, p));
     } else {
-        loss_kernel<<<p.B, LOSS_THREADS, p.N <= LOSS_SMEM_FLOATS ? (size_t)p.N * 4 : 0, s>>>(p);
+        KGE_CUDA_CHECK(h, launch_dependent(loss_kernel, dim3(p.B), dim3(LOSS_THREADS), p.N <= LOSS_SMEM_FLOATS ? (size_t)p.N * 4 : 0, s, p));
     }
     stage_end(h, ST_LOSS, s);
     KGE_LAUNCH_CHECK(h);
@@ -1338,12 +1349,14 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     KGE_LAUNCH_CHECK(h);
     if (side) KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_t, 0));
     }
+    // the update follows the chain kernel directly: join the id sort here, where it has long finished
+    if (dedup_side) KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_seg, 0));
     stage_begin(h, ST_CHAIN, s);
     {
         const int grid = (row_warps * 32 + 255) / 256 + 1;
-        if (nch == 1) chain_kernel<1><<<grid, 256, 0, s>>>(p);
-        else if (nch == 2) chain_kernel<2><<<grid, 256, 0, s>>>(p);
-        else chain_kernel<4><<<grid, 256, 0, s>>>(p);
+        if (nch == 1) KGE_CUDA_CHECK(h, launch_dependent(chain_kernel<1>, dim3(grid), dim3(256), 0, s, p));
+        else if (nch == 2) KGE_CUDA_CHECK(h, launch_dependent(chain_kernel<2>, dim3(grid), dim3(256), 0, s, p));
+        else KGE_CUDA_CHECK(h, launch_dependent(chain_kernel<4>, dim3(grid), dim3(256), 0, s, p));
     }
     stage_end(h, ST_CHAIN, s);
     KGE_LAUNCH_CHECK(h);

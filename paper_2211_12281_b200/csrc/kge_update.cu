@@ -304,6 +304,7 @@ __device__ __forceinline__ void piece_sum(const UpdateJob& J, const UpdateParams
 
 __global__ void __launch_bounds__(256, 3) piece_kernel(UpdateParams p) {
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    grid_dependency_wait();
     if (gw >= p.warp_begin[p.njobs]) return;
     int j = 0;
     while (j + 1 < p.njobs && gw >= p.warp_begin[j + 1]) ++j;
@@ -371,7 +372,7 @@ int launch_update(kge_handle* h, uint64_t step, float lr, cudaStream_t s) {
     up.corr2 = (float)(1.0 - std::pow((double)c.beta2, (double)(step + 1)));
     const int warps = up.warp_begin[up.njobs];
     stage_begin(h, ST_UPDATE, s);
-    piece_kernel<<<(warps * 32 + 255) / 256, 256, 0, s>>>(up);
+    KGE_CUDA_CHECK(h, launch_dependent(piece_kernel, dim3((warps * 32 + 255) / 256), dim3(256), 0, s, up));
     stage_end(h, ST_UPDATE, s);
     KGE_LAUNCH_CHECK(h);
     return KGE_OK;
