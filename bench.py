@@ -96,7 +96,7 @@ STAGE_OPS = {
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
 # summarised in profiles/train_step_c2_transe_l1_launches.md (None once the kernel has changed since).
-NCU_TRAFFIC_BYTES = {("c2_transe_l1", "accum_q"): 5.27e6, ("c2_transe_l1", "accum_t"): 5.27e6, ("c2_transe_l1", "block"): 1.07e6}
+NCU_TRAFFIC_BYTES = {}
 
 
 def cfg_kwargs(w, seed):
@@ -352,7 +352,11 @@ def run_ours(args, w, name):
     per_stage_us = {k: 1e3 * v[0] / v[1] for k, v in stages.items() if v[1] > 0}
     kind = f"{w['score']}{w['p_norm']}"
     ops = STAGE_OPS.get(kind, {})
-    compute_stages = [s for s in ("block", "accum_q", "accum_t") if s in per_stage_us]
+    if "accum_q" in per_stage_us and "accum_t" not in per_stage_us:     # dQ and dT share one launch
+        per_stage_us["accum"] = per_stage_us.pop("accum_q")
+        ops = dict(ops, accum=ops.get("accum_q", 0) + ops.get("accum_t", 0))
+    # tensor-core step: "block" is the statistics pass and "loss" the gradient pass, each one B x N x d contraction
+    compute_stages = [s for s in ("block", "accum", "accum_q", "accum_t") + (("loss",) if w.get("tc") else ()) if s in per_stage_us]
     dominant = max(compute_stages, key=lambda s: per_stage_us[s])
     roofline = None
     if w.get("tc"):

@@ -262,7 +262,12 @@ int kge_bind(kge_handle* h, float* ent, float* rel, float* relw, float* ent_stat
         if (rc != KGE_OK) return rc;
     }
     if (!h->streams_ready) {
-        KGE_CUDA_CHECK(h, cudaStreamCreateWithFlags(&h->side[0], cudaStreamNonBlocking));
+        // side[0] carries the sort of the touched ids, a few small kernels the update waits for:
+        // at the highest priority their CTAs take the next free slots instead of queueing behind
+        // the score and gradient kernels' hundreds of CTAs
+        int prio_least = 0, prio_greatest = 0;
+        KGE_CUDA_CHECK(h, cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
+        KGE_CUDA_CHECK(h, cudaStreamCreateWithPriority(&h->side[0], cudaStreamNonBlocking, prio_greatest));
         KGE_CUDA_CHECK(h, cudaStreamCreateWithFlags(&h->side[1], cudaStreamNonBlocking));
         cudaEvent_t* evs[4] = {&h->ev_ids, &h->ev_loss, &h->ev_seg, &h->ev_t};
         for (cudaEvent_t* e : evs) KGE_CUDA_CHECK(h, cudaEventCreateWithFlags(e, cudaEventDisableTiming));

@@ -820,7 +820,7 @@ inline size_t accum_tma_smem(int d4) {
 
 // ACC_WARPS warps per CTA, 32 / ACC_WARPS owner rows per warp (8 rows while the registers last).
 template <int KIND, int NCH, bool OWNER_Q, int ACC_WARPS>
-__global__ void __launch_bounds__(32 * ACC_WARPS) accum_tma_kernel(AccArgs a) {
+__device__ __forceinline__ void accum_tma_body(const AccArgs& a, const int block_x, const int block_y) {
     constexpr int ACC_RPW = ACC_ROWS / ACC_WARPS;
     constexpr int ACC_THREADS = 32 * ACC_WARPS;
     constexpr int ACC_WPT = ACC_ROWS * ACC_CC / ACC_THREADS;   // weights of a tile handled per thread
@@ -832,9 +832,9 @@ __global__ void __launch_bounds__(32 * ACC_WARPS) accum_tma_kernel(AccArgs a) {
     uint64_t* bars = reinterpret_cast<uint64_t*>(Csum + 8 * 32);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int r0 = blockIdx.x * ACC_ROWS;
+    const int r0 = block_x * ACC_ROWS;
     const int per = ((a.oth_rows + a.split - 1) / a.split + ACC_CC - 1) / ACC_CC * ACC_CC;
-    const int c_begin = blockIdx.y * per;
+    const int c_begin = block_y * per;
     const int c_end = min(a.oth_rows, c_begin + per);
     const int nchunk = c_end > c_begin ? (c_end - c_begin + ACC_CC - 1) / ACC_CC : 0;
 
@@ -936,7 +936,7 @@ __global__ void __launch_bounds__(32 * ACC_WARPS) accum_tma_kernel(AccArgs a) {
         for (int j = 0; j < NCH; ++j) {
             const int r = r0 + warp * ACC_RPW + i, c = lane + 32 * j;
             if (r >= a.own_rows || c >= d4) continue;
-            reinterpret_cast<float4*>(a.out)[((int64_t)blockIdx.y * a.own_rows + r) * d4 + c] = acc[i][j];
+            reinterpret_cast<float4*>(a.out)[((int64_t)block_y * a.own_rows + r) * d4 + c] = acc[i][j];
         }
     if (KIND == KIND_L1 && !OWNER_Q) {
         Csum[warp * 32 + lane] = csum;
@@ -944,9 +944,19 @@ __global__ void __launch_bounds__(32 * ACC_WARPS) accum_tma_kernel(AccArgs a) {
         if (warp == 0 && r0 + lane < a.own_rows) {
             float t = 0.f;
             for (int w = 0; w < ACC_WARPS; ++w) t += Csum[w * 32 + lane];
-            a.csum[(int64_t)blockIdx.y * a.own_rows + r0 + lane] = t;
+            a.csum[(int64_t)block_y * a.own_rows + r0 + lane] = t;
         }
     }
+}
+
+// Both accumulations of a step in one launch: blockIdx.z = 0 owns query rows (dQ), 1 owns
+// negative rows (dT); the grid spans the larger of the two shapes.
+template <int KIND, int NCH, int ACC_WARPS>
+__global__ void __launch_bounds__(32 * ACC_WARPS) accum_tma_kernel(AccArgs aq, AccArgs at) {
+    const int own_rows = blockIdx.z == 0 ? aq.own_rows : at.own_rows, split = blockIdx.z == 0 ? aq.split : at.split;
+    if ((int)blockIdx.x * ACC_ROWS >= own_rows || (int)blockIdx.y >= split) return;
+    if (blockIdx.z == 0) accum_tma_body<KIND, NCH, true, ACC_WARPS>(aq, blockIdx.x, blockIdx.y);
+    else accum_tma_body<KIND, NCH, false, ACC_WARPS>(at, blockIdx.x, blockIdx.y);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1180,26 +1190,42 @@ cudaError_t launch_block_tma(const TrainParams& p, cudaStream_t s) {
     return launch_dependent(block_tma_kernel<KIND>, grid, dim3(FTHREADS), smem, s, p);
 }
 
-template <int KIND, int NCH, bool OWNER_Q>
-cudaError_t launch_accum_tma_inst(const AccArgs& a, cudaStream_t s) {
+template <int KIND, int NCH>
+cudaError_t launch_accum_tma_inst(const AccArgs& aq, const AccArgs& at, cudaStream_t s) {
     constexpr int WARPS = NCH == 4 ? 8 : 4;
-    const size_t smem = accum_tma_smem(a.d4);
+    const size_t smem = accum_tma_smem(aq.d4);
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(accum_tma_kernel<KIND, NCH, OWNER_Q, WARPS>,
+        cudaError_t e = cudaFuncSetAttribute(accum_tma_kernel<KIND, NCH, WARPS>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)accum_tma_smem(kMaxDim / 4));
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    dim3 grid((a.own_rows + ACC_ROWS - 1) / ACC_ROWS, a.split);
-    return launch_dependent(accum_tma_kernel<KIND, NCH, OWNER_Q, WARPS>, grid, dim3(32 * WARPS), smem, s, a);
+    dim3 grid((std::max(aq.own_rows, at.own_rows) + ACC_ROWS - 1) / ACC_ROWS, std::max(aq.split, at.split), 2);
+    return launch_dependent(accum_tma_kernel<KIND, NCH, WARPS>, grid, dim3(32 * WARPS), smem, s, aq, at);
 }
 
+template <int KIND>
+cudaError_t launch_accum_tma_kind(const AccArgs& aq, const AccArgs& at, cudaStream_t s) {
+    if (aq.d4 <= 32) return launch_accum_tma_inst<KIND, 1>(aq, at, s);
+    if (aq.d4 <= 64) return launch_accum_tma_inst<KIND, 2>(aq, at, s);
+    return launch_accum_tma_inst<KIND, 4>(aq, at, s);
+}
+
+// dQ and dT of the pair kinds whose operands are plain rows, in one launch.
+cudaError_t launch_accum_tma(int kind, const AccArgs& aq, const AccArgs& at, cudaStream_t s) {
+    switch (kind) {
+        case KIND_L1: return launch_accum_tma_kind<KIND_L1>(aq, at, s);
+        case KIND_L2: return launch_accum_tma_kind<KIND_L2>(aq, at, s);
+        case KIND_CL1: return launch_accum_tma_kind<KIND_CL1>(aq, at, s);
+        default: return launch_accum_tma_kind<KIND_DOT>(aq, at, s);
+    }
+}
+
+// TransH: one launch per owner side.
 template <int KIND, int NCH, bool OWNER_Q>
 cudaError_t launch_accum_inst(const AccArgs& a, cudaStream_t s) {
-    constexpr bool TH = KIND == KIND_TH_L1 || KIND == KIND_TH_L2;
-    if (!TH) return launch_accum_tma_inst<TH ? KIND_L1 : KIND, NCH, OWNER_Q>(a, s);
-    size_t smem = (size_t)ACC_CC * a.d4 * 16 * ((TH && !OWNER_Q) ? 2 : 1) + (size_t)ACC_CC * ACC_LDW * 4 * (TH ? 3 : 1);
+    const size_t smem = (size_t)ACC_CC * a.d4 * 16 * (OWNER_Q ? 1 : 2) + (size_t)ACC_CC * ACC_LDW * 4 * 3;
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(accum_kernel<KIND, NCH, OWNER_Q>,
@@ -1221,14 +1247,8 @@ cudaError_t launch_accum_kind(const AccArgs& a, cudaStream_t s) {
 
 template <bool OWNER_Q>
 cudaError_t launch_accum(int kind, const AccArgs& a, cudaStream_t s) {
-    switch (kind) {
-        case KIND_L1: return launch_accum_kind<KIND_L1, OWNER_Q>(a, s);
-        case KIND_L2: return launch_accum_kind<KIND_L2, OWNER_Q>(a, s);
-        case KIND_CL1: return launch_accum_kind<KIND_CL1, OWNER_Q>(a, s);
-        case KIND_DOT: return launch_accum_kind<KIND_DOT, OWNER_Q>(a, s);
-        case KIND_TH_L1: return launch_accum_kind<KIND_TH_L1, OWNER_Q>(a, s);
-        default: return launch_accum_kind<KIND_TH_L2, OWNER_Q>(a, s);
-    }
+    if (kind == KIND_TH_L1) return launch_accum_kind<KIND_TH_L1, OWNER_Q>(a, s);
+    return launch_accum_kind<KIND_TH_L2, OWNER_Q>(a, s);
 }
 
 }  // namespace
@@ -1329,25 +1349,33 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     aq.own = p.w.Q; aq.oth = p.w.Tneg; aq.what = p.w.What; aq.G = p.w.F; aq.U = p.w.U; aq.Cc = p.w.Cc;
     aq.own_rows = p.B; aq.oth_rows = p.N; aq.N = p.N; aq.d4 = p.d4; aq.split = p.split_q;
     aq.out = p.w.dQpart; aq.out2 = p.w.dWpart; aq.csum = nullptr; aq.status = p.w.status;
-    // the two accumulations are independent: with a side stream they run concurrently
-    if (side) {
-        KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_loss, s));
-        KGE_CUDA_CHECK(h, cudaStreamWaitEvent(side, h->ev_loss, 0));
-    }
-    cudaStream_t sq = side ? side : s;
-    stage_begin(h, ST_ACCUM_Q, sq);
-    KGE_CUDA_CHECK(h, launch_accum<true>(p.kind, aq, sq));
-    stage_end(h, ST_ACCUM_Q, sq);
-    KGE_LAUNCH_CHECK(h);
-    if (side) KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_t, side));
     AccArgs at = aq;
     at.own = p.w.Tneg; at.oth = p.w.Q; at.own_rows = p.N; at.oth_rows = p.B; at.split = p.split_t;
     at.out = p.w.dTpart; at.out2 = nullptr; at.csum = p.w.Cpart;
-    stage_begin(h, ST_ACCUM_T, s);
-    KGE_CUDA_CHECK(h, launch_accum<false>(p.kind, at, s));
-    stage_end(h, ST_ACCUM_T, s);
-    KGE_LAUNCH_CHECK(h);
-    if (side) KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_t, 0));
+    if (p.kind != KIND_TH_L1 && p.kind != KIND_TH_L2) {
+        // the two accumulations are independent: one launch holds both
+        stage_begin(h, ST_ACCUM_Q, s);
+        KGE_CUDA_CHECK(h, launch_accum_tma(p.kind, aq, at, s));
+        stage_end(h, ST_ACCUM_Q, s);
+        KGE_LAUNCH_CHECK(h);
+    } else {
+        // TransH: two launches, concurrent when there is a side stream
+        if (side) {
+            KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_loss, s));
+            KGE_CUDA_CHECK(h, cudaStreamWaitEvent(side, h->ev_loss, 0));
+        }
+        cudaStream_t sq = side ? side : s;
+        stage_begin(h, ST_ACCUM_Q, sq);
+        KGE_CUDA_CHECK(h, launch_accum<true>(p.kind, aq, sq));
+        stage_end(h, ST_ACCUM_Q, sq);
+        KGE_LAUNCH_CHECK(h);
+        if (side) KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_t, side));
+        stage_begin(h, ST_ACCUM_T, s);
+        KGE_CUDA_CHECK(h, launch_accum<false>(p.kind, at, s));
+        stage_end(h, ST_ACCUM_T, s);
+        KGE_LAUNCH_CHECK(h);
+        if (side) KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_t, 0));
+    }
     }
     // the update follows the chain kernel directly: join the id sort here, where it has long finished
     if (dedup_side) KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_seg, 0));
