@@ -33,6 +33,7 @@ constexpr int TC_STAGES = 4;
 constexpr int TC_EPI_WARPS = 8;                           // epilogue warps of the training kernels: TC_EPI_GROUPS per tensor-memory lane quarter
 constexpr int TC_EPI_WARPS_TOPK = 16;                     // the filter epilogue of full-entity scoring profits from more
 constexpr int TC_EPI_GROUPS = TC_EPI_WARPS / 4;
+constexpr int TC_GRAD_STAGE_BYTES = 2048;                 // per epilogue warp: 32 rows x 32 bf16 columns on their way to memory
 constexpr int TC_PIECE = TC_BN / TC_EPI_GROUPS;           // columns of a 128-wide tile per piece of loss statistics
 __host__ __device__ constexpr int tc_epi_warps(int epi) { return (epi & 3) == 3 ? TC_EPI_WARPS_TOPK : TC_EPI_WARPS; }   // 3 = EPI_TOPK
 __host__ __device__ constexpr int tc_threads(int epi) { return 32 * (2 + tc_epi_warps(epi)); }
@@ -56,10 +57,11 @@ struct TcGemmParams {
     // fused loss epilogues (EPI_STATS, EPI_GRAD): the score is acc, or for l2 != 0 the distance score above
     int l2, loss;
     float gamma, adv_temp, ce_c, loss_scale;
-    float4* stat_part;                    // [M, pieces] per column piece of a tile: (max, sum exp, weighted loss sum, -)
+    int row_pieces;                       // pieces of TC_PIECE columns per row of stat_part / grow_part
+    float4* stat_part;                    // [M, row_pieces] per column piece: (max, sum exp, weighted loss sum, -)
     const float2* row_stat;               // [M] (max, 1 / normaliser) of the whole row
     uint16_t* Gb; int64_t ldg;            // [M, ldg] bf16 dL/dF (divided by the distance for l2)
-    float* grow_part;                     // [M, pieces] sums of the written values per column piece
+    float* grow_part;                     // [M, row_pieces] sums of the written values per column piece
     float* gcol_part;                     // [4 * tiles_m, N] sums per 32-row piece (l2 only)
     // full-entity scoring (EPI_TOPK): rows are queries, columns the entities [n_base, n_base + N)
     int m_fastest;                        // walk the row tiles of one column tile first (the column tile stays in L2)
@@ -233,8 +235,8 @@ __device__ __forceinline__ void tc_epilogue_stats(const TcGemmParams& p, const T
         if (valid1 == 32) tc_stats_chunk<L2, CE, true>(p, v1, rn, ncol + 32, valid1, k1, k0, m, z, l);
         else if (valid1 > 0) tc_stats_chunk<L2, CE, false>(p, v1, rn, ncol + 32, valid1, k1, k0, m, z, l);
     }
-    if (row < p.M)
-        p.stat_part[(int64_t)row * (TC_EPI_GROUPS * p.tiles_n) + (it.n0 / TC_BN) * TC_EPI_GROUPS + col_off / TC_PIECE] = make_float4(m, z, l, 0.f);
+    const int piece = (it.n0 + col_off) / TC_PIECE;
+    if (row < p.M && piece < p.row_pieces) p.stat_part[(int64_t)row * p.row_pieces + piece] = make_float4(m, z, l, 0.f);
 }
 
 __device__ __forceinline__ uint16_t bf16_bits(float v) {
@@ -257,8 +259,14 @@ __device__ __forceinline__ float tc_grad_one(const TcGemmParams& p, float acc, f
 
 // Second pass: dL/dF from the recomputed score and the row's final (base-2 max, 1 / normaliser),
 // written as bf16 for the two backward contractions (which read it K-major and MN-major).
+// A warp's 32 rows x 32 columns of bf16 pass through `stage` (2 KB of shared memory of its own)
+// on their way out, so that a store instruction writes whole 32-byte sectors: eight rows x 64
+// contiguous bytes instead of 16 bytes in each of 32 rows.  The 16-byte chunk c of row r sits at
+// chunk c ^ ((r >> 1) & 3) of the row: both the row-wise writes and the 8-row reads then touch
+// every bank once.
 template <bool L2, bool CE>
-__device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr) {
+__device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr,
+                                                 uint4* stage) {
     const bool rin = row < p.M;
     const float rn = (L2 && rin) ? p.row_norm2[row] : 0.f;
     const float2 st = rin ? p.row_stat[row] : make_float2(0.f, 0.f);
@@ -285,16 +293,24 @@ __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const Tc
             const __nv_bfloat162 pr = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
             g2[i] = *reinterpret_cast<const uint32_t*>(&pr);
         }
-        if (valid > 0) {
-            uint16_t* dst = p.Gb + (int64_t)row * p.ldg + ncol;
-            if (valid == 32) {
+        if (ncol + 32 <= p.N) {       // warp-uniform: all 32 columns lie inside the problem
+            const int sw = (lane >> 1) & 3;
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    reinterpret_cast<uint4*>(dst)[i] = make_uint4(g2[4 * i], g2[4 * i + 1], g2[4 * i + 2], g2[4 * i + 3]);
-            } else {
+            for (int i = 0; i < 4; ++i)
+                stage[lane * 4 + (i ^ sw)] = make_uint4(g2[4 * i], g2[4 * i + 1], g2[4 * i + 2], g2[4 * i + 3]);
+            __syncwarp();
+            const int row0 = row - lane;             // first of this warp's 32 rows
 #pragma unroll
-                for (int i = 0; i < 32; ++i) if (i < valid) dst[i] = (uint16_t)(g2[i >> 1] >> ((i & 1) * 16));
+            for (int i = 0; i < 4; ++i) {
+                const int r = i * 8 + (lane >> 2), c = lane & 3;
+                const uint4 val = stage[r * 4 + (c ^ ((r >> 1) & 3))];
+                if (row0 + r < p.M) *reinterpret_cast<uint4*>(p.Gb + (int64_t)(row0 + r) * p.ldg + ncol + c * 8) = val;
             }
+            __syncwarp();
+        } else if (valid > 0) {
+            uint16_t* dst = p.Gb + (int64_t)row * p.ldg + ncol;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) if (i < valid) dst[i] = (uint16_t)(g2[i >> 1] >> ((i & 1) * 16));
         }
         if (L2) {   // the norm expansion also needs the sums of what the contractions will see
 #pragma unroll
@@ -318,7 +334,8 @@ __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const Tc
                 p.gcol_part[(int64_t)((it.m0 / TC_BM) * 4 + ((row - it.m0) >> 5)) * p.N + ncol + lane] = v[0];
         }
     }
-    if (L2 && rin) p.grow_part[(int64_t)row * (TC_EPI_GROUPS * p.tiles_n) + (it.n0 / TC_BN) * TC_EPI_GROUPS + col_off / TC_PIECE] = rsum;
+    const int piece = (it.n0 + col_off) / TC_PIECE;
+    if (L2 && rin && piece < p.row_pieces) p.grow_part[(int64_t)row * p.row_pieces + piece] = rsum;
 }
 
 // Largest float below x (x finite or -inf; -inf maps to itself).
@@ -404,10 +421,16 @@ __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const Tc
 // this thread's tensor-memory lane (taddr points at the first of them).
 template <int EPI, int WIDTH>
 __device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr, int32_t* beat_sm) {
-    static_assert((EPI & 3) == EPI_STORE || (EPI & 3) == EPI_TOPK || WIDTH == TC_PIECE, "the fused loss epilogues work on fixed pieces of a 128-column tile");
-    if ((EPI & 3) == EPI_STATS) { tc_epilogue_stats<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, col_off, taddr); return; }
+    static_assert((EPI & 3) == EPI_STORE || (EPI & 3) == EPI_TOPK || WIDTH % TC_PIECE == 0, "the fused loss epilogues work on pieces of TC_PIECE columns");
+    if ((EPI & 3) == EPI_STATS || (EPI & 3) == EPI_GRAD) {
+#pragma unroll 1
+        for (int c = 0; c < WIDTH; c += TC_PIECE) {
+            if ((EPI & 3) == EPI_STATS) tc_epilogue_stats<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, col_off + c, taddr + (uint32_t)c);
+            else tc_epilogue_grad<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, col_off + c, taddr + (uint32_t)c, reinterpret_cast<uint4*>(beat_sm));
+        }
+        return;
+    }
     if ((EPI & 3) == EPI_TOPK) { tc_epilogue_topk<WIDTH>(p, it, row, col_off, taddr, beat_sm); return; }
-    if ((EPI & 3) == EPI_GRAD) { tc_epilogue_grad<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, col_off, taddr); return; }
     float* const Cout = p.C + (int64_t)it.z * p.split_stride;
 #pragma unroll 1
     for (int c0 = col_off; c0 < col_off + WIDTH; c0 += 32) {
@@ -546,7 +569,9 @@ __global__ void __launch_bounds__(tc_threads(EPI)) tc_gemm_kernel(const __grid_c
             if (!ok || *stop) { if (lane == 0) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); } break; }
             const TcItem it = tc_item(p, item);
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cgrp * (BN / EG));
-            tc_epilogue<EPI, BN / EG>(p, it, it.m0 + quarter * 32 + lane, cgrp * (BN / EG), taddr, beat_sm);
+            // scratch after the barriers: the rank counts of EPI_TOPK, or 2 KB per epilogue warp for EPI_GRAD's stores
+            int32_t* scratch = (EPI & 3) == EPI_GRAD ? beat_sm + (warp - 2) * (TC_GRAD_STAGE_BYTES / 4) : beat_sm;
+            tc_epilogue<EPI, BN / EG>(p, it, it.m0 + quarter * 32 + lane, cgrp * (BN / EG), taddr, scratch);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
@@ -665,7 +690,9 @@ template <int EPI, int BN = 128, bool A_MN = false, bool B_MN = false>
 cudaError_t launch_gemm_inst(const unsigned char* tmA, const unsigned char* tmB, const TcGemmParams& p, int num_sms, cudaStream_t s,
                              size_t extra_smem = 0) {
     constexpr size_t smem = tc_smem_bytes(BN);
-    constexpr size_t extra_max = (EPI & 3) == EPI_TOPK ? (size_t)TC_BEAT_ROWS_MAX * 4 : 0;
+    constexpr size_t extra_max = (EPI & 3) == EPI_TOPK ? (size_t)TC_BEAT_ROWS_MAX * 4
+                               : ((EPI & 3) == EPI_GRAD ? (size_t)tc_epi_warps(EPI) * TC_GRAD_STAGE_BYTES : 0);
+    if ((EPI & 3) == EPI_GRAD) extra_smem = extra_max;
     static bool configured = false;
     if (!configured) {
         const cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<EPI, BN, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -678,19 +705,23 @@ cudaError_t launch_gemm_inst(const unsigned char* tmA, const unsigned char* tmB,
     return cudaSuccess;
 }
 
-// Scores Q . T^T with one of the fused loss epilogues.
-cudaError_t launch_fused(int pass, bool l2, bool ce, kge_handle* h, const TcGemmParams& p, cudaStream_t s) {
+// Scores Q . T^T with one of the fused loss epilogues, in tiles of BN columns.
+template <int BN>
+cudaError_t launch_fused_bn(int pass, bool l2, bool ce, kge_handle* h, const TcGemmParams& p, cudaStream_t s) {
     const int key = (pass == EPI_GRAD ? 4 : 0) | (l2 ? 2 : 0) | (ce ? 1 : 0);
     switch (key) {
-        case 0: return launch_gemm_inst<EPI_STATS>(h->tm_q, h->tm_t, p, h->num_sms, s);
-        case 1: return launch_gemm_inst<EPI_STATS | EPI_CE>(h->tm_q, h->tm_t, p, h->num_sms, s);
-        case 2: return launch_gemm_inst<EPI_STATS | EPI_L2>(h->tm_q, h->tm_t, p, h->num_sms, s);
-        case 3: return launch_gemm_inst<EPI_STATS | EPI_L2 | EPI_CE>(h->tm_q, h->tm_t, p, h->num_sms, s);
-        case 4: return launch_gemm_inst<EPI_GRAD>(h->tm_q, h->tm_t, p, h->num_sms, s);
-        case 5: return launch_gemm_inst<EPI_GRAD | EPI_CE>(h->tm_q, h->tm_t, p, h->num_sms, s);
-        case 6: return launch_gemm_inst<EPI_GRAD | EPI_L2>(h->tm_q, h->tm_t, p, h->num_sms, s);
-        default: return launch_gemm_inst<EPI_GRAD | EPI_L2 | EPI_CE>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        case 0: return launch_gemm_inst<EPI_STATS, BN>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        case 1: return launch_gemm_inst<EPI_STATS | EPI_CE, BN>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        case 2: return launch_gemm_inst<EPI_STATS | EPI_L2, BN>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        case 3: return launch_gemm_inst<EPI_STATS | EPI_L2 | EPI_CE, BN>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        case 4: return launch_gemm_inst<EPI_GRAD, BN>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        case 5: return launch_gemm_inst<EPI_GRAD | EPI_CE, BN>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        case 6: return launch_gemm_inst<EPI_GRAD | EPI_L2, BN>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        default: return launch_gemm_inst<EPI_GRAD | EPI_L2 | EPI_CE, BN>(h->tm_q, h->tm_t, p, h->num_sms, s);
     }
+}
+cudaError_t launch_fused(int pass, bool l2, bool ce, kge_handle* h, const TcGemmParams& p, cudaStream_t s) {
+    return p.bn == 256 ? launch_fused_bn<256>(pass, l2, ce, h, p, s) : launch_fused_bn<128>(pass, l2, ce, h, p, s);
 }
 }  // namespace
 
@@ -703,8 +734,11 @@ int launch_tc_forward(kge_handle* h, cudaStream_t s) {
     TcGemmParams p{};
     p.M = c.batch; p.N = c.num_neg; p.K = c.dim;
     p.kb_per_split = (p.K + TC_BK - 1) / TC_BK; p.split_stride = 0;
-    p.bn = TC_BN;
-    p.tiles_m = (p.M + TC_BM - 1) / TC_BM; p.tiles_n = (p.N + TC_BN - 1) / TC_BN; p.items = p.tiles_m * p.tiles_n;
+    // 256-column tiles halve the operand bytes fetched per score (the row tile is shared by twice
+    // the columns); narrow problems keep 128 so that the tiles still spread over the SMs
+    p.bn = (p.N >= 1024 && (int64_t)((p.M + TC_BM - 1) / TC_BM) * ((p.N + 255) / 256) >= h->num_sms) ? 256 : TC_BN;
+    p.tiles_m = (p.M + TC_BM - 1) / TC_BM; p.tiles_n = (p.N + p.bn - 1) / p.bn; p.items = p.tiles_m * p.tiles_n;
+    p.row_pieces = TC_EPI_GROUPS * ((p.N + TC_BN - 1) / TC_BN);
     p.C = nullptr; p.ldc = 0;
     p.row_norm2 = w.qn2; p.col_norm2 = w.tn2;
     p.status = w.status;
@@ -719,14 +753,14 @@ int launch_tc_forward(kge_handle* h, cudaStream_t s) {
     stage_end(h, ST_BLOCK, s);
     KGE_LAUNCH_CHECK(h);
     stage_begin(h, ST_LOSS, s);
-    CombineParams cp{p.stat_part, TC_EPI_GROUPS * p.tiles_n, p.M, w.fpos, c.loss, c.gamma, c.ce_correction, c.loss_scale,
+    CombineParams cp{p.stat_part, p.row_pieces, p.M, w.fpos, c.loss, c.gamma, c.ce_correction, c.loss_scale,
                      reinterpret_cast<float2*>(w.row_stat), w.Lrow, w.gpos};
     stats_combine_kernel<<<(p.M * 32 + 255) / 256, 256, 0, s>>>(cp);
     KGE_LAUNCH_CHECK(h);
     KGE_CUDA_CHECK(h, launch_fused(EPI_GRAD, p.l2 != 0, ce, h, p, s));
     KGE_LAUNCH_CHECK(h);
     if (p.l2) {
-        grad_sums_kernel<<<(p.M + p.N + 255) / 256, 256, 0, s>>>(w.grow_part, TC_EPI_GROUPS * p.tiles_n, w.Grow, p.M,
+        grad_sums_kernel<<<(p.M + p.N + 255) / 256, 256, 0, s>>>(w.grow_part, p.row_pieces, w.Grow, p.M,
                                                                  w.gcol_part, 4 * p.tiles_m, w.Gcol, p.N);
         KGE_LAUNCH_CHECK(h);
     }

@@ -161,6 +161,18 @@ def test_tensor_core_score_block(oracle64, score, p, d):
     _run(oracle64, prob, steps=1)
 
 
+@pytest.mark.parametrize("score,p,loss,N", [("distmult", 1, "softmax", 2400), ("transe", 2, "logsigmoid", 2500),
+                                            ("complex", 1, "logsigmoid", 2560)])
+def test_tensor_core_wide_tiles(oracle64, score, p, loss, N):
+    """Enough tiles to fill every SM, which switches the fused forward passes to 256-column
+    tiles: N = 2400 leaves the last tile's upper half outside the problem (its statistics pieces
+    do not exist), N = 2500 a ragged last piece, N = 2560 none."""
+    prob = Problem(E=20000, R=9, T=60000, d=64, score=score, p_norm=p, loss=loss, B=2048, N=N, P=2,
+                   ce_correction=0.3, gamma=4.0 if score == "transe" else 0.0, adv_temp=0.5 if loss == "logsigmoid" else 0.0,
+                   lr=0.05, graph_seed=11, relation_zipf=1.0, tc=True)
+    _run(oracle64, prob, steps=1)
+
+
 def test_tensor_core_path_refuses_what_it_cannot_do():
     import paper_2211_12281_b200 as K
     for kw in (dict(score="transe", p_norm=1, dim=128), dict(score="rotate", p_norm=2, dim=128),
