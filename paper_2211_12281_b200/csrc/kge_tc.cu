@@ -41,7 +41,7 @@ constexpr uint32_t TC_A_BYTES = TC_BM * TC_BK * 2;
 constexpr uint32_t TC_MN_GROUP_BYTES = 64 * TC_BK * 2;    // MN-major operand: 64 contiguous elements x 64 K rows per TMA box
 __host__ __device__ constexpr uint32_t tc_stage_bytes(int bn) { return TC_A_BYTES + (uint32_t)bn * TC_BK * 2; }
 __host__ __device__ constexpr size_t tc_smem_bytes(int bn) { return 1024 + (size_t)TC_STAGES * tc_stage_bytes(bn) + 128; }
-constexpr int TC_BEAT_ROWS_MAX = 20 * 1024;                // queries whose rank counts fit in shared memory beside the stages
+constexpr int TC_BEAT_ROWS_MAX = 8 * 1024;                 // queries whose rank counts fit in shared memory beside the 256-column stages
 
 enum { EPI_STORE = 0, EPI_STATS = 1, EPI_GRAD = 2, EPI_TOPK = 3, EPI_L2 = 4, EPI_CE = 8 };   // L2 / CE: flags of the fused loss epilogues
 
@@ -338,6 +338,19 @@ __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const Tc
     if (L2 && rin && piece < p.row_pieces) p.grow_part[(int64_t)row * p.row_pieces + piece] = rsum;
 }
 
+// 1.0f if a > b, else 0.0f, in one instruction.
+__device__ __forceinline__ float one_if_gt(float a, float b) {
+    float r;
+    asm("set.gt.f32.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+    return r;
+}
+// Maximum of three in one instruction.
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
 // Largest float below x (x finite or -inf; -inf maps to itself).
 __device__ __forceinline__ float float_below(float x) {
     if (x == 0.f) return __uint_as_float(0x80000001u);
@@ -380,9 +393,13 @@ __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const Tc
         // rank of the true tail
         if (tt >= 0) {
             if (tt < e0 || tt >= e0 + 32) {
+                // counted in floating point (exact: at most 32 per chain) on four independent chains:
+                // the comparison yields 1.0f and the additions go to the FMA pipe
                 const float c = tt >= e0 + 32 ? ft_lo : ft;
+                float n[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int i = 0; i < 32; ++i) beat += v[i] > c ? 1 : 0;
+                for (int i = 0; i < 32; ++i) n[i & 3] += one_if_gt(v[i], c);
+                beat += (int)((n[0] + n[1]) + (n[2] + n[3]));
             } else {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
@@ -392,9 +409,11 @@ __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const Tc
             }
         }
         // candidates: anything ordered before the current k-th best
-        float vmax = v[0];
+        float vm[4];           // a tree of three-input maxima, not a chain of 31
 #pragma unroll
-        for (int i = 1; i < 32; ++i) vmax = fmaxf(vmax, v[i]);
+        for (int j = 0; j < 4; ++j)
+            vm[j] = max3(max3(v[8 * j], v[8 * j + 1], v[8 * j + 2]), max3(v[8 * j + 3], v[8 * j + 4], v[8 * j + 5]), fmaxf(v[8 * j + 6], v[8 * j + 7]));
+        const float vmax = fmaxf(max3(vm[0], vm[1], vm[2]), vm[3]);
         if (vmax > thr_lo) {   // rare once the threshold has tightened
 #pragma unroll
             for (int i = 0; i < 32; ++i) {     // (padded columns hold -inf and never pass)
@@ -502,6 +521,15 @@ __global__ void __launch_bounds__(tc_threads(EPI)) tc_gemm_kernel(const __grid_c
     if (warp == 0) {
         if (lane == 0) {
             int ring = 0;    // slices issued so far: stage = ring % STAGES, phase = ring / STAGES
+            // Without K splits and with a slice count that divides the ring, slice kb of every item
+            // lands in the same stages, so the operand that consecutive items share (the row tile
+            // when column tiles vary fastest, the column tile otherwise) is still there from the item
+            // before: it is fetched again only when it changes.  keep[s] = first row (or column) of
+            // the shared operand held by stage s.
+            const bool reuse = p.kb_per_split == kb_total && TC_STAGES % kb_total == 0;
+            int keep[TC_STAGES];
+#pragma unroll
+            for (int s = 0; s < TC_STAGES; ++s) keep[s] = -1;
             for (int item = item_begin; item < item_end && !*stop; ++item) {
                 const TcItem it = tc_item(p, item);
                 const int kb0 = it.z * p.kb_per_split, nkb = min(p.kb_per_split, kb_total - kb0);
@@ -509,16 +537,23 @@ __global__ void __launch_bounds__(tc_threads(EPI)) tc_gemm_kernel(const __grid_c
                     const int s = ring % TC_STAGES;
                     if (!mbar_wait_bounded(&empty[s], ((ring / TC_STAGES) & 1) ^ 1)) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); break; }
                     unsigned char* sa = base + (size_t)s * TC_STAGE_BYTES;
-                    mbar_arrive_expect_tx(&full[s], TC_STAGE_BYTES);
+                    const int shared_at = p.m_fastest ? it.n0 : it.m0;
+                    bool have = false;
+#pragma unroll
+                    for (int q = 0; q < TC_STAGES; ++q) if (q == s) { have = reuse && keep[q] == shared_at; keep[q] = shared_at; }
+                    const bool load_a = !(have && !p.m_fastest), load_b = !(have && p.m_fastest);
+                    mbar_arrive_expect_tx(&full[s], (load_a ? TC_A_BYTES : 0u) + (load_b ? TC_STAGE_BYTES - TC_A_BYTES : 0u));
                     const int k0 = (kb0 + kb) * TC_BK;
-                    if (A_MN) {
+                    if (!load_a) {
+                    } else if (A_MN) {
 #pragma unroll
                         for (int g = 0; g < TC_BM / 64; ++g) tma_load_2d(sa + g * TC_MN_GROUP_BYTES, &tmA, it.m0 + 64 * g, k0, &full[s]);
                     } else {
                         tma_load_2d(sa, &tmA, k0, it.m0, &full[s]);
                     }
                     unsigned char* sb = sa + TC_A_BYTES;
-                    if (B_MN) {
+                    if (!load_b) {
+                    } else if (B_MN) {
 #pragma unroll
                         for (int g = 0; g < BN / 64; ++g) tma_load_2d(sb + g * TC_MN_GROUP_BYTES, &tmB, it.n0 + 64 * g, k0, &full[s]);
                     } else {
@@ -844,8 +879,8 @@ int launch_tc_infer_chunk(kge_handle* h, int nq, int64_t e_lo, int64_t e_hi, con
     TcGemmParams p{};
     p.M = nq; p.N = (int)(e_hi - e_lo); p.K = h->cfg.dim;
     p.kb_per_split = (p.K + TC_BK - 1) / TC_BK;
-    p.bn = TC_BN;
-    p.tiles_m = (p.M + TC_BM - 1) / TC_BM; p.tiles_n = (p.N + TC_BN - 1) / TC_BN;
+    p.bn = 256;      // a row tile of queries is shared by 256 entities
+    p.tiles_m = (p.M + TC_BM - 1) / TC_BM; p.tiles_n = (p.N + p.bn - 1) / p.bn;
     if ((int64_t)p.tiles_m * p.tiles_n > 0x7fffffff) return KGE_ERR_BAD_ARG;
     p.items = p.tiles_m * p.tiles_n;
     p.status = w.status;
@@ -853,9 +888,9 @@ int launch_tc_infer_chunk(kge_handle* h, int nq, int64_t e_lo, int64_t e_hi, con
     p.thr = w.thr; p.thr_id = w.thr_id; p.ftrue = w.iftrue; p.tt = true_tails;
     p.cand_cnt = w.cand_cnt; p.beat_tmp = w.beat_tmp; p.cand_score = w.cand_score; p.cand_id = w.cand_id;
     p.cand_cap = kCandCap; p.overflow = w.status + 1;
-    p.beat_rows = std::min(nq, TC_BEAT_ROWS_MAX);
+    p.beat_rows = std::min(nq, TC_BEAT_ROWS_MAX);   // the other rows count with global atomics
     // (the table's tensor map covers all rows; the kernel offsets its row coordinate by n_base)
-    KGE_CUDA_CHECK(h, launch_gemm_inst<EPI_TOPK>(h->tm_iq, h->tm_eb, p, h->num_sms, s, (size_t)p.beat_rows * 4));
+    KGE_CUDA_CHECK(h, (launch_gemm_inst<EPI_TOPK, 256>(h->tm_iq, h->tm_eb, p, h->num_sms, s, (size_t)p.beat_rows * 4)));
     KGE_LAUNCH_CHECK(h);
     return KGE_OK;
 }
