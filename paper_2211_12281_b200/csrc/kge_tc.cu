@@ -370,7 +370,9 @@ __device__ __forceinline__ float float_below(float x) {
 template <int WIDTH>
 __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr, int32_t* beat_sm) {
     const bool rin = row < p.M;
-    float thr = 0.f, ft = 0.f; int32_t thr_id = 0, tt = -1;
+    // rows outside the problem stay in the loop (the warp votes below need every lane): no true
+    // tail, and a threshold nothing exceeds
+    float thr = INFINITY, ft = 0.f; int32_t thr_id = 0, tt = -1;
     if (rin) {
         thr = p.thr[row]; thr_id = p.thr_id[row];
         if (p.tt) { ft = p.ftrue[row]; tt = p.tt[row]; }
@@ -381,26 +383,27 @@ __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const Tc
     for (int c0 = col_off; c0 < col_off + WIDTH; c0 += 32) {
         float v[32];
         tmem_ld32(taddr + (uint32_t)(c0 - col_off), v);
-        if (!rin) continue;
         const int ncol = it.n0 + c0;
-        const int valid = min(32, p.N - ncol);
+        const int valid = min(32, p.N - ncol);          // the same for every lane
         if (valid <= 0) continue;
         const int32_t e0 = (int32_t)(p.n_base + ncol);
         if (valid != 32) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) if (i >= valid) v[i] = -INFINITY;   // never counted, never a candidate
         }
-        // rank of the true tail
-        if (tt >= 0) {
-            if (tt < e0 || tt >= e0 + 32) {
-                // counted in floating point (exact: at most 32 per chain) on four independent chains:
+        // rank of the true tail.  The branch is taken by the whole warp (a vote), so that the
+        // element-by-element form stays out of the instruction stream of the common case.
+        if (p.tt) {
+            const bool inside = tt >= e0 && tt < e0 + 32;
+            if (!__any_sync(0xffffffffu, inside)) {
+                // counted in floating point (exact: at most 8 per chain) on four independent chains:
                 // the comparison yields 1.0f and the additions go to the FMA pipe
                 const float c = tt >= e0 + 32 ? ft_lo : ft;
                 float n[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int i = 0; i < 32; ++i) n[i & 3] += one_if_gt(v[i], c);
-                beat += (int)((n[0] + n[1]) + (n[2] + n[3]));
-            } else {
+                if (tt >= 0) beat += (int)((n[0] + n[1]) + (n[2] + n[3]));
+            } else if (tt >= 0) {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
                     const int32_t e = e0 + i;
@@ -414,18 +417,20 @@ __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const Tc
         for (int j = 0; j < 4; ++j)
             vm[j] = max3(max3(v[8 * j], v[8 * j + 1], v[8 * j + 2]), max3(v[8 * j + 3], v[8 * j + 4], v[8 * j + 5]), fmaxf(v[8 * j + 6], v[8 * j + 7]));
         const float vmax = fmaxf(max3(vm[0], vm[1], vm[2]), vm[3]);
-        if (vmax > thr_lo) {   // rare once the threshold has tightened
+        if (__any_sync(0xffffffffu, vmax > thr_lo)) {   // rare once the threshold has tightened
+            if (vmax > thr_lo) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {     // (padded columns hold -inf and never pass)
-                const float f = v[i];
-                const int32_t e = e0 + i;
-                if (f > thr || (f == thr && e < thr_id && f != -INFINITY)) {
-                    const int slot = atomicAdd(&p.cand_cnt[row], 1);
-                    if (slot < p.cand_cap) {
-                        p.cand_score[(int64_t)row * p.cand_cap + slot] = f;
-                        p.cand_id[(int64_t)row * p.cand_cap + slot] = e;
-                    } else {
-                        *p.overflow = 1;   // the host redoes this chunk in pieces that cannot overflow
+                for (int i = 0; i < 32; ++i) {     // (padded columns hold -inf and never pass)
+                    const float f = v[i];
+                    const int32_t e = e0 + i;
+                    if (f > thr || (f == thr && e < thr_id && f != -INFINITY)) {
+                        const int slot = atomicAdd(&p.cand_cnt[row], 1);
+                        if (slot < p.cand_cap) {
+                            p.cand_score[(int64_t)row * p.cand_cap + slot] = f;
+                            p.cand_id[(int64_t)row * p.cand_cap + slot] = e;
+                        } else {
+                            *p.overflow = 1;   // the host redoes this chunk in pieces that cannot overflow
+                        }
                     }
                 }
             }
@@ -481,7 +486,7 @@ __device__ __forceinline__ TcItem tc_item(const TcGemmParams& p, int64_t item) {
 // the operand is read MN-major (its tensor map has the contraction index as rows), which is how
 // dL/dF, Q and T serve as transposed operands without a transposed copy.
 template <int EPI, int BN = 128, bool A_MN = false, bool B_MN = false>
-__global__ void __launch_bounds__(tc_threads(EPI)) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
+__global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
                                                              const __grid_constant__ CUtensorMap tmB, TcGemmParams p) {
     constexpr uint32_t TC_STAGE_BYTES = tc_stage_bytes(BN);
     constexpr uint32_t TC_TMEM_COLS = 2 * BN;          // two fp32 accumulators, used in turn
