@@ -215,18 +215,22 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+// One test of the barrier phase `parity`.  The hardware may park the thread for up to about
+// `hint_ns` while the phase is incomplete (it wakes as soon as the phase completes), so a waiting
+// thread does not fill its scheduler's issue slots with polls.
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, uint32_t hint_ns = 2000u) {
     uint32_t ok;
     asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns) : "memory");
     return ok != 0;
 }
-// Polls the barrier phase `parity` a bounded number of times; false = gave up.
+// Waits for the barrier phase `parity` a bounded number of times (each up to the hint above,
+// then a short sleep: seconds in all); false = gave up.
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
     for (int i = 0; i < (1 << 20); ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (i > 128) __nanosleep(64);
+        if (i > 16) __nanosleep(256);
     }
     return false;
 }
