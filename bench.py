@@ -96,7 +96,7 @@ STAGE_OPS = {
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
 # summarised in profiles/train_step_c2_transe_l1_launches.md (None once the kernel has changed since).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {("c2_transe_l1", "accum"): 5.29e6, ("c2_transe_l1", "block"): 1.07e6}
 
 
 def cfg_kwargs(w, seed):

@@ -378,6 +378,7 @@ __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const Tc
         if (p.tt) { ft = p.ftrue[row]; tt = p.tt[row]; }
     }
     const float thr_lo = float_below(thr), ft_lo = float_below(ft);
+    const int lane = threadIdx.x & 31;
     int beat = 0;
 #pragma unroll 1
     for (int c0 = col_off; c0 < col_off + WIDTH; c0 += 32) {
@@ -417,21 +418,32 @@ __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const Tc
         for (int j = 0; j < 4; ++j)
             vm[j] = max3(max3(v[8 * j], v[8 * j + 1], v[8 * j + 2]), max3(v[8 * j + 3], v[8 * j + 4], v[8 * j + 5]), fmaxf(v[8 * j + 6], v[8 * j + 7]));
         const float vmax = fmaxf(max3(vm[0], vm[1], vm[2]), vm[3]);
-        if (__any_sync(0xffffffffu, vmax > thr_lo)) {   // rare once the threshold has tightened
-            if (vmax > thr_lo) {
+        // Rare once the threshold has tightened, but one warp of the sixteen that share a tile
+        // meets it at most tiles, and the tile waits for its slowest warp.  So the warp takes the
+        // flagged lanes one at a time and spreads that lane's 32 scores over its 32 lanes (one
+        // shuffle per score): the ordering test and the append then run once per lane, not 32
+        // times in a row.
+        unsigned pending = __ballot_sync(0xffffffffu, vmax > thr_lo);
+        while (pending) {
+            const int src = __ffs(pending) - 1;
+            pending &= pending - 1;
+            float f = 0.f;
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {     // (padded columns hold -inf and never pass)
-                    const float f = v[i];
-                    const int32_t e = e0 + i;
-                    if (f > thr || (f == thr && e < thr_id && f != -INFINITY)) {
-                        const int slot = atomicAdd(&p.cand_cnt[row], 1);
-                        if (slot < p.cand_cap) {
-                            p.cand_score[(int64_t)row * p.cand_cap + slot] = f;
-                            p.cand_id[(int64_t)row * p.cand_cap + slot] = e;
-                        } else {
-                            *p.overflow = 1;   // the host redoes this chunk in pieces that cannot overflow
-                        }
-                    }
+            for (int i = 0; i < 32; ++i) {
+                const float t = __shfl_sync(0xffffffffu, v[i], src);
+                if (lane == i) f = t;
+            }
+            const float thr_s = __shfl_sync(0xffffffffu, thr, src);
+            const int32_t id_s = __shfl_sync(0xffffffffu, thr_id, src);
+            const int row_s = __shfl_sync(0xffffffffu, row, src);
+            const int32_t e = e0 + lane;
+            if (f > thr_s || (f == thr_s && e < id_s && f != -INFINITY)) {     // (padded columns hold -inf and never pass)
+                const int slot = atomicAdd(&p.cand_cnt[row_s], 1);
+                if (slot < p.cand_cap) {
+                    p.cand_score[(int64_t)row_s * p.cand_cap + slot] = f;
+                    p.cand_id[(int64_t)row_s * p.cand_cap + slot] = e;
+                } else {
+                    *p.overflow = 1;   // the host redoes this chunk in pieces that cannot overflow
                 }
             }
         }
