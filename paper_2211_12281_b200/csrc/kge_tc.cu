@@ -40,7 +40,7 @@ __host__ __device__ constexpr int tc_threads(int epi) { return 32 * (2 + tc_epi_
 constexpr uint32_t TC_A_BYTES = TC_BM * TC_BK * 2;
 constexpr uint32_t TC_MN_GROUP_BYTES = 64 * TC_BK * 2;    // MN-major operand: 64 contiguous elements x 64 K rows per TMA box
 __host__ __device__ constexpr uint32_t tc_stage_bytes(int bn) { return TC_A_BYTES + (uint32_t)bn * TC_BK * 2; }
-__host__ __device__ constexpr size_t tc_smem_bytes(int bn) { return 1024 + (size_t)TC_STAGES * tc_stage_bytes(bn) + 128; }
+__host__ __device__ constexpr size_t tc_smem_bytes(int bn) { return 1024 + (size_t)TC_STAGES * tc_stage_bytes(bn) + 256; }
 constexpr int TC_BEAT_ROWS_MAX = 8 * 1024;                 // queries whose rank counts fit in shared memory beside the 256-column stages
 
 enum { EPI_STORE = 0, EPI_STATS = 1, EPI_GRAD = 2, EPI_TOPK = 3, EPI_L2 = 4, EPI_CE = 8 };   // L2 / CE: flags of the fused loss epilogues
@@ -501,17 +501,18 @@ template <int EPI, int BN = 128, bool A_MN = false, bool B_MN = false>
 __global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
                                                              const __grid_constant__ CUtensorMap tmB, TcGemmParams p) {
     constexpr uint32_t TC_STAGE_BYTES = tc_stage_bytes(BN);
-    constexpr uint32_t TC_TMEM_COLS = 2 * BN;          // two fp32 accumulators, used in turn
+    constexpr int NACC = 512 / BN;                      // fp32 accumulators in tensor memory, used in turn: all 512 columns
+    constexpr uint32_t TC_TMEM_COLS = NACC * BN;
     constexpr int EW = tc_epi_warps(EPI), EG = EW / 4, TC_THREADS = tc_threads(EPI);
     extern __shared__ unsigned char tc_smem_raw[];
     unsigned char* base = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
     uint64_t* full = reinterpret_cast<uint64_t*>(base + (size_t)TC_STAGES * TC_STAGE_BYTES);
     uint64_t* empty = full + TC_STAGES;
     uint64_t* acc_full = empty + TC_STAGES;      // [2] accumulator buffer written
-    uint64_t* acc_empty = acc_full + 2;          // [2] accumulator buffer drained by all epilogue warps
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    uint64_t* acc_empty = acc_full + NACC;       // [NACC] accumulator buffer drained by all epilogue warps
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + NACC);
     volatile uint32_t* stop = tmem_slot + 1;     // set by a warp whose wait ran out
-    int32_t* beat_sm = reinterpret_cast<int32_t*>(base + (size_t)TC_STAGES * TC_STAGE_BYTES + 128);   // [beat_rows], EPI_TOPK
+    int32_t* beat_sm = reinterpret_cast<int32_t*>(base + (size_t)TC_STAGES * TC_STAGE_BYTES + 256);   // [beat_rows], EPI_TOPK
     if ((EPI & 3) == EPI_TOPK)
         for (int i = threadIdx.x; i < p.beat_rows; i += TC_THREADS) beat_sm[i] = 0;
 
@@ -522,7 +523,7 @@ __global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __gri
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < TC_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EW); }
+        for (int b = 0; b < NACC; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EW); }
         *stop = 0;
         mbar_init_fence();
     }
@@ -589,9 +590,9 @@ __global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __gri
             for (int item = item_begin, local = 0; item < item_end && ok && !*stop; ++item, ++local) {
                 const TcItem it = tc_item(p, item);
                 const int nkb = min(p.kb_per_split, kb_total - it.z * p.kb_per_split);
-                const int buf = local & 1;
+                const int buf = local % NACC;
                 // the epilogue warps must have drained this buffer (two items ago)
-                if (!mbar_wait_bounded(&acc_empty[buf], ((local >> 1) & 1) ^ 1)) { ok = false; break; }
+                if (!mbar_wait_bounded(&acc_empty[buf], ((local / NACC) & 1) ^ 1)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_acc = tmem_base + (uint32_t)buf * BN;
                 for (int kb = 0; kb < nkb; ++kb, ++ring) {
@@ -615,8 +616,8 @@ __global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __gri
         const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
         const int cgrp = (warp - 2) >> 2;              // which group of the tile's columns
         for (int item = item_begin, local = 0; item < item_end; ++item, ++local) {
-            const int buf = local & 1;
-            const bool ok = mbar_wait_bounded(&acc_full[buf], (local >> 1) & 1);
+            const int buf = local % NACC;
+            const bool ok = mbar_wait_bounded(&acc_full[buf], (local / NACC) & 1);
             tc_fence_after();
             if (!ok || *stop) { if (lane == 0) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); } break; }
             const TcItem it = tc_item(p, item);
