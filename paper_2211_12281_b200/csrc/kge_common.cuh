@@ -168,6 +168,8 @@ int launch_update(kge_handle* h, uint64_t step, float lr, cudaStream_t s);
 int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows);
 int tc_backward_tile_cols(int cols);
 int tc_pieces_per_tile();
+// The dT contraction of the dot-product kinds with a single K split is the negatives' gradient rows: it writes them in place.
+bool tc_negatives_direct(const kge_handle* h);
 int launch_tc_backward(kge_handle* h, cudaStream_t s, cudaStream_t side);
 int launch_tc_forward(kge_handle* h, cudaStream_t s);
 int launch_cast_bf16(kge_handle* h, const float* src, uint16_t* dst, int64_t count, cudaStream_t s);

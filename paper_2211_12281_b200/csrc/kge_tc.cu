@@ -842,6 +842,10 @@ int launch_tc_bwd_gemm(kge_handle* h, const unsigned char* tmA, const unsigned c
 }
 }  // namespace
 
+bool tc_negatives_direct(const kge_handle* h) {
+    return h->cfg.prec == KGE_PREC_BF16_TC && h->kind == KIND_DOT && h->split_t == 1;
+}
+
 // Columns per tile of a backward contraction whose output rows are `cols` wide.
 int tc_backward_tile_cols(int cols) { return cols > 128 ? 256 : 128; }
 
@@ -865,7 +869,9 @@ int launch_tc_backward(kge_handle* h, cudaStream_t s, cudaStream_t side) {
     stage_end(h, ST_ACCUM_Q, s);
     if (rc != KGE_OK) return rc;
     stage_begin(h, ST_ACCUM_T, s);
-    rc = launch_tc_bwd_gemm<true>(h, h->tm_g64, h->tm_q64, N, d, B, h->split_t, w.dTpart, d, s);
+    // one split and no correction term: these rows are final, so they go where the update reads them
+    float* dT_out = tc_negatives_direct(h) ? w.grad_ent + (size_t)2 * B * d : w.dTpart;
+    rc = launch_tc_bwd_gemm<true>(h, h->tm_g64, h->tm_q64, N, d, B, h->split_t, dT_out, d, s);
     stage_end(h, ST_ACCUM_T, s);
     return rc;
 }

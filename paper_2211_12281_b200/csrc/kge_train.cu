@@ -25,6 +25,7 @@ struct TrainParams {
     int slots_per_bucket;
     SampleParams sp;
     int tc_l2;          // TransE p = 2 with tensor-core backward: the splits hold C.T and C^T.Q, C = dL/dF / distance
+    int neg_direct;     // the dT contraction wrote the negatives' gradient rows itself (one K split, no correction term)
     Workspace w;
 };
 
@@ -987,7 +988,7 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
         return;
     }
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (warp >= p.B + p.N) return;
+    if (warp >= p.B + (p.neg_direct ? 0 : p.N)) return;
     const int d4 = p.d4;
     float4* gent = reinterpret_cast<float4*>(p.w.grad_ent);
     if (warp >= p.B) {
@@ -1271,6 +1272,7 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     p.sp.heads = h->ws.heads; p.sp.rels = h->ws.rels; p.sp.tails = h->ws.tails; p.sp.negs = h->ws.negs;
     p.slots_per_bucket = c.batch / (c.head_part < 0 ? c.num_parts * c.num_parts : c.num_parts);
     p.tc_l2 = c.prec == KGE_PREC_BF16_TC && p.kind == KIND_L2;
+    p.neg_direct = tc_negatives_direct(h) ? 1 : 0;
     p.w = h->ws;
     const int nch = p.d4 <= 32 ? 1 : (p.d4 <= 64 ? 2 : 4);
 
@@ -1381,7 +1383,7 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     if (dedup_side) KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_seg, 0));
     stage_begin(h, ST_CHAIN, s);
     {
-        const int grid = (row_warps * 32 + 255) / 256 + 1;
+        const int grid = ((p.neg_direct ? p.B : row_warps) * 32 + 255) / 256 + 1;
         if (nch == 1) KGE_CUDA_CHECK(h, launch_dependent(chain_kernel<1>, dim3(grid), dim3(256), 0, s, p));
         else if (nch == 2) KGE_CUDA_CHECK(h, launch_dependent(chain_kernel<2>, dim3(grid), dim3(256), 0, s, p));
         else KGE_CUDA_CHECK(h, launch_dependent(chain_kernel<4>, dim3(grid), dim3(256), 0, s, p));
