@@ -302,7 +302,7 @@ __device__ __forceinline__ void piece_sum(const UpdateJob& J, const UpdateParams
     apply_row<V, NCH>(J, p, J.uniq[u], g, lane);
 }
 
-__global__ void __launch_bounds__(256, 3) piece_kernel(UpdateParams p) {
+__global__ void __launch_bounds__(256, 4) piece_kernel(UpdateParams p) {
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     grid_dependency_wait();
     if (gw >= p.warp_begin[p.njobs]) return;
