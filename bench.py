@@ -90,7 +90,7 @@ STAGE_OPS = {
     "transe1": dict(block=2, accum_q=2, accum_t=2),     # sub, |.|+add  /  compare, predicated add
     "rotate1": dict(block=3.5, accum_q=5, accum_t=5),   # per real coordinate; one sqrt / rsqrt per complex pair
     "distmult1": dict(block=1, accum_q=1, accum_t=1),   # one FMA
-    "transh1": dict(block=4, accum_q=11, accum_t=8),     # w.t dot, residual, |.| / residual again, sign, two or three accumulations
+    "transh1": dict(block=4, accum_q=6, accum_t=5),      # w.t dot, residual, |.| / residual again (2), compare, one or two predicated adds, one FMA
 }
 
 

@@ -240,6 +240,27 @@ __device__ __forceinline__ void pair_update(float& acc, float4 q, float4 t) {
     }
 }
 
+// acc += w where x > 0: one compare and one predicated add (two adds sharing the compare in the
+// second form).  With sign(x) = 2 [x > 0] - 1 a sum of w sign(x) is 2 P - (sum of w), P the sum
+// these accumulate; the value at x == 0 is a free choice of sub-gradient of |x| (here -1).
+__device__ __forceinline__ void add_if_pos(float& acc, float x, float w) {
+    asm("{\n .reg .pred p;\n setp.gt.f32 p, %1, 0f00000000;\n @p add.f32 %0, %0, %2;\n}\n" : "+f"(acc) : "f"(x), "f"(w));
+}
+__device__ __forceinline__ void add2_if_pos(float& acc1, float& acc2, float x, float w1, float w2) {
+    asm("{\n .reg .pred p;\n setp.gt.f32 p, %2, 0f00000000;\n @p add.f32 %0, %0, %3;\n @p add.f32 %1, %1, %4;\n}\n"
+        : "+f"(acc1), "+f"(acc2) : "f"(x), "f"(w1), "f"(w2));
+}
+__device__ __forceinline__ void f4add_if_pos(float4& acc, float4 x, float w) {
+    add_if_pos(acc.x, x.x, w); add_if_pos(acc.y, x.y, w); add_if_pos(acc.z, x.z, w); add_if_pos(acc.w, x.w, w);
+}
+__device__ __forceinline__ void f4add_w_if_pos(float& acc, float4 x, float4 w) {   // acc += sum of w_k over the x_k > 0
+    add_if_pos(acc, x.x, w.x); add_if_pos(acc, x.y, w.y); add_if_pos(acc, x.z, w.z); add_if_pos(acc, x.w, w.w);
+}
+__device__ __forceinline__ void f4add2_if_pos(float4& acc1, float4& acc2, float4 x, float w1, float w2) {
+    add2_if_pos(acc1.x, acc2.x, x.x, w1, w2); add2_if_pos(acc1.y, acc2.y, x.y, w1, w2);
+    add2_if_pos(acc1.z, acc2.z, x.z, w1, w2); add2_if_pos(acc1.w, acc2.w, x.w, w1, w2);
+}
+
 template <int KIND, int MODE>
 __global__ void __launch_bounds__(256) block_kernel(TrainParams p) {
     constexpr bool TH = KIND == KIND_TH_L1 || KIND == KIND_TH_L2;
@@ -254,6 +275,7 @@ __global__ void __launch_bounds__(256) block_kernel(TrainParams p) {
     const float4* Wg = reinterpret_cast<const float4*>(p.w.What);
 
     float acc[4][4], u[4][4];
+    float wsum[4] = {0.f, 0.f, 0.f, 0.f};   // TransH p = 1, second pass: sum of the normal's coordinates per query row
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -296,6 +318,10 @@ __global__ void __launch_bounds__(256) block_kernel(TrainParams p) {
                     tv[i] = *reinterpret_cast<const float4*>(&Ts[(tx + 16 * i) * LDS + kk]);
                     if (TH) wv[i] = *reinterpret_cast<const float4*>(&Ws[(ty + 16 * i) * LDS + kk]);
                 }
+                if (KIND == KIND_TH_L1 && MODE == 1) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) wsum[i] += (wv[i].x + wv[i].y) + (wv[i].z + wv[i].w);
+                }
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -311,7 +337,7 @@ __global__ void __launch_bounds__(256) block_kernel(TrainParams p) {
                                 if (KIND == KIND_TH_L1) acc[i][j] += fabsf(x.x) + fabsf(x.y) + fabsf(x.z) + fabsf(x.w);
                                 else acc[i][j] += f4dot(x, x);
                             } else {
-                                if (KIND == KIND_TH_L1) acc[i][j] += f4dot(f4sgn(x), wv[i]);
+                                if (KIND == KIND_TH_L1) f4add_w_if_pos(acc[i][j], x, wv[i]);
                                 else acc[i][j] += f4dot(x, wv[i]);
                             }
                         }
@@ -328,7 +354,8 @@ __global__ void __launch_bounds__(256) block_kernel(TrainParams p) {
             if (b >= p.B || n >= p.N) continue;
             const int64_t o = (int64_t)b * p.N + n;
             if (MODE == 1) {
-                p.w.Cc[o] = -p.w.F[o] * acc[i][j];   // F holds G (p=1) or G / distance (p=2) by now
+                const float sw = KIND == KIND_TH_L1 ? 2.f * acc[i][j] - wsum[i] : acc[i][j];   // p = 1: acc holds P
+                p.w.Cc[o] = -p.w.F[o] * sw;          // F holds G (p=1) or G / distance (p=2) by now
             } else {
                 float f = acc[i][j];
                 if (KIND == KIND_L1 || KIND == KIND_CL1 || KIND == KIND_TH_L1) f = -f;
@@ -699,7 +726,9 @@ __global__ void __launch_bounds__(256) accum_kernel(AccArgs a) {
     const int c_begin = blockIdx.y * per;
     const int c_end = min(a.oth_rows, c_begin + per);
 
-    float4 A[4][NCH], Wn[TH && OWNER_Q ? 4 : 1][NCH], acc[4][NCH], acc2[TH && OWNER_Q ? 4 : 1][NCH];
+    constexpr bool TH1 = KIND == KIND_TH_L1;   // sign sums as 2 P - (sum of the weights): see add_if_pos
+    float4 A[4][NCH], Wn[TH && OWNER_Q ? 4 : 1][NCH], acc[4][NCH], acc2[TH ? 4 : 1][NCH], acc3[TH1 && OWNER_Q ? 4 : 1][NCH];
+    float sg[4] = {0.f, 0.f, 0.f, 0.f}, sug[4] = {0.f, 0.f, 0.f, 0.f};   // TH1: sums of g and of u g over this split, per owner row
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -708,10 +737,9 @@ __global__ void __launch_bounds__(256) accum_kernel(AccArgs a) {
             const bool in = r < a.own_rows && c < d4;
             A[i][j] = in ? reinterpret_cast<const float4*>(a.own)[(int64_t)r * d4 + c] : f4zero();
             acc[i][j] = f4zero();
-            if (TH && OWNER_Q) {
-                Wn[i][j] = in ? reinterpret_cast<const float4*>(a.what)[(int64_t)r * d4 + c] : f4zero();
-                acc2[i][j] = f4zero();
-            }
+            if (TH && OWNER_Q) Wn[i][j] = in ? reinterpret_cast<const float4*>(a.what)[(int64_t)r * d4 + c] : f4zero();
+            if (TH) acc2[i][j] = f4zero();
+            if (TH1 && OWNER_Q) acc3[i][j] = f4zero();
         }
 
     for (int c0 = c_begin; c0 < c_end; c0 += ACC_CC) {
@@ -742,6 +770,11 @@ __global__ void __launch_bounds__(256) accum_kernel(AccArgs a) {
                 uw[0] = u4.x; uw[1] = u4.y; uw[2] = u4.z; uw[3] = u4.w;
                 cw[0] = c4.x; cw[1] = c4.y; cw[2] = c4.z; cw[3] = c4.w;
             }
+            float ugw[4] = {0.f, 0.f, 0.f, 0.f};
+            if (TH1) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { ugw[i] = uw[i] * gw[i]; sg[i] += gw[i]; sug[i] += ugw[i]; }
+            }
 #pragma unroll
             for (int j = 0; j < NCH; ++j) {
                 const int c = lane + 32 * j;
@@ -754,17 +787,27 @@ __global__ void __launch_bounds__(256) accum_kernel(AccArgs a) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const float4 x = f4fma(uw[i], Wn[i][j], f4sub(A[i][j], bv));
-                        const float4 S = KIND == KIND_TH_L1 ? f4scale(-gw[i], f4sgn(x)) : f4scale(-gw[i], x);
-                        acc[i][j] = f4add(acc[i][j], S);
-                        acc2[i][j] = f4fma(cw[i], bv, f4fma(uw[i], S, acc2[i][j]));
+                        if (TH1) {      // acc = P (weights g), acc3 = P (weights u g), acc2 = sum of c t
+                            f4add2_if_pos(acc[i][j], acc3[i][j], x, gw[i], ugw[i]);
+                            acc2[i][j] = f4fma(cw[i], bv, acc2[i][j]);
+                        } else {
+                            const float4 S = f4scale(-gw[i], x);
+                            acc[i][j] = f4add(acc[i][j], S);
+                            acc2[i][j] = f4fma(cw[i], bv, f4fma(uw[i], S, acc2[i][j]));
+                        }
                     }
                 } else {                // own = t_n (A); other = q_b (bv) with its normal wv
                     const float4 wv = W2s[cc * d4 + c];
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const float4 x = f4fma(uw[i], wv, f4sub(bv, A[i][j]));
-                        const float4 S = KIND == KIND_TH_L1 ? f4scale(-gw[i], f4sgn(x)) : f4scale(-gw[i], x);
-                        acc[i][j] = f4fma(cw[i], wv, f4sub(acc[i][j], S));
+                        if (TH1) {      // acc = P (weights g), acc2 = sum of c w
+                            f4add_if_pos(acc[i][j], x, gw[i]);
+                            acc2[i][j] = f4fma(cw[i], wv, acc2[i][j]);
+                        } else {
+                            const float4 S = f4scale(-gw[i], x);
+                            acc[i][j] = f4fma(cw[i], wv, f4sub(acc[i][j], S));
+                        }
                     }
                 }
             }
@@ -778,6 +821,18 @@ __global__ void __launch_bounds__(256) accum_kernel(AccArgs a) {
             const int r = r0 + warp * 4 + i, c = lane + 32 * j;
             if (r >= a.own_rows || c >= d4) continue;
             const int64_t o = ((int64_t)blockIdx.y * a.own_rows + r) * d4 + c;
+            if (TH1) {
+                const float4 P = acc[i][j], C = acc2[i][j];
+                if (OWNER_Q) {   // -sum g sign(x) = (sum g) - 2 P;  sum (c t - u g sign(x)) = C - 2 P_u + (sum u g)
+                    const float4 Pu = acc3[OWNER_Q ? i : 0][j];
+                    acc[i][j] = make_float4(sg[i] - 2.f * P.x, sg[i] - 2.f * P.y, sg[i] - 2.f * P.z, sg[i] - 2.f * P.w);
+                    acc2[i][j] = make_float4(C.x - 2.f * Pu.x + sug[i], C.y - 2.f * Pu.y + sug[i], C.z - 2.f * Pu.z + sug[i],
+                                             C.w - 2.f * Pu.w + sug[i]);
+                } else {         // sum (c w + g sign(x)) = C + 2 P - (sum g)
+                    acc[i][j] = make_float4(C.x + 2.f * P.x - sg[i], C.y + 2.f * P.y - sg[i], C.z + 2.f * P.z - sg[i],
+                                            C.w + 2.f * P.w - sg[i]);
+                }
+            }
             reinterpret_cast<float4*>(a.out)[o] = acc[i][j];
             if (TH && OWNER_Q) reinterpret_cast<float4*>(a.out2)[o] = acc2[i][j];
         }
