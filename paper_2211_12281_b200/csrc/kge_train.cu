@@ -726,7 +726,9 @@ __global__ void __launch_bounds__(256) accum_kernel(AccArgs a) {
     const int c_begin = blockIdx.y * per;
     const int c_end = min(a.oth_rows, c_begin + per);
 
-    constexpr bool TH1 = KIND == KIND_TH_L1;   // sign sums as 2 P - (sum of the weights): see add_if_pos
+    // sign sums as 2 P - (sum of the weights): see add_if_pos (not for the widest rows of the query side, whose three
+    // accumulators per row would not fit the register file)
+    constexpr bool TH1 = KIND == KIND_TH_L1 && !(OWNER_Q && NCH == 4);
     float4 A[4][NCH], Wn[TH && OWNER_Q ? 4 : 1][NCH], acc[4][NCH], acc2[TH ? 4 : 1][NCH], acc3[TH1 && OWNER_Q ? 4 : 1][NCH];
     float sg[4] = {0.f, 0.f, 0.f, 0.f}, sug[4] = {0.f, 0.f, 0.f, 0.f};   // TH1: sums of g and of u g over this split, per owner row
 #pragma unroll
@@ -791,7 +793,7 @@ __global__ void __launch_bounds__(256) accum_kernel(AccArgs a) {
                             f4add2_if_pos(acc[i][j], acc3[i][j], x, gw[i], ugw[i]);
                             acc2[i][j] = f4fma(cw[i], bv, acc2[i][j]);
                         } else {
-                            const float4 S = f4scale(-gw[i], x);
+                            const float4 S = KIND == KIND_TH_L1 ? f4scale(-gw[i], f4sgn(x)) : f4scale(-gw[i], x);
                             acc[i][j] = f4add(acc[i][j], S);
                             acc2[i][j] = f4fma(cw[i], bv, f4fma(uw[i], S, acc2[i][j]));
                         }
@@ -805,7 +807,7 @@ __global__ void __launch_bounds__(256) accum_kernel(AccArgs a) {
                             f4add_if_pos(acc[i][j], x, gw[i]);
                             acc2[i][j] = f4fma(cw[i], wv, acc2[i][j]);
                         } else {
-                            const float4 S = f4scale(-gw[i], x);
+                            const float4 S = KIND == KIND_TH_L1 ? f4scale(-gw[i], f4sgn(x)) : f4scale(-gw[i], x);
                             acc[i][j] = f4fma(cw[i], wv, f4sub(acc[i][j], S));
                         }
                     }

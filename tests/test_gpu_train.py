@@ -145,6 +145,16 @@ def test_wide_rows_and_many_splits(oracle64):
     _run(oracle64, prob, steps=1)
 
 
+@pytest.mark.parametrize("d", [128, 256, 384])
+def test_transh_l1_row_widths(oracle64, d):
+    """TransH p = 1 at one, two and four 128-float slices per lane: the backward takes its sign
+    sums as predicated adds for the first two and element by element on the query side of the
+    widest rows."""
+    prob = Problem(E=800, R=6, T=20000, d=d, score="transh", p_norm=1, loss="logsigmoid", B=96, N=80, P=2,
+                   gamma=6.0, adv_temp=0.5, lr=0.05, graph_seed=12, relation_zipf=1.0)
+    _run(oracle64, prob, steps=1)
+
+
 @pytest.mark.parametrize("score,p", [("distmult", 1), ("complex", 1), ("transe", 2)])
 @pytest.mark.parametrize("d", [64, 192, 256])
 def test_tensor_core_score_block(oracle64, score, p, d):
