@@ -32,7 +32,7 @@ import kge_synth
 METRIC = "positive triples/sec (fwd+bwd+update, N shared negs)"
 UNIT = "triples/s"
 
-# BASELINE configs[1]: 100,000 entities, 500 relations (Zipf 1.0), 2,000,000 triples with
+# The headline configuration: 100,000 entities, 500 relations (Zipf 1.0), 2,000,000 triples with
 # Zipf(1.1) degrees, d = 128 fp32, log-sigmoid loss with margin 12 (self-adversarial
 # temperature 1), B = N = 1,024, P = 4, SGD lr 0.05.
 WORKLOADS = {
@@ -42,7 +42,7 @@ WORKLOADS = {
     "c2_rotate_l1": dict(E=100_000, R=500, T=2_000_000, d=128, score="rotate", p_norm=1, loss="logsigmoid",
                          opt="sgd", B=1024, N=1024, P=4, gamma=12.0, adv_temp=1.0, lr=0.05,
                          entity_zipf=1.1, relation_zipf=1.0, graph_seed=1),
-    # BASELINE configs[2]: 10,000,000 entities, 1,000 relations (Zipf 1.0), 100,000,000 Zipf(1.1) triples,
+    # The 10 M-entity configuration: 10,000,000 entities, 1,000 relations (Zipf 1.0), 100,000,000 Zipf(1.1) triples,
     # d = 256, sampled-softmax loss with the paper's correction, B = 4,096 x N = 16,384, P = 8, Adam on
     # touched rows, bf16 tensor-core score block.  Tables are drawn on the device (10 GB + 20 GB of state).
     "c3_distmult": dict(E=10_000_000, R=1000, T=100_000_000, d=256, score="distmult", p_norm=1, loss="softmax",
@@ -51,11 +51,11 @@ WORKLOADS = {
     "c3_complex": dict(E=10_000_000, R=1000, T=100_000_000, d=256, score="complex", p_norm=1, loss="softmax",
                        opt="adam", B=4096, N=16384, P=8, gamma=0.0, adv_temp=0.0, lr=0.001, tc=True,
                        ce_correction="paper", entity_zipf=1.1, relation_zipf=1.0, graph_seed=2, device_tables=True),
-    # a tenth of configs[2]'s graph and table with the same batch shape: quick runs of the tensor-core step
+    # a tenth of the 10 M-entity configuration's graph and table with the same batch shape: quick runs of the tensor-core step
     "c3s_distmult": dict(E=1_000_000, R=1000, T=10_000_000, d=256, score="distmult", p_norm=1, loss="softmax",
                          opt="adam", B=4096, N=16384, P=8, gamma=0.0, adv_temp=0.0, lr=0.001, tc=True,
                          ce_correction="paper", entity_zipf=1.1, relation_zipf=1.0, graph_seed=2, device_tables=True),
-    # BASELINE configs[3]: 91,000,000 entities (46.6 GB table), 1,400 relations, d = 128, B = N = 8,192, P = 16, row-wise
+    # The 91 M-entity training configuration: 91,000,000 entities (46.6 GB table), 1,400 relations, d = 128, B = N = 8,192, P = 16, row-wise
     # Adagrad, log-sigmoid loss with margin 12.  The graph is cut to 60 M of the 600 M triples (host-side preprocessing;
     # the step does not depend on the graph's size).  TransE-L2 on tensor cores, TransH on CUDA cores.
     "c4_transe_l2": dict(E=91_000_000, R=1400, T=60_000_000, d=128, score="transe", p_norm=2, loss="logsigmoid",
@@ -69,7 +69,7 @@ WORKLOADS = {
                         entity_zipf=1.1, relation_zipf=0.0, graph_seed=0),
 }
 
-# BASELINE configs[4]: 15,000 (h, r) queries against all 91,000,000 entities of d = 128, top-10 and the
+# The full-entity scoring configuration: 15,000 (h, r) queries against all 91,000,000 entities of d = 128, top-10 and the
 # rank of a designated true tail.  The "s" variants keep the query batch and shrink the table.
 INFER_WORKLOADS = {
     "c5_transe_l1": dict(E=91_000_000, R=1400, d=128, Q=15000, K=10, score="transe", p_norm=1),

@@ -1,6 +1,6 @@
-"""Parity at the benchmark's full table sizes, on what the oracle can afford: the rows one step
+"""Parity at the full table sizes of the large configurations, on what the oracle can afford: the rows one step
 touches.  The GPU runs the step on the whole table (10 M x 256 fp32 plus Adam state for
-configs[2]); the rows of the batch are pulled out before and after, the ids are renumbered
+the 10 M-entity configuration); the rows of the batch are pulled out before and after, the ids are renumbered
 densely, and the fp64 oracle runs the same step on that compact problem -- every quantity of
 the step depends on the tables only through the rows the batch names, and the sampled-softmax
 correction c is passed as a number, so the compact problem has the same answer."""
@@ -26,7 +26,7 @@ def test_config3_full_table_step_on_touched_rows(oracle64, score):
     free, _ = torch.cuda.mem_get_info()
     if free < 45e9:
         pytest.skip("needs 45 GB of free device memory")
-    # configs[2] with a graph of 20 M triples instead of 100 M (the step never sees the graph's size)
+    # the 10 M-entity configuration with a graph of 20 M triples instead of 100 M (the step never sees the graph's size)
     E, R, T, d, B, N, P = 10_000_000, 1000, 20_000_000, 256, 4096, 16384, 8
     lr, c = 1e-3, float(np.log((E - 1) / N))
     kw = dict(num_entities=E, num_relations=R, dim=d, score=score, loss="softmax", opt="adam", batch=B, num_neg=N,
@@ -89,7 +89,7 @@ def test_config3_full_table_step_on_touched_rows(oracle64, score):
 
 @pytest.mark.parametrize("score,p_norm,tc", [("transe", 2, True), ("transh", 1, False)])
 def test_config4_full_table_step_on_touched_rows(oracle64, score, p_norm, tc):
-    """configs[3]: 91,000,000 entities of d = 128 (a 46.6 GB table), B = N = 8,192, P = 16, row-wise
+    """the 91 M-entity training configuration: 91,000,000 entities of d = 128 (a 46.6 GB table), B = N = 8,192, P = 16, row-wise
     Adagrad, log-sigmoid loss with margin 12; TransE-L2 on tensor cores (norm expansion), TransH on
     CUDA cores.  The graph is cut to 20 M triples (the step never sees its size)."""
     import torch
@@ -161,7 +161,7 @@ def test_config4_full_table_step_on_touched_rows(oracle64, score, p_norm, tc):
 
 @pytest.mark.parametrize("score,tc", [("transe", False), ("distmult", True)])
 def test_config5_full_table_topk_properties(oracle32, oracle64, score, tc):
-    """configs[4]: queries against all 91,000,000 entities (46.6 GB table), top-10 and rank.  The
+    """the full-entity scoring configuration: queries against all 91,000,000 entities (46.6 GB table), top-10 and rank.  The
     oracle cannot hold the table, so the lists are checked by what fixes them: every reported
     score is the oracle's score of that (query, entity) pair; the list is ordered by (score
     descending, id ascending) with distinct ids; no entity of a 400,000-row sample is ordered

@@ -82,7 +82,7 @@ def test_tensor_core_topk_against_bf16_operand_oracle(oracle64, score):
 
 
 def test_config1_mrr_after_training(oracle32, oracle64):
-    """BASELINE configs[0]: 10 SGD steps, then MRR of the first 100 triples ranked against
+    """The small configuration: 10 SGD steps, then MRR of the first 100 triples ranked against
     all 1,000 entities.  Inference parity is taken on the GPU's own trained tables."""
     prob = Problem(E=1000, R=10, T=20000, d=32, score="distmult", loss="logsigmoid", B=64, N=128, P=2,
                    lr=0.1, seed=0, graph_seed=0)

@@ -7,7 +7,7 @@ from parity_util import GpuSide, OracleSide, Problem
 pytestmark = pytest.mark.gpu
 
 CASES = {
-    # BASELINE configs[0] and configs[1] shapes
+    # the small configuration and the headline configuration (shapes)
     "c1": dict(E=1000, R=10, T=20000, d=32, score="distmult", B=64, N=128, P=2, seed=0),
     "c2": dict(E=100000, R=500, T=2000000, d=128, score="transe", B=1024, N=1024, P=4, seed=0,
                graph_seed=1, relation_zipf=1.0),

@@ -204,7 +204,7 @@ def test_repeated_rows_one_entity_everywhere(oracle64):
 
 
 def test_config1_ten_sgd_steps_free_running(oracle64):
-    """BASELINE configs[0]: 10 SGD steps of DistMult with internal sampling, both sides
+    """The small configuration: 10 SGD steps of DistMult with internal sampling, both sides
     running freely from the same initial tables."""
     prob = Problem(E=1000, R=10, T=20000, d=32, score="distmult", loss="logsigmoid", B=64, N=128, P=2,
                    lr=0.1, seed=0, graph_seed=0)
@@ -228,7 +228,7 @@ def test_config1_ten_sgd_steps_free_running(oracle64):
 
 @pytest.mark.parametrize("score,p", [("transe", 1), ("rotate", 1)])
 def test_config2_full_size_step(oracle64, score, p):
-    """BASELINE configs[1] at full size, in the launch configuration the benchmark times:
+    """The headline configuration at full size, in the launch configuration the benchmark times:
     100,000 entities, d = 128, B = N = 1,024, P = 4, log-sigmoid with margin 12, SGD 0.05."""
     prob = Problem(E=100000, R=500, T=2000000, d=128, score=score, p_norm=p, loss="logsigmoid",
                    B=1024, N=1024, P=4, gamma=12.0, adv_temp=1.0, lr=0.05, seed=0, graph_seed=1,
