@@ -519,6 +519,27 @@ struct WarpReduce {    // one warp works on one row
     __device__ __forceinline__ float max(float v) const { return warp_max(v); }
 };
 
+template <int WPR>     // WPR neighbouring warps work on one row; every warp of the CTA calls each reduction
+struct GroupReduce {
+    float* sm;         // [2][warps of the CTA], the halves used in turn so that one barrier per reduction is enough
+    int warp, lane;
+    mutable int turn;
+    template <class Op>
+    __device__ __forceinline__ float across(float v, Op op) const {
+        float* slot = sm + (turn & 1) * (LOSS_THREADS / 32);
+        ++turn;
+        if (lane == 0) slot[warp] = v;
+        __syncthreads();
+        const int first = warp / WPR * WPR;
+        float t = slot[first];
+#pragma unroll
+        for (int i = 1; i < WPR; ++i) t = op(t, slot[first + i]);
+        return t;
+    }
+    __device__ __forceinline__ float sum(float v) const { return across(warp_sum(v), [](float a, float c) { return a + c; }); }
+    __device__ __forceinline__ float max(float v) const { return across(warp_max(v), [](float a, float c) { return fmaxf(a, c); }); }
+};
+
 // How a thread reaches its share of a row of scores: element i of count(), read with get(i),
 // dL/dF written back with put(i, g).
 struct StridedRow {    // scores in shared or global memory, covered as t0, t0 + stride, ...
@@ -651,22 +672,29 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_warp_kernel(TrainParams p) 
     loss_row(p, b, sr, lane == 0, WarpReduce{});
 }
 
-// One warp per positive with the whole row in registers (N = 128 * V4): every pass over the row
-// is unrolled, so the exponentials of a lane's 4 * V4 scores are independent instructions.
-template <int V4>
+// WPR warps per positive with the whole row in registers (N = 128 * V4 * WPR): every pass over the
+// row is unrolled, so the exponentials of a lane's 4 * V4 scores are independent instructions.
+// With WPR > 1 the warps of a row exchange their partial maxima and sums through shared memory.
+template <int V4, int WPR>
 __global__ void __launch_bounds__(LOSS_THREADS) loss_reg_kernel(TrainParams p) {
+    __shared__ float red_sm[2 * (LOSS_THREADS / 32)];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = blockIdx.x * (LOSS_THREADS / 32) + warp;
+    const int row = blockIdx.x * (LOSS_THREADS / 32 / WPR) + warp / WPR, part = warp % WPR;
     grid_dependency_wait();
     allow_dependents();
-    if (b >= p.B) return;
+    if (WPR == 1 && row >= p.B) return;
+    const bool valid = row < p.B;
+    const int b = valid ? row : p.B - 1;          // a CTA's spare warps shadow the last row: they take part in the barriers
     float4* Frow = reinterpret_cast<float4*>(p.w.F + (int64_t)b * p.N);
     RegisterRow<V4> rr;
 #pragma unroll
-    for (int j = 0; j < V4; ++j) rr.f[j] = Frow[j * 32 + lane];
-    loss_row(p, b, rr, lane == 0, WarpReduce{});
+    for (int j = 0; j < V4; ++j) rr.f[j] = Frow[(j * WPR + part) * 32 + lane];
+    if (WPR == 1) loss_row(p, b, rr, lane == 0, WarpReduce{});
+    else loss_row(p, b, rr, valid && part == 0 && lane == 0, GroupReduce<WPR>{red_sm, warp, lane, 0});
+    if (valid) {
 #pragma unroll
-    for (int j = 0; j < V4; ++j) Frow[j * 32 + lane] = rr.g[j];
+        for (int j = 0; j < V4; ++j) Frow[(j * WPR + part) * 32 + lane] = rr.g[j];
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1379,11 +1407,12 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
             configured = true;
         }
     }
-    constexpr int loss_rows = LOSS_THREADS / 32;
-    const int loss_grid = (p.B + loss_rows - 1) / loss_rows;
-    if (p.N == 256) KGE_CUDA_CHECK(h, launch_dependent(loss_reg_kernel<2>, dim3(loss_grid), dim3(LOSS_THREADS), 0, s, p));
-    else if (p.N == 512) KGE_CUDA_CHECK(h, launch_dependent(loss_reg_kernel<4>, dim3(loss_grid), dim3(LOSS_THREADS), 0, s, p));
-    else if (p.N == 1024) KGE_CUDA_CHECK(h, launch_dependent(loss_reg_kernel<8>, dim3(loss_grid), dim3(LOSS_THREADS), 0, s, p));
+    // rows of 256 / 512 / 1024 scores in registers, 2 / 4 / 4 warps per row (one warp per row leaves most of the SM idle:
+    // 80 -> 75.5 us per step at B = N = 1024)
+    constexpr int warps = LOSS_THREADS / 32;
+    if (p.N == 256) KGE_CUDA_CHECK(h, (launch_dependent(loss_reg_kernel<1, 2>, dim3((p.B + warps / 2 - 1) / (warps / 2)), dim3(LOSS_THREADS), 0, s, p)));
+    else if (p.N == 512) KGE_CUDA_CHECK(h, (launch_dependent(loss_reg_kernel<1, 4>, dim3((p.B + warps / 4 - 1) / (warps / 4)), dim3(LOSS_THREADS), 0, s, p)));
+    else if (p.N == 1024) KGE_CUDA_CHECK(h, (launch_dependent(loss_reg_kernel<2, 4>, dim3((p.B + warps / 4 - 1) / (warps / 4)), dim3(LOSS_THREADS), 0, s, p)));
     else if (p.N <= LOSS_WARP_MAX_N && (p.N & 3) == 0) {
         constexpr int rows = LOSS_THREADS / 32;
         KGE_CUDA_CHECK(h, launch_dependent(loss_warp_kernel, dim3((p.B + rows - 1) / rows), dim3(LOSS_THREADS), (size_t)rows * p.N * 4, s, p));

@@ -145,6 +145,16 @@ def test_wide_rows_and_many_splits(oracle64):
     _run(oracle64, prob, steps=1)
 
 
+@pytest.mark.parametrize("N,loss", [(256, "logsigmoid"), (512, "softmax"), (1024, "softmax"), (512, "logsigmoid")])
+def test_loss_rows_in_registers(oracle64, N, loss):
+    """Rows of 256 / 512 / 1024 scores are held in registers by 2 / 4 / 4 warps that exchange their
+    partial maxima and sums through shared memory; B = 37 leaves a CTA with spare warps."""
+    prob = Problem(E=3000, R=5, T=20000, d=32, score="transe", p_norm=1, loss=loss, B=37, N=N, P=1,
+                   gamma=6.0, adv_temp=1.0 if loss == "logsigmoid" else 0.0, ce_correction=0.2, lr=0.05, graph_seed=13,
+                   relation_zipf=1.0)
+    _run(oracle64, prob, steps=1)
+
+
 @pytest.mark.parametrize("d", [128, 256, 384])
 def test_transh_l1_row_widths(oracle64, d):
     """TransH p = 1 at one, two and four 128-float slices per lane: the backward takes its sign
