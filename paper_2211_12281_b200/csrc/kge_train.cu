@@ -1051,6 +1051,31 @@ __global__ void __launch_bounds__(32 * ACC_WARPS) accum_tma_kernel(AccArgs aq, A
 // the gradient rows of the head, the positive tail and the relation.  Warps [B, B+N): add
 // the row splits of dT and write the gradient row of the negative tail.
 // ------------------------------------------------------------------------------------------
+// Sum of n split partials first[0], first[stride], ... in ascending order.  Eight loads are issued
+// before the first addition: a loop of load-then-add would pay one trip to L2 per split.
+__device__ __forceinline__ float4 sum_splits(const float4* first, int64_t stride, int n) {
+    float4 s = f4zero();
+    for (int s0 = 0; s0 < n; s0 += 8) {
+        float4 v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = s0 + i < n ? first[(int64_t)(s0 + i) * stride] : f4zero();
+#pragma unroll
+        for (int i = 0; i < 8; ++i) s = f4add(s, v[i]);
+    }
+    return s;
+}
+__device__ __forceinline__ float sum_splits(const float* first, int64_t stride, int n) {
+    float s = 0.f;
+    for (int s0 = 0; s0 < n; s0 += 8) {
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = s0 + i < n ? first[(int64_t)(s0 + i) * stride] : 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) s += v[i];
+    }
+    return s;
+}
+
 template <int kMaxChunks>
 __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
     const int lane = threadIdx.x & 31;
@@ -1080,11 +1105,9 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
         const int n = warp - p.B;
         const float4* part = reinterpret_cast<const float4*>(p.w.dTpart);
         float wsum = 0.f;   // TransE p = 1: the splits hold P, the gradient is 2 P - (column sum of dL/dF)
-        if (p.kind == KIND_L1)
-            for (int sp = 0; sp < p.split_t; ++sp) wsum += p.w.Cpart[(int64_t)sp * p.N + n];
+        if (p.kind == KIND_L1) wsum = sum_splits(p.w.Cpart + n, p.N, p.split_t);
         for (int c = lane; c < d4; c += 32) {
-            float4 s = f4zero();
-            for (int sp = 0; sp < p.split_t; ++sp) s = f4add(s, part[((int64_t)sp * p.N + n) * d4 + c]);
+            float4 s = sum_splits(part + (int64_t)n * d4 + c, (int64_t)p.N * d4, p.split_t);
             if (p.kind == KIND_L1) s = make_float4(2.f * s.x - wsum, 2.f * s.y - wsum, 2.f * s.z - wsum, 2.f * s.w - wsum);
             if (p.tc_l2) {   // dT_n = sum_b C_bn (q_b - t_n) = (C^T Q)_n - (column sum of C) t_n
                 const float cs = p.w.Gcol[n];
@@ -1111,9 +1134,7 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
         const bool in = c < d4;
         h[i] = in ? hrow[c] : f4zero(); t[i] = in ? trow[c] : f4zero(); q[i] = in ? qrow[c] : f4zero();
         float4 s = f4zero();
-        if (in)
-            for (int sp = 0; sp < p.split_q; ++sp)
-                s = f4add(s, reinterpret_cast<const float4*>(p.w.dQpart)[((int64_t)sp * p.B + b) * d4 + c]);
+        if (in) s = sum_splits(reinterpret_cast<const float4*>(p.w.dQpart) + (int64_t)b * d4 + c, (int64_t)p.B * d4, p.split_q);
         if (p.kind == KIND_L1 && in) {   // the splits hold P; dQ = (row sum of dL/dF) - 2 P
             const float rs = p.w.Grow[b];
             s = make_float4(rs - 2.f * s.x, rs - 2.f * s.y, rs - 2.f * s.z, rs - 2.f * s.w);
@@ -1140,9 +1161,7 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
             const float4 wraw = in ? wrow[c] : f4zero();
             nrm2 += f4dot(wraw, wraw);
             float4 s = f4zero();
-            if (in)
-                for (int sp = 0; sp < p.split_q; ++sp)
-                    s = f4add(s, reinterpret_cast<const float4*>(p.w.dWpart)[((int64_t)sp * p.B + b) * d4 + c]);
+            if (in) s = sum_splits(reinterpret_cast<const float4*>(p.w.dWpart) + (int64_t)b * d4 + c, (int64_t)p.B * d4, p.split_q);
             dwh[i] = s;
             u += f4dot(wh[i], t[i]); a += f4dot(wh[i], h[i]);
         }
