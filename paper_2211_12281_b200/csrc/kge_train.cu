@@ -221,6 +221,7 @@ __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
 constexpr int TB = 64, TN = 64, KC = 32, LDS = KC + 4;
 
 __device__ __forceinline__ float approx_sqrt(float x) { float r; asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+__device__ __forceinline__ float approx_rsqrt(float x) { float r; asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
 
 template <int KIND>
 __device__ __forceinline__ void pair_update(float& acc, float4 q, float4 t) {
@@ -728,11 +729,13 @@ __device__ __forceinline__ void acc_update(float4& acc, float4 a, float4 b, floa
     } else if (KIND == KIND_L2) {  // w already holds G / distance
         acc = f4fma(w, f4sub(b, a), acc);
     } else {                       // KIND_CL1: acc -= w * (a - b) / |a - b| per complex component
+        // one special-function reciprocal square root per complex component (relative error 2^-22, as in the forward)
         float xr = a.x - b.x, xi = a.y - b.y, m2 = fmaf(xr, xr, xi * xi);
-        float s = m2 > 0.f ? w * rsqrtf(m2) : 0.f;
+        // (a zero modulus has xr = xi = 0, so the finite factor from the floor contributes nothing)
+        float s = w * approx_rsqrt(fmaxf(m2, 1e-37f));
         acc.x = fmaf(-s, xr, acc.x); acc.y = fmaf(-s, xi, acc.y);
         xr = a.z - b.z; xi = a.w - b.w; m2 = fmaf(xr, xr, xi * xi);
-        s = m2 > 0.f ? w * rsqrtf(m2) : 0.f;
+        s = w * approx_rsqrt(fmaxf(m2, 1e-37f));
         acc.z = fmaf(-s, xr, acc.z); acc.w = fmaf(-s, xi, acc.w);
     }
 }
