@@ -161,7 +161,8 @@ int kge_train_step_host(kge_handle* h, uint64_t step, float lr,
  * (score descending, entity id ascending) -- unused places (k > |E|) hold id -1 and -inf.
  * If true_tails is given, out_ranks[q] (int32) = 1 + number of entities ordered before the
  * true tail under the same order; neither the head nor the true tail is filtered.  nq must
- * not exceed the max_queries the workspace was sized for, k not its topk.
+ * not exceed the max_queries the workspace was sized for, k not its topk.  nq = 0 is a no-op that
+ * returns KGE_OK (the array arguments may then be NULL).
  * Synchronises `stream` (candidate-list occupancy is checked between entity chunks).
  */
 int kge_score_all_topk(kge_handle* h, const int32_t* q_heads, const int32_t* q_rels, int32_t nq, int32_t k,

@@ -395,7 +395,8 @@ int kge_train_step_host(kge_handle* h, uint64_t step, float lr, const int32_t* h
 int kge_score_all_topk(kge_handle* h, const int32_t* q_heads, const int32_t* q_rels, int32_t nq, int32_t k,
                        const int32_t* true_tails, int32_t* out_ids, float* out_scores, int32_t* out_ranks,
                        void* stream) {
-    if (!h || !q_heads || !q_rels || !out_ids || !out_scores || nq < 0 || k <= 0) return KGE_ERR_BAD_ARG;
+    if (!h || nq < 0 || k <= 0) return KGE_ERR_BAD_ARG;
+    if (nq > 0 && (!q_heads || !q_rels || !out_ids || !out_scores)) return KGE_ERR_BAD_ARG;   // an empty batch may pass NULL
     if (out_ranks && !true_tails) return KGE_ERR_BAD_ARG;
     if (!h->bound) return KGE_ERR_NOT_READY;
     if (nq > h->max_queries || k > h->topk) return KGE_ERR_WORKSPACE;

@@ -106,6 +106,20 @@ def test_k_larger_than_entities_and_single_query(oracle32):
     assert (ids[0, 9:] == -1).all() and np.isneginf(sc[0, 9:]).all()
 
 
+def test_empty_query_batch_is_a_no_op(oracle32):
+    """nq = 0: the call returns success, launches nothing and leaves the outputs alone."""
+    prob = Problem(E=9, R=2, T=50, d=16, score="transe", p_norm=1, B=4, N=4, P=1, graph_seed=12)
+    gpu = GpuSide(prob, max_queries=4, topk=3, load_graph=False)
+    t = gpu.torch
+    dev = gpu.ent.device
+    ids = t.full((1, 3), 77, dtype=t.int32, device=dev); sc = t.full((1, 3), 5.0, dtype=t.float32, device=dev)
+    empty = t.empty(0, dtype=t.int32, device=dev)
+    before = gpu.kge.launch_count()
+    gpu.kge.score_all_topk(empty, empty, 3, None, ids, sc, None)
+    assert gpu.kge.get_status() == 0 and gpu.kge.launch_count() == before
+    assert (ids.cpu().numpy() == 77).all() and (sc.cpu().numpy() == 5.0).all()
+
+
 def test_rising_scores_take_the_overflow_path(oracle32):
     """Scores that grow with the entity id make every entity of a chunk beat the current
     k-th best, which fills the candidate list; the library must redo the chunk in pieces."""

@@ -202,6 +202,14 @@ def test_tensor_core_path_refuses_what_it_cannot_do():
         assert e.value.code == -5
 
 
+@pytest.mark.parametrize("score,p", [("transe", 1), ("distmult", 1), ("transh", 1)])
+def test_smallest_problem(oracle64, score, p):
+    """One positive, one negative, one partition, four coordinates: every tile, chunk and piece is ragged."""
+    prob = Problem(E=5, R=1, T=6, d=4, score=score, p_norm=p, loss="logsigmoid", B=1, N=1, P=1,
+                   gamma=1.0 if score != "distmult" else 0.0, adv_temp=1.0, lr=0.1, graph_seed=14)
+    _run(oracle64, prob, steps=2)
+
+
 def test_repeated_rows_one_entity_everywhere(oracle64):
     """One entity is head, tail and negative several times; one relation for the whole batch."""
     prob = Problem(E=64, R=2, T=2000, d=32, score="distmult", loss="logsigmoid", B=16, N=16, P=1, lr=0.1)
