@@ -145,13 +145,50 @@ __global__ void query_setup_kernel(InferParams p) {
     p.w.cand_cnt[q] = 0; p.w.beat_tmp[q] = 0; p.w.beat[q] = 0;
 }
 
+constexpr int IQ = 64, IE = 64, IKC = 32, ILD = IKC + 4;
+
+// Epilogue of a 64 x 64 score tile: rank counting against the true tail, threshold filter into the
+// candidate lists.  Thread (tx, ty) holds the pairs (q0 + ty + 16 i, e0 + tx + 16 j).
+template <int KIND>
+__device__ __forceinline__ void score_tile_epilogue(const InferParams& p, const float (&acc)[4][4], int q0, int64_t e0, int tx, int ty) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int q = q0 + ty + 16 * i;
+        const bool qin = q < p.nq;
+        float thr = 0.f, ft = 0.f; int32_t thr_id = 0, tt = 0;
+        if (qin) {
+            thr = p.w.thr[q]; thr_id = p.w.thr_id[q];
+            if (p.tt) { ft = p.w.iftrue[q]; tt = p.tt[q]; }
+        }
+        int beat = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t e = e0 + tx + 16 * j;
+            if (!qin || e >= p.e_hi) continue;
+            const float f = canon_finish(KIND, acc[i][j]);
+            if (p.tt && ordered_before(f, (int32_t)e, ft, tt)) ++beat;
+            if (ordered_before(f, (int32_t)e, thr, thr_id)) {
+                const int slot = atomicAdd(&p.w.cand_cnt[q], 1);
+                if (slot < kCandCap) {
+                    p.w.cand_score[(int64_t)q * kCandCap + slot] = f;
+                    p.w.cand_id[(int64_t)q * kCandCap + slot] = (int32_t)e;
+                } else {
+                    p.w.status[1] = 1;   // this chunk overflowed a list: the host redoes it in small pieces
+                }
+            }
+        }
+        // the 16 lanes sharing a query row are contiguous: one atomic per row and tile
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) beat += __shfl_xor_sync(0xffffffffu, beat, o);
+        if (tx == 0 && beat > 0) atomicAdd(&p.w.beat_tmp[q], beat);
+    }
+}
+
 // ------------------------------------------------------------------------------------------
 // score tile: 64 queries x 64 entities per CTA, 4 x 4 pairs per thread.  Consecutive CTAs
 // walk the query tiles of one entity tile, so an entity tile is fetched from HBM once and
 // served to the other query tiles by L2.
 // ------------------------------------------------------------------------------------------
-constexpr int IQ = 64, IE = 64, IKC = 32, ILD = IKC + 4;
-
 template <int KIND>
 __global__ void __launch_bounds__(256) score_tile_kernel(InferParams p) {
     constexpr bool TH = KIND == KIND_TH_L1 || KIND == KIND_TH_L2;
@@ -219,38 +256,113 @@ __global__ void __launch_bounds__(256) score_tile_kernel(InferParams p) {
             __syncthreads();
         }
     }
-    // epilogue: rank counting against the true tail, threshold filter into the candidate lists
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int q = q0 + ty + 16 * i;
-        const bool qin = q < p.nq;
-        float thr = 0.f, ft = 0.f; int32_t thr_id = 0, tt = 0;
-        if (qin) {
-            thr = p.w.thr[q]; thr_id = p.w.thr_id[q];
-            if (p.tt) { ft = p.w.iftrue[q]; tt = p.tt[q]; }
-        }
-        int beat = 0;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int64_t e = e0 + tx + 16 * j;
-            if (!qin || e >= p.e_hi) continue;
-            const float f = canon_finish(KIND, acc[i][j]);
-            if (p.tt && ordered_before(f, (int32_t)e, ft, tt)) ++beat;
-            if (ordered_before(f, (int32_t)e, thr, thr_id)) {
-                const int slot = atomicAdd(&p.w.cand_cnt[q], 1);
-                if (slot < kCandCap) {
-                    p.w.cand_score[(int64_t)q * kCandCap + slot] = f;
-                    p.w.cand_id[(int64_t)q * kCandCap + slot] = (int32_t)e;
-                } else {
-                    p.w.status[1] = 1;   // this chunk overflowed a list: the host redoes it in small pieces
-                }
-            }
-        }
-        // the 16 lanes sharing a query row are contiguous: one atomic per row and tile
-#pragma unroll
-        for (int o = 8; o > 0; o >>= 1) beat += __shfl_xor_sync(0xffffffffu, beat, o);
-        if (tx == 0 && beat > 0) atomicAdd(&p.w.beat_tmp[q], beat);
+    score_tile_epilogue<KIND>(p, acc, q0, e0, tx, ty);
+}
+
+// ------------------------------------------------------------------------------------------
+// score tile, kinds that are a function of (q, t) alone: the same 64 x 64 tile and the same
+// operation order (one accumulator per pair, coordinates ascending), but the 64 query rows and
+// 64 entity rows arrive by one asynchronous bulk copy per row into padded shared-memory rows (up
+// to 128 coordinates per stage, two stages for longer rows), so a CTA waits once per stage instead
+// of loading and synchronising every 32 coordinates.
+// ------------------------------------------------------------------------------------------
+constexpr int IKT = 128;
+__host__ __device__ inline int infer_tma_kc(int d) { return d < IKT ? d : IKT; }
+__host__ __device__ inline int infer_tma_stages(int d) { return d > IKT ? 2 : 1; }
+inline size_t infer_tma_smem(int d) {
+    return (size_t)infer_tma_stages(d) * (IQ + IE) * (infer_tma_kc(d) + 4) * sizeof(float) + 2 * sizeof(uint64_t);
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(256) score_tile_tma_kernel(InferParams p) {
+    extern __shared__ __align__(128) unsigned char smraw[];
+    constexpr int ROWS = IQ + IE;        // rows [0, IQ) of a stage hold queries, the rest entities
+    const int kc = infer_tma_kc(p.d), ld = kc + 4, nstage = infer_tma_stages(p.d);
+    const int nchunk = (p.d + kc - 1) / kc;
+    float* base = reinterpret_cast<float*>(smraw);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smraw + (size_t)nstage * ROWS * ld * sizeof(float));
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int qt = blockIdx.x % p.q_tiles;
+    const int64_t et = blockIdx.x / p.q_tiles;
+    const int q0 = qt * IQ;
+    const int64_t e0 = p.e_lo + et * IE;
+
+    if (tid == 0) {
+        for (int st = 0; st < nstage; ++st) mbar_init(&bars[st], ROWS);
+        mbar_init_fence();
     }
+    __syncthreads();
+
+    auto issue = [&](int chunk, int stage) {     // thread r < ROWS owns row r of the stage
+        if (tid >= ROWS) return;
+        const bool isq = tid < IQ;
+        const int64_t g = isq ? q0 + tid : e0 + (tid - IQ);
+        const bool in = isq ? g < p.nq : g < p.e_hi;
+        float* dst = base + ((size_t)stage * ROWS + tid) * ld;
+        const int k0 = chunk * kc, len = min(kc, p.d - k0);
+        if (in) {
+            const float* src = (isq ? p.w.iq : p.ent) + g * p.d + k0;
+            mbar_arrive_expect_tx(&bars[stage], (uint32_t)len * 4u);
+            bulk_g2s(dst, src, (uint32_t)len * 4u, &bars[stage]);
+        } else {
+            if (chunk < nstage)   // rows outside the problem stay zero for the whole kernel
+                for (int k = 0; k < kc; k += 4) *reinterpret_cast<float4*>(dst + k) = make_float4(0.f, 0.f, 0.f, 0.f);
+            mbar_arrive(&bars[stage]);
+        }
+    };
+    issue(0, 0);
+    if (nstage > 1 && nchunk > 1) issue(1, 1);
+
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int chunk = 0; chunk < nchunk; ++chunk) {
+        const int stage = chunk % nstage;
+        const bool ok = mbar_wait_bounded(&bars[stage], (uint32_t)(chunk / nstage) & 1u);
+        if (!__syncthreads_and(ok)) {
+            if (tid == 0) set_status(p.w.status, KGE_ERR_TIMEOUT);
+            // give copies still in flight a bounded chance to land before shared memory is released
+            for (int st = 0; st < nstage; ++st) (void)mbar_wait_bounded(&bars[st], (uint32_t)(chunk / nstage) & 1u);
+            return;
+        }
+        const float* Qs = base + (size_t)stage * ROWS * ld;
+        const float* Ts = Qs + IQ * ld;
+        const int len = min(kc, p.d - chunk * kc);
+#pragma unroll 2
+        for (int kk = 0; kk < len; kk += 4) {
+            float4 qv[4], tv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                qv[i] = *reinterpret_cast<const float4*>(&Qs[(ty + 16 * i) * ld + kk]);
+                tv[i] = *reinterpret_cast<const float4*>(&Ts[(tx + 16 * i) * ld + kk]);
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) canon_update<KIND>(acc[i][j], qv[i], tv[j]);
+        }
+        if (chunk + nstage < nchunk) {
+            __syncthreads();             // every thread is done reading this stage
+            issue(chunk + nstage, stage);
+        }
+    }
+    score_tile_epilogue<KIND>(p, acc, q0, e0, tx, ty);
+}
+
+template <int KIND>
+cudaError_t launch_score_tile_tma(const InferParams& p, unsigned grid, cudaStream_t s) {
+    static bool configured = false;
+    if (!configured) {
+        const cudaError_t e = cudaFuncSetAttribute(score_tile_tma_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)infer_tma_smem(kMaxDim));
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    score_tile_tma_kernel<KIND><<<grid, 256, infer_tma_smem(p.d), s>>>(p);
+    return cudaSuccess;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -330,17 +442,18 @@ __global__ void finish_kernel(InferParams p, int32_t* out_ids, float* out_scores
     if (out_ranks) out_ranks[q] = 1 + p.w.beat[q];
 }
 
-void launch_score_tiles(const InferParams& p, cudaStream_t s) {
+cudaError_t launch_score_tiles(const InferParams& p, cudaStream_t s) {
     const int64_t e_tiles = (p.e_hi - p.e_lo + IE - 1) / IE;
     const unsigned grid = (unsigned)(e_tiles * p.q_tiles);
     switch (p.kind) {
-        case KIND_L1: score_tile_kernel<KIND_L1><<<grid, 256, 0, s>>>(p); break;
-        case KIND_L2: score_tile_kernel<KIND_L2><<<grid, 256, 0, s>>>(p); break;
-        case KIND_CL1: score_tile_kernel<KIND_CL1><<<grid, 256, 0, s>>>(p); break;
-        case KIND_DOT: score_tile_kernel<KIND_DOT><<<grid, 256, 0, s>>>(p); break;
+        case KIND_L1: return launch_score_tile_tma<KIND_L1>(p, grid, s);
+        case KIND_L2: return launch_score_tile_tma<KIND_L2>(p, grid, s);
+        case KIND_CL1: return launch_score_tile_tma<KIND_CL1>(p, grid, s);
+        case KIND_DOT: return launch_score_tile_tma<KIND_DOT>(p, grid, s);
         case KIND_TH_L1: score_tile_kernel<KIND_TH_L1><<<grid, 256, 0, s>>>(p); break;
         default: score_tile_kernel<KIND_TH_L2><<<grid, 256, 0, s>>>(p); break;
     }
+    return cudaSuccess;
 }
 
 }  // namespace
@@ -371,7 +484,7 @@ int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int3
     }
     auto score_chunk = [&](const InferParams& ip) -> int {
         if (tc) return launch_tc_infer_chunk(h, nq, ip.e_lo, ip.e_hi, true_tails, s);
-        launch_score_tiles(ip, s);
+        KGE_CUDA_CHECK(h, launch_score_tiles(ip, s));
         KGE_LAUNCH_CHECK(h);
         return KGE_OK;
     };
