@@ -1300,7 +1300,7 @@ cudaError_t launch_block_tma(const TrainParams& p, cudaStream_t s) {
 
 template <int KIND, int NCH>
 cudaError_t launch_accum_tma_inst(const AccArgs& aq, const AccArgs& at, cudaStream_t s) {
-    constexpr int WARPS = (NCH == 4 || KIND == KIND_CL1) ? 8 : 4;   // the complex pairs wait on special-function results: more warps hide that
+    constexpr int WARPS = NCH == 4 ? 8 : 4;
     const size_t smem = accum_tma_smem(aq.d4);
     static bool configured = false;
     if (!configured) {
