@@ -27,6 +27,9 @@
  *   graph_build        : brute-force bucket membership + stable order on tiny graphs.
  *   sample_batch       : exact per-bucket / per-partition counts (Eq. 3, Eq. 4),
  *                        chi-square of the cube-root relation law.
+ *   bf16_round         : hand-worked IEEE bit patterns (ties to even both ways, carries,
+ *                        negatives, subnormals, the largest finite value) and an independent
+ *                        rounding routine on 10^5 random floats.
  *   score              : TransE 0 at h=t,r=0; DistMult symmetry; ComplEx -> DistMult
  *                        with zero imaginary parts; RotatE zero phase -> complex L1;
  *                        TransH special cases; numpy.linalg.norm for the L2 forms.
@@ -264,6 +267,9 @@ static real bf16_round(real v) { /* round-to-nearest-even to 8 significand bits 
     memcpy(&f, &u, 4);
     return (real)f;
 }
+
+/* The operand rounding of the tensor-core variant, exported so that it can be pinned on bit patterns. */
+real kgeo_bf16_round(real v) { return bf16_round(v); }
 
 /* TransH unit normal: w / max(||w||_2, 1e-12). */
 static real unit_normal(int32_t d, const real *w, real *what) {

@@ -92,6 +92,8 @@ class Oracle:
         L.kgeo_icbrt_weight.restype = C.c_uint64
         L.kgeo_icbrt_weight.argtypes = [C.c_uint64]
         L.kgeo_score.restype = R
+        L.kgeo_bf16_round.restype = R
+        L.kgeo_bf16_round.argtypes = [R]
         L.kgeo_score_grad.restype = None
         L.kgeo_row_loss.restype = R
         L.kgeo_batch_loss.restype = C.c_double
@@ -153,6 +155,10 @@ class Oracle:
         return heads, rels, tails, negs
 
     # -- scores / losses ----------------------------------------------------------
+    def bf16_round(self, v):
+        """The operand rounding of the bf16 variant (nearest, ties to even), as a Python float."""
+        return float(self.lib.kgeo_bf16_round(self.creal(v)))
+
     def score(self, score, p, h, r, t, w=None, bf16=0):
         score = SCORE_NAMES[score] if isinstance(score, str) else score
         h, r, t = self.arr(h), self.arr(r), self.arr(t)

@@ -103,6 +103,97 @@ def test_bf16_operand_variant_is_close_and_exact_on_bf16_inputs(oracle64):
     assert oracle64.score("transe", 2, h, np.zeros(d), t, bf16=1) == pytest.approx(-np.linalg.norm(h - t), rel=1e-13)
 
 
+def _f32(bits):
+    return float(np.array([bits], dtype=np.uint32).view(np.float32)[0])
+
+
+# (fp32 input bits, bf16 result as the upper 16 bits) worked out by hand from the IEEE definition of
+# round-to-nearest-even to an 8-bit significand: bf16 keeps the upper 16 bits of the fp32 pattern, the
+# lower 16 bits are the discarded fraction (0x8000 = exactly half a unit in the last kept place).
+BF16_PATTERNS = [
+    (0x3F800000, 0x3F80),   # 1.0 is representable
+    (0x3F808000, 0x3F80),   # 1 + 2^-8: a tie, kept mantissa 0000000 is even -> down to 1.0
+    (0x3F818000, 0x3F82),   # 1 + 3 2^-8: a tie, kept mantissa 0000001 is odd -> up to 1 + 2^-6
+    (0x3F808001, 0x3F81),   # just above the tie -> up
+    (0x3F807FFF, 0x3F80),   # just below the tie -> down
+    (0x3F810001, 0x3F81),   # just above a representable value -> stays
+    (0xBF808000, 0xBF80),   # the negative twins: rounding is symmetric in the sign
+    (0xBF818000, 0xBF82),
+    (0xBF808001, 0xBF81),
+    (0x3FFF8000, 0x4000),   # 2 - 2^-8: a tie with kept mantissa 1111111 (odd) -> carries into the exponent: 2.0
+    (0x3FFF7FFF, 0x3FFF),   # just below it -> 2 - 2^-7
+    (0x7F7F7FFF, 0x7F7F),   # the largest input that stays finite
+    (0x7F7FFFFF, 0x7F80),   # the largest finite fp32 lies above the last tie -> +inf
+    (0x7F7F8000, 0x7F80),   # that tie itself: kept mantissa odd -> up -> +inf
+    (0x00000001, 0x0000),   # smallest fp32 subnormal -> +0
+    (0x00008000, 0x0000),   # half of the smallest bf16 subnormal: a tie -> even -> +0
+    (0x00008001, 0x0001),   # just above -> the smallest bf16 subnormal 2^-133
+    (0x00018000, 0x0002),   # 1.5 x 2^-133: a tie, odd -> up to 2^-132
+    (0x007F8000, 0x0080),   # subnormal that rounds up into the smallest normal 2^-126
+    (0x80008000, 0x8000),   # -0 result keeps its sign
+]
+
+
+def test_bf16_round_hand_worked_bit_patterns(oracle64, oracle32):
+    for o in (oracle64, oracle32):
+        for bits, want_hi in BF16_PATTERNS:
+            got = np.array([o.bf16_round(_f32(bits))], dtype=np.float32).view(np.uint32)[0]
+            assert got == want_hi << 16, (hex(bits), hex(got), hex(want_hi << 16))
+    # a few of the same as plain numbers
+    assert oracle64.bf16_round(1 + 2.0 ** -8) == 1.0
+    assert oracle64.bf16_round(1 + 3 * 2.0 ** -8) == 1 + 2.0 ** -6
+    assert oracle64.bf16_round(-(1 + 2.0 ** -8 + 2.0 ** -20)) == -(1 + 2.0 ** -7)
+    assert oracle64.bf16_round(2 - 2.0 ** -8) == 2.0
+    assert oracle64.bf16_round(3.3895313892515355e38) == 3.3895313892515355e38     # (2 - 2^-7) 2^127, the largest bf16
+    assert oracle64.bf16_round(float(np.finfo(np.float32).max)) == float("inf")
+
+
+def test_bf16_round_against_an_independent_routine_on_random_floats(oracle64):
+    """torch's float -> bfloat16 conversion (round to nearest even) on 10^5 random bit patterns of
+    every magnitude, and exact rational arithmetic on a sample of them."""
+    import torch
+    from fractions import Fraction
+    rng = np.random.default_rng(11)
+    bits = rng.integers(0, 2 ** 32, size=100_000, dtype=np.uint64).astype(np.uint32)
+    x = bits.view(np.float32)
+    x = x[np.isfinite(x)]
+    want = torch.from_numpy(x.copy()).to(torch.bfloat16).to(torch.float32).numpy()
+    got = np.array([oracle64.bf16_round(float(v)) for v in x], dtype=np.float32)
+    assert (got.view(np.uint32) == want.view(np.uint32)).all()
+    # the definition itself on normal numbers: nearest multiple of 2^(e-7), ties to the even multiple
+    for v in x[:2000]:
+        if v == 0 or abs(float(v)) < 2.0 ** -120 or abs(float(v)) > 2.0 ** 120:
+            continue
+        fr = Fraction(float(v))
+        e = int(np.floor(np.log2(abs(float(v)))))
+        while Fraction(2) ** e > abs(fr):
+            e -= 1
+        while Fraction(2) ** (e + 1) <= abs(fr):
+            e += 1
+        ulp = Fraction(2) ** (e - 7)
+        n = fr / ulp
+        lo = n.numerator // n.denominator
+        rem = n - lo
+        k = lo + (1 if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and lo % 2 == 1) else 0)
+        assert Fraction(oracle64.bf16_round(float(v))) == k * ulp, float(v)
+
+
+def test_bf16_norm_expansion_clamps_negative_squared_distance(oracle64):
+    """TransE p = 2 in the bf16 variant is -sqrt(max(|q|^2 + |t|^2 - 2 bf16(q).bf16(t), 0)).  With q = t the
+    exact distance is 0, but the rounded cross term differs from |q|^2: operands that round up in magnitude
+    make the expansion negative, which must clamp to a score of exactly 0 (not NaN); operands that round
+    down leave 2 d (x^2 - bf16(x)^2) > 0, whose root is the score."""
+    d = 4
+    up = 1 + 0.75 * 2.0 ** -7          # rounds to 1 + 2^-7: bf16(q).bf16(t) > |q|^2
+    f = oracle64.score("transe", 2, np.full(d, up), np.zeros(d), np.full(d, up), bf16=1)
+    assert f == 0.0 and not np.isnan(f)
+    down = 1 + 0.25 * 2.0 ** -7        # rounds to 1.0
+    f = oracle64.score("transe", 2, np.full(d, down), np.zeros(d), np.full(d, down), bf16=1)
+    assert f == pytest.approx(-np.sqrt(2 * d * (down * down - 1.0)), rel=1e-12)
+    # the exact variant scores 0 in both cases
+    assert oracle64.score("transe", 2, np.full(d, up), np.zeros(d), np.full(d, up)) == 0.0
+
+
 # ----------------------------------------------------------------------------- losses
 def test_sampled_softmax_uniform_scores_closed_forms(oracle64):
     N, E = 37, 1000
