@@ -121,6 +121,27 @@ int kge_graph_load(kge_handle* h, const int32_t* heads /*[host]*/, const int32_t
                    const int32_t* tails /*[host]*/, int64_t n, void* stream);
 
 /*
+ * The same preprocessing for triple lists that already live in device memory (heads, rels, tails:
+ * device int32 [n], read only, n < 2^31), done entirely on the device: keys counted with integer
+ * atomics, the canonical order made by a stable least-significant-digit radix sort of the triple
+ * indices, weights in 128-bit integer arithmetic.  The result is bit-identical to kge_graph_load on
+ * the same list.  Synchronises `stream`; same error codes (KGE_ERR_UNSUPPORTED if P^2 |R| > 2^31).
+ */
+int kge_graph_load_device(kge_handle* h, const int32_t* heads, const int32_t* rels, const int32_t* tails,
+                          int64_t n, void* stream);
+
+/*
+ * Optional initialisation of the bound tables on the device (the paper prescribes none): entity rows
+ * and relation rows N(0, std^2), RotatE phases uniform in (-pi, pi), TransH normals N(0, std^2);
+ * optimiser state zero.  Element (row, 4c + j) comes from word j of Philox4x32-10 with key = seed and
+ * counter (row lo, row hi, c, stream) -- stream 2 entities, 3 relations, 4 normals -- through the
+ * uniform u = ((word >> 9) + 1/2) 2^-23 and, for normal entries, Box-Muller on the word pairs (0, 1)
+ * and (2, 3): std sqrt(-2 ln u_a) (cos, sin)(2 pi u_b).  A table is a pure function of (seed, shape).
+ * Enqueues on `stream` and returns.
+ */
+int kge_init_tables(kge_handle* h, float std, void* stream);
+
+/*
  * Draw the batch of step `step` (Section 4 "Training", Eq. 3 and Eq. 4): B positives, with
  * replacement, B/P^2 from every bucket (or B/P from each T_{i,j} of head_part i), the
  * relation by p(r) ~ n_r^(1/3) and the triple uniform within (bucket, r); N negatives,
@@ -185,8 +206,8 @@ int kge_score_all_topk(kge_handle* h, const int32_t* q_heads, const int32_t* q_r
  * current); make that first call outside any stream capture.  All calls share the one
  * array: it keeps the previous call's contents (this entry point clears what must start at
  * zero), and two calls that overlap on the same GPU -- from different streams or threads --
- * race on it, so serialise them.  Synchronises `stream`; returns 0, an argument error, or the
- * code recorded on the device (KGE_ERR_ID_RANGE).
+ * race on it, so serialise them.  Synchronises `stream`; returns 0, an argument error,
+ * KGE_ERR_CUDA, or the code recorded on the device (KGE_ERR_ID_RANGE, KGE_ERR_TIMEOUT).
  */
 int kge_score_all_topk_static(const kge_config* cfg /*[host]*/, const float* ent, const float* rel,
                               const float* relw, const int32_t* q_heads, const int32_t* q_rels, int32_t nq,
@@ -200,6 +221,14 @@ int kge_score_all_topk_static(const kge_config* cfg /*[host]*/, const float* ent
  */
 int kge_eval_mrr(kge_handle* h, const int32_t* q_heads, const int32_t* q_rels, const int32_t* true_tails,
                  int32_t nq, int32_t k_cutoff, double* mrr_out /*[host]*/, void* stream);
+
+/*
+ * The same mean over ranks the caller already has (the out_ranks of kge_score_all_topk, [nq] int32 on
+ * the device), so that a caller who needs the lists and the metric scores the table once.  The sum is
+ * taken in fp64 on the device in a fixed order.  mrr_out: [host] double.  Synchronises `stream`.
+ */
+int kge_mrr_from_ranks(kge_handle* h, const int32_t* ranks, int32_t nq, int32_t k_cutoff,
+                       double* mrr_out /*[host]*/, void* stream);
 
 /* Synchronise `stream`, return the sticky device status word (0 or a negative code), clear it. */
 int kge_get_status(kge_handle* h, void* stream);
@@ -242,10 +271,36 @@ typedef enum {
     KGE_TAP_ENT_PERM = 8,  /* [2B+N] int32 source positions, stably sorted by id */
     KGE_TAP_REL_UNIQ = 9, KGE_TAP_REL_SEG = 10, KGE_TAP_REL_PERM = 11,
     KGE_TAP_LROW = 12,     /* [B] per-positive loss */
-    KGE_TAP_BATCH = 13     /* [3B+N] int32 heads | rels | tails | negs used by the step */
+    KGE_TAP_BATCH = 13,    /* [3B+N] int32 heads | rels | tails | negs used by the step */
+    KGE_TAP_GRAPH_H = 14, KGE_TAP_GRAPH_R = 15, KGE_TAP_GRAPH_T = 16,   /* [T] int32 triples in canonical order */
+    KGE_TAP_GRAPH_OFF = 17,   /* [P*P*(R+1)] int64 first sorted index of relation r in bucket (i, j) */
+    KGE_TAP_GRAPH_WCUM = 18   /* [P*P*(R+1)] uint64 running sums of the cube-root weights per bucket */
 } kge_tap_t;
 size_t kge_debug_bytes(kge_handle* h, int tap, void* stream);
 int kge_debug_export(kge_handle* h, int tap, void* dst /*[host]*/, size_t bytes, void* stream);
+
+/*
+ * Parity tap of the B x N score block F_bn = f(q_b, t_n) (scoring-function table): while scores_out
+ * (a caller-owned device array of B * N floats, 16-byte aligned) is set, every kge_train_step also
+ * writes the block there, row-major [B, N] -- a device copy before the loss overwrites the block on
+ * the fp32 path, one extra contraction on the tensor-core path (which never stores the block).
+ * NULL switches the tap off.  Never on a timed path.
+ */
+int kge_debug_capture_scores(kge_handle* h, float* scores_out);
+
+/*
+ * Every wait of a kernel on an asynchronous copy or a barrier is a bounded loop of `tries`
+ * attempts (default 2^20, seconds in all; 0 restores the default).  A test shortens it here;
+ * kge_debug_wait_probe then launches one thread block that waits on a barrier nothing arrives at:
+ * the wait runs out after `tries` attempts, the kernel records KGE_ERR_TIMEOUT in the status word
+ * and returns -- the give-up path every kernel of the library shares -- and the context stays usable.
+ */
+/* Parity tap of the table generator: the raw Philox words of kge_init_tables for a [rows, width]
+ * table of stream `stream_id`, as bit patterns in out (device, rows * width words). */
+int kge_debug_init_words(kge_handle* h, float* out, int64_t rows, int32_t width, uint32_t stream_id, void* stream);
+
+int kge_debug_set_wait_limit(kge_handle* h, int32_t tries);
+int kge_debug_wait_probe(kge_handle* h, void* stream);
 
 #ifdef __cplusplus
 }

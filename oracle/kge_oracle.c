@@ -21,15 +21,24 @@
  * Compile with -O2 -fno-fast-math -ffp-contract=off so that nothing is fused or
  * reassociated beyond what is written.
  *
+ * Sub-gradient of |x| at x = 0 (p = 1 distances): 0 by default.  Any value in [-1, 1] is a valid
+ * sub-gradient there; a third build with -DKGEO_L1_TIE_SIGN=-1 takes sign(0) = -1 (the left
+ * derivative) and exists only so that a test on constructed exact ties can check, coordinate by
+ * coordinate, which sub-gradient the CUDA library takes.  It differs from the default build at
+ * exact ties only (pinned by a closed form on TransE).
+ *
  * Parity pins (tests/test_oracle_*.py, all CPU):
  *   philox4x32_10      : cross-checked against cuRAND's host Philox generator.
  *   mulhi64, icbrt     : Python big-integer arithmetic.
+ *   init_table         : moments and Kolmogorov-Smirnov tests against the normal / uniform laws,
+ *                        independence of neighbouring entries, the raw words against philox.
  *   graph_build        : brute-force bucket membership + stable order on tiny graphs.
  *   sample_batch       : exact per-bucket / per-partition counts (Eq. 3, Eq. 4),
  *                        chi-square of the cube-root relation law.
  *   bf16_round         : hand-worked IEEE bit patterns (ties to even both ways, carries,
  *                        negatives, subnormals, the largest finite value) and an independent
  *                        rounding routine on 10^5 random floats.
+ *   query_vector       : numpy restatement per model; f(h, r, t) recovered from (q, t) alone.
  *   score              : TransE 0 at h=t,r=0; DistMult symmetry; ComplEx -> DistMult
  *                        with zero imaginary parts; RotatE zero phase -> complex L1;
  *                        TransH special cases; numpy.linalg.norm for the L2 forms.
@@ -46,6 +55,9 @@
 
 #ifndef KGEO_F32
 #define KGEO_F32 0
+#endif
+#ifndef KGEO_L1_TIE_SIGN
+#define KGEO_L1_TIE_SIGN 0
 #endif
 
 #if KGEO_F32
@@ -131,6 +143,44 @@ static void draw2x64(uint64_t seed, uint64_t step, uint32_t slot, uint32_t strea
     kgeo_philox4x32_10(ctr, key, o);
     *x64 = (uint64_t)o[0] | ((uint64_t)o[1] << 32);
     *y64 = (uint64_t)o[2] | ((uint64_t)o[3] << 32);
+}
+
+/* ------------------------------------------------------------------------- */
+/* Table initialisation.  The paper prescribes none; this is the library's     */
+/* recipe: element (row, 4c + j) of a [rows, width] table comes from word j of  */
+/* Philox with counter (row lo, row hi, c, stream) under the seed, through the   */
+/* uniform u = ((word >> 9) + 1/2) 2^-23 in (0, 1).  kind 0: normal entries by   */
+/* Box-Muller on the word pairs (0, 1) and (2, 3): std sqrt(-2 ln u_a) times      */
+/* (cos, sin)(2 pi u_b).  kind 1: phases (2u - 1) pi.  kind 2: the raw words      */
+/* (as bit patterns).  Computed in fp64, stored as fp32 like every table.         */
+/* ------------------------------------------------------------------------- */
+void kgeo_init_table(uint64_t seed, uint32_t stream, int64_t rows, int32_t width, double std,
+                     int32_t kind, float *out) {
+    const double PI = 3.14159265358979323846;
+    for (int64_t row = 0; row < rows; ++row) {
+        for (int32_t c = 0; 4 * c < width; ++c) {
+            uint32_t ctr[4] = { (uint32_t)row, (uint32_t)((uint64_t)row >> 32), (uint32_t)c, stream };
+            uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+            uint32_t x[4];
+            kgeo_philox4x32_10(ctr, key, x);
+            double u[4], v[4];
+            for (int j = 0; j < 4; ++j) u[j] = ((double)(x[j] >> 9) + 0.5) / 8388608.0;
+            if (kind == 1) {
+                for (int j = 0; j < 4; ++j) v[j] = (2.0 * u[j] - 1.0) * PI;
+            } else {
+                for (int j = 0; j < 4; j += 2) {
+                    double rad = std * sqrt(-2.0 * log(u[j]));
+                    v[j] = rad * cos(2.0 * PI * u[j + 1]);
+                    v[j + 1] = rad * sin(2.0 * PI * u[j + 1]);
+                }
+            }
+            for (int j = 0; j < 4 && 4 * c + j < width; ++j) {
+                float f = (float)v[j];
+                if (kind == 2) memcpy(&f, &x[j], 4);
+                out[row * width + 4 * c + j] = f;
+            }
+        }
+    }
 }
 
 /* ------------------------------------------------------------------------- */
@@ -334,6 +384,30 @@ static void dot_query(int32_t score, int32_t d, const real *h, const real *r, re
 }
 
 /*
+ * Per-query vector q of the scoring-function table, the part of f(h, r, t) that does not depend
+ * on the tail: TransE h + r; TransH (h - (w^.h) w^) + r with w^ the unit normal; RotatE h o e^{i r};
+ * DistMult r o h; ComplEx r h.  The score is then a function of (q, t) (and w^ for TransH).
+ */
+void kgeo_query_vector(int32_t score, int32_t d, const real *h, const real *r, const real *w, real *q) {
+    if (score == SC_DISTMULT || score == SC_COMPLEX) { dot_query(score, d, h, r, q); return; }
+    if (score == SC_TRANSE) { for (int k = 0; k < d; ++k) q[k] = h[k] + r[k]; return; }
+    if (score == SC_ROTATE) {
+        for (int k = 0; k < d / 2; ++k) {
+            real cs = R_COS(r[k]), sn = R_SIN(r[k]);
+            q[2 * k] = R_FMA(h[2 * k], cs, -(h[2 * k + 1] * sn));
+            q[2 * k + 1] = R_FMA(h[2 * k], sn, h[2 * k + 1] * cs);
+        }
+        return;
+    }
+    real *what = (real *)malloc(sizeof(real) * (size_t)d);
+    unit_normal(d, w, what);
+    real a = 0;
+    for (int k = 0; k < d; ++k) a = R_FMA(what[k], h[k], a);
+    for (int k = 0; k < d; ++k) q[k] = R_FMA(-a, what[k], h[k]) + r[k];
+    free(what);
+}
+
+/*
  * f(h, r, t).  `w` is the TransH normal (ignored otherwise); `scratch` holds 3*d reals.
  * bf16 = 1 rounds the two operands of the contraction to bf16 first (dot-product
  * models: q and t; TransE-L2: q = h + r and t inside the cross term only).
@@ -415,7 +489,7 @@ static void score_grad_one(int32_t score, int32_t p, int32_t d, real g,
             s[2 * k + 1] = m > 0 ? -x[2 * k + 1] / m : 0;
         }
     } else {
-        for (int k = 0; k < d; ++k) s[k] = x[k] > 0 ? (real)-1 : (x[k] < 0 ? (real)1 : (real)0);
+        for (int k = 0; k < d; ++k) s[k] = x[k] > 0 ? (real)-1 : (x[k] < 0 ? (real)1 : -(real)KGEO_L1_TIE_SIGN);
     }
     if (score == SC_TRANSE) { /* x = h + r - t */
         for (int k = 0; k < d; ++k) {

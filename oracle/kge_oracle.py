@@ -62,14 +62,19 @@ def lib_path(precision: str) -> Path:
     return _HERE / f"libkge_oracle_{precision}.so"
 
 
+# build name -> extra defines.  "f64_tie" is the fp64 build whose sub-gradient of |x| at 0 is -1
+# instead of 0 (see the header of kge_oracle.c); only the exact-tie tests load it.
+_BUILDS = {"f64": ["-DKGEO_F32=0"], "f32": ["-DKGEO_F32=1"], "f64_tie": ["-DKGEO_F32=0", "-DKGEO_L1_TIE_SIGN=-1"]}
+
+
 def build(force: bool = False) -> None:
-    """Compile both precisions with gcc (no fast-math, no contraction, OpenMP over rows)."""
-    for prec, flag in (("f64", "0"), ("f32", "1")):
+    """Compile every build with gcc (no fast-math, no contraction, OpenMP over rows)."""
+    for prec, flags in _BUILDS.items():
         out = lib_path(prec)
         if not force and out.exists() and out.stat().st_mtime >= _SRC.stat().st_mtime:
             continue
         cmd = ["gcc", "-std=c11", "-O2", "-fno-fast-math", "-ffp-contract=off", "-fopenmp", "-fPIC",
-               "-shared", f"-DKGEO_F32={flag}", str(_SRC), "-o", str(out), "-lm"]
+               "-shared", *flags, str(_SRC), "-o", str(out), "-lm"]
         subprocess.run(cmd, check=True)
 
 
@@ -79,11 +84,11 @@ def _p(a, ctype):
 
 class Oracle:
     def __init__(self, precision: str = "f64"):
-        assert precision in ("f64", "f32")
+        assert precision in _BUILDS
         build()
         self.precision = precision
-        self.real = np.float64 if precision == "f64" else np.float32
-        self.creal = C.c_double if precision == "f64" else C.c_float
+        self.real = np.float32 if precision == "f32" else np.float64
+        self.creal = C.c_float if precision == "f32" else C.c_double
         self.lib = C.CDLL(str(lib_path(precision)))
         assert self.lib.kgeo_real_bytes() == np.dtype(self.real).itemsize
         L, R = self.lib, self.creal
@@ -95,6 +100,8 @@ class Oracle:
         L.kgeo_bf16_round.restype = R
         L.kgeo_bf16_round.argtypes = [R]
         L.kgeo_score_grad.restype = None
+        L.kgeo_init_table.restype = None
+        L.kgeo_query_vector.restype = None
         L.kgeo_row_loss.restype = R
         L.kgeo_batch_loss.restype = C.c_double
         L.kgeo_batch_grads.restype = C.c_double
@@ -124,6 +131,13 @@ class Oracle:
 
     def icbrt_weight(self, n):
         return int(self.lib.kgeo_icbrt_weight(C.c_uint64(n)))
+
+    def init_table(self, seed, stream, rows, width, std=1.0, kind=0):
+        """fp32 [rows, width] table of the library's initialisation recipe (kind 0 normal, 1 phases, 2 raw words)."""
+        out = np.empty((rows, width), dtype=np.float32)
+        self.lib.kgeo_init_table(C.c_uint64(seed), C.c_uint32(stream), C.c_int64(rows), C.c_int32(width), C.c_double(std),
+                                 C.c_int32(kind), _p(out, C.c_float))
+        return out
 
     # -- graph + sampler --------------------------------------------------------
     def graph_build(self, E, R, P, h, r, t):
@@ -166,6 +180,15 @@ class Oracle:
         R = self.creal
         return float(self.lib.kgeo_score(C.c_int32(score), C.c_int32(p), C.c_int32(len(h)), C.c_int32(bf16),
                                          _p(h, R), _p(r, R), _p(w, R), _p(t, R)))
+
+    def query_vector(self, score, h, r, w=None):
+        score = SCORE_NAMES[score] if isinstance(score, str) else score
+        h, r = self.arr(h), self.arr(r)
+        w = None if w is None else self.arr(w)
+        R = self.creal
+        q = np.empty_like(h)
+        self.lib.kgeo_query_vector(C.c_int32(score), C.c_int32(len(h)), _p(h, R), _p(r, R), _p(w, R), _p(q, R))
+        return q
 
     def score_grad(self, score, p, g, h, r, t, w=None):
         score = SCORE_NAMES[score] if isinstance(score, str) else score

@@ -21,8 +21,10 @@ LOSS_NAMES = {"logsigmoid": LOSS_LOGSIGMOID, "softmax": LOSS_SAMPLED_SOFTMAX}
 OPT_NAMES = {"sgd": OPT_SGD, "adam": OPT_ADAM, "adagrad": OPT_ROWWISE_ADAGRAD}
 
 TAPS = dict(Q=0, FPOS=1, G=2, GRAD_ENT=3, GRAD_REL=4, GRAD_RELW=5, ENT_UNIQ=6, ENT_SEG=7, ENT_PERM=8,
-            REL_UNIQ=9, REL_SEG=10, REL_PERM=11, LROW=12, BATCH=13)
-_INT_TAPS = {"ENT_UNIQ", "ENT_SEG", "ENT_PERM", "REL_UNIQ", "REL_SEG", "REL_PERM", "BATCH"}
+            REL_UNIQ=9, REL_SEG=10, REL_PERM=11, LROW=12, BATCH=13, GRAPH_H=14, GRAPH_R=15, GRAPH_T=16,
+            GRAPH_OFF=17, GRAPH_WCUM=18)
+_INT_TAPS = {"ENT_UNIQ", "ENT_SEG", "ENT_PERM", "REL_UNIQ", "REL_SEG", "REL_PERM", "BATCH", "GRAPH_H", "GRAPH_R", "GRAPH_T"}
+_I64_TAPS = {"GRAPH_OFF": "int64", "GRAPH_WCUM": "uint64"}
 
 KGE_ERR_NO_EXTENSION = -10
 
@@ -75,6 +77,9 @@ SIGNATURES = {
     "kge_workspace_bytes": (C.c_size_t, [_vp, C.c_int64, C.c_int32, C.c_int32]),
     "kge_bind": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_size_t, C.c_int64, C.c_int32, C.c_int32, _vp]),
     "kge_graph_load": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int64, _vp]),
+    "kge_graph_load_device": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int64, _vp]),
+    "kge_init_tables": (C.c_int, [_vp, C.c_float, _vp]),
+    "kge_debug_init_words": (C.c_int, [_vp, _vp, C.c_int64, C.c_int32, C.c_uint32, _vp]),
     "kge_sample_batch": (C.c_int, [_vp, C.c_uint64, _vp, _vp, _vp, _vp, _vp]),
     "kge_train_step": (C.c_int, [_vp, C.c_uint64, C.c_float, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kge_train_step_host": (C.c_int, [_vp, C.c_uint64, C.c_float, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -82,6 +87,10 @@ SIGNATURES = {
     "kge_score_all_topk_static": (C.c_int, [C.POINTER(KgeConfig), _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32, _vp, _vp, _vp,
                                             _vp, _vp]),
     "kge_eval_mrr": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int32, C.c_int32, C.POINTER(C.c_double), _vp]),
+    "kge_mrr_from_ranks": (C.c_int, [_vp, _vp, C.c_int32, C.c_int32, C.POINTER(C.c_double), _vp]),
+    "kge_debug_capture_scores": (C.c_int, [_vp, _vp]),
+    "kge_debug_set_wait_limit": (C.c_int, [_vp, C.c_int32]),
+    "kge_debug_wait_probe": (C.c_int, [_vp, _vp]),
     "kge_get_status": (C.c_int, [_vp, _vp]),
     "kge_launch_count": (C.c_int64, [_vp]),
     "kge_profile": (C.c_int, [_vp, C.c_int]),
@@ -186,6 +195,17 @@ class Kge:
         self._check(lib().kge_graph_load(self._h, _ptr(heads), _ptr(rels), _ptr(tails), len(heads), _stream()),
                     "kge_graph_load")
 
+    def graph_load_device(self, heads, rels, tails):
+        """heads / rels / tails: int32 device tensors."""
+        self._check(lib().kge_graph_load_device(self._h, _ptr(heads), _ptr(rels), _ptr(tails), heads.numel(), _stream()),
+                    "kge_graph_load_device")
+
+    def init_tables(self, std):
+        self._check(lib().kge_init_tables(self._h, std, _stream()), "kge_init_tables")
+
+    def debug_init_words(self, out, rows, width, stream_id):
+        self._check(lib().kge_debug_init_words(self._h, _ptr(out), rows, width, stream_id, _stream()), "kge_debug_init_words")
+
     def sample_batch(self, step, heads, rels, tails, negs):
         self._check(lib().kge_sample_batch(self._h, step, _ptr(heads), _ptr(rels), _ptr(tails), _ptr(negs), _stream()),
                     "kge_sample_batch")
@@ -209,6 +229,23 @@ class Kge:
         self._check(lib().kge_eval_mrr(self._h, _ptr(q_heads), _ptr(q_rels), _ptr(true_tails), q_heads.numel(),
                                        k_cutoff, C.byref(out), _stream()), "kge_eval_mrr")
         return out.value
+
+    def mrr_from_ranks(self, ranks, k_cutoff=10) -> float:
+        out = C.c_double(0.0)
+        self._check(lib().kge_mrr_from_ranks(self._h, _ptr(ranks), ranks.numel(), k_cutoff, C.byref(out), _stream()),
+                    "kge_mrr_from_ranks")
+        return out.value
+
+    def debug_capture_scores(self, scores_out):
+        """scores_out: float32 device tensor of B * N elements, or None to switch the tap off."""
+        self._capture = scores_out
+        self._check(lib().kge_debug_capture_scores(self._h, _ptr(scores_out)), "kge_debug_capture_scores")
+
+    def debug_set_wait_limit(self, tries: int):
+        self._check(lib().kge_debug_set_wait_limit(self._h, tries), "kge_debug_set_wait_limit")
+
+    def debug_wait_probe(self):
+        self._check(lib().kge_debug_wait_probe(self._h, _stream()), "kge_debug_wait_probe")
 
     def get_status(self) -> int:
         return int(lib().kge_get_status(self._h, _stream()))
@@ -234,7 +271,10 @@ class Kge:
         import numpy as np
         code = TAPS[tap]
         nbytes = int(lib().kge_debug_bytes(self._h, code, _stream()))
-        out = np.empty(nbytes // 4, dtype=np.int32 if tap in _INT_TAPS else np.float32)
+        if tap in _I64_TAPS:
+            out = np.empty(nbytes // 8, dtype=_I64_TAPS[tap])
+        else:
+            out = np.empty(nbytes // 4, dtype=np.int32 if tap in _INT_TAPS else np.float32)
         if nbytes:
             self._check(lib().kge_debug_export(self._h, code, _ptr(out), nbytes, _stream()), "kge_debug_export")
         return out

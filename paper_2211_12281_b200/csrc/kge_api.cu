@@ -56,9 +56,12 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
     w.status = cv.take<int32_t>(64);
     w.loss = reinterpret_cast<float*>(w.status ? w.status + 8 : nullptr);
     w.counts = w.status ? w.status + 16 : nullptr;
+    w.mrr = reinterpret_cast<double*>(w.status ? w.status + 32 : nullptr);
     w.gh = cv.take<int32_t>(T); w.gr = cv.take<int32_t>(T); w.gt = cv.take<int32_t>(T);
     w.off = cv.take<int64_t>(P * P * (R + 1));
     w.wcum = cv.take<uint64_t>(P * P * (R + 1));
+    w.gstart = T > 0 ? cv.take<uint64_t>(P * P * R + 1) : nullptr;
+    w.ghist = T > 0 ? cv.take<uint32_t>(graph_hist_words(T)) : nullptr;
     w.heads = cv.take<int32_t>(3 * B + N);
     if (w.heads) { w.rels = w.heads + B; w.tails = w.rels + B; w.negs = w.tails + B; }
     w.Q = cv.take<float>(B * d);
@@ -131,6 +134,35 @@ uint64_t icbrt_weight(uint64_t n) {
     return lo;
 }
 
+// Mean of (rank <= cutoff ? 1 / rank : 0) over nq ranks in fp64 by one CTA: every thread adds its
+// strided share in ascending order, the 256 partial sums are added by a fixed tree, so the result
+// is the same on every run.
+__global__ void __launch_bounds__(256) mrr_kernel(const int32_t* ranks, int nq, int cutoff, double* out) {
+    __shared__ double part[256];
+    double acc = 0.0;
+    for (int q = threadIdx.x; q < nq; q += 256) {
+        const int32_t r = ranks[q];
+        if (r >= 1 && (cutoff == 0 || r <= cutoff)) acc += 1.0 / (double)r;
+    }
+    part[threadIdx.x] = acc;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if ((int)threadIdx.x < o) part[threadIdx.x] += part[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *out = part[0] / (double)nq;
+}
+
+// One CTA that waits on a barrier nothing ever arrives at: the bounded wait runs out, the kernel
+// records KGE_ERR_TIMEOUT and returns.  Exercises the give-up path every kernel of the library shares.
+__global__ void wait_probe_kernel(int32_t* status, int limit) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) { mbar_init(&bar, 1); mbar_init_fence(); }
+    __syncthreads();
+    const bool ok = mbar_wait_bounded(&bar, 0u, limit);
+    if (!__syncthreads_and(ok) && threadIdx.x == 0) set_status(status, KGE_ERR_TIMEOUT);
+}
+
 }  // namespace
 
 extern "C" {
@@ -170,6 +202,9 @@ int kge_create(const kge_config* cfg, kge_handle** out) {
     h->bound = h->graph_loaded = false;
     h->streams_ready = false;
     h->launches = 0;
+    h->wait_limit = kDefaultWaitLimit;
+    h->capture_scores = nullptr;
+    h->cuda_err[0] = '\0';
     h->num_sms = 148;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) == cudaSuccess &&
@@ -325,6 +360,47 @@ int kge_graph_load(kge_handle* h, const int32_t* heads, const int32_t* rels, con
     return KGE_OK;
 }
 
+int kge_graph_load_device(kge_handle* h, const int32_t* heads, const int32_t* rels, const int32_t* tails, int64_t n,
+                          void* stream) {
+    if (!h || !heads || !rels || !tails || n < 0) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    if (n != h->num_triples) return KGE_ERR_WORKSPACE;
+    const kge_config& c = h->cfg;
+    // keys and triple indices are sorted as 32-bit words
+    if (n > ((int64_t)1 << 31) || (int64_t)c.num_parts * c.num_parts * c.num_relations > ((int64_t)1 << 31)) return KGE_ERR_UNSUPPORTED;
+    h->graph_loaded = false;
+    const int rc = launch_graph_build_device(h, heads, rels, tails, n, static_cast<cudaStream_t>(stream));
+    if (rc != KGE_OK) return rc;
+    h->graph_loaded = true;
+    return KGE_OK;
+}
+
+int kge_init_tables(kge_handle* h, float std, void* stream) {
+    if (!h || !(std >= 0.f)) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    const kge_config& c = h->cfg;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int rc = launch_init_table(h, h->ent, c.num_entities, c.dim, std, 0, 2u, s);
+    if (rc == KGE_OK) rc = launch_init_table(h, h->rel, c.num_relations, h->kw, std, c.score == KGE_ROTATE ? 1 : 0, 3u, s);
+    if (rc == KGE_OK && h->relw) rc = launch_init_table(h, h->relw, c.num_relations, c.dim, std, 0, 4u, s);
+    if (rc != KGE_OK) return rc;
+    // optimiser state starts at zero
+    const size_t per = c.opt == KGE_OPT_ADAM ? 2 : 1;
+    if (c.opt != KGE_OPT_SGD) {
+        const bool adam = c.opt == KGE_OPT_ADAM;
+        KGE_CUDA_CHECK(h, cudaMemsetAsync(h->ent_state, 0, (size_t)c.num_entities * (adam ? per * c.dim : 1) * sizeof(float), s));
+        KGE_CUDA_CHECK(h, cudaMemsetAsync(h->rel_state, 0, (size_t)c.num_relations * (adam ? per * h->kw : 1) * sizeof(float), s));
+        if (h->relw_state)
+            KGE_CUDA_CHECK(h, cudaMemsetAsync(h->relw_state, 0, (size_t)c.num_relations * (adam ? per * c.dim : 1) * sizeof(float), s));
+    }
+    return KGE_OK;
+}
+
+int kge_debug_init_words(kge_handle* h, float* out, int64_t rows, int32_t width, uint32_t stream_id, void* stream) {
+    if (!h || !out || rows < 0 || width <= 0) return KGE_ERR_BAD_ARG;
+    return launch_init_table(h, out, rows, width, 1.f, 2, stream_id, static_cast<cudaStream_t>(stream));
+}
+
 int kge_sample_batch(kge_handle* h, uint64_t step, int32_t* heads, int32_t* rels, int32_t* tails, int32_t* negs,
                      void* stream) {
     if (!h || !heads || !rels || !tails || !negs) return KGE_ERR_BAD_ARG;
@@ -405,23 +481,47 @@ int kge_score_all_topk(kge_handle* h, const int32_t* q_heads, const int32_t* q_r
                               static_cast<cudaStream_t>(stream));
 }
 
+int kge_mrr_from_ranks(kge_handle* h, const int32_t* ranks, int32_t nq, int32_t k_cutoff, double* mrr_out, void* stream) {
+    if (!h || !ranks || !mrr_out || nq <= 0 || k_cutoff < 0) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    mrr_kernel<<<1, 256, 0, s>>>(ranks, nq, k_cutoff, h->ws.mrr);
+    KGE_LAUNCH_CHECK(h);
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(mrr_out, h->ws.mrr, sizeof(double), cudaMemcpyDeviceToHost, s));
+    KGE_CUDA_CHECK(h, cudaStreamSynchronize(s));
+    return KGE_OK;
+}
+
 int kge_eval_mrr(kge_handle* h, const int32_t* q_heads, const int32_t* q_rels, const int32_t* true_tails,
                  int32_t nq, int32_t k_cutoff, double* mrr_out, void* stream) {
     if (!h || !q_heads || !q_rels || !true_tails || !mrr_out || nq <= 0 || k_cutoff < 0) return KGE_ERR_BAD_ARG;
     if (!h->bound) return KGE_ERR_NOT_READY;
     if (nq > h->max_queries || h->topk < 1) return KGE_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    Workspace& w = h->ws;
-    // a k = 1 search whose lists are discarded; only the ranks are used
-    int rc = run_score_all_topk(h, q_heads, q_rels, nq, 1, true_tails, nullptr, nullptr, w.beat_tmp, s);
+    // a k = 1 search whose lists are discarded; only the ranks are used (they land in the workspace)
+    const int rc = run_score_all_topk(h, q_heads, q_rels, nq, 1, true_tails, nullptr, nullptr, h->ws.beat_tmp, s);
     if (rc != KGE_OK) return rc;
-    std::vector<int32_t> ranks(nq);
-    KGE_CUDA_CHECK(h, cudaMemcpyAsync(ranks.data(), w.beat_tmp, nq * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
-    KGE_CUDA_CHECK(h, cudaStreamSynchronize(s));
-    double acc = 0.0;
-    for (int32_t q = 0; q < nq; ++q)
-        if (k_cutoff == 0 || ranks[q] <= k_cutoff) acc += 1.0 / (double)ranks[q];
-    *mrr_out = acc / nq;
+    return kge_mrr_from_ranks(h, h->ws.beat_tmp, nq, k_cutoff, mrr_out, stream);
+}
+
+int kge_debug_set_wait_limit(kge_handle* h, int32_t tries) {
+    if (!h || tries < 0) return KGE_ERR_BAD_ARG;
+    h->wait_limit = tries == 0 ? kDefaultWaitLimit : tries;
+    return KGE_OK;
+}
+
+int kge_debug_wait_probe(kge_handle* h, void* stream) {
+    if (!h) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    wait_probe_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(h->ws.status, h->wait_limit);
+    KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
+}
+
+int kge_debug_capture_scores(kge_handle* h, float* scores_out) {
+    if (!h) return KGE_ERR_BAD_ARG;
+    if (scores_out && (reinterpret_cast<uintptr_t>(scores_out) % 16) != 0) return KGE_ERR_BAD_ARG;
+    h->capture_scores = scores_out;
     return KGE_OK;
 }
 
@@ -473,7 +573,7 @@ const char* kge_error_string(int code) {
     }
 }
 
-const char* kge_last_cuda_error(const kge_handle* h) { return h ? h->cuda_err.c_str() : ""; }
+const char* kge_last_cuda_error(const kge_handle* h) { return h ? h->cuda_err : ""; }
 
 size_t kge_debug_bytes(kge_handle* h, int tap, void* stream) {
     if (!h || !h->bound) return 0;
@@ -499,6 +599,9 @@ size_t kge_debug_bytes(kge_handle* h, int tap, void* stream) {
         case KGE_TAP_REL_SEG: return ((size_t)counts[1] + 1) * 4;
         case KGE_TAP_REL_PERM: return B * 4;
         case KGE_TAP_BATCH: return (3 * B + N) * 4;
+        case KGE_TAP_GRAPH_H: case KGE_TAP_GRAPH_R: case KGE_TAP_GRAPH_T: return h->graph_loaded ? (size_t)h->num_triples * 4 : 0;
+        case KGE_TAP_GRAPH_OFF: case KGE_TAP_GRAPH_WCUM:
+            return h->graph_loaded ? (size_t)c.num_parts * c.num_parts * (c.num_relations + 1) * 8 : 0;
         default: return 0;
     }
 }
@@ -525,6 +628,11 @@ int kge_debug_export(kge_handle* h, int tap, void* dst, size_t bytes, void* stre
         case KGE_TAP_REL_SEG: src = w.rel_seg; break;
         case KGE_TAP_REL_PERM: src = w.rel_perm; break;
         case KGE_TAP_BATCH: src = w.heads; break;
+        case KGE_TAP_GRAPH_H: src = w.gh; break;
+        case KGE_TAP_GRAPH_R: src = w.gr; break;
+        case KGE_TAP_GRAPH_T: src = w.gt; break;
+        case KGE_TAP_GRAPH_OFF: src = w.off; break;
+        case KGE_TAP_GRAPH_WCUM: src = w.wcum; break;
         default: return KGE_ERR_BAD_ARG;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);

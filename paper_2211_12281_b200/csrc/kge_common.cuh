@@ -5,9 +5,10 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#include <string>
+#include <cstdio>
 
 #include "../../include/kge.h"
+#include "kge_device_once.h"
 
 namespace kge {
 
@@ -42,6 +43,8 @@ struct Workspace {
     int32_t *gh, *gr, *gt; // [T]
     int64_t* off;          // [P*P*(R+1)]
     uint64_t* wcum;        // [P*P*(R+1)]
+    uint64_t* gstart;      // [P*P*R + 1] on-device preprocessing: triples per key, then first sorted index per key
+    uint32_t* ghist;       // [256 * tiles + 1] on-device preprocessing: digit-major tile histograms of a radix pass
     // batch
     int32_t *heads, *rels, *tails, *negs;  // contiguous [3B+N]
     float *Q, *What, *Tneg;                // [B,d], [B,d] (TransH), [N,d]
@@ -66,6 +69,7 @@ struct Workspace {
     uint64_t *ent_tkeys, *rel_tkeys;       // tile-sorted (id, position) keys, padded to whole tiles
     float *part_ent, *part_rel, *part_relw;  // [list length, width] partial sums of long segments
     // inference
+    double* mrr;                           // [1] mean reciprocal rank of the last kge_eval_mrr (in the header block)
     float *iq, *iwhat, *iftrue;            // [maxq,d], [maxq,d], [maxq]
     uint16_t *iqb, *Eb;                    // [maxq,d], [E,d] bf16 query vectors and entity table (tensor-core inference)
     float *thr;                            // [maxq] current k-th best score (-inf until the list is full)
@@ -116,16 +120,20 @@ struct kge_handle {
     bool streams_ready;
     cudaStream_t side[2];
     cudaEvent_t ev_ids, ev_loss, ev_seg, ev_t;
-    std::string cuda_err;
+    int wait_limit;         // tries of every bounded barrier wait in this handle's kernels (kDefaultWaitLimit unless a test shortens it)
+    float* capture_scores;  // debug: the training step also writes the B x N score block here (caller's device array), or NULL
+    char cuda_err[256];     // text of the last failed CUDA call (a fixed buffer: reporting an error allocates nothing)
 };
 
 namespace kge {
+
+constexpr int kDefaultWaitLimit = 1 << 20;   // tries of a bounded barrier wait: seconds in all
 
 #define KGE_CUDA_CHECK(h, expr)                                   \
     do {                                                          \
         cudaError_t e_ = (expr);                                  \
         if (e_ != cudaSuccess) {                                  \
-            (h)->cuda_err = std::string(#expr) + ": " + cudaGetErrorString(e_); \
+            std::snprintf((h)->cuda_err, sizeof((h)->cuda_err), "%s: %s", #expr, cudaGetErrorString(e_)); \
             return KGE_ERR_CUDA;                                  \
         }                                                         \
     } while (0)
@@ -135,10 +143,20 @@ namespace kge {
         (h)->launches += 1;                                       \
         cudaError_t e_ = cudaGetLastError();                      \
         if (e_ != cudaSuccess) {                                  \
-            (h)->cuda_err = std::string("kernel launch: ") + cudaGetErrorString(e_); \
+            std::snprintf((h)->cuda_err, sizeof((h)->cuda_err), "kernel launch: %s", cudaGetErrorString(e_)); \
             return KGE_ERR_CUDA;                                  \
         }                                                         \
     } while (0)
+
+// Runs `set` (a cudaFuncSetAttribute call) once per device: the attribute belongs to the device
+// that is current when it is set, so a process that uses several GPUs must set it on each.
+template <class F>
+inline cudaError_t once_per_device(DeviceOnce& flags, F&& set) {
+    int dev = -1;
+    const cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    return static_cast<cudaError_t>(flags.run(dev, set));
+}
 
 inline void stage_begin(kge_handle* h, int id, cudaStream_t s) {
     if (h->prof.on) { cudaEventRecord(h->prof.a[id], s); }
@@ -175,6 +193,11 @@ int launch_tc_forward(kge_handle* h, cudaStream_t s);
 int launch_cast_bf16(kge_handle* h, const float* src, uint16_t* dst, int64_t count, cudaStream_t s);
 int launch_tc_infer_chunk(kge_handle* h, int nq, int64_t e_lo, int64_t e_hi, const int32_t* true_tails, cudaStream_t s);
 int dedup_tiles(int n);     // sort tiles of a list of n ids
+// On-device graph preprocessing and table initialisation (kge_graph.cu).
+size_t graph_hist_words(int64_t num_triples);
+int launch_graph_build_device(kge_handle* h, const int32_t* heads, const int32_t* rels, const int32_t* tails, int64_t n,
+                              cudaStream_t s);
+int launch_init_table(kge_handle* h, float* out, int64_t rows, int width, float std, int kind, uint32_t stream_id, cudaStream_t s);
 int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int32_t nq, int32_t k,
                        const int32_t* true_tails, int32_t* out_ids, float* out_scores, int32_t* out_ranks,
                        cudaStream_t s);
@@ -227,10 +250,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, ui
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns) : "memory");
     return ok != 0;
 }
-// Waits for the barrier phase `parity` a bounded number of times (each up to the hint above,
-// then a short sleep: seconds in all); false = gave up.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-    for (int i = 0; i < (1 << 20); ++i) {
+// Waits for the barrier phase `parity` at most `limit` times (each up to the hint above, then a
+// short sleep: seconds in all at the default limit); false = gave up.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, int limit) {
+    for (int i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (i > 16) __nanosleep(256);
     }

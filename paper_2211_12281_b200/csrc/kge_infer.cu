@@ -27,6 +27,7 @@ struct InferParams {
     const int32_t *qh, *qr, *tt;   // tt may be NULL
     int64_t e_lo, e_hi;            // entity range of this launch
     int q_tiles;
+    int wait_limit;                // tries of a bounded barrier wait
     Workspace w;
 };
 
@@ -321,11 +322,11 @@ __global__ void __launch_bounds__(256) score_tile_tma_kernel(InferParams p) {
 
     for (int chunk = 0; chunk < nchunk; ++chunk) {
         const int stage = chunk % nstage;
-        const bool ok = mbar_wait_bounded(&bars[stage], (uint32_t)(chunk / nstage) & 1u);
+        const bool ok = mbar_wait_bounded(&bars[stage], (uint32_t)(chunk / nstage) & 1u, p.wait_limit);
         if (!__syncthreads_and(ok)) {
             if (tid == 0) set_status(p.w.status, KGE_ERR_TIMEOUT);
             // give copies still in flight a bounded chance to land before shared memory is released
-            for (int st = 0; st < nstage; ++st) (void)mbar_wait_bounded(&bars[st], (uint32_t)(chunk / nstage) & 1u);
+            for (int st = 0; st < nstage; ++st) (void)mbar_wait_bounded(&bars[st], (uint32_t)(chunk / nstage) & 1u, p.wait_limit);
             return;
         }
         const float* Qs = base + (size_t)stage * ROWS * ld;
@@ -354,13 +355,11 @@ __global__ void __launch_bounds__(256) score_tile_tma_kernel(InferParams p) {
 
 template <int KIND>
 cudaError_t launch_score_tile_tma(const InferParams& p, unsigned grid, cudaStream_t s) {
-    static bool configured = false;
-    if (!configured) {
-        const cudaError_t e = cudaFuncSetAttribute(score_tile_tma_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)infer_tma_smem(kMaxDim));
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static DeviceOnce configured;
+    const cudaError_t e = once_per_device(configured, [] {
+        return cudaFuncSetAttribute(score_tile_tma_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)infer_tma_smem(kMaxDim));
+    });
+    if (e != cudaSuccess) return e;
     score_tile_tma_kernel<KIND><<<grid, 256, infer_tma_smem(p.d), s>>>(p);
     return cudaSuccess;
 }
@@ -468,6 +467,7 @@ int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int3
     p.ent = h->ent; p.rel = h->rel; p.relw = h->relw;
     p.qh = qh; p.qr = qr; p.tt = true_tails;
     p.q_tiles = (nq + IQ - 1) / IQ;
+    p.wait_limit = h->wait_limit;
     p.w = h->ws;
     p.e_lo = 0; p.e_hi = 0;
     const int qblocks = (nq + 127) / 128;
@@ -566,7 +566,7 @@ extern "C" int kge_score_all_topk_static(const kge_config* cfg, const float* ent
     if (nq > kStaticMaxQueries || k > kStaticMaxTopk || c.dim > kMaxDim) return KGE_ERR_WORKSPACE;
     if (nq == 0) return KGE_OK;
 
-    kge_handle h;                       // plain host object on the stack; nothing in it is heap-backed here
+    kge_handle h{};                     // plain host object on the stack, every field zero; nothing in it is heap-backed
     h.cfg = c;
     h.kw = c.score == KGE_ROTATE ? c.dim / 2 : c.dim;
     h.kind = kind_of(c);
@@ -574,6 +574,9 @@ extern "C" int kge_score_all_topk_static(const kge_config* cfg, const float* ent
     h.ent_state = h.rel_state = h.relw_state = nullptr;
     h.launches = 0; h.bound = true; h.graph_loaded = false;
     h.max_queries = kStaticMaxQueries; h.topk = kStaticMaxTopk;
+    h.num_sms = 148; h.split_q = h.split_t = 1; h.num_triples = 0;
+    h.ws_base = nullptr; h.ws_bytes = 0; h.streams_ready = false;
+    h.wait_limit = kDefaultWaitLimit; h.capture_scores = nullptr;
 
     // Set-up, once per device and with that device current: in host code the array's name is
     // only a stand-in, so its device address has to be asked for.
@@ -615,5 +618,5 @@ extern "C" int kge_score_all_topk_static(const kge_config* cfg, const float* ent
     int32_t word = 0;
     KGE_CUDA_CHECK(&h, cudaMemcpyAsync(&word, w.status, 4, cudaMemcpyDeviceToHost, s));
     KGE_CUDA_CHECK(&h, cudaStreamSynchronize(s));
-    return word;   // 0, or the code a kernel recorded (an id outside its table)
+    return word;   // 0, or the code a kernel recorded (an id outside its table, a bounded wait that ran out)
 }

@@ -54,6 +54,7 @@ struct TcGemmParams {
     int64_t split_stride;                 // floats between the output slabs of consecutive K splits
     const float *row_norm2, *col_norm2;   // norm expansion: |q_b|^2 [M], |t_n|^2 [N]
     int32_t* status;
+    int wait_limit;                       // tries of a bounded barrier wait
     // fused loss epilogues (EPI_STATS, EPI_GRAD): the score is acc, or for l2 != 0 the distance score above
     int l2, loss;
     float gamma, adv_temp, ce_c, loss_scale;
@@ -468,12 +469,17 @@ __device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem&
     }
     if ((EPI & 3) == EPI_TOPK) { tc_epilogue_topk<WIDTH>(p, it, row, col_off, taddr, beat_sm); return; }
     float* const Cout = p.C + (int64_t)it.z * p.split_stride;
+    const float rn = ((EPI & EPI_L2) && row < p.M) ? p.row_norm2[row] : 0.f;
 #pragma unroll 1
     for (int c0 = col_off; c0 < col_off + WIDTH; c0 += 32) {
         float v[32];
         tmem_ld32(taddr + (uint32_t)(c0 - col_off), v);
         if (row >= p.M) continue;
         const int ncol = it.n0 + c0;
+        if (EPI & EPI_L2) {   // the debug tap of the score block: the distance score of the norm expansion, as the fused epilogues form it
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = ncol + i < p.N ? tc_score<true>(p, v[i], rn, ncol + i) : 0.f;
+        }
         float* dst = Cout + (int64_t)row * p.ldc + ncol;
         if (ncol + 32 <= p.N && (p.ldc & 3) == 0) {
 #pragma unroll
@@ -553,7 +559,7 @@ __global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __gri
                 const int kb0 = it.z * p.kb_per_split, nkb = min(p.kb_per_split, kb_total - kb0);
                 for (int kb = 0; kb < nkb; ++kb, ++ring) {
                     const int s = ring % TC_STAGES;
-                    if (!mbar_wait_bounded(&empty[s], ((ring / TC_STAGES) & 1) ^ 1)) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); break; }
+                    if (!mbar_wait_bounded(&empty[s], ((ring / TC_STAGES) & 1) ^ 1, p.wait_limit)) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); break; }
                     unsigned char* sa = base + (size_t)s * TC_STAGE_BYTES;
                     const int shared_at = p.m_fastest ? it.n0 : it.m0;
                     bool have = false;
@@ -592,12 +598,12 @@ __global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __gri
                 const int nkb = min(p.kb_per_split, kb_total - it.z * p.kb_per_split);
                 const int buf = local % NACC;
                 // the epilogue warps must have drained this buffer (two items ago)
-                if (!mbar_wait_bounded(&acc_empty[buf], ((local / NACC) & 1) ^ 1)) { ok = false; break; }
+                if (!mbar_wait_bounded(&acc_empty[buf], ((local / NACC) & 1) ^ 1, p.wait_limit)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_acc = tmem_base + (uint32_t)buf * BN;
                 for (int kb = 0; kb < nkb; ++kb, ++ring) {
                     const int s = ring % TC_STAGES;
-                    if (!mbar_wait_bounded(&full[s], (ring / TC_STAGES) & 1)) { ok = false; break; }
+                    if (!mbar_wait_bounded(&full[s], (ring / TC_STAGES) & 1, p.wait_limit)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = smem_u32(base + (size_t)s * TC_STAGE_BYTES);
 #pragma unroll
@@ -617,7 +623,7 @@ __global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __gri
         const int cgrp = (warp - 2) >> 2;              // which group of the tile's columns
         for (int item = item_begin, local = 0; item < item_end; ++item, ++local) {
             const int buf = local % NACC;
-            const bool ok = mbar_wait_bounded(&acc_full[buf], (local / NACC) & 1);
+            const bool ok = mbar_wait_bounded(&acc_full[buf], (local / NACC) & 1, p.wait_limit);
             tc_fence_after();
             if (!ok || *stop) { if (lane == 0) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); } break; }
             const TcItem it = tc_item(p, item);
@@ -662,7 +668,7 @@ EncodeTiledFn encode_tiled_fn() {
 // matrix reads as zero.
 int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
     EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) { h->cuda_err = "cuTensorMapEncodeTiled is not available from this driver"; return KGE_ERR_CUDA; }
+    if (!fn) { std::snprintf(h->cuda_err, sizeof(h->cuda_err), "cuTensorMapEncodeTiled is not available from this driver"); return KGE_ERR_CUDA; }
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
     const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
@@ -670,7 +676,7 @@ int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t 
     const CUresult r = fn(static_cast<CUtensorMap*>(map_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
                           dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) { h->cuda_err = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r); return KGE_ERR_CUDA; }
+    if (r != CUDA_SUCCESS) { std::snprintf(h->cuda_err, sizeof(h->cuda_err), "cuTensorMapEncodeTiled failed with code %d", (int)r); return KGE_ERR_CUDA; }
     return KGE_OK;
 }
 
@@ -746,13 +752,11 @@ cudaError_t launch_gemm_inst(const unsigned char* tmA, const unsigned char* tmB,
     constexpr size_t extra_max = (EPI & 3) == EPI_TOPK ? (size_t)TC_BEAT_ROWS_MAX * 4
                                : ((EPI & 3) == EPI_GRAD ? (size_t)tc_epi_warps(EPI) * TC_GRAD_STAGE_BYTES : 0);
     if ((EPI & 3) == EPI_GRAD) extra_smem = extra_max;
-    static bool configured = false;
-    if (!configured) {
-        const cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<EPI, BN, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)(smem + extra_max));
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static DeviceOnce configured;
+    const cudaError_t e = once_per_device(configured, [] {
+        return cudaFuncSetAttribute(tc_gemm_kernel<EPI, BN, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(smem + extra_max));
+    });
+    if (e != cudaSuccess) return e;
     tc_gemm_kernel<EPI, BN, A_MN, B_MN><<<std::min(p.items, num_sms), tc_threads(EPI), smem + extra_smem, s>>>(
         *reinterpret_cast<const CUtensorMap*>(tmA), *reinterpret_cast<const CUtensorMap*>(tmB), p);
     return cudaSuccess;
@@ -794,13 +798,23 @@ int launch_tc_forward(kge_handle* h, cudaStream_t s) {
     p.row_pieces = TC_EPI_GROUPS * ((p.N + TC_BN - 1) / TC_BN);
     p.C = nullptr; p.ldc = 0;
     p.row_norm2 = w.qn2; p.col_norm2 = w.tn2;
-    p.status = w.status;
+    p.status = w.status; p.wait_limit = h->wait_limit;
     p.l2 = h->kind == KIND_L2; p.loss = c.loss;
     p.gamma = c.gamma; p.adv_temp = c.adv_temp; p.ce_c = c.ce_correction; p.loss_scale = c.loss_scale;
     p.stat_part = reinterpret_cast<float4*>(w.stat_part); p.row_stat = reinterpret_cast<const float2*>(w.row_stat);
     p.Gb = w.Gb; p.ldg = (c.num_neg + 7) / 8 * 8;
     p.grow_part = w.grow_part; p.gcol_part = w.gcol_part;
     const bool ce = c.loss == KGE_LOSS_SAMPLED_SOFTMAX;
+    if (h->capture_scores) {
+        // debug tap: this path never stores the score block, so an extra contraction writes it (fp32 [B, N]) with the
+        // same mainloop and, for the norm expansion, the same score formula as the fused epilogues
+        TcGemmParams cp = p;
+        cp.bn = TC_BN; cp.tiles_n = (p.N + TC_BN - 1) / TC_BN; cp.items = cp.tiles_m * cp.tiles_n;
+        cp.C = h->capture_scores; cp.ldc = p.N;
+        if (p.l2) KGE_CUDA_CHECK(h, (launch_gemm_inst<EPI_STORE | EPI_L2, 128>(h->tm_q, h->tm_t, cp, h->num_sms, s)));
+        else KGE_CUDA_CHECK(h, (launch_gemm_inst<EPI_STORE, 128>(h->tm_q, h->tm_t, cp, h->num_sms, s)));
+        KGE_LAUNCH_CHECK(h);
+    }
     stage_begin(h, ST_BLOCK, s);
     KGE_CUDA_CHECK(h, launch_fused(EPI_STATS, p.l2 != 0, ce, h, p, s));
     stage_end(h, ST_BLOCK, s);
@@ -831,7 +845,7 @@ int launch_tc_bwd_gemm(kge_handle* h, const unsigned char* tmA, const unsigned c
     const int kb = (K + TC_BK - 1) / TC_BK;
     p.kb_per_split = (kb + split - 1) / split;
     p.C = C; p.ldc = ldc; p.split_stride = (int64_t)M * ldc;
-    p.status = h->ws.status;
+    p.status = h->ws.status; p.wait_limit = h->wait_limit;
     p.bn = tc_backward_tile_cols(N);
     p.tiles_m = (M + TC_BM - 1) / TC_BM; p.tiles_n = (N + p.bn - 1) / p.bn;
     p.items = p.tiles_m * p.tiles_n * ((kb + p.kb_per_split - 1) / p.kb_per_split);
@@ -907,7 +921,7 @@ int launch_tc_infer_chunk(kge_handle* h, int nq, int64_t e_lo, int64_t e_hi, con
     p.tiles_m = (p.M + TC_BM - 1) / TC_BM; p.tiles_n = (p.N + p.bn - 1) / p.bn;
     if ((int64_t)p.tiles_m * p.tiles_n > 0x7fffffff) return KGE_ERR_BAD_ARG;
     p.items = p.tiles_m * p.tiles_n;
-    p.status = w.status;
+    p.status = w.status; p.wait_limit = h->wait_limit;
     p.m_fastest = 1; p.n_base = e_lo;
     p.thr = w.thr; p.thr_id = w.thr_id; p.ftrue = w.iftrue; p.tt = true_tails;
     p.cand_cnt = w.cand_cnt; p.beat_tmp = w.beat_tmp; p.cand_score = w.cand_score; p.cand_id = w.cand_id;

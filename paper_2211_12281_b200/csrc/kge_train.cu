@@ -26,6 +26,7 @@ struct TrainParams {
     SampleParams sp;
     int tc_l2;          // TransE p = 2 with tensor-core backward: the splits hold C.T and C^T.Q, C = dL/dF / distance
     int neg_direct;     // the dT contraction wrote the negatives' gradient rows itself (one K split, no correction term)
+    int wait_limit;     // tries of a bounded barrier wait
     Workspace w;
 };
 
@@ -38,7 +39,11 @@ __device__ __forceinline__ float4 f4fma(float s, float4 a, float4 c) {
     return make_float4(fmaf(s, a.x, c.x), fmaf(s, a.y, c.y), fmaf(s, a.z, c.z), fmaf(s, a.w, c.w));
 }
 __device__ __forceinline__ float f4dot(float4 a, float4 b) { return a.x * b.x + a.y * b.y + a.z * b.z + a.w * b.w; }
-__device__ __forceinline__ float sgnf(float x) { return (x > 0.f ? 1.f : 0.f) - (x < 0.f ? 1.f : 0.f); }
+// The sub-gradient of |x| that every p = 1 kernel of this library uses: +1 for x > 0, -1 otherwise.
+// At x == 0 any value in [-1, 1] is a sub-gradient; the score-block backward counts the pairs with
+// x > 0 (see add_if_pos), which fixes -1 there, and the positive pair takes the same value so that
+// a step has one convention.
+__device__ __forceinline__ float sgnf(float x) { return x > 0.f ? 1.f : -1.f; }
 __device__ __forceinline__ float4 f4sgn(float4 a) { return make_float4(sgnf(a.x), sgnf(a.y), sgnf(a.z), sgnf(a.w)); }
 // Four floats rounded to bf16 (nearest even), packed in memory order.
 __device__ __forceinline__ uint2 pack_bf16x4(float4 v) {
@@ -243,7 +248,7 @@ __device__ __forceinline__ void pair_update(float& acc, float4 q, float4 t) {
 
 // acc += w where x > 0: one compare and one predicated add (two adds sharing the compare in the
 // second form).  With sign(x) = 2 [x > 0] - 1 a sum of w sign(x) is 2 P - (sum of w), P the sum
-// these accumulate; the value at x == 0 is a free choice of sub-gradient of |x| (here -1).
+// these accumulate; the value at x == 0 is a free choice of sub-gradient of |x| (-1: see sgnf).
 __device__ __forceinline__ void add_if_pos(float& acc, float x, float w) {
     asm("{\n .reg .pred p;\n setp.gt.f32 p, %1, 0f00000000;\n @p add.f32 %0, %0, %2;\n}\n" : "+f"(acc) : "f"(x), "f"(w));
 }
@@ -429,11 +434,11 @@ __global__ void __launch_bounds__(FTHREADS) block_tma_kernel(TrainParams p) {
 
     for (int chunk = 0; chunk < nchunk; ++chunk) {
         const int stage = chunk % nstage;
-        const bool ok = mbar_wait_bounded(&bars[stage], (uint32_t)(chunk / nstage) & 1u);
+        const bool ok = mbar_wait_bounded(&bars[stage], (uint32_t)(chunk / nstage) & 1u, p.wait_limit);
         if (!__syncthreads_and(ok)) {
             if (tid == 0) set_status(p.w.status, KGE_ERR_TIMEOUT);
             // give copies still in flight a bounded chance to land before shared memory is released
-            for (int st = 0; st < nstage; ++st) (void)mbar_wait_bounded(&bars[st], (uint32_t)(chunk / nstage) & 1u);
+            for (int st = 0; st < nstage; ++st) (void)mbar_wait_bounded(&bars[st], (uint32_t)(chunk / nstage) & 1u, p.wait_limit);
             return;
         }
         const float* Qs = base + (size_t)stage * ROWS * ld;
@@ -713,6 +718,7 @@ struct AccArgs {
     float *out, *out2;          // [split, own_rows, d]; out2: TransH normal gradient (OWNER_Q)
     float *csum;                // [split, own_rows] weight sums per owner row (TransE p = 1, owner = negatives)
     int32_t* status;
+    int wait_limit;             // tries of a bounded barrier wait
 };
 
 constexpr int ACC_ROWS = 32, ACC_CC = 32, ACC_LDW = 36;
@@ -721,11 +727,11 @@ template <int KIND>
 __device__ __forceinline__ void acc_update(float4& acc, float4 a, float4 b, float w) {
     if (KIND == KIND_DOT) {
         acc = f4fma(w, b, acc);
-    } else if (KIND == KIND_L1) {  // acc -= w * sign(a - b)
-        acc.x += (a.x < b.x ? w : 0.f) - (a.x > b.x ? w : 0.f);
-        acc.y += (a.y < b.y ? w : 0.f) - (a.y > b.y ? w : 0.f);
-        acc.z += (a.z < b.z ? w : 0.f) - (a.z > b.z ? w : 0.f);
-        acc.w += (a.w < b.w ? w : 0.f) - (a.w > b.w ? w : 0.f);
+    } else if (KIND == KIND_L1) {  // acc -= w * sign(a - b), sign as in sgnf
+        acc.x += a.x > b.x ? -w : w;
+        acc.y += a.y > b.y ? -w : w;
+        acc.z += a.z > b.z ? -w : w;
+        acc.w += a.w > b.w ? -w : w;
     } else if (KIND == KIND_L2) {  // w already holds G / distance
         acc = f4fma(w, f4sub(b, a), acc);
     } else {                       // KIND_CL1: acc -= w * (a - b) / |a - b| per complex component
@@ -878,8 +884,8 @@ __global__ void __launch_bounds__(256) accum_kernel(AccArgs a) {
 // of the next chunk is prefetched through registers while the current chunk is consumed.
 //
 // TransE p = 1: the term is w * sign(q - t).  Writing sign = 2 [q > t] - 1 (the value at an
-// exact tie is a free choice of sub-gradient of |x| at 0; this kernel takes -1, the positive
-// pair in the chain kernel takes 0), the sum becomes 2 P - (sum of the weights) with
+// exact tie is a free choice of sub-gradient of |x| at 0; the whole step takes -1, see sgnf),
+// the sum becomes 2 P - (sum of the weights) with
 // P = sum of w over the pairs with q > t: one compare and one predicated add per element.
 // The kernel accumulates P; the weight sums come from the loss kernel (rows) and from this
 // kernel's own pass over the weight tiles (columns, OWNER_Q = false).
@@ -983,10 +989,10 @@ __device__ __forceinline__ void accum_tma_body(const AccArgs& a, const int block
             if (tid == 0) issue_rows(chunk + 1, cur ^ 1);
             load_weights(chunk + 1);
         }
-        const bool ok = mbar_wait_bounded(&bars[cur], (uint32_t)(chunk >> 1) & 1u);
+        const bool ok = mbar_wait_bounded(&bars[cur], (uint32_t)(chunk >> 1) & 1u, a.wait_limit);
         if (!__syncthreads_and(ok)) {
             if (tid == 0) set_status(a.status, KGE_ERR_TIMEOUT);
-            (void)mbar_wait_bounded(&bars[cur ^ 1], (uint32_t)((chunk + 1) >> 1) & 1u);
+            (void)mbar_wait_bounded(&bars[cur ^ 1], (uint32_t)((chunk + 1) >> 1) & 1u, a.wait_limit);
             return;
         }
         const int ccmax = min(ACC_CC, c_end - (c_begin + chunk * ACC_CC));
@@ -1287,13 +1293,11 @@ void launch_block(const TrainParams& p, cudaStream_t s) {
 template <int KIND>
 cudaError_t launch_block_tma(const TrainParams& p, cudaStream_t s) {
     const size_t smem = block_tma_smem(p.d);
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(block_tma_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)block_tma_smem(kMaxDim));
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static DeviceOnce configured;
+    const cudaError_t e = once_per_device(configured, [] {
+        return cudaFuncSetAttribute(block_tma_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)block_tma_smem(kMaxDim));
+    });
+    if (e != cudaSuccess) return e;
     dim3 grid((p.N + TN - 1) / TN, (p.B + FTQ - 1) / FTQ);
     return launch_dependent(block_tma_kernel<KIND>, grid, dim3(FTHREADS), smem, s, p);
 }
@@ -1302,13 +1306,12 @@ template <int KIND, int NCH>
 cudaError_t launch_accum_tma_inst(const AccArgs& aq, const AccArgs& at, cudaStream_t s) {
     constexpr int WARPS = NCH == 4 ? 8 : 4;
     const size_t smem = accum_tma_smem(aq.d4);
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(accum_tma_kernel<KIND, NCH, WARPS>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)accum_tma_smem(kMaxDim / 4));
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static DeviceOnce configured;
+    const cudaError_t e = once_per_device(configured, [] {
+        return cudaFuncSetAttribute(accum_tma_kernel<KIND, NCH, WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)accum_tma_smem(kMaxDim / 4));
+    });
+    if (e != cudaSuccess) return e;
     dim3 grid((std::max(aq.own_rows, at.own_rows) + ACC_ROWS - 1) / ACC_ROWS, std::max(aq.split, at.split), 2);
     return launch_dependent(accum_tma_kernel<KIND, NCH, WARPS>, grid, dim3(32 * WARPS), smem, s, aq, at);
 }
@@ -1334,13 +1337,11 @@ cudaError_t launch_accum_tma(int kind, const AccArgs& aq, const AccArgs& at, cud
 template <int KIND, int NCH, bool OWNER_Q>
 cudaError_t launch_accum_inst(const AccArgs& a, cudaStream_t s) {
     const size_t smem = (size_t)ACC_CC * a.d4 * 16 * (OWNER_Q ? 1 : 2) + (size_t)ACC_CC * ACC_LDW * 4 * 3;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(accum_kernel<KIND, NCH, OWNER_Q>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static DeviceOnce configured;
+    const cudaError_t e = once_per_device(configured, [] {
+        return cudaFuncSetAttribute(accum_kernel<KIND, NCH, OWNER_Q>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    });
+    if (e != cudaSuccess) return e;
     dim3 grid((a.own_rows + ACC_ROWS - 1) / ACC_ROWS, a.split);
     accum_kernel<KIND, NCH, OWNER_Q><<<grid, 256, smem, s>>>(a);
     return cudaSuccess;
@@ -1380,6 +1381,7 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     p.slots_per_bucket = c.batch / (c.head_part < 0 ? c.num_parts * c.num_parts : c.num_parts);
     p.tc_l2 = c.prec == KGE_PREC_BF16_TC && p.kind == KIND_L2;
     p.neg_direct = tc_negatives_direct(h) ? 1 : 0;
+    p.wait_limit = h->wait_limit;
     p.w = h->ws;
     const int nch = p.d4 <= 32 ? 1 : (p.d4 <= 64 ? 2 : 4);
 
@@ -1418,16 +1420,17 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     }
     stage_end(h, ST_BLOCK, s);
     KGE_LAUNCH_CHECK(h);
+    if (h->capture_scores)   // debug tap: the loss kernel is about to overwrite the scores in place
+        KGE_CUDA_CHECK(h, cudaMemcpyAsync(h->capture_scores, p.w.F, (size_t)p.B * p.N * sizeof(float), cudaMemcpyDeviceToDevice, s));
     stage_begin(h, ST_LOSS, s);
     {
-        static bool configured = false;
-        if (!configured) {
-            KGE_CUDA_CHECK(h, cudaFuncSetAttribute(loss_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   LOSS_SMEM_FLOATS * 4));
-            KGE_CUDA_CHECK(h, cudaFuncSetAttribute(loss_warp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   LOSS_THREADS / 32 * LOSS_WARP_MAX_N * 4));
-            configured = true;
-        }
+        static DeviceOnce configured;
+        KGE_CUDA_CHECK(h, once_per_device(configured, [] {
+            const cudaError_t e = cudaFuncSetAttribute(loss_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, LOSS_SMEM_FLOATS * 4);
+            if (e != cudaSuccess) return e;
+            return cudaFuncSetAttribute(loss_warp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        LOSS_THREADS / 32 * LOSS_WARP_MAX_N * 4);
+        }));
     }
     // rows of 256 / 512 / 1024 scores in registers, 2 / 4 / 4 warps per row (one warp per row leaves most of the SM idle:
     // 80 -> 75.5 us per step at B = N = 1024)
@@ -1458,7 +1461,7 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     AccArgs aq;
     aq.own = p.w.Q; aq.oth = p.w.Tneg; aq.what = p.w.What; aq.G = p.w.F; aq.U = p.w.U; aq.Cc = p.w.Cc;
     aq.own_rows = p.B; aq.oth_rows = p.N; aq.N = p.N; aq.d4 = p.d4; aq.split = p.split_q;
-    aq.out = p.w.dQpart; aq.out2 = p.w.dWpart; aq.csum = nullptr; aq.status = p.w.status;
+    aq.out = p.w.dQpart; aq.out2 = p.w.dWpart; aq.csum = nullptr; aq.status = p.w.status; aq.wait_limit = h->wait_limit;
     AccArgs at = aq;
     at.own = p.w.Tneg; at.oth = p.w.Q; at.own_rows = p.N; at.oth_rows = p.B; at.split = p.split_t;
     at.out = p.w.dTpart; at.out2 = nullptr; at.csum = p.w.Cpart;

@@ -22,3 +22,10 @@ def oracle64():
 def oracle32():
     from oracle.kge_oracle import Oracle
     return Oracle("f32")
+
+
+@pytest.fixture(scope="session")
+def oracle64_tie():
+    """The fp64 oracle built with sign(0) = -1 as the sub-gradient of |x| at an exact tie."""
+    from oracle.kge_oracle import Oracle
+    return Oracle("f64_tie")

@@ -71,3 +71,34 @@ def test_missing_library_fails_loudly(K, monkeypatch, tmp_path):
     with pytest.raises(K.KgeError) as e:
         binding.lib()
     assert e.value.code == binding.KGE_ERR_NO_EXTENSION
+
+
+def test_per_device_once_bookkeeping(tmp_path):
+    """Settings that CUDA keeps per device (a kernel's opt-in to large dynamic shared memory) are applied
+    once per device ordinal, not once per process: exercised on the host with made-up ordinals."""
+    import subprocess
+    src = tmp_path / "once.cpp"
+    src.write_text(r"""
+#include <cassert>
+#include "kge_device_once.h"
+int main() {
+    kge::DeviceOnce once;
+    int calls = 0;
+    auto ok = [&] { ++calls; return 0; };
+    auto fail = [&] { ++calls; return 7; };
+    assert(once.run(0, ok) == 0 && calls == 1);
+    assert(once.run(0, ok) == 0 && calls == 1);          // device 0 is configured: not again
+    assert(once.run(1, ok) == 0 && calls == 2);          // a second GPU of the same process gets its own call
+    assert(once.run(1, ok) == 0 && calls == 2);
+    assert(once.run(2, fail) == 7 && calls == 3);        // a failure is reported and not remembered
+    assert(once.run(2, ok) == 0 && calls == 4);
+    assert(once.run(kge::kMaxDevices, ok) == 0 && once.run(kge::kMaxDevices, ok) == 0 && calls == 6);   // beyond the table: every time
+    assert(once.run(-1, ok) == 0 && calls == 7);
+    kge::DeviceOnce other;                               // another kernel's flags are independent
+    assert(other.run(0, ok) == 0 && calls == 8);
+    return 0;
+}
+""")
+    exe = tmp_path / "once"
+    subprocess.run(["g++", "-std=c++17", "-I", str(ROOT / "paper_2211_12281_b200" / "csrc"), str(src), "-o", str(exe)], check=True)
+    assert subprocess.run([str(exe)]).returncode == 0

@@ -52,6 +52,11 @@ def test_topk_rank_mrr_against_fp32_oracle(oracle32, oracle64, score, p):
     assert abs(mrr - oracle64.mrr(o_ranks, 10)) <= 1e-3
     mrr0 = gpu.kge.eval_mrr(gpu.dev_i32(qh), gpu.dev_i32(qr), gpu.dev_i32(tt), 0)
     assert abs(mrr0 - oracle64.mrr(o_ranks, 0)) <= 1e-3
+    # the same metric from ranks the caller already holds (no second pass over the table)
+    ranks_dev = gpu.dev_i32(ranks)
+    assert gpu.kge.mrr_from_ranks(ranks_dev, 10) == mrr and gpu.kge.mrr_from_ranks(ranks_dev, 0) == mrr0
+    if score != "rotate":
+        assert abs(mrr - oracle64.mrr(o_ranks, 10)) <= 1e-12 and abs(mrr0 - oracle64.mrr(o_ranks, 0)) <= 1e-12
 
 
 @pytest.mark.parametrize("score", ["distmult", "complex"])

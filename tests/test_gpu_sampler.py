@@ -30,6 +30,19 @@ def test_sampled_indices_bit_exact(oracle64, name):
     assert gpu.kge.get_status() == 0
 
 
+@pytest.mark.parametrize("name", ["c2", "ragged_head2", "c1"])
+def test_step_that_samples_its_own_batch_uses_the_oracles_batch(oracle64, name):
+    """kge_train_step with no ids draws the batch inside its gather kernel (the cumulative weights of a
+    bucket staged per thread block): at the headline shape (R = 500 weights per bucket, B = N = 1,024) and
+    with a fixed head partition and a ragged last shard the ids it used are the oracle's, bit for bit."""
+    prob = Problem(**CASES[name])
+    gpu, orc = GpuSide(prob), OracleSide(prob, oracle64)
+    for step in (0, 1, 7, 2**32 + 5):
+        gpu.kge.train_step(step, 0.01)
+        assert (gpu.kge.debug_export("BATCH") == np.concatenate(orc.sample(step))).all(), (name, step)
+    assert gpu.kge.get_status() == 0
+
+
 def test_graph_load_reports_empty_bucket_and_bad_ids():
     import paper_2211_12281_b200 as K
     prob = Problem(E=40, R=5, T=4, d=16, score="transe", B=8, N=4, P=2)

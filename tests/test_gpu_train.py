@@ -14,7 +14,7 @@ MODELS = [("transe", 1), ("transe", 2), ("transh", 1), ("transh", 2), ("rotate",
           ("distmult", 1), ("complex", 1)]
 
 
-def _check_step(gpu, orc, step, batch, *, taps=True, rows_atol=2e-6):
+def _check_step(gpu, orc, step, batch, *, taps=True, rows_atol=2e-6, warm_adam=False):
     prob = gpu.prob
     B, N, d = prob.B, prob.N, prob.d
     # tensor-core path: the scores come from bf16-rounded operands (matched by the oracle, so dL/dF
@@ -35,12 +35,27 @@ def _check_step(gpu, orc, step, batch, *, taps=True, rows_atol=2e-6):
     loss_dev = gpu.torch.zeros(1, dtype=gpu.torch.float32, device=gpu.ent.device)
     want = orc.grads(batch) if taps else None
     grads_for_adam = (want or orc.grads(batch)) if prob.opt == "adam" else None
+    fwd = orc.o.batch_loss(orc.cfg, orc.ent, orc.rel, orc.relw, *batch) if taps else None     # at the pre-step tables
+    qvec = None
+    if taps:
+        wrow = lambda b: None if orc.relw is None else orc.relw[batch[1][b]]
+        qvec = np.stack([orc.o.query_vector(prob.score, orc.ent[batch[0][b]], orc.rel[batch[1][b]], wrow(b)) for b in range(B)])
+        scores_dev = gpu.torch.full((B, N), float("nan"), dtype=gpu.torch.float32, device=gpu.ent.device)
+        gpu.kge.debug_capture_scores(scores_dev)
     gpu.kge.train_step(step, prob.lr, *dev, loss_out=loss_dev)
+    gpu.kge.debug_capture_scores(None)
     assert gpu.kge.get_status() == 0
     loss_o = orc.step(step, batch)
     assert_close(loss_dev.item(), loss_o, atol=1e-5, what="loss")
     if taps:
         kge = gpu.kge
+        # forward taps, element by element: per-query vectors, positive scores, the B x N score block, per-positive loss.
+        # Relative 1e-4; the absolute term covers values that are cancelling sums of d products of O(1 / d) terms
+        # (the tensor-core block: the same operand rounding on both sides, another accumulation order).
+        assert_close(kge.debug_export("Q").reshape(B, d), qvec, atol=2e-6, what="Q")
+        assert_close(kge.debug_export("FPOS"), fwd["fpos"], atol=2e-6, what="positive scores")
+        assert_close(scores_dev.cpu().numpy(), fwd["F"], atol=2e-6, what="score block F")
+        assert_close(kge.debug_export("LROW"), fwd["Lrow"], atol=1e-5, what="per-positive loss")
         l2 = prob.kw["p_norm"] == 2 and prob.score in ("transe", "transh", "rotate")
         G = kge.debug_export("G").reshape(B, N)
         if l2:   # the tap holds dL/dF divided by the distance; undo with the oracle's distances
@@ -69,7 +84,7 @@ def _check_step(gpu, orc, step, batch, *, taps=True, rows_atol=2e-6):
             assert (kge.debug_export(pre + "_PERM") == perm).all()
     ent, rel, relw = gpu.tables()
     if prob.opt == "adam":
-        _check_adam_tables(prob, batch, grads_for_adam, (ent, rel, relw), (orc.ent, orc.rel, orc.relw), rows_atol)
+        _check_adam_tables(prob, batch, grads_for_adam, (ent, rel, relw), (orc.ent, orc.rel, orc.relw), rows_atol, warm=warm_adam)
     else:
         assert_close(ent, orc.ent, atol=rows_atol, what="entity table")
         assert_close(rel, orc.rel, atol=rows_atol, what="relation table")
@@ -81,7 +96,7 @@ def _check_step(gpu, orc, step, batch, *, taps=True, rows_atol=2e-6):
             assert_close(got.cpu().numpy(), want_s, atol=2e-5 * float(np.abs(want_s).max()) + 1e-12, what=name)
 
 
-def _check_adam_tables(prob, batch, g, got, want, rows_atol):
+def _check_adam_tables(prob, batch, g, got, want, rows_atol, warm=False):
     """Adam divides by sqrt(v) + eps, so its step is discontinuous where a gradient
     coordinate is zero: there fp32 rounding noise (1e-9) against the exact zero (the softmax
     probabilities of a row sum to one, so e.g. a TransE-L1 coordinate with every tail on the
@@ -96,6 +111,9 @@ def _check_adam_tables(prob, batch, g, got, want, rows_atol):
         np.add.at(tabs[2], rels, g["dw"])
     for name, gt, a, b in zip(("entity", "relation", "normal"), tabs, got, want):
         if gt is None:
+            continue
+        if warm:     # second moments well away from zero: the step is continuous in g, every coordinate is compared
+            assert_close(a, b, atol=rows_atol, what=name + " table (all coordinates, warm moments)")
             continue
         ill = np.abs(gt) < 1e-4 * np.abs(gt).max()
         a, b = np.asarray(a, np.float64), np.asarray(b, np.float64)
@@ -133,6 +151,95 @@ def test_optimisers_with_state(oracle64, opt, score, p):
     prob = Problem(E=300, R=5, T=10000, d=32, score=score, p_norm=p, loss="softmax", opt=opt, B=64, N=96, P=2,
                    ce_correction=0.1, lr=0.01, graph_seed=4, relation_zipf=1.0)
     _run(oracle64, prob, steps=3, taps=False)
+
+
+@pytest.mark.parametrize("score,p", [("transe", 1), ("complex", 1), ("transh", 2), ("rotate", 1)])
+def test_adam_from_warm_moments_every_coordinate(oracle64, score, p):
+    """Adam's step m^ / (sqrt(v^) + eps) is discontinuous in the gradient only where v is zero (the first
+    time a row is touched).  From moments that are already warm -- here every row starts with second
+    moments of the size of a squared gradient -- the step is continuous, so ALL coordinates of the
+    updated tables and of both moments are held to the normal tolerance, at global steps 2, 3 and 4."""
+    prob = Problem(E=300, R=5, T=10000, d=32, score=score, p_norm=p, loss="softmax", opt="adam", B=64, N=96, P=2,
+                   ce_correction=0.1, lr=0.01, graph_seed=4, relation_zipf=1.0)
+    gpu, orc = GpuSide(prob), OracleSide(prob, oracle64)
+    g0 = orc.grads(orc.sample(0))
+    gs = float(np.sqrt(np.mean(g0["dh"] ** 2))) + 1e-6                  # a typical gradient magnitude
+    rng = np.random.default_rng(9)
+    for st in gpu.states:
+        if st is None:
+            continue
+        w = st.shape[1] // 2
+        init = np.concatenate([rng.standard_normal((st.shape[0], w)) * gs,                  # first moments
+                               rng.uniform(0.5, 1.5, (st.shape[0], w)) * gs * gs], axis=1)   # second moments > 0
+        st.copy_(gpu.torch.from_numpy(init.astype(np.float32)))
+    for step in (2, 3, 4):
+        batch = orc.sample(step)
+        orc.set_tables(*gpu.tables(), states=[None if s is None else s.cpu().numpy() for s in gpu.states])
+        _check_step(gpu, orc, step, batch, taps=False, warm_adam=True)
+
+
+def test_l1_exact_ties_take_one_sub_gradient_everywhere(oracle64, oracle64_tie):
+    """Tables of small integers make q_k = t_k happen in a large share of the (query, negative, coordinate)
+    elements, and for the positive pair too.  |x| has every value in [-1, 1] as a sub-gradient at 0; the
+    oracle's default is 0, the CUDA library takes -1 (the left derivative) in every kernel of the step.
+    Checked coordinate by coordinate: (i) against the oracle build whose sub-gradient at 0 is -1 (TransE
+    and TransH, all gradient rows and the updated tables); (ii) for TransE against the default oracle
+    plus the closed-form difference  d(dh) = +sum over ties of dL/dF,  d(dt) = -sum over ties of dL/dF."""
+    for score in ("transe", "transh"):
+        prob = Problem(E=60, R=4, T=3000, d=16, score=score, p_norm=1, loss="logsigmoid", B=32, N=40, P=2,
+                       gamma=4.0, adv_temp=0.5, lr=0.05, graph_seed=15)
+        rng = np.random.default_rng(15)
+        prob.ent = rng.integers(-2, 3, prob.ent.shape).astype(np.float32)
+        prob.rel = rng.integers(-1, 2, prob.rel.shape).astype(np.float32)
+        if score == "transh":
+            prob.relw = np.zeros_like(prob.relw)
+            prob.relw[np.arange(prob.R), np.arange(prob.R)] = 2.0      # axis-aligned normals: the projection stays in the integers
+        gpu, o_tie, o_def = GpuSide(prob), OracleSide(prob, oracle64_tie), OracleSide(prob, oracle64)
+        batch = o_def.sample(0)
+        batch[2][:8] = batch[0][:8]                                     # a few positives with t = h: the positive pair ties where r = 0
+        B, N, d = prob.B, prob.N, prob.d
+        want, base = o_tie.grads(batch), o_def.grads(batch)
+        fwd = oracle64.batch_loss(o_def.cfg, o_def.ent, o_def.rel, o_def.relw, *batch)
+        gpu.kge.train_step(0, prob.lr, *[gpu.dev_i32(a) for a in batch])
+        assert gpu.kge.get_status() == 0
+        ge = gpu.kge.debug_export("GRAD_ENT").reshape(2 * B + N, d)
+        scale = max(np.abs(want["dh"]).max(), np.abs(want["dtneg"]).max())
+        for got, key in ((ge[:B], "dh"), (ge[B:2 * B], "dtpos"), (ge[2 * B:], "dtneg"),
+                         (gpu.kge.debug_export("GRAD_REL").reshape(B, d), "dr")):
+            assert_close(got, want[key], atol=2e-5 * scale, what=f"{score} {key} against the sign(0) = -1 oracle")
+        if score == "transh":
+            assert_close(gpu.kge.debug_export("GRAD_RELW").reshape(B, d), want["dw"], atol=2e-5 * np.abs(want["dw"]).max(), what="dw")
+            continue
+        q = o_def.ent[batch[0]] + o_def.rel[batch[1]]
+        tie_neg = q[:, None, :] == o_def.ent[batch[3]][None, :, :]              # [B, N, d]
+        tie_pos = q == o_def.ent[batch[2]]
+        assert tie_neg.mean() > 0.1 and tie_pos.sum() > 0
+        G, gpos = base["G"], base["gpos"]
+        d_dh = np.einsum("bn,bnk->bk", G, tie_neg) + gpos[:, None] * tie_pos
+        assert_close(ge[:B], base["dh"] + d_dh, atol=2e-5 * scale, what="dh = default oracle + tie weights")
+        assert_close(ge[B:2 * B], base["dtpos"] - gpos[:, None] * tie_pos, atol=2e-5 * scale, what="dtpos")
+        assert_close(ge[2 * B:], base["dtneg"] - np.einsum("bn,bnk->nk", G, tie_neg), atol=2e-5 * scale, what="dtneg")
+        assert np.abs(d_dh).max() > 100 * 2e-5 * scale                           # the difference is far above the tolerance
+        assert fwd["loss"] > 0
+        o_tie.step(0, batch)
+        assert_close(gpu.tables()[0], o_tie.ent, atol=2e-6, what="entity table")
+        assert_close(gpu.tables()[1], o_tie.rel, atol=2e-6, what="relation table")
+
+
+def test_bounded_wait_runs_out_and_the_context_stays_usable(oracle64):
+    """Every wait of a kernel on an asynchronous copy or a barrier is a bounded loop.  With the limit cut to
+    32 tries, a thread block that waits on a barrier nothing arrives at gives up, records KGE_ERR_TIMEOUT
+    (-11) and returns; the status clears, and a normal step on the same handle then runs clean."""
+    prob = Problem(E=500, R=7, T=20000, d=32, score="transe", p_norm=1, B=64, N=64, P=2, gamma=6.0, lr=0.05)
+    gpu, orc = GpuSide(prob), OracleSide(prob, oracle64)
+    gpu.kge.debug_set_wait_limit(32)
+    gpu.kge.debug_wait_probe()
+    assert gpu.kge.get_status() == -11
+    assert gpu.kge.get_status() == 0
+    gpu.kge.debug_set_wait_limit(0)                 # back to the default
+    orc._pre = (orc.ent.copy(), orc.rel.copy(), None)
+    _check_step(gpu, orc, 0, orc.sample(0), taps=True)
+    assert gpu.kge.get_status() == 0
 
 
 def test_wide_rows_and_many_splits(oracle64):

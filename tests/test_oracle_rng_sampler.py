@@ -204,3 +204,36 @@ def test_negative_sampler_uniform_within_partition(oracle64):
         hits += np.bincount(oracle64.sample_batch(cfg, step, g)[3], minlength=E)
     exp = N * 10 / E
     assert ((hits - exp) ** 2 / exp).sum() < 27.9     # chi2(9 dof) 0.999 quantile
+
+
+# ----------------------------------------------------------------------------- table initialisation
+def test_init_table_laws_and_words(oracle64):
+    """The initialisation recipe: normal entries with the requested standard deviation (moments and a
+    Kolmogorov-Smirnov test), uniform phases in (-pi, pi), no correlation between the two outputs of a
+    Box-Muller pair or between neighbouring rows, raw words equal to philox of (row, c, stream), and
+    tables of different streams / seeds unrelated."""
+    from scipy import stats
+    rows, width, std = 4000, 52, 0.25
+    a = oracle64.init_table(7, 2, rows, width, std).astype(np.float64)
+    n = a.size
+    assert abs(a.mean()) < 5 * std / np.sqrt(n) and abs(a.std() - std) < 5 * std / np.sqrt(2 * n)
+    assert stats.kstest(a.ravel() / std, "norm").pvalue > 1e-3
+    assert abs(stats.kurtosis(a.ravel())) < 0.05 and abs(stats.skew(a.ravel())) < 0.03
+    for x, y in ((a[:, 0::2], a[:, 1::2]), (a[:-1], a[1:]), (a[:, :-4], a[:, 4:])):
+        assert abs(np.corrcoef(x.ravel(), y.ravel())[0, 1]) < 5 / np.sqrt(x.size)
+    # Box-Muller radius: z0^2 + z1^2 = -2 std^2 ln u is exponentially distributed with mean 2 std^2
+    r2 = (a[:, 0::2] ** 2 + a[:, 1::2] ** 2).ravel() / (2 * std * std)
+    assert stats.kstest(r2, "expon").pvalue > 1e-3
+    ph = oracle64.init_table(7, 3, rows, 6, kind=1).astype(np.float64)          # width 6: a ragged group of four
+    assert ph.min() > -np.pi - 1e-6 and ph.max() < np.pi + 1e-6
+    assert stats.kstest((ph.ravel() + np.pi) / (2 * np.pi), "uniform").pvalue > 1e-3
+    words = oracle64.init_table(7, 2, 50, 8, kind=2).view(np.uint32)
+    for row, c in ((0, 0), (49, 1), (17, 0)):
+        assert (words[row, 4 * c:4 * c + 4] == oracle64.philox([row, 0, c, 2], [7, 0])).all()
+    big = oracle64.init_table(2 ** 40 + 9, 4, 3, 4, kind=2).view(np.uint32)
+    assert (big[2] == oracle64.philox([2, 0, 0, 4], [9, 2 ** 8])).all()            # the seed's upper half is the second key word
+    assert abs(np.corrcoef(a.ravel(), oracle64.init_table(7, 4, rows, width, std).ravel())[0, 1]) < 5 / np.sqrt(n)
+    assert abs(np.corrcoef(a.ravel(), oracle64.init_table(8, 2, rows, width, std).ravel())[0, 1]) < 5 / np.sqrt(n)
+    # the uniform behind every entry is (k + 1/2) 2^-23: recover it from a phase and check it is on that grid
+    k = (ph.ravel() / np.pi + 1) / 2 * 2 ** 23 - 0.5
+    assert np.abs(k - np.round(k)).max() < 2e-1      # fp32 storage of the phase leaves about 0.1 of a grid step

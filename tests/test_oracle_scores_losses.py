@@ -103,6 +103,63 @@ def test_bf16_operand_variant_is_close_and_exact_on_bf16_inputs(oracle64):
     assert oracle64.score("transe", 2, h, np.zeros(d), t, bf16=1) == pytest.approx(-np.linalg.norm(h - t), rel=1e-13)
 
 
+def test_query_vector_is_the_tail_independent_part_of_every_score(oracle64):
+    """q per model against numpy, and f(h, r, t) recovered from (q, t) alone."""
+    rng = np.random.default_rng(21)
+    d = 12
+    h, r, t, w = rng.standard_normal((4, d))
+    c = lambda v: v[0::2] + 1j * v[1::2]
+    q = oracle64.query_vector("transe", h, r)
+    assert q == pytest.approx(h + r, rel=1e-15)
+    for p in (1, 2):
+        assert oracle64.score("transe", p, h, r, t) == pytest.approx(-np.linalg.norm(q - t, ord=p), rel=1e-13)
+    q = oracle64.query_vector("distmult", h, r)
+    assert q == pytest.approx(r * h, rel=1e-15)
+    assert oracle64.score("distmult", 1, h, r, t) == pytest.approx(q @ t, rel=1e-12)
+    q = oracle64.query_vector("complex", h, r)
+    assert c(q) == pytest.approx(c(r) * c(h), rel=1e-13)
+    assert oracle64.score("complex", 1, h, r, t) == pytest.approx(q @ t, rel=1e-12)      # real dot of the interleaved rows
+    ph = rng.uniform(-np.pi, np.pi, d // 2)
+    q = oracle64.query_vector("rotate", h, ph)
+    assert c(q) == pytest.approx(c(h) * np.exp(1j * ph), rel=1e-13)
+    assert oracle64.score("rotate", 1, h, ph, t) == pytest.approx(-np.abs(c(q) - c(t)).sum(), rel=1e-13)
+    assert oracle64.score("rotate", 2, h, ph, t) == pytest.approx(-np.linalg.norm(q - t), rel=1e-13)
+    q = oracle64.query_vector("transh", h, r, w=w)
+    what = w / np.linalg.norm(w)
+    assert q == pytest.approx(h - (what @ h) * what + r, rel=1e-12)
+    for p in (1, 2):
+        x = (q - t) + (what @ t) * what
+        assert oracle64.score("transh", p, h, r, t, w=w) == pytest.approx(-np.linalg.norm(x, ord=p), rel=1e-12)
+
+
+def test_tie_build_differs_from_the_default_only_at_exact_ties(oracle64, oracle64_tie):
+    """The build with sign(0) = -1: identical gradients on generic inputs for every model; on TransE p = 1
+    with integer rows the difference is the closed form -g [x_k = 0] on dh, dr and +g [x_k = 0] on dt."""
+    rng = np.random.default_rng(22)
+    d = 8
+    for score, p in (("transe", 1), ("transe", 2), ("transh", 1), ("transh", 2), ("rotate", 1), ("distmult", 1), ("complex", 1)):
+        h, t, w = rng.standard_normal((3, d))
+        r = rng.standard_normal(d // 2 if score == "rotate" else d)
+        a = oracle64.score_grad(score, p, 0.7, h, r, t, w=w if score == "transh" else None)
+        b = oracle64_tie.score_grad(score, p, 0.7, h, r, t, w=w if score == "transh" else None)
+        for x, y in zip(a, b):
+            assert x is None or (x == y).all()
+    h = np.array([1., 2., -1., 0., 3., 0., 2., 1.]); r = np.array([0., -1., 1., 0., 0., 2., 1., -1.])
+    t = np.array([1., 0., 0., 0., 2., 2., 5., 0.])          # x = h + r - t = (0, 1, 0, 0, 1, 0, -2, 0)
+    tie = (h + r - t) == 0
+    assert tie.sum() == 5
+    g = 0.3
+    dh0, dr0, _, dt0 = oracle64.score_grad("transe", 1, g, h, r, t)
+    dh1, dr1, _, dt1 = oracle64_tie.score_grad("transe", 1, g, h, r, t)
+    # f = -sum |x|: df/dx = -sign(x); at a tie the default build has 0 and the tie build -(-1) = +1
+    assert (dh0[tie] == 0).all() and (dt0[tie] == 0).all()
+    assert dh1 - dh0 == pytest.approx(g * tie) and dr1 - dr0 == pytest.approx(g * tie) and dt1 - dt0 == pytest.approx(-g * tie)
+    # p = 2 and the dot-product models have no such kink: the builds agree on these rows too
+    for score, p in (("transe", 2), ("distmult", 1)):
+        for x, y in zip(oracle64.score_grad(score, p, g, h, r, t), oracle64_tie.score_grad(score, p, g, h, r, t)):
+            assert x is None or (x == y).all()
+
+
 def _f32(bits):
     return float(np.array([bits], dtype=np.uint32).view(np.float32)[0])
 

@@ -34,7 +34,7 @@ def _both(gpu, prob, qh, qr, tt, k):
 
 
 @pytest.mark.parametrize("score,p", [("transe", 1), ("transh", 2), ("complex", 1)])
-def test_static_entry_point_matches_workspace_entry_point_twice(score, p):
+def test_static_entry_point_matches_workspace_entry_point_twice(oracle32, score, p):
     E, R, d, k = 3000, 6, 48, 10
     prob = Problem(E=E, R=R, T=100, d=d, score=score, p_norm=p, B=4, N=4, P=1, graph_seed=21)
     prob.ent[2500] = prob.ent[3]            # an exact tie
@@ -46,6 +46,9 @@ def test_static_entry_point_matches_workspace_entry_point_twice(score, p):
         assert (rk_a == rk_b).all(), call
         assert (sc_a == sc_b).all(), call               # same kernels, same arithmetic: identical scores
         assert (ids_a >= 0).all() and (rk_a >= 1).all()
+        # and on its own feet: the fp32 oracle's lists and ranks, bit for bit
+        o_ids, _, o_ranks = oracle32.score_all_topk(prob.oracle_cfg(), prob.ent, prob.rel, prob.relw, qh, qr, k, true_tails=tt)
+        assert (ids_b == o_ids).all() and (rk_b == o_ranks).all(), call
 
 
 def test_static_entry_point_rejects_sizes_beyond_its_fixed_array():
