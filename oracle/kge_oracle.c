@@ -43,7 +43,10 @@
  *                        with zero imaginary parts; RotatE zero phase -> complex L1;
  *                        TransH special cases; numpy.linalg.norm for the L2 forms.
  *   batch_loss         : closed forms (log(N+1), log|E|, 2 log 2), softmax sums to 1.
- *   batch_grads        : central finite differences of batch_loss in fp64.
+ *   batch_grads        : central finite differences of batch_loss in fp64 (also with the
+ *                        L3 regulariser switched on, both forms).
+ *   l3_term            : hand values (1, -2, 2) -> 17^(1/3) and 17; homogeneity.
+ *   lr_linear_decay    : end points, midpoint, linearity.
  *   dedup/update_rows  : naive scatter when all ids differ; hand sums when they repeat;
  *                        independent numpy restatement of an SGD step.
  *   score_all_topk     : numpy argsort brute force; duplicated rows (exact ties).
@@ -104,6 +107,9 @@ typedef struct {
     double gamma, adv_temp, ce_correction, loss_scale;
     double lr, beta1, beta2, eps;
     uint64_t seed;
+    double reg_lambda;     /* lambda_S of the L3 regulariser on the gathered entity rows (0 = off) */
+    int32_t reg_form;      /* 0: sum of the norms ||e||_3 as printed; 1: sum of the cubes ||e||_3^3 */
+    int32_t _pad2;
 } kgeo_config;
 
 int kgeo_real_bytes(void) { return (int)sizeof(real); }
@@ -584,6 +590,43 @@ real kgeo_row_loss(const kgeo_config *c, real fpos, const real *F, int32_t N,
     return row_loss(c, fpos, F, N, w_fixed, gpos, G);
 }
 
+/* ------------------------------------------------------------------------- */
+/* Regularisation (Section 3.1 "Regularisation"): lambda_S Omega_S with          */
+/* Omega_S = sum over the batch of (||h||_3 + ||t||_3) + sum over the shared     */
+/* negatives of ||t'||_3, one term per occurrence of a row.  There is no feature  */
+/* projection here, so the final embedding is the shallow one and Omega_T equals  */
+/* Omega_S.  The term is added to the micro-batch loss as it stands (it is not    */
+/* multiplied by loss_scale).  reg_form 1 takes the cube of each norm instead     */
+/* (the form of the regulariser's source, Lacroix et al. 2018).                   */
+/* ------------------------------------------------------------------------- */
+real kgeo_l3_term(int32_t form, int32_t d, const real *e) {
+    real s3 = 0;
+    for (int k = 0; k < d; ++k) s3 += R_FABS(e[k]) * e[k] * e[k];
+    return form == 1 ? s3 : (real)cbrt((double)s3);
+}
+
+/* g[k] += lam * d(term)/d e[k]; the norm has zero gradient at e = 0. */
+static void l3_term_grad(int32_t form, int32_t d, real lam, const real *e, real *g) {
+    real s3 = 0;
+    for (int k = 0; k < d; ++k) s3 += R_FABS(e[k]) * e[k] * e[k];
+    if (form == 1) { for (int k = 0; k < d; ++k) g[k] += lam * 3 * e[k] * R_FABS(e[k]); return; }
+    if (!(s3 > 0)) return;
+    real n = (real)cbrt((double)s3);
+    for (int k = 0; k < d; ++k) g[k] += lam * e[k] * R_FABS(e[k]) / (n * n);
+}
+
+static double batch_regulariser(const kgeo_config *c, const real *ent, const int32_t *heads,
+                                const int32_t *tails, const int32_t *negs) {
+    if (c->reg_lambda == 0) return 0;
+    const int32_t d = c->dim;
+    double omega = 0;
+    for (int32_t b = 0; b < c->batch; ++b)
+        omega += (double)kgeo_l3_term(c->reg_form, d, ent + (size_t)heads[b] * d)
+               + (double)kgeo_l3_term(c->reg_form, d, ent + (size_t)tails[b] * d);
+    for (int32_t n = 0; n < c->num_neg; ++n) omega += (double)kgeo_l3_term(c->reg_form, d, ent + (size_t)negs[n] * d);
+    return c->reg_lambda * omega;
+}
+
 static const real *relw_row(const real *relw, int64_t r, int32_t d) {
     return relw ? relw + (size_t)r * d : NULL;
 }
@@ -620,7 +663,7 @@ double kgeo_batch_loss(const kgeo_config *c, const real *ent, const real *rel, c
     }
     for (int32_t b = 0; b < B; ++b) { total += (double)Lrow[b]; if (Lrow_out) Lrow_out[b] = Lrow[b]; }
     free(Lrow);
-    return c->loss_scale * total;
+    return c->loss_scale * total + batch_regulariser(c, ent, heads, tails, negs);
 }
 
 /*
@@ -680,10 +723,18 @@ double kgeo_batch_grads(const kgeo_config *c, const real *ent, const real *rel, 
         }
         free(scratch); free(Frow);
     }
+    if (c->reg_lambda != 0) {   /* one term per occurrence: its gradient joins that occurrence's row */
+        const real lam = (real)c->reg_lambda;
+        for (int32_t b = 0; b < B; ++b) {
+            l3_term_grad(c->reg_form, d, lam, ent + (size_t)heads[b] * d, dh + (size_t)b * d);
+            l3_term_grad(c->reg_form, d, lam, ent + (size_t)tails[b] * d, dtpos + (size_t)b * d);
+        }
+        for (int32_t n = 0; n < N; ++n) l3_term_grad(c->reg_form, d, lam, ent + (size_t)negs[n] * d, dtneg + (size_t)n * d);
+    }
     double total = 0;
     for (int32_t b = 0; b < B; ++b) total += (double)Lrow[b];
     free(Lrow);
-    return c->loss_scale * total;
+    return c->loss_scale * total + batch_regulariser(c, ent, heads, tails, negs);
 }
 
 /* ------------------------------------------------------------------------- */
@@ -859,6 +910,12 @@ int kgeo_score_all_topk(const kgeo_config *c, const real *ent, const real *rel, 
         free(scratch);
     }
     return ERR_OK;
+}
+
+/* Learning rate decayed linearly to zero over the course of training (Section 5). */
+double kgeo_lr_linear_decay(double lr0, uint64_t step, uint64_t total_steps) {
+    if (total_steps == 0 || step >= total_steps) return 0.0;
+    return lr0 * (1.0 - (double)step / (double)total_steps);
 }
 
 /* mean over queries of (rank <= k_cut ? 1/rank : 0); k_cut = 0 means no cut-off. */

@@ -41,13 +41,14 @@ class Config(C.Structure):
         ("loss_scale", C.c_double),
         ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
         ("seed", C.c_uint64),
+        ("reg_lambda", C.c_double), ("reg_form", C.c_int32), ("_pad2", C.c_int32),
     ]
 
 
 def make_config(*, num_entities, num_relations, dim, score, p_norm=1, loss="logsigmoid", opt="sgd",
                 bf16_operands=0, batch=1, num_neg=1, num_parts=1, head_part=-1, sample_mode=0,
                 gamma=0.0, adv_temp=0.0, ce_correction=0.0, loss_scale=1.0, lr=0.1,
-                beta1=0.9, beta2=0.999, eps=None, seed=0) -> Config:
+                beta1=0.9, beta2=0.999, eps=None, seed=0, reg_lambda=0.0, reg_form=0) -> Config:
     score = SCORE_NAMES[score] if isinstance(score, str) else int(score)
     loss = LOSS_NAMES[loss] if isinstance(loss, str) else int(loss)
     opt = OPT_NAMES[opt] if isinstance(opt, str) else int(opt)
@@ -55,7 +56,7 @@ def make_config(*, num_entities, num_relations, dim, score, p_norm=1, loss="logs
         eps = 1e-10 if opt == OPT_ROWWISE_ADAGRAD else 1e-8
     return Config(num_entities, num_relations, dim, score, p_norm, loss, opt, bf16_operands,
                   batch, num_neg, num_parts, head_part, sample_mode, 0,
-                  gamma, adv_temp, ce_correction, loss_scale, lr, beta1, beta2, eps, seed)
+                  gamma, adv_temp, ce_correction, loss_scale, lr, beta1, beta2, eps, seed, reg_lambda, reg_form, 0)
 
 
 def lib_path(precision: str) -> Path:
@@ -107,6 +108,9 @@ class Oracle:
         L.kgeo_batch_grads.restype = C.c_double
         L.kgeo_train_step.restype = C.c_double
         L.kgeo_mrr.restype = C.c_double
+        L.kgeo_l3_term.restype = R
+        L.kgeo_lr_linear_decay.restype = C.c_double
+        L.kgeo_lr_linear_decay.argtypes = [C.c_double, C.c_uint64, C.c_uint64]
         L.kgeo_dedup.restype = C.c_int32
 
     # -- helpers ------------------------------------------------------------
@@ -189,6 +193,13 @@ class Oracle:
         q = np.empty_like(h)
         self.lib.kgeo_query_vector(C.c_int32(score), C.c_int32(len(h)), _p(h, R), _p(r, R), _p(w, R), _p(q, R))
         return q
+
+    def l3_term(self, form, e):
+        e = self.arr(e)
+        return float(self.lib.kgeo_l3_term(C.c_int32(form), C.c_int32(len(e)), _p(e, self.creal)))
+
+    def lr_linear_decay(self, lr0, step, total_steps):
+        return float(self.lib.kgeo_lr_linear_decay(lr0, step, total_steps))
 
     def score_grad(self, score, p, g, h, r, t, w=None):
         score = SCORE_NAMES[score] if isinstance(score, str) else score

@@ -369,6 +369,7 @@ int kge_graph_load_device(kge_handle* h, const int32_t* heads, const int32_t* re
     // keys and triple indices are sorted as 32-bit words
     if (n > ((int64_t)1 << 31) || (int64_t)c.num_parts * c.num_parts * c.num_relations > ((int64_t)1 << 31)) return KGE_ERR_UNSUPPORTED;
     h->graph_loaded = false;
+    if (n == 0) return KGE_ERR_EMPTY_BUCKET;      // every bucket is empty
     const int rc = launch_graph_build_device(h, heads, rels, tails, n, static_cast<cudaStream_t>(stream));
     if (rc != KGE_OK) return rc;
     h->graph_loaded = true;

@@ -302,15 +302,39 @@ def _tiny_problem(rng, score, E=7, R=3, d=4, B=3, N=5):
     return ent, rel, relw, heads, rels, tails, negs
 
 
+def test_l3_regulariser_term_and_lr_decay_closed_forms(oracle64):
+    e = np.array([1.0, -2.0, 2.0, 0.0])
+    assert oracle64.l3_term(0, e) == pytest.approx(17.0 ** (1 / 3), rel=1e-15)       # ||e||_3 = (1 + 8 + 8)^(1/3)
+    assert oracle64.l3_term(1, e) == pytest.approx(17.0, rel=1e-15)
+    assert oracle64.l3_term(0, -3 * e) == pytest.approx(3 * 17.0 ** (1 / 3), rel=1e-14)  # a norm is homogeneous
+    assert oracle64.l3_term(0, np.zeros(4)) == 0.0
+    # the batch term counts every occurrence of a row: lambda (sum over heads, tails, negatives)
+    rng = np.random.default_rng(3)
+    ent, rel, relw, heads, rels, tails, negs = _tiny_problem(rng, "distmult")
+    kw = dict(num_entities=7, num_relations=3, dim=4, score="distmult", batch=3, num_neg=5, loss_scale=0.5)
+    base = oracle64.batch_loss(make_config(**kw), ent, rel, None, heads, rels, tails, negs)["loss"]
+    for form in (0, 1):
+        omega = sum(np.sum(np.abs(ent[i]) ** 3) ** (1.0 if form else 1 / 3) for i in np.concatenate([heads, tails, negs]))
+        got = oracle64.batch_loss(make_config(**kw, reg_lambda=0.3, reg_form=form), ent, rel, None, heads, rels, tails, negs)["loss"]
+        assert got == pytest.approx(base + 0.3 * omega, rel=1e-13)                   # added as it stands, not times loss_scale
+    # linear decay to zero (Section 5)
+    assert oracle64.lr_linear_decay(0.05, 0, 1000) == 0.05 and oracle64.lr_linear_decay(0.05, 1000, 1000) == 0.0
+    assert oracle64.lr_linear_decay(0.05, 500, 1000) == pytest.approx(0.025, rel=1e-15)
+    assert oracle64.lr_linear_decay(0.05, 2000, 1000) == 0.0
+    steps = np.arange(0, 1000, 37)
+    lrs = np.array([oracle64.lr_linear_decay(0.05, int(s), 1000) for s in steps])
+    assert np.allclose(np.diff(lrs), -0.05 * 37 / 1000, rtol=1e-12, atol=0)
+
+
 @pytest.mark.parametrize("score,p", MODELS)
-@pytest.mark.parametrize("loss", ["logsigmoid", "softmax"])
-def test_batch_grads_match_central_finite_differences(oracle64, score, p, loss):
+@pytest.mark.parametrize("loss,reg", [("logsigmoid", None), ("softmax", None), ("softmax", 0), ("logsigmoid", 1)])
+def test_batch_grads_match_central_finite_differences(oracle64, score, p, loss, reg):
     rng = np.random.default_rng(100 * MODELS.index((score, p)) + len(loss))
     ent, rel, relw, heads, rels, tails, negs = _tiny_problem(rng, score)
     E, d = ent.shape
     cfg = make_config(num_entities=E, num_relations=len(rel), dim=d, score=score, p_norm=p, loss=loss,
                       batch=3, num_neg=5, gamma=1.5 if loss == "logsigmoid" else 0.0, adv_temp=0.8,
-                      ce_correction=0.4, loss_scale=0.5)
+                      ce_correction=0.4, loss_scale=0.5, reg_lambda=0.0 if reg is None else 0.37, reg_form=reg or 0)
     out = oracle64.batch_grads(cfg, ent, rel, relw, heads, rels, tails, negs)
     base = oracle64.batch_loss(cfg, ent, rel, relw, heads, rels, tails, negs)
     assert out["loss"] == pytest.approx(base["loss"], rel=1e-14)
