@@ -85,7 +85,9 @@ typedef struct {
     float lr;               /* default learning rate (kge_train_step takes one per call) */
     float beta1, beta2;     /* Adam */
     float eps;              /* Adam / Adagrad denominator epsilon */
-    uint64_t seed;          /* sampler seed (Philox key) */
+    uint64_t seed;          /* sampler seed (Philox key); also keys kge_init_tables */
+    float reg_lambda;       /* lambda_S >= 0 of the L3 regulariser (Section 3.1 "Regularisation"); 0 = off */
+    int32_t reg_form;       /* 0: sum of the norms ||e||_3 as printed; 1: sum of the cubes ||e||_3^3 */
 } kge_config;
 
 /* Validate the configuration and create the handle.  Allocates nothing on the device. */
@@ -161,6 +163,10 @@ int kge_sample_batch(kge_handle* h, uint64_t step, int32_t* heads, int32_t* rels
  * are taken at the pre-step tables.  If heads/rels/tails/negs are all NULL the batch of
  * `step` is sampled internally exactly as kge_sample_batch would.  `step` also drives Adam's
  * bias correction (t = step + 1).  loss_out: one float, loss_scale * sum_b L_b (may be NULL).
+ * With reg_lambda > 0 the L3 regulariser of Section 3.1 "Regularisation" on the gathered entity rows,
+ * lambda_S Omega_S with Omega_S = sum_b (||h_b||_3 + ||t_b||_3) + sum_n ||t'_n||_3 (one term per
+ * occurrence of a row; without a feature projection Omega_T = Omega_S), is added to the loss as it
+ * stands (not times loss_scale) and its gradient to the rows' gradients.
  */
 int kge_train_step(kge_handle* h, uint64_t step, float lr,
                    const int32_t* heads, const int32_t* rels, const int32_t* tails, const int32_t* negs,
@@ -229,6 +235,30 @@ int kge_eval_mrr(kge_handle* h, const int32_t* q_heads, const int32_t* q_rels, c
  */
 int kge_mrr_from_ranks(kge_handle* h, const int32_t* ranks, int32_t nq, int32_t k_cutoff,
                        double* mrr_out /*[host]*/, void* stream);
+
+/* Learning rate of step `step` when lr0 is decayed linearly to zero over total_steps steps (the
+ * recipe of Section 5): lr0 (1 - step / total_steps), 0 from total_steps on.  Pure host arithmetic;
+ * pass the result to kge_train_step. */
+float kge_lr_linear_decay(float lr0, uint64_t step, uint64_t total_steps);
+
+/*
+ * Power-rank ensemble (Section 3.2 "Ensemble", Eq. 2).  lists: device int32 [num_models, nq, k_list],
+ * lists[m][q] = the top-k_list tails of model m for query q in rank order (the out_ids of
+ * kge_score_all_topk; places holding -1 are skipped).  Every entity of a query's lists gets
+ * s(t) = sum over the models, in ascending model order, of table[k - 1] if t is the k-th entry of the
+ * model's list and table[k_list] if it is in none of its places; out_ids [nq, top_n] receives the
+ * top_n entities by (s descending, entity id ascending), out_scores [nq, top_n] (device fp64, may be
+ * NULL) their s; places beyond the number of distinct entities hold -1 and -inf.  The sums are fp64
+ * additions of the table's entries in that fixed order.  At most 16,384 list entries per query
+ * (num_models * k_list; else KGE_ERR_WORKSPACE).  Enqueues on `stream` and returns.
+ *
+ * kge_ensemble_rank_scores fills the table [host, k_list + 1 doubles] for a power p != 0 as Eq. 2
+ * defines it: table[k - 1] = -sgn(p) k^p for k = 1 .. k_list, table[k_list] = -(k_list + 1)^p if
+ * p > 0, else 0 (the paper settles on p = -0.5).  Copy it to the device for kge_ensemble_topk.
+ */
+int kge_ensemble_rank_scores(double power, int32_t k_list, double* table /*[host]*/);
+int kge_ensemble_topk(const int32_t* lists, int32_t num_models, int32_t nq, int32_t k_list, const double* table,
+                      int32_t top_n, int32_t* out_ids, double* out_scores, void* stream);
 
 /* Synchronise `stream`, return the sticky device status word (0 or a negative code), clear it. */
 int kge_get_status(kge_handle* h, void* stream);

@@ -46,13 +46,14 @@ class KgeConfig(C.Structure):
         ("gamma", C.c_float), ("adv_temp", C.c_float), ("ce_correction", C.c_float), ("loss_scale", C.c_float),
         ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
         ("seed", C.c_uint64),
+        ("reg_lambda", C.c_float), ("reg_form", C.c_int32),
     ]
 
     @classmethod
     def make(cls, *, num_entities, num_relations, dim, score, p_norm=1, loss="logsigmoid", opt="sgd",
              prec=PREC_FP32, batch=1, num_neg=1, num_parts=1, head_part=-1, sample_mode=0,
              gamma=0.0, adv_temp=0.0, ce_correction=0.0, loss_scale=1.0, lr=0.1,
-             beta1=0.9, beta2=0.999, eps=None, seed=0) -> "KgeConfig":
+             beta1=0.9, beta2=0.999, eps=None, seed=0, reg_lambda=0.0, reg_form=0) -> "KgeConfig":
         score = SCORE_NAMES[score] if isinstance(score, str) else int(score)
         loss = LOSS_NAMES[loss] if isinstance(loss, str) else int(loss)
         opt = OPT_NAMES[opt] if isinstance(opt, str) else int(opt)
@@ -60,7 +61,7 @@ class KgeConfig(C.Structure):
             eps = 1e-10 if opt == OPT_ROWWISE_ADAGRAD else 1e-8
         return cls(num_entities, num_relations, dim, score, p_norm, loss, opt, prec, batch, num_neg,
                    num_parts, head_part, sample_mode, 0, gamma, adv_temp, ce_correction, loss_scale,
-                   lr, beta1, beta2, eps, seed)
+                   lr, beta1, beta2, eps, seed, reg_lambda, reg_form)
 
 
 def library_path() -> Path:
@@ -91,6 +92,9 @@ SIGNATURES = {
     "kge_debug_capture_scores": (C.c_int, [_vp, _vp]),
     "kge_debug_set_wait_limit": (C.c_int, [_vp, C.c_int32]),
     "kge_debug_wait_probe": (C.c_int, [_vp, _vp]),
+    "kge_lr_linear_decay": (C.c_float, [C.c_float, C.c_uint64, C.c_uint64]),
+    "kge_ensemble_rank_scores": (C.c_int, [C.c_double, C.c_int32, _vp]),
+    "kge_ensemble_topk": (C.c_int, [_vp, C.c_int32, C.c_int32, C.c_int32, _vp, C.c_int32, _vp, _vp, _vp]),
     "kge_get_status": (C.c_int, [_vp, _vp]),
     "kge_launch_count": (C.c_int64, [_vp]),
     "kge_profile": (C.c_int, [_vp, C.c_int]),
@@ -143,6 +147,22 @@ def score_all_topk_static(cfg: KgeConfig, ent, rel, relw, q_heads, q_rels, k, tr
     return int(lib().kge_score_all_topk_static(C.byref(cfg), _ptr(ent), _ptr(rel), _ptr(relw), _ptr(q_heads),
                                                _ptr(q_rels), q_heads.numel(), k, _ptr(true_tails), _ptr(out_ids),
                                                _ptr(out_scores), _ptr(out_ranks), _stream()))
+
+
+def ensemble_rank_scores(power: float, k_list: int):
+    """kge_ensemble_rank_scores: the table of Eq. 2's rank scores as a numpy float64 array [k_list + 1]."""
+    import numpy as np
+    table = np.empty(k_list + 1, dtype=np.float64)
+    rc = int(lib().kge_ensemble_rank_scores(power, k_list, _ptr(table)))
+    if rc != 0:
+        raise KgeError(rc, "kge_ensemble_rank_scores", lib().kge_error_string(rc).decode())
+    return table
+
+
+def ensemble_topk(lists, table, top_n, out_ids, out_scores=None) -> int:
+    """kge_ensemble_topk on device tensors: lists int32 [M, nq, K], table float64 [K + 1]."""
+    m, nq, k = lists.shape
+    return int(lib().kge_ensemble_topk(_ptr(lists), m, nq, k, _ptr(table), top_n, _ptr(out_ids), _ptr(out_scores), _stream()))
 
 
 class Kge:

@@ -68,6 +68,7 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
     w.What = th ? cv.take<float>(B * d) : nullptr;
     w.Tneg = cv.take<float>(N * d);
     w.fpos = cv.take<float>(B); w.gpos = cv.take<float>(B); w.Lrow = cv.take<float>(B);
+    w.reg_s3 = c.reg_lambda > 0.f ? cv.take<float>(2 * B + N) : nullptr;
     const bool tc = c.prec == KGE_PREC_BF16_TC;
     w.Qb = tc ? cv.take<uint16_t>(B * d) : nullptr;
     w.Tb = tc ? cv.take<uint16_t>(N * d) : nullptr;
@@ -182,6 +183,7 @@ int kge_create(const kge_config* cfg, kge_handle** out) {
     if (c.head_part >= c.num_parts || c.head_part < -1) return KGE_ERR_BAD_ARG;
     if (c.sample_mode != 0 && c.sample_mode != 1) return KGE_ERR_BAD_ARG;
     if (!(c.adv_temp >= 0.f)) return KGE_ERR_BAD_ARG;
+    if (!(c.reg_lambda >= 0.f) || (c.reg_form != 0 && c.reg_form != 1)) return KGE_ERR_BAD_ARG;
     if ((int64_t)c.batch * c.num_neg > ((int64_t)1 << 31)) return KGE_ERR_BAD_ARG;
     const int64_t P = c.num_parts;
     if (c.num_neg % P != 0) return KGE_ERR_DIVISIBILITY;
@@ -524,6 +526,11 @@ int kge_debug_capture_scores(kge_handle* h, float* scores_out) {
     if (scores_out && (reinterpret_cast<uintptr_t>(scores_out) % 16) != 0) return KGE_ERR_BAD_ARG;
     h->capture_scores = scores_out;
     return KGE_OK;
+}
+
+float kge_lr_linear_decay(float lr0, uint64_t step, uint64_t total_steps) {
+    if (total_steps == 0 || step >= total_steps) return 0.f;
+    return (float)((double)lr0 * (1.0 - (double)step / (double)total_steps));
 }
 
 int kge_get_status(kge_handle* h, void* stream) {

@@ -49,6 +49,7 @@ struct Workspace {
     int32_t *heads, *rels, *tails, *negs;  // contiguous [3B+N]
     float *Q, *What, *Tneg;                // [B,d], [B,d] (TransH), [N,d]
     float *fpos, *gpos, *Lrow;             // [B]
+    float *reg_s3;                         // [2B+N] sum of |e_k|^3 of the gathered rows [heads | tails | negs] (L3 regulariser), or NULL
     uint16_t *Qb, *Tb;                     // [B,d], [N,d] bf16 copies of Q and Tneg (tensor-core scoring)
     uint16_t *Gb;                          // bf16 [B,ldN] dL/dF (ldN = N rounded up to 8)
     float *Gcol;                           // [N] column sums of dL/dF (TransE p=2 on tensor cores)

@@ -857,7 +857,8 @@ int launch_tc_bwd_gemm(kge_handle* h, const unsigned char* tmA, const unsigned c
 }  // namespace
 
 bool tc_negatives_direct(const kge_handle* h) {
-    return h->cfg.prec == KGE_PREC_BF16_TC && h->kind == KIND_DOT && h->split_t == 1;
+    // (with the regulariser on, the chain kernel still has a term to add to every negative's row)
+    return h->cfg.prec == KGE_PREC_BF16_TC && h->kind == KIND_DOT && h->split_t == 1 && !(h->cfg.reg_lambda > 0.f);
 }
 
 // Columns per tile of a backward contraction whose output rows are `cols` wide.

@@ -27,6 +27,8 @@ struct TrainParams {
     int tc_l2;          // TransE p = 2 with tensor-core backward: the splits hold C.T and C^T.Q, C = dL/dF / distance
     int neg_direct;     // the dT contraction wrote the negatives' gradient rows itself (one K split, no correction term)
     int wait_limit;     // tries of a bounded barrier wait
+    float reg_lambda;   // L3 regulariser on the gathered entity rows (0 = off)
+    int reg_form;       // 0: norms, 1: cubes
     Workspace w;
 };
 
@@ -39,6 +41,21 @@ __device__ __forceinline__ float4 f4fma(float s, float4 a, float4 c) {
     return make_float4(fmaf(s, a.x, c.x), fmaf(s, a.y, c.y), fmaf(s, a.z, c.z), fmaf(s, a.w, c.w));
 }
 __device__ __forceinline__ float f4dot(float4 a, float4 b) { return a.x * b.x + a.y * b.y + a.z * b.z + a.w * b.w; }
+// L3 regulariser (Section 3.1 "Regularisation"): a lane's share of sum_k |e_k|^3, and c * e_k |e_k| (the gradient's shape).
+__device__ __forceinline__ float f4cube(float4 a) {
+    return fabsf(a.x) * a.x * a.x + fabsf(a.y) * a.y * a.y + fabsf(a.z) * a.z * a.z + fabsf(a.w) * a.w * a.w;
+}
+__device__ __forceinline__ float4 f4reg(float c, float4 a) {
+    return make_float4(c * a.x * fabsf(a.x), c * a.y * fabsf(a.y), c * a.z * fabsf(a.z), c * a.w * fabsf(a.w));
+}
+// Factor of e_k |e_k| in the gradient of lambda * (term of one row) given s3 = sum_k |e_k|^3:
+// norm: lambda / ||e||_3^2 (0 at e = 0); cube: 3 lambda.
+__device__ __forceinline__ float reg_coef(float lambda, int form, float s3) {
+    if (form == 1) return 3.f * lambda;
+    if (!(s3 > 0.f)) return 0.f;
+    const float n = cbrtf(s3);
+    return lambda / (n * n);
+}
 // The sub-gradient of |x| that every p = 1 kernel of this library uses: +1 for x > 0, -1 otherwise.
 // At x == 0 any value in [-1, 1] is a sub-gradient; the score-block backward counts the pairs with
 // x > 0 (see add_if_pos), which fixes -1 there, and the positive pair takes the same value so that
@@ -93,7 +110,7 @@ __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
         const int64_t id = checked_id(neg, p.E, p.w.status);
         const float4* src = reinterpret_cast<const float4*>(p.ent) + id * d4;
         float4* dst = reinterpret_cast<float4*>(p.w.Tneg) + (int64_t)n * d4;
-        float nrm2 = 0.f;
+        float nrm2 = 0.f, s3 = 0.f;
         for (int c = lane; c < d4; c += 32) {
             const float4 v = src[c];
             dst[c] = v;
@@ -101,8 +118,10 @@ __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
                 reinterpret_cast<uint2*>(p.w.Tb)[(int64_t)n * d4 + c] = pack_bf16x4(v);
                 nrm2 += f4dot(v, v);
             }
+            if (p.w.reg_s3) s3 += f4cube(v);
         }
         if (p.w.Tb) { nrm2 = warp_sum(nrm2); if (lane == 0) p.w.tn2[n] = nrm2; }
+        if (p.w.reg_s3) { s3 = warp_sum(s3); if (lane == 0) p.w.reg_s3[2 * p.B + n] = s3; }
         return;
     }
     const int b = warp;
@@ -128,6 +147,13 @@ __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
         h[i] = c < d4 ? hrow[c] : f4zero();
         t[i] = c < d4 ? trow[c] : f4zero();
         q[i] = f4zero(); wh[i] = f4zero();
+    }
+    if (p.w.reg_s3) {
+        float sh = 0.f, st = 0.f;
+#pragma unroll
+        for (int i = 0; i < kMaxChunks; ++i) { sh += f4cube(h[i]); st += f4cube(t[i]); }
+        sh = warp_sum(sh); st = warp_sum(st);
+        if (lane == 0) { p.w.reg_s3[b] = sh; p.w.reg_s3[p.B + b] = st; }
     }
     if (p.score == KGE_ROTATE) {
         const float2* th = reinterpret_cast<const float2*>(p.rel) + rid * d4;  // d/2 phases = d4 float2
@@ -1094,13 +1120,18 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
         __shared__ float lsum[8];
         float v = 0.f;
         for (int b = threadIdx.x; b < p.B; b += 256) v += p.w.Lrow[b];
+        v *= p.loss_scale;
+        if (p.w.reg_s3) {   // lambda Omega: one term per gathered row, added as it stands
+            float om = 0.f;
+            for (int i = threadIdx.x; i < 2 * p.B + p.N; i += 256) { const float s3 = p.w.reg_s3[i]; om += p.reg_form == 1 ? s3 : cbrtf(s3); }
+            v = fmaf(p.reg_lambda, om, v);
+        }
         v = warp_sum(v);
         if (lane == 0) lsum[threadIdx.x >> 5] = v;
         __syncthreads();
         if (threadIdx.x == 0) {
             float t = 0.f;
             for (int i = 0; i < 8; ++i) t += lsum[i];
-            t *= p.loss_scale;
             *p.w.loss = t;
             if (p.loss_out) *p.loss_out = t;
         }
@@ -1115,6 +1146,7 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
         const float4* part = reinterpret_cast<const float4*>(p.w.dTpart);
         float wsum = 0.f;   // TransE p = 1: the splits hold P, the gradient is 2 P - (column sum of dL/dF)
         if (p.kind == KIND_L1) wsum = sum_splits(p.w.Cpart + n, p.N, p.split_t);
+        const float creg = p.w.reg_s3 ? reg_coef(p.reg_lambda, p.reg_form, p.w.reg_s3[2 * p.B + n]) : 0.f;
         for (int c = lane; c < d4; c += 32) {
             float4 s = sum_splits(part + (int64_t)n * d4 + c, (int64_t)p.N * d4, p.split_t);
             if (p.kind == KIND_L1) s = make_float4(2.f * s.x - wsum, 2.f * s.y - wsum, 2.f * s.z - wsum, 2.f * s.w - wsum);
@@ -1123,6 +1155,7 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
                 const float4 t = reinterpret_cast<const float4*>(p.w.Tneg)[(int64_t)n * d4 + c];
                 s = make_float4(s.x - cs * t.x, s.y - cs * t.y, s.z - cs * t.z, s.w - cs * t.w);
             }
+            if (p.w.reg_s3) s = f4add(s, f4reg(creg, reinterpret_cast<const float4*>(p.w.Tneg)[(int64_t)n * d4 + c]));
             gent[(int64_t)(2 * p.B + n) * d4 + c] = s;
         }
         return;
@@ -1156,6 +1189,9 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
     }
     float4* gh = gent + (int64_t)b * d4;
     float4* gt = gent + (int64_t)(p.B + b) * d4;
+    // L3 regulariser: its gradient joins the head's and the positive tail's rows where they are stored
+    const float creg_h = p.w.reg_s3 ? reg_coef(p.reg_lambda, p.reg_form, p.w.reg_s3[b]) : 0.f;
+    const float creg_t = p.w.reg_s3 ? reg_coef(p.reg_lambda, p.reg_form, p.w.reg_s3[p.B + b]) : 0.f;
 
     if (p.score == KGE_TRANSH) {
         const float4* whrow = reinterpret_cast<const float4*>(p.w.What) + (int64_t)b * d4;
@@ -1212,8 +1248,8 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
         for (int i = 0; i < kMaxChunks; ++i) {
             const int c = lane + 32 * i;
             if (c >= d4) continue;
-            gh[c] = f4fma(-wdq, wh[i], dq[i]);
-            gt[c] = dt[i];
+            gh[c] = f4add(f4fma(-wdq, wh[i], dq[i]), f4reg(creg_h, h[i]));
+            gt[c] = f4add(dt[i], f4reg(creg_t, t[i]));
             gr[c] = dq[i];
             gw[c] = clamped ? f4scale(inv, dwh[i]) : f4scale(inv, f4fma(-wdw, wh[i], dwh[i]));
         }
@@ -1254,9 +1290,9 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
             const float2 ph = th[c];
             float s0, c0, s1, c1;
             sincosf(ph.x, &s0, &c0); sincosf(ph.y, &s1, &c1);
-            gh[c] = make_float4(dq[i].x * c0 + dq[i].y * s0, -dq[i].x * s0 + dq[i].y * c0,
-                                dq[i].z * c1 + dq[i].w * s1, -dq[i].z * s1 + dq[i].w * c1);
-            gt[c] = dt[i];
+            gh[c] = f4add(make_float4(dq[i].x * c0 + dq[i].y * s0, -dq[i].x * s0 + dq[i].y * c0,
+                                      dq[i].z * c1 + dq[i].w * s1, -dq[i].z * s1 + dq[i].w * c1), f4reg(creg_h, h[i]));
+            gt[c] = f4add(dt[i], f4reg(creg_t, t[i]));
             gr[c] = make_float2(-dq[i].x * q[i].y + dq[i].y * q[i].x, -dq[i].z * q[i].w + dq[i].w * q[i].z);
         }
         return;
@@ -1267,16 +1303,17 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
     for (int i = 0; i < kMaxChunks; ++i) {
         const int c = lane + 32 * i;
         if (c >= d4) continue;
-        gt[c] = dt[i];
+        gt[c] = f4add(dt[i], f4reg(creg_t, t[i]));
+        const float4 rg = f4reg(creg_h, h[i]);
         if (p.score == KGE_TRANSE) {
-            gh[c] = dq[i]; gr[c] = dq[i];
+            gh[c] = f4add(dq[i], rg); gr[c] = dq[i];
         } else if (p.score == KGE_DISTMULT) {
             const float4 r = rrow[c];
-            gh[c] = f4mul(dq[i], r); gr[c] = f4mul(dq[i], h[i]);
+            gh[c] = f4add(f4mul(dq[i], r), rg); gr[c] = f4mul(dq[i], h[i]);
         } else {  // ComplEx: q = r * h
             const float4 r = rrow[c];
-            gh[c] = make_float4(dq[i].x * r.x + dq[i].y * r.y, -dq[i].x * r.y + dq[i].y * r.x,
-                                dq[i].z * r.z + dq[i].w * r.w, -dq[i].z * r.w + dq[i].w * r.z);
+            gh[c] = f4add(make_float4(dq[i].x * r.x + dq[i].y * r.y, -dq[i].x * r.y + dq[i].y * r.x,
+                                      dq[i].z * r.z + dq[i].w * r.w, -dq[i].z * r.w + dq[i].w * r.z), rg);
             gr[c] = make_float4(dq[i].x * h[i].x + dq[i].y * h[i].y, -dq[i].x * h[i].y + dq[i].y * h[i].x,
                                 dq[i].z * h[i].z + dq[i].w * h[i].w, -dq[i].z * h[i].w + dq[i].w * h[i].z);
         }
@@ -1382,6 +1419,7 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     p.tc_l2 = c.prec == KGE_PREC_BF16_TC && p.kind == KIND_L2;
     p.neg_direct = tc_negatives_direct(h) ? 1 : 0;
     p.wait_limit = h->wait_limit;
+    p.reg_lambda = c.reg_lambda; p.reg_form = c.reg_form;
     p.w = h->ws;
     const int nch = p.d4 <= 32 ? 1 : (p.d4 <= 64 ? 2 : 4);
 

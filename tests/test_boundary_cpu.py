@@ -30,8 +30,9 @@ def test_library_exports_every_declared_symbol(K):
 
 
 def test_config_struct_matches_header_layout(K):
-    # 2 x int64 + 12 x int32 + 8 x float + uint64 = 104 bytes, seed 8-byte aligned
-    assert C.sizeof(K.KgeConfig) == 104 and K.KgeConfig.seed.offset == 96 and K.KgeConfig.gamma.offset == 64
+    # 2 x int64 + 12 x int32 + 8 x float + uint64 + float + int32 = 112 bytes, seed 8-byte aligned
+    assert C.sizeof(K.KgeConfig) == 112 and K.KgeConfig.seed.offset == 96 and K.KgeConfig.gamma.offset == 64
+    assert K.KgeConfig.reg_lambda.offset == 104 and K.KgeConfig.reg_form.offset == 108
 
 
 def _create(K, **over):

@@ -242,6 +242,44 @@ def test_bounded_wait_runs_out_and_the_context_stays_usable(oracle64):
     assert gpu.kge.get_status() == 0
 
 
+@pytest.mark.parametrize("score,p,form,tc", [("transe", 1, 0, False), ("distmult", 1, 1, False), ("transh", 2, 0, False),
+                                             ("rotate", 1, 1, False), ("complex", 1, 0, True), ("transe", 2, 1, True)])
+def test_l3_regulariser(oracle64, score, p, form, tc):
+    """lambda_S Omega_S on the gathered rows (Section 3.1 "Regularisation"), both forms, on the CUDA-core and the
+    tensor-core path (where the negatives' gradient rows otherwise bypass the chain kernel): the loss, every
+    gradient row and the updated tables against the oracle; one entity is head, tail and negative at once."""
+    d = 64 if tc else 40
+    prob = Problem(E=400, R=6, T=20000, d=d, score=score, p_norm=p, loss="softmax" if tc else "logsigmoid", B=128, N=128, P=2,
+                   gamma=4.0 if score in ("transe", "transh", "rotate") and not tc else 0.0, adv_temp=0.0 if tc else 0.5,
+                   ce_correction=0.2, loss_scale=0.5, lr=0.05, graph_seed=16, relation_zipf=1.0, tc=tc,
+                   reg_lambda=0.07, reg_form=form)
+    prob.ent[5] = 0.0                                   # a zero row: the norm has zero gradient there
+    gpu, orc = GpuSide(prob), OracleSide(prob, oracle64)
+    batch = [a.copy() for a in orc.sample(0)]
+    batch[0][:3] = 9; batch[2][3:5] = 9; batch[3][:4] = 9; batch[3][7] = 5; batch[0][10] = 5
+    orc._pre = (orc.ent.copy(), orc.rel.copy(), None if orc.relw is None else orc.relw.copy())
+    unreg = oracle64.batch_loss(Problem.oracle_cfg(_without_reg(prob)), orc.ent, orc.rel, orc.relw, *batch)["loss"]
+    _check_step(gpu, orc, 0, batch)
+    assert gpu.kge.get_status() == 0
+    reg = oracle64.batch_loss(orc.cfg, *orc._pre, *batch)["loss"] - unreg
+    assert reg > 0.05 * abs(unreg)                      # the term is a visible share of the loss
+
+
+def _without_reg(prob):
+    import copy
+    q = copy.copy(prob)
+    q.kw = dict(prob.kw, reg_lambda=0.0)
+    return q
+
+
+def test_lr_linear_decay_helper(oracle64):
+    import paper_2211_12281_b200 as K
+    f = K.lib().kge_lr_linear_decay
+    for lr0, step, total in ((0.05, 0, 1000), (0.05, 500, 1000), (0.05, 999, 1000), (0.05, 1000, 1000), (0.05, 5000, 1000),
+                             (3e-3, 1234567, 5_000_000), (1.0, 7, 0)):
+        assert f(lr0, step, total) == pytest.approx(oracle64.lr_linear_decay(np.float32(lr0), step, total), rel=1e-6, abs=0)
+
+
 def test_wide_rows_and_many_splits(oracle64):
     # d = 256 (two slices per lane), B << N so the dQ accumulation is split over columns
     prob = Problem(E=2000, R=11, T=40000, d=256, score="distmult", loss="softmax", B=32, N=640, P=4,
