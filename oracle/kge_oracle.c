@@ -47,6 +47,8 @@
  *                        L3 regulariser switched on, both forms).
  *   l3_term            : hand values (1, -2, 2) -> 17^(1/3) and 17; homogeneity.
  *   lr_linear_decay    : end points, midpoint, linearity.
+ *   ensemble_topk      : a hand-worked 3-model example (p = -0.5, p = 1), reciprocal-rank fusion (p = -1)
+ *                        restated in numpy, invariance under a permutation of the models, the id tie rule.
  *   dedup/update_rows  : naive scatter when all ids differ; hand sums when they repeat;
  *                        independent numpy restatement of an SGD step.
  *   score_all_topk     : numpy argsort brute force; duplicated rows (exact ties).
@@ -909,6 +911,56 @@ int kgeo_score_all_topk(const kgeo_config *c, const real *ent, const real *rel, 
         }
         free(scratch);
     }
+    return ERR_OK;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Power-rank ensemble (Section 3.2 "Ensemble", Eq. 2).  lists[m][q][0..K) are  */
+/* model m's top-K tails of query q in rank order (-1 = unused place).  Brute     */
+/* force: every entity that occurs in one of the query's lists gets                */
+/*   s(t) = sum over m ascending of  -sgn(p) k^p  if t is the k-th of list m,       */
+/*                                   -[p > 0] (K + 1)^p  if t is not in list m,     */
+/* and the top_n by (s descending, id ascending) are returned (entities in no list  */
+/* have the lowest possible score and cannot reach the top when K >= top_n).        */
+/* Always fp64.                                                                     */
+/* ------------------------------------------------------------------------- */
+int kgeo_ensemble_topk(const int32_t *lists, int32_t M, int32_t nq, int32_t K, double p, int32_t top_n,
+                       int32_t *out_ids, double *out_scores) {
+    if (M <= 0 || K <= 0 || top_n <= 0 || p == 0.0) return ERR_BAD_ARG;
+    const double sgn = p > 0 ? 1.0 : -1.0;
+    const double absent = p > 0 ? -pow((double)K + 1.0, p) : 0.0;
+    int32_t *cand = (int32_t *)malloc(sizeof(int32_t) * (size_t)M * K);
+    double *cs = (double *)malloc(sizeof(double) * (size_t)M * K);
+    for (int32_t q = 0; q < nq; ++q) {
+        int32_t nc = 0;
+        for (int32_t m = 0; m < M; ++m)
+            for (int32_t k = 0; k < K; ++k) {
+                int32_t id = lists[((size_t)m * nq + q) * K + k];
+                if (id < 0) continue;
+                int seen = 0;
+                for (int32_t c = 0; c < nc; ++c) if (cand[c] == id) { seen = 1; break; }
+                if (!seen) cand[nc++] = id;
+            }
+        for (int32_t c = 0; c < nc; ++c) {
+            double s = 0;
+            for (int32_t m = 0; m < M; ++m) {
+                int present = 0;
+                for (int32_t k = 0; k < K; ++k)
+                    if (lists[((size_t)m * nq + q) * K + k] == cand[c]) { s += -sgn * pow((double)(k + 1), p); present = 1; }
+                if (!present) s += absent;
+            }
+            cs[c] = s;
+        }
+        for (int32_t r = 0; r < top_n; ++r) {
+            int32_t best = -1;
+            for (int32_t c = 0; c < nc; ++c)
+                if (cand[c] >= 0 && (best < 0 || cs[c] > cs[best] || (cs[c] == cs[best] && cand[c] < cand[best]))) best = c;
+            out_ids[(size_t)q * top_n + r] = best >= 0 ? cand[best] : -1;
+            out_scores[(size_t)q * top_n + r] = best >= 0 ? cs[best] : -(double)INFINITY;
+            if (best >= 0) cand[best] = -1;
+        }
+    }
+    free(cand); free(cs);
     return ERR_OK;
 }
 

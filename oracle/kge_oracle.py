@@ -293,6 +293,17 @@ class Oracle:
             raise ValueError(f"kgeo_score_all_topk failed: {rc}")
         return ids, sc, ranks
 
+    def ensemble_topk(self, lists, power, top_n=10):
+        """lists: int32 [M, nq, K].  Returns (ids [nq, top_n], scores [nq, top_n] float64)."""
+        lists = np.ascontiguousarray(lists, dtype=np.int32)
+        M, nq, K = lists.shape
+        ids, sc = np.empty((nq, top_n), np.int32), np.empty((nq, top_n), np.float64)
+        rc = self.lib.kgeo_ensemble_topk(_p(lists, C.c_int32), C.c_int32(M), C.c_int32(nq), C.c_int32(K), C.c_double(power),
+                                         C.c_int32(top_n), _p(ids, C.c_int32), _p(sc, C.c_double))
+        if rc != 0:
+            raise ValueError(f"kgeo_ensemble_topk failed: {rc}")
+        return ids, sc
+
     def mrr(self, ranks, k_cut=0):
         ranks = np.ascontiguousarray(ranks, dtype=np.int64)
         return float(self.lib.kgeo_mrr(_p(ranks, C.c_int64), C.c_int32(len(ranks)), C.c_int32(k_cut)))
