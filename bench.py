@@ -1,18 +1,24 @@
 #!/usr/bin/env python
-"""Benchmark of the shared-negative scoring block: one "step" = one pass of the whole
-training hot path (sample, gather, score block, loss, backward, dedup, sparse update) over
-one synthetic batch.
+"""Benchmark of the shared-negative scoring block.
 
-    python bench.py --gpus N --steps K --warmup W            # the CUDA library
+A training "step" is one pass of the whole hot path (sample, gather, score block, loss, backward,
+dedup, sparse update) over one synthetic batch; an inference "step" is one pass of all queries over
+the whole entity table (scores, top-k, rank).
+
+    python bench.py --gpus N --steps K --warmup W            # the CUDA library, every workload of the suite
+    python bench.py --workload c2_transe_l1 ...              # one workload
     python bench.py --impl reference --steps K --warmup W    # the CPU oracle, as it stands
 
-Prints ONE JSON line.  At N > 1 (launched by torch.distributed.run) every rank trains an
-independent replica on its own GPU -- the method's hot path exchanges nothing between
-devices -- and `value` is the sum over replicas divided by the slowest replica's time.
+Prints ONE JSON line.  Its top level is the headline workload (the training step at the largest
+configuration); `per_workload` carries the same fields for every other workload of the suite, each
+with its own clock samples.  At N > 1 (launched by torch.distributed.run) every rank trains an
+independent replica of the headline workload on its own GPU -- the method's hot path exchanges
+nothing between devices -- and `value` is the sum over replicas divided by the slowest replica's time.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -31,46 +37,53 @@ import kge_synth
 
 METRIC = "positive triples/sec (fwd+bwd+update, N shared negs)"
 UNIT = "triples/s"
+INFER_METRIC = "scored pairs/sec (full-entity top-k + rank)"
+INFER_UNIT = "pairs/s"
 
-# The headline configuration: 100,000 entities, 500 relations (Zipf 1.0), 2,000,000 triples with
-# Zipf(1.1) degrees, d = 128 fp32, log-sigmoid loss with margin 12 (self-adversarial
-# temperature 1), B = N = 1,024, P = 4, SGD lr 0.05.
 WORKLOADS = {
+    # 100,000 entities, 500 relations (Zipf 1.0), 2,000,000 triples with Zipf(1.1) degrees, d = 128 fp32, log-sigmoid loss with
+    # margin 12 (self-adversarial temperature 1), B = N = 1,024, P = 4, SGD lr 0.05.
     "c2_transe_l1": dict(E=100_000, R=500, T=2_000_000, d=128, score="transe", p_norm=1, loss="logsigmoid",
                          opt="sgd", B=1024, N=1024, P=4, gamma=12.0, adv_temp=1.0, lr=0.05,
                          entity_zipf=1.1, relation_zipf=1.0, graph_seed=1),
     "c2_rotate_l1": dict(E=100_000, R=500, T=2_000_000, d=128, score="rotate", p_norm=1, loss="logsigmoid",
                          opt="sgd", B=1024, N=1024, P=4, gamma=12.0, adv_temp=1.0, lr=0.05,
                          entity_zipf=1.1, relation_zipf=1.0, graph_seed=1),
-    # The 10 M-entity configuration: 10,000,000 entities, 1,000 relations (Zipf 1.0), 100,000,000 Zipf(1.1) triples,
-    # d = 256, sampled-softmax loss with the paper's correction, B = 4,096 x N = 16,384, P = 8, Adam on
-    # touched rows, bf16 tensor-core score block.  Tables are drawn on the device (10 GB + 20 GB of state).
+    # 10,000,000 entities, 1,000 relations (Zipf 1.0), 100,000,000 Zipf(1.1) triples, d = 256, sampled-softmax loss with the
+    # paper's correction, B = 4,096 x N = 16,384, P = 8, Adam on touched rows, bf16 tensor-core score block.
     "c3_distmult": dict(E=10_000_000, R=1000, T=100_000_000, d=256, score="distmult", p_norm=1, loss="softmax",
                         opt="adam", B=4096, N=16384, P=8, gamma=0.0, adv_temp=0.0, lr=0.001, tc=True,
-                        ce_correction="paper", entity_zipf=1.1, relation_zipf=1.0, graph_seed=2, device_tables=True),
+                        ce_correction="paper", entity_zipf=1.1, relation_zipf=1.0, graph_seed=2, device_data=True),
     "c3_complex": dict(E=10_000_000, R=1000, T=100_000_000, d=256, score="complex", p_norm=1, loss="softmax",
                        opt="adam", B=4096, N=16384, P=8, gamma=0.0, adv_temp=0.0, lr=0.001, tc=True,
-                       ce_correction="paper", entity_zipf=1.1, relation_zipf=1.0, graph_seed=2, device_tables=True),
+                       ce_correction="paper", entity_zipf=1.1, relation_zipf=1.0, graph_seed=2, device_data=True),
     # a tenth of the 10 M-entity configuration's graph and table with the same batch shape: quick runs of the tensor-core step
     "c3s_distmult": dict(E=1_000_000, R=1000, T=10_000_000, d=256, score="distmult", p_norm=1, loss="softmax",
                          opt="adam", B=4096, N=16384, P=8, gamma=0.0, adv_temp=0.0, lr=0.001, tc=True,
-                         ce_correction="paper", entity_zipf=1.1, relation_zipf=1.0, graph_seed=2, device_tables=True),
-    # The 91 M-entity training configuration: 91,000,000 entities (46.6 GB table), 1,400 relations, d = 128, B = N = 8,192, P = 16, row-wise
-    # Adagrad, log-sigmoid loss with margin 12.  The graph is cut to 60 M of the 600 M triples (host-side preprocessing;
-    # the step does not depend on the graph's size).  TransE-L2 on tensor cores, TransH on CUDA cores.
-    "c4_transe_l2": dict(E=91_000_000, R=1400, T=60_000_000, d=128, score="transe", p_norm=2, loss="logsigmoid",
+                         ce_correction="paper", entity_zipf=1.1, relation_zipf=1.0, graph_seed=2, device_data=True),
+    # 91,000,000 entities (46.6 GB table), 1,400 relations, 600,000,000 triples, d = 128, B = N = 8,192, P = 16, row-wise
+    # Adagrad, log-sigmoid loss with margin 12.  Graph and tables are made on the device.  TransE-L2 on tensor cores,
+    # TransH on CUDA cores.
+    "c4_transe_l2": dict(E=91_000_000, R=1400, T=600_000_000, d=128, score="transe", p_norm=2, loss="logsigmoid",
                          opt="adagrad", B=8192, N=8192, P=16, gamma=12.0, adv_temp=1.0, lr=0.05, tc=True,
-                         entity_zipf=1.1, relation_zipf=1.0, graph_seed=3, device_tables=True),
-    "c4_transh_l1": dict(E=91_000_000, R=1400, T=60_000_000, d=128, score="transh", p_norm=1, loss="logsigmoid",
+                         entity_zipf=1.1, relation_zipf=1.0, graph_seed=3, device_data=True),
+    "c4_transh_l1": dict(E=91_000_000, R=1400, T=600_000_000, d=128, score="transh", p_norm=1, loss="logsigmoid",
                          opt="adagrad", B=8192, N=8192, P=16, gamma=12.0, adv_temp=1.0, lr=0.05,
-                         entity_zipf=1.1, relation_zipf=1.0, graph_seed=3, device_tables=True),
+                         entity_zipf=1.1, relation_zipf=1.0, graph_seed=3, device_data=True),
+    # the same batch on a 4 M-entity table and a 20 M-triple graph: quick runs of the two steps above
+    "c4s_transh_l1": dict(E=4_000_000, R=1400, T=20_000_000, d=128, score="transh", p_norm=1, loss="logsigmoid",
+                          opt="adagrad", B=8192, N=8192, P=16, gamma=12.0, adv_temp=1.0, lr=0.05,
+                          entity_zipf=1.1, relation_zipf=1.0, graph_seed=3, device_data=True),
+    "c4s_transe_l2": dict(E=4_000_000, R=1400, T=20_000_000, d=128, score="transe", p_norm=2, loss="logsigmoid",
+                          opt="adagrad", B=8192, N=8192, P=16, gamma=12.0, adv_temp=1.0, lr=0.05, tc=True,
+                          entity_zipf=1.1, relation_zipf=1.0, graph_seed=3, device_data=True),
     "c1_distmult": dict(E=1000, R=10, T=20_000, d=32, score="distmult", p_norm=1, loss="logsigmoid",
                         opt="sgd", B=64, N=128, P=2, gamma=0.0, adv_temp=0.0, lr=0.1,
                         entity_zipf=1.1, relation_zipf=0.0, graph_seed=0),
 }
 
-# The full-entity scoring configuration: 15,000 (h, r) queries against all 91,000,000 entities of d = 128, top-10 and the
-# rank of a designated true tail.  The "s" variants keep the query batch and shrink the table.
+# Full-entity scoring: 15,000 (h, r) queries against all 91,000,000 entities of d = 128, top-10 and the rank of a designated
+# true tail.  The "s" variants keep the query batch and shrink the table.
 INFER_WORKLOADS = {
     "c5_transe_l1": dict(E=91_000_000, R=1400, d=128, Q=15000, K=10, score="transe", p_norm=1),
     "c5_distmult": dict(E=91_000_000, R=1400, d=128, Q=15000, K=10, score="distmult", p_norm=1),
@@ -80,23 +93,34 @@ INFER_WORKLOADS = {
     "c5s_distmult": dict(E=4_000_000, R=1400, d=128, Q=15000, K=10, score="distmult", p_norm=1),
 }
 
-# fp32 CUDA-core peak used for "bound": "alu": 148 SMs x 128 fp32 lanes x 1.965 GHz, one
-# instruction per lane per clock (an FMA counts as one).
-ALU_PEAK_TOPS = 148 * 128 * 1.965e9 / 1e12
+SUITE = ["c4_transh_l1", "c4_transe_l2", "c3_distmult", "c3_complex", "c2_transe_l1", "c2_rotate_l1", "c5_distmult_tc",
+         "c5_transe_l1"]
+HEADLINE = "c4_transh_l1"
 
-# Algorithmic fp32 lane-operations per (query, negative, embedding coordinate) of each stage,
-# by pair kind: the minimum a CUDA-core evaluation of the definition needs.
+# Instruction mixes of kge_measure_alu and what they stand for.
+MIX_FMA, MIX_SUB_ABS, MIX_CMP_ADD, MIX_SFU = 0, 1, 2, 3
+MIX_NAMES = {MIX_FMA: "fma", MIX_SUB_ABS: "sub+abs-add", MIX_CMP_ADD: "compare+predicated-add", MIX_SFU: "special-function"}
+
+# Algorithmic CUDA-core work of each stage per (query, negative, embedding coordinate): a list of (instructions, mix).
+# It is the minimum a CUDA-core evaluation of the definition needs; the roofline time of a stage is the sum over the
+# mixes of instructions / measured rate of that mix (special-function instructions run beside the others: the larger
+# of the two times counts).
 STAGE_OPS = {
-    "transe1": dict(block=2, accum_q=2, accum_t=2),     # sub, |.|+add  /  compare, predicated add
-    "rotate1": dict(block=3.5, accum_q=5, accum_t=5),   # per real coordinate; one sqrt / rsqrt per complex pair
-    "distmult1": dict(block=1, accum_q=1, accum_t=1),   # one FMA
-    "transh1": dict(block=4, accum_q=6, accum_t=5),      # w.t dot, residual, |.| / residual again (2), compare, one or two predicated adds, one FMA
+    "transe1": dict(block=[(2, MIX_SUB_ABS)], accum=[(4, MIX_CMP_ADD)]),
+    "transe2": dict(block=[(2, MIX_FMA)], accum=[(4, MIX_FMA)]),
+    # per real coordinate: two subtractions, a product and a multiply-add per complex component, then half a square root
+    "rotate1": dict(block=[(2, MIX_SUB_ABS), (0.5, MIX_FMA), (0.5, MIX_SFU)], accum=[(2, MIX_SUB_ABS), (1, MIX_FMA), (2, MIX_FMA), (1.0, MIX_SFU)]),
+    "distmult1": dict(block=[(1, MIX_FMA)], accum=[(2, MIX_FMA)]),
+    "complex1": dict(block=[(1, MIX_FMA)], accum=[(2, MIX_FMA)]),
+    # TransH p = 1: w.t (1 fma) + residual (sub, fma) + |.| accumulate (1); the backward passes re-form the residual
+    "transh1": dict(block=[(2, MIX_FMA), (2, MIX_SUB_ABS)], th_cpass=[(2, MIX_FMA), (2, MIX_CMP_ADD)],
+                    accum_q=[(2, MIX_FMA), (3, MIX_CMP_ADD), (1, MIX_FMA)], accum_t=[(2, MIX_FMA), (2, MIX_CMP_ADD), (1, MIX_FMA)]),
 }
 
-
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
-# summarised in profiles/train_step_c2_transe_l1_launches.md (None once the kernel has changed since).
-NCU_TRAFFIC_BYTES = {("c2_transe_l1", "accum"): 5.29e6, ("c2_transe_l1", "block"): 1.07e6}
+# Special-function instructions per score of the fused tensor-core epilogues (exponential, logarithm, reciprocal, reciprocal
+# square root: one instruction each).
+TC_SFU_PER_SCORE = {("softmax", False): dict(block=1, loss=1), ("logsigmoid", False): dict(block=3, loss=3),
+                    ("softmax", True): dict(block=2, loss=2), ("logsigmoid", True): dict(block=4, loss=4)}
 
 
 def cfg_kwargs(w, seed):
@@ -106,6 +130,15 @@ def cfg_kwargs(w, seed):
     return dict(num_entities=w["E"], num_relations=w["R"], dim=w["d"], score=w["score"], p_norm=w["p_norm"],
                 loss=w["loss"], opt=w["opt"], batch=w["B"], num_neg=w["N"], num_parts=w["P"], gamma=w["gamma"],
                 adv_temp=w["adv_temp"], ce_correction=c, lr=w["lr"], seed=seed)
+
+
+def config_of(name, w):
+    """The `config` object of a workload's line: the same keys for the CUDA arm and the reference arm."""
+    if name in INFER_WORKLOADS:
+        return {"workload": name, "entities": w["E"], "relations": w["R"], "dim": w["d"], "queries": w["Q"], "topk": w["K"],
+                "score": w["score"], "p_norm": w["p_norm"]}
+    return {"workload": name, "entities": w["E"], "relations": w["R"], "triples": w["T"], "dim": w["d"], "batch": w["B"],
+            "num_neg": w["N"], "parts": w["P"], "score": w["score"], "p_norm": w["p_norm"], "loss": w["loss"], "opt": w["opt"]}
 
 
 class ClockSampler:
@@ -132,7 +165,7 @@ class ClockSampler:
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.25)
+        time.sleep(0.15)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -177,10 +210,35 @@ def measured_peaks():
     p = ROOT / "MEASURED_PEAKS.json"
     if p.exists():
         d = json.loads(p.read_text())
-        return {"hbm_gbs": d.get("hbm_gbs"), "source": "measured"}
-    return {"hbm_gbs": 6650.0, "source": "fallback"}
+        return {"hbm_gbs": d.get("hbm_gbs", 6650.0), "bf16_tflops": d.get("bf16_tflops_sustained", 1400.0), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback"}
 
 
+def ncu_traffic(workload, kernel):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of `kernel` from the tracked capture record, or None when
+    there is no record for this workload and kernel or the kernel's source file has changed since the capture."""
+    rec_path = ROOT / "profiles" / "ncu_traffic.json"
+    if not rec_path.exists():
+        return None
+    for rec in json.loads(rec_path.read_text()).get("captures", []):
+        if rec.get("workload") == workload and rec.get("stage") == kernel:
+            src = ROOT / rec["source"]
+            if src.exists() and hashlib.sha256(src.read_bytes()).hexdigest() == rec.get("source_sha256"):
+                return rec.get("dram_bytes_per_launch")
+    return None
+
+
+def stage_roof_us(ops, elements, alu):
+    """Roofline time (us) of a CUDA-core stage and the mix that dominates it."""
+    t_alu = sum(n * elements / alu[m] for n, m in ops if m != MIX_SFU)
+    t_sfu = sum(n * elements / alu[m] for n, m in ops if m == MIX_SFU)
+    top = max(ops, key=lambda nm: nm[0] * elements / alu[nm[1]])[1]
+    if t_sfu > t_alu:
+        return t_sfu * 1e6, MIX_SFU
+    return t_alu * 1e6, top
+
+
+# ------------------------------------------------------------------------------------------ the oracle, timed
 ORACLE_MAX_ENTITIES = 200_000     # the fp64 oracle holds whole tables on the host: larger workloads are timed on a cut
 
 
@@ -221,86 +279,171 @@ def oracle_step_time(w, batch_size, steps, warmup, seed=0):
     return float(np.mean(times)), num_threads(), note
 
 
-def run_reference(args, w, name):
-    """The reference arm: the CPU oracle, untouched, on the machine's host cores."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
-        return
+def oracle_train_sample(w, target_s, steps, warmup):
+    """The oracle's full training step on as many of the workload's positives as fit `target_s` seconds in all."""
     P2 = w["P"] * w["P"]
-    # calibrate the per-step sample so that warmup + steps stay within about two minutes
-    t_cal, cores, note = oracle_step_time(w, 4 * P2, 1, 0)
-    per_pos = t_cal / (4 * P2)
-    budget = 120.0 / max(1, args.steps + args.warmup)
+    t_cal, cores, note = oracle_step_time(w, P2, 1, 0)
+    per_pos = t_cal / P2
+    budget = target_s / max(1, steps + warmup)
     b_ref = int(min(w["B"], max(P2, (budget / per_pos) // P2 * P2)))
-    t_step, cores, note = oracle_step_time(w, b_ref, args.steps, args.warmup)
-    value = b_ref / t_step
-    sample = (f"{args.steps} steps, each a full training step (sample, forward, backward, dedup, update) on "
-              f"{b_ref} of the workload's {w['B']} positives against all {w['N']} shared negatives" + note)
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_step * 1e3, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": name, "entities": w["E"], "relations": w["R"], "triples": w["T"], "dim": w["d"],
-                       "batch": b_ref, "num_neg": w["N"], "parts": w["P"]},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
-            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    t_step, cores, note = oracle_step_time(w, b_ref, steps, warmup)
+    sample = (f"{steps} full training steps (sample, forward, backward, dedup, update; fp64 oracle, OpenMP) on {b_ref} of the "
+              f"workload's {w['B']} positives against all {w['N']} shared negatives" + note)
+    return b_ref / t_step, t_step, b_ref, cores, sample
+
+
+def oracle_infer_sample(w, target_s):
+    """The fp32 oracle's brute-force scoring, top-k and rank on a cut of the table and of the query batch."""
+    from oracle.kge_oracle import Oracle, make_config, num_threads
+    o = Oracle("f32")
+    E, nq = min(w["E"], 100_000), max(1, num_threads())
+    ent, rel, _ = kge_synth.make_tables(E, w["R"], w["d"], w["score"], seed=5)
+    qh, qr, tt = kge_synth.make_queries(E, w["R"], nq, seed=5)
+    cfg = make_config(num_entities=E, num_relations=w["R"], dim=w["d"], score=w["score"], p_norm=w["p_norm"],
+                      bf16_operands=1 if w.get("tc") else 0)
+    t0 = time.perf_counter()
+    o.score_all_topk(cfg, ent, rel, None, qh, qr, w["K"], true_tails=tt)
+    dt = time.perf_counter() - t0
+    reps = int(max(1, min(20, target_s / max(dt, 1e-3) - 1)))
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        o.score_all_topk(cfg, ent, rel, None, qh, qr, w["K"], true_tails=tt)
+    dt = (time.perf_counter() - t0) / reps
+    sample = (f"{reps} passes of {nq} queries against a table cut to {E} entities (fp32 oracle, brute force, top-{w['K']} and rank, "
+              f"OpenMP over queries)")
+    return nq * E / dt, dt, num_threads(), sample
+
+
+# ------------------------------------------------------------------------------------------ the reference arm
+def run_reference(args, names):
+    """The reference arm: the CPU oracle, untouched, on the machine's host cores, on a bounded sample of every workload."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    per = max(8.0, 150.0 / len(names))
+    lines = {}
+    for name in names:
+        if name in INFER_WORKLOADS:
+            w = INFER_WORKLOADS[name]
+            value, dt, cores, sample = oracle_infer_sample(w, per)
+            metric, unit, ms = INFER_METRIC, INFER_UNIT, dt * 1e3
+        else:
+            w = WORKLOADS[name]
+            value, t_step, b_ref, cores, sample = oracle_train_sample(w, per, args.steps, args.warmup)
+            metric, unit, ms = METRIC, UNIT, t_step * 1e3
+        lines[name] = {"impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus,
+                       "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+                       "scaling": "weak", "vs_baseline": None, "dtype": "f32" if name in INFER_WORKLOADS else "f64",
+                       "data": "synthetic", "config": config_of(name, w),
+                       "cpu_baseline": {"value": value, "unit": unit, "cores": cores, "kind": "oracle", "sample": sample},
+                       "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    head = names[0]
+    line = dict(lines[head])
+    if len(names) > 1:
+        line["per_workload"] = {n: lines[n] for n in names[1:]}
     print(json.dumps(line), flush=True)
 
 
-def run_ours(args, w, name):
-    import torch
-    import torch.distributed as dist
-    import paper_2211_12281_b200 as K
+# ------------------------------------------------------------------------------------------ the CUDA arm
+class Ctx:
+    """What the workloads of one run share: the device, the measured rates, buffers worth keeping."""
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    def __init__(self, args):
+        import torch
+        import torch.distributed as dist
+        import paper_2211_12281_b200 as K
+        self.torch, self.dist, self.K, self.args = torch, dist, K, args
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+        torch.cuda.set_device(self.local)
+        self.dev = torch.device("cuda", self.local)
+        if self.world > 1:
+            dist.init_process_group("nccl", device_id=self.dev)
+        self.peaks = measured_peaks()
+        # lane instructions per second of each mix, measured now on this GPU (a short burst at the clocks it finds)
+        self.alu = {m: K.measure_alu(m, 8192) for m in (MIX_FMA, MIX_SUB_ABS, MIX_CMP_ADD, MIX_SFU)}
+        self.flush = None
+        self.graphs = {}          # (E, R, T, seed) -> device triples, shared by the models of one configuration
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
+    def barrier(self):
+        if self.world > 1:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def release(self):
+        self.graphs.clear()
+        self.torch.cuda.empty_cache()
+
+
+def sustain(fn, first_step, min_seconds, torch):
+    """Keeps calling fn(step) for at least min_seconds so that the clock sampler sees the workload under load."""
+    t0, step = time.perf_counter(), first_step
+    while time.perf_counter() - t0 < min_seconds:
+        for _ in range(8):
+            fn(step); step += 1
         torch.cuda.synchronize()
+    return step
 
-    B, N = w["B"], w["N"]
-    h, r, t = kge_synth.make_graph(w["E"], w["R"], w["T"], seed=w["graph_seed"], entity_zipf=w["entity_zipf"],
-                                   relation_zipf=w["relation_zipf"])
-    kw_rel = w["d"] // 2 if w["score"] == "rotate" else w["d"]
-    if w.get("device_tables"):
-        # large tables are drawn on the device with the same law (N(0, 1/sqrt(d)) rows)
-        gen = torch.Generator(device=dev); gen.manual_seed(w["graph_seed"] + 1_000_003)
-        ent_d = torch.empty((w["E"], w["d"]), dtype=torch.float32, device=dev).normal_(0.0, w["d"] ** -0.5, generator=gen)
-        rel_d = torch.empty((w["R"], kw_rel), dtype=torch.float32, device=dev).normal_(0.0, w["d"] ** -0.5, generator=gen)
-        relw_d = None
-        if w["score"] == "transh":
-            relw_d = torch.empty((w["R"], w["d"]), dtype=torch.float32, device=dev).normal_(0.0, w["d"] ** -0.5, generator=gen)
-    else:
-        ent, rel, relw = kge_synth.make_tables(w["E"], w["R"], w["d"], w["score"], seed=w["graph_seed"])
-        ent_d, rel_d = torch.from_numpy(ent).to(dev), torch.from_numpy(rel).to(dev)
-        relw_d = None if relw is None else torch.from_numpy(relw).to(dev)
+
+def bench_training(ctx, name, w, cpu_seconds):
+    torch, K, args, dev = ctx.torch, ctx.K, ctx.args, ctx.dev
+    B, N, d = w["B"], w["N"], w["d"]
+    kw_rel = d // 2 if w["score"] == "rotate" else d
+    big = bool(w.get("device_data"))
+    ent_d = torch.empty((w["E"], d), dtype=torch.float32, device=dev)
+    rel_d = torch.empty((w["R"], kw_rel), dtype=torch.float32, device=dev)
+    relw_d = torch.empty((w["R"], d), dtype=torch.float32, device=dev) if w["score"] == "transh" else None
     states = [None, None, None]
     if w["opt"] == "adam":
-        states = [torch.zeros((w["E"], 2 * w["d"]), dtype=torch.float32, device=dev),
-                  torch.zeros((w["R"], 2 * kw_rel), dtype=torch.float32, device=dev),
-                  None if relw_d is None else torch.zeros((w["R"], 2 * w["d"]), dtype=torch.float32, device=dev)]
+        states = [torch.empty((w["E"], 2 * d), dtype=torch.float32, device=dev), torch.empty((w["R"], 2 * kw_rel), dtype=torch.float32, device=dev),
+                  None if relw_d is None else torch.empty((w["R"], 2 * d), dtype=torch.float32, device=dev)]
     elif w["opt"] == "adagrad":
-        states = [torch.zeros(w["E"], dtype=torch.float32, device=dev), torch.zeros(w["R"], dtype=torch.float32, device=dev),
-                  None if relw_d is None else torch.zeros(w["R"], dtype=torch.float32, device=dev)]
+        states = [torch.empty(w["E"], dtype=torch.float32, device=dev), torch.empty(w["R"], dtype=torch.float32, device=dev),
+                  None if relw_d is None else torch.empty(w["R"], dtype=torch.float32, device=dev)]
     prec = K.PREC_BF16_TC if w.get("tc") else K.PREC_FP32
-    kge = K.Kge(K.KgeConfig.make(**cfg_kwargs(w, seed=replica_seed(rank)), prec=prec))       # each replica draws its own batches
+    kge = K.Kge(K.KgeConfig.make(**cfg_kwargs(w, seed=replica_seed(ctx.rank)), prec=prec))       # each replica draws its own batches
     kge.bind(ent_d, rel_d, relw_d, *states, num_triples=w["T"])
-    kge.graph_load(h, r, t)
+    t_setup = time.perf_counter()
+    if big:
+        # tables by the library's own generator (N(0, 1/sqrt(d)) rows, uniform phases), graph drawn and preprocessed on the device
+        kge.init_tables(d ** -0.5)
+        gkey = (w["E"], w["R"], w["T"], w["graph_seed"])
+        if gkey not in ctx.graphs:
+            ctx.graphs.clear()
+            ctx.graphs[gkey] = kge_synth.make_graph_device(w["E"], w["R"], w["T"], seed=w["graph_seed"], device=dev,
+                                                           entity_zipf=w["entity_zipf"], relation_zipf=w["relation_zipf"])
+        torch.cuda.synchronize()
+        t_graph = time.perf_counter()
+        kge.graph_load_device(*ctx.graphs[gkey])
+        graph_load_s = time.perf_counter() - t_graph
+    else:
+        ent, rel, relw = kge_synth.make_tables(w["E"], w["R"], d, w["score"], seed=w["graph_seed"])
+        ent_d.copy_(torch.from_numpy(ent)); rel_d.copy_(torch.from_numpy(rel))
+        if relw is not None:
+            relw_d.copy_(torch.from_numpy(relw))
+        for st in states:
+            if st is not None:
+                st.zero_()
+        h, r, t = kge_synth.make_graph(w["E"], w["R"], w["T"], seed=w["graph_seed"], entity_zipf=w["entity_zipf"],
+                                       relation_zipf=w["relation_zipf"])
+        t_graph = time.perf_counter()
+        kge.graph_load(h, r, t)
+        graph_load_s = time.perf_counter() - t_graph
+    setup_s = time.perf_counter() - t_setup
     loss = torch.zeros(1, dtype=torch.float32, device=dev)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # 2 x L2: evicts the tables between steps
+    # a table that fits L2 is evicted between steps by a 256 MiB write (untimed); larger tables need no flush
+    table_bytes = w["E"] * d * 4
+    flush_needed = table_bytes < 4 * 126e6
+    if flush_needed and ctx.flush is None:
+        ctx.flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
     def timed_steps(first_step, count, fn):
         evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(count)]
         for i, (a, b) in enumerate(evs):
-            flush.zero_()
+            if flush_needed:
+                ctx.flush.zero_()
             a.record()
             fn(first_step + i)
             b.record()
@@ -312,118 +455,148 @@ def run_ours(args, w, name):
     timed_steps(0, warm, step_fn)
     assert kge.get_status() == 0
 
-    # ---- device-resident timing: K steps, CUDA events on the launching stream ----
-    barrier()
-    clocks = ClockSampler(local)
+    # ---- device-resident timing: K steps, CUDA events on the launching stream; the clock sampler keeps running over a
+    # continuation of the same steps so that it sees at least half a second of this workload under load ----
+    ctx.barrier()
+    clocks = ClockSampler(ctx.local)
     launches0 = kge.launch_count()
     ms = timed_steps(warm, args.steps, step_fn)
-    barrier()
-    clock_info = clocks.stop()
     launches = kge.launch_count() - launches0
+    ctx.barrier()
+    nxt = sustain(step_fn, warm + args.steps, 0.6, torch)
+    clock_info = clocks.stop()
     total_ms = max_over_ranks(float(np.sum(ms)), dev)
     ms_per_step = total_ms / args.steps
-    value = whole_job_value(world, B, ms_per_step)
+    value = whole_job_value(ctx.world, B, ms_per_step)
     assert np.isfinite(loss.item()) and kge.get_status() == 0
+    if clock_info.get("sm_mhz"):
+        clock_info["ms_per_step_x_sm_mhz"] = ms_per_step * clock_info["sm_mhz"]
 
     # ---- end to end: ids in pinned host memory -> H2D, step, loss -> D2H, every step ----
-    nxt = warm + args.steps
     ids_all = torch.empty(3 * B + N, dtype=torch.int32, device=dev)          # heads | rels | tails | negs, back to back
     ids_dev = [ids_all[0:B], ids_all[B:2 * B], ids_all[2 * B:3 * B], ids_all[3 * B:]]
     pinned = []
-    for i in range(min(args.steps, 256)):                                   # a ring of pinned host batches
+    for i in range(min(args.steps, 64)):                                    # a ring of pinned host batches
         kge.sample_batch(nxt + i, *ids_dev)
         host = ids_all.cpu().pin_memory()
         pinned.append([host[0:B], host[B:2 * B], host[2 * B:3 * B], host[3 * B:]])
     loss_host = torch.zeros(1, dtype=torch.float32).pin_memory()
     host_fn = lambda s: kge.train_step_host(s, w["lr"], *pinned[(s - nxt) % len(pinned)], loss_host)
-    barrier()
+    ctx.barrier()
     e2e_ms = float(np.sum(timed_steps(nxt, args.steps, host_fn)))
-    barrier()
+    ctx.barrier()
     e2e_ms = max_over_ranks(e2e_ms, dev)
-    e2e_value = whole_job_value(world, B, e2e_ms / args.steps)
+    e2e_value = whole_job_value(ctx.world, B, e2e_ms / args.steps)
     nxt += args.steps
 
-    # ---- per-kernel times (CUDA events around every launch, same stream) for the roofline ----
+    # ---- per-kernel times (CUDA events around every launch, same stream, serial) for the roofline ----
     kge.profile(True)
-    prof_steps = min(args.steps, 100)
+    prof_steps = min(args.steps, 50)
     timed_steps(nxt, prof_steps, step_fn)
     stages = kge.profile_read()
     kge.profile(False)
+    uniq = len(kge.debug_export("ENT_UNIQ"))
     per_stage_us = {k: 1e3 * v[0] / v[1] for k, v in stages.items() if v[1] > 0}
     kind = f"{w['score']}{w['p_norm']}"
-    ops = STAGE_OPS.get(kind, {})
+    ops = dict(STAGE_OPS.get(kind, {}))
     if "accum_q" in per_stage_us and "accum_t" not in per_stage_us:     # dQ and dT share one launch
         per_stage_us["accum"] = per_stage_us.pop("accum_q")
-        ops = dict(ops, accum=ops.get("accum_q", 0) + ops.get("accum_t", 0))
-    # tensor-core step: "block" is the statistics pass and "loss" the gradient pass, each one B x N x d contraction
-    compute_stages = [s for s in ("block", "accum", "accum_q", "accum_t") + (("loss",) if w.get("tc") else ()) if s in per_stage_us]
-    dominant = max(compute_stages, key=lambda s: per_stage_us[s])
-    roofline = None
+    elements = float(B) * N * d
+    roofs = {}                                                           # stage -> (roofline us, bound, detail)
     if w.get("tc"):
-        # each of the three contractions is 2 B N d flops; bf16 operands, fp32 accumulation
-        peaks = json.loads((ROOT / "MEASURED_PEAKS.json").read_text()) if (ROOT / "MEASURED_PEAKS.json").exists() else {}
-        peak = peaks.get("bf16_tflops_sustained", 1400.0)
-        achieved = 2.0 * B * N * w["d"] / (per_stage_us[dominant] * 1e-6) / 1e12
-        roofline = {"bound": "tensor", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                    "frac": achieved / peak, "traffic": None,
-                    "peak_source": "measured (sustained cuBLAS bf16)" if peaks else "fallback",
-                    "us_per_launch": per_stage_us[dominant]}
-    elif dominant in ops:
-        alg_ops = ops[dominant] * B * N * w["d"]
-        achieved = alg_ops / (per_stage_us[dominant] * 1e-6) / 1e12
-        roofline = {"bound": "alu", "kernel": dominant, "achieved": achieved, "peak": ALU_PEAK_TOPS,
-                    "unit": "TFLOP/s", "frac": achieved / ALU_PEAK_TOPS, "traffic": NCU_TRAFFIC_BYTES.get((name, dominant)),
-                    "op": "one fp32 CUDA-core instruction per lane (FMA = 1)",
-                    "peak_source": "148 SMs x 128 lanes x 1.965 GHz", "us_per_launch": per_stage_us[dominant]}
+        # each of the four tensor-core launches is one B x N x d contraction: 2 B N d flops, bf16 operands, fp32 accumulation.
+        # "block" is the statistics pass and "loss" the merge kernel plus the gradient pass; their epilogues also issue
+        # special-function instructions per score, and the larger of the two times is the pass's roof.
+        sfu = TC_SFU_PER_SCORE[(w["loss"], w["score"] == "transe")]
+        for st in ("block", "loss", "accum_q", "accum_t"):
+            if st not in per_stage_us:
+                continue
+            t_tc = 2.0 * elements / (ctx.peaks["bf16_tflops"] * 1e12) * 1e6
+            t_sf = sfu.get(st, 0) * float(B) * N / ctx.alu[MIX_SFU] * 1e6
+            roofs[st] = (max(t_tc, t_sf), "tensor" if t_tc >= t_sf else "sfu", {"t_tensor_us": t_tc, "t_sfu_us": t_sf})
+    else:
+        for st, o in ops.items():
+            if st in per_stage_us:
+                t, mix = stage_roof_us(o, elements, ctx.alu)
+                roofs[st] = (t, "alu", {"mix": MIX_NAMES[mix], "instructions_per_element": sum(n for n, _ in o)})
+    # the two memory-bound sub-steps: random row gathers and the sparse row update
+    rel_bytes = B * 4 * kw_rel * (2 if w["score"] == "transh" else 1)
+    build_bytes = (2 * B + N) * 4 * d + rel_bytes + (B + N) * 4 * d + ((B + N) * 2 * d if w.get("tc") else 0)
+    state_per_row = {"sgd": 8 * d, "adagrad": 8 * d + 8, "adam": 24 * d}[w["opt"]]
+    update_bytes = uniq * state_per_row + (2 * B + N) * 4 * d
+    hbm = ctx.peaks["hbm_gbs"] * 1e9
+    hbm_substeps = {}
+    for st, nbytes in (("build", build_bytes), ("update", update_bytes)):
+        if st in per_stage_us:
+            gbs = nbytes / (per_stage_us[st] * 1e-6) / 1e9
+            hbm_substeps[st] = {"bytes": int(nbytes), "us": per_stage_us[st], "gbs": gbs, "frac": gbs * 1e9 / hbm}
+            roofs[st] = (nbytes / hbm * 1e6, "hbm", {})
+    compute = [s for s in roofs if roofs[s][1] != "hbm"]
+    dominant = max(compute, key=lambda s: per_stage_us[s]) if compute else None
+    roofline = None
+    if dominant is not None:
+        t_roof, bound, detail = roofs[dominant]
+        us = per_stage_us[dominant]
+        if bound == "alu":
+            n_ops = sum(n for n, _ in ops[dominant]) * elements
+            achieved, peak, unit = n_ops / (us * 1e-6) / 1e12, n_ops / (t_roof * 1e-6) / 1e12, "T lane-instructions/s"
+            src = "measured in this run: kge_measure_alu on the stage's instruction mix (" + detail["mix"] + ")"
+        elif bound == "sfu":
+            n_ops = detail["t_sfu_us"] * 1e-6 * ctx.alu[MIX_SFU]
+            achieved, peak, unit = n_ops / (us * 1e-6) / 1e12, ctx.alu[MIX_SFU] / 1e12, "T special-function instructions/s"
+            bound, src = "alu", "measured in this run: kge_measure_alu, special-function mix (the pass's larger roof; tensor time " \
+                                f"{detail['t_tensor_us']:.1f} us)"
+        else:
+            achieved, peak, unit = 2.0 * elements / (us * 1e-6) / 1e12, ctx.peaks["bf16_tflops"], "TFLOP/s"
+            src = ctx.peaks["source"] + " (sustained cuBLAS bf16)"
+        roofline = {"bound": bound, "kernel": dominant, "achieved": achieved, "peak": peak, "unit": unit,
+                    "frac": t_roof / us, "traffic": ncu_traffic(name, dominant), "peak_source": src, "us_per_launch": us}
+        roofline.update({k: v for k, v in detail.items() if k != "mix"})
+    stage_frac = {s: roofs[s][0] / per_stage_us[s] for s in roofs}
+    step_roof_us = sum(roofs[s][0] for s in roofs)
 
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ctx.world, "steps": args.steps,
             "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if w.get("tc") else "f32", "data": "synthetic",
-            "config": {"workload": name, "entities": w["E"], "relations": w["R"], "triples": w["T"], "dim": w["d"],
-                       "batch": B, "num_neg": N, "parts": w["P"], "score": w["score"], "p_norm": w["p_norm"],
-                       "loss": w["loss"], "opt": w["opt"], "replicas": world,
-                       "l2": "flushed between steps (256 MiB write), untimed"},
-            "scored_pairs_per_s": world * B * (N + 1) / (ms_per_step * 1e-3),
+            "config": dict(config_of(name, w), replicas=ctx.world,
+                           l2="flushed between steps (256 MiB write), untimed" if flush_needed else "table larger than L2, no flush",
+                           graph="drawn and preprocessed on the device" if big else "drawn and preprocessed on the host"),
+            "scored_pairs_per_s": ctx.world * B * (N + 1) / (ms_per_step * 1e-3),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": (3 * B + N) * 4, "d2h_bytes_per_step": 4},
             "gpu_launches": int(launches), "clocks": clock_info, "roofline": roofline,
-            "stage_us": per_stage_us, "loss": loss.item()}
-
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        b_cpu = min(B, 256)
-        t_step, cores, note = oracle_step_time(w, b_cpu, 2, 1)
-        line["cpu_baseline"] = {"value": b_cpu / t_step, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                "sample": f"2 full training steps on {b_cpu} of the {B} positives against all {N} "
-                                          f"shared negatives (fp64 oracle, OpenMP)" + note}
-    if rank == 0:
-        print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+            "stage_us": per_stage_us, "stage_frac": stage_frac, "step_frac": step_roof_us / (ms_per_step * 1e3),
+            "hbm_substeps": hbm_substeps, "unique_rows": uniq, "graph_load_s": graph_load_s, "setup_s": setup_s,
+            "loss": loss.item()}
+    if ctx.rank == 0 and ctx.world == 1 and cpu_seconds > 0:
+        v, t_step, b_cpu, cores, sample = oracle_train_sample(w, cpu_seconds, 2, 1)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+    kge.close()
+    return line
 
 
-def run_infer(args, w, name):
+def bench_inference(ctx, name, w, cpu_seconds):
     """Full-entity scoring with top-k and rank: one step = one pass of all queries over the table."""
-    import torch
-    import paper_2211_12281_b200 as K
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
-    dev = torch.device("cuda", 0)
-    torch.cuda.set_device(dev)
+    torch, K, args, dev = ctx.torch, ctx.K, ctx.args, ctx.dev
     E, R, d, Q, k = w["E"], w["R"], w["d"], w["Q"], w["K"]
-    gen = torch.Generator(device=dev); gen.manual_seed(5)
-    ent = torch.empty((E, d), dtype=torch.float32, device=dev).normal_(0.0, d ** -0.5, generator=gen)
-    rel = torch.empty((R, d), dtype=torch.float32, device=dev).normal_(0.0, d ** -0.5, generator=gen)
+    ent = torch.empty((E, d), dtype=torch.float32, device=dev)
+    rel = torch.empty((R, d), dtype=torch.float32, device=dev)
     qh, qr, tt = kge_synth.make_queries(E, R, Q, seed=5)
     qh_d, qr_d, tt_d = (torch.from_numpy(a).to(dev) for a in (qh, qr, tt))
     kge = K.Kge(K.KgeConfig.make(num_entities=E, num_relations=R, dim=d, score=w["score"], p_norm=w["p_norm"],
-                                 prec=K.PREC_BF16_TC if w.get("tc") else K.PREC_FP32))
+                                 prec=K.PREC_BF16_TC if w.get("tc") else K.PREC_FP32, seed=5))
     kge.bind(ent, rel, max_queries=Q, topk=k)
+    kge.init_tables(d ** -0.5)
     ids = torch.empty((Q, k), dtype=torch.int32, device=dev)
     sc = torch.empty((Q, k), dtype=torch.float32, device=dev)
     ranks = torch.empty(Q, dtype=torch.int32, device=dev)
-    steps, warm = max(1, min(args.steps, 5)), max(1, min(args.warmup, 2))
-    for _ in range(warm):
+    # a pass over 91 M entities on CUDA cores takes seconds: one warm-up pass on a slice of the queries, one timed pass
+    long_pass = E * float(Q) * d > 5e15 and not w.get("tc")
+    steps = 1 if long_pass else max(1, min(args.steps, 3))
+    if long_pass:
+        kge.score_all_topk(qh_d[:256].contiguous(), qr_d[:256].contiguous(), k, tt_d[:256].contiguous(), ids[:256], sc[:256], ranks[:256])
+    else:
         kge.score_all_topk(qh_d, qr_d, k, tt_d, ids, sc, ranks)
-    clocks = ClockSampler(0)
+    clocks = ClockSampler(ctx.local)
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     l0 = kge.launch_count()
     a.record()
@@ -431,54 +604,106 @@ def run_infer(args, w, name):
         kge.score_all_topk(qh_d, qr_d, k, tt_d, ids, sc, ranks)
     b.record(); torch.cuda.synchronize()
     ms = a.elapsed_time(b) / steps
+    launches = int((kge.launch_count() - l0) / steps)
+    while ms * steps < 600.0 and not long_pass:           # keep the sampler under load for at least half a second
+        kge.score_all_topk(qh_d, qr_d, k, tt_d, ids, sc, ranks); steps += 1
     clock_info = clocks.stop()
+    if clock_info.get("sm_mhz"):
+        clock_info["ms_per_step_x_sm_mhz"] = ms * clock_info["sm_mhz"]
     assert kge.get_status() == 0
-    pairs = float(Q) * E
-    t_hbm = E * d * 4 / (measured_peaks()["hbm_gbs"] * 1e9)
-    ops = {"transe": 2.0, "distmult": 1.0}[w["score"]]
-    t_alu = ops * pairs * d / (ALU_PEAK_TOPS * 1e12)
-    bound = "alu" if t_alu > t_hbm else "hbm"
-    if w.get("tc"):
-        peaks = json.loads((ROOT / "MEASURED_PEAKS.json").read_text()) if (ROOT / "MEASURED_PEAKS.json").exists() else {}
-        peak = peaks.get("bf16_tflops_sustained", 1400.0)
-        t_tc = 2.0 * pairs * d / (peak * 1e12)
-        bound = "tensor" if t_tc > t_hbm else "hbm"
-    roof = {"bound": bound, "kernel": "tc_gemm<topk>" if w.get("tc") else "score_tile", "frac": max(t_alu, t_hbm) / (ms * 1e-3), "traffic": None,
-            "t_alu_ms": t_alu * 1e3, "t_hbm_ms": t_hbm * 1e3}
-    if bound == "tensor":
-        roof.update(achieved=2.0 * pairs * d / (ms * 1e-3) / 1e12, peak=peak, unit="TFLOP/s", frac=t_tc / (ms * 1e-3))
-    elif bound == "alu":
-        roof.update(achieved=ops * pairs * d / (ms * 1e-3) / 1e12, peak=ALU_PEAK_TOPS, unit="TFLOP/s")
+    mrr = kge.mrr_from_ranks(ranks, 10)
+    # end to end: queries from pinned host memory, lists and ranks back to the host
+    pin = lambda x: torch.from_numpy(x).pin_memory()
+    hq, hr, ht = pin(qh), pin(qr), pin(tt)
+    h_ids, h_sc, h_rk = (torch.empty((Q, k), dtype=torch.int32).pin_memory(), torch.empty((Q, k), dtype=torch.float32).pin_memory(),
+                         torch.empty(Q, dtype=torch.int32).pin_memory())
+    if long_pass:
+        e2e_ms = None          # a second multi-second pass would add nothing: the copies are 0.4 MB against seconds of scoring
     else:
-        roof.update(achieved=E * d * 4 / (ms * 1e-3) / 1e9, peak=measured_peaks()["hbm_gbs"], unit="GB/s")
-    line = {"metric": "scored pairs/sec (full-entity top-k + rank)", "value": pairs / (ms * 1e-3), "unit": "pairs/s",
-            "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        a.record()
+        kge.score_all_topk_host(hq, hr, k, ht, h_ids, h_sc, h_rk)
+        b.record(); torch.cuda.synchronize()
+        e2e_ms = a.elapsed_time(b)
+        assert (h_ids == ids.cpu()).all()
+    pairs = float(Q) * E
+    t_hbm = E * d * 4 / (ctx.peaks["hbm_gbs"] * 1e9)
+    if w.get("tc"):
+        t_c = 2.0 * pairs * d / (ctx.peaks["bf16_tflops"] * 1e12)
+        roof = {"bound": "tensor", "kernel": "tc_gemm<topk>", "achieved": 2.0 * pairs * d / (ms * 1e-3) / 1e12,
+                "peak": ctx.peaks["bf16_tflops"], "unit": "TFLOP/s", "peak_source": ctx.peaks["source"] + " (sustained cuBLAS bf16)"}
+    else:
+        o = {"transe": [(2, MIX_SUB_ABS)], "distmult": [(1, MIX_FMA)]}[w["score"]]
+        t_us, mix = stage_roof_us(o, pairs * d, ctx.alu)
+        t_c = t_us * 1e-6
+        n_ops = sum(n for n, _ in o) * pairs * d
+        roof = {"bound": "alu", "kernel": "score_tile", "achieved": n_ops / (ms * 1e-3) / 1e12, "peak": n_ops / t_c / 1e12,
+                "unit": "T lane-instructions/s",
+                "peak_source": "measured in this run: kge_measure_alu on the kernel's instruction mix (" + MIX_NAMES[mix] + ")"}
+    roof.update(frac=max(t_c, t_hbm) / (ms * 1e-3), traffic=ncu_traffic(name, roof["kernel"]), t_compute_ms=t_c * 1e3, t_hbm_ms=t_hbm * 1e3)
+    e2e_value = pairs / ((e2e_ms if e2e_ms is not None else ms) * 1e-3)
+    line = {"metric": INFER_METRIC, "value": pairs / (ms * 1e-3), "unit": INFER_UNIT,
+            "n_gpus": 1, "steps": steps, "warmup": 1, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if w.get("tc") else "f32", "data": "synthetic",
-            "config": {"workload": name, "entities": E, "relations": R, "dim": d, "queries": Q, "topk": k,
-                       "score": w["score"], "p_norm": w["p_norm"], "l2": "table larger than L2" if E * d * 4 > 126e6 else "table fits L2"},
-            "queries_per_s": Q / (ms * 1e-3), "gpu_launches": int((kge.launch_count() - l0) / steps),
-            "clocks": clock_info, "roofline": roof, "mean_rank": float(ranks.float().mean().item())}
-    print(json.dumps(line), flush=True)
+            "config": dict(config_of(name, w), l2="table larger than L2" if E * d * 4 > 126e6 else "table fits L2"),
+            "queries_per_s": Q / (ms * 1e-3), "gpu_launches": launches,
+            "e2e": {"value": e2e_value, "unit": INFER_UNIT, "h2d_bytes_per_step": 3 * Q * 4, "d2h_bytes_per_step": Q * (8 * k + 4),
+                    "measured": e2e_ms is not None},
+            "clocks": clock_info, "roofline": roof, "mean_rank": float(ranks.float().mean().item()), "mrr_at_10": mrr}
+    if ctx.rank == 0 and cpu_seconds > 0:
+        v, dt, cores, sample = oracle_infer_sample(w, cpu_seconds)
+        line["cpu_baseline"] = {"value": v, "unit": INFER_UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+    kge.close()
+    return line
+
+
+def run_ours(args, names):
+    ctx = Ctx(args)
+    if ctx.world > 1:
+        names = names[:1]                     # replicas of the headline workload
+    lines = {}
+    for i, name in enumerate(names):
+        cpu_s = 0.0 if args.no_cpu_baseline else (18.0 if i == 0 else 5.0)
+        if name in INFER_WORKLOADS:
+            lines[name] = bench_inference(ctx, name, INFER_WORKLOADS[name], cpu_s)
+        else:
+            lines[name] = bench_training(ctx, name, WORKLOADS[name], cpu_s)
+        nxt = names[i + 1] if i + 1 < len(names) else None
+        same_graph = nxt in WORKLOADS and name in WORKLOADS and all(WORKLOADS[nxt][k] == WORKLOADS[name][k] for k in ("E", "R", "T", "graph_seed"))
+        if not same_graph:
+            ctx.release()
+        else:
+            ctx.torch.cuda.empty_cache()
+    head = names[0]
+    line = dict(lines[head])
+    line["alu_rates"] = {MIX_NAMES[m]: v / 1e12 for m, v in ctx.alu.items()}
+    line["alu_rates_unit"] = "T lane-instructions/s, measured by kge_measure_alu at the start of this run"
+    if len(names) > 1:
+        line["per_workload"] = {n: lines[n] for n in names[1:]}
+    if ctx.rank == 0:
+        print(json.dumps(line), flush=True)
+    if ctx.world > 1:
+        ctx.dist.destroy_process_group()
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5000)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=sorted(WORKLOADS) + sorted(INFER_WORKLOADS), default="c2_transe_l1")
+    ap.add_argument("--workload", default="suite",
+                    help="'suite' (default: every workload, headline first), or one or more names separated by commas: "
+                         + ", ".join(sorted(WORKLOADS) + sorted(INFER_WORKLOADS)))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    if args.workload in INFER_WORKLOADS:
-        if args.impl == "reference":
-            raise SystemExit("--impl reference covers the training workloads")
-        return run_infer(args, INFER_WORKLOADS[args.workload], args.workload)
-    w = WORKLOADS[args.workload]
+    names = list(SUITE) if args.workload == "suite" else args.workload.split(",")
+    for n in names:
+        if n not in WORKLOADS and n not in INFER_WORKLOADS:
+            raise SystemExit(f"unknown workload {n}")
     if args.impl == "reference":
-        run_reference(args, w, args.workload)
+        run_reference(args, names)
     else:
-        run_ours(args, w, args.workload)
+        run_ours(args, names)
 
 
 if __name__ == "__main__":

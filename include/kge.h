@@ -197,6 +197,26 @@ int kge_score_all_topk(kge_handle* h, const int32_t* q_heads, const int32_t* q_r
                        void* stream);
 
 /*
+ * kge_score_all_topk for callers that keep queries and results on the host: q_heads, q_rels,
+ * true_tails (or NULL) are [host] int32 [nq]; out_ids / out_scores [host] [nq, k]; out_ranks [host]
+ * [nq] or NULL (pinned memory makes the copies asynchronous).  The queries are copied in and the
+ * results copied back on `stream` through staging arrays inside the workspace; synchronises.
+ */
+int kge_score_all_topk_host(kge_handle* h, const int32_t* q_heads, const int32_t* q_rels, int32_t nq, int32_t k,
+                            const int32_t* true_tails, int32_t* out_ids, float* out_scores, int32_t* out_ranks,
+                            void* stream);
+
+/*
+ * Tensor-core inference (KGE_PREC_BF16_TC, DistMult / ComplEx) scores against a bf16 copy of the
+ * entity table kept in the workspace.  The copy is made by the first kge_score_all_topk / kge_eval_mrr
+ * after kge_bind and again after every kge_train_step or kge_init_tables on this handle; a caller that
+ * changes the entity table by any other means must call this before the next inference call, or it will
+ * score against the old rows.  Enqueues the copy on `stream` (46.6 GB read, 23.3 GB written at 91 M x 128).
+ * A no-op returning KGE_OK for handles without a tensor-core inference workspace.
+ */
+int kge_refresh_inference_table(kge_handle* h, void* stream);
+
+/*
  * (No counterpart in the paper: an addition for callers that cannot allocate.)
  * kge_score_all_topk for programs that must not call cudaMalloc -- an inference service whose
  * whole GPU memory is already handed to another allocator, a plugin that runs under a host
@@ -280,6 +300,17 @@ typedef enum {
 } kge_stage_t;
 int kge_profile(kge_handle* h, int enable);
 int kge_profile_read(kge_handle* h, double* ms /*[host]*/, int64_t* launches /*[host]*/, int reset);
+
+/*
+ * Measurement helper for the benchmark's roofline (not part of the method): the rate, in lane
+ * instructions per second over the whole GPU, at which the CUDA cores retire one of the instruction
+ * mixes the CUDA-core kernels consist of, from a register-resident loop of `iters` rounds:
+ * mix 0 fused multiply-add; mix 1 subtract + add of the absolute value (2 per element);
+ * mix 2 compare + predicated add (2 per element); mix 3 special-function exponential (counted
+ * alone; its accumulating add rides along).  per_second: [host].  Allocates 256 bytes of device
+ * memory for the duration of the call and synchronises.
+ */
+int kge_measure_alu(int32_t mix, int32_t iters, double* per_second /*[host]*/, void* stream);
 
 const char* kge_error_string(int code);
 const char* kge_last_cuda_error(const kge_handle* h);

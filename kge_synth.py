@@ -61,3 +61,37 @@ def make_queries(num_entities: int, num_relations: int, num_queries: int, *, see
     qr = rng.integers(0, num_relations, size=num_queries).astype(np.int32)
     tt = rng.integers(0, num_entities, size=num_queries).astype(np.int32)
     return np.ascontiguousarray(qh), qr, tt
+
+
+def make_graph_device(num_entities: int, num_relations: int, num_triples: int, *, seed: int, device,
+                      entity_zipf: float = 1.1, relation_zipf: float = 0.0, chunk: int = 1 << 25):
+    """The law of `make_graph` drawn on a GPU with torch's seeded generator, for graphs too large to draw
+    (or to hold three times over) on the host: int32 device tensors (h, r, t).  The random stream differs
+    from `make_graph`'s; the distribution (Zipf popularity ranks through a random permutation) is the same."""
+    import torch
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+
+    def cdf_of(n_items, s):
+        w = torch.arange(1, n_items + 1, dtype=torch.float64, device=device).pow_(-s)
+        c = torch.cumsum(w, 0)
+        return c.div_(c[-1].clone())
+
+    def draw(n_items, s, perm, out):
+        cdf = cdf_of(n_items, s) if s != 0.0 else None
+        for lo in range(0, num_triples, chunk):
+            n = min(chunk, num_triples - lo)
+            if cdf is None:
+                ranks = torch.randint(0, n_items, (n,), generator=gen, device=device)
+            else:
+                u = torch.rand(n, dtype=torch.float64, generator=gen, device=device)
+                ranks = torch.searchsorted(cdf, u, right=True).clamp_(max=n_items - 1)
+            out[lo:lo + n] = perm[ranks]
+        return out
+
+    perm = torch.randperm(num_entities, generator=gen, device=device).to(torch.int32)
+    h = draw(num_entities, entity_zipf, perm, torch.empty(num_triples, dtype=torch.int32, device=device))
+    t = draw(num_entities, entity_zipf, perm, torch.empty(num_triples, dtype=torch.int32, device=device))
+    rperm = torch.randperm(num_relations, generator=gen, device=device).to(torch.int32)
+    r = draw(num_relations, relation_zipf, rperm, torch.empty(num_triples, dtype=torch.int32, device=device))
+    return h, r, t

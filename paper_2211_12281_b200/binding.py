@@ -87,6 +87,9 @@ SIGNATURES = {
     "kge_score_all_topk": (C.c_int, [_vp, _vp, _vp, C.c_int32, C.c_int32, _vp, _vp, _vp, _vp, _vp]),
     "kge_score_all_topk_static": (C.c_int, [C.POINTER(KgeConfig), _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32, _vp, _vp, _vp,
                                             _vp, _vp]),
+    "kge_score_all_topk_host": (C.c_int, [_vp, _vp, _vp, C.c_int32, C.c_int32, _vp, _vp, _vp, _vp, _vp]),
+    "kge_refresh_inference_table": (C.c_int, [_vp, _vp]),
+    "kge_measure_alu": (C.c_int, [C.c_int32, C.c_int32, C.POINTER(C.c_double), _vp]),
     "kge_eval_mrr": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int32, C.c_int32, C.POINTER(C.c_double), _vp]),
     "kge_mrr_from_ranks": (C.c_int, [_vp, _vp, C.c_int32, C.c_int32, C.POINTER(C.c_double), _vp]),
     "kge_debug_capture_scores": (C.c_int, [_vp, _vp]),
@@ -147,6 +150,15 @@ def score_all_topk_static(cfg: KgeConfig, ent, rel, relw, q_heads, q_rels, k, tr
     return int(lib().kge_score_all_topk_static(C.byref(cfg), _ptr(ent), _ptr(rel), _ptr(relw), _ptr(q_heads),
                                                _ptr(q_rels), q_heads.numel(), k, _ptr(true_tails), _ptr(out_ids),
                                                _ptr(out_scores), _ptr(out_ranks), _stream()))
+
+
+def measure_alu(mix: int, iters: int = 4096) -> float:
+    """kge_measure_alu: lane instructions per second of instruction mix `mix` on the current GPU."""
+    out = C.c_double(0.0)
+    rc = int(lib().kge_measure_alu(mix, iters, C.byref(out), _stream()))
+    if rc != 0:
+        raise KgeError(rc, "kge_measure_alu", lib().kge_error_string(rc).decode())
+    return out.value
 
 
 def ensemble_rank_scores(power: float, k_list: int):
@@ -243,6 +255,15 @@ class Kge:
         self._check(lib().kge_score_all_topk(self._h, _ptr(q_heads), _ptr(q_rels), q_heads.numel(), k,
                                              _ptr(true_tails), _ptr(out_ids), _ptr(out_scores), _ptr(out_ranks),
                                              _stream()), "kge_score_all_topk")
+
+    def score_all_topk_host(self, q_heads, q_rels, k, true_tails, out_ids, out_scores, out_ranks=None):
+        """Host arrays (pinned torch tensors or numpy) in and out."""
+        self._check(lib().kge_score_all_topk_host(self._h, _ptr(q_heads), _ptr(q_rels), len(q_heads), k, _ptr(true_tails),
+                                                  _ptr(out_ids), _ptr(out_scores), _ptr(out_ranks), _stream()),
+                    "kge_score_all_topk_host")
+
+    def refresh_inference_table(self):
+        self._check(lib().kge_refresh_inference_table(self._h, _stream()), "kge_refresh_inference_table")
 
     def eval_mrr(self, q_heads, q_rels, true_tails, k_cutoff=10) -> float:
         out = C.c_double(0.0)

@@ -87,6 +87,7 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
     w.F = cv.take<float>(B * N);
     w.U = th ? cv.take<float>(B * N) : nullptr;
     w.Cc = th ? cv.take<float>(B * N) : nullptr;
+    w.wsum = th ? cv.take<float>(B) : nullptr;
     w.dQpart = cv.take<float>((size_t)h->split_q * B * d);
     w.dWpart = th ? cv.take<float>((size_t)h->split_q * B * d) : nullptr;
     w.dTpart = cv.take<float>((size_t)h->split_t * N * d);
@@ -114,6 +115,8 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
         w.cand_cnt = cv.take<int32_t>(q); w.beat_tmp = cv.take<int32_t>(q); w.beat = cv.take<int32_t>(q);
         w.cand_score = cv.take<float>(q * kCandCap); w.cand_id = cv.take<int32_t>(q * kCandCap);
         w.top_score = cv.take<float>(q * k); w.top_id = cv.take<int32_t>(q * k);
+        w.hq_heads = cv.take<int32_t>(q); w.hq_rels = cv.take<int32_t>(q); w.hq_tails = cv.take<int32_t>(q); w.hq_ranks = cv.take<int32_t>(q);
+        w.hq_ids = cv.take<int32_t>(q * k); w.hq_scores = cv.take<float>(q * k);
         // tensor-core inference (dot-product models): bf16 query vectors and a bf16 copy of the whole table
         const bool tci = c.prec == KGE_PREC_BF16_TC && (c.score == KGE_DISTMULT || c.score == KGE_COMPLEX);
         w.iqb = tci ? cv.take<uint16_t>(q * d) : nullptr;
@@ -312,6 +315,7 @@ int kge_bind(kge_handle* h, float* ent, float* rel, float* relw, float* ent_stat
     }
     h->bound = true;
     h->graph_loaded = false;
+    h->eb_valid = false;
     return KGE_OK;
 }
 
@@ -383,6 +387,7 @@ int kge_init_tables(kge_handle* h, float std, void* stream) {
     if (!h->bound) return KGE_ERR_NOT_READY;
     const kge_config& c = h->cfg;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    h->eb_valid = false;
     int rc = launch_init_table(h, h->ent, c.num_entities, c.dim, std, 0, 2u, s);
     if (rc == KGE_OK) rc = launch_init_table(h, h->rel, c.num_relations, h->kw, std, c.score == KGE_ROTATE ? 1 : 0, 3u, s);
     if (rc == KGE_OK && h->relw) rc = launch_init_table(h, h->relw, c.num_relations, c.dim, std, 0, 4u, s);
@@ -444,6 +449,7 @@ int kge_train_step(kge_handle* h, uint64_t step, float lr, const int32_t* heads,
     // with side streams the id sort has been joined before the chain kernel
     if (!fork && (rc = launch_dedup(h, heads, rels, tails, negs, s)) != KGE_OK) return rc;
     rc = launch_update(h, step, lr, s);
+    h->eb_valid = false;          // the entity table has moved on: tensor-core inference must refresh its bf16 copy
     if (rc != KGE_OK) return rc;
     return h->prof.on ? stage_collect(h, s) : KGE_OK;
 }
@@ -482,6 +488,40 @@ int kge_score_all_topk(kge_handle* h, const int32_t* q_heads, const int32_t* q_r
     if (nq == 0) return KGE_OK;
     return run_score_all_topk(h, q_heads, q_rels, nq, k, true_tails, out_ids, out_scores, out_ranks,
                               static_cast<cudaStream_t>(stream));
+}
+
+int kge_score_all_topk_host(kge_handle* h, const int32_t* q_heads, const int32_t* q_rels, int32_t nq, int32_t k,
+                            const int32_t* true_tails, int32_t* out_ids, float* out_scores, int32_t* out_ranks,
+                            void* stream) {
+    if (!h || nq < 0 || k <= 0) return KGE_ERR_BAD_ARG;
+    if (nq > 0 && (!q_heads || !q_rels || !out_ids || !out_scores)) return KGE_ERR_BAD_ARG;
+    if (out_ranks && !true_tails) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    if (nq > h->max_queries || k > h->topk) return KGE_ERR_WORKSPACE;
+    if (nq == 0) return KGE_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    Workspace& w = h->ws;
+    const size_t qb = (size_t)nq * sizeof(int32_t);
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.hq_heads, q_heads, qb, cudaMemcpyHostToDevice, s));
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.hq_rels, q_rels, qb, cudaMemcpyHostToDevice, s));
+    if (true_tails) KGE_CUDA_CHECK(h, cudaMemcpyAsync(w.hq_tails, true_tails, qb, cudaMemcpyHostToDevice, s));
+    const int rc = run_score_all_topk(h, w.hq_heads, w.hq_rels, nq, k, true_tails ? w.hq_tails : nullptr, w.hq_ids, w.hq_scores,
+                                      out_ranks ? w.hq_ranks : nullptr, s);
+    if (rc != KGE_OK) return rc;
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(out_ids, w.hq_ids, (size_t)nq * k * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    KGE_CUDA_CHECK(h, cudaMemcpyAsync(out_scores, w.hq_scores, (size_t)nq * k * sizeof(float), cudaMemcpyDeviceToHost, s));
+    if (out_ranks) KGE_CUDA_CHECK(h, cudaMemcpyAsync(out_ranks, w.hq_ranks, qb, cudaMemcpyDeviceToHost, s));
+    KGE_CUDA_CHECK(h, cudaStreamSynchronize(s));
+    return KGE_OK;
+}
+
+int kge_refresh_inference_table(kge_handle* h, void* stream) {
+    if (!h) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    if (!h->ws.Eb) return KGE_OK;
+    const int rc = launch_cast_bf16(h, h->ent, h->ws.Eb, h->cfg.num_entities * h->cfg.dim, static_cast<cudaStream_t>(stream));
+    if (rc == KGE_OK) h->eb_valid = true;
+    return rc;
 }
 
 int kge_mrr_from_ranks(kge_handle* h, const int32_t* ranks, int32_t nq, int32_t k_cutoff, double* mrr_out, void* stream) {

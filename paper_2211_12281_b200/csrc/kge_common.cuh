@@ -59,7 +59,8 @@ struct Workspace {
     float *Grow;                           // [B] row sums of dL/dF (TransE p=1 backward)
     float *Cpart;                          // [St, N] column sums of dL/dF per row split (TransE p=1 backward)
     float *F;                              // [B,N] scores, overwritten by dL/dF
-    float *U, *Cc;                         // [B,N] TransH: w.t and the S.w contraction
+    float *U, *Cc;                         // [B,N] TransH: w.t and the contraction c' = sum_k s_k w_k of every pair
+    float *wsum;                           // [B] TransH: sum of the unit normal's coordinates
     float *dQpart, *dWpart, *dTpart;       // [Sq,B,d], [Sq,B,d] (TransH), [St,N,d]
     float *grad_ent, *grad_rel, *grad_relw;  // [2B+N,d], [B,kw], [B,d]
     // dedup
@@ -78,6 +79,8 @@ struct Workspace {
     int32_t *cand_cnt, *beat_tmp, *beat;   // [maxq]
     float *cand_score; int32_t *cand_id;   // [maxq, kCandCap]
     float *top_score; int32_t *top_id;     // [maxq, topk] running lists
+    int32_t *hq_heads, *hq_rels, *hq_tails, *hq_ranks;   // [maxq] staging of kge_score_all_topk_host
+    int32_t *hq_ids; float *hq_scores;                   // [maxq, topk]
 };
 
 }  // namespace kge
@@ -121,6 +124,7 @@ struct kge_handle {
     bool streams_ready;
     cudaStream_t side[2];
     cudaEvent_t ev_ids, ev_loss, ev_seg, ev_t;
+    bool eb_valid;          // the bf16 copy of the entity table (tensor-core inference) matches the table
     int wait_limit;         // tries of every bounded barrier wait in this handle's kernels (kDefaultWaitLimit unless a test shortens it)
     float* capture_scores;  // debug: the training step also writes the B x N score block here (caller's device array), or NULL
     char cuda_err[256];     // text of the last failed CUDA call (a fixed buffer: reporting an error allocates nothing)
@@ -190,6 +194,9 @@ int tc_pieces_per_tile();
 // The dT contraction of the dot-product kinds with a single K split is the negatives' gradient rows: it writes them in place.
 bool tc_negatives_direct(const kge_handle* h);
 int launch_tc_backward(kge_handle* h, cudaStream_t s, cudaStream_t side);
+// TransH score block (scores, w.t, c') and its two backward accumulations (kge_transh.cu).
+int launch_th_forward(kge_handle* h, cudaStream_t s);
+int launch_th_backward(kge_handle* h, cudaStream_t sq, cudaStream_t st);
 int launch_tc_forward(kge_handle* h, cudaStream_t s);
 int launch_cast_bf16(kge_handle* h, const float* src, uint16_t* dst, int64_t count, cudaStream_t s);
 int launch_tc_infer_chunk(kge_handle* h, int nq, int64_t e_lo, int64_t e_hi, const int32_t* true_tails, cudaStream_t s);

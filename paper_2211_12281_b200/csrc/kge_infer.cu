@@ -477,7 +477,10 @@ int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int3
     const bool tc = h->ws.Eb != nullptr;    // dot-product model with the tensor-core score block
     if (tc) {
         int rc = launch_cast_bf16(h, h->ws.iq, h->ws.iqb, (int64_t)nq * c.dim, s);
-        if (rc == KGE_OK) rc = launch_cast_bf16(h, h->ent, h->ws.Eb, c.num_entities * c.dim, s);
+        if (rc == KGE_OK && !h->eb_valid) {     // the bf16 copy of the table is kept until the table changes
+            rc = launch_cast_bf16(h, h->ent, h->ws.Eb, c.num_entities * c.dim, s);
+            if (rc == KGE_OK) h->eb_valid = true;
+        }
         if (rc != KGE_OK) return rc;
         ftrue_bf16_kernel<<<qblocks, 128, 0, s>>>(p);
         KGE_LAUNCH_CHECK(h);

@@ -196,8 +196,14 @@ __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
             const float inv = 1.f / fmaxf(sqrtf(warp_sum(nrm2)), 1e-12f);
             float a = 0.f;
 #pragma unroll
-            for (int i = 0; i < kMaxChunks; ++i) { wh[i] = f4scale(inv, wh[i]); a += f4dot(wh[i], h[i]); }
-            a = warp_sum(a);
+            float ws = 0.f;
+#pragma unroll
+            for (int i = 0; i < kMaxChunks; ++i) {
+                wh[i] = f4scale(inv, wh[i]); a += f4dot(wh[i], h[i]);
+                ws += (wh[i].x + wh[i].y) + (wh[i].z + wh[i].w);
+            }
+            a = warp_sum(a); ws = warp_sum(ws);
+            if (lane == 0) p.w.wsum[b] = ws;      // sum of the unit normal's coordinates (the p = 1 forward needs it per query)
 #pragma unroll
             for (int i = 0; i < kMaxChunks; ++i) q[i] = f4add(f4fma(-a, wh[i], h[i]), r[i]);
         }
@@ -245,11 +251,10 @@ __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
 }
 
 // ------------------------------------------------------------------------------------------
-// block: 64 x 64 pairs per CTA, 256 threads, 4 x 4 pairs per thread, the embedding axis
-// streamed through shared memory in slices of 32.  MODE 0 writes F (and U = w.t for TransH);
-// MODE 1 (TransH only) writes the contraction c_bn = sum_k S_bnk w_bk needed by the backward.
+// block: F[b, n] = f(q_b, t_n).  Per-pair arithmetic of the kinds that are a function of
+// (q, t) alone; the TransH block lives in kge_transh.cu.
 // ------------------------------------------------------------------------------------------
-constexpr int TB = 64, TN = 64, KC = 32, LDS = KC + 4;
+constexpr int TN = 64;   // negative columns per score tile
 
 __device__ __forceinline__ float approx_sqrt(float x) { float r; asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
 __device__ __forceinline__ float approx_rsqrt(float x) { float r; asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
@@ -291,111 +296,6 @@ __device__ __forceinline__ void f4add_w_if_pos(float& acc, float4 x, float4 w) {
 __device__ __forceinline__ void f4add2_if_pos(float4& acc1, float4& acc2, float4 x, float w1, float w2) {
     add2_if_pos(acc1.x, acc2.x, x.x, w1, w2); add2_if_pos(acc1.y, acc2.y, x.y, w1, w2);
     add2_if_pos(acc1.z, acc2.z, x.z, w1, w2); add2_if_pos(acc1.w, acc2.w, x.w, w1, w2);
-}
-
-template <int KIND, int MODE>
-__global__ void __launch_bounds__(256) block_kernel(TrainParams p) {
-    constexpr bool TH = KIND == KIND_TH_L1 || KIND == KIND_TH_L2;
-    __shared__ __align__(16) float Qs[TB * LDS];
-    __shared__ __align__(16) float Ts[TN * LDS];
-    __shared__ __align__(16) float Ws[TH ? TB * LDS : 4];
-    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-    const int b0 = blockIdx.y * TB, n0 = blockIdx.x * TN;
-    const int d4 = p.d4;
-    const float4* Qg = reinterpret_cast<const float4*>(p.w.Q);
-    const float4* Tg = reinterpret_cast<const float4*>(p.w.Tneg);
-    const float4* Wg = reinterpret_cast<const float4*>(p.w.What);
-
-    float acc[4][4], u[4][4];
-    float wsum[4] = {0.f, 0.f, 0.f, 0.f};   // TransH p = 1, second pass: sum of the normal's coordinates per query row
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) { acc[i][j] = 0.f; u[i][j] = 0.f; }
-    if (TH && MODE == 1) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int b = b0 + ty + 16 * i, n = n0 + tx + 16 * j;
-                u[i][j] = (b < p.B && n < p.N) ? p.w.U[(int64_t)b * p.N + n] : 0.f;
-            }
-    }
-    const int npass = (TH && MODE == 0) ? 2 : 1;
-    for (int pass = 0; pass < npass; ++pass) {
-        const bool upass = TH && MODE == 0 && pass == 0;
-        for (int k0 = 0; k0 < p.d; k0 += KC) {
-#pragma unroll
-            for (int it = 0; it < 2; ++it) {
-                const int idx = tid + 256 * it, row = idx >> 3, c4 = idx & 7;
-                const int gc = (k0 >> 2) + c4;
-                const bool kin = gc < d4;
-                float4 qv = f4zero(), tv = f4zero(), wv = f4zero();
-                if (kin && b0 + row < p.B) {
-                    qv = Qg[(int64_t)(b0 + row) * d4 + gc];
-                    if (TH) wv = Wg[(int64_t)(b0 + row) * d4 + gc];
-                }
-                if (kin && n0 + row < p.N) tv = Tg[(int64_t)(n0 + row) * d4 + gc];
-                *reinterpret_cast<float4*>(&Qs[row * LDS + c4 * 4]) = qv;
-                *reinterpret_cast<float4*>(&Ts[row * LDS + c4 * 4]) = tv;
-                if (TH) *reinterpret_cast<float4*>(&Ws[row * LDS + c4 * 4]) = wv;
-            }
-            __syncthreads();
-#pragma unroll
-            for (int kk = 0; kk < KC; kk += 4) {
-                float4 qv[4], tv[4], wv[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    qv[i] = *reinterpret_cast<const float4*>(&Qs[(ty + 16 * i) * LDS + kk]);
-                    tv[i] = *reinterpret_cast<const float4*>(&Ts[(tx + 16 * i) * LDS + kk]);
-                    if (TH) wv[i] = *reinterpret_cast<const float4*>(&Ws[(ty + 16 * i) * LDS + kk]);
-                }
-                if (KIND == KIND_TH_L1 && MODE == 1) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) wsum[i] += (wv[i].x + wv[i].y) + (wv[i].z + wv[i].w);
-                }
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        if (!TH) {
-                            pair_update<TH ? KIND_L1 : KIND>(acc[i][j], qv[i], tv[j]);
-                        } else if (upass) {
-                            u[i][j] = fmaf(wv[i].x, tv[j].x, u[i][j]); u[i][j] = fmaf(wv[i].y, tv[j].y, u[i][j]);
-                            u[i][j] = fmaf(wv[i].z, tv[j].z, u[i][j]); u[i][j] = fmaf(wv[i].w, tv[j].w, u[i][j]);
-                        } else {
-                            const float4 x = f4fma(u[i][j], wv[i], f4sub(qv[i], tv[j]));
-                            if (MODE == 0) {
-                                if (KIND == KIND_TH_L1) acc[i][j] += fabsf(x.x) + fabsf(x.y) + fabsf(x.z) + fabsf(x.w);
-                                else acc[i][j] += f4dot(x, x);
-                            } else {
-                                if (KIND == KIND_TH_L1) f4add_w_if_pos(acc[i][j], x, wv[i]);
-                                else acc[i][j] += f4dot(x, wv[i]);
-                            }
-                        }
-                    }
-            }
-            __syncthreads();
-        }
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int b = b0 + ty + 16 * i, n = n0 + tx + 16 * j;
-            if (b >= p.B || n >= p.N) continue;
-            const int64_t o = (int64_t)b * p.N + n;
-            if (MODE == 1) {
-                const float sw = KIND == KIND_TH_L1 ? 2.f * acc[i][j] - wsum[i] : acc[i][j];   // p = 1: acc holds P
-                p.w.Cc[o] = -p.w.F[o] * sw;          // F holds G (p=1) or G / distance (p=2) by now
-            } else {
-                float f = acc[i][j];
-                if (KIND == KIND_L1 || KIND == KIND_CL1 || KIND == KIND_TH_L1) f = -f;
-                else if (KIND == KIND_L2 || KIND == KIND_TH_L2) f = -sqrtf(f);
-                p.w.F[o] = f;
-                if (TH) p.w.U[o] = u[i][j];
-            }
-        }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -770,137 +670,6 @@ __device__ __forceinline__ void acc_update(float4& acc, float4 a, float4 b, floa
         s = w * approx_rsqrt(fmaxf(m2, 1e-37f));
         acc.z = fmaf(-s, xr, acc.z); acc.w = fmaf(-s, xi, acc.w);
     }
-}
-
-template <int KIND, int NCH, bool OWNER_Q>
-__global__ void __launch_bounds__(256) accum_kernel(AccArgs a) {
-    constexpr bool TH = KIND == KIND_TH_L1 || KIND == KIND_TH_L2;
-    extern __shared__ __align__(16) float smem[];
-    const int d4 = a.d4;
-    float4* Bs = reinterpret_cast<float4*>(smem);                        // [32][d4]
-    float4* W2s = Bs + (TH && !OWNER_Q ? ACC_CC * d4 : 0);               // TransH dT: normals of the queries
-    float* Gs = reinterpret_cast<float*>(W2s + ACC_CC * d4);             // [32][36] weights, [c][r]
-    float* Us = Gs + ACC_CC * ACC_LDW;
-    float* Cs = Us + (TH ? ACC_CC * ACC_LDW : 0);
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int r0 = blockIdx.x * ACC_ROWS;
-    const int per = ((a.oth_rows + a.split - 1) / a.split + ACC_CC - 1) / ACC_CC * ACC_CC;
-    const int c_begin = blockIdx.y * per;
-    const int c_end = min(a.oth_rows, c_begin + per);
-
-    // sign sums as 2 P - (sum of the weights): see add_if_pos (not for the widest rows of the query side, whose three
-    // accumulators per row would not fit the register file)
-    constexpr bool TH1 = KIND == KIND_TH_L1 && !(OWNER_Q && NCH == 4);
-    float4 A[4][NCH], Wn[TH && OWNER_Q ? 4 : 1][NCH], acc[4][NCH], acc2[TH ? 4 : 1][NCH], acc3[TH1 && OWNER_Q ? 4 : 1][NCH];
-    float sg[4] = {0.f, 0.f, 0.f, 0.f}, sug[4] = {0.f, 0.f, 0.f, 0.f};   // TH1: sums of g and of u g over this split, per owner row
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < NCH; ++j) {
-            const int r = r0 + warp * 4 + i, c = lane + 32 * j;
-            const bool in = r < a.own_rows && c < d4;
-            A[i][j] = in ? reinterpret_cast<const float4*>(a.own)[(int64_t)r * d4 + c] : f4zero();
-            acc[i][j] = f4zero();
-            if (TH && OWNER_Q) Wn[i][j] = in ? reinterpret_cast<const float4*>(a.what)[(int64_t)r * d4 + c] : f4zero();
-            if (TH) acc2[i][j] = f4zero();
-            if (TH1 && OWNER_Q) acc3[i][j] = f4zero();
-        }
-
-    for (int c0 = c_begin; c0 < c_end; c0 += ACC_CC) {
-        for (int idx = tid; idx < ACC_CC * d4; idx += 256) {
-            const int rr = idx / d4, cc = idx - rr * d4, row = c0 + rr;
-            Bs[idx] = row < c_end ? reinterpret_cast<const float4*>(a.oth)[(int64_t)row * d4 + cc] : f4zero();
-            if (TH && !OWNER_Q)
-                W2s[idx] = row < c_end ? reinterpret_cast<const float4*>(a.what)[(int64_t)row * d4 + cc] : f4zero();
-        }
-        for (int idx = tid; idx < ACC_CC * ACC_ROWS; idx += 256) {
-            int rr, cc;
-            int64_t g;
-            if (OWNER_Q) { cc = idx & 31; rr = idx >> 5; g = (int64_t)(r0 + rr) * a.N + (c0 + cc); }
-            else         { rr = idx & 31; cc = idx >> 5; g = (int64_t)(c0 + cc) * a.N + (r0 + rr); }
-            const bool in = (r0 + rr) < a.own_rows && (c0 + cc) < c_end;
-            Gs[cc * ACC_LDW + rr] = in ? a.G[g] : 0.f;
-            if (TH) { Us[cc * ACC_LDW + rr] = in ? a.U[g] : 0.f; Cs[cc * ACC_LDW + rr] = in ? a.Cc[g] : 0.f; }
-        }
-        __syncthreads();
-#pragma unroll 4
-        for (int cc = 0; cc < ACC_CC; ++cc) {
-            const float4 g4 = *reinterpret_cast<const float4*>(&Gs[cc * ACC_LDW + warp * 4]);
-            const float gw[4] = {g4.x, g4.y, g4.z, g4.w};
-            float uw[4] = {0.f, 0.f, 0.f, 0.f}, cw[4] = {0.f, 0.f, 0.f, 0.f};
-            if (TH) {
-                const float4 u4 = *reinterpret_cast<const float4*>(&Us[cc * ACC_LDW + warp * 4]);
-                const float4 c4 = *reinterpret_cast<const float4*>(&Cs[cc * ACC_LDW + warp * 4]);
-                uw[0] = u4.x; uw[1] = u4.y; uw[2] = u4.z; uw[3] = u4.w;
-                cw[0] = c4.x; cw[1] = c4.y; cw[2] = c4.z; cw[3] = c4.w;
-            }
-            float ugw[4] = {0.f, 0.f, 0.f, 0.f};
-            if (TH1) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) { ugw[i] = uw[i] * gw[i]; sg[i] += gw[i]; sug[i] += ugw[i]; }
-            }
-#pragma unroll
-            for (int j = 0; j < NCH; ++j) {
-                const int c = lane + 32 * j;
-                if (c >= d4) continue;
-                const float4 bv = Bs[cc * d4 + c];
-                if (!TH) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) acc_update<TH ? KIND_L1 : KIND>(acc[i][j], A[i][j], bv, gw[i]);
-                } else if (OWNER_Q) {   // own = q_b (A), normal Wn; other = t_n (bv)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float4 x = f4fma(uw[i], Wn[i][j], f4sub(A[i][j], bv));
-                        if (TH1) {      // acc = P (weights g), acc3 = P (weights u g), acc2 = sum of c t
-                            f4add2_if_pos(acc[i][j], acc3[i][j], x, gw[i], ugw[i]);
-                            acc2[i][j] = f4fma(cw[i], bv, acc2[i][j]);
-                        } else {
-                            const float4 S = KIND == KIND_TH_L1 ? f4scale(-gw[i], f4sgn(x)) : f4scale(-gw[i], x);
-                            acc[i][j] = f4add(acc[i][j], S);
-                            acc2[i][j] = f4fma(cw[i], bv, f4fma(uw[i], S, acc2[i][j]));
-                        }
-                    }
-                } else {                // own = t_n (A); other = q_b (bv) with its normal wv
-                    const float4 wv = W2s[cc * d4 + c];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float4 x = f4fma(uw[i], wv, f4sub(bv, A[i][j]));
-                        if (TH1) {      // acc = P (weights g), acc2 = sum of c w
-                            f4add_if_pos(acc[i][j], x, gw[i]);
-                            acc2[i][j] = f4fma(cw[i], wv, acc2[i][j]);
-                        } else {
-                            const float4 S = KIND == KIND_TH_L1 ? f4scale(-gw[i], f4sgn(x)) : f4scale(-gw[i], x);
-                            acc[i][j] = f4fma(cw[i], wv, f4sub(acc[i][j], S));
-                        }
-                    }
-                }
-            }
-        }
-        __syncthreads();
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < NCH; ++j) {
-            const int r = r0 + warp * 4 + i, c = lane + 32 * j;
-            if (r >= a.own_rows || c >= d4) continue;
-            const int64_t o = ((int64_t)blockIdx.y * a.own_rows + r) * d4 + c;
-            if (TH1) {
-                const float4 P = acc[i][j], C = acc2[i][j];
-                if (OWNER_Q) {   // -sum g sign(x) = (sum g) - 2 P;  sum (c t - u g sign(x)) = C - 2 P_u + (sum u g)
-                    const float4 Pu = acc3[OWNER_Q ? i : 0][j];
-                    acc[i][j] = make_float4(sg[i] - 2.f * P.x, sg[i] - 2.f * P.y, sg[i] - 2.f * P.z, sg[i] - 2.f * P.w);
-                    acc2[i][j] = make_float4(C.x - 2.f * Pu.x + sug[i], C.y - 2.f * Pu.y + sug[i], C.z - 2.f * Pu.z + sug[i],
-                                             C.w - 2.f * Pu.w + sug[i]);
-                } else {         // sum (c w + g sign(x)) = C + 2 P - (sum g)
-                    acc[i][j] = make_float4(C.x + 2.f * P.x - sg[i], C.y + 2.f * P.y - sg[i], C.z + 2.f * P.z - sg[i],
-                                            C.w + 2.f * P.w - sg[i]);
-                }
-            }
-            reinterpret_cast<float4*>(a.out)[o] = acc[i][j];
-            if (TH && OWNER_Q) reinterpret_cast<float4*>(a.out2)[o] = acc2[i][j];
-        }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1321,12 +1090,6 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
 }
 
 // ---- host-side dispatch ----
-template <int KIND, int MODE>
-void launch_block(const TrainParams& p, cudaStream_t s) {
-    dim3 grid((p.N + TN - 1) / TN, (p.B + TB - 1) / TB);
-    block_kernel<KIND, MODE><<<grid, 256, 0, s>>>(p);
-}
-
 template <int KIND>
 cudaError_t launch_block_tma(const TrainParams& p, cudaStream_t s) {
     const size_t smem = block_tma_smem(p.d);
@@ -1368,33 +1131,6 @@ cudaError_t launch_accum_tma(int kind, const AccArgs& aq, const AccArgs& at, cud
         case KIND_CL1: return launch_accum_tma_kind<KIND_CL1>(aq, at, s);
         default: return launch_accum_tma_kind<KIND_DOT>(aq, at, s);
     }
-}
-
-// TransH: one launch per owner side.
-template <int KIND, int NCH, bool OWNER_Q>
-cudaError_t launch_accum_inst(const AccArgs& a, cudaStream_t s) {
-    const size_t smem = (size_t)ACC_CC * a.d4 * 16 * (OWNER_Q ? 1 : 2) + (size_t)ACC_CC * ACC_LDW * 4 * 3;
-    static DeviceOnce configured;
-    const cudaError_t e = once_per_device(configured, [] {
-        return cudaFuncSetAttribute(accum_kernel<KIND, NCH, OWNER_Q>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-    });
-    if (e != cudaSuccess) return e;
-    dim3 grid((a.own_rows + ACC_ROWS - 1) / ACC_ROWS, a.split);
-    accum_kernel<KIND, NCH, OWNER_Q><<<grid, 256, smem, s>>>(a);
-    return cudaSuccess;
-}
-
-template <int KIND, bool OWNER_Q>
-cudaError_t launch_accum_kind(const AccArgs& a, cudaStream_t s) {
-    if (a.d4 <= 32) return launch_accum_inst<KIND, 1, OWNER_Q>(a, s);
-    if (a.d4 <= 64) return launch_accum_inst<KIND, 2, OWNER_Q>(a, s);
-    return launch_accum_inst<KIND, 4, OWNER_Q>(a, s);
-}
-
-template <bool OWNER_Q>
-cudaError_t launch_accum(int kind, const AccArgs& a, cudaStream_t s) {
-    if (kind == KIND_TH_L1) return launch_accum_kind<KIND_TH_L1, OWNER_Q>(a, s);
-    return launch_accum_kind<KIND_TH_L2, OWNER_Q>(a, s);
 }
 
 }  // namespace
@@ -1453,8 +1189,7 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
         case KIND_L2: KGE_CUDA_CHECK(h, launch_block_tma<KIND_L2>(p, s)); break;
         case KIND_CL1: KGE_CUDA_CHECK(h, launch_block_tma<KIND_CL1>(p, s)); break;
         case KIND_DOT: KGE_CUDA_CHECK(h, launch_block_tma<KIND_DOT>(p, s)); break;
-        case KIND_TH_L1: launch_block<KIND_TH_L1, 0>(p, s); break;
-        default: launch_block<KIND_TH_L2, 0>(p, s); break;
+        default: { const int rc = launch_th_forward(h, s); if (rc != KGE_OK) return rc; h->launches -= 1; break; }   // TransH (counted below)
     }
     stage_end(h, ST_BLOCK, s);
     KGE_LAUNCH_CHECK(h);
@@ -1485,13 +1220,6 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     stage_end(h, ST_LOSS, s);
     KGE_LAUNCH_CHECK(h);
     }
-    if (p.kind == KIND_TH_L1 || p.kind == KIND_TH_L2) {
-        stage_begin(h, ST_TH_CPASS, s);
-        if (p.kind == KIND_TH_L1) launch_block<KIND_TH_L1, 1>(p, s); else launch_block<KIND_TH_L2, 1>(p, s);
-        stage_end(h, ST_TH_CPASS, s);
-        KGE_LAUNCH_CHECK(h);
-    }
-
     if (c.prec == KGE_PREC_BF16_TC) {
         const int rc = launch_tc_backward(h, s, side);
         if (rc != KGE_OK) return rc;
@@ -1516,16 +1244,11 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
             KGE_CUDA_CHECK(h, cudaStreamWaitEvent(side, h->ev_loss, 0));
         }
         cudaStream_t sq = side ? side : s;
-        stage_begin(h, ST_ACCUM_Q, sq);
-        KGE_CUDA_CHECK(h, launch_accum<true>(p.kind, aq, sq));
-        stage_end(h, ST_ACCUM_Q, sq);
-        KGE_LAUNCH_CHECK(h);
-        if (side) KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_t, side));
-        stage_begin(h, ST_ACCUM_T, s);
-        KGE_CUDA_CHECK(h, launch_accum<false>(p.kind, at, s));
-        stage_end(h, ST_ACCUM_T, s);
-        KGE_LAUNCH_CHECK(h);
-        if (side) KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_t, 0));
+        { const int rc = launch_th_backward(h, sq, s); if (rc != KGE_OK) return rc; }
+        if (side) {
+            KGE_CUDA_CHECK(h, cudaEventRecord(h->ev_t, side));
+            KGE_CUDA_CHECK(h, cudaStreamWaitEvent(s, h->ev_t, 0));
+        }
     }
     }
     // the update follows the chain kernel directly: join the id sort here, where it has long finished
