@@ -112,9 +112,12 @@ STAGE_OPS = {
     "rotate1": dict(block=[(2, MIX_SUB_ABS), (0.5, MIX_FMA), (0.5, MIX_SFU)], accum=[(2, MIX_SUB_ABS), (1, MIX_FMA), (2, MIX_FMA), (1.0, MIX_SFU)]),
     "distmult1": dict(block=[(1, MIX_FMA)], accum=[(2, MIX_FMA)]),
     "complex1": dict(block=[(1, MIX_FMA)], accum=[(2, MIX_FMA)]),
-    # TransH p = 1: w.t (1 fma) + residual (sub, fma) + |.| accumulate (1); the backward passes re-form the residual
-    "transh1": dict(block=[(2, MIX_FMA), (2, MIX_SUB_ABS)], th_cpass=[(2, MIX_FMA), (2, MIX_CMP_ADD)],
-                    accum_q=[(2, MIX_FMA), (3, MIX_CMP_ADD), (1, MIX_FMA)], accum_t=[(2, MIX_FMA), (2, MIX_CMP_ADD), (1, MIX_FMA)]),
+    # TransH p = 1.  forward: w.t (fma), threshold fma(u, w, q), residual and |.| accumulate (sub + abs-add), the pair's
+    # contraction sum_k sign(x_k) w_k (compare + predicated add).  backward: threshold (fma), compare, one predicated add
+    # per sign sum (two on the query side), one fma for the c t (c w) term.
+    "transh1": dict(block=[(2, MIX_FMA), (2, MIX_SUB_ABS), (2, MIX_CMP_ADD)],
+                    accum_q=[(2, MIX_FMA), (3, MIX_CMP_ADD)], accum_t=[(2, MIX_FMA), (2, MIX_CMP_ADD)]),
+    "transh2": dict(block=[(5, MIX_FMA)], accum_q=[(5, MIX_FMA)], accum_t=[(4, MIX_FMA)]),
 }
 
 # Special-function instructions per score of the fused tensor-core epilogues (exponential, logarithm, reciprocal, reciprocal

@@ -34,6 +34,31 @@ int pick_split(int rows, int cols, int num_sms) {
     return std::max(1, (cols + per - 1) / per);
 }
 
+// The same choice for launches of many more CTAs than the GPU holds at once (TransH at large batches).
+int pick_split_waves(int rows, int cols, int num_sms, int ctas_per_sm) {
+    // One CTA covers 32 owner rows and walks its share of the reduced dimension in chunks of 32.  The CTAs of a launch
+    // run in waves of num_sms * ctas_per_sm; the number of column splits (at most 16, none empty) is the one that
+    // leaves the last wave fullest, with at least about two waves so that the CTAs' start-up overlaps other CTAs'
+    // work, and the fewer splits among equals (every split adds a partial slab for the chain kernel to sum).
+    const int row_ctas = (rows + 31) / 32;
+    const int slots = num_sms * ctas_per_sm;
+    const int max_split = std::max(1, std::min(16, (cols + 31) / 32));
+    int best = 1;
+    double best_score = -1.0;
+    for (int s = 1; s <= max_split; ++s) {
+        const int per = ((cols + s - 1) / s + 31) / 32 * 32;
+        const int real = (cols + per - 1) / per;                   // splits that are not empty
+        if (real != s) continue;
+        const int n = row_ctas * s;
+        const int waves = (n + slots - 1) / slots;
+        double score = (double)n / ((double)waves * slots);        // how full the waves are
+        if (n < 2 * slots) score *= 0.9;                           // fewer than two waves: nothing hides a CTA's start-up
+        score -= 0.002 * s;
+        if (score > best_score) { best_score = score; best = s; }
+    }
+    return best;
+}
+
 // Tensor-core contraction [rows, cols] over `depth` on persistent CTAs (one per SM): as many K
 // splits as still give every SM at most one tile (or one split when there are more tiles than
 // SMs), each at least four 64-wide slices deep, at most 16, none empty.
@@ -217,8 +242,14 @@ int kge_create(const kge_config* cfg, kge_handle** out) {
         h->num_sms = sms;
     else
         (void)cudaGetLastError();
-    h->split_q = pick_split(c.batch, c.num_neg, h->num_sms);
-    h->split_t = pick_split(c.num_neg, c.batch, h->num_sms);
+    // resident CTAs per SM of the TransH accumulation kernels: two (128 registers x 256 threads, 70-90 KB of shared memory)
+    if (c.score == KGE_TRANSH) {
+        h->split_q = pick_split_waves(c.batch, c.num_neg, h->num_sms, 2);
+        h->split_t = pick_split_waves(c.num_neg, c.batch, h->num_sms, 2);
+    } else {
+        h->split_q = pick_split(c.batch, c.num_neg, h->num_sms);
+        h->split_t = pick_split(c.num_neg, c.batch, h->num_sms);
+    }
     if (c.prec == KGE_PREC_BF16_TC) {   // the backward contractions run as 128 x 128 tensor-core tiles split over K
         h->split_q = pick_split_tc(c.batch, c.dim, c.num_neg, h->num_sms);
         h->split_t = pick_split_tc(c.num_neg, c.dim, c.batch, h->num_sms);

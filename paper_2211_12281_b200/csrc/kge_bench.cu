@@ -33,7 +33,7 @@ __global__ void __launch_bounds__(MB_THREADS) alu_mix_kernel(float* out, float s
 #pragma unroll
             for (int j = 0; j < MB_ACC; ++j) {
                 if (MIX == 0) {
-                    acc[j] = fmaf(q[j], t[r], acc[j]);
+                    acc[j] = fmaf(t[r], w, acc[j]);      // (two of the three operands are shared by the round: no register-bank stalls)
                 } else if (MIX == 1) {
                     asm volatile("{\n .reg .f32 x;\n sub.f32 x, %1, %2;\n abs.f32 x, x;\n add.f32 %0, %0, x;\n}\n" : "+f"(acc[j]) : "f"(q[j]), "f"(t[r]));
                 } else if (MIX == 2) {

@@ -264,8 +264,7 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
         float* T0 = Tl + (size_t)buf * NT * HA_CC * HA_LDW;
 #pragma unroll
         for (int e = 0; e < HA_WPT; ++e) {
-            const int idx = tid + HA_THREADS * e;
-            const int rr = OWNER_Q ? idx >> 5 : idx & 31, cc = OWNER_Q ? idx & 31 : idx >> 5;
+            const int rr = OWNER_Q ? warp + HA_WARPS * e : lane, cc = OWNER_Q ? lane : warp + HA_WARPS * e;
             const int o = cc * HA_LDW + rr;
             T0[o] = greg[e];
             T0[HA_CC * HA_LDW + o] = ureg[e];
