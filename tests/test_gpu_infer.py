@@ -59,6 +59,24 @@ def test_topk_rank_mrr_against_fp32_oracle(oracle32, oracle64, score, p):
         assert abs(mrr - oracle64.mrr(o_ranks, 10)) <= 1e-12 and abs(mrr0 - oracle64.mrr(o_ranks, 0)) <= 1e-12
 
 
+@pytest.mark.parametrize("score,p,d", [("transe", 1, 128), ("distmult", 1, 40), ("transe", 2, 64), ("complex", 1, 128)])
+def test_many_query_tiles_stream_past_resident_entity_tiles(oracle32, score, p, d):
+    """With four or more 64-query tiles and rows of at most 128 floats a thread block keeps its entity tile and streams
+    the query tiles past it (double buffer): 300 queries (a ragged fifth tile), 3,000 entities (ragged last tile, chunks
+    1024 + 1024 + 952), exact ties; ids, scores and ranks bit-exact against the fp32 oracle."""
+    import kge_synth
+    E, R, K, nq = 3000, 9, 10, 300
+    prob = Problem(E=E, R=R, T=100, d=d, score=score, p_norm=p, B=4, N=4, P=1, graph_seed=19)
+    prob.ent[2900] = prob.ent[17]; prob.ent[1] = prob.ent[0]
+    qh, qr, tt = kge_synth.make_queries(E, R, nq, seed=19)
+    tt[0] = qh[0]; tt[1] = 2900; tt[2] = 17
+    gpu = GpuSide(prob, max_queries=nq, topk=K, load_graph=False)
+    ids, sc, ranks = _infer(gpu, qh, qr, tt, K)
+    o_ids, o_sc, o_ranks = oracle32.score_all_topk(prob.oracle_cfg(), prob.ent, prob.rel, prob.relw, qh, qr, K, true_tails=tt)
+    assert (ids == o_ids).all() and (ranks == o_ranks).all()
+    assert (sc == o_sc).all() or np.allclose(sc, o_sc, rtol=1e-6)
+
+
 @pytest.mark.parametrize("score", ["distmult", "complex"])
 def test_tensor_core_topk_against_bf16_operand_oracle(oracle64, score):
     """Full-entity scoring on tensor cores (bf16 operands, fp32 accumulation) against the oracle
