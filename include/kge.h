@@ -207,6 +207,37 @@ int kge_score_all_topk_host(kge_handle* h, const int32_t* q_heads, const int32_t
                             void* stream);
 
 /*
+ * Full-entity inference with the entity table sharded row-wise over several devices (Section 4 "Inference": the heads of
+ * the queries are shared between the workers, every worker scores all queries against its own shard and returns its
+ * top-K, and a final top-K over the D K gathered candidates selects the predictions).  The handle is bound to ONE shard:
+ * its num_entities rows are the entities [ent_base, ent_base + num_entities) of the whole table; relation tables are whole
+ * on every device.  Entity ids in q_heads, true_tails and in the outputs are ids of the whole table.  The library does
+ * not communicate: between these calls the caller sums or gathers the small per-query arrays over the devices.
+ *
+ *   kge_shard_query_vectors  qvec_out [nq, d]: the query vector of every query whose head lies in this shard, zeros for
+ *                            the others.  Summed over the shards (each head lies in exactly one) this is every query's
+ *                            vector, bit for bit as a single device builds it.
+ *   kge_shard_true_scores    ftrue_out [nq]: the score of the true tail, from the summed query vectors, for the true
+ *                            tails that lie in this shard; zeros for the others.  Sum over the shards.
+ *   kge_shard_score_topk     the summed qvec (and ftrue, true_tails, or all three NULL) against this shard: out_ids /
+ *                            out_scores [nq, k] its k best tails as in kge_score_all_topk, out_beat [nq] the number of
+ *                            its entities ordered before the true tail.  Synchronises `stream`.
+ *   kge_merge_topk           cand_ids / cand_scores [nq, per_query] (the shards' lists side by side, per_query <= 2048,
+ *                            places holding id -1 ignored) -> out_ids / out_scores [nq, k], the k best under (score
+ *                            descending, id ascending).  The rank of the true tail is 1 + the sum of the shards' out_beat.
+ * nq must not exceed the max_queries the workspace was sized for, k not its topk.
+ */
+int kge_shard_query_vectors(kge_handle* h, const int32_t* q_heads, const int32_t* q_rels, int32_t nq, int64_t ent_base,
+                            float* qvec_out, void* stream);
+int kge_shard_true_scores(kge_handle* h, const float* qvec, const int32_t* q_rels, const int32_t* true_tails, int32_t nq,
+                          int64_t ent_base, float* ftrue_out, void* stream);
+int kge_shard_score_topk(kge_handle* h, const float* qvec, const int32_t* q_rels, int32_t nq, int32_t k, const float* ftrue,
+                         const int32_t* true_tails, int64_t ent_base, int32_t* out_ids, float* out_scores, int32_t* out_beat,
+                         void* stream);
+int kge_merge_topk(const int32_t* cand_ids, const float* cand_scores, int32_t nq, int32_t per_query, int32_t k,
+                   int32_t* out_ids, float* out_scores, void* stream);
+
+/*
  * Tensor-core inference (KGE_PREC_BF16_TC, DistMult / ComplEx) scores against a bf16 copy of the
  * entity table kept in the workspace.  The copy is made by the first kge_score_all_topk / kge_eval_mrr
  * after kge_bind and again after every kge_train_step or kge_init_tables on this handle; a caller that

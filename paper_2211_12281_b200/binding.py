@@ -89,6 +89,10 @@ SIGNATURES = {
                                             _vp, _vp]),
     "kge_score_all_topk_host": (C.c_int, [_vp, _vp, _vp, C.c_int32, C.c_int32, _vp, _vp, _vp, _vp, _vp]),
     "kge_refresh_inference_table": (C.c_int, [_vp, _vp]),
+    "kge_shard_query_vectors": (C.c_int, [_vp, _vp, _vp, C.c_int32, C.c_int64, _vp, _vp]),
+    "kge_shard_true_scores": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int32, C.c_int64, _vp, _vp]),
+    "kge_shard_score_topk": (C.c_int, [_vp, _vp, _vp, C.c_int32, C.c_int32, _vp, _vp, C.c_int64, _vp, _vp, _vp, _vp]),
+    "kge_merge_topk": (C.c_int, [_vp, _vp, C.c_int32, C.c_int32, C.c_int32, _vp, _vp, _vp]),
     "kge_measure_alu": (C.c_int, [C.c_int32, C.c_int32, C.POINTER(C.c_double), _vp]),
     "kge_eval_mrr": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int32, C.c_int32, C.POINTER(C.c_double), _vp]),
     "kge_mrr_from_ranks": (C.c_int, [_vp, _vp, C.c_int32, C.c_int32, C.POINTER(C.c_double), _vp]),
@@ -159,6 +163,12 @@ def measure_alu(mix: int, iters: int = 4096) -> float:
     if rc != 0:
         raise KgeError(rc, "kge_measure_alu", lib().kge_error_string(rc).decode())
     return out.value
+
+
+def merge_topk(cand_ids, cand_scores, k, out_ids, out_scores) -> int:
+    """kge_merge_topk on device tensors: cand_* [nq, per_query] -> out_* [nq, k]."""
+    nq, per_query = cand_ids.shape
+    return int(lib().kge_merge_topk(_ptr(cand_ids), _ptr(cand_scores), nq, per_query, k, _ptr(out_ids), _ptr(out_scores), _stream()))
 
 
 def ensemble_rank_scores(power: float, k_list: int):
@@ -261,6 +271,19 @@ class Kge:
         self._check(lib().kge_score_all_topk_host(self._h, _ptr(q_heads), _ptr(q_rels), len(q_heads), k, _ptr(true_tails),
                                                   _ptr(out_ids), _ptr(out_scores), _ptr(out_ranks), _stream()),
                     "kge_score_all_topk_host")
+
+    def shard_query_vectors(self, q_heads, q_rels, ent_base, qvec_out):
+        self._check(lib().kge_shard_query_vectors(self._h, _ptr(q_heads), _ptr(q_rels), q_heads.numel(), ent_base, _ptr(qvec_out),
+                                                  _stream()), "kge_shard_query_vectors")
+
+    def shard_true_scores(self, qvec, q_rels, true_tails, ent_base, ftrue_out):
+        self._check(lib().kge_shard_true_scores(self._h, _ptr(qvec), _ptr(q_rels), _ptr(true_tails), q_rels.numel(), ent_base,
+                                                _ptr(ftrue_out), _stream()), "kge_shard_true_scores")
+
+    def shard_score_topk(self, qvec, q_rels, k, ftrue, true_tails, ent_base, out_ids, out_scores, out_beat=None):
+        self._check(lib().kge_shard_score_topk(self._h, _ptr(qvec), _ptr(q_rels), q_rels.numel(), k, _ptr(ftrue), _ptr(true_tails),
+                                               ent_base, _ptr(out_ids), _ptr(out_scores), _ptr(out_beat), _stream()),
+                    "kge_shard_score_topk")
 
     def refresh_inference_table(self):
         self._check(lib().kge_refresh_inference_table(self._h, _stream()), "kge_refresh_inference_table")

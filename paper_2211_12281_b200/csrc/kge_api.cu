@@ -546,6 +546,41 @@ int kge_score_all_topk_host(kge_handle* h, const int32_t* q_heads, const int32_t
     return KGE_OK;
 }
 
+int kge_shard_query_vectors(kge_handle* h, const int32_t* q_heads, const int32_t* q_rels, int32_t nq, int64_t ent_base,
+                            float* qvec_out, void* stream) {
+    if (!h || !q_heads || !q_rels || !qvec_out || nq <= 0 || ent_base < 0) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    if (nq > h->max_queries) return KGE_ERR_WORKSPACE;
+    return run_shard_query_vectors(h, q_heads, q_rels, nq, ent_base, qvec_out, static_cast<cudaStream_t>(stream));
+}
+
+int kge_shard_true_scores(kge_handle* h, const float* qvec, const int32_t* q_rels, const int32_t* true_tails, int32_t nq,
+                          int64_t ent_base, float* ftrue_out, void* stream) {
+    if (!h || !qvec || !q_rels || !true_tails || !ftrue_out || nq <= 0 || ent_base < 0) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    if (nq > h->max_queries) return KGE_ERR_WORKSPACE;
+    return run_shard_true_scores(h, qvec, q_rels, true_tails, nq, ent_base, ftrue_out, static_cast<cudaStream_t>(stream));
+}
+
+int kge_shard_score_topk(kge_handle* h, const float* qvec, const int32_t* q_rels, int32_t nq, int32_t k, const float* ftrue,
+                         const int32_t* true_tails, int64_t ent_base, int32_t* out_ids, float* out_scores, int32_t* out_beat,
+                         void* stream) {
+    if (!h || !qvec || !q_rels || !out_ids || !out_scores || nq <= 0 || k <= 0 || ent_base < 0) return KGE_ERR_BAD_ARG;
+    if ((out_beat != nullptr) != (true_tails != nullptr) || (true_tails != nullptr) != (ftrue != nullptr)) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    if (nq > h->max_queries || k > h->topk) return KGE_ERR_WORKSPACE;
+    if (ent_base + h->cfg.num_entities > INT32_MAX) return KGE_ERR_BAD_ARG;     // ids stay 32-bit
+    const ShardScoring shard{ent_base, qvec, ftrue};
+    return run_score_all_topk(h, nullptr, q_rels, nq, k, true_tails, out_ids, out_scores, out_beat, static_cast<cudaStream_t>(stream), &shard);
+}
+
+int kge_merge_topk(const int32_t* cand_ids, const float* cand_scores, int32_t nq, int32_t per_query, int32_t k, int32_t* out_ids,
+                   float* out_scores, void* stream) {
+    if (!cand_ids || !cand_scores || !out_ids || !out_scores || nq < 0 || per_query <= 0 || k <= 0) return KGE_ERR_BAD_ARG;
+    if (nq == 0) return KGE_OK;
+    return run_merge_topk(cand_ids, cand_scores, nq, per_query, k, out_ids, out_scores, static_cast<cudaStream_t>(stream));
+}
+
 int kge_refresh_inference_table(kge_handle* h, void* stream) {
     if (!h) return KGE_ERR_BAD_ARG;
     if (!h->bound) return KGE_ERR_NOT_READY;

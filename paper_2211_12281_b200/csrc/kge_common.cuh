@@ -199,16 +199,24 @@ int launch_th_forward(kge_handle* h, cudaStream_t s);
 int launch_th_backward(kge_handle* h, cudaStream_t sq, cudaStream_t st);
 int launch_tc_forward(kge_handle* h, cudaStream_t s);
 int launch_cast_bf16(kge_handle* h, const float* src, uint16_t* dst, int64_t count, cudaStream_t s);
-int launch_tc_infer_chunk(kge_handle* h, int nq, int64_t e_lo, int64_t e_hi, const int32_t* true_tails, cudaStream_t s);
+int launch_tc_infer_chunk(kge_handle* h, int nq, int64_t e_lo, int64_t e_hi, const int32_t* true_tails, int64_t id_base, cudaStream_t s);
 int dedup_tiles(int n);     // sort tiles of a list of n ids
 // On-device graph preprocessing and table initialisation (kge_graph.cu).
 size_t graph_hist_words(int64_t num_triples);
 int launch_graph_build_device(kge_handle* h, const int32_t* heads, const int32_t* rels, const int32_t* tails, int64_t n,
                               cudaStream_t s);
 int launch_init_table(kge_handle* h, float* out, int64_t rows, int width, float std, int kind, uint32_t stream_id, cudaStream_t s);
+// Sharded inference: the bound table holds the entities [ent_base, ent_base + E) of a larger table; query vectors
+// (and true-tail scores) were assembled from all shards, ids are global, out_ranks receives the shard's beat counts.
+struct ShardScoring { int64_t ent_base; const float* qvec; const float* ftrue; };
 int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int32_t nq, int32_t k,
                        const int32_t* true_tails, int32_t* out_ids, float* out_scores, int32_t* out_ranks,
-                       cudaStream_t s);
+                       cudaStream_t s, const ShardScoring* shard = nullptr);
+int run_shard_query_vectors(kge_handle* h, const int32_t* qh, const int32_t* qr, int32_t nq, int64_t ent_base, float* qvec_out, cudaStream_t s);
+int run_shard_true_scores(kge_handle* h, const float* qvec, const int32_t* qr, const int32_t* true_tails, int32_t nq, int64_t ent_base,
+                          float* ftrue_out, cudaStream_t s);
+int run_merge_topk(const int32_t* cand_ids, const float* cand_scores, int32_t nq, int32_t per_query, int32_t k, int32_t* out_ids,
+                   float* out_scores, cudaStream_t s);
 
 #ifdef __CUDACC__
 // ---- device helpers ----

@@ -14,6 +14,8 @@
 #include <cmath>
 #include <vector>
 
+#include <cuda_bf16.h>
+
 #include "kge_common.cuh"
 
 namespace kge {
@@ -28,6 +30,12 @@ struct InferParams {
     int64_t e_lo, e_hi;            // entity range of this launch
     int q_tiles;
     int wait_limit;                // tries of a bounded barrier wait
+    // sharded inference (Section 4 "Inference"): the bound table is the shard [id_base, id_base + E) of a larger one;
+    // query vectors and true-tail scores come from outside (they need rows of other shards), ids are global
+    int64_t id_base;
+    const float* ext_q;            // [nq, d] finished query vectors, or NULL: build them from qh, qr
+    const float* ext_ftrue;        // [nq] scores of the true tails, or NULL: score them here
+    int raw_beat;                  // out_ranks receives the shard's count of entities ordered before the true tail, not 1 + count
     Workspace w;
 };
 
@@ -79,14 +87,18 @@ __device__ __forceinline__ bool ordered_before(float fa, int32_t ia, float fb, i
 // query set-up: one thread per query builds q (and the TransH unit normal) sequentially,
 // scores the true tail, and resets the query's running state.
 // ------------------------------------------------------------------------------------------
-__global__ void query_setup_kernel(InferParams p) {
-    const int q = blockIdx.x * blockDim.x + threadIdx.x;
-    if (q >= p.nq) return;
+// TransH: the unit normal of relation rid into wh, sequentially.
+__device__ __forceinline__ void unit_normal_seq(const InferParams& p, int64_t rid, float* wh) {
+    const float* w = p.relw + rid * p.d;
+    float s = 0.f;
+    for (int k = 0; k < p.d; ++k) s = __fmaf_rn(w[k], w[k], s);
+    const float den = fmaxf(__fsqrt_rn(s), 1e-12f);
+    for (int k = 0; k < p.d; ++k) wh[k] = __fdiv_rn(w[k], den);
+}
+
+// Query vector of (head row h, relation rid) into qv (and the TransH unit normal into wh), sequentially.
+__device__ __forceinline__ void build_query_seq(const InferParams& p, const float* h, int64_t rid, float* qv, float* wh) {
     const int d = p.d;
-    const float* h = p.ent + checked_id(p.qh[q], p.E, p.w.status) * d;
-    const int64_t rid = checked_id(p.qr[q], p.R, p.w.status);
-    float* qv = p.w.iq + (int64_t)q * d;
-    float* wh = p.score == KGE_TRANSH ? p.w.iwhat + (int64_t)q * d : nullptr;
     if (p.score == KGE_TRANSE) {
         const float* r = p.rel + rid * d;
         for (int k = 0; k < d; ++k) qv[k] = __fadd_rn(h[k], r[k]);
@@ -108,16 +120,17 @@ __global__ void query_setup_kernel(InferParams p) {
         }
     } else {  // TransH
         const float* r = p.rel + rid * d;
-        const float* w = p.relw + rid * d;
-        float s = 0.f;
-        for (int k = 0; k < d; ++k) s = __fmaf_rn(w[k], w[k], s);
-        const float den = fmaxf(__fsqrt_rn(s), 1e-12f);
+        unit_normal_seq(p, rid, wh);
         float a = 0.f;
-        for (int k = 0; k < d; ++k) { wh[k] = __fdiv_rn(w[k], den); a = __fmaf_rn(wh[k], h[k], a); }
+        for (int k = 0; k < d; ++k) a = __fmaf_rn(wh[k], h[k], a);
         for (int k = 0; k < d; ++k) qv[k] = __fadd_rn(__fmaf_rn(-a, wh[k], h[k]), r[k]);
     }
-    if (p.tt) {
-        const float* t = p.ent + checked_id(p.tt[q], p.E, p.w.status) * d;
+}
+
+// Canonical score of (query vector qv, unit normal wh, tail row t).
+__device__ __forceinline__ float score_seq(const InferParams& p, const float* qv, const float* wh, const float* t) {
+    const int d = p.d;
+    {
         float acc = 0.f;
         if (p.score == KGE_TRANSH) {
             float u = 0.f;
@@ -136,8 +149,25 @@ __global__ void query_setup_kernel(InferParams p) {
                 else canon_update<KIND_CL1>(acc, q4, t4);
             }
         }
-        p.w.iftrue[q] = canon_finish(p.kind, acc);
+        return canon_finish(p.kind, acc);
     }
+}
+
+__global__ void query_setup_kernel(InferParams p) {
+    const int q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.nq) return;
+    const int d = p.d;
+    const int64_t rid = checked_id(p.qr[q], p.R, p.w.status);
+    float* qv = p.w.iq + (int64_t)q * d;
+    float* wh = p.score == KGE_TRANSH ? p.w.iwhat + (int64_t)q * d : nullptr;
+    if (p.ext_q) {   // sharded: the query vector was built by the shard that holds the head
+        for (int k = 0; k < d; ++k) qv[k] = p.ext_q[(int64_t)q * d + k];
+        if (wh) unit_normal_seq(p, rid, wh);
+    } else {
+        build_query_seq(p, p.ent + checked_id(p.qh[q], p.E, p.w.status) * d, rid, qv, wh);
+    }
+    if (p.ext_ftrue) p.w.iftrue[q] = p.ext_ftrue[q];
+    else if (p.tt) p.w.iftrue[q] = score_seq(p, qv, wh, p.ent + checked_id(p.tt[q], p.E, p.w.status) * d);
     for (int j = 0; j < p.k; ++j) {
         p.w.top_score[(int64_t)q * p.k + j] = -INFINITY;
         p.w.top_id[(int64_t)q * p.k + j] = INT_MAX;
@@ -167,12 +197,13 @@ __device__ __forceinline__ void score_tile_epilogue(const InferParams& p, const 
             const int64_t e = e0 + tx + 16 * j;
             if (!qin || e >= p.e_hi) continue;
             const float f = canon_finish(KIND, acc[i][j]);
-            if (p.tt && ordered_before(f, (int32_t)e, ft, tt)) ++beat;
-            if (ordered_before(f, (int32_t)e, thr, thr_id)) {
+            const int32_t ge = (int32_t)(e + p.id_base);       // the id the caller knows the entity by
+            if (p.tt && ordered_before(f, ge, ft, tt)) ++beat;
+            if (ordered_before(f, ge, thr, thr_id)) {
                 const int slot = atomicAdd(&p.w.cand_cnt[q], 1);
                 if (slot < kCandCap) {
                     p.w.cand_score[(int64_t)q * kCandCap + slot] = f;
-                    p.w.cand_id[(int64_t)q * kCandCap + slot] = (int32_t)e;
+                    p.w.cand_id[(int64_t)q * kCandCap + slot] = ge;
                 } else {
                     p.w.status[1] = 1;   // this chunk overflowed a list: the host redoes it in small pieces
                 }
@@ -423,6 +454,78 @@ __global__ void ftrue_bf16_kernel(InferParams p) {
     p.w.iftrue[q] = acc;
 }
 
+// ---- sharded inference: the pieces that need rows of one shard only ----
+// Query vectors of the queries whose head lies in this shard; zeros for the others, so that a sum over the shards
+// (every head lies in exactly one) gives every query's vector exactly.
+__global__ void shard_query_kernel(InferParams p, float* qvec_out, float* wh_scratch) {
+    const int q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.nq) return;
+    const int64_t hid = (int64_t)p.qh[q] - p.id_base;
+    float* qv = qvec_out + (int64_t)q * p.d;
+    if (hid < 0 || hid >= p.E) { for (int k = 0; k < p.d; ++k) qv[k] = 0.f; return; }
+    const int64_t rid = checked_id(p.qr[q], p.R, p.w.status);
+    build_query_seq(p, p.ent + hid * p.d, rid, qv, p.score == KGE_TRANSH ? wh_scratch + (int64_t)q * p.d : nullptr);
+}
+
+// Scores of the true tails that lie in this shard, from finished query vectors; zeros for the others.  bf16_rows: the
+// tensor-core arithmetic (query vector and tail row rounded to bf16, fp32 accumulation).
+__global__ void shard_ftrue_kernel(InferParams p, const float* qvec, float* wh_scratch, float* f_out, const uint16_t* bf16_rows) {
+    const int q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.nq) return;
+    const int64_t tid = (int64_t)p.tt[q] - p.id_base;
+    if (tid < 0 || tid >= p.E) { f_out[q] = 0.f; return; }
+    const float* qv = qvec + (int64_t)q * p.d;
+    if (bf16_rows) {
+        const uint16_t* tb = bf16_rows + tid * p.d;
+        float acc = 0.f;
+        for (int k = 0; k < p.d; ++k) {
+            const __nv_bfloat16 qb = __float2bfloat16_rn(qv[k]);
+            acc = __fmaf_rn(__bfloat162float(qb), __uint_as_float((uint32_t)tb[k] << 16), acc);
+        }
+        f_out[q] = acc;
+        return;
+    }
+    float* wh = nullptr;
+    if (p.score == KGE_TRANSH) { wh = wh_scratch + (int64_t)q * p.d; unit_normal_seq(p, checked_id(p.qr[q], p.R, p.w.status), wh); }
+    f_out[q] = score_seq(p, qv, wh, p.ent + tid * p.d);
+}
+
+// Final top-k of a query over the candidates gathered from all shards: one CTA per query sorts per_query (score, id)
+// pairs under (score descending, id ascending); unused places (id -1) sort last.
+constexpr int MERGE_THREADS = 128, MERGE_MAX = 2048;
+__global__ void __launch_bounds__(MERGE_THREADS) merge_topk_kernel(const int32_t* cand_ids, const float* cand_scores, int per_query, int k,
+                                                                   int32_t* out_ids, float* out_scores) {
+    __shared__ float ss[MERGE_MAX];
+    __shared__ int32_t si[MERGE_MAX];
+    const int q = blockIdx.x, tid = threadIdx.x;
+    int n2 = 1;
+    while (n2 < per_query) n2 <<= 1;
+    for (int i = tid; i < n2; i += MERGE_THREADS) {
+        float s = -INFINITY; int32_t id = INT_MAX;
+        if (i < per_query) {
+            id = cand_ids[(int64_t)q * per_query + i]; s = cand_scores[(int64_t)q * per_query + i];
+            if (id < 0) { id = INT_MAX; s = -INFINITY; }
+        }
+        ss[i] = s; si[i] = id;
+    }
+    __syncthreads();
+    for (int size = 2; size <= n2; size <<= 1)
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            for (int t = tid; t < n2 / 2; t += MERGE_THREADS) {
+                const int lo = 2 * t - (t & (stride - 1)), hi = lo + stride;
+                const bool up = (lo & size) == 0;
+                const float a = ss[lo], b = ss[hi]; const int32_t ia = si[lo], ib = si[hi];
+                if (ordered_before(b, ib, a, ia) == up) { ss[lo] = b; si[lo] = ib; ss[hi] = a; si[hi] = ia; }
+            }
+            __syncthreads();
+        }
+    for (int i = tid; i < k; i += MERGE_THREADS) {
+        const bool have = i < n2 && si[i] != INT_MAX;
+        out_ids[(int64_t)q * k + i] = have ? si[i] : -1;
+        out_scores[(int64_t)q * k + i] = have ? ss[i] : -INFINITY;
+    }
+}
+
 __global__ void reset_chunk_kernel(InferParams p) {
     const int q = blockIdx.x * blockDim.x + threadIdx.x;
     if (q < p.nq) { p.w.cand_cnt[q] = 0; p.w.beat_tmp[q] = 0; }
@@ -438,7 +541,7 @@ __global__ void finish_kernel(InferParams p, int32_t* out_ids, float* out_scores
             out_ids[(int64_t)q * p.k + j] = id == INT_MAX ? -1 : id;
             out_scores[(int64_t)q * p.k + j] = p.w.top_score[(int64_t)q * p.k + j];
         }
-    if (out_ranks) out_ranks[q] = 1 + p.w.beat[q];
+    if (out_ranks) out_ranks[q] = (p.raw_beat ? 0 : 1) + p.w.beat[q];
 }
 
 cudaError_t launch_score_tiles(const InferParams& p, cudaStream_t s) {
@@ -457,9 +560,8 @@ cudaError_t launch_score_tiles(const InferParams& p, cudaStream_t s) {
 
 }  // namespace
 
-int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int32_t nq, int32_t k,
-                       const int32_t* true_tails, int32_t* out_ids, float* out_scores, int32_t* out_ranks,
-                       cudaStream_t s) {
+namespace {
+InferParams infer_params(kge_handle* h, const int32_t* qh, const int32_t* qr, int32_t nq, int32_t k, const int32_t* true_tails) {
     const kge_config& c = h->cfg;
     InferParams p;
     p.nq = nq; p.k = k; p.d = c.dim; p.d4 = c.dim / 4; p.score = c.score; p.kind = h->kind;
@@ -468,8 +570,48 @@ int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int3
     p.qh = qh; p.qr = qr; p.tt = true_tails;
     p.q_tiles = (nq + IQ - 1) / IQ;
     p.wait_limit = h->wait_limit;
+    p.id_base = 0; p.ext_q = nullptr; p.ext_ftrue = nullptr; p.raw_beat = 0;
     p.w = h->ws;
     p.e_lo = 0; p.e_hi = 0;
+    return p;
+}
+}  // namespace
+
+int run_shard_query_vectors(kge_handle* h, const int32_t* qh, const int32_t* qr, int32_t nq, int64_t ent_base, float* qvec_out, cudaStream_t s) {
+    InferParams p = infer_params(h, qh, qr, nq, 1, nullptr);
+    p.id_base = ent_base;
+    shard_query_kernel<<<(nq + 127) / 128, 128, 0, s>>>(p, qvec_out, h->ws.iwhat);
+    KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
+}
+
+int run_shard_true_scores(kge_handle* h, const float* qvec, const int32_t* qr, const int32_t* true_tails, int32_t nq, int64_t ent_base,
+                          float* ftrue_out, cudaStream_t s) {
+    InferParams p = infer_params(h, nullptr, qr, nq, 1, true_tails);
+    p.id_base = ent_base;
+    if (h->ws.Eb && !h->eb_valid) {       // tensor-core arithmetic scores against the bf16 copy of the shard
+        const int rc = launch_cast_bf16(h, h->ent, h->ws.Eb, h->cfg.num_entities * h->cfg.dim, s);
+        if (rc != KGE_OK) return rc;
+        h->eb_valid = true;
+    }
+    shard_ftrue_kernel<<<(nq + 127) / 128, 128, 0, s>>>(p, qvec, h->ws.iwhat, ftrue_out, h->ws.Eb);
+    KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
+}
+
+int run_merge_topk(const int32_t* cand_ids, const float* cand_scores, int32_t nq, int32_t per_query, int32_t k, int32_t* out_ids,
+                   float* out_scores, cudaStream_t s) {
+    if (per_query > MERGE_MAX) return KGE_ERR_WORKSPACE;
+    merge_topk_kernel<<<nq, MERGE_THREADS, 0, s>>>(cand_ids, cand_scores, per_query, k, out_ids, out_scores);
+    return cudaGetLastError() == cudaSuccess ? KGE_OK : KGE_ERR_CUDA;
+}
+
+int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int32_t nq, int32_t k,
+                       const int32_t* true_tails, int32_t* out_ids, float* out_scores, int32_t* out_ranks,
+                       cudaStream_t s, const ShardScoring* shard) {
+    const kge_config& c = h->cfg;
+    InferParams p = infer_params(h, qh, qr, nq, k, true_tails);
+    if (shard) { p.id_base = shard->ent_base; p.ext_q = shard->qvec; p.ext_ftrue = shard->ftrue; p.raw_beat = 1; }
     const int qblocks = (nq + 127) / 128;
     query_setup_kernel<<<qblocks, 128, 0, s>>>(p);
     KGE_LAUNCH_CHECK(h);
@@ -482,11 +624,13 @@ int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int3
             if (rc == KGE_OK) h->eb_valid = true;
         }
         if (rc != KGE_OK) return rc;
-        ftrue_bf16_kernel<<<qblocks, 128, 0, s>>>(p);
-        KGE_LAUNCH_CHECK(h);
+        if (!p.ext_ftrue) {
+            ftrue_bf16_kernel<<<qblocks, 128, 0, s>>>(p);
+            KGE_LAUNCH_CHECK(h);
+        }
     }
     auto score_chunk = [&](const InferParams& ip) -> int {
-        if (tc) return launch_tc_infer_chunk(h, nq, ip.e_lo, ip.e_hi, true_tails, s);
+        if (tc) return launch_tc_infer_chunk(h, nq, ip.e_lo, ip.e_hi, true_tails, ip.id_base, s);
         KGE_CUDA_CHECK(h, launch_score_tiles(ip, s));
         KGE_LAUNCH_CHECK(h);
         return KGE_OK;
@@ -616,7 +760,7 @@ extern "C" int kge_score_all_topk_static(const kge_config* cfg, const float* ent
     // the array still holds the previous call's words: the status header must start at zero
     // (the per-query state is rewritten by the query set-up kernel)
     KGE_CUDA_CHECK(&h, cudaMemsetAsync(w.status, 0, 256, s));
-    int rc = run_score_all_topk(&h, q_heads, q_rels, nq, k, true_tails, out_ids, out_scores, out_ranks, s);
+    int rc = run_score_all_topk(&h, q_heads, q_rels, nq, k, true_tails, out_ids, out_scores, out_ranks, s, nullptr);
     if (rc != KGE_OK) return rc;
     int32_t word = 0;
     KGE_CUDA_CHECK(&h, cudaMemcpyAsync(&word, w.status, 4, cudaMemcpyDeviceToHost, s));

@@ -67,6 +67,7 @@ struct TcGemmParams {
     // full-entity scoring (EPI_TOPK): rows are queries, columns the entities [n_base, n_base + N)
     int m_fastest;                        // walk the row tiles of one column tile first (the column tile stays in L2)
     int64_t n_base;
+    int64_t id_base;                      // the caller's id of table row 0 (sharded inference)
     const float *thr, *ftrue;             // [M] current k-th best score; score of the true tail
     const int32_t *thr_id, *tt;           // [M] its id; true tail ids (or NULL)
     int32_t *cand_cnt, *beat_tmp;         // [M] candidates appended in this chunk; entities ordered before the true tail
@@ -388,7 +389,7 @@ __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const Tc
         const int ncol = it.n0 + c0;
         const int valid = min(32, p.N - ncol);          // the same for every lane
         if (valid <= 0) continue;
-        const int32_t e0 = (int32_t)(p.n_base + ncol);
+        const int32_t e0 = (int32_t)(p.n_base + p.id_base + ncol);
         if (valid != 32) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) if (i >= valid) v[i] = -INFINITY;   // never counted, never a candidate
@@ -913,7 +914,7 @@ int launch_cast_bf16(kge_handle* h, const float* src, uint16_t* dst, int64_t cou
 
 // One chunk of full-entity scoring on tensor cores: the bf16 query vectors against the bf16
 // rows [e_lo, e_hi) of the entity table, survivors appended to the candidate lists.
-int launch_tc_infer_chunk(kge_handle* h, int nq, int64_t e_lo, int64_t e_hi, const int32_t* true_tails, cudaStream_t s) {
+int launch_tc_infer_chunk(kge_handle* h, int nq, int64_t e_lo, int64_t e_hi, const int32_t* true_tails, int64_t id_base, cudaStream_t s) {
     const Workspace& w = h->ws;
     TcGemmParams p{};
     p.M = nq; p.N = (int)(e_hi - e_lo); p.K = h->cfg.dim;
@@ -923,7 +924,7 @@ int launch_tc_infer_chunk(kge_handle* h, int nq, int64_t e_lo, int64_t e_hi, con
     if ((int64_t)p.tiles_m * p.tiles_n > 0x7fffffff) return KGE_ERR_BAD_ARG;
     p.items = p.tiles_m * p.tiles_n;
     p.status = w.status; p.wait_limit = h->wait_limit;
-    p.m_fastest = 1; p.n_base = e_lo;
+    p.m_fastest = 1; p.n_base = e_lo; p.id_base = id_base;
     p.thr = w.thr; p.thr_id = w.thr_id; p.ftrue = w.iftrue; p.tt = true_tails;
     p.cand_cnt = w.cand_cnt; p.beat_tmp = w.beat_tmp; p.cand_score = w.cand_score; p.cand_id = w.cand_id;
     p.cand_cap = kCandCap; p.overflow = w.status + 1;

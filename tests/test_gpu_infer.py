@@ -60,10 +60,9 @@ def test_topk_rank_mrr_against_fp32_oracle(oracle32, oracle64, score, p):
 
 
 @pytest.mark.parametrize("score,p,d", [("transe", 1, 128), ("distmult", 1, 40), ("transe", 2, 64), ("complex", 1, 128)])
-def test_many_query_tiles_stream_past_resident_entity_tiles(oracle32, score, p, d):
-    """With four or more 64-query tiles and rows of at most 128 floats a thread block keeps its entity tile and streams
-    the query tiles past it (double buffer): 300 queries (a ragged fifth tile), 3,000 entities (ragged last tile, chunks
-    1024 + 1024 + 952), exact ties; ids, scores and ranks bit-exact against the fp32 oracle."""
+def test_five_query_tiles_with_a_ragged_last_one(oracle32, score, p, d):
+    """300 queries (a ragged fifth 64-query tile) against 3,000 entities (ragged last tile, chunks 1024 + 1024 + 952)
+    with exact ties: ids, scores and ranks bit-exact against the fp32 oracle."""
     import kge_synth
     E, R, K, nq = 3000, 9, 10, 300
     prob = Problem(E=E, R=R, T=100, d=d, score=score, p_norm=p, B=4, N=4, P=1, graph_seed=19)
