@@ -47,6 +47,9 @@
  *                        L3 regulariser switched on, both forms).
  *   l3_term            : hand values (1, -2, 2) -> 17^(1/3) and 17; homogeneity.
  *   lr_linear_decay    : end points, midpoint, linearity.
+ *   encoder_*          : e = e_S + M e_F against numpy for one slot; central finite differences of the
+ *                        encoder batch loss in every coordinate of M_H, M_T and the shallow rows; the
+ *                        shared-matrix step against the sum of the two gradients.
  *   ensemble_topk      : a hand-worked 3-model example (p = -0.5, p = 1), reciprocal-rank fusion (p = -1)
  *                        restated in numpy, invariance under a permutation of the models, the id tie rule.
  *   dedup/update_rows  : naive scatter when all ids differ; hand sums when they repeat;
@@ -855,6 +858,143 @@ double kgeo_train_step(const kgeo_config *c, double lr, uint64_t step,
         kgeo_update_rows(c, lr, step, relw, relw_state, d, uniq, seg, perm, U, rows);
     }
     free(dh); free(dtp); free(dr); free(dw); free(dtn); free(G); free(gpos);
+    free(ids); free(uniq); free(seg); free(perm); free(rows);
+    return loss;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Encoder (Section 3.1 "Encoder", Eq. 1): the embedding of an entity is its     */
+/* trainable shallow row plus a linear projection of its fixed text features,     */
+/*   e = e_S + M_H e_F  as a head,   e = e_S + M_T e_F  as a tail (positive or     */
+/* negative), M_H, M_T in R^{d x |e_F|} trainable (optionally one shared matrix).  */
+/* The batch functions below build the final embeddings of the batch's 2B + N      */
+/* slots [heads | tails | negs] as a compact table and hand it to the functions    */
+/* above, so that scores, losses and their derivatives are exactly those already   */
+/* pinned; the chain rule then gives                                               */
+/*   dL/de_S[id] += dL/de[slot]   and   dL/dM_X += dL/de[slot] (x) e_F[id].         */
+/* bf16_operands = 1 also rounds M to bf16 inside the projection (the features are  */
+/* stored as bf16 values already), as the tensor-core projection does.              */
+/* ------------------------------------------------------------------------- */
+static void encoder_slots(const kgeo_config *c, int32_t F, const real *ent, const real *feat,
+                          const real *MH, const real *MT,
+                          const int32_t *heads, const int32_t *tails, const int32_t *negs, real *slots) {
+    const int32_t B = c->batch, N = c->num_neg, d = c->dim;
+    for (int32_t s = 0; s < 2 * B + N; ++s) {
+        const int32_t id = s < B ? heads[s] : (s < 2 * B ? tails[s - B] : negs[s - 2 * B]);
+        const real *M = s < B ? MH : MT;
+        const real *f = feat + (size_t)id * F;
+        for (int k = 0; k < d; ++k) {
+            real acc = 0;
+            for (int j = 0; j < F; ++j) {
+                real m = M[(size_t)k * F + j];
+                acc = R_FMA(c->bf16_operands ? bf16_round(m) : m, f[j], acc);
+            }
+            slots[(size_t)s * d + k] = ent[(size_t)id * d + k] + acc;
+        }
+    }
+}
+
+static void slot_batch(int32_t B, int32_t N, int32_t *h, int32_t *t, int32_t *n) {
+    for (int32_t b = 0; b < B; ++b) { h[b] = b; t[b] = B + b; }
+    for (int32_t i = 0; i < N; ++i) n[i] = 2 * B + i;
+}
+
+/* Batch loss with the encoder (feat: [E, F] features, MH / MT: [d, F]). */
+double kgeo_encoder_batch_loss(const kgeo_config *c, int32_t F, const real *ent, const real *feat,
+                               const real *MH, const real *MT, const real *rel, const real *relw,
+                               const int32_t *heads, const int32_t *rels, const int32_t *tails, const int32_t *negs) {
+    const int32_t B = c->batch, N = c->num_neg, d = c->dim;
+    real *slots = (real *)malloc(sizeof(real) * (size_t)(2 * B + N) * d);
+    int32_t *sh = (int32_t *)malloc(sizeof(int32_t) * (size_t)(2 * B + N)), *st = sh + B, *sn = sh + 2 * B;
+    encoder_slots(c, F, ent, feat, MH, MT, heads, tails, negs, slots);
+    slot_batch(B, N, sh, st, sn);
+    kgeo_config cc = *c; cc.num_entities = 2 * B + N;
+    double loss = kgeo_batch_loss(&cc, slots, rel, relw, sh, rels, st, sn, NULL, NULL, NULL, NULL);
+    free(slots); free(sh);
+    return loss;
+}
+
+/*
+ * Gradients with the encoder.  Outputs: the per-slot rows dh[B,d], dtpos[B,d], dtneg[N,d] (= dL/de of the slot,
+ * which is also the gradient of the slot's shallow row), dr, dw as in kgeo_batch_grads, and the dense dMH[d,F],
+ * dMT[d,F] (overwritten; with MH == MT the caller adds the two).
+ */
+double kgeo_encoder_batch_grads(const kgeo_config *c, int32_t F, const real *ent, const real *feat,
+                                const real *MH, const real *MT, const real *rel, const real *relw,
+                                const int32_t *heads, const int32_t *rels, const int32_t *tails, const int32_t *negs,
+                                real *dh, real *dtpos, real *dr, real *dw, real *dtneg, real *dMH, real *dMT) {
+    const int32_t B = c->batch, N = c->num_neg, d = c->dim;
+    real *slots = (real *)malloc(sizeof(real) * (size_t)(2 * B + N) * d);
+    int32_t *sh = (int32_t *)malloc(sizeof(int32_t) * (size_t)(2 * B + N)), *st = sh + B, *sn = sh + 2 * B;
+    real *G = (real *)malloc(sizeof(real) * (size_t)B * N), *gpos = (real *)malloc(sizeof(real) * (size_t)B);
+    encoder_slots(c, F, ent, feat, MH, MT, heads, tails, negs, slots);
+    slot_batch(B, N, sh, st, sn);
+    kgeo_config cc = *c; cc.num_entities = 2 * B + N;
+    double loss = kgeo_batch_grads(&cc, slots, rel, relw, sh, rels, st, sn, dh, dtpos, dr, dw, dtneg, G, gpos);
+    memset(dMH, 0, sizeof(real) * (size_t)d * F);
+    memset(dMT, 0, sizeof(real) * (size_t)d * F);
+    for (int32_t s = 0; s < 2 * B + N; ++s) {          /* slots in ascending order */
+        const int32_t id = s < B ? heads[s] : (s < 2 * B ? tails[s - B] : negs[s - 2 * B]);
+        const real *g = s < B ? dh + (size_t)s * d : (s < 2 * B ? dtpos + (size_t)(s - B) * d : dtneg + (size_t)(s - 2 * B) * d);
+        real *dM = s < B ? dMH : dMT;
+        const real *f = feat + (size_t)id * F;
+        for (int k = 0; k < d; ++k)
+            for (int j = 0; j < F; ++j) dM[(size_t)k * F + j] += g[k] * f[j];
+    }
+    free(slots); free(sh); free(G); free(gpos);
+    return loss;
+}
+
+/* Dense optimiser step on a [rows, width] matrix (the projection matrices): every row is "touched". */
+static void update_dense(const kgeo_config *c, double lr, uint64_t step, real *M, real *state, int32_t rows, int32_t width, const real *g) {
+    int32_t *ids = (int32_t *)malloc(sizeof(int32_t) * (size_t)rows * 3 + sizeof(int32_t));
+    int32_t *uniq = ids, *seg = ids + rows, *perm = ids + 2 * rows + 1;
+    const real **gr = (const real **)malloc(sizeof(real *) * (size_t)rows);
+    for (int32_t r = 0; r < rows; ++r) { uniq[r] = r; seg[r] = r; perm[r] = r; gr[r] = g + (size_t)r * width; }
+    seg[rows] = rows;
+    kgeo_update_rows(c, lr, step, M, state, width, uniq, seg, perm, rows, gr);
+    free(ids); free(gr);
+}
+
+/*
+ * One training step with the encoder, in place: shallow rows, relation rows (and normals) as in kgeo_train_step, the
+ * projection matrices by the same optimiser rule applied densely (Adam state [d, 2F]; row-wise Adagrad one value per
+ * row of M).  shared != 0: MH and MT are one matrix (pass the same pointer twice) and its gradient is dMH + dMT.
+ */
+double kgeo_encoder_train_step(const kgeo_config *c, int32_t F, int32_t shared, double lr, uint64_t step,
+                               real *ent, const real *feat, real *MH, real *MT, real *rel, real *relw,
+                               real *ent_state, real *MH_state, real *MT_state, real *rel_state, real *relw_state,
+                               const int32_t *heads, const int32_t *rels, const int32_t *tails, const int32_t *negs) {
+    const int32_t B = c->batch, N = c->num_neg, d = c->dim;
+    const int kw = rel_width(c->score, d);
+    real *dh = (real *)malloc(sizeof(real) * (size_t)B * d), *dtp = (real *)malloc(sizeof(real) * (size_t)B * d);
+    real *dr = (real *)malloc(sizeof(real) * (size_t)B * kw), *dw = relw ? (real *)malloc(sizeof(real) * (size_t)B * d) : NULL;
+    real *dtn = (real *)malloc(sizeof(real) * (size_t)N * d);
+    real *dMH = (real *)malloc(sizeof(real) * (size_t)d * F), *dMT = (real *)malloc(sizeof(real) * (size_t)d * F);
+    double loss = kgeo_encoder_batch_grads(c, F, ent, feat, MH, MT, rel, relw, heads, rels, tails, negs, dh, dtp, dr, dw, dtn, dMH, dMT);
+    const int32_t ne = 2 * B + N;
+    int32_t *ids = (int32_t *)malloc(sizeof(int32_t) * (size_t)ne), *uniq = (int32_t *)malloc(sizeof(int32_t) * (size_t)ne);
+    int32_t *seg = (int32_t *)malloc(sizeof(int32_t) * ((size_t)ne + 1)), *perm = (int32_t *)malloc(sizeof(int32_t) * (size_t)ne);
+    const real **rows = (const real **)malloc(sizeof(real *) * (size_t)ne);
+    for (int32_t b = 0; b < B; ++b) { ids[b] = heads[b]; rows[b] = dh + (size_t)b * d; ids[B + b] = tails[b]; rows[B + b] = dtp + (size_t)b * d; }
+    for (int32_t n = 0; n < N; ++n) { ids[2 * B + n] = negs[n]; rows[2 * B + n] = dtn + (size_t)n * d; }
+    int32_t U = kgeo_dedup(ids, ne, uniq, seg, perm);
+    kgeo_update_rows(c, lr, step, ent, ent_state, d, uniq, seg, perm, U, rows);
+    for (int32_t b = 0; b < B; ++b) rows[b] = dr + (size_t)b * kw;
+    U = kgeo_dedup(rels, B, uniq, seg, perm);
+    kgeo_update_rows(c, lr, step, rel, rel_state, kw, uniq, seg, perm, U, rows);
+    if (relw) {
+        for (int32_t b = 0; b < B; ++b) rows[b] = dw + (size_t)b * d;
+        kgeo_update_rows(c, lr, step, relw, relw_state, d, uniq, seg, perm, U, rows);
+    }
+    if (shared) {
+        for (size_t i = 0; i < (size_t)d * F; ++i) dMH[i] += dMT[i];
+        update_dense(c, lr, step, MH, MH_state, d, F, dMH);
+    } else {
+        update_dense(c, lr, step, MH, MH_state, d, F, dMH);
+        update_dense(c, lr, step, MT, MT_state, d, F, dMT);
+    }
+    free(dh); free(dtp); free(dr); free(dw); free(dtn); free(dMH); free(dMT);
     free(ids); free(uniq); free(seg); free(perm); free(rows);
     return loss;
 }

@@ -275,6 +275,48 @@ class Oracle:
                                               _p(heads, C.c_int32), _p(rels, C.c_int32), _p(tails, C.c_int32),
                                               _p(negs, C.c_int32)))
 
+    # -- encoder (Eq. 1) -------------------------------------------------------------------
+    def encoder_batch_loss(self, cfg, ent, feat, MH, MT, rel, relw, heads, rels, tails, negs):
+        ent, feat, MH, MT, rel = map(self.arr, (ent, feat, MH, MT, rel))
+        relw = None if relw is None else self.arr(relw)
+        heads, rels, tails, negs = map(self._i32, (heads, rels, tails, negs))
+        R = self.creal
+        self.lib.kgeo_encoder_batch_loss.restype = C.c_double
+        return float(self.lib.kgeo_encoder_batch_loss(C.byref(cfg), C.c_int32(feat.shape[1]), _p(ent, R), _p(feat, R), _p(MH, R), _p(MT, R),
+                                                      _p(rel, R), _p(relw, R), _p(heads, C.c_int32), _p(rels, C.c_int32),
+                                                      _p(tails, C.c_int32), _p(negs, C.c_int32)))
+
+    def encoder_batch_grads(self, cfg, ent, feat, MH, MT, rel, relw, heads, rels, tails, negs):
+        ent, feat, MH, MT, rel = map(self.arr, (ent, feat, MH, MT, rel))
+        relw = None if relw is None else self.arr(relw)
+        heads, rels, tails, negs = map(self._i32, (heads, rels, tails, negs))
+        R = self.creal
+        B, N, d, F = cfg.batch, cfg.num_neg, cfg.dim, feat.shape[1]
+        kw = d // 2 if cfg.score == ROTATE else d
+        dh, dtpos, dtneg = np.empty((B, d), self.real), np.empty((B, d), self.real), np.empty((N, d), self.real)
+        dr = np.empty((B, kw), self.real)
+        dw = None if relw is None else np.empty((B, d), self.real)
+        dMH, dMT = np.empty((d, F), self.real), np.empty((d, F), self.real)
+        self.lib.kgeo_encoder_batch_grads.restype = C.c_double
+        loss = self.lib.kgeo_encoder_batch_grads(C.byref(cfg), C.c_int32(F), _p(ent, R), _p(feat, R), _p(MH, R), _p(MT, R), _p(rel, R),
+                                                 _p(relw, R), _p(heads, C.c_int32), _p(rels, C.c_int32), _p(tails, C.c_int32),
+                                                 _p(negs, C.c_int32), _p(dh, R), _p(dtpos, R), _p(dr, R), _p(dw, R), _p(dtneg, R),
+                                                 _p(dMH, R), _p(dMT, R))
+        return dict(loss=float(loss), dh=dh, dtpos=dtpos, dr=dr, dw=dw, dtneg=dtneg, dMH=dMH, dMT=dMT)
+
+    def encoder_train_step(self, cfg, shared, lr, step, ent, feat, MH, MT, rel, relw, ent_state, MH_state, MT_state, rel_state,
+                           relw_state, heads, rels, tails, negs):
+        """In place on arrays of this build's real type.  shared: MH and MT must be the same array."""
+        R = self.creal
+        for a in (ent, feat, MH, MT, rel, relw, ent_state, MH_state, MT_state, rel_state, relw_state):
+            assert a is None or (a.dtype == self.real and a.flags.c_contiguous)
+        heads, rels, tails, negs = map(self._i32, (heads, rels, tails, negs))
+        self.lib.kgeo_encoder_train_step.restype = C.c_double
+        return float(self.lib.kgeo_encoder_train_step(C.byref(cfg), C.c_int32(feat.shape[1]), C.c_int32(1 if shared else 0), C.c_double(lr),
+                                                      C.c_uint64(step), _p(ent, R), _p(feat, R), _p(MH, R), _p(MT, R), _p(rel, R), _p(relw, R),
+                                                      _p(ent_state, R), _p(MH_state, R), _p(MT_state, R), _p(rel_state, R), _p(relw_state, R),
+                                                      _p(heads, C.c_int32), _p(rels, C.c_int32), _p(tails, C.c_int32), _p(negs, C.c_int32)))
+
     # -- inference ------------------------------------------------------------------------
     def score_all_topk(self, cfg: Config, ent, rel, relw, qh, qr, K, true_tails=None, ent_lo=0, ent_hi=None):
         ent, rel = self.arr(ent), self.arr(rel)
