@@ -88,6 +88,8 @@ typedef struct {
     uint64_t seed;          /* sampler seed (Philox key); also keys kge_init_tables */
     float reg_lambda;       /* lambda_S >= 0 of the L3 regulariser (Section 3.1 "Regularisation"); 0 = off */
     int32_t reg_form;       /* 0: sum of the norms ||e||_3 as printed; 1: sum of the cubes ||e||_3^3 */
+    int32_t feat_dim;       /* |e_F| of the feature-projection encoder (Eq. 1); 0 = no encoder; % 64 == 0 (the paper's is 768) */
+    int32_t feat_shared;    /* 1: M_H and M_T are one matrix */
 } kge_config;
 
 /* Validate the configuration and create the handle.  Allocates nothing on the device. */
@@ -109,6 +111,20 @@ int kge_bind(kge_handle* h, float* ent, float* rel, float* relw,
              float* ent_state, float* rel_state, float* relw_state,
              void* workspace, size_t workspace_bytes,
              int64_t num_triples, int32_t max_queries, int32_t topk, void* stream);
+
+/*
+ * Feature-projection encoder (Section 3.1 "Encoder", Eq. 1; handles created with feat_dim = F > 0): the embedding of an
+ * entity is its shallow row plus a linear projection of its fixed text features, e = e_S + M_H e_F as a head and
+ * e = e_S + M_T e_F as a (positive or negative) tail.  feat: [E, F] bf16 features (read only); MH, MT: [d, F] fp32
+ * trainable matrices (the same pointer twice when feat_shared = 1); *_state: their optimiser state (Adam [d, 2F],
+ * row-wise Adagrad [d], NULL for SGD).  Call after kge_bind.  kge_train_step then projects the features of the batch's
+ * 2B + N slots on tensor cores (bf16 operands, fp32 accumulation -- the (B + N) |e_F| d term of the cost model in
+ * Section 4.1), adds the projections to the gathered rows, and after the backward forms dM_H = sum_b dL/de_b (x) e_F and
+ * dM_T likewise (tensor cores, gradient rows rounded to bf16) and steps the matrices with the handle's optimiser, every
+ * row of a matrix touched; the shallow rows' gradients are the slots' gradient rows as before.  The regulariser applies to
+ * the final embeddings (Omega_T).  Full-entity scoring is not offered on handles with an encoder (KGE_ERR_UNSUPPORTED).
+ */
+int kge_bind_features(kge_handle* h, const uint16_t* feat, float* MH, float* MT, float* MH_state, float* MT_state, void* stream);
 
 /*
  * Graph preprocessing (Section 4 "Partitioning"): logical partition part(e) = e div S,

@@ -108,7 +108,7 @@ typedef struct {
     int32_t batch, num_neg, num_parts;
     int32_t head_part;     /* -1: slots spread over all P*P buckets; i: micro-batch B_i */
     int32_t sample_mode;   /* 0: cube-root relation law; 1: uniform over the bucket */
-    int32_t _pad;
+    int32_t bf16_projection; /* 1: the encoder's projection M e_F takes M rounded to bf16 (tensor-core variant) */
     double gamma, adv_temp, ce_correction, loss_scale;
     double lr, beta1, beta2, eps;
     uint64_t seed;
@@ -872,7 +872,7 @@ double kgeo_train_step(const kgeo_config *c, double lr, uint64_t step,
 /* above, so that scores, losses and their derivatives are exactly those already   */
 /* pinned; the chain rule then gives                                               */
 /*   dL/de_S[id] += dL/de[slot]   and   dL/dM_X += dL/de[slot] (x) e_F[id].         */
-/* bf16_operands = 1 also rounds M to bf16 inside the projection (the features are  */
+/* bf16_projection = 1 rounds M to bf16 inside the projection (the features are     */
 /* stored as bf16 values already), as the tensor-core projection does.              */
 /* ------------------------------------------------------------------------- */
 static void encoder_slots(const kgeo_config *c, int32_t F, const real *ent, const real *feat,
@@ -887,7 +887,7 @@ static void encoder_slots(const kgeo_config *c, int32_t F, const real *ent, cons
             real acc = 0;
             for (int j = 0; j < F; ++j) {
                 real m = M[(size_t)k * F + j];
-                acc = R_FMA(c->bf16_operands ? bf16_round(m) : m, f[j], acc);
+                acc = R_FMA(c->bf16_projection ? bf16_round(m) : m, f[j], acc);
             }
             slots[(size_t)s * d + k] = ent[(size_t)id * d + k] + acc;
         }

@@ -36,7 +36,7 @@ class Config(C.Structure):
         ("dim", C.c_int32), ("score", C.c_int32), ("p_norm", C.c_int32), ("loss", C.c_int32),
         ("opt", C.c_int32), ("bf16_operands", C.c_int32),
         ("batch", C.c_int32), ("num_neg", C.c_int32), ("num_parts", C.c_int32),
-        ("head_part", C.c_int32), ("sample_mode", C.c_int32), ("_pad", C.c_int32),
+        ("head_part", C.c_int32), ("sample_mode", C.c_int32), ("bf16_projection", C.c_int32),
         ("gamma", C.c_double), ("adv_temp", C.c_double), ("ce_correction", C.c_double),
         ("loss_scale", C.c_double),
         ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
@@ -48,14 +48,14 @@ class Config(C.Structure):
 def make_config(*, num_entities, num_relations, dim, score, p_norm=1, loss="logsigmoid", opt="sgd",
                 bf16_operands=0, batch=1, num_neg=1, num_parts=1, head_part=-1, sample_mode=0,
                 gamma=0.0, adv_temp=0.0, ce_correction=0.0, loss_scale=1.0, lr=0.1,
-                beta1=0.9, beta2=0.999, eps=None, seed=0, reg_lambda=0.0, reg_form=0) -> Config:
+                beta1=0.9, beta2=0.999, eps=None, seed=0, reg_lambda=0.0, reg_form=0, bf16_projection=0) -> Config:
     score = SCORE_NAMES[score] if isinstance(score, str) else int(score)
     loss = LOSS_NAMES[loss] if isinstance(loss, str) else int(loss)
     opt = OPT_NAMES[opt] if isinstance(opt, str) else int(opt)
     if eps is None:
         eps = 1e-10 if opt == OPT_ROWWISE_ADAGRAD else 1e-8
     return Config(num_entities, num_relations, dim, score, p_norm, loss, opt, bf16_operands,
-                  batch, num_neg, num_parts, head_part, sample_mode, 0,
+                  batch, num_neg, num_parts, head_part, sample_mode, bf16_projection,
                   gamma, adv_temp, ce_correction, loss_scale, lr, beta1, beta2, eps, seed, reg_lambda, reg_form, 0)
 
 

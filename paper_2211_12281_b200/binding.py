@@ -46,14 +46,14 @@ class KgeConfig(C.Structure):
         ("gamma", C.c_float), ("adv_temp", C.c_float), ("ce_correction", C.c_float), ("loss_scale", C.c_float),
         ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
         ("seed", C.c_uint64),
-        ("reg_lambda", C.c_float), ("reg_form", C.c_int32),
+        ("reg_lambda", C.c_float), ("reg_form", C.c_int32), ("feat_dim", C.c_int32), ("feat_shared", C.c_int32),
     ]
 
     @classmethod
     def make(cls, *, num_entities, num_relations, dim, score, p_norm=1, loss="logsigmoid", opt="sgd",
              prec=PREC_FP32, batch=1, num_neg=1, num_parts=1, head_part=-1, sample_mode=0,
              gamma=0.0, adv_temp=0.0, ce_correction=0.0, loss_scale=1.0, lr=0.1,
-             beta1=0.9, beta2=0.999, eps=None, seed=0, reg_lambda=0.0, reg_form=0) -> "KgeConfig":
+             beta1=0.9, beta2=0.999, eps=None, seed=0, reg_lambda=0.0, reg_form=0, feat_dim=0, feat_shared=0) -> "KgeConfig":
         score = SCORE_NAMES[score] if isinstance(score, str) else int(score)
         loss = LOSS_NAMES[loss] if isinstance(loss, str) else int(loss)
         opt = OPT_NAMES[opt] if isinstance(opt, str) else int(opt)
@@ -61,7 +61,7 @@ class KgeConfig(C.Structure):
             eps = 1e-10 if opt == OPT_ROWWISE_ADAGRAD else 1e-8
         return cls(num_entities, num_relations, dim, score, p_norm, loss, opt, prec, batch, num_neg,
                    num_parts, head_part, sample_mode, 0, gamma, adv_temp, ce_correction, loss_scale,
-                   lr, beta1, beta2, eps, seed, reg_lambda, reg_form)
+                   lr, beta1, beta2, eps, seed, reg_lambda, reg_form, feat_dim, feat_shared)
 
 
 def library_path() -> Path:
@@ -77,6 +77,7 @@ SIGNATURES = {
     "kge_destroy": (None, [_vp]),
     "kge_workspace_bytes": (C.c_size_t, [_vp, C.c_int64, C.c_int32, C.c_int32]),
     "kge_bind": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_size_t, C.c_int64, C.c_int32, C.c_int32, _vp]),
+    "kge_bind_features": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kge_graph_load": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int64, _vp]),
     "kge_graph_load_device": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int64, _vp]),
     "kge_init_tables": (C.c_int, [_vp, C.c_float, _vp]),
@@ -231,6 +232,12 @@ class Kge:
         self._check(lib().kge_bind(self._h, _ptr(ent), _ptr(rel), _ptr(relw), _ptr(ent_state), _ptr(rel_state),
                                    _ptr(relw_state), C.c_void_p(ws.data_ptr()), ws.numel(), num_triples,
                                    max_queries, topk, _stream()), "kge_bind")
+
+    def bind_features(self, feat, MH, MT, MH_state=None, MT_state=None):
+        """feat: bfloat16 [E, F] device tensor; MH, MT: float32 [d, F] (the same tensor twice for a shared matrix)."""
+        self._keep += [feat, MH, MT, MH_state, MT_state]
+        self._check(lib().kge_bind_features(self._h, _ptr(feat), _ptr(MH), _ptr(MT), _ptr(MH_state), _ptr(MT_state), _stream()),
+                    "kge_bind_features")
 
     def graph_load(self, heads, rels, tails):
         """heads / rels / tails: numpy int32 host arrays."""

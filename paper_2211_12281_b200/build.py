@@ -16,7 +16,7 @@ CSRC = PKG / "csrc"
 LIB = PKG / "libkge.so"
 OBJ = PKG / "_build"
 SOURCES = ["kge_api.cu", "kge_sample.cu", "kge_train.cu", "kge_tc.cu", "kge_update.cu", "kge_infer.cu",
-           "kge_graph.cu", "kge_ensemble.cu", "kge_bench.cu", "kge_transh.cu"]
+           "kge_graph.cu", "kge_ensemble.cu", "kge_bench.cu", "kge_transh.cu", "kge_encoder.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 

@@ -94,6 +94,14 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
     w.Tneg = cv.take<float>(N * d);
     w.fpos = cv.take<float>(B); w.gpos = cv.take<float>(B); w.Lrow = cv.take<float>(B);
     w.reg_s3 = c.reg_lambda > 0.f ? cv.take<float>(2 * B + N) : nullptr;
+    if (c.feat_dim > 0) {
+        const size_t F = c.feat_dim;
+        w.Fb = cv.take<uint16_t>((2 * B + N) * F);
+        w.Mb = cv.take<uint16_t>(2 * d * F);
+        w.proj = cv.take<float>((2 * B + N) * d);
+        w.Gslot = cv.take<uint16_t>((2 * B + N) * d);
+        w.dMpart = cv.take<float>((size_t)2 * h->split_m * d * F);
+    }
     const bool tc = c.prec == KGE_PREC_BF16_TC;
     w.Qb = tc ? cv.take<uint16_t>(B * d) : nullptr;
     w.Tb = tc ? cv.take<uint16_t>(N * d) : nullptr;
@@ -212,6 +220,9 @@ int kge_create(const kge_config* cfg, kge_handle** out) {
     if (c.sample_mode != 0 && c.sample_mode != 1) return KGE_ERR_BAD_ARG;
     if (!(c.adv_temp >= 0.f)) return KGE_ERR_BAD_ARG;
     if (!(c.reg_lambda >= 0.f) || (c.reg_form != 0 && c.reg_form != 1)) return KGE_ERR_BAD_ARG;
+    if (c.feat_dim < 0 || (c.feat_shared != 0 && c.feat_shared != 1)) return KGE_ERR_BAD_ARG;
+    // the projection runs on tensor cores: 64-element slices of the feature axis, 16-byte aligned bf16 rows of width d
+    if (c.feat_dim > 0 && (c.feat_dim % 64 != 0 || c.dim % 8 != 0)) return KGE_ERR_UNSUPPORTED;
     if ((int64_t)c.batch * c.num_neg > ((int64_t)1 << 31)) return KGE_ERR_BAD_ARG;
     const int64_t P = c.num_parts;
     if (c.num_neg % P != 0) return KGE_ERR_DIVISIBILITY;
@@ -254,6 +265,10 @@ int kge_create(const kge_config* cfg, kge_handle** out) {
         h->split_q = pick_split_tc(c.batch, c.dim, c.num_neg, h->num_sms);
         h->split_t = pick_split_tc(c.num_neg, c.dim, c.batch, h->num_sms);
     }
+    h->split_m = 1;
+    h->features_bound = false;
+    if (c.feat_dim > 0)   // dM = dE^T . F: [d, F] over the batch's slots, split over the slots so that every SM has a tile
+        h->split_m = pick_split_tc(c.dim, c.feat_dim, c.batch, h->num_sms);
     *out = h;
     return KGE_OK;
 }
@@ -347,6 +362,22 @@ int kge_bind(kge_handle* h, float* ent, float* rel, float* relw, float* ent_stat
     h->bound = true;
     h->graph_loaded = false;
     h->eb_valid = false;
+    return KGE_OK;
+}
+
+int kge_bind_features(kge_handle* h, const uint16_t* feat, float* MH, float* MT, float* MH_state, float* MT_state, void* stream) {
+    (void)stream;
+    if (!h || !feat || !MH || !MT) return KGE_ERR_BAD_ARG;
+    if (h->cfg.feat_dim <= 0) return KGE_ERR_UNSUPPORTED;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    if ((h->cfg.feat_shared != 0) != (MH == MT)) return KGE_ERR_BAD_ARG;
+    if (h->cfg.opt != KGE_OPT_SGD && (!MH_state || !MT_state)) return KGE_ERR_BAD_ARG;
+    auto misaligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) % 16) != 0; };
+    if (misaligned(feat) || misaligned(MH) || misaligned(MT)) return KGE_ERR_BAD_ARG;
+    h->feat = feat; h->MH = MH; h->MT = MT; h->MH_state = MH_state; h->MT_state = MT_state;
+    const int rc = encoder_make_maps(h);
+    if (rc != KGE_OK) return rc;
+    h->features_bound = true;
     return KGE_OK;
 }
 
@@ -467,12 +498,17 @@ int kge_train_step(kge_handle* h, uint64_t step, float lr, const int32_t* heads,
         // triple bucket and the bucket's cumulative weights fit its shared memory.
         const kge_config& c = h->cfg;
         const int buckets = c.head_part < 0 ? c.num_parts * c.num_parts : c.num_parts;
-        fused = fork && (c.batch / buckets) % 8 == 0 && c.num_relations + 1 <= 4096;
+        // (with an encoder the ids must exist before the gather: the features of the batch are projected first)
+        fused = fork && (c.batch / buckets) % 8 == 0 && c.num_relations + 1 <= 4096 && c.feat_dim == 0;
         if (!fused) {
             rc = launch_sample(h, step, w.heads, w.rels, w.tails, w.negs, s);
             if (rc != KGE_OK) return rc;
         }
         heads = w.heads; rels = w.rels; tails = w.tails; negs = w.negs;
+    }
+    if (h->cfg.feat_dim > 0) {
+        if (!h->features_bound) return KGE_ERR_NOT_READY;
+        if ((rc = launch_encoder_forward(h, heads, tails, negs, s)) != KGE_OK) return rc;
     }
     rc = launch_forward_backward(h, heads, rels, tails, negs, loss_out, s, fork ? h->side[1] : nullptr,
                                  fork ? h->side[0] : nullptr, fused, step);
@@ -480,6 +516,7 @@ int kge_train_step(kge_handle* h, uint64_t step, float lr, const int32_t* heads,
     // with side streams the id sort has been joined before the chain kernel
     if (!fork && (rc = launch_dedup(h, heads, rels, tails, negs, s)) != KGE_OK) return rc;
     rc = launch_update(h, step, lr, s);
+    if (rc == KGE_OK && h->cfg.feat_dim > 0) rc = launch_encoder_backward(h, step, lr, s);
     h->eb_valid = false;          // the entity table has moved on: tensor-core inference must refresh its bf16 copy
     if (rc != KGE_OK) return rc;
     return h->prof.on ? stage_collect(h, s) : KGE_OK;
@@ -515,6 +552,7 @@ int kge_score_all_topk(kge_handle* h, const int32_t* q_heads, const int32_t* q_r
     if (nq > 0 && (!q_heads || !q_rels || !out_ids || !out_scores)) return KGE_ERR_BAD_ARG;   // an empty batch may pass NULL
     if (out_ranks && !true_tails) return KGE_ERR_BAD_ARG;
     if (!h->bound) return KGE_ERR_NOT_READY;
+    if (h->cfg.feat_dim > 0) return KGE_ERR_UNSUPPORTED;      // full-entity scoring reads shallow rows only
     if (nq > h->max_queries || k > h->topk) return KGE_ERR_WORKSPACE;
     if (nq == 0) return KGE_OK;
     return run_score_all_topk(h, q_heads, q_rels, nq, k, true_tails, out_ids, out_scores, out_ranks,

@@ -49,6 +49,12 @@ struct Workspace {
     int32_t *heads, *rels, *tails, *negs;  // contiguous [3B+N]
     float *Q, *What, *Tneg;                // [B,d], [B,d] (TransH), [N,d]
     float *fpos, *gpos, *Lrow;             // [B]
+    // feature-projection encoder (Eq. 1)
+    uint16_t *Fb;                          // [2B+N, F] bf16 features of the batch's slots [heads | tails | negs]
+    uint16_t *Mb;                          // [2][d, F] bf16 copies of M_H, M_T
+    float *proj;                           // [2B+N, d] M e_F of every slot (added to the gathered rows)
+    uint16_t *Gslot;                       // [2B+N, d] bf16 copy of the slots' gradient rows
+    float *dMpart;                         // [2][splits][d, F] partial gradients of M_H, M_T
     float *reg_s3;                         // [2B+N] sum of |e_k|^3 of the gathered rows [heads | tails | negs] (L3 regulariser), or NULL
     uint16_t *Qb, *Tb;                     // [B,d], [N,d] bf16 copies of Q and Tneg (tensor-core scoring)
     uint16_t *Gb;                          // bf16 [B,ldN] dL/dF (ldN = N rounded up to 8)
@@ -121,6 +127,13 @@ struct kge_handle {
     // read MN-major) for dQ; Gb and Qb (64-row boxes, read MN-major) for dT
     alignas(64) unsigned char tm_q[128], tm_t[128], tm_g[128], tm_g64[128], tm_t64[128], tm_q64[128];
     alignas(64) unsigned char tm_iq[128], tm_eb[128];   // inference: bf16 query vectors and bf16 entity table
+    // encoder: features of the head / tail+negative slots and M_H / M_T (K-major, 128-row boxes) for the projection; the
+    // slots' gradient rows and features again (MN-major, 64-row boxes) for dM = dE^T . F
+    alignas(64) unsigned char tm_fh[128], tm_ft[128], tm_mh[128], tm_mt[128], tm_gh64[128], tm_gt64[128], tm_fh64[128], tm_ft64[128];
+    const uint16_t* feat;   // [E, F] bf16 text features (fixed)
+    float *MH, *MT, *MH_state, *MT_state;   // [d, F] projection matrices and their optimiser state
+    int split_m;            // K splits of the two dM contractions
+    bool features_bound;
     bool streams_ready;
     cudaStream_t side[2];
     cudaEvent_t ev_ids, ev_loss, ev_seg, ev_t;
@@ -198,6 +211,14 @@ int launch_tc_backward(kge_handle* h, cudaStream_t s, cudaStream_t side);
 int launch_th_forward(kge_handle* h, cudaStream_t s);
 int launch_th_backward(kge_handle* h, cudaStream_t sq, cudaStream_t st);
 int launch_tc_forward(kge_handle* h, cudaStream_t s);
+int launch_tc_gemm_nt(kge_handle* h, const unsigned char* tmA, const unsigned char* tmB, int M, int N, int K, float* C, int64_t ldc,
+                      cudaStream_t s);
+int launch_tc_gemm_tn(kge_handle* h, const unsigned char* tmA64, const unsigned char* tmB64, int M, int N, int K, int split, float* C,
+                      int64_t ldc, cudaStream_t s);
+// Feature-projection encoder (kge_encoder.cu): M e_F of the batch's slots before the gather; dM and the dense step after the backward.
+int encoder_make_maps(kge_handle* h);
+int launch_encoder_forward(kge_handle* h, const int32_t* heads, const int32_t* tails, const int32_t* negs, cudaStream_t s);
+int launch_encoder_backward(kge_handle* h, uint64_t step, float lr, cudaStream_t s);
 int launch_cast_bf16(kge_handle* h, const float* src, uint16_t* dst, int64_t count, cudaStream_t s);
 int launch_tc_infer_chunk(kge_handle* h, int nq, int64_t e_lo, int64_t e_hi, const int32_t* true_tails, int64_t id_base, cudaStream_t s);
 int dedup_tiles(int n);     // sort tiles of a list of n ids

@@ -857,6 +857,27 @@ int launch_tc_bwd_gemm(kge_handle* h, const unsigned char* tmA, const unsigned c
 }
 }  // namespace
 
+// Plain contractions for the feature-projection encoder, on the same kernel.
+//   C[M, N] = A[M, K] . B[N, K]^T   (both operands K-major: tensor maps with 128-row boxes)
+int launch_tc_gemm_nt(kge_handle* h, const unsigned char* tmA, const unsigned char* tmB, int M, int N, int K, float* C, int64_t ldc,
+                      cudaStream_t s) {
+    TcGemmParams p{};
+    p.M = M; p.N = N; p.K = K;
+    p.kb_per_split = (K + TC_BK - 1) / TC_BK;
+    p.C = C; p.ldc = ldc; p.split_stride = 0;
+    p.status = h->ws.status; p.wait_limit = h->wait_limit;
+    p.bn = TC_BN;
+    p.tiles_m = (M + TC_BM - 1) / TC_BM; p.tiles_n = (N + p.bn - 1) / p.bn; p.items = p.tiles_m * p.tiles_n;
+    KGE_CUDA_CHECK(h, (launch_gemm_inst<EPI_STORE, 128>(tmA, tmB, p, h->num_sms, s)));
+    KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
+}
+//   C[split][M, N] = A[K, M]^T . B[K, N] over K slices of each split (both operands MN-major: 64-row boxes)
+int launch_tc_gemm_tn(kge_handle* h, const unsigned char* tmA64, const unsigned char* tmB64, int M, int N, int K, int split, float* C,
+                      int64_t ldc, cudaStream_t s) {
+    return launch_tc_bwd_gemm<true>(h, tmA64, tmB64, M, N, K, split, C, ldc, s);
+}
+
 bool tc_negatives_direct(const kge_handle* h) {
     // (with the regulariser on, the chain kernel still has a term to add to every negative's row)
     return h->cfg.prec == KGE_PREC_BF16_TC && h->kind == KIND_DOT && h->split_t == 1 && !(h->cfg.reg_lambda > 0.f);

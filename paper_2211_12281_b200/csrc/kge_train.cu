@@ -27,6 +27,7 @@ struct TrainParams {
     int tc_l2;          // TransE p = 2 with tensor-core backward: the splits hold C.T and C^T.Q, C = dL/dF / distance
     int neg_direct;     // the dT contraction wrote the negatives' gradient rows itself (one K split, no correction term)
     int wait_limit;     // tries of a bounded barrier wait
+    const float* proj;  // feature-projection encoder: [2B+N, d] M e_F of the slots [heads | tails | negs], added to the rows read; or NULL
     float reg_lambda;   // L3 regulariser on the gathered entity rows (0 = off)
     int reg_form;       // 0: norms, 1: cubes
     Workspace w;
@@ -111,8 +112,10 @@ __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
         const float4* src = reinterpret_cast<const float4*>(p.ent) + id * d4;
         float4* dst = reinterpret_cast<float4*>(p.w.Tneg) + (int64_t)n * d4;
         float nrm2 = 0.f, s3 = 0.f;
+        const float4* pj = p.proj ? reinterpret_cast<const float4*>(p.proj) + (int64_t)(2 * p.B + n) * d4 : nullptr;
         for (int c = lane; c < d4; c += 32) {
-            const float4 v = src[c];
+            float4 v = src[c];
+            if (pj) v = f4add(v, pj[c]);       // e = e_S + M_T e_F
             dst[c] = v;
             if (p.w.Tb) {   // tensor-core scoring: bf16 copy and the squared norm of the unrounded row
                 reinterpret_cast<uint2*>(p.w.Tb)[(int64_t)n * d4 + c] = pack_bf16x4(v);
@@ -146,6 +149,10 @@ __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
         const int c = lane + 32 * i;
         h[i] = c < d4 ? hrow[c] : f4zero();
         t[i] = c < d4 ? trow[c] : f4zero();
+        if (p.proj && c < d4) {                // e = e_S + M_H e_F (head), e_S + M_T e_F (tail)
+            h[i] = f4add(h[i], reinterpret_cast<const float4*>(p.proj)[(int64_t)b * d4 + c]);
+            t[i] = f4add(t[i], reinterpret_cast<const float4*>(p.proj)[(int64_t)(p.B + b) * d4 + c]);
+        }
         q[i] = f4zero(); wh[i] = f4zero();
     }
     if (p.w.reg_s3) {
@@ -944,6 +951,10 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
         const int c = lane + 32 * i;
         const bool in = c < d4;
         h[i] = in ? hrow[c] : f4zero(); t[i] = in ? trow[c] : f4zero(); q[i] = in ? qrow[c] : f4zero();
+        if (p.proj && in) {                    // the final embeddings, as the gather kernel formed them
+            h[i] = f4add(h[i], reinterpret_cast<const float4*>(p.proj)[(int64_t)b * d4 + c]);
+            t[i] = f4add(t[i], reinterpret_cast<const float4*>(p.proj)[(int64_t)(p.B + b) * d4 + c]);
+        }
         float4 s = f4zero();
         if (in) s = sum_splits(reinterpret_cast<const float4*>(p.w.dQpart) + (int64_t)b * d4 + c, (int64_t)p.B * d4, p.split_q);
         if (p.kind == KIND_L1 && in) {   // the splits hold P; dQ = (row sum of dL/dF) - 2 P
@@ -1156,6 +1167,7 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     p.neg_direct = tc_negatives_direct(h) ? 1 : 0;
     p.wait_limit = h->wait_limit;
     p.reg_lambda = c.reg_lambda; p.reg_form = c.reg_form;
+    p.proj = c.feat_dim > 0 ? h->ws.proj : nullptr;
     p.w = h->ws;
     const int nch = p.d4 <= 32 ? 1 : (p.d4 <= 64 ? 2 : 4);
 

@@ -44,7 +44,8 @@ class Problem:
         return self.d // 2 if self.score == "rotate" else self.d
 
     def oracle_cfg(self):
-        return oracle_config(**self.kw, bf16_operands=1 if self.tc else 0)
+        kw = {k: v for k, v in self.kw.items() if k not in ("feat_dim", "feat_shared")}     # (the oracle's encoder takes them as arguments)
+        return oracle_config(**kw, bf16_operands=1 if self.tc else 0)
 
     def state_shapes(self):
         if self.opt == "sgd":

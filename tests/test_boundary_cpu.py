@@ -30,8 +30,8 @@ def test_library_exports_every_declared_symbol(K):
 
 
 def test_config_struct_matches_header_layout(K):
-    # 2 x int64 + 12 x int32 + 8 x float + uint64 + float + int32 = 112 bytes, seed 8-byte aligned
-    assert C.sizeof(K.KgeConfig) == 112 and K.KgeConfig.seed.offset == 96 and K.KgeConfig.gamma.offset == 64
+    # 2 x int64 + 12 x int32 + 8 x float + uint64 + float + 3 x int32 = 120 bytes, seed 8-byte aligned
+    assert C.sizeof(K.KgeConfig) == 120 and K.KgeConfig.seed.offset == 96 and K.KgeConfig.gamma.offset == 64
     assert K.KgeConfig.reg_lambda.offset == 104 and K.KgeConfig.reg_form.offset == 108
 
 
