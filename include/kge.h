@@ -189,6 +189,34 @@ int kge_train_step(kge_handle* h, uint64_t step, float lr,
                    float* loss_out, void* stream);
 
 /*
+ * Pieces of the training step for an entity table sharded row-wise over several devices (Section 4 "Training": worker i
+ * holds the shard E_i, processes the micro-batch B_i whose heads lie in E_i, receives the rows of its B positive tails and
+ * N negatives from their owners by a balanced AllToAll -- B/D + N/D rows from every worker, Eq. 3 and Eq. 4 -- and, not
+ * spelled out in the paper, returns their gradient rows the same way).  The library does not communicate; the caller
+ * moves the rows between devices between these calls (paper_2211_12281_b200/sharded.py does, with torch.distributed).
+ *
+ *   kge_gather_rows      rows_out [n, d] = the shard's rows of the n whole-table ids `ids` (all must lie in
+ *                        [ent_base, ent_base + num_entities), else KGE_ERR_ID_RANGE is recorded): what an owner sends.
+ *   kge_train_gradients  forward and backward of one batch exactly as kge_train_step, but nothing is de-duplicated or
+ *                        updated: the gradient rows of the slots [heads | tails | negs] ([2B+N, d]), of the relations
+ *                        ([B, k]) and of the TransH normals ([B, d]) stay in the workspace, where kge_gradient_rows
+ *                        points.  The ids index the bound table (a worker binds its shard extended by B + N rows that
+ *                        hold the received tails and negatives, and renumbers the batch accordingly).
+ *   kge_apply_gradients  table (0 entities, 1 relations, 2 TransH normals) receives n (row id, gradient row) pairs:
+ *                        stable sort by id, one optimiser step per distinct row with its gradients added in ascending
+ *                        list position -- the step's own de-duplication and update on a list of the caller's.  scratch:
+ *                        device memory of kge_apply_scratch_bytes(h, table, n) bytes, 256-byte aligned.
+ * All three enqueue on `stream` and return.
+ */
+int kge_gather_rows(kge_handle* h, const int32_t* ids, int32_t n, int64_t ent_base, float* rows_out, void* stream);
+int kge_train_gradients(kge_handle* h, uint64_t step, const int32_t* heads, const int32_t* rels, const int32_t* tails,
+                        const int32_t* negs, float* loss_out, void* stream);
+int kge_gradient_rows(kge_handle* h, float** grad_ent /*[host]*/, float** grad_rel /*[host]*/, float** grad_relw /*[host]*/);
+size_t kge_apply_scratch_bytes(const kge_handle* h, int32_t table, int32_t n);
+int kge_apply_gradients(kge_handle* h, int32_t table, const int32_t* ids, const float* grads, int32_t n, uint64_t step, float lr,
+                        void* scratch, size_t scratch_bytes, void* stream);
+
+/*
  * The same step for callers that keep the batch on the host: ids are [host] arrays (pinned
  * memory makes the copies asynchronous), copied in on `stream` (as one copy when the four
  * lists lie back to back in the order heads, rels, tails, negs); the loss is copied back to

@@ -84,6 +84,11 @@ SIGNATURES = {
     "kge_debug_init_words": (C.c_int, [_vp, _vp, C.c_int64, C.c_int32, C.c_uint32, _vp]),
     "kge_sample_batch": (C.c_int, [_vp, C.c_uint64, _vp, _vp, _vp, _vp, _vp]),
     "kge_train_step": (C.c_int, [_vp, C.c_uint64, C.c_float, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "kge_gather_rows": (C.c_int, [_vp, _vp, C.c_int32, C.c_int64, _vp, _vp]),
+    "kge_train_gradients": (C.c_int, [_vp, C.c_uint64, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "kge_gradient_rows": (C.c_int, [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp)]),
+    "kge_apply_scratch_bytes": (C.c_size_t, [_vp, C.c_int32, C.c_int32]),
+    "kge_apply_gradients": (C.c_int, [_vp, C.c_int32, _vp, _vp, C.c_int32, C.c_uint64, C.c_float, _vp, C.c_size_t, _vp]),
     "kge_train_step_host": (C.c_int, [_vp, C.c_uint64, C.c_float, _vp, _vp, _vp, _vp, _vp, _vp]),
     "kge_score_all_topk": (C.c_int, [_vp, _vp, _vp, C.c_int32, C.c_int32, _vp, _vp, _vp, _vp, _vp]),
     "kge_score_all_topk_static": (C.c_int, [C.POINTER(KgeConfig), _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32, _vp, _vp, _vp,
@@ -262,6 +267,31 @@ class Kge:
     def train_step(self, step, lr, heads=None, rels=None, tails=None, negs=None, loss_out=None):
         self._check(lib().kge_train_step(self._h, step, lr, _ptr(heads), _ptr(rels), _ptr(tails), _ptr(negs),
                                          _ptr(loss_out), _stream()), "kge_train_step")
+
+    def gather_rows(self, ids, ent_base, rows_out):
+        self._check(lib().kge_gather_rows(self._h, _ptr(ids), ids.numel(), ent_base, _ptr(rows_out), _stream()), "kge_gather_rows")
+
+    def train_gradients(self, step, heads, rels, tails, negs, loss_out=None):
+        self._check(lib().kge_train_gradients(self._h, step, _ptr(heads), _ptr(rels), _ptr(tails), _ptr(negs), _ptr(loss_out), _stream()),
+                    "kge_train_gradients")
+
+    def gradient_rows(self):
+        """Device addresses (ints) of the gradient rows of the last step: (entity slots [2B+N, d], relations [B, k], normals [B, d])."""
+        a, b, c = _vp(), _vp(), _vp()
+        self._check(lib().kge_gradient_rows(self._h, C.byref(a), C.byref(b), C.byref(c)), "kge_gradient_rows")
+        return a.value, b.value, c.value
+
+    def apply_gradients(self, table, ids, grads, step, lr, scratch=None):
+        """table: 0 entities, 1 relations, 2 normals; ids int32 [n], grads float32 [n, width] device tensors."""
+        import torch
+        n = ids.numel()
+        need = int(lib().kge_apply_scratch_bytes(self._h, table, n))
+        if scratch is None or scratch.numel() < need + 256:
+            scratch = torch.empty(need + 256, dtype=torch.uint8, device=ids.device)
+        off = (-scratch.data_ptr()) % 256
+        self._check(lib().kge_apply_gradients(self._h, table, _ptr(ids), _ptr(grads), n, step, lr, C.c_void_p(scratch.data_ptr() + off),
+                                              need, _stream()), "kge_apply_gradients")
+        return scratch
 
     def train_step_host(self, step, lr, heads, rels, tails, negs, loss_out):
         """ids and loss_out are host arrays (pinned torch tensors or numpy)."""

@@ -522,6 +522,51 @@ int kge_train_step(kge_handle* h, uint64_t step, float lr, const int32_t* heads,
     return h->prof.on ? stage_collect(h, s) : KGE_OK;
 }
 
+int kge_train_gradients(kge_handle* h, uint64_t step, const int32_t* heads, const int32_t* rels, const int32_t* tails,
+                        const int32_t* negs, float* loss_out, void* stream) {
+    if (!h || !heads || !rels || !tails || !negs) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    if (h->cfg.feat_dim > 0) return KGE_ERR_UNSUPPORTED;
+    // forward and backward only, in order on the caller's stream: no sort of the touched ids, no update
+    return launch_forward_backward(h, heads, rels, tails, negs, loss_out, static_cast<cudaStream_t>(stream), nullptr, nullptr, false, step);
+}
+
+int kge_gradient_rows(kge_handle* h, float** grad_ent, float** grad_rel, float** grad_relw) {
+    if (!h) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    if (grad_ent) *grad_ent = h->ws.grad_ent;
+    if (grad_rel) *grad_rel = h->ws.grad_rel;
+    if (grad_relw) *grad_relw = h->ws.grad_relw;
+    return KGE_OK;
+}
+
+int kge_gather_rows(kge_handle* h, const int32_t* ids, int32_t n, int64_t ent_base, float* rows_out, void* stream) {
+    if (!h || !ids || !rows_out || n < 0 || ent_base < 0) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    if (n == 0) return KGE_OK;
+    return launch_gather_rows(h, ids, n, ent_base, rows_out, static_cast<cudaStream_t>(stream));
+}
+
+size_t kge_apply_scratch_bytes(const kge_handle* h, int32_t table, int32_t n) {
+    if (!h || n <= 0 || table < 0 || table > 2) return 0;
+    return apply_scratch_bytes(n, table == 1 ? h->kw : h->cfg.dim);
+}
+
+int kge_apply_gradients(kge_handle* h, int32_t table, const int32_t* ids, const float* grads, int32_t n, uint64_t step, float lr,
+                        void* scratch, size_t scratch_bytes, void* stream) {
+    if (!h || !ids || !grads || n < 0 || table < 0 || table > 2) return KGE_ERR_BAD_ARG;
+    if (!h->bound) return KGE_ERR_NOT_READY;
+    if (n == 0) return KGE_OK;
+    float* tab = table == 0 ? h->ent : (table == 1 ? h->rel : h->relw);
+    float* state = table == 0 ? h->ent_state : (table == 1 ? h->rel_state : h->relw_state);
+    if (!tab) return KGE_ERR_BAD_ARG;
+    const int width = table == 1 ? h->kw : h->cfg.dim;
+    if (!scratch || (reinterpret_cast<uintptr_t>(scratch) % 256) != 0 || scratch_bytes < apply_scratch_bytes(n, width)) return KGE_ERR_WORKSPACE;
+    const int64_t rows = table == 0 ? h->cfg.num_entities : h->cfg.num_relations;
+    h->eb_valid = false;
+    return launch_apply_gradients(h, tab, state, rows, width, ids, grads, n, step, lr, scratch, static_cast<cudaStream_t>(stream));
+}
+
 int kge_train_step_host(kge_handle* h, uint64_t step, float lr, const int32_t* heads, const int32_t* rels,
                         const int32_t* tails, const int32_t* negs, float* loss_out, void* stream) {
     if (!h || !heads || !rels || !tails || !negs) return KGE_ERR_BAD_ARG;

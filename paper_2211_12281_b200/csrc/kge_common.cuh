@@ -200,6 +200,11 @@ int launch_dedup(kge_handle* h, const int32_t* heads, const int32_t* rels, const
                  const int32_t* negs, cudaStream_t s);
 // Segment sums of the gradient rows and the optimiser step (needs both of the above).
 int launch_update(kge_handle* h, uint64_t step, float lr, cudaStream_t s);
+// Pieces of the multi-device training step: rows of this shard for a list of ids; one list of (id, gradient row) pairs applied to a table.
+int launch_gather_rows(kge_handle* h, const int32_t* ids, int n, int64_t base, float* out, cudaStream_t s);
+size_t apply_scratch_bytes(int n, int width);
+int launch_apply_gradients(kge_handle* h, float* table, float* state, int64_t rows, int width, const int32_t* ids, const float* grads,
+                           int n, uint64_t step, float lr, void* scratch, cudaStream_t s);
 // Tensor-core score block: F from the bf16 operand copies; tensor maps are made at bind time.
 int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows);
 int tc_backward_tile_cols(int cols);

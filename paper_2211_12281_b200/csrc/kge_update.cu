@@ -352,6 +352,85 @@ int launch_dedup(kge_handle* h, const int32_t* heads, const int32_t* rels, const
     return KGE_OK;
 }
 
+// ---- one list of (row id, gradient row) pairs applied to one table, with caller-provided scratch ----
+namespace {
+struct ApplyScratch {
+    int32_t *perm, *sorted, *uniq, *seg, *segof, *done, *count, *dummy;
+    uint64_t* tkeys;
+    float* part;
+    size_t bytes;
+};
+// Carves the scratch of a list of n rows of `width` floats (base == nullptr: measures only).
+ApplyScratch carve_apply(char* base, int n, int width) {
+    size_t used = 0;
+    auto take = [&](size_t bytes) { char* p = base ? base + used : nullptr; used += (bytes + 255) / 256 * 256; return p; };
+    ApplyScratch a{};
+    a.perm = reinterpret_cast<int32_t*>(take((size_t)n * 4)); a.sorted = reinterpret_cast<int32_t*>(take((size_t)n * 4));
+    a.uniq = reinterpret_cast<int32_t*>(take((size_t)n * 4)); a.seg = reinterpret_cast<int32_t*>(take(((size_t)n + 1) * 4));
+    a.segof = reinterpret_cast<int32_t*>(take((size_t)n * 4)); a.done = reinterpret_cast<int32_t*>(take((size_t)n * 4));
+    a.count = reinterpret_cast<int32_t*>(take(256)); a.dummy = reinterpret_cast<int32_t*>(take(256));
+    a.tkeys = reinterpret_cast<uint64_t*>(take((size_t)dedup_tiles(n) * SORT_TILE * 8));
+    a.part = reinterpret_cast<float*>(take((size_t)n * width * 4));
+    a.bytes = used;
+    return a;
+}
+}  // namespace
+
+namespace {
+// One warp per requested row: out[i] = table[ids[i] - base] (an id outside the shard is reported and reads row 0).
+__global__ void __launch_bounds__(256) gather_rows_kernel(const float* table, int64_t rows, int d4, const int32_t* ids, int n, int64_t base,
+                                                          float* out, int32_t* status) {
+    const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (i >= n) return;
+    int64_t r = (int64_t)ids[i] - base;
+    if (r < 0 || r >= rows) { set_status(status, KGE_ERR_ID_RANGE); r = 0; }
+    const float4* src = reinterpret_cast<const float4*>(table) + r * d4;
+    float4* dst = reinterpret_cast<float4*>(out) + (int64_t)i * d4;
+    for (int c = lane; c < d4; c += 32) dst[c] = src[c];
+}
+}  // namespace
+
+int launch_gather_rows(kge_handle* h, const int32_t* ids, int n, int64_t base, float* out, cudaStream_t s) {
+    gather_rows_kernel<<<(n * 32 + 255) / 256, 256, 0, s>>>(h->ent, h->cfg.num_entities, h->cfg.dim / 4, ids, n, base, out, h->ws.status);
+    KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
+}
+
+size_t apply_scratch_bytes(int n, int width) { return carve_apply(nullptr, n, width).bytes; }
+
+// table[ids[i]] receives the gradient row grads[i] for i < n: stable sort of the ids, one update per distinct row with
+// the row's gradients added in ascending list position, by the handle's optimiser rule (the same kernels as the step's
+// own update).  `rows`: height of the table; state: the table's optimiser state.
+int launch_apply_gradients(kge_handle* h, float* table, float* state, int64_t rows, int width, const int32_t* ids, const float* grads,
+                           int n, uint64_t step, float lr, void* scratch, cudaStream_t s) {
+    const kge_config& c = h->cfg;
+    ApplyScratch a = carve_apply(static_cast<char*>(scratch), n, width);
+    DedupParams dp;
+    dp.ent = IdList{ids, ids, ids, n, 0, 0, rows, a.perm, a.sorted, a.uniq, a.seg, a.segof, a.done, nullptr, a.tkeys, a.count};
+    // (the kernels serve two lists at once: the second one is empty here)
+    dp.rel = IdList{ids, ids, ids, 0, 0, 0, rows, a.dummy, a.dummy, a.dummy, a.dummy, a.dummy, a.dummy, nullptr, a.tkeys, a.dummy + 32};
+    dp.ent_tiles = dedup_tiles(n);
+    dp.status = h->ws.status;
+    tile_sort_kernel<<<dp.ent_tiles, SORT_THREADS, 0, s>>>(dp);
+    KGE_LAUNCH_CHECK(h);
+    rank_kernel<<<dp.ent_tiles * (SORT_TILE / RANK_THREADS), RANK_THREADS, 0, s>>>(dp);
+    KGE_LAUNCH_CHECK(h);
+    segment_kernel<<<2, SEG_THREADS, 0, s>>>(dp);
+    KGE_LAUNCH_CHECK(h);
+    UpdateParams up;
+    up.njobs = 1;
+    up.job[0] = UpdateJob{table, state, grads, a.part, a.uniq, a.seg, a.perm, a.sorted, a.segof, a.done, width, n};
+    up.job[1] = up.job[0]; up.job[2] = up.job[0];
+    up.warp_begin[0] = 0; up.warp_begin[1] = n; up.warp_begin[2] = n; up.warp_begin[3] = n;
+    up.opt = c.opt;
+    up.lr = lr; up.beta1 = c.beta1; up.beta2 = c.beta2; up.eps = c.eps;
+    up.corr1 = (float)(1.0 - std::pow((double)c.beta1, (double)(step + 1)));
+    up.corr2 = (float)(1.0 - std::pow((double)c.beta2, (double)(step + 1)));
+    KGE_CUDA_CHECK(h, launch_dependent(piece_kernel, dim3((n * 32 + 255) / 256), dim3(256), 0, s, up));
+    KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
+}
+
 int launch_update(kge_handle* h, uint64_t step, float lr, cudaStream_t s) {
     const kge_config& c = h->cfg;
     Workspace& w = h->ws;
