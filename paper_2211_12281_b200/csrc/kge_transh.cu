@@ -52,10 +52,13 @@ __host__ __device__ inline int hb_kc(int d) { return d < HB_KC ? d : HB_KC; }
 __host__ __device__ inline int hb_stages(int d) { return d > HB_KC ? 2 : 1; }
 inline size_t hb_smem(int d) { return (size_t)hb_stages(d) * HB_ROWS * (hb_kc(d) + 4) * sizeof(float) + 2 * sizeof(uint64_t); }
 
-template <bool P1>
+// KC: the chunk length when it is known at compile time (rows of at least HB_KC floats), so that
+// every shared-memory address of the inner loops is one base per operand plus a constant; 0: rows
+// shorter than HB_KC, chunk length = row length.
+template <bool P1, int KC>
 __global__ void __launch_bounds__(HB_THREADS, 2) th_block_kernel(ThFwdParams p) {
     extern __shared__ __align__(128) unsigned char smraw[];
-    const int kc = hb_kc(p.d), ld = kc + 4, nstage = hb_stages(p.d);
+    const int kc = KC ? KC : hb_kc(p.d), ld = kc + 4, nstage = hb_stages(p.d);
     const int nchunk = (p.d + kc - 1) / kc;
     const int nload = nchunk > 1 ? 2 * nchunk : 1;       // both sweeps read every chunk; a single chunk stays where it is
     float* base = reinterpret_cast<float*>(smraw);
@@ -207,11 +210,13 @@ inline size_t ha_smem() {
 
 // OWNER_Q: owner rows are queries (own = Q, oth = Tneg); else negatives (own = Tneg, oth = Q, whose normals come along).
 // The sums run over the other side's rows in ascending order inside a split; the chain kernel adds the splits in order.
-template <bool P1, bool OWNER_Q>
+// FULL_SLAB: every column slab is HA_SLAB floats wide (d a multiple of HA_SLAB), so the row stride
+// of the staged rows is a compile-time constant.
+template <bool P1, bool OWNER_Q, bool FULL_SLAB>
 __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
     extern __shared__ __align__(128) unsigned char smraw[];
     constexpr int NT = OWNER_Q ? 4 : 3;                      // weight tiles: g, u, c (and u g for the query side)
-    const int k0 = blockIdx.z * HA_SLAB, kc = min(HA_SLAB, a.d - k0), d4s = kc >> 2;
+    const int k0 = blockIdx.z * HA_SLAB, kc = FULL_SLAB ? HA_SLAB : min(HA_SLAB, a.d - k0), d4s = kc >> 2;
     float4* Bs = reinterpret_cast<float4*>(smraw);                                   // [2][32][d4s] rows of the other side
     float4* Ws = Bs + 2 * HA_CC * (HA_SLAB / 4);                                     // [2][32][d4s] their normals (owner = negatives)
     float* Tl = reinterpret_cast<float*>(Ws + (OWNER_Q ? 0 : 2 * HA_CC * (HA_SLAB / 4)));   // [2][NT][32][36] weight tiles, [c][r]
@@ -322,7 +327,10 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
             }
         }
         if (act) {
-#pragma unroll 2
+            // not unrolled: with two or more iterations in flight the compiler keeps the next
+            // iteration's 20 loaded values in a second register set and copies them over (about
+            // 18 register moves per 80 arithmetic instructions, measured)
+#pragma unroll 1
             for (int cc = 0; cc < ccmax; ++cc) {
                 static_assert(HA_RPW == 4, "one float4 of each weight tile per warp");
                 const float4 g4 = *reinterpret_cast<const float4*>(&Gc[cc * HA_LDW + warp * HA_RPW]);
@@ -400,22 +408,26 @@ template <bool P1>
 cudaError_t launch_fwd(const ThFwdParams& p, cudaStream_t s) {
     static DeviceOnce configured;
     const cudaError_t e = once_per_device(configured, [] {
-        return cudaFuncSetAttribute(th_block_kernel<P1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hb_smem(kMaxDim));
+        const cudaError_t e0 = cudaFuncSetAttribute(th_block_kernel<P1, HB_KC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hb_smem(kMaxDim));
+        return e0 != cudaSuccess ? e0 : cudaFuncSetAttribute(th_block_kernel<P1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hb_smem(HB_KC));
     });
     if (e != cudaSuccess) return e;
     dim3 grid((p.N + HB_T - 1) / HB_T, (p.B + HB_Q - 1) / HB_Q);
-    return launch_dependent(th_block_kernel<P1>, grid, dim3(HB_THREADS), hb_smem(p.d), s, p);
+    if (p.d >= HB_KC) return launch_dependent(th_block_kernel<P1, HB_KC>, grid, dim3(HB_THREADS), hb_smem(p.d), s, p);
+    return launch_dependent(th_block_kernel<P1, 0>, grid, dim3(HB_THREADS), hb_smem(p.d), s, p);
 }
 
 template <bool P1, bool OWNER_Q>
 cudaError_t launch_acc(const ThAccArgs& a, cudaStream_t s) {
     static DeviceOnce configured;
     const cudaError_t e = once_per_device(configured, [] {
-        return cudaFuncSetAttribute(th_accum_kernel<P1, OWNER_Q>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ha_smem<OWNER_Q>());
+        const cudaError_t e0 = cudaFuncSetAttribute(th_accum_kernel<P1, OWNER_Q, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ha_smem<OWNER_Q>());
+        return e0 != cudaSuccess ? e0 : cudaFuncSetAttribute(th_accum_kernel<P1, OWNER_Q, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ha_smem<OWNER_Q>());
     });
     if (e != cudaSuccess) return e;
     dim3 grid((a.own_rows + HA_ROWS - 1) / HA_ROWS, a.split, (a.d + HA_SLAB - 1) / HA_SLAB);
-    th_accum_kernel<P1, OWNER_Q><<<grid, HA_THREADS, ha_smem<OWNER_Q>(), s>>>(a);
+    if (a.d % HA_SLAB == 0) th_accum_kernel<P1, OWNER_Q, true><<<grid, HA_THREADS, ha_smem<OWNER_Q>(), s>>>(a);
+    else th_accum_kernel<P1, OWNER_Q, false><<<grid, HA_THREADS, ha_smem<OWNER_Q>(), s>>>(a);
     return cudaSuccess;
 }
 
