@@ -151,7 +151,7 @@ constexpr int kDefaultWaitLimit = 1 << 20;   // tries of a bounded barrier wait:
     do {                                                          \
         cudaError_t e_ = (expr);                                  \
         if (e_ != cudaSuccess) {                                  \
-            std::snprintf((h)->cuda_err, sizeof((h)->cuda_err), "%s: %s", #expr, cudaGetErrorString(e_)); \
+            std::snprintf((h)->cuda_err, sizeof((h)->cuda_err), "%.160s: %s", #expr, cudaGetErrorString(e_)); \
             return KGE_ERR_CUDA;                                  \
         }                                                         \
     } while (0)

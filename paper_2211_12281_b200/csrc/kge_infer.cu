@@ -178,10 +178,26 @@ __global__ void query_setup_kernel(InferParams p) {
 
 constexpr int IQ = 64, IE = 64, IKC = 32, ILD = IKC + 4;
 
+// Largest float below x (x finite).
+__device__ __forceinline__ float float_below(float x) {
+    if (x == 0.f) return __uint_as_float(0x80000001u);
+    const uint32_t b = __float_as_uint(x);
+    return __uint_as_float(x > 0.f ? b - 1u : b + 1u);
+}
+
 // Epilogue of a 64 x 64 score tile: rank counting against the true tail, threshold filter into the
 // candidate lists.  Thread (tx, ty) holds the pairs (q0 + ty + 16 i, e0 + tx + 16 j).
+// The tile's 64 entity ids are consecutive.  If the reference id (the true tail, or the id of the
+// current k-th best) is not among them, "ordered before (f0, id0)" is the same plain comparison
+// for the whole row of the tile: f >= f0 when the tile lies below id0, f > f0 when above, and
+// f >= f0 is f > (largest float below f0).  So the common case costs one compare per pair and
+// test; a row whose reference id falls inside the tile, a ragged last tile and non-finite
+// reference scores take the element-by-element form.
 template <int KIND>
 __device__ __forceinline__ void score_tile_epilogue(const InferParams& p, const float (&acc)[4][4], int q0, int64_t e0, int tx, int ty) {
+    const int64_t g0 = e0 + p.id_base;                  // the id the caller knows the tile's first entity by
+    const bool whole = e0 + IE <= p.e_hi;
+    int beat_all = 0;                                   // four rows' counts, one byte each (at most 4 per thread, 64 per row)
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int q = q0 + ty + 16 * i;
@@ -191,28 +207,50 @@ __device__ __forceinline__ void score_tile_epilogue(const InferParams& p, const 
             thr = p.w.thr[q]; thr_id = p.w.thr_id[q];
             if (p.tt) { ft = p.w.iftrue[q]; tt = p.tt[q]; }
         }
+        auto append = [&](float f, int32_t ge) {
+            const int slot = atomicAdd(&p.w.cand_cnt[q], 1);
+            if (slot < kCandCap) {
+                p.w.cand_score[(int64_t)q * kCandCap + slot] = f;
+                p.w.cand_id[(int64_t)q * kCandCap + slot] = ge;
+            } else {
+                p.w.status[1] = 1;   // this chunk overflowed a list: the host redoes it in small pieces
+            }
+        };
+        const bool thr_out = thr_id < g0 || thr_id >= g0 + IE, tt_out = tt < g0 || tt >= g0 + IE;
+        const bool plain = whole && qin && thr_out && tt_out && fabsf(thr) < INFINITY && fabsf(ft) < INFINITY;
         int beat = 0;
+        if (plain) {
+            const float thr_c = thr_id >= g0 + IE ? float_below(thr) : thr;
+            const float ft_c = tt >= g0 + IE ? float_below(ft) : ft;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int64_t e = e0 + tx + 16 * j;
-            if (!qin || e >= p.e_hi) continue;
-            const float f = canon_finish(KIND, acc[i][j]);
-            const int32_t ge = (int32_t)(e + p.id_base);       // the id the caller knows the entity by
-            if (p.tt && ordered_before(f, ge, ft, tt)) ++beat;
-            if (ordered_before(f, ge, thr, thr_id)) {
-                const int slot = atomicAdd(&p.w.cand_cnt[q], 1);
-                if (slot < kCandCap) {
-                    p.w.cand_score[(int64_t)q * kCandCap + slot] = f;
-                    p.w.cand_id[(int64_t)q * kCandCap + slot] = ge;
-                } else {
-                    p.w.status[1] = 1;   // this chunk overflowed a list: the host redoes it in small pieces
-                }
+            for (int j = 0; j < 4; ++j) {
+                const float f = canon_finish(KIND, acc[i][j]);
+                beat += f > ft_c ? 1 : 0;
+                if (f > thr_c) append(f, (int32_t)(g0 + tx + 16 * j));
+            }
+            if (!p.tt) beat = 0;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int64_t e = e0 + tx + 16 * j;
+                if (!qin || e >= p.e_hi) continue;
+                const float f = canon_finish(KIND, acc[i][j]);
+                const int32_t ge = (int32_t)(e + p.id_base);
+                if (p.tt && ordered_before(f, ge, ft, tt)) ++beat;
+                if (ordered_before(f, ge, thr, thr_id)) append(f, ge);
             }
         }
-        // the 16 lanes sharing a query row are contiguous: one atomic per row and tile
+        beat_all |= beat << (8 * i);
+    }
+    // the 16 lanes sharing a query row are contiguous: one atomic per row and tile
 #pragma unroll
-        for (int o = 8; o > 0; o >>= 1) beat += __shfl_xor_sync(0xffffffffu, beat, o);
-        if (tx == 0 && beat > 0) atomicAdd(&p.w.beat_tmp[q], beat);
+    for (int o = 8; o > 0; o >>= 1) beat_all += __shfl_xor_sync(0xffffffffu, beat_all, o);
+    if (tx == 0 && beat_all != 0) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int beat = (beat_all >> (8 * i)) & 0xff;
+            if (beat > 0) atomicAdd(&p.w.beat_tmp[q0 + ty + 16 * i], beat);
+        }
     }
 }
 
@@ -305,11 +343,13 @@ inline size_t infer_tma_smem(int d) {
     return (size_t)infer_tma_stages(d) * (IQ + IE) * (infer_tma_kc(d) + 4) * sizeof(float) + 2 * sizeof(uint64_t);
 }
 
-template <int KIND>
+// KC: the stage length when known at compile time (rows of at least IKT floats; shared-memory
+// addresses of the inner loop are then constants off one base per operand), 0: shorter rows.
+template <int KIND, int KC>
 __global__ void __launch_bounds__(256) score_tile_tma_kernel(InferParams p) {
     extern __shared__ __align__(128) unsigned char smraw[];
     constexpr int ROWS = IQ + IE;        // rows [0, IQ) of a stage hold queries, the rest entities
-    const int kc = infer_tma_kc(p.d), ld = kc + 4, nstage = infer_tma_stages(p.d);
+    const int kc = KC ? KC : infer_tma_kc(p.d), ld = kc + 4, nstage = infer_tma_stages(p.d);
     const int nchunk = (p.d + kc - 1) / kc;
     float* base = reinterpret_cast<float*>(smraw);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smraw + (size_t)nstage * ROWS * ld * sizeof(float));
@@ -388,10 +428,12 @@ template <int KIND>
 cudaError_t launch_score_tile_tma(const InferParams& p, unsigned grid, cudaStream_t s) {
     static DeviceOnce configured;
     const cudaError_t e = once_per_device(configured, [] {
-        return cudaFuncSetAttribute(score_tile_tma_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)infer_tma_smem(kMaxDim));
+        const cudaError_t e0 = cudaFuncSetAttribute(score_tile_tma_kernel<KIND, IKT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)infer_tma_smem(kMaxDim));
+        return e0 != cudaSuccess ? e0 : cudaFuncSetAttribute(score_tile_tma_kernel<KIND, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)infer_tma_smem(IKT));
     });
     if (e != cudaSuccess) return e;
-    score_tile_tma_kernel<KIND><<<grid, 256, infer_tma_smem(p.d), s>>>(p);
+    if (p.d >= IKT) score_tile_tma_kernel<KIND, IKT><<<grid, 256, infer_tma_smem(p.d), s>>>(p);
+    else score_tile_tma_kernel<KIND, 0><<<grid, 256, infer_tma_smem(p.d), s>>>(p);
     return cudaSuccess;
 }
 

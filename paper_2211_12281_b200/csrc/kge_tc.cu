@@ -241,10 +241,6 @@ __device__ __forceinline__ void tc_epilogue_stats(const TcGemmParams& p, const T
     if (row < p.M && piece < p.row_pieces) p.stat_part[(int64_t)row * p.row_pieces + piece] = make_float4(m, z, l, 0.f);
 }
 
-__device__ __forceinline__ uint16_t bf16_bits(float v) {
-    const __nv_bfloat16 b = __float2bfloat16_rn(v);
-    return *reinterpret_cast<const uint16_t*>(&b);
-}
 __device__ __forceinline__ float bf16_value(uint16_t bits) { return __uint_as_float((uint32_t)bits << 16); }
 
 // dL/dF of one pair from its accumulator: scale = loss_scale / normaliser, k0 already holds minus

@@ -59,7 +59,7 @@ __device__ __forceinline__ float reg_coef(float lambda, int form, float s3) {
 }
 // The sub-gradient of |x| that every p = 1 kernel of this library uses: +1 for x > 0, -1 otherwise.
 // At x == 0 any value in [-1, 1] is a sub-gradient; the score-block backward counts the pairs with
-// x > 0 (see add_if_pos), which fixes -1 there, and the positive pair takes the same value so that
+// x > 0 (see add_if_gt), which fixes -1 there, and the positive pair takes the same value so that
 // a step has one convention.
 __device__ __forceinline__ float sgnf(float x) { return x > 0.f ? 1.f : -1.f; }
 __device__ __forceinline__ float4 f4sgn(float4 a) { return make_float4(sgnf(a.x), sgnf(a.y), sgnf(a.z), sgnf(a.w)); }
@@ -202,7 +202,6 @@ __global__ void __launch_bounds__(256) build_kernel(TrainParams p) {
             }
             const float inv = 1.f / fmaxf(sqrtf(warp_sum(nrm2)), 1e-12f);
             float a = 0.f;
-#pragma unroll
             float ws = 0.f;
 #pragma unroll
             for (int i = 0; i < kMaxChunks; ++i) {
@@ -284,27 +283,6 @@ __device__ __forceinline__ void pair_update(float& acc, float4 q, float4 t) {
     }
 }
 
-// acc += w where x > 0: one compare and one predicated add (two adds sharing the compare in the
-// second form).  With sign(x) = 2 [x > 0] - 1 a sum of w sign(x) is 2 P - (sum of w), P the sum
-// these accumulate; the value at x == 0 is a free choice of sub-gradient of |x| (-1: see sgnf).
-__device__ __forceinline__ void add_if_pos(float& acc, float x, float w) {
-    asm("{\n .reg .pred p;\n setp.gt.f32 p, %1, 0f00000000;\n @p add.f32 %0, %0, %2;\n}\n" : "+f"(acc) : "f"(x), "f"(w));
-}
-__device__ __forceinline__ void add2_if_pos(float& acc1, float& acc2, float x, float w1, float w2) {
-    asm("{\n .reg .pred p;\n setp.gt.f32 p, %2, 0f00000000;\n @p add.f32 %0, %0, %3;\n @p add.f32 %1, %1, %4;\n}\n"
-        : "+f"(acc1), "+f"(acc2) : "f"(x), "f"(w1), "f"(w2));
-}
-__device__ __forceinline__ void f4add_if_pos(float4& acc, float4 x, float w) {
-    add_if_pos(acc.x, x.x, w); add_if_pos(acc.y, x.y, w); add_if_pos(acc.z, x.z, w); add_if_pos(acc.w, x.w, w);
-}
-__device__ __forceinline__ void f4add_w_if_pos(float& acc, float4 x, float4 w) {   // acc += sum of w_k over the x_k > 0
-    add_if_pos(acc, x.x, w.x); add_if_pos(acc, x.y, w.y); add_if_pos(acc, x.z, w.z); add_if_pos(acc, x.w, w.w);
-}
-__device__ __forceinline__ void f4add2_if_pos(float4& acc1, float4& acc2, float4 x, float w1, float w2) {
-    add2_if_pos(acc1.x, acc2.x, x.x, w1, w2); add2_if_pos(acc1.y, acc2.y, x.y, w1, w2);
-    add2_if_pos(acc1.z, acc2.z, x.z, w1, w2); add2_if_pos(acc1.w, acc2.w, x.w, w1, w2);
-}
-
 // ------------------------------------------------------------------------------------------
 // block, kinds that are a function of (q, t) alone: 32 x 64 pairs per CTA, 4 x 4 per thread.
 // The 32 query rows and 64 negative rows of the tile are brought into shared memory by one
@@ -321,11 +299,14 @@ inline size_t block_tma_smem(int d) {
     return (size_t)block_tma_stages(d) * (FTQ + TN) * (block_tma_kc(d) + 4) * sizeof(float) + 2 * sizeof(uint64_t);
 }
 
-template <int KIND>
+// KC: the stage length when it is known at compile time (rows of at least FKC floats): every
+// shared-memory address of the inner loop is then one base per operand plus a constant, which
+// removes two integer instructions per 128-bit load.  0: shorter rows, stage length = row length.
+template <int KIND, int KC>
 __global__ void __launch_bounds__(FTHREADS) block_tma_kernel(TrainParams p) {
     extern __shared__ __align__(128) unsigned char smraw[];
     constexpr int ROWS = FTQ + TN;       // rows [0, FTQ) of a stage hold queries, the rest negatives
-    const int kc = block_tma_kc(p.d), ld = kc + 4, nstage = block_tma_stages(p.d);
+    const int kc = KC ? KC : block_tma_kc(p.d), ld = kc + 4, nstage = block_tma_stages(p.d);
     const int nchunk = (p.d + kc - 1) / kc;
     float* base = reinterpret_cast<float*>(smraw);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smraw + (size_t)nstage * ROWS * ld * sizeof(float));
@@ -377,7 +358,8 @@ __global__ void __launch_bounds__(FTHREADS) block_tma_kernel(TrainParams p) {
         const float* Qs = base + (size_t)stage * ROWS * ld;
         const float* Ts = Qs + FTQ * ld;
         const int len = min(kc, p.d - chunk * kc);
-#pragma unroll 2
+        // (measured: the plain L1 loop is fastest rolled, the others unrolled twice)
+#pragma unroll (KIND == KIND_L1 ? 1 : 2)
         for (int kk = 0; kk < len; kk += 4) {
             float4 qv[4], tv[4];
 #pragma unroll
@@ -716,13 +698,15 @@ inline size_t accum_tma_smem(int d4) {
 }
 
 // ACC_WARPS warps per CTA, 32 / ACC_WARPS owner rows per warp (8 rows while the registers last).
-template <int KIND, int NCH, bool OWNER_Q, int ACC_WARPS>
+// FULL: the rows are exactly 32 * NCH float4 long, so the row stride of the staged rows is a
+// compile-time constant and no lane is idle.
+template <int KIND, int NCH, bool OWNER_Q, int ACC_WARPS, bool FULL>
 __device__ __forceinline__ void accum_tma_body(const AccArgs& a, const int block_x, const int block_y) {
     constexpr int ACC_RPW = ACC_ROWS / ACC_WARPS;
     constexpr int ACC_THREADS = 32 * ACC_WARPS;
     constexpr int ACC_WPT = ACC_ROWS * ACC_CC / ACC_THREADS;   // weights of a tile handled per thread
     extern __shared__ __align__(128) unsigned char smraw[];
-    const int d4 = a.d4;
+    const int d4 = FULL ? 32 * NCH : a.d4;
     float4* Bs = reinterpret_cast<float4*>(smraw);                                  // [2][32][d4]
     float* Gs = reinterpret_cast<float*>(Bs + 2 * ACC_CC * d4);                     // [2][32][36], [c][r]
     float* Csum = Gs + 2 * ACC_CC * ACC_LDW;                                        // [warps][32]
@@ -807,7 +791,8 @@ __device__ __forceinline__ void accum_tma_body(const AccArgs& a, const int block
                 if (cc < ccmax) csum += Gc[cc * ACC_LDW + lane];
             }
         }
-#pragma unroll 2
+        // rolled: unrolled, the compiler holds the next iteration's operands in a second register set and copies them over
+#pragma unroll 1
         for (int cc = 0; cc < ccmax; ++cc) {
             float gw[ACC_RPW];
 #pragma unroll
@@ -818,7 +803,7 @@ __device__ __forceinline__ void accum_tma_body(const AccArgs& a, const int block
 #pragma unroll
             for (int j = 0; j < NCH; ++j) {
                 const int c = lane + 32 * j;
-                if (c >= d4) continue;
+                if (!FULL && c >= d4) continue;
                 const float4 bv = Bc[cc * d4 + c];
 #pragma unroll
                 for (int i = 0; i < ACC_RPW; ++i) acc_update2<KIND, OWNER_Q>(acc[i][j], A[i][j], bv, gw[i]);
@@ -848,12 +833,12 @@ __device__ __forceinline__ void accum_tma_body(const AccArgs& a, const int block
 
 // Both accumulations of a step in one launch: blockIdx.z = 0 owns query rows (dQ), 1 owns
 // negative rows (dT); the grid spans the larger of the two shapes.
-template <int KIND, int NCH, int ACC_WARPS>
-__global__ void __launch_bounds__(32 * ACC_WARPS) accum_tma_kernel(AccArgs aq, AccArgs at) {
+template <int KIND, int NCH, int ACC_WARPS, bool FULL>
+__global__ void __launch_bounds__(32 * ACC_WARPS, NCH == 1 ? 4 : 1) accum_tma_kernel(AccArgs aq, AccArgs at) {
     const int own_rows = blockIdx.z == 0 ? aq.own_rows : at.own_rows, split = blockIdx.z == 0 ? aq.split : at.split;
     if ((int)blockIdx.x * ACC_ROWS >= own_rows || (int)blockIdx.y >= split) return;
-    if (blockIdx.z == 0) accum_tma_body<KIND, NCH, true, ACC_WARPS>(aq, blockIdx.x, blockIdx.y);
-    else accum_tma_body<KIND, NCH, false, ACC_WARPS>(at, blockIdx.x, blockIdx.y);
+    if (blockIdx.z == 0) accum_tma_body<KIND, NCH, true, ACC_WARPS, FULL>(aq, blockIdx.x, blockIdx.y);
+    else accum_tma_body<KIND, NCH, false, ACC_WARPS, FULL>(at, blockIdx.x, blockIdx.y);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1106,11 +1091,13 @@ cudaError_t launch_block_tma(const TrainParams& p, cudaStream_t s) {
     const size_t smem = block_tma_smem(p.d);
     static DeviceOnce configured;
     const cudaError_t e = once_per_device(configured, [] {
-        return cudaFuncSetAttribute(block_tma_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)block_tma_smem(kMaxDim));
+        const cudaError_t e0 = cudaFuncSetAttribute(block_tma_kernel<KIND, FKC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)block_tma_smem(kMaxDim));
+        return e0 != cudaSuccess ? e0 : cudaFuncSetAttribute(block_tma_kernel<KIND, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)block_tma_smem(FKC));
     });
     if (e != cudaSuccess) return e;
     dim3 grid((p.N + TN - 1) / TN, (p.B + FTQ - 1) / FTQ);
-    return launch_dependent(block_tma_kernel<KIND>, grid, dim3(FTHREADS), smem, s, p);
+    if (p.d >= FKC) return launch_dependent(block_tma_kernel<KIND, FKC>, grid, dim3(FTHREADS), smem, s, p);
+    return launch_dependent(block_tma_kernel<KIND, 0>, grid, dim3(FTHREADS), smem, s, p);
 }
 
 template <int KIND, int NCH>
@@ -1119,12 +1106,15 @@ cudaError_t launch_accum_tma_inst(const AccArgs& aq, const AccArgs& at, cudaStre
     const size_t smem = accum_tma_smem(aq.d4);
     static DeviceOnce configured;
     const cudaError_t e = once_per_device(configured, [] {
-        return cudaFuncSetAttribute(accum_tma_kernel<KIND, NCH, WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)accum_tma_smem(kMaxDim / 4));
+        const cudaError_t e0 = cudaFuncSetAttribute(accum_tma_kernel<KIND, NCH, WARPS, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                    (int)accum_tma_smem(kMaxDim / 4));
+        return e0 != cudaSuccess ? e0 : cudaFuncSetAttribute(accum_tma_kernel<KIND, NCH, WARPS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                             (int)accum_tma_smem(kMaxDim / 4));
     });
     if (e != cudaSuccess) return e;
     dim3 grid((std::max(aq.own_rows, at.own_rows) + ACC_ROWS - 1) / ACC_ROWS, std::max(aq.split, at.split), 2);
-    return launch_dependent(accum_tma_kernel<KIND, NCH, WARPS>, grid, dim3(32 * WARPS), smem, s, aq, at);
+    if (aq.d4 == 32 * NCH) return launch_dependent(accum_tma_kernel<KIND, NCH, WARPS, true>, grid, dim3(32 * WARPS), smem, s, aq, at);
+    return launch_dependent(accum_tma_kernel<KIND, NCH, WARPS, false>, grid, dim3(32 * WARPS), smem, s, aq, at);
 }
 
 template <int KIND>
