@@ -301,6 +301,16 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     }
     return false;
 }
+// The same for a single thread that shares its scheduler with working warps (the copy-issuing and
+// MMA-issuing threads of the tensor-core kernel): it sleeps between tests from the first miss on,
+// so its polls do not take issue slots from the warps that do the arithmetic.
+__device__ __forceinline__ bool mbar_wait_idle(uint64_t* bar, uint32_t parity, int limit) {
+    for (int i = 0; i < limit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(96);
+    }
+    return false;
+}
 // dst (shared) and src (global) 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"

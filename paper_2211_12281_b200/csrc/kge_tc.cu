@@ -186,6 +186,26 @@ __device__ __forceinline__ float tc_score(const TcGemmParams& p, float acc, floa
 }
 
 
+// Per-row inputs of an epilogue, read before the accumulator is waited for.
+struct TcRowState {
+    float rn;                 // squared norm of the row (norm expansion)
+    float2 st;                // EPI_GRAD: the row's (base-2 maximum, 1 / normaliser)
+    float thr, ft;            // EPI_TOPK: current k-th best score, score of the true tail
+    int32_t thr_id, tt;       //           its id, the true tail's id
+};
+template <int EPI>
+__device__ __forceinline__ TcRowState tc_row_state(const TcGemmParams& p, int row) {
+    TcRowState r{0.f, make_float2(0.f, 0.f), INFINITY, 0.f, 0, -1};
+    if (row >= p.M) return r;   // rows outside the problem: no true tail, a threshold nothing exceeds
+    if ((EPI & EPI_L2) != 0) r.rn = p.row_norm2[row];
+    if ((EPI & 3) == EPI_GRAD) r.st = p.row_stat[row];
+    if ((EPI & 3) == EPI_TOPK) {
+        r.thr = p.thr[row]; r.thr_id = p.thr_id[row];
+        if (p.tt) { r.ft = p.ftrue[row]; r.tt = p.tt[row]; }
+    }
+    return r;
+}
+
 // One chunk of 32 scores of the first pass.  FULL: all 32 columns lie inside the problem (no
 // per-element masking); otherwise the first `valid` do.
 template <bool L2, bool CE, bool FULL>
@@ -220,8 +240,8 @@ __device__ __forceinline__ void tc_stats_chunk(const TcGemmParams& p, float (&v)
 // exponent is x = a f for the self-adversarial weights and x = f + c for the sampled softmax;
 // it is carried in base 2 (y = x log2 e), so an exponential is one ex2 of a difference.
 template <bool L2, bool CE>
-__device__ __forceinline__ void tc_epilogue_stats(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr) {
-    const float rn = (L2 && row < p.M) ? p.row_norm2[row] : 0.f;
+__device__ __forceinline__ void tc_epilogue_stats(const TcGemmParams& p, const TcItem& it, int row, const TcRowState& rs, int col_off, uint32_t taddr) {
+    const float rn = rs.rn;
     const float k1 = CE ? kLog2e : p.adv_temp * kLog2e, k0 = CE ? p.ce_c * kLog2e : 0.f;
     float m = -INFINITY, z = 0.f, l = 0.f;
     static_assert(TC_PIECE == 64, "two chunks of 32 columns per piece");
@@ -263,11 +283,11 @@ __device__ __forceinline__ float tc_grad_one(const TcGemmParams& p, float acc, f
 // chunk c ^ ((r >> 1) & 3) of the row: both the row-wise writes and the 8-row reads then touch
 // every bank once.
 template <bool L2, bool CE>
-__device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr,
+__device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const TcItem& it, int row, const TcRowState& rs, int col_off, uint32_t taddr,
                                                  uint4* stage) {
     const bool rin = row < p.M;
-    const float rn = (L2 && rin) ? p.row_norm2[row] : 0.f;
-    const float2 st = rin ? p.row_stat[row] : make_float2(0.f, 0.f);
+    const float rn = rs.rn;
+    const float2 st = rs.st;
     const float k1 = CE ? kLog2e : p.adv_temp * kLog2e, k0 = (CE ? p.ce_c * kLog2e : 0.f) - st.x;
     const float scale = p.loss_scale * st.y;
     const int lane = threadIdx.x & 31;
@@ -366,25 +386,18 @@ __device__ __forceinline__ float float_below(float x) {
 // id takes the element-by-element form, so the common case costs a compare-and-count per score
 // for the rank and one maximum per score for the candidate test.
 template <int WIDTH>
-__device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr, int32_t* beat_sm) {
+__device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const TcItem& it, int row, const TcRowState& rs, int col_off, uint32_t taddr, int32_t* beat_sm) {
     const bool rin = row < p.M;
-    // rows outside the problem stay in the loop (the warp votes below need every lane): no true
-    // tail, and a threshold nothing exceeds
-    float thr = INFINITY, ft = 0.f; int32_t thr_id = 0, tt = -1;
-    if (rin) {
-        thr = p.thr[row]; thr_id = p.thr_id[row];
-        if (p.tt) { ft = p.ftrue[row]; tt = p.tt[row]; }
-    }
+    // rows outside the problem stay in the loop (the warp votes below need every lane): their state
+    // holds no true tail and a threshold nothing exceeds
+    const float thr = rs.thr, ft = rs.ft; const int32_t thr_id = rs.thr_id, tt = rs.tt;
     const float thr_lo = float_below(thr), ft_lo = float_below(ft);
     const int lane = threadIdx.x & 31;
     int beat = 0;
-#pragma unroll 1
-    for (int c0 = col_off; c0 < col_off + WIDTH; c0 += 32) {
-        float v[32];
-        tmem_ld32(taddr + (uint32_t)(c0 - col_off), v);
+    auto chunk = [&](float (&v)[32], int c0) {
         const int ncol = it.n0 + c0;
         const int valid = min(32, p.N - ncol);          // the same for every lane
-        if (valid <= 0) continue;
+        if (valid <= 0) return;
         const int32_t e0 = (int32_t)(p.n_base + p.id_base + ncol);
         if (valid != 32) {
 #pragma unroll
@@ -445,6 +458,16 @@ __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const Tc
                 }
             }
         }
+    };
+    static_assert(WIDTH % 64 == 0, "two chunks of 32 columns are requested from tensor memory at a time");
+#pragma unroll 1
+    for (int c0 = col_off; c0 < col_off + WIDTH; c0 += 64) {
+        float v0[32], v1[32];
+        tmem_ld32_issue(taddr + (uint32_t)(c0 - col_off), v0);
+        tmem_ld32_issue(taddr + (uint32_t)(c0 - col_off) + 32u, v1);
+        tmem_ld_wait();
+        chunk(v0, c0);
+        chunk(v1, c0 + 32);
     }
     if (rin && beat > 0) {
         if (row < p.beat_rows) atomicAdd(&beat_sm[row], beat); else atomicAdd(&p.beat_tmp[row], beat);
@@ -454,19 +477,19 @@ __device__ __forceinline__ void tc_epilogue_topk(const TcGemmParams& p, const Tc
 // Epilogue of one warp on one item: WIDTH columns [col_off, col_off + WIDTH) of the tile row held by
 // this thread's tensor-memory lane (taddr points at the first of them).
 template <int EPI, int WIDTH>
-__device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem& it, int row, int col_off, uint32_t taddr, int32_t* beat_sm) {
+__device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem& it, int row, const TcRowState& rs, int col_off, uint32_t taddr, int32_t* beat_sm) {
     static_assert((EPI & 3) == EPI_STORE || (EPI & 3) == EPI_TOPK || WIDTH % TC_PIECE == 0, "the fused loss epilogues work on pieces of TC_PIECE columns");
     if ((EPI & 3) == EPI_STATS || (EPI & 3) == EPI_GRAD) {
 #pragma unroll 1
         for (int c = 0; c < WIDTH; c += TC_PIECE) {
-            if ((EPI & 3) == EPI_STATS) tc_epilogue_stats<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, col_off + c, taddr + (uint32_t)c);
-            else tc_epilogue_grad<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, col_off + c, taddr + (uint32_t)c, reinterpret_cast<uint4*>(beat_sm));
+            if ((EPI & 3) == EPI_STATS) tc_epilogue_stats<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, rs, col_off + c, taddr + (uint32_t)c);
+            else tc_epilogue_grad<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, rs, col_off + c, taddr + (uint32_t)c, reinterpret_cast<uint4*>(beat_sm));
         }
         return;
     }
-    if ((EPI & 3) == EPI_TOPK) { tc_epilogue_topk<WIDTH>(p, it, row, col_off, taddr, beat_sm); return; }
+    if ((EPI & 3) == EPI_TOPK) { tc_epilogue_topk<WIDTH>(p, it, row, rs, col_off, taddr, beat_sm); return; }
     float* const Cout = p.C + (int64_t)it.z * p.split_stride;
-    const float rn = ((EPI & EPI_L2) && row < p.M) ? p.row_norm2[row] : 0.f;
+    const float rn = rs.rn;
 #pragma unroll 1
     for (int c0 = col_off; c0 < col_off + WIDTH; c0 += 32) {
         float v[32];
@@ -495,6 +518,19 @@ __device__ __forceinline__ TcItem tc_item(const TcGemmParams& p, int64_t item) {
     if (p.m_fastest) return TcItem{0, (int)(item % p.tiles_m) * TC_BM, (int)(item / p.tiles_m) * p.bn};
     const int tn = (int)(item % p.tiles_n), r = (int)(item / p.tiles_n);
     return TcItem{r / p.tiles_m, (r % p.tiles_m) * TC_BM, tn * p.bn};
+}
+// The same walk one item at a time: the divisions are paid once per CTA, not once per item and warp.
+__device__ __forceinline__ void tc_item_next(const TcGemmParams& p, TcItem& it) {
+    if (p.m_fastest) {
+        it.m0 += TC_BM;
+        if (it.m0 >= p.tiles_m * TC_BM) { it.m0 = 0; it.n0 += p.bn; }
+    } else {
+        it.n0 += p.bn;
+        if (it.n0 >= p.tiles_n * p.bn) {
+            it.n0 = 0; it.m0 += TC_BM;
+            if (it.m0 >= p.tiles_m * TC_BM) { it.m0 = 0; ++it.z; }
+        }
+    }
 }
 
 // BN: columns per tile (128, or 256 for the backward contractions of wide rows); A_MN / B_MN:
@@ -551,12 +587,12 @@ __global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __gri
             int keep[TC_STAGES];
 #pragma unroll
             for (int s = 0; s < TC_STAGES; ++s) keep[s] = -1;
-            for (int item = item_begin; item < item_end && !*stop; ++item) {
-                const TcItem it = tc_item(p, item);
+            TcItem it = tc_item(p, item_begin);
+            for (int item = item_begin; item < item_end && !*stop; ++item, tc_item_next(p, it)) {
                 const int kb0 = it.z * p.kb_per_split, nkb = min(p.kb_per_split, kb_total - kb0);
                 for (int kb = 0; kb < nkb; ++kb, ++ring) {
                     const int s = ring % TC_STAGES;
-                    if (!mbar_wait_bounded(&empty[s], ((ring / TC_STAGES) & 1) ^ 1, p.wait_limit)) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); break; }
+                    if (!mbar_wait_idle(&empty[s], ((ring / TC_STAGES) & 1) ^ 1, p.wait_limit)) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); break; }
                     unsigned char* sa = base + (size_t)s * TC_STAGE_BYTES;
                     const int shared_at = p.m_fastest ? it.n0 : it.m0;
                     bool have = false;
@@ -590,17 +626,17 @@ __global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __gri
             constexpr uint32_t idesc = umma_idesc_bf16(TC_BM, BN, A_MN, B_MN);
             int ring = 0;
             bool ok = true;
-            for (int item = item_begin, local = 0; item < item_end && ok && !*stop; ++item, ++local) {
-                const TcItem it = tc_item(p, item);
+            TcItem it = tc_item(p, item_begin);
+            for (int item = item_begin, local = 0; item < item_end && ok && !*stop; ++item, ++local, tc_item_next(p, it)) {
                 const int nkb = min(p.kb_per_split, kb_total - it.z * p.kb_per_split);
                 const int buf = local % NACC;
                 // the epilogue warps must have drained this buffer (two items ago)
-                if (!mbar_wait_bounded(&acc_empty[buf], ((local / NACC) & 1) ^ 1, p.wait_limit)) { ok = false; break; }
+                if (!mbar_wait_idle(&acc_empty[buf], ((local / NACC) & 1) ^ 1, p.wait_limit)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_acc = tmem_base + (uint32_t)buf * BN;
                 for (int kb = 0; kb < nkb; ++kb, ++ring) {
                     const int s = ring % TC_STAGES;
-                    if (!mbar_wait_bounded(&full[s], (ring / TC_STAGES) & 1, p.wait_limit)) { ok = false; break; }
+                    if (!mbar_wait_idle(&full[s], (ring / TC_STAGES) & 1, p.wait_limit)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = smem_u32(base + (size_t)s * TC_STAGE_BYTES);
 #pragma unroll
@@ -618,16 +654,18 @@ __global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __gri
     } else {
         const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
         const int cgrp = (warp - 2) >> 2;              // which group of the tile's columns
-        for (int item = item_begin, local = 0; item < item_end; ++item, ++local) {
+        TcItem it = tc_item(p, item_begin);
+        for (int item = item_begin, local = 0; item < item_end; ++item, ++local, tc_item_next(p, it)) {
             const int buf = local % NACC;
+            // what the epilogue needs of its row does not depend on the accumulator: fetched before the wait
+            const TcRowState rs = tc_row_state<EPI>(p, it.m0 + quarter * 32 + lane);
             const bool ok = mbar_wait_bounded(&acc_full[buf], (local / NACC) & 1, p.wait_limit);
             tc_fence_after();
             if (!ok || *stop) { if (lane == 0) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); } break; }
-            const TcItem it = tc_item(p, item);
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cgrp * (BN / EG));
             // scratch after the barriers: the rank counts of EPI_TOPK, or 2 KB per epilogue warp for EPI_GRAD's stores
             int32_t* scratch = (EPI & 3) == EPI_GRAD ? beat_sm + (warp - 2) * (TC_GRAD_STAGE_BYTES / 4) : beat_sm;
-            tc_epilogue<EPI, BN / EG>(p, it, it.m0 + quarter * 32 + lane, cgrp * (BN / EG), taddr, scratch);
+            tc_epilogue<EPI, BN / EG>(p, it, it.m0 + quarter * 32 + lane, rs, cgrp * (BN / EG), taddr, scratch);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
