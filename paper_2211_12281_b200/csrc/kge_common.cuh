@@ -294,10 +294,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, ui
 }
 // Waits for the barrier phase `parity` at most `limit` times (each up to the hint above, then a
 // short sleep: seconds in all at the default limit); false = gave up.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, int limit) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, int limit, int spin = 16, unsigned sleep_ns = 256) {
     for (int i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (i > 16) __nanosleep(256);
+        if (i > spin) __nanosleep(sleep_ns);
     }
     return false;
 }

@@ -30,6 +30,7 @@ namespace {
 
 constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 64;      // BK bf16 = one 128-byte swizzle row
 constexpr int TC_STAGES = 4;
+constexpr int TC_RING_MAX = 8;                            // barriers are laid out for the deepest ring (resident column tile, below)
 constexpr int TC_EPI_WARPS = 8;                           // epilogue warps of the training kernels: TC_EPI_GROUPS per tensor-memory lane quarter
 constexpr int TC_EPI_WARPS_TOPK = 16;                     // the filter epilogue of full-entity scoring profits from more
 constexpr int TC_EPI_GROUPS = TC_EPI_WARPS / 4;
@@ -75,6 +76,7 @@ struct TcGemmParams {
     int cand_cap;
     int32_t* overflow;                    // set when a candidate list is full
     int beat_rows;                        // rows whose rank counts are gathered in shared memory first (0: global atomics)
+    int resident_b;                       // EPI_TOPK: the column tile has a buffer of its own and the ring holds row tiles only
 };
 
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
@@ -543,13 +545,21 @@ __global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __gri
     constexpr int NACC = 512 / BN;                      // fp32 accumulators in tensor memory, used in turn: all 512 columns
     constexpr uint32_t TC_TMEM_COLS = NACC * BN;
     constexpr int EW = tc_epi_warps(EPI), EG = EW / 4, TC_THREADS = tc_threads(EPI);
+    // For the epilogues that are bound by special-function instructions and row-dependent loads
+    // (the norm-expansion kinds) the epilogue warps form two groups that take the CTA's items in
+    // turn, so the epilogues of consecutive items overlap; measured faster there (log-sigmoid
+    // L2 passes 164 -> 156 us at B = N = 8192) and slower for the others, which stay one group.
+    constexpr int EGRP = ((EPI & EPI_L2) != 0 && (EPI & 3) != EPI_STORE && EG % 2 == 0) ? 2 : 1;
+    constexpr int GW = EW / EGRP, GCOLS = BN / (GW / 4);       // warps per group; columns per warp
     extern __shared__ unsigned char tc_smem_raw[];
     unsigned char* base = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
     uint64_t* full = reinterpret_cast<uint64_t*>(base + (size_t)TC_STAGES * TC_STAGE_BYTES);
-    uint64_t* empty = full + TC_STAGES;
-    uint64_t* acc_full = empty + TC_STAGES;      // [2] accumulator buffer written
+    uint64_t* empty = full + TC_RING_MAX;
+    uint64_t* acc_full = empty + TC_RING_MAX;    // [NACC] accumulator buffer written
     uint64_t* acc_empty = acc_full + NACC;       // [NACC] accumulator buffer drained by all epilogue warps
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + NACC);
+    uint64_t* b_full = acc_empty + NACC;         // resident column tile: loaded / no longer read by any MMA
+    uint64_t* b_free = b_full + 1;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b_free + 1);
     volatile uint32_t* stop = tmem_slot + 1;     // set by a warp whose wait ran out
     int32_t* beat_sm = reinterpret_cast<int32_t*>(base + (size_t)TC_STAGES * TC_STAGE_BYTES + 256);   // [beat_rows], EPI_TOPK
     if ((EPI & 3) == EPI_TOPK)
@@ -561,8 +571,9 @@ __global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __gri
     const int kb_total = (p.K + TC_BK - 1) / TC_BK;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int b = 0; b < NACC; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EW); }
+        for (int s = 0; s < TC_RING_MAX; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        mbar_init(b_full, 1); mbar_init(b_free, 1);
+        for (int b = 0; b < NACC; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], GW); }
         *stop = 0;
         mbar_init_fence();
     }
@@ -575,7 +586,76 @@ __global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __gri
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == 0) {
+    // Full-entity scoring with rows of at most 128 coordinates: the column (entity) tile of the
+    // current run of items sits in a buffer of its own (2 x 32 KB) and the rest of the stage memory
+    // is a ring of eight 16 KB row-tile slices, four items deep.  With the column tile kept inside
+    // the ring stages instead, only two items were in flight and the MMAs waited for copies.
+    const bool resident = (EPI & 3) == EPI_TOPK && BN == 256 && p.resident_b != 0;
+    constexpr uint32_t RES_B_BYTES = 2u * 256u * TC_BK * 2u;          // two slices of the column tile
+    constexpr int RES_RING = 8;
+    if (warp == 0 && resident) {
+        if (lane == 0) {
+            int ring = 0, btile = 0, cur_n0 = -1;
+            TcItem it = tc_item(p, item_begin);
+            for (int item = item_begin; item < item_end && !*stop; ++item, tc_item_next(p, it)) {
+                bool ok = true;
+                if (it.n0 != cur_n0) {      // a new column tile: every MMA on the previous one must be done
+                    cur_n0 = it.n0;
+                    ok = mbar_wait_idle(b_free, (btile & 1) ^ 1, p.wait_limit);
+                    if (ok) {
+                        mbar_arrive_expect_tx(b_full, (uint32_t)kb_total * (256u * TC_BK * 2u));
+                        for (int kb = 0; kb < kb_total; ++kb)
+#pragma unroll
+                            for (int g = 0; g < 2; ++g)
+                                tma_load_2d(base + (size_t)kb * (256 * TC_BK * 2) + g * (128 * TC_BK * 2), &tmB, kb * TC_BK,
+                                            (int)p.n_base + it.n0 + 128 * g, b_full);
+                        ++btile;
+                    }
+                }
+                for (int kb = 0; kb < kb_total && ok; ++kb, ++ring) {
+                    const int s = ring % RES_RING;
+                    ok = mbar_wait_idle(&empty[s], ((ring / RES_RING) & 1) ^ 1, p.wait_limit);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(&full[s], TC_A_BYTES);
+                    tma_load_2d(base + RES_B_BYTES + (size_t)s * TC_A_BYTES, &tmA, kb * TC_BK, it.m0, &full[s]);
+                }
+                if (!ok) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); break; }
+            }
+        }
+    } else if (warp == 1 && resident) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(TC_BM, BN, false, false);
+            int ring = 0, btile = 0, cur_n0 = -1;
+            bool ok = true;
+            TcItem it = tc_item(p, item_begin);
+            for (int item = item_begin, local = 0; item < item_end && ok && !*stop; ++item, ++local) {
+                const int buf = local % NACC;
+                if (it.n0 != cur_n0) {
+                    cur_n0 = it.n0;
+                    if (!mbar_wait_idle(b_full, btile & 1, p.wait_limit)) { ok = false; break; }
+                    ++btile;
+                }
+                if (!mbar_wait_idle(&acc_empty[buf], ((local / NACC) & 1) ^ 1, p.wait_limit)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tmem_acc = tmem_base + (uint32_t)buf * BN;
+                for (int kb = 0; kb < kb_total; ++kb, ++ring) {
+                    const int s = ring % RES_RING;
+                    if (!mbar_wait_idle(&full[s], (ring / RES_RING) & 1, p.wait_limit)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(base + RES_B_BYTES + (size_t)s * TC_A_BYTES);
+                    const uint32_t sb = smem_u32(base + (size_t)kb * (256 * TC_BK * 2));
+#pragma unroll
+                    for (int k = 0; k < TC_BK / 16; ++k)
+                        umma_bf16(tmem_acc, umma_desc_k_sw128(sa + k * 32), umma_desc_k_sw128(sb + k * 32), idesc, (kb | k) != 0);
+                    umma_commit(&empty[s]);
+                }
+                umma_commit(&acc_full[buf]);           // also after a failed wait, so the epilogue warps wake up
+                tc_item_next(p, it);
+                if (item + 1 >= item_end || it.n0 != cur_n0) umma_commit(b_free);   // the last MMAs that read this column tile
+            }
+            if (!ok) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); }
+        }
+    } else if (warp == 0) {
         if (lane == 0) {
             int ring = 0;    // slices issued so far: stage = ring % STAGES, phase = ring / STAGES
             // Without K splits and with a slice count that divides the ring, slice kb of every item
@@ -653,19 +733,24 @@ __global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __gri
         }
     } else {
         const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
-        const int cgrp = (warp - 2) >> 2;              // which group of the tile's columns
-        TcItem it = tc_item(p, item_begin);
-        for (int item = item_begin, local = 0; item < item_end; ++item, ++local, tc_item_next(p, it)) {
-            const int buf = local % NACC;
+        const int egrp = (warp - 2) / GW;              // which items
+        const int cgrp = ((warp - 2) % GW) >> 2;       // which group of the tile's columns
+        TcItem it = tc_item(p, min(item_begin + egrp, p.items - 1));
+        for (int item = item_begin + egrp, local = egrp; item < item_end; item += EGRP, local += EGRP) {
+            if (local != egrp) {
+#pragma unroll
+                for (int g = 0; g < EGRP; ++g) tc_item_next(p, it);
+            }
             // what the epilogue needs of its row does not depend on the accumulator: fetched before the wait
             const TcRowState rs = tc_row_state<EPI>(p, it.m0 + quarter * 32 + lane);
+            const int buf = local % NACC;
             const bool ok = mbar_wait_bounded(&acc_full[buf], (local / NACC) & 1, p.wait_limit);
             tc_fence_after();
             if (!ok || *stop) { if (lane == 0) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); } break; }
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cgrp * (BN / EG));
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cgrp * GCOLS);
             // scratch after the barriers: the rank counts of EPI_TOPK, or 2 KB per epilogue warp for EPI_GRAD's stores
             int32_t* scratch = (EPI & 3) == EPI_GRAD ? beat_sm + (warp - 2) * (TC_GRAD_STAGE_BYTES / 4) : beat_sm;
-            tc_epilogue<EPI, BN / EG>(p, it, it.m0 + quarter * 32 + lane, rs, cgrp * (BN / EG), taddr, scratch);
+            tc_epilogue<EPI, GCOLS>(p, it, it.m0 + quarter * 32 + lane, rs, cgrp * GCOLS, taddr, scratch);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
@@ -984,6 +1069,7 @@ int launch_tc_infer_chunk(kge_handle* h, int nq, int64_t e_lo, int64_t e_hi, con
     p.cand_cnt = w.cand_cnt; p.beat_tmp = w.beat_tmp; p.cand_score = w.cand_score; p.cand_id = w.cand_id;
     p.cand_cap = kCandCap; p.overflow = w.status + 1;
     p.beat_rows = std::min(nq, TC_BEAT_ROWS_MAX);   // the other rows count with global atomics
+    p.resident_b = p.kb_per_split <= 2 ? 1 : 0;     // the column tile's two slices fit beside an eight-stage ring of row-tile slices
     // (the table's tensor map covers all rows; the kernel offsets its row coordinate by n_base)
     KGE_CUDA_CHECK(h, (launch_gemm_inst<EPI_TOPK, 256>(h->tm_iq, h->tm_eb, p, h->num_sms, s, (size_t)p.beat_rows * 4)));
     KGE_LAUNCH_CHECK(h);

@@ -76,14 +76,18 @@ def test_five_query_tiles_with_a_ragged_last_one(oracle32, score, p, d):
     assert (sc == o_sc).all() or np.allclose(sc, o_sc, rtol=1e-6)
 
 
-@pytest.mark.parametrize("score", ["distmult", "complex"])
-def test_tensor_core_topk_against_bf16_operand_oracle(oracle64, score):
+@pytest.mark.parametrize("score,E,d", [("distmult", 5000, 64), ("complex", 5000, 64), ("distmult", 70000, 128),
+                                       ("complex", 40000, 256)])
+def test_tensor_core_topk_against_bf16_operand_oracle(oracle64, score, E, d):
     """Full-entity scoring on tensor cores (bf16 operands, fp32 accumulation) against the oracle
     with bf16-rounded operands.  The accumulation order differs, so the lists are compared as
     sets with a near-tie audit (2e-2 relative is the stated bound of this path; 1e-4 is used),
-    ranks within 2, MRR within 1e-3.  E = 5000 leaves ragged 128-wide tiles, nq = 200 two row tiles."""
+    ranks within 2, MRR within 1e-3.  E = 5000 leaves ragged 128-wide tiles, nq = 200 two row tiles.
+    d = 64 and 128 keep the entity tile in a buffer of its own (one and two slices); at E = 70,000 the
+    later chunks give every thread block runs of items that cross from one entity tile to the
+    next.  d = 256 takes the plain ring of whole stages."""
     import kge_synth
-    E, R, d, K, nq = 5000, 9, 64, 10, 200
+    R, K, nq = 9, 10, 200
     prob = Problem(E=E, R=R, T=100, d=d, score=score, p_norm=1, B=8, N=8, P=1, graph_seed=12, tc=True)
     qh, qr, tt = kge_synth.make_queries(E, R, nq, seed=12)
     tt[0] = qh[0]
