@@ -659,6 +659,118 @@ def bench_inference(ctx, name, w, cpu_seconds):
     return line
 
 
+def time_calls(torch, fn, warm, count):
+    """Mean milliseconds per call of fn(i) over `count` calls after `warm` untimed ones (CUDA events on the current stream)."""
+    for i in range(warm):
+        fn(i)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record()
+    for i in range(count):
+        fn(warm + i)
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / count
+
+
+def bench_next_rows(ctx):
+    """Short device-timed runs of what the library offers beyond the plain step and the plain full-entity pass: the L3
+    regulariser, the feature-projection encoder (Eq. 1), the power-rank ensemble (Eq. 2), full-entity scoring over three
+    row shards and the two-worker training protocol of Section 4 (both on this one GPU, the collectives as in-process
+    exchanges).  Reported beside the workloads, not part of `value`."""
+    import numpy as np
+    torch, K, dev = ctx.torch, ctx.K, ctx.dev
+    from paper_2211_12281_b200.sharded import BessRank, GpuShard, bess_train_step_program, run_lockstep, sharded_score_all_topk_sequential
+    out = {}
+    w = WORKLOADS["c2_transe_l1"]
+    E, R, d, B, N = w["E"], w["R"], w["d"], w["B"], w["N"]
+    ent, rel, _ = kge_synth.make_tables(E, R, d, "transe", seed=w["graph_seed"])
+    h, r, t = kge_synth.make_graph(E, R, w["T"], seed=w["graph_seed"], entity_zipf=w["entity_zipf"], relation_zipf=w["relation_zipf"])
+    loss = torch.zeros(1, dtype=torch.float32, device=dev)
+
+    def c2_handle(**extra):
+        ent_d, rel_d = torch.from_numpy(ent.copy()).to(dev), torch.from_numpy(rel.copy()).to(dev)
+        kge = K.Kge(K.KgeConfig.make(**dict(cfg_kwargs(w, seed=0), **extra)))
+        kge.bind(ent_d, rel_d, None, num_triples=w["T"])
+        kge.graph_load(h, r, t)
+        return kge
+
+    # ---- plain step, then the same with the regulariser, then with the encoder (768 bf16 features per entity)
+    kge = c2_handle()
+    out["c2_step_ms"] = time_calls(torch, lambda s: kge.train_step(s, w["lr"], loss_out=loss), 5, 50)
+    kge = c2_handle(reg_lambda=1e-3)
+    out["c2_step_with_l3_regulariser_ms"] = time_calls(torch, lambda s: kge.train_step(s, w["lr"], loss_out=loss), 5, 50)
+    assert kge.get_status() == 0
+    F = 768
+    kge = c2_handle(feat_dim=F)
+    gen = torch.Generator(device=dev); gen.manual_seed(5)
+    feat = (torch.randn((E, F), generator=gen, device=dev) / F ** 0.5).to(torch.bfloat16)
+    MH = torch.randn((d, F), generator=gen, device=dev) * 0.05
+    MT = torch.randn((d, F), generator=gen, device=dev) * 0.05
+    kge.bind_features(feat, MH, MT)
+    out["c2_step_with_encoder_ms"] = time_calls(torch, lambda s: kge.train_step(s, w["lr"], loss_out=loss), 5, 50)
+    out["encoder_feature_dim"] = F
+    assert kge.get_status() == 0
+    del kge, feat
+
+    # ---- ensemble: 85 models' top-100 lists of 15,000 queries -> top-10 (Eq. 2, p = -0.5)
+    M, nq, kl = 85, 15000, 100
+    lists = torch.randint(0, 1_000_000, (M, nq, kl), generator=gen, device=dev, dtype=torch.int32)
+    table = torch.from_numpy(K.ensemble_rank_scores(-0.5, kl)).to(dev)
+    e_ids = torch.empty((nq, 10), dtype=torch.int32, device=dev); e_sc = torch.empty((nq, 10), dtype=torch.float64, device=dev)
+    ms = time_calls(torch, lambda i: K.ensemble_topk(lists, table, 10, e_ids, e_sc), 2, 5)
+    out["ensemble"] = {"models": M, "queries": nq, "list_length": kl, "ms": ms, "queries_per_s": nq / (ms * 1e-3)}
+    del lists
+
+    # ---- full-entity scoring over three row shards, one after the other on this GPU, against one handle on the whole table
+    Es, nqs, k = 3_000_000, 2048, 10
+    ent_s = torch.randn((Es, d), generator=gen, device=dev) * d ** -0.5
+    rel_s = torch.randn((R, d), generator=gen, device=dev) * d ** -0.5
+    qh, qr, tt = (torch.from_numpy(x).to(dev) for x in kge_synth.make_queries(Es, R, nqs, seed=9))
+    icfg = dict(num_entities=Es, num_relations=R, dim=d, score="transe", p_norm=1, batch=4, num_neg=4)
+    whole = K.Kge(K.KgeConfig.make(**icfg)); whole.bind(ent_s, rel_s, None, max_queries=nqs, topk=k)
+    ids = torch.empty((nqs, k), dtype=torch.int32, device=dev); sc = torch.empty((nqs, k), dtype=torch.float32, device=dev)
+    ranks = torch.empty(nqs, dtype=torch.int32, device=dev)
+    ms_whole = time_calls(torch, lambda i: whole.score_all_topk(qh, qr, k, tt, ids, sc, ranks), 1, 2)
+    D = 3
+    S = (Es + D - 1) // D
+    shards = []
+    for j in range(D):
+        lo, hi = j * S, min(Es, (j + 1) * S)
+        sh = K.Kge(K.KgeConfig.make(**dict(icfg, num_entities=hi - lo))); sh.bind(ent_s[lo:hi], rel_s, None, max_queries=nqs, topk=k)
+        shards.append(GpuShard(sh, lo))
+    res = []
+    ms_sharded = time_calls(torch, lambda i: res.append(sharded_score_all_topk_sequential(shards, qh, qr, k, tt)), 1, 2)
+    same = bool((res[-1][0] == ids).all() and (res[-1][2] == ranks).all())
+    out["sharded_inference"] = {"entities": Es, "queries": nqs, "shards": D, "ms_whole_table": ms_whole, "ms_three_shards_in_turn": ms_sharded,
+                                "identical_to_whole_table": same}
+    del whole, shards, ent_s, res
+
+    # ---- two workers of the Section 4 training protocol in lockstep on this GPU: B = 512 positives per worker, N = 1024
+    D, Bw = 2, B // 2
+    S = (E + D - 1) // D
+    kw = dict(cfg_kwargs(w, seed=0), batch=Bw, num_parts=D)
+    workers = []
+    for i in range(D):
+        lo, hi = i * S, min(E, (i + 1) * S)
+        rows = hi - lo
+        ent_ext = torch.zeros((rows + Bw + N, d), dtype=torch.float32, device=dev)
+        ent_ext[:rows] = torch.from_numpy(ent[lo:hi]).to(dev)
+        rel_i = torch.from_numpy(rel.copy()).to(dev)
+        mine = (h // S) == i
+        sampler = K.Kge(K.KgeConfig.make(**dict(kw, head_part=i)))
+        sampler.bind(ent_ext, rel_i, None, num_triples=int(mine.sum()))
+        sampler.graph_load(np.ascontiguousarray(h[mine]), np.ascontiguousarray(r[mine]), np.ascontiguousarray(t[mine]))
+        compute = K.Kge(K.KgeConfig.make(**dict(kw, num_entities=rows + Bw + N, num_parts=1)))
+        compute.bind(ent_ext, rel_i, None)
+        workers.append(BessRank(i, D, sampler, compute, ent_ext, rows, S))
+    ms = time_calls(torch, lambda s: run_lockstep([bess_train_step_program(wk, s, w["lr"]) for wk in workers]), 3, 20)
+    assert all(wk.compute.get_status() == 0 and wk.sampler.get_status() == 0 for wk in workers)
+    out["two_worker_training_step"] = {"workers": D, "positives_per_worker": Bw, "negatives": N, "ms_per_global_step": ms,
+                                       "note": "both workers on this GPU, one after the other; exchanges are in-process"}
+    return out
+
+
 def run_ours(args, names):
     ctx = Ctx(args)
     if ctx.world > 1:
@@ -682,6 +794,9 @@ def run_ours(args, names):
     line["alu_rates_unit"] = "T lane-instructions/s, measured by kge_measure_alu at the start of this run"
     if len(names) > 1:
         line["per_workload"] = {n: lines[n] for n in names[1:]}
+    if args.next_rows or (args.workload == "suite" and ctx.world == 1):
+        ctx.release()
+        line["next_rows"] = bench_next_rows(ctx)
     if ctx.rank == 0:
         print(json.dumps(line), flush=True)
     if ctx.world > 1:
@@ -698,6 +813,8 @@ def main():
                     help="'suite' (default: every workload, headline first), or one or more names separated by commas: "
                          + ", ".join(sorted(WORKLOADS) + sorted(INFER_WORKLOADS)))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--next-rows", action="store_true",
+                    help="also time the regulariser, the encoder, the ensemble, sharded inference and the two-worker step (part of the suite)")
     args = ap.parse_args()
     names = list(SUITE) if args.workload == "suite" else args.workload.split(",")
     for n in names:
