@@ -39,7 +39,11 @@ extern "C" {
 typedef struct kge_handle kge_handle; /* host-side object */
 
 /* Scoring functions: the table "Scoring functions" (Section 3.1). */
-typedef enum { KGE_TRANSE = 0, KGE_TRANSH = 1, KGE_ROTATE = 2, KGE_DISTMULT = 3, KGE_COMPLEX = 4 } kge_score_t;
+typedef enum { KGE_TRANSE = 0, KGE_TRANSH = 1, KGE_ROTATE = 2, KGE_DISTMULT = 3, KGE_COMPLEX = 4,
+               KGE_ROTATE_REAL_L1 = 5   /* RotatE with p = 1 read literally: the sum of |x_k| over the d real coordinates of
+                                           h o r - t (the scoring-function table identifies C^(d/2) with R^d), not the sum of
+                                           complex moduli that KGE_ROTATE takes; with p = 2 the two are the same */
+} kge_score_t;
 /* Loss functions: Section 3.1 "Loss Functions". */
 typedef enum { KGE_LOSS_LOGSIGMOID = 0, KGE_LOSS_SAMPLED_SOFTMAX = 1 } kge_loss_t;
 /* The paper names no optimiser; these are the textbook rules applied to touched rows only. */

@@ -42,7 +42,7 @@ def make_tables(num_entities: int, num_relations: int, dim: int, score: str, *, 
     rng = np.random.default_rng(seed + 1_000_003)
     std = 1.0 / np.sqrt(dim)
     ent = (rng.standard_normal((num_entities, dim)) * std).astype(np.float32)
-    if score == "rotate":
+    if score in ("rotate", "rotate_real_l1"):
         rel = rng.uniform(-np.pi, np.pi, size=(num_relations, dim // 2)).astype(np.float32)
     else:
         rel = (rng.standard_normal((num_relations, dim)) * std).astype(np.float32)

@@ -90,7 +90,9 @@ typedef double real;
 #define R_COS cos
 #endif
 
-enum { SC_TRANSE = 0, SC_TRANSH = 1, SC_ROTATE = 2, SC_DISTMULT = 3, SC_COMPLEX = 4 };
+enum { SC_TRANSE = 0, SC_TRANSH = 1, SC_ROTATE = 2, SC_DISTMULT = 3, SC_COMPLEX = 4,
+       SC_ROTATE_REAL = 5 };   /* RotatE with the norm taken literally over the d real coordinates (see distance_norm) */
+static int is_rotate(int32_t score) { return score == SC_ROTATE || score == SC_ROTATE_REAL; }
 enum { LOSS_LOGSIGMOID = 0, LOSS_SAMPLED_SOFTMAX = 1 };
 enum { OPT_SGD = 0, OPT_ADAM = 1, OPT_ROWWISE_ADAGRAD = 2 };
 enum { ERR_OK = 0, ERR_BAD_ARG = -1, ERR_DIVISIBILITY = -2, ERR_EMPTY_BUCKET = -3 };
@@ -317,7 +319,7 @@ int kgeo_sample_batch(const kgeo_config *c, uint64_t step,
 /* the raw rows.  Complex rows are interleaved (re0, im0, re1, im1, ...).      */
 /* RotatE's L1 is the sum of complex moduli (the cited RotatE definition).     */
 /* ------------------------------------------------------------------------- */
-static int rel_width(int32_t score, int32_t d) { return score == SC_ROTATE ? d / 2 : d; }
+static int rel_width(int32_t score, int32_t d) { return is_rotate(score) ? d / 2 : d; }
 
 static real bf16_round(real v) { /* round-to-nearest-even to 8 significand bits */
     float f = (float)v;
@@ -402,7 +404,7 @@ static void dot_query(int32_t score, int32_t d, const real *h, const real *r, re
 void kgeo_query_vector(int32_t score, int32_t d, const real *h, const real *r, const real *w, real *q) {
     if (score == SC_DISTMULT || score == SC_COMPLEX) { dot_query(score, d, h, r, q); return; }
     if (score == SC_TRANSE) { for (int k = 0; k < d; ++k) q[k] = h[k] + r[k]; return; }
-    if (score == SC_ROTATE) {
+    if (is_rotate(score)) {
         for (int k = 0; k < d / 2; ++k) {
             real cs = R_COS(r[k]), sn = R_SIN(r[k]);
             q[2 * k] = R_FMA(h[2 * k], cs, -(h[2 * k + 1] * sn));
@@ -508,7 +510,7 @@ static void score_grad_one(int32_t score, int32_t p, int32_t d, real g,
             if (dr) dr[k] += g * s[k];
             if (dt) dt[k] -= g * s[k];
         }
-    } else if (score == SC_ROTATE) { /* x = h e^{i theta} - t */
+    } else if (is_rotate(score)) { /* x = h e^{i theta} - t */
         for (int k = 0; k < d / 2; ++k) {
             real cs = R_COS(r[k]), sn = R_SIN(r[k]);
             real sre = s[2 * k], sim = s[2 * k + 1];

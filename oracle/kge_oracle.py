@@ -22,10 +22,11 @@ import numpy as np
 _HERE = Path(__file__).resolve().parent
 _SRC = _HERE / "kge_oracle.c"
 
-TRANSE, TRANSH, ROTATE, DISTMULT, COMPLEX = range(5)
+TRANSE, TRANSH, ROTATE, DISTMULT, COMPLEX, ROTATE_REAL_L1 = range(6)
 LOSS_LOGSIGMOID, LOSS_SAMPLED_SOFTMAX = range(2)
 OPT_SGD, OPT_ADAM, OPT_ROWWISE_ADAGRAD = range(3)
-SCORE_NAMES = {"transe": TRANSE, "transh": TRANSH, "rotate": ROTATE, "distmult": DISTMULT, "complex": COMPLEX}
+SCORE_NAMES = {"transe": TRANSE, "transh": TRANSH, "rotate": ROTATE, "distmult": DISTMULT, "complex": COMPLEX,
+               "rotate_real_l1": ROTATE_REAL_L1}   # RotatE with the norm over the d real coordinates
 LOSS_NAMES = {"logsigmoid": LOSS_LOGSIGMOID, "softmax": LOSS_SAMPLED_SOFTMAX}
 OPT_NAMES = {"sgd": OPT_SGD, "adam": OPT_ADAM, "adagrad": OPT_ROWWISE_ADAGRAD}
 
@@ -242,7 +243,7 @@ class Oracle:
         heads, rels, tails, negs = map(self._i32, (heads, rels, tails, negs))
         R = self.creal
         B, N, d = cfg.batch, cfg.num_neg, cfg.dim
-        kw = d // 2 if cfg.score == ROTATE else d
+        kw = d // 2 if cfg.score in (ROTATE, ROTATE_REAL_L1) else d
         dh, dtpos, dtneg = np.empty((B, d), self.real), np.empty((B, d), self.real), np.empty((N, d), self.real)
         dr = np.empty((B, kw), self.real)
         dw = None if relw is None else np.empty((B, d), self.real)
@@ -292,7 +293,7 @@ class Oracle:
         heads, rels, tails, negs = map(self._i32, (heads, rels, tails, negs))
         R = self.creal
         B, N, d, F = cfg.batch, cfg.num_neg, cfg.dim, feat.shape[1]
-        kw = d // 2 if cfg.score == ROTATE else d
+        kw = d // 2 if cfg.score in (ROTATE, ROTATE_REAL_L1) else d
         dh, dtpos, dtneg = np.empty((B, d), self.real), np.empty((B, d), self.real), np.empty((N, d), self.real)
         dr = np.empty((B, kw), self.real)
         dw = None if relw is None else np.empty((B, d), self.real)

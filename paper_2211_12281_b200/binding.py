@@ -12,11 +12,12 @@ from pathlib import Path
 
 _PKG = Path(__file__).resolve().parent
 
-TRANSE, TRANSH, ROTATE, DISTMULT, COMPLEX = range(5)
+TRANSE, TRANSH, ROTATE, DISTMULT, COMPLEX, ROTATE_REAL_L1 = range(6)
 LOSS_LOGSIGMOID, LOSS_SAMPLED_SOFTMAX = range(2)
 OPT_SGD, OPT_ADAM, OPT_ROWWISE_ADAGRAD = range(3)
 PREC_FP32, PREC_BF16_TC = range(2)
-SCORE_NAMES = {"transe": TRANSE, "transh": TRANSH, "rotate": ROTATE, "distmult": DISTMULT, "complex": COMPLEX}
+SCORE_NAMES = {"transe": TRANSE, "transh": TRANSH, "rotate": ROTATE, "distmult": DISTMULT, "complex": COMPLEX,
+               "rotate_real_l1": ROTATE_REAL_L1}
 LOSS_NAMES = {"logsigmoid": LOSS_LOGSIGMOID, "softmax": LOSS_SAMPLED_SOFTMAX}
 OPT_NAMES = {"sgd": OPT_SGD, "adam": OPT_ADAM, "adagrad": OPT_ROWWISE_ADAGRAD}
 

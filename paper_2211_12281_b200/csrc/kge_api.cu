@@ -210,7 +210,7 @@ int kge_create(const kge_config* cfg, kge_handle** out) {
     if (c.num_entities <= 0 || c.num_entities > INT32_MAX || c.num_relations <= 0 || c.num_relations > INT32_MAX)
         return KGE_ERR_BAD_ARG;
     if (c.dim <= 0 || c.dim % 4 != 0 || c.dim > kMaxDim) return KGE_ERR_BAD_ARG;
-    if (c.score < KGE_TRANSE || c.score > KGE_COMPLEX) return KGE_ERR_BAD_ARG;
+    if (c.score < KGE_TRANSE || c.score > KGE_ROTATE_REAL_L1) return KGE_ERR_BAD_ARG;
     if (c.p_norm != 1 && c.p_norm != 2) return KGE_ERR_BAD_ARG;
     if (c.loss != KGE_LOSS_LOGSIGMOID && c.loss != KGE_LOSS_SAMPLED_SOFTMAX) return KGE_ERR_BAD_ARG;
     if (c.opt < KGE_OPT_SGD || c.opt > KGE_OPT_ROWWISE_ADAGRAD) return KGE_ERR_BAD_ARG;
@@ -238,8 +238,10 @@ int kge_create(const kge_config* cfg, kge_handle** out) {
     kge_handle* h = new (std::nothrow) kge_handle();
     if (!h) return KGE_ERR_BAD_ARG;
     h->cfg = c;
-    h->kw = c.score == KGE_ROTATE ? c.dim / 2 : c.dim;
     h->kind = kind_of(c);
+    // RotatE with the real L1 norm differs from RotatE in the pair arithmetic (`kind`) only: from here on it is RotatE
+    if (c.score == KGE_ROTATE_REAL_L1) h->cfg.score = KGE_ROTATE;
+    h->kw = h->cfg.score == KGE_ROTATE ? c.dim / 2 : c.dim;
     h->bound = h->graph_loaded = false;
     h->streams_ready = false;
     h->launches = 0;

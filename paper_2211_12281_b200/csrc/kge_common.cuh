@@ -29,6 +29,7 @@ inline Kind kind_of(const kge_config& c) {
     switch (c.score) {
         case KGE_TRANSE: return c.p_norm == 1 ? KIND_L1 : KIND_L2;
         case KGE_ROTATE: return c.p_norm == 1 ? KIND_CL1 : KIND_L2;
+        case KGE_ROTATE_REAL_L1: return c.p_norm == 1 ? KIND_L1 : KIND_L2;   // the same query vector and chain rule, the real norm
         case KGE_TRANSH: return c.p_norm == 1 ? KIND_TH_L1 : KIND_TH_L2;
         default: return KIND_DOT;
     }

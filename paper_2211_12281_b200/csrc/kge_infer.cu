@@ -748,7 +748,7 @@ extern "C" int kge_score_all_topk_static(const kge_config* cfg, const float* ent
     if (out_ranks && !true_tails) return KGE_ERR_BAD_ARG;
     const kge_config& c = *cfg;
     if (c.num_entities <= 0 || c.num_entities > INT32_MAX || c.num_relations <= 0 || c.num_relations > INT32_MAX ||
-        c.dim <= 0 || c.dim % 4 != 0 || c.score < KGE_TRANSE || c.score > KGE_COMPLEX ||
+        c.dim <= 0 || c.dim % 4 != 0 || c.score < KGE_TRANSE || c.score > KGE_ROTATE_REAL_L1 ||
         (c.p_norm != 1 && c.p_norm != 2) || (c.score == KGE_TRANSH && !relw))
         return KGE_ERR_BAD_ARG;
     // the fixed scratch bounds the problem: refuse anything it cannot hold
@@ -757,8 +757,9 @@ extern "C" int kge_score_all_topk_static(const kge_config* cfg, const float* ent
 
     kge_handle h{};                     // plain host object on the stack, every field zero; nothing in it is heap-backed
     h.cfg = c;
-    h.kw = c.score == KGE_ROTATE ? c.dim / 2 : c.dim;
     h.kind = kind_of(c);
+    if (c.score == KGE_ROTATE_REAL_L1) h.cfg.score = KGE_ROTATE;      // the same query vector, the real norm (see kge_create)
+    h.kw = h.cfg.score == KGE_ROTATE ? c.dim / 2 : c.dim;
     h.ent = const_cast<float*>(ent); h.rel = const_cast<float*>(rel); h.relw = const_cast<float*>(relw);
     h.ent_state = h.rel_state = h.relw_state = nullptr;
     h.launches = 0; h.bound = true; h.graph_loaded = false;

@@ -41,7 +41,7 @@ class Problem:
 
     @property
     def rel_width(self):
-        return self.d // 2 if self.score == "rotate" else self.d
+        return self.d // 2 if self.score in ("rotate", "rotate_real_l1") else self.d
 
     def oracle_cfg(self):
         kw = {k: v for k, v in self.kw.items() if k not in ("feat_dim", "feat_shared")}     # (the oracle's encoder takes them as arguments)

@@ -21,7 +21,7 @@ def _infer(gpu, qh, qr, tt, K):
 
 
 @pytest.mark.parametrize("score,p", [("transe", 1), ("transe", 2), ("distmult", 1), ("complex", 1),
-                                     ("transh", 1), ("transh", 2), ("rotate", 2), ("rotate", 1)])
+                                     ("transh", 1), ("transh", 2), ("rotate", 2), ("rotate", 1), ("rotate_real_l1", 1)])
 def test_topk_rank_mrr_against_fp32_oracle(oracle32, oracle64, score, p):
     import kge_synth
     E, R, d, K, nq = 5000, 9, 40, 10, 70          # chunks 1024, 1024, 2048, 904; ragged tiles
@@ -33,7 +33,7 @@ def test_topk_rank_mrr_against_fp32_oracle(oracle32, oracle64, score, p):
     ids, sc, ranks = _infer(gpu, qh, qr, tt, K)
     cfg = prob.oracle_cfg()
     o_ids, o_sc, o_ranks = oracle32.score_all_topk(cfg, prob.ent, prob.rel, prob.relw, qh, qr, K, true_tails=tt)
-    if score == "rotate":
+    if score in ("rotate", "rotate_real_l1"):
         # sin / cos come from different math libraries: compare as sets, audit near-ties
         r_ids, r_sc, r_ranks = oracle64.score_all_topk(cfg, prob.ent, prob.rel, prob.relw, qh, qr, K + 5, true_tails=tt)
         for q in range(nq):
@@ -55,7 +55,7 @@ def test_topk_rank_mrr_against_fp32_oracle(oracle32, oracle64, score, p):
     # the same metric from ranks the caller already holds (no second pass over the table)
     ranks_dev = gpu.dev_i32(ranks)
     assert gpu.kge.mrr_from_ranks(ranks_dev, 10) == mrr and gpu.kge.mrr_from_ranks(ranks_dev, 0) == mrr0
-    if score != "rotate":
+    if score not in ("rotate", "rotate_real_l1"):
         assert abs(mrr - oracle64.mrr(o_ranks, 10)) <= 1e-12 and abs(mrr0 - oracle64.mrr(o_ranks, 0)) <= 1e-12
 
 

@@ -11,7 +11,7 @@ from parity_util import GpuSide, OracleSide, Problem, assert_close
 pytestmark = pytest.mark.gpu
 
 MODELS = [("transe", 1), ("transe", 2), ("transh", 1), ("transh", 2), ("rotate", 1), ("rotate", 2),
-          ("distmult", 1), ("complex", 1)]
+          ("distmult", 1), ("complex", 1), ("rotate_real_l1", 1)]
 
 
 def _check_step(gpu, orc, step, batch, *, taps=True, rows_atol=2e-6, warm_adam=False):
@@ -56,7 +56,7 @@ def _check_step(gpu, orc, step, batch, *, taps=True, rows_atol=2e-6, warm_adam=F
         assert_close(kge.debug_export("FPOS"), fwd["fpos"], atol=2e-6, what="positive scores")
         assert_close(scores_dev.cpu().numpy(), fwd["F"], atol=2e-6, what="score block F")
         assert_close(kge.debug_export("LROW"), fwd["Lrow"], atol=1e-5, what="per-positive loss")
-        l2 = prob.kw["p_norm"] == 2 and prob.score in ("transe", "transh", "rotate")
+        l2 = prob.kw["p_norm"] == 2 and prob.score in ("transe", "transh", "rotate", "rotate_real_l1")
         G = kge.debug_export("G").reshape(B, N)
         if l2:   # the tap holds dL/dF divided by the distance; undo with the oracle's distances
             F = orc.o.batch_loss(orc.cfg, *orc._pre, *batch)["F"]
@@ -139,7 +139,7 @@ def _run(oracle64, prob, steps=2, taps=True, external_batch=None):
 def test_step_taps_and_tables_all_models(oracle64, score, p, loss):
     # B = 72 and N = 70 leave ragged 64-wide tiles; d = 40 leaves a ragged 32-wide slice
     prob = Problem(E=500, R=7, T=20000, d=40, score=score, p_norm=p, loss=loss, B=72, N=70, P=2,
-                   gamma=6.0 if loss == "logsigmoid" and score in ("transe", "transh", "rotate") else 0.0,
+                   gamma=6.0 if loss == "logsigmoid" and score in ("transe", "transh", "rotate", "rotate_real_l1") else 0.0,
                    adv_temp=1.0 if loss == "logsigmoid" else 0.0, ce_correction=0.5, loss_scale=0.25,
                    lr=0.05, graph_seed=3, relation_zipf=1.0)
     _run(oracle64, prob)

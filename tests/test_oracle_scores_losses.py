@@ -9,12 +9,13 @@ import pytest
 from oracle.kge_oracle import make_config
 
 MODELS = [("transe", 1), ("transe", 2), ("transh", 1), ("transh", 2), ("rotate", 1), ("rotate", 2),
-          ("distmult", 1), ("complex", 1)]
+          ("distmult", 1), ("complex", 1), ("rotate_real_l1", 1)]
+ROTATE = ("rotate", "rotate_real_l1")
 
 
 def _rows(rng, d, score):
     h, t = rng.standard_normal(d), rng.standard_normal(d)
-    r = rng.uniform(-np.pi, np.pi, d // 2) if score == "rotate" else rng.standard_normal(d)
+    r = rng.uniform(-np.pi, np.pi, d // 2) if score in ROTATE else rng.standard_normal(d)
     w = rng.standard_normal(d) if score == "transh" else None
     return h, r, w, t
 
@@ -66,8 +67,15 @@ def test_rotate_special_phases_and_numpy_complex(oracle64):
     assert oracle64.score("rotate", 1, h, np.full(d // 2, np.pi), t) == pytest.approx(-np.abs(-hc - tc).sum(), rel=1e-12)
     th = rng.uniform(-np.pi, np.pi, d // 2)
     assert oracle64.score("rotate", 1, h, th, t) == pytest.approx(-np.abs(hc * np.exp(1j * th) - tc).sum(), rel=1e-12)
-    # L1 over moduli differs from the literal real L1 (|Re| + |Im|)
+    # L1 over moduli differs from the literal real L1 (|Re| + |Im|), which is the other score id
     assert oracle64.score("rotate", 1, h, zero, t) != pytest.approx(-np.abs(h - t).sum())
+    assert oracle64.score("rotate_real_l1", 1, h, zero, t) == pytest.approx(-np.abs(h - t).sum(), rel=1e-13)
+    q = hc * np.exp(1j * th) - tc
+    assert oracle64.score("rotate_real_l1", 1, h, th, t) == pytest.approx(-(np.abs(q.real) + np.abs(q.imag)).sum(), rel=1e-12)
+    # with p = 2 the real norm is the complex one: the two ids agree
+    assert oracle64.score("rotate_real_l1", 2, h, th, t) == oracle64.score("rotate", 2, h, th, t)
+    # |Re| + |Im| >= modulus, component by component
+    assert oracle64.score("rotate_real_l1", 1, h, th, t) <= oracle64.score("rotate", 1, h, th, t)
 
 
 def test_transh_special_cases(oracle64):
@@ -294,7 +302,7 @@ def test_logsigmoid_closed_forms(oracle64):
 # ----------------------------------------------------------------------------- gradients
 def _tiny_problem(rng, score, E=7, R=3, d=4, B=3, N=5):
     ent = rng.standard_normal((E, d)) * 0.7
-    rel = rng.uniform(-np.pi, np.pi, (R, d // 2)) if score == "rotate" else rng.standard_normal((R, d)) * 0.7
+    rel = rng.uniform(-np.pi, np.pi, (R, d // 2)) if score in ROTATE else rng.standard_normal((R, d)) * 0.7
     relw = rng.standard_normal((R, d)) if score == "transh" else None
     # repeated rows on purpose: entity 2 is a head, a tail and a negative; relation 1 twice
     heads = np.array([2, 0, 5], np.int32); rels = np.array([1, 1, 0], np.int32)
