@@ -217,9 +217,9 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback"}
 
 
-def ncu_traffic(workload, kernel):
-    """dram__bytes_read.sum + dram__bytes_write.sum per launch of `kernel` from the tracked capture record, or None when
-    there is no record for this workload and kernel or the kernel's source file has changed since the capture."""
+def ncu_record(workload, kernel):
+    """The tracked ncu capture record of this workload's `kernel`, or None when there is none or the kernel's source file
+    has changed since the capture."""
     rec_path = ROOT / "profiles" / "ncu_traffic.json"
     if not rec_path.exists():
         return None
@@ -227,8 +227,20 @@ def ncu_traffic(workload, kernel):
         if rec.get("workload") == workload and rec.get("stage") == kernel:
             src = ROOT / rec["source"]
             if src.exists() and hashlib.sha256(src.read_bytes()).hexdigest() == rec.get("source_sha256"):
-                return rec.get("dram_bytes_per_launch")
+                return rec
     return None
+
+
+def ncu_traffic(workload, kernel):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of `kernel` from the tracked capture record, or None."""
+    rec = ncu_record(workload, kernel)
+    return None if rec is None else rec.get("dram_bytes_per_launch")
+
+
+def ncu_tensor_active(workload, kernel):
+    """sm__pipe_tensor_cycles_active (% of peak) of a tensor-core pass from the tracked capture record, or None."""
+    rec = ncu_record(workload, kernel)
+    return None if rec is None else rec.get("tensor_pipe_active_pct")
 
 
 def stage_roof_us(ops, elements, alu):
@@ -554,6 +566,8 @@ def bench_training(ctx, name, w, cpu_seconds):
             src = ctx.peaks["source"] + " (sustained cuBLAS bf16)"
         roofline = {"bound": bound, "kernel": dominant, "achieved": achieved, "peak": peak, "unit": unit,
                     "frac": t_roof / us, "traffic": ncu_traffic(name, dominant), "peak_source": src, "us_per_launch": us}
+        if w.get("tc"):      # tensor pipe activity of the four passes under ncu (tracked capture of the same kernels)
+            roofline["tensor_pipe_active_ncu_pct"] = {st: ncu_tensor_active(name, st) for st in ("block", "loss", "accum_q", "accum_t")}
         roofline.update({k: v for k, v in detail.items() if k != "mix"})
     stage_frac = {s: roofs[s][0] / per_stage_us[s] for s in roofs}
     step_roof_us = sum(roofs[s][0] for s in roofs)
@@ -643,6 +657,8 @@ def bench_inference(ctx, name, w, cpu_seconds):
                 "unit": "T lane-instructions/s",
                 "peak_source": "measured in this run: kge_measure_alu on the kernel's instruction mix (" + MIX_NAMES[mix] + ")"}
     roof.update(frac=max(t_c, t_hbm) / (ms * 1e-3), traffic=ncu_traffic(name, roof["kernel"]), t_compute_ms=t_c * 1e3, t_hbm_ms=t_hbm * 1e3)
+    if w.get("tc"):
+        roof["tensor_pipe_active_ncu_pct"] = ncu_tensor_active(name, roof["kernel"])
     e2e_value = pairs / ((e2e_ms if e2e_ms is not None else ms) * 1e-3)
     line = {"metric": INFER_METRIC, "value": pairs / (ms * 1e-3), "unit": INFER_UNIT,
             "n_gpus": 1, "steps": steps, "warmup": 1, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
