@@ -261,9 +261,46 @@ __device__ __forceinline__ void ordered_sum(const V* rows, int wv, int count, In
 // One warp per sorted position.  A warp whose position opens a segment of at most PIECE rows
 // sums it and updates the row.  In a longer segment every PIECE-th position sums its piece
 // into the partial buffer (row index = the piece's first sorted position).
+//
+// Most segments are short, and for those everything follows from the sorted ids around r alone:
+// lane l reads sorted[r - PIECE + l].  Position r opens a segment if sorted[r - 1] differs; the run
+// of equal ids from r on is its length if it ends within PIECE positions; a position inside a
+// segment and less than PIECE from its start never starts a piece.  So the common case needs the
+// ids and the permutation in one round trip to memory and the gradient rows in the next (the table
+// row is pulled into L2 meanwhile), instead of a chain through the segment tables; only positions
+// in segments longer than PIECE take the general path.
 template <typename V, int NCH>
 __device__ __forceinline__ void piece_sum(const UpdateJob& J, const UpdateParams& p, int r, int lane) {
     const int wv = J.width / VecOps<V>::LEN;
+    {
+        const int pos = r - PIECE + lane;
+        const int32_t sv = pos < 0 ? -1 : (pos < J.n ? J.sorted[pos] : -2);
+        const int32_t after = r + PIECE < J.n ? J.sorted[r + PIECE] : -2;
+        const int32_t src = (lane < PIECE && r + lane < J.n) ? J.perm[r + lane] : 0;
+        const int32_t id = __shfl_sync(0xffffffffu, sv, PIECE);
+        const bool head = __shfl_sync(0xffffffffu, sv, PIECE - 1) != id;
+        const bool far = __shfl_sync(0xffffffffu, sv, 0) == id;          // PIECE or more positions into a segment
+        const unsigned same = __ballot_sync(0xffffffffu, sv == id) >> PIECE;
+        const int run = __ffs(~same) - 1;                                // ids equal to mine from r on, at most PIECE
+        if (!head && !far) return;
+        if (head && (run < PIECE || after != id)) {
+            const int64_t row = id;
+            const int row_lines = (J.width * 4 + 127) / 128;
+            const char* base = reinterpret_cast<const char*>(J.table + row * J.width);
+            if (lane < row_lines) asm volatile("prefetch.global.L2 [%0];" ::"l"(base + lane * 128));
+            if (p.opt == KGE_OPT_ADAM) {
+                const char* sb = reinterpret_cast<const char*>(J.state + row * 2 * J.width);
+                for (int ln = lane; ln < 2 * row_lines; ln += 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(sb + ln * 128));
+            }
+            V g[NCH];
+#pragma unroll
+            for (int i = 0; i < NCH; ++i) g[i] = VecOps<V>::zero();
+            ordered_sum<V, NCH>(reinterpret_cast<const V*>(J.grads), wv, run,
+                                [&](int s) { return (int64_t)__shfl_sync(0xffffffffu, src, s); }, g, lane);
+            apply_row<V, NCH>(J, p, row, g, lane);
+            return;
+        }
+    }
     const int u = J.seg_of[r];
     const int s0 = J.seg[u], s1 = J.seg[u + 1];
     const int len = s1 - s0;
