@@ -116,7 +116,7 @@ class Oracle:
 
     # -- helpers ------------------------------------------------------------
     def arr(self, a):
-        """Contiguous array in this build's real type (tables enter as fp32 values)."""
+        """Contiguous array in the loaded variant's real type (tables enter as fp32 values)."""
         return np.ascontiguousarray(np.asarray(a), dtype=self.real)
 
     @staticmethod
@@ -265,7 +265,7 @@ class Oracle:
 
     def train_step(self, cfg: Config, lr, step, ent, rel, relw, ent_state, rel_state, relw_state,
                    heads, rels, tails, negs):
-        """In place on arrays of this build's real type (use ``arr`` first). Returns the loss."""
+        """In place on arrays of the loaded variant's real type (use ``arr`` first). Returns the loss."""
         R = self.creal
         for a in (ent, rel, relw, ent_state, rel_state, relw_state):
             assert a is None or (a.dtype == self.real and a.flags.c_contiguous)
@@ -307,7 +307,7 @@ class Oracle:
 
     def encoder_train_step(self, cfg, shared, lr, step, ent, feat, MH, MT, rel, relw, ent_state, MH_state, MT_state, rel_state,
                            relw_state, heads, rels, tails, negs):
-        """In place on arrays of this build's real type.  shared: MH and MT must be the same array."""
+        """In place on arrays of the loaded variant's real type.  shared: MH and MT must be the same array."""
         R = self.creal
         for a in (ent, feat, MH, MT, rel, relw, ent_state, MH_state, MT_state, rel_state, relw_state):
             assert a is None or (a.dtype == self.real and a.flags.c_contiguous)
