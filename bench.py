@@ -523,10 +523,11 @@ def bench_training(ctx, name, w, cpu_seconds):
         # "block" is the statistics pass and "loss" the merge kernel plus the gradient pass; their epilogues also issue
         # special-function instructions per score, and the larger of the two times is the pass's roof.
         sfu = TC_SFU_PER_SCORE[(w["loss"], w["score"] == "transe")]
-        for st in ("block", "loss", "accum_q", "accum_t"):
+        for st in ("block", "loss", "accum_q", "accum_t", "accum"):
             if st not in per_stage_us:
                 continue
-            t_tc = 2.0 * elements / (ctx.peaks["bf16_tflops"] * 1e12) * 1e6
+            # ("accum": both backward contractions in one launch)
+            t_tc = (2 if st == "accum" else 1) * 2.0 * elements / (ctx.peaks["bf16_tflops"] * 1e12) * 1e6
             t_sf = sfu.get(st, 0) * float(B) * N / ctx.alu[MIX_SFU] * 1e6
             roofs[st] = (max(t_tc, t_sf), "tensor" if t_tc >= t_sf else "sfu", {"t_tensor_us": t_tc, "t_sfu_us": t_sf})
     else:
@@ -562,12 +563,12 @@ def bench_training(ctx, name, w, cpu_seconds):
             bound, src = "alu", "measured in this run: kge_measure_alu, special-function mix (the pass's larger roof; tensor time " \
                                 f"{detail['t_tensor_us']:.1f} us)"
         else:
-            achieved, peak, unit = 2.0 * elements / (us * 1e-6) / 1e12, ctx.peaks["bf16_tflops"], "TFLOP/s"
+            achieved, peak, unit = (2 if dominant == "accum" else 1) * 2.0 * elements / (us * 1e-6) / 1e12, ctx.peaks["bf16_tflops"], "TFLOP/s"
             src = ctx.peaks["source"] + " (sustained cuBLAS bf16)"
         roofline = {"bound": bound, "kernel": dominant, "achieved": achieved, "peak": peak, "unit": unit,
                     "frac": t_roof / us, "traffic": ncu_traffic(name, dominant), "peak_source": src, "us_per_launch": us}
         if w.get("tc"):      # tensor pipe activity of the four passes under ncu (tracked capture of the same kernels)
-            roofline["tensor_pipe_active_ncu_pct"] = {st: ncu_tensor_active(name, st) for st in ("block", "loss", "accum_q", "accum_t")}
+            roofline["tensor_pipe_active_ncu_pct"] = {st: ncu_tensor_active(name, st) for st in ("block", "loss", "accum")}
         roofline.update({k: v for k, v in detail.items() if k != "mix"})
     stage_frac = {s: roofs[s][0] / per_stage_us[s] for s in roofs}
     step_roof_us = sum(roofs[s][0] for s in roofs)

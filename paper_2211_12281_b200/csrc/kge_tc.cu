@@ -764,6 +764,164 @@ __global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __gri
         for (int i = threadIdx.x; i < p.beat_rows; i += TC_THREADS) { const int32_t b = beat_sm[i]; if (b) atomicAdd(&p.beat_tmp[i], b); }
 }
 
+// ------------------------------------------------------------------------------------------
+// Both backward contractions of a step in one launch:
+//   problem 0   dQ partial[z] = G . T     A = dL/dF read K-major,  B = negatives read MN-major
+//   problem 1   dT partial[z] = G^T . Q   A = dL/dF read MN-major, B = queries read MN-major
+// Launched one after the other, each gave every CTA a single item, so the pipeline fill, the drain
+// of the accumulator and the launch were exposed twice (11-18 us of 41-47 us at B = 4096,
+// N = 16384, d = 256).  Here the items of both problems form one list that the CTAs take in
+// strides, two items per CTA at the shapes above, and the second item's MMAs run under the first
+// item's drain (the accumulators are used in turn, as in tc_gemm_kernel).  Plain stores of fp32
+// tiles; warp roles, barriers and bounded waits as in tc_gemm_kernel.
+// ------------------------------------------------------------------------------------------
+struct DualProb {
+    int M, N, kb_total, kb_per_split, tiles_m, tiles_n, items;
+    float* C; int64_t ldc, split_stride;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(32 * (2 + TC_EPI_WARPS), 1) tc_gemm_dual_kernel(const __grid_constant__ CUtensorMap tmA0,
+                                                                                    const __grid_constant__ CUtensorMap tmB0,
+                                                                                    const __grid_constant__ CUtensorMap tmA1,
+                                                                                    const __grid_constant__ CUtensorMap tmB1,
+                                                                                    DualProb q0, DualProb q1, int32_t* status, int wait_limit) {
+    constexpr uint32_t STAGE_BYTES = tc_stage_bytes(BN);
+    constexpr int NACC = 512 / BN;
+    constexpr uint32_t TMEM_COLS = NACC * BN;
+    constexpr int EW = TC_EPI_WARPS, EG = EW / 4;
+    extern __shared__ unsigned char tc_smem_raw[];
+    unsigned char* base = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
+    uint64_t* full = reinterpret_cast<uint64_t*>(base + (size_t)TC_STAGES * STAGE_BYTES);
+    uint64_t* empty = full + TC_RING_MAX;
+    uint64_t* acc_full = empty + TC_RING_MAX;
+    uint64_t* acc_empty = acc_full + NACC;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + NACC);
+    volatile uint32_t* stop = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total = q0.items + q1.items;
+    // item -> (problem, K split, first row, first column); column tile fastest inside a problem
+    auto prob_of = [&](int item) { return item < q0.items ? 0 : 1; };
+    auto item_of = [&](const DualProb& q, int local_item) {
+        const int tn = local_item % q.tiles_n, r = local_item / q.tiles_n;
+        return TcItem{r / q.tiles_m, (r % q.tiles_m) * TC_BM, tn * BN};
+    };
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int b = 0; b < NACC; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EW); }
+        *stop = 0;
+        mbar_init_fence();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int ring = 0;
+            for (int item = blockIdx.x; item < total && !*stop; item += gridDim.x) {
+                const int which = prob_of(item);
+                const DualProb q = which ? q1 : q0;
+                const TcItem it = item_of(q, which ? item - q0.items : item);
+                const CUtensorMap* ta = which ? &tmA1 : &tmA0;
+                const CUtensorMap* tb = which ? &tmB1 : &tmB0;
+                const int kb0 = it.z * q.kb_per_split, nkb = min(q.kb_per_split, q.kb_total - kb0);
+                for (int kb = 0; kb < nkb; ++kb, ++ring) {
+                    const int s = ring % TC_STAGES;
+                    if (!mbar_wait_idle(&empty[s], ((ring / TC_STAGES) & 1) ^ 1, wait_limit)) { *stop = 1; set_status(status, KGE_ERR_TIMEOUT); break; }
+                    unsigned char* sa = base + (size_t)s * STAGE_BYTES;
+                    mbar_arrive_expect_tx(&full[s], STAGE_BYTES);
+                    const int k0 = (kb0 + kb) * TC_BK;
+                    if (which) {      // dL/dF with the contraction index as rows: two boxes of 64 output rows
+#pragma unroll
+                        for (int g = 0; g < TC_BM / 64; ++g) tma_load_2d(sa + g * TC_MN_GROUP_BYTES, ta, it.m0 + 64 * g, k0, &full[s]);
+                    } else {
+                        tma_load_2d(sa, ta, k0, it.m0, &full[s]);
+                    }
+#pragma unroll
+                    for (int g = 0; g < BN / 64; ++g) tma_load_2d(sa + TC_A_BYTES + g * TC_MN_GROUP_BYTES, tb, it.n0 + 64 * g, k0, &full[s]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_k = umma_idesc_bf16(TC_BM, BN, false, true), idesc_mn = umma_idesc_bf16(TC_BM, BN, true, true);
+            int ring = 0;
+            bool ok = true;
+            for (int item = blockIdx.x, local = 0; item < total && ok && !*stop; item += gridDim.x, ++local) {
+                const int which = prob_of(item);
+                const DualProb q = which ? q1 : q0;
+                const TcItem it = item_of(q, which ? item - q0.items : item);
+                const int nkb = min(q.kb_per_split, q.kb_total - it.z * q.kb_per_split);
+                const int buf = local % NACC;
+                if (!mbar_wait_idle(&acc_empty[buf], ((local / NACC) & 1) ^ 1, wait_limit)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tmem_acc = tmem_base + (uint32_t)buf * BN;
+                for (int kb = 0; kb < nkb; ++kb, ++ring) {
+                    const int s = ring % TC_STAGES;
+                    if (!mbar_wait_idle(&full[s], (ring / TC_STAGES) & 1, wait_limit)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(base + (size_t)s * STAGE_BYTES);
+#pragma unroll
+                    for (int k = 0; k < TC_BK / 16; ++k) {
+                        const uint64_t ad = which ? umma_desc_mn_sw128(sa + k * 2048) : umma_desc_k_sw128(sa + k * 32);
+                        const uint64_t bd = umma_desc_mn_sw128(sa + TC_A_BYTES + k * 2048);
+                        umma_bf16(tmem_acc, ad, bd, which ? idesc_mn : idesc_k, (kb | k) != 0);
+                    }
+                    umma_commit(&empty[s]);
+                }
+                umma_commit(&acc_full[buf]);           // also after a failed wait, so the epilogue warps wake up
+            }
+            if (!ok) { *stop = 1; set_status(status, KGE_ERR_TIMEOUT); }
+        }
+    } else {
+        const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
+        const int cgrp = (warp - 2) >> 2;              // which half of the tile's columns
+        constexpr int COLS = BN / EG;
+        for (int item = blockIdx.x, local = 0; item < total; item += gridDim.x, ++local) {
+            const int buf = local % NACC;
+            const bool ok = mbar_wait_bounded(&acc_full[buf], (local / NACC) & 1, wait_limit);
+            tc_fence_after();
+            if (!ok || *stop) { if (lane == 0) { *stop = 1; set_status(status, KGE_ERR_TIMEOUT); } break; }
+            const int which = prob_of(item);
+            const DualProb q = which ? q1 : q0;
+            const TcItem it = item_of(q, which ? item - q0.items : item);
+            const int row = it.m0 + quarter * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cgrp * COLS);
+            float* const Cout = q.C + (int64_t)it.z * q.split_stride;
+#pragma unroll 1
+            for (int c0 = cgrp * COLS; c0 < (cgrp + 1) * COLS; c0 += 32) {
+                float v[32];
+                tmem_ld32(taddr + (uint32_t)(c0 - cgrp * COLS), v);
+                if (row >= q.M) continue;
+                const int ncol = it.n0 + c0;
+                float* dst = Cout + (int64_t)row * q.ldc + ncol;
+                if (ncol + 32 <= q.N && (q.ldc & 3) == 0) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) if (ncol + i < q.N) dst[i] = v[i];
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -976,6 +1134,36 @@ int launch_tc_bwd_gemm(kge_handle* h, const unsigned char* tmA, const unsigned c
 }
 }  // namespace
 
+namespace {
+DualProb dual_prob(int M, int N, int K, int split, float* C, int64_t ldc, int bn) {
+    DualProb q{};
+    q.M = M; q.N = N;
+    q.kb_total = (K + TC_BK - 1) / TC_BK;
+    q.kb_per_split = (q.kb_total + split - 1) / split;
+    q.tiles_m = (M + TC_BM - 1) / TC_BM; q.tiles_n = (N + bn - 1) / bn;
+    q.items = q.tiles_m * q.tiles_n * ((q.kb_total + q.kb_per_split - 1) / q.kb_per_split);
+    q.C = C; q.ldc = ldc; q.split_stride = (int64_t)M * ldc;
+    return q;
+}
+template <int BN>
+cudaError_t launch_gemm_dual(kge_handle* h, const DualProb& q0, const DualProb& q1, cudaStream_t s) {
+    constexpr size_t smem = tc_smem_bytes(BN);
+    static DeviceOnce configured;
+    const cudaError_t e = once_per_device(configured, [] {
+        return cudaFuncSetAttribute(tc_gemm_dual_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    });
+    if (e != cudaSuccess) return e;
+    // as few CTAs as give the same number of rounds: SMs left over serve the id sort that runs beside this launch
+    const int total = q0.items + q1.items;
+    const int rounds = (total + h->num_sms - 1) / h->num_sms;
+    const int grid = (total + rounds - 1) / rounds;
+    tc_gemm_dual_kernel<BN><<<grid, 32 * (2 + TC_EPI_WARPS), smem, s>>>(
+        *reinterpret_cast<const CUtensorMap*>(h->tm_g), *reinterpret_cast<const CUtensorMap*>(h->tm_t64),
+        *reinterpret_cast<const CUtensorMap*>(h->tm_g64), *reinterpret_cast<const CUtensorMap*>(h->tm_q64), q0, q1, h->ws.status, h->wait_limit);
+    return cudaSuccess;
+}
+}  // namespace
+
 // Plain contractions for the feature-projection encoder, on the same kernel.
 //   C[M, N] = A[M, K] . B[N, K]^T   (both operands K-major: tensor maps with 128-row boxes)
 int launch_tc_gemm_nt(kge_handle* h, const unsigned char* tmA, const unsigned char* tmB, int M, int N, int K, float* C, int64_t ldc,
@@ -1019,17 +1207,16 @@ int launch_tc_backward(kge_handle* h, cudaStream_t s, cudaStream_t side) {
     const kge_config& c = h->cfg;
     Workspace& w = h->ws;
     const int B = c.batch, N = c.num_neg, d = c.dim;
-    (void)side;   // both contractions are persistent kernels that fill the device: run them in order
-    stage_begin(h, ST_ACCUM_Q, s);
-    int rc = launch_tc_bwd_gemm<false>(h, h->tm_g, h->tm_t64, B, d, N, h->split_q, w.dQpart, d, s);
-    stage_end(h, ST_ACCUM_Q, s);
-    if (rc != KGE_OK) return rc;
-    stage_begin(h, ST_ACCUM_T, s);
-    // one split and no correction term: these rows are final, so they go where the update reads them
+    (void)side;
+    // one split and no correction term: the negatives' rows are final, so they go where the update reads them
     float* dT_out = tc_negatives_direct(h) ? w.grad_ent + (size_t)2 * B * d : w.dTpart;
-    rc = launch_tc_bwd_gemm<true>(h, h->tm_g64, h->tm_q64, N, d, B, h->split_t, dT_out, d, s);
-    stage_end(h, ST_ACCUM_T, s);
-    return rc;
+    const int bn = tc_backward_tile_cols(d);
+    const DualProb q0 = dual_prob(B, d, N, h->split_q, w.dQpart, d, bn), q1 = dual_prob(N, d, B, h->split_t, dT_out, d, bn);
+    stage_begin(h, ST_ACCUM_Q, s);        // (both contractions: the profile reports them as one stage)
+    KGE_CUDA_CHECK(h, bn == 256 ? launch_gemm_dual<256>(h, q0, q1, s) : launch_gemm_dual<128>(h, q0, q1, s));
+    stage_end(h, ST_ACCUM_Q, s);
+    KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
 }
 
 
