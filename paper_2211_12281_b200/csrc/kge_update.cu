@@ -99,38 +99,45 @@ __global__ void __launch_bounds__(RANK_THREADS) rank_kernel(DedupParams p) {
     if (key != ~0ull) { L.perm[rank] = (int32_t)(uint32_t)key; L.sorted[rank] = (int32_t)(key >> 32); }
 }
 
-// blockIdx.x = 0: entity list, 1: relation list.
+// blockIdx.x = 0: entity list, 1: relation list.  One CTA walks the sorted list 1024 positions at a
+// time (coalesced reads): a position opens a segment if its id differs from the one before it, and
+// the number of openings up to a position (a ballot scan inside each warp, warp totals through
+// shared memory, a running carry between rounds) is the index of its segment.
 __global__ void __launch_bounds__(SEG_THREADS) segment_kernel(DedupParams p) {
     __shared__ int32_t warp_tot[SEG_THREADS / 32];
+    __shared__ int32_t carry_sm;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const IdList& L = blockIdx.x == 0 ? p.ent : p.rel;
     const int n = L.n();
-    const int per = (n + SEG_THREADS - 1) / SEG_THREADS;
-    const int r0 = min(n, tid * per), r1 = min(n, r0 + per);
-    int cnt = 0;
-    int32_t prev = r0 > 0 && r0 < n ? L.sorted[r0 - 1] : -1;
-    for (int r = r0; r < r1; ++r) { const int32_t id = L.sorted[r]; cnt += id != prev; prev = id; }
-    int incl = cnt;   // inclusive scan of the per-thread segment-head counts
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    if (lane == 31) warp_tot[warp] = incl;
+    if (tid == 0) carry_sm = 0;
     __syncthreads();
-    int before = 0, total = 0;
-    for (int w = 0; w < SEG_THREADS / 32; ++w) { if (w < warp) before += warp_tot[w]; total += warp_tot[w]; }
-    int u = before + incl - cnt;
-    prev = r0 > 0 && r0 < n ? L.sorted[r0 - 1] : -1;
-    for (int r = r0; r < r1; ++r) {
-        const int32_t id = L.sorted[r];
-        if (id != prev) { L.uniq[u] = id; L.seg[u] = r; ++u; }
-        L.seg_of[r] = u - 1;
-        L.seg_done[r] = 0;
-        if (L.seg_done2) L.seg_done2[r] = 0;
-        prev = id;
+    // (ids are non-negative: position 0 opens a segment; the next round's ids are requested before this round's scan)
+    auto id_at = [&](int r) { return (r >= 0 && r < n) ? L.sorted[r] : -1; };
+    int32_t id_nx = id_at(tid), prev_nx = id_at(tid - 1);
+    for (int base = 0; base < n; base += SEG_THREADS) {
+        const int r = base + tid;
+        const int32_t id = id_nx, prev = prev_nx;
+        id_nx = id_at(r + SEG_THREADS); prev_nx = id_at(r + SEG_THREADS - 1);
+        const bool head = r < n && id != prev;
+        const unsigned mask = __ballot_sync(0xffffffffu, head);
+        const int incl = __popc(mask & (0xffffffffu >> (31 - lane)));
+        if (lane == 0) warp_tot[warp] = __popc(mask);
+        __syncthreads();
+        int before = 0, total = 0;
+        for (int w = 0; w < SEG_THREADS / 32; ++w) { const int t = warp_tot[w]; if (w < warp) before += t; total += t; }
+        const int carry = carry_sm;
+        if (r < n) {
+            const int u = carry + before + incl - 1;
+            if (head) { L.uniq[u] = id; L.seg[u] = r; }
+            L.seg_of[r] = u;
+            L.seg_done[r] = 0;
+            if (L.seg_done2) L.seg_done2[r] = 0;
+        }
+        __syncthreads();
+        if (tid == 0) carry_sm = carry + total;
+        __syncthreads();
     }
-    if (tid == 0) { L.seg[total] = n; *L.count = total; }
+    if (tid == 0) { L.seg[carry_sm] = n; *L.count = carry_sm; }
 }
 
 struct UpdateJob {
