@@ -36,8 +36,14 @@ constexpr int TC_EPI_WARPS_TOPK = 16;                     // the filter epilogue
 constexpr int TC_EPI_GROUPS = TC_EPI_WARPS / 4;
 constexpr int TC_GRAD_STAGE_BYTES = 2048;                 // per epilogue warp: 32 rows x 32 bf16 columns on their way to memory
 constexpr int TC_PIECE = TC_BN / TC_EPI_GROUPS;           // columns of a 128-wide tile per piece of loss statistics
-__host__ __device__ constexpr int tc_epi_warps(int epi) { return (epi & 3) == 3 ? TC_EPI_WARPS_TOPK : TC_EPI_WARPS; }   // 3 = EPI_TOPK
-__host__ __device__ constexpr int tc_threads(int epi) { return 32 * (2 + tc_epi_warps(epi)); }
+// The fused loss epilogues on 256-column tiles run on sixteen warps as well (64 columns = one piece of statistics per warp):
+// measured against eight, C3 passes 41.5 / 58.0 -> 39.4 / 53.8 us, the special-function-bound C4 passes 98.7 / 154.7 -> 98.9 / 135.8 us,
+// although sixteen warps leave 96 registers per thread and the norm-expansion variants spill a little.
+constexpr int TC_FUSED_WARPS_256 = 16;
+__host__ __device__ constexpr int tc_epi_warps(int epi, int bn = 128) {   // 3 = EPI_TOPK, 1 / 2 = the fused loss epilogues
+    return (epi & 3) == 3 ? TC_EPI_WARPS_TOPK : ((((epi & 3) == 1 || (epi & 3) == 2) && bn == 256) ? TC_FUSED_WARPS_256 : TC_EPI_WARPS);
+}
+__host__ __device__ constexpr int tc_threads(int epi, int bn = 128) { return 32 * (2 + tc_epi_warps(epi, bn)); }
 constexpr uint32_t TC_A_BYTES = TC_BM * TC_BK * 2;
 constexpr uint32_t TC_MN_GROUP_BYTES = 64 * TC_BK * 2;    // MN-major operand: 64 contiguous elements x 64 K rows per TMA box
 __host__ __device__ constexpr uint32_t tc_stage_bytes(int bn) { return TC_A_BYTES + (uint32_t)bn * TC_BK * 2; }
@@ -539,12 +545,12 @@ __device__ __forceinline__ void tc_item_next(const TcGemmParams& p, TcItem& it) 
 // the operand is read MN-major (its tensor map has the contraction index as rows), which is how
 // dL/dF, Q and T serve as transposed operands without a transposed copy.
 template <int EPI, int BN = 128, bool A_MN = false, bool B_MN = false>
-__global__ void __launch_bounds__(tc_threads(EPI), 1) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
+__global__ void __launch_bounds__(tc_threads(EPI, BN), 1) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
                                                              const __grid_constant__ CUtensorMap tmB, TcGemmParams p) {
     constexpr uint32_t TC_STAGE_BYTES = tc_stage_bytes(BN);
     constexpr int NACC = 512 / BN;                      // fp32 accumulators in tensor memory, used in turn: all 512 columns
     constexpr uint32_t TC_TMEM_COLS = NACC * BN;
-    constexpr int EW = tc_epi_warps(EPI), EG = EW / 4, TC_THREADS = tc_threads(EPI);
+    constexpr int EW = tc_epi_warps(EPI, BN), EG = EW / 4, TC_THREADS = tc_threads(EPI, BN);
     // For the epilogues that are bound by special-function instructions and row-dependent loads
     // (the norm-expansion kinds) the epilogue warps form two groups that take the CTA's items in
     // turn, so the epilogues of consecutive items overlap; measured faster there (log-sigmoid
@@ -1028,14 +1034,14 @@ cudaError_t launch_gemm_inst(const unsigned char* tmA, const unsigned char* tmB,
                              size_t extra_smem = 0) {
     constexpr size_t smem = tc_smem_bytes(BN);
     constexpr size_t extra_max = (EPI & 3) == EPI_TOPK ? (size_t)TC_BEAT_ROWS_MAX * 4
-                               : ((EPI & 3) == EPI_GRAD ? (size_t)tc_epi_warps(EPI) * TC_GRAD_STAGE_BYTES : 0);
+                               : ((EPI & 3) == EPI_GRAD ? (size_t)tc_epi_warps(EPI, BN) * TC_GRAD_STAGE_BYTES : 0);
     if ((EPI & 3) == EPI_GRAD) extra_smem = extra_max;
     static DeviceOnce configured;
     const cudaError_t e = once_per_device(configured, [] {
         return cudaFuncSetAttribute(tc_gemm_kernel<EPI, BN, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(smem + extra_max));
     });
     if (e != cudaSuccess) return e;
-    tc_gemm_kernel<EPI, BN, A_MN, B_MN><<<std::min(p.items, num_sms), tc_threads(EPI), smem + extra_smem, s>>>(
+    tc_gemm_kernel<EPI, BN, A_MN, B_MN><<<std::min(p.items, num_sms), tc_threads(EPI, BN), smem + extra_smem, s>>>(
         *reinterpret_cast<const CUtensorMap*>(tmA), *reinterpret_cast<const CUtensorMap*>(tmB), p);
     return cudaSuccess;
 }
