@@ -551,11 +551,11 @@ __global__ void __launch_bounds__(tc_threads(EPI, BN), 1) tc_gemm_kernel(const _
     constexpr int NACC = 512 / BN;                      // fp32 accumulators in tensor memory, used in turn: all 512 columns
     constexpr uint32_t TC_TMEM_COLS = NACC * BN;
     constexpr int EW = tc_epi_warps(EPI, BN), EG = EW / 4, TC_THREADS = tc_threads(EPI, BN);
-    // For the epilogues that are bound by special-function instructions and row-dependent loads
-    // (the norm-expansion kinds) the epilogue warps form two groups that take the CTA's items in
-    // turn, so the epilogues of consecutive items overlap; measured faster there (log-sigmoid
-    // L2 passes 164 -> 156 us at B = N = 8192) and slower for the others, which stay one group.
-    constexpr int EGRP = ((EPI & EPI_L2) != 0 && (EPI & 3) != EPI_STORE && EG % 2 == 0) ? 2 : 1;
+    // In the gradient pass of the norm-expansion kinds (bound by special-function instructions, with row- and
+    // column-dependent loads) the epilogue warps form two groups that take the CTA's items in turn, so the epilogues
+    // of consecutive items overlap: measured faster there (136 against 146 us at B = N = 8192) and slower or equal
+    // in every other pass, which stay one group.
+    constexpr int EGRP = ((EPI & EPI_L2) != 0 && (EPI & 3) == EPI_GRAD && EG % 2 == 0) ? 2 : 1;
     constexpr int GW = EW / EGRP, GCOLS = BN / (GW / 4);       // warps per group; columns per warp
     extern __shared__ unsigned char tc_smem_raw[];
     unsigned char* base = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
