@@ -523,6 +523,8 @@ def bench_training(ctx, name, w, cpu_seconds):
         # "block" is the statistics pass and "loss" the merge kernel plus the gradient pass; their epilogues also issue
         # special-function instructions per score, and the larger of the two times is the pass's roof.
         sfu = TC_SFU_PER_SCORE[(w["loss"], w["score"] == "transe")]
+        if w["loss"] == "logsigmoid" and w["score"] == "transe" and w.get("adv_temp") == 1.0 and w.get("gamma", 0.0) <= 80.0:
+            sfu = dict(block=3, loss=3)      # temperature 1: the weight and the loss term share one exponential
         for st in ("block", "loss", "accum_q", "accum_t", "accum"):
             if st not in per_stage_us:
                 continue

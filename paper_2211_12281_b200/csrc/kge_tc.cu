@@ -50,7 +50,8 @@ __host__ __device__ constexpr uint32_t tc_stage_bytes(int bn) { return TC_A_BYTE
 __host__ __device__ constexpr size_t tc_smem_bytes(int bn) { return 1024 + (size_t)TC_STAGES * tc_stage_bytes(bn) + 256; }
 constexpr int TC_BEAT_ROWS_MAX = 8 * 1024;                 // queries whose rank counts fit in shared memory beside the 256-column stages
 
-enum { EPI_STORE = 0, EPI_STATS = 1, EPI_GRAD = 2, EPI_TOPK = 3, EPI_L2 = 4, EPI_CE = 8 };   // L2 / CE: flags of the fused loss epilogues
+enum { EPI_STORE = 0, EPI_STATS = 1, EPI_GRAD = 2, EPI_TOPK = 3, EPI_L2 = 4, EPI_CE = 8,    // L2 / CE: flags of the fused loss epilogues
+       EPI_A1 = 16 };   // log-sigmoid loss of a distance score with self-adversarial temperature exactly 1 (see tc_stats_chunk)
 
 struct TcGemmParams {
     int M, N, K;
@@ -216,7 +217,11 @@ __device__ __forceinline__ TcRowState tc_row_state(const TcGemmParams& p, int ro
 
 // One chunk of 32 scores of the first pass.  FULL: all 32 columns lie inside the problem (no
 // per-element masking); otherwise the first `valid` do.
-template <bool L2, bool CE, bool FULL>
+// A1 (distance scores f <= 0, log-sigmoid loss, temperature a = 1): the weight exponential and the loss term share one
+// exponential.  With e = 2^(y - m) the weight term, exp(gamma + f) = K e with K = exp(gamma) 2^m (one special-function
+// instruction per chunk and lane; K <= exp(gamma) because f <= 0), and softplus(gamma + f) = log(1 + K e): three
+// special-function instructions per score (distance, exponential, logarithm) instead of four.
+template <bool L2, bool CE, bool FULL, bool A1 = false>
 __device__ __forceinline__ void tc_stats_chunk(const TcGemmParams& p, float (&v)[32], float rn, int ncol, int valid,
                                                float k1, float k0, float& m, float& z, float& l) {
     // four independent chains each for the maximum and the sums: a single chain of 32 dependent
@@ -232,12 +237,14 @@ __device__ __forceinline__ void tc_stats_chunk(const TcGemmParams& p, float (&v)
     const float cm = fmaxf(fmaxf(cmv[0], cmv[1]), fmaxf(cmv[2], cmv[3]));
     if (cm > m) { const float r = fast_exp2(m - cm); z *= r; l *= r; m = cm; }
     float zv[4] = {0.f, 0.f, 0.f, 0.f}, lv[4] = {0.f, 0.f, 0.f, 0.f};
+    const float kexp = A1 ? fast_exp2(fmaf(p.gamma, kLog2e, m)) : 0.f;      // exp(gamma) 2^m
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
         float e = fast_exp2((CE ? v[i] : fmaf(v[i], k1, k0)) - m);
         if (!FULL && i >= valid) e = 0.f;
         zv[i & 3] += e;
-        if (!CE) lv[i & 3] = fmaf(e, tc_softplus(p.gamma + v[i]), lv[i & 3]);
+        if (A1) lv[i & 3] = fmaf(e, kLn2 * fast_log2(fmaf(kexp, e, 1.f)), lv[i & 3]);
+        else if (!CE) lv[i & 3] = fmaf(e, tc_softplus(p.gamma + v[i]), lv[i & 3]);
     }
     z += (zv[0] + zv[1]) + (zv[2] + zv[3]);
     if (!CE) l += (lv[0] + lv[1]) + (lv[2] + lv[3]);
@@ -247,7 +254,7 @@ __device__ __forceinline__ void tc_stats_chunk(const TcGemmParams& p, float (&v)
 // sum) over this thread's 64 columns of one row, rescaled whenever the maximum moves.  The
 // exponent is x = a f for the self-adversarial weights and x = f + c for the sampled softmax;
 // it is carried in base 2 (y = x log2 e), so an exponential is one ex2 of a difference.
-template <bool L2, bool CE>
+template <bool L2, bool CE, bool A1>
 __device__ __forceinline__ void tc_epilogue_stats(const TcGemmParams& p, const TcItem& it, int row, const TcRowState& rs, int col_off, uint32_t taddr) {
     const float rn = rs.rn;
     const float k1 = CE ? kLog2e : p.adv_temp * kLog2e, k0 = CE ? p.ce_c * kLog2e : 0.f;
@@ -260,10 +267,10 @@ __device__ __forceinline__ void tc_epilogue_stats(const TcGemmParams& p, const T
     if (row < p.M) {
         const int ncol = it.n0 + col_off;
         const int valid0 = min(32, p.N - ncol), valid1 = min(32, p.N - ncol - 32);   // columns inside the problem (may be <= 0)
-        if (valid0 == 32) tc_stats_chunk<L2, CE, true>(p, v0, rn, ncol, valid0, k1, k0, m, z, l);
-        else if (valid0 > 0) tc_stats_chunk<L2, CE, false>(p, v0, rn, ncol, valid0, k1, k0, m, z, l);
-        if (valid1 == 32) tc_stats_chunk<L2, CE, true>(p, v1, rn, ncol + 32, valid1, k1, k0, m, z, l);
-        else if (valid1 > 0) tc_stats_chunk<L2, CE, false>(p, v1, rn, ncol + 32, valid1, k1, k0, m, z, l);
+        if (valid0 == 32) tc_stats_chunk<L2, CE, true, A1>(p, v0, rn, ncol, valid0, k1, k0, m, z, l);
+        else if (valid0 > 0) tc_stats_chunk<L2, CE, false, A1>(p, v0, rn, ncol, valid0, k1, k0, m, z, l);
+        if (valid1 == 32) tc_stats_chunk<L2, CE, true, A1>(p, v1, rn, ncol + 32, valid1, k1, k0, m, z, l);
+        else if (valid1 > 0) tc_stats_chunk<L2, CE, false, A1>(p, v1, rn, ncol + 32, valid1, k1, k0, m, z, l);
     }
     const int piece = (it.n0 + col_off) / TC_PIECE;
     if (row < p.M && piece < p.row_pieces) p.stat_part[(int64_t)row * p.row_pieces + piece] = make_float4(m, z, l, 0.f);
@@ -273,12 +280,16 @@ __device__ __forceinline__ float bf16_value(uint16_t bits) { return __uint_as_fl
 
 // dL/dF of one pair from its accumulator: scale = loss_scale / normaliser, k0 already holds minus
 // the row's base-2 maximum.
-template <bool L2, bool CE>
-__device__ __forceinline__ float tc_grad_one(const TcGemmParams& p, float acc, float rn, int col, float k1, float k0, float scale) {
+// A1: sigmoid(gamma + f) = t / (1 + t) with t = exp(gamma + f) = krow e, e the weight exponential 2^(y - max) and
+// krow = exp(gamma) 2^max per row: one reciprocal instead of an exponential and a reciprocal.
+template <bool L2, bool CE, bool A1>
+__device__ __forceinline__ float tc_grad_one(const TcGemmParams& p, float acc, float rn, int col, float k1, float k0, float scale, float krow) {
     float inv;
     const float f = tc_score_inv<L2>(p, acc, rn, col, inv);
-    float g = scale * fast_exp2(fmaf(f, k1, k0));
-    if (!CE) g *= tc_sigmoid(p.gamma + f);
+    const float e = fast_exp2(fmaf(f, k1, k0));
+    float g = scale * e;
+    if (A1) { const float t = krow * e; g *= t * fast_rcp(1.f + t); }
+    else if (!CE) g *= tc_sigmoid(p.gamma + f);
     if (L2) g *= inv;
     return g;
 }
@@ -290,7 +301,7 @@ __device__ __forceinline__ float tc_grad_one(const TcGemmParams& p, float acc, f
 // contiguous bytes instead of 16 bytes in each of 32 rows.  The 16-byte chunk c of row r sits at
 // chunk c ^ ((r >> 1) & 3) of the row: both the row-wise writes and the 8-row reads then touch
 // every bank once.
-template <bool L2, bool CE>
+template <bool L2, bool CE, bool A1>
 __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const TcItem& it, int row, const TcRowState& rs, int col_off, uint32_t taddr,
                                                  uint4* stage) {
     const bool rin = row < p.M;
@@ -298,6 +309,7 @@ __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const Tc
     const float2 st = rs.st;
     const float k1 = CE ? kLog2e : p.adv_temp * kLog2e, k0 = (CE ? p.ce_c * kLog2e : 0.f) - st.x;
     const float scale = p.loss_scale * st.y;
+    const float krow = A1 ? fast_exp2(fmaf(p.gamma, kLog2e, st.x)) : 0.f;     // exp(gamma) 2^(row maximum)
     const int lane = threadIdx.x & 31;
     float rsum = 0.f;
 #pragma unroll 1
@@ -309,10 +321,10 @@ __device__ __forceinline__ void tc_epilogue_grad(const TcGemmParams& p, const Tc
         uint32_t g2[16];     // bf16 pairs in memory order
         if (valid == 32) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = tc_grad_one<L2, CE>(p, v[i], rn, ncol + i, k1, k0, scale);
+            for (int i = 0; i < 32; ++i) v[i] = tc_grad_one<L2, CE, A1>(p, v[i], rn, ncol + i, k1, k0, scale, krow);
         } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = i < valid ? tc_grad_one<L2, CE>(p, v[i], rn, ncol + i, k1, k0, scale) : 0.f;
+            for (int i = 0; i < 32; ++i) v[i] = i < valid ? tc_grad_one<L2, CE, A1>(p, v[i], rn, ncol + i, k1, k0, scale, krow) : 0.f;
         }
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
@@ -490,8 +502,8 @@ __device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem&
     if ((EPI & 3) == EPI_STATS || (EPI & 3) == EPI_GRAD) {
 #pragma unroll 1
         for (int c = 0; c < WIDTH; c += TC_PIECE) {
-            if ((EPI & 3) == EPI_STATS) tc_epilogue_stats<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, rs, col_off + c, taddr + (uint32_t)c);
-            else tc_epilogue_grad<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0>(p, it, row, rs, col_off + c, taddr + (uint32_t)c, reinterpret_cast<uint4*>(beat_sm));
+            if ((EPI & 3) == EPI_STATS) tc_epilogue_stats<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0, (EPI & EPI_A1) != 0>(p, it, row, rs, col_off + c, taddr + (uint32_t)c);
+            else tc_epilogue_grad<(EPI & EPI_L2) != 0, (EPI & EPI_CE) != 0, (EPI & EPI_A1) != 0>(p, it, row, rs, col_off + c, taddr + (uint32_t)c, reinterpret_cast<uint4*>(beat_sm));
         }
         return;
     }
@@ -1049,6 +1061,11 @@ cudaError_t launch_gemm_inst(const unsigned char* tmA, const unsigned char* tmB,
 // Scores Q . T^T with one of the fused loss epilogues, in tiles of BN columns.
 template <int BN>
 cudaError_t launch_fused_bn(int pass, bool l2, bool ce, kge_handle* h, const TcGemmParams& p, cudaStream_t s) {
+    // the shared-exponential form of the log-sigmoid distance epilogues: temperature exactly 1, exp(gamma) finite
+    if (l2 && !ce && p.adv_temp == 1.f && p.gamma <= 80.f) {
+        if (pass == EPI_GRAD) return launch_gemm_inst<EPI_GRAD | EPI_L2 | EPI_A1, BN>(h->tm_q, h->tm_t, p, h->num_sms, s);
+        return launch_gemm_inst<EPI_STATS | EPI_L2 | EPI_A1, BN>(h->tm_q, h->tm_t, p, h->num_sms, s);
+    }
     const int key = (pass == EPI_GRAD ? 4 : 0) | (l2 ? 2 : 0) | (ce ? 1 : 0);
     switch (key) {
         case 0: return launch_gemm_inst<EPI_STATS, BN>(h->tm_q, h->tm_t, p, h->num_sms, s);

@@ -326,16 +326,27 @@ def test_tensor_core_score_block(oracle64, score, p, d):
     _run(oracle64, prob, steps=1)
 
 
-@pytest.mark.parametrize("score,p,loss,N", [("distmult", 1, "softmax", 2400), ("transe", 2, "logsigmoid", 2500),
-                                            ("complex", 1, "logsigmoid", 2560)])
-def test_tensor_core_wide_tiles(oracle64, score, p, loss, N):
+@pytest.mark.parametrize("score,p,loss,N,a", [("distmult", 1, "softmax", 2400, 0.0), ("transe", 2, "logsigmoid", 2500, 0.5),
+                                              ("complex", 1, "logsigmoid", 2560, 0.5), ("transe", 2, "logsigmoid", 2500, 1.0)])
+def test_tensor_core_wide_tiles(oracle64, score, p, loss, N, a):
     """Enough tiles to fill every SM, which switches the fused forward passes to 256-column
     tiles: N = 2400 leaves the last tile's upper half outside the problem (its statistics pieces
-    do not exist), N = 2500 a ragged last piece, N = 2560 none."""
+    do not exist), N = 2500 a ragged last piece, N = 2560 none.  Temperature 1 with a distance score
+    takes the epilogues that share one exponential between the weight and the loss term."""
     prob = Problem(E=20000, R=9, T=60000, d=64, score=score, p_norm=p, loss=loss, B=2048, N=N, P=2,
-                   ce_correction=0.3, gamma=4.0 if score == "transe" else 0.0, adv_temp=0.5 if loss == "logsigmoid" else 0.0,
+                   ce_correction=0.3, gamma=4.0 if score == "transe" else 0.0, adv_temp=a,
                    lr=0.05, graph_seed=11, relation_zipf=1.0, tc=True)
     _run(oracle64, prob, steps=1)
+
+
+@pytest.mark.parametrize("gamma", [12.0, 0.5, 90.0])
+def test_tensor_core_distance_logsigmoid_temperature_one(oracle64, gamma):
+    """TransE-L2 on tensor cores, log-sigmoid loss with self-adversarial temperature exactly 1 (128-column tiles
+    here): margin 12 as in the large configuration, a small margin, and one beyond the range of the
+    shared-exponential form (the general epilogues take over there)."""
+    prob = Problem(E=3000, R=9, T=30000, d=128, score="transe", p_norm=2, loss="logsigmoid", B=200, N=300, P=2,
+                   gamma=gamma, adv_temp=1.0, lr=0.05, graph_seed=18, relation_zipf=1.0, tc=True)
+    _run(oracle64, prob, steps=2)
 
 
 def test_tensor_core_path_refuses_what_it_cannot_do():
