@@ -332,6 +332,7 @@ int kge_bind(kge_handle* h, float* ent, float* rel, float* relw, float* ent_stat
     h->ws_base = static_cast<char*>(workspace);
     h->ws_bytes = workspace_bytes;
     h->num_triples = num_triples; h->max_queries = max_queries; h->topk = topk;
+    h->tiles32_ready = false;       // (tensor maps of the inference tiles are encoded at the first full-entity call)
     layout(h, h->ws_base, num_triples, max_queries, topk, &h->ws);
     KGE_CUDA_CHECK(h, cudaMemsetAsync(h->ws.status, 0, 256, static_cast<cudaStream_t>(stream)));
     if (h->cfg.prec == KGE_PREC_BF16_TC) {

@@ -128,6 +128,8 @@ struct kge_handle {
     // read MN-major) for dQ; Gb and Qb (64-row boxes, read MN-major) for dT
     alignas(64) unsigned char tm_q[128], tm_t[128], tm_g[128], tm_g64[128], tm_t64[128], tm_q64[128];
     alignas(64) unsigned char tm_iq[128], tm_eb[128];   // inference: bf16 query vectors and bf16 entity table
+    alignas(64) unsigned char tm_iq32[128], tm_ent32[128];   // inference on CUDA cores: fp32 query vectors and entity table in 64-row x 32-float boxes
+    bool tiles32_ready;
     // encoder: features of the head / tail+negative slots and M_H / M_T (K-major, 128-row boxes) for the projection; the
     // slots' gradient rows and features again (MN-major, 64-row boxes) for dM = dE^T . F
     alignas(64) unsigned char tm_fh[128], tm_ft[128], tm_mh[128], tm_mt[128], tm_gh64[128], tm_gt64[128], tm_fh64[128], tm_ft64[128];
@@ -208,6 +210,8 @@ int launch_apply_gradients(kge_handle* h, float* table, float* state, int64_t ro
                            int n, uint64_t step, float lr, void* scratch, cudaStream_t s);
 // Tensor-core score block: F from the bf16 operand copies; tensor maps are made at bind time.
 int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows);
+// Tensor map of a row-major fp32 matrix [rows, cols] read in boxes of 64 rows x 32 floats with the 128-byte swizzle.
+int tc_make_f32_tile_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols);
 int tc_backward_tile_cols(int cols);
 int tc_pieces_per_tile();
 // The dT contraction of the dot-product kinds with a single K split is the negatives' gradient rows: it writes them in place.

@@ -16,6 +16,8 @@
 
 #include <cuda_bf16.h>
 
+#include <cuda.h>
+
 #include "kge_common.cuh"
 
 namespace kge {
@@ -193,8 +195,31 @@ __device__ __forceinline__ float float_below(float x) {
 // f >= f0 is f > (largest float below f0).  So the common case costs one compare per pair and
 // test; a row whose reference id falls inside the tile, a ragged last tile and non-finite
 // reference scores take the element-by-element form.
+//
+// `cuts` (optional, shared memory, one entry per query row of the tile): the two comparison values of a row in the
+// plain case, worked out once per row by score_tile_row_cuts while the tile's rows are still on their way, so that
+// the sixteen threads of a row do not each load the row's state and form them again.
+__device__ __forceinline__ void score_tile_row_cuts(const InferParams& p, int q0, int64_t e0, int row, float4* cuts) {
+    const int64_t g0 = e0 + p.id_base;
+    const int q = q0 + row;
+    float4 c = make_float4(0.f, INFINITY, 0.f, 0.f);     // (x: candidate cut, y: rank cut, z: 1 = plain case)
+    if (q < p.nq && e0 + IE <= p.e_hi) {
+        const float thr = p.w.thr[q]; const int32_t thr_id = p.w.thr_id[q];
+        float ft = 0.f; int32_t tt = -1;
+        if (p.tt) { ft = p.w.iftrue[q]; tt = p.tt[q]; }
+        const bool thr_out = thr_id < g0 || thr_id >= g0 + IE, tt_out = !p.tt || tt < g0 || tt >= g0 + IE;
+        if (thr_out && tt_out && fabsf(thr) < INFINITY && fabsf(ft) < INFINITY) {
+            c.x = thr_id >= g0 + IE ? float_below(thr) : thr;
+            c.y = !p.tt ? INFINITY : (tt >= g0 + IE ? float_below(ft) : ft);     // without true tails nothing is counted
+            c.z = 1.f;
+        }
+    }
+    cuts[row] = c;
+}
+
 template <int KIND>
-__device__ __forceinline__ void score_tile_epilogue(const InferParams& p, const float (&acc)[4][4], int q0, int64_t e0, int tx, int ty) {
+__device__ __forceinline__ void score_tile_epilogue(const InferParams& p, const float (&acc)[4][4], int q0, int64_t e0, int tx, int ty,
+                                                    const float4* cuts = nullptr) {
     const int64_t g0 = e0 + p.id_base;                  // the id the caller knows the tile's first entity by
     const bool whole = e0 + IE <= p.e_hi;
     int beat_all = 0;                                   // four rows' counts, one byte each (at most 4 per thread, 64 per row)
@@ -202,6 +227,30 @@ __device__ __forceinline__ void score_tile_epilogue(const InferParams& p, const 
     for (int i = 0; i < 4; ++i) {
         const int q = q0 + ty + 16 * i;
         const bool qin = q < p.nq;
+        if (cuts) {
+            const float4 c = cuts[ty + 16 * i];
+            if (c.z != 0.f) {
+                int beat = 0;
+                float f[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { f[j] = canon_finish(KIND, acc[i][j]); beat += f[j] > c.y ? 1 : 0; }
+                if (fmaxf(fmaxf(f[0], f[1]), fmaxf(f[2], f[3])) > c.x) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (f[j] > c.x) {
+                            const int slot = atomicAdd(&p.w.cand_cnt[q], 1);
+                            if (slot < kCandCap) {
+                                p.w.cand_score[(int64_t)q * kCandCap + slot] = f[j];
+                                p.w.cand_id[(int64_t)q * kCandCap + slot] = (int32_t)(g0 + tx + 16 * j);
+                            } else {
+                                p.w.status[1] = 1;
+                            }
+                        }
+                }
+                beat_all |= beat << (8 * i);
+                continue;
+            }
+        }
         float thr = 0.f, ft = 0.f; int32_t thr_id = 0, tt = 0;
         if (qin) {
             thr = p.w.thr[q]; thr_id = p.w.thr_id[q];
@@ -222,11 +271,14 @@ __device__ __forceinline__ void score_tile_epilogue(const InferParams& p, const 
         if (plain) {
             const float thr_c = thr_id >= g0 + IE ? float_below(thr) : thr;
             const float ft_c = tt >= g0 + IE ? float_below(ft) : ft;
+            float f[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float f = canon_finish(KIND, acc[i][j]);
-                beat += f > ft_c ? 1 : 0;
-                if (f > thr_c) append(f, (int32_t)(g0 + tx + 16 * j));
+            for (int j = 0; j < 4; ++j) { f[j] = canon_finish(KIND, acc[i][j]); beat += f[j] > ft_c ? 1 : 0; }
+            // candidates are rare once the threshold has tightened: one test of the largest of the four
+            // instead of four divergent branches
+            if (fmaxf(fmaxf(f[0], f[1]), fmaxf(f[2], f[3])) > thr_c) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) if (f[j] > thr_c) append(f[j], (int32_t)(g0 + tx + 16 * j));
             }
             if (!p.tt) beat = 0;
         } else {
@@ -275,6 +327,8 @@ __global__ void __launch_bounds__(256) score_tile_kernel(InferParams p) {
     const float4* Wg = reinterpret_cast<const float4*>(p.w.iwhat);
     const float4* Tg = reinterpret_cast<const float4*>(p.ent);
 
+    __shared__ float4 cuts[IQ];
+    if (tid >= 256 - IQ) score_tile_row_cuts(p, q0, e0, tid - (256 - IQ), cuts);     // (read after the barriers of the loop below)
     float acc[4][4], u[4][4];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
@@ -326,7 +380,7 @@ __global__ void __launch_bounds__(256) score_tile_kernel(InferParams p) {
             __syncthreads();
         }
     }
-    score_tile_epilogue<KIND>(p, acc, q0, e0, tx, ty);
+    score_tile_epilogue<KIND>(p, acc, q0, e0, tx, ty, cuts);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -384,6 +438,8 @@ __global__ void __launch_bounds__(256) score_tile_tma_kernel(InferParams p) {
     };
     issue(0, 0);
     if (nstage > 1 && nchunk > 1) issue(1, 1);
+    __shared__ float4 cuts[IQ];
+    if (tid >= 256 - IQ) score_tile_row_cuts(p, q0, e0, tid - (256 - IQ), cuts);     // (read after the barrier that follows the first wait)
 
     float acc[4][4];
 #pragma unroll
@@ -421,7 +477,117 @@ __global__ void __launch_bounds__(256) score_tile_tma_kernel(InferParams p) {
             issue(chunk + nstage, stage);
         }
     }
-    score_tile_epilogue<KIND>(p, acc, q0, e0, tx, ty);
+    score_tile_epilogue<KIND>(p, acc, q0, e0, tx, ty, cuts);
+}
+
+// ------------------------------------------------------------------------------------------
+// The same score tile for rows of at least 128 floats, staged by the TMA engine's tensor copies:
+// eight copies per stage (four 64-row x 32-float boxes of the queries, four of the entities, 128-byte
+// swizzle) issued by one thread, instead of one bulk copy per row issued lane by lane (128 per
+// tile, about 5 % of the kernel's instructions).  A box holds a row's 32 floats as eight 16-byte
+// units, unit u of row r at position u ^ (r & 7): a thread's rows all share r & 7, so its eight
+// unit offsets are computed once and every 128-bit read is base + constant + one of them, without
+// bank conflicts.  What a box covers beyond the matrix reads as zero, and adding the term of a
+// zero pair leaves every accumulator as it is, so ragged rows keep the canonical order and value.
+// ------------------------------------------------------------------------------------------
+constexpr int ITB_BOX_BYTES = 64 * 128, ITB_CHUNK_BYTES = 4 * ITB_BOX_BYTES, ITB_STAGE_BYTES = 2 * ITB_CHUNK_BYTES;
+inline size_t infer_tensor_smem(int d) { return 1024 + (size_t)infer_tma_stages(d) * ITB_STAGE_BYTES + 2 * sizeof(uint64_t); }
+__device__ __forceinline__ void tile_load_2d(void* dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(256, 3) score_tile_tensor_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmE,
+                                                                   InferParams p) {
+    extern __shared__ unsigned char smraw_t[];
+    unsigned char* base = smraw_t + ((1024u - (smem_u32(smraw_t) & 1023u)) & 1023u);       // swizzled boxes want 1024-byte alignment
+    const int nstage = infer_tma_stages(p.d);
+    const int nchunk = (p.d + IKT - 1) / IKT;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base + (size_t)nstage * ITB_STAGE_BYTES);
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int qt = blockIdx.x % p.q_tiles;
+    const int64_t et = blockIdx.x / p.q_tiles;
+    const int q0 = qt * IQ;
+    const int64_t e0 = p.e_lo + et * IE;
+
+    if (tid == 0) {
+        for (int st = 0; st < nstage; ++st) mbar_init(&bars[st], 1);
+        mbar_init_fence();
+    }
+    __syncthreads();
+    auto issue = [&](int chunk, int stage) {
+        if (tid != 0) return;
+        unsigned char* qs = base + (size_t)stage * ITB_STAGE_BYTES;
+        mbar_arrive_expect_tx(&bars[stage], (uint32_t)ITB_STAGE_BYTES);
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            tile_load_2d(qs + b * ITB_BOX_BYTES, &tmQ, chunk * IKT + 32 * b, q0, &bars[stage]);
+            tile_load_2d(qs + ITB_CHUNK_BYTES + b * ITB_BOX_BYTES, &tmE, chunk * IKT + 32 * b, (int)e0, &bars[stage]);
+        }
+    };
+    issue(0, 0);
+    if (nstage > 1 && nchunk > 1) issue(1, 1);
+    __shared__ float4 cuts[IQ];
+    if (tid >= 256 - IQ) score_tile_row_cuts(p, q0, e0, tid - (256 - IQ), cuts);     // (read after the barrier that follows the first wait)
+
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    uint32_t qoff[8], toff[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) { qoff[u] = (uint32_t)((u ^ (ty & 7)) << 4); toff[u] = (uint32_t)((u ^ (tx & 7)) << 4); }
+
+    for (int chunk = 0; chunk < nchunk; ++chunk) {
+        const int stage = chunk % nstage;
+        const bool ok = mbar_wait_bounded(&bars[stage], (uint32_t)(chunk / nstage) & 1u, p.wait_limit);
+        if (!__syncthreads_and(ok)) {
+            if (tid == 0) set_status(p.w.status, KGE_ERR_TIMEOUT);
+            for (int st = 0; st < nstage; ++st) (void)mbar_wait_bounded(&bars[st], (uint32_t)(chunk / nstage) & 1u, p.wait_limit);
+            return;
+        }
+        const unsigned char* qrow = base + (size_t)stage * ITB_STAGE_BYTES + ty * 128;
+        const unsigned char* trow = base + (size_t)stage * ITB_STAGE_BYTES + ITB_CHUNK_BYTES + tx * 128;
+        const int nbox = (min(IKT, p.d - chunk * IKT) + 31) / 32;
+#pragma unroll 1
+        for (int b = 0; b < nbox; ++b) {
+            const unsigned char* qb = qrow + b * ITB_BOX_BYTES;
+            const unsigned char* tb = trow + b * ITB_BOX_BYTES;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                float4 qv[4], tv[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    qv[i] = *reinterpret_cast<const float4*>(qb + i * (16 * 128) + qoff[u]);
+                    tv[i] = *reinterpret_cast<const float4*>(tb + i * (16 * 128) + toff[u]);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) canon_update<KIND>(acc[i][j], qv[i], tv[j]);
+            }
+        }
+        if (chunk + nstage < nchunk) {
+            __syncthreads();             // every thread is done reading this stage
+            issue(chunk + nstage, stage);
+        }
+    }
+    score_tile_epilogue<KIND>(p, acc, q0, e0, tx, ty, cuts);
+}
+
+template <int KIND>
+cudaError_t launch_score_tile_tensor(const kge_handle* h, const InferParams& p, unsigned grid, cudaStream_t s) {
+    static DeviceOnce configured;
+    const cudaError_t e = once_per_device(configured, [] {
+        return cudaFuncSetAttribute(score_tile_tensor_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)infer_tensor_smem(kMaxDim));
+    });
+    if (e != cudaSuccess) return e;
+    score_tile_tensor_kernel<KIND><<<grid, 256, infer_tensor_smem(p.d), s>>>(*reinterpret_cast<const CUtensorMap*>(h->tm_iq32),
+                                                                            *reinterpret_cast<const CUtensorMap*>(h->tm_ent32), p);
+    return cudaSuccess;
 }
 
 template <int KIND>
@@ -586,9 +752,18 @@ __global__ void finish_kernel(InferParams p, int32_t* out_ids, float* out_scores
     if (out_ranks) out_ranks[q] = (p.raw_beat ? 0 : 1) + p.w.beat[q];
 }
 
-cudaError_t launch_score_tiles(const InferParams& p, cudaStream_t s) {
+cudaError_t launch_score_tiles(const kge_handle* h, const InferParams& p, cudaStream_t s) {
     const int64_t e_tiles = (p.e_hi - p.e_lo + IE - 1) / IE;
     const unsigned grid = (unsigned)(e_tiles * p.q_tiles);
+    if (h->tiles32_ready && p.d >= IKT) {      // rows of at least 128 floats: tiles staged by tensor copies
+        switch (p.kind) {
+            case KIND_L1: return launch_score_tile_tensor<KIND_L1>(h, p, grid, s);
+            case KIND_L2: return launch_score_tile_tensor<KIND_L2>(h, p, grid, s);
+            case KIND_CL1: return launch_score_tile_tensor<KIND_CL1>(h, p, grid, s);
+            case KIND_DOT: return launch_score_tile_tensor<KIND_DOT>(h, p, grid, s);
+            default: break;
+        }
+    }
     switch (p.kind) {
         case KIND_L1: return launch_score_tile_tma<KIND_L1>(p, grid, s);
         case KIND_L2: return launch_score_tile_tma<KIND_L2>(p, grid, s);
@@ -671,9 +846,16 @@ int run_score_all_topk(kge_handle* h, const int32_t* qh, const int32_t* qr, int3
             KGE_LAUNCH_CHECK(h);
         }
     }
+    if (!tc && !h->tiles32_ready && c.dim >= IKT && h->kind != KIND_TH_L1 && h->kind != KIND_TH_L2) {
+        // tensor maps of the fp32 query vectors and of the entity table (host-side encoding, nothing allocated)
+        int rc = tc_make_f32_tile_map(h, h->tm_iq32, h->ws.iq, h->max_queries, c.dim);
+        if (rc == KGE_OK) rc = tc_make_f32_tile_map(h, h->tm_ent32, h->ent, c.num_entities, c.dim);
+        if (rc != KGE_OK) return rc;
+        h->tiles32_ready = true;
+    }
     auto score_chunk = [&](const InferParams& ip) -> int {
         if (tc) return launch_tc_infer_chunk(h, nq, ip.e_lo, ip.e_hi, true_tails, ip.id_base, s);
-        KGE_CUDA_CHECK(h, launch_score_tiles(ip, s));
+        KGE_CUDA_CHECK(h, launch_score_tiles(h, ip, s));
         KGE_LAUNCH_CHECK(h);
         return KGE_OK;
     };

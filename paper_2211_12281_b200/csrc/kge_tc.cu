@@ -976,6 +976,20 @@ int tc_make_operand_map(kge_handle* h, void* map_out, const void* base, int64_t 
     return KGE_OK;
 }
 
+int tc_make_f32_tile_map(kge_handle* h, void* map_out, const void* base, int64_t rows, int64_t cols) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) { std::snprintf(h->cuda_err, sizeof(h->cuda_err), "cuTensorMapEncodeTiled is not available from this driver"); return KGE_ERR_CUDA; }
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 4};
+    const cuuint32_t box[2] = {32, 64};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(static_cast<CUtensorMap*>(map_out), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base),
+                          dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { std::snprintf(h->cuda_err, sizeof(h->cuda_err), "cuTensorMapEncodeTiled failed with code %d", (int)r); return KGE_ERR_CUDA; }
+    return KGE_OK;
+}
+
 namespace {
 
 // One warp per positive merges the per-piece statistics of its row (and the positive score,
