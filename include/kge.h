@@ -81,7 +81,11 @@ typedef struct {
     int32_t head_part;      /* -1: slots spread evenly over all P*P buckets, bucket-major;
                                i >= 0: the micro-batch B_i of Eq. 3 (all heads in partition i) */
     int32_t sample_mode;    /* 0: cube-root relation law of Section 4 "Training"; 1: uniform over the bucket */
-    int32_t _reserved;
+    int32_t contract;       /* TransH with fp32 arithmetic: where the backward's two contractions with per-pair coefficients
+                               (sum_n c_bn t_n and sum_b c_bn w_b, c = -dL/dF . sum_k s_k w_k) run.  0: on the tensor cores, as
+                               bf16 two-term splits of both operands with all four products accumulated in fp32 (2^-17 relative
+                               per term), from 2^22 pairs per block and dim % 32 == 0 on, else on the CUDA cores in fp32;
+                               1: on the tensor cores whenever dim % 32 == 0; 2: always on the CUDA cores.  Ignored elsewhere. */
     float gamma;            /* margin of the log-sigmoid loss */
     float adv_temp;         /* a >= 0, self-adversarial temperature (0 = uniform weights 1/N) */
     float ce_correction;    /* c of the sampled-softmax loss; the paper's value is log((|E|-1)/N) */

@@ -43,7 +43,7 @@ class KgeConfig(C.Structure):
         ("dim", C.c_int32), ("score", C.c_int32), ("p_norm", C.c_int32), ("loss", C.c_int32),
         ("opt", C.c_int32), ("prec", C.c_int32),
         ("batch", C.c_int32), ("num_neg", C.c_int32), ("num_parts", C.c_int32),
-        ("head_part", C.c_int32), ("sample_mode", C.c_int32), ("_reserved", C.c_int32),
+        ("head_part", C.c_int32), ("sample_mode", C.c_int32), ("contract", C.c_int32),
         ("gamma", C.c_float), ("adv_temp", C.c_float), ("ce_correction", C.c_float), ("loss_scale", C.c_float),
         ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
         ("seed", C.c_uint64),
@@ -54,14 +54,14 @@ class KgeConfig(C.Structure):
     def make(cls, *, num_entities, num_relations, dim, score, p_norm=1, loss="logsigmoid", opt="sgd",
              prec=PREC_FP32, batch=1, num_neg=1, num_parts=1, head_part=-1, sample_mode=0,
              gamma=0.0, adv_temp=0.0, ce_correction=0.0, loss_scale=1.0, lr=0.1,
-             beta1=0.9, beta2=0.999, eps=None, seed=0, reg_lambda=0.0, reg_form=0, feat_dim=0, feat_shared=0) -> "KgeConfig":
+             beta1=0.9, beta2=0.999, eps=None, seed=0, reg_lambda=0.0, reg_form=0, feat_dim=0, feat_shared=0, contract=0) -> "KgeConfig":
         score = SCORE_NAMES[score] if isinstance(score, str) else int(score)
         loss = LOSS_NAMES[loss] if isinstance(loss, str) else int(loss)
         opt = OPT_NAMES[opt] if isinstance(opt, str) else int(opt)
         if eps is None:
             eps = 1e-10 if opt == OPT_ROWWISE_ADAGRAD else 1e-8
         return cls(num_entities, num_relations, dim, score, p_norm, loss, opt, prec, batch, num_neg,
-                   num_parts, head_part, sample_mode, 0, gamma, adv_temp, ce_correction, loss_scale,
+                   num_parts, head_part, sample_mode, contract, gamma, adv_temp, ce_correction, loss_scale,
                    lr, beta1, beta2, eps, seed, reg_lambda, reg_form, feat_dim, feat_shared)
 
 

@@ -121,9 +121,14 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
     w.U = th ? cv.take<float>(B * N) : nullptr;
     w.Cc = th ? cv.take<float>(B * N) : nullptr;
     w.wsum = th ? cv.take<float>(B) : nullptr;
+    const size_t Np = (N + 63) / 64 * 64;
+    w.Csb = h->th_tc ? cv.take<uint16_t>(B * 2 * Np) : nullptr;
+    w.Tsb = h->th_tc ? cv.take<uint16_t>(N * 2 * d) : nullptr;
+    w.Wsb = h->th_tc ? cv.take<uint16_t>(B * 2 * d) : nullptr;
+    const size_t xs = (size_t)th_contract_slabs(h);      // slabs the tensor-core contractions add behind the splits' own
     w.dQpart = cv.take<float>((size_t)h->split_q * B * d);
-    w.dWpart = th ? cv.take<float>((size_t)h->split_q * B * d) : nullptr;
-    w.dTpart = cv.take<float>((size_t)h->split_t * N * d);
+    w.dWpart = th ? cv.take<float>(((size_t)h->split_q + xs) * B * d) : nullptr;
+    w.dTpart = cv.take<float>(((size_t)h->split_t + xs) * N * d);
     w.grad_ent = cv.take<float>((2 * B + N) * d);
     w.grad_rel = cv.take<float>(B * kw);
     w.grad_relw = th ? cv.take<float>(B * d) : nullptr;
@@ -218,6 +223,7 @@ int kge_create(const kge_config* cfg, kge_handle** out) {
     if (c.batch <= 0 || c.num_neg <= 0 || c.num_parts <= 0) return KGE_ERR_BAD_ARG;
     if (c.head_part >= c.num_parts || c.head_part < -1) return KGE_ERR_BAD_ARG;
     if (c.sample_mode != 0 && c.sample_mode != 1) return KGE_ERR_BAD_ARG;
+    if (c.contract < 0 || c.contract > 2) return KGE_ERR_BAD_ARG;
     if (!(c.adv_temp >= 0.f)) return KGE_ERR_BAD_ARG;
     if (!(c.reg_lambda >= 0.f) || (c.reg_form != 0 && c.reg_form != 1)) return KGE_ERR_BAD_ARG;
     if (c.feat_dim < 0 || (c.feat_shared != 0 && c.feat_shared != 1)) return KGE_ERR_BAD_ARG;
@@ -266,6 +272,18 @@ int kge_create(const kge_config* cfg, kge_handle** out) {
     if (c.prec == KGE_PREC_BF16_TC) {   // the backward contractions run as 128 x 128 tensor-core tiles split over K
         h->split_q = pick_split_tc(c.batch, c.dim, c.num_neg, h->num_sms);
         h->split_t = pick_split_tc(c.num_neg, c.dim, c.batch, h->num_sms);
+    }
+    // TransH, fp32: the backward's two contractions with per-pair coefficients go to the tensor cores as bf16
+    // two-term splits once a block has enough pairs to pay for the extra launch (`contract`: 0 automatic, 1 always
+    // where the shapes allow, 2 never)
+    h->th_tc = c.score == KGE_TRANSH && c.prec == KGE_PREC_FP32 && c.dim % 32 == 0 && c.contract != 2 &&
+               (c.contract == 1 || (int64_t)c.batch * c.num_neg >= ((int64_t)1 << 22));
+    h->th_gsplit = 1;
+    if (h->th_tc) {   // K splits: as many as still give every SM at most one tile, each at least eight 64-wide slices deep, at most 4
+        const int bn = 2 * c.dim > 128 ? 256 : 128;
+        const int tiles = ((c.batch + 127) / 128 + (c.num_neg + 127) / 128) * ((2 * c.dim + bn - 1) / bn);
+        const int kb = 2 * ((std::min(c.batch, c.num_neg) + 63) / 64);
+        h->th_gsplit = std::max(1, std::min(std::min(h->num_sms / tiles, kb / 8), 4));
     }
     h->split_m = 1;
     h->features_bound = false;
@@ -348,6 +366,16 @@ int kge_bind(kge_handle* h, float* ent, float* rel, float* relw, float* ent_stat
             rc = tc_make_operand_map(h, h->tm_iq, h->ws.iqb, max_queries, d, d, 128);
             if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_eb, h->ws.Eb, h->cfg.num_entities, d, d, 128);
         }
+        if (rc != KGE_OK) return rc;
+    }
+    if (h->th_tc) {
+        const int64_t B = h->cfg.batch, N = h->cfg.num_neg, d = h->cfg.dim, Np = (N + 63) / 64 * 64;
+        // (the padding columns of the coefficient splits are never written: zero once, zero for good)
+        KGE_CUDA_CHECK(h, cudaMemsetAsync(h->ws.Csb, 0, (size_t)B * 2 * Np * 2, static_cast<cudaStream_t>(stream)));
+        int rc = tc_make_operand_map(h, h->tm_cs, h->ws.Csb, B, 2 * Np, 2 * Np, 128);
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_cs64, h->ws.Csb, B, 2 * Np, 2 * Np, 64);
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_ts64, h->ws.Tsb, N, 2 * d, 2 * d, 64);
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_ws64, h->ws.Wsb, B, 2 * d, 2 * d, 64);
         if (rc != KGE_OK) return rc;
     }
     if (!h->streams_ready) {

@@ -68,6 +68,10 @@ struct Workspace {
     float *F;                              // [B,N] scores, overwritten by dL/dF
     float *U, *Cc;                         // [B,N] TransH: w.t and the contraction c' = sum_k s_k w_k of every pair
     float *wsum;                           // [B] TransH: sum of the unit normal's coordinates
+    // TransH with the backward's two per-pair-coefficient contractions on tensor cores: bf16 two-term splits
+    // (x = x1 + x2 up to 2^-17 relative) of c = -dL/dF c' as [B, 2 Np] = [c1 | c2] (Np = N rounded up to 64,
+    // padding kept zero), of the negatives as [N, 2d] = [t1 | t2] and of the unit normals as [B, 2d]
+    uint16_t *Csb, *Tsb, *Wsb;
     float *dQpart, *dWpart, *dTpart;       // [Sq,B,d], [Sq,B,d] (TransH), [St,N,d]
     float *grad_ent, *grad_rel, *grad_relw;  // [2B+N,d], [B,kw], [B,d]
     // dedup
@@ -119,6 +123,8 @@ struct kge_handle {
     int64_t num_triples;
     int32_t max_queries, topk;
     int split_q, split_t;   // column splits of the two backward accumulations
+    bool th_tc;             // TransH: sum_n c_bn t_n and sum_b c_bn w_b as tensor-core contractions of bf16 splits
+    int th_gsplit;          // K splits of each of those contractions (each leaves two partial slabs)
     bool bound, graph_loaded;
     int64_t launches;
     int num_sms;
@@ -127,6 +133,7 @@ struct kge_handle {
     // TMA tensor maps (tensor-core path): Qb, Tb (128-row boxes) for the scores; Gb (128-row boxes) and Tb (64-row boxes,
     // read MN-major) for dQ; Gb and Qb (64-row boxes, read MN-major) for dT
     alignas(64) unsigned char tm_q[128], tm_t[128], tm_g[128], tm_g64[128], tm_t64[128], tm_q64[128];
+    alignas(64) unsigned char tm_cs[128], tm_cs64[128], tm_ts64[128], tm_ws64[128];   // TransH splits: Csb K-major / MN-major, Tsb, Wsb
     alignas(64) unsigned char tm_iq[128], tm_eb[128];   // inference: bf16 query vectors and bf16 entity table
     alignas(64) unsigned char tm_iq32[128], tm_ent32[128];   // inference on CUDA cores: fp32 query vectors and entity table in 64-row x 32-float boxes
     bool tiles32_ready;
@@ -220,6 +227,8 @@ int launch_tc_backward(kge_handle* h, cudaStream_t s, cudaStream_t side);
 // TransH score block (scores, w.t, c') and its two backward accumulations (kge_transh.cu).
 int launch_th_forward(kge_handle* h, cudaStream_t s);
 int launch_th_backward(kge_handle* h, cudaStream_t sq, cudaStream_t st);
+int th_contract_slabs(const kge_handle* h);          // partial slabs the tensor-core contractions add per side (0 when off)
+int launch_th_contract_gemm(kge_handle* h, cudaStream_t s);
 int launch_tc_forward(kge_handle* h, cudaStream_t s);
 int launch_tc_gemm_nt(kge_handle* h, const unsigned char* tmA, const unsigned char* tmB, int M, int N, int K, float* C, int64_t ldc,
                       cudaStream_t s);

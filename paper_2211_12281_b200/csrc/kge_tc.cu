@@ -796,6 +796,12 @@ __global__ void __launch_bounds__(tc_threads(EPI, BN), 1) tc_gemm_kernel(const _
 struct DualProb {
     int M, N, kb_total, kb_per_split, tiles_m, tiles_n, items;
     float* C; int64_t ldc, split_stride;
+    // K in segments of seg_kb slices: the B operand's K coordinate starts over with every segment, and an MN-major
+    // A operand moves a_seg_x columns to the right per segment instead of going on downwards (its segments lie
+    // side by side in memory).  One segment = a plain contraction.
+    int seg_kb, a_seg_x;
+    // fold > 0: output column c goes to column c % fold of slab c / fold (slabs fold_stride floats apart)
+    int fold; int64_t fold_stride;
 };
 
 template <int BN>
@@ -856,15 +862,17 @@ __global__ void __launch_bounds__(32 * (2 + TC_EPI_WARPS), 1) tc_gemm_dual_kerne
                     if (!mbar_wait_idle(&empty[s], ((ring / TC_STAGES) & 1) ^ 1, wait_limit)) { *stop = 1; set_status(status, KGE_ERR_TIMEOUT); break; }
                     unsigned char* sa = base + (size_t)s * STAGE_BYTES;
                     mbar_arrive_expect_tx(&full[s], STAGE_BYTES);
-                    const int k0 = (kb0 + kb) * TC_BK;
+                    const int kblk = kb0 + kb, seg = kblk / q.seg_kb;
+                    const int k0 = kblk * TC_BK, kseg = (kblk - seg * q.seg_kb) * TC_BK;
                     if (which) {      // dL/dF with the contraction index as rows: two boxes of 64 output rows
 #pragma unroll
-                        for (int g = 0; g < TC_BM / 64; ++g) tma_load_2d(sa + g * TC_MN_GROUP_BYTES, ta, it.m0 + 64 * g, k0, &full[s]);
+                        for (int g = 0; g < TC_BM / 64; ++g)
+                            tma_load_2d(sa + g * TC_MN_GROUP_BYTES, ta, it.m0 + 64 * g + seg * q.a_seg_x, kseg, &full[s]);
                     } else {
                         tma_load_2d(sa, ta, k0, it.m0, &full[s]);
                     }
 #pragma unroll
-                    for (int g = 0; g < BN / 64; ++g) tma_load_2d(sa + TC_A_BYTES + g * TC_MN_GROUP_BYTES, tb, it.n0 + 64 * g, k0, &full[s]);
+                    for (int g = 0; g < BN / 64; ++g) tma_load_2d(sa + TC_A_BYTES + g * TC_MN_GROUP_BYTES, tb, it.n0 + 64 * g, kseg, &full[s]);
                 }
             }
         }
@@ -921,6 +929,7 @@ __global__ void __launch_bounds__(32 * (2 + TC_EPI_WARPS), 1) tc_gemm_dual_kerne
                 if (row >= q.M) continue;
                 const int ncol = it.n0 + c0;
                 float* dst = Cout + (int64_t)row * q.ldc + ncol;
+                if (q.fold > 0) dst += (int64_t)(ncol / q.fold) * (q.fold_stride - q.fold);     // (32-column pieces never straddle a fold)
                 if (ncol + 32 <= q.N && (q.ldc & 3) == 0) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
@@ -1180,10 +1189,12 @@ DualProb dual_prob(int M, int N, int K, int split, float* C, int64_t ldc, int bn
     q.tiles_m = (M + TC_BM - 1) / TC_BM; q.tiles_n = (N + bn - 1) / bn;
     q.items = q.tiles_m * q.tiles_n * ((q.kb_total + q.kb_per_split - 1) / q.kb_per_split);
     q.C = C; q.ldc = ldc; q.split_stride = (int64_t)M * ldc;
+    q.seg_kb = q.kb_total; q.a_seg_x = 0; q.fold = 0; q.fold_stride = 0;
     return q;
 }
 template <int BN>
-cudaError_t launch_gemm_dual(kge_handle* h, const DualProb& q0, const DualProb& q1, cudaStream_t s) {
+cudaError_t launch_gemm_dual(kge_handle* h, const unsigned char* tmA0, const unsigned char* tmB0, const unsigned char* tmA1,
+                             const unsigned char* tmB1, const DualProb& q0, const DualProb& q1, cudaStream_t s) {
     constexpr size_t smem = tc_smem_bytes(BN);
     static DeviceOnce configured;
     const cudaError_t e = once_per_device(configured, [] {
@@ -1195,8 +1206,8 @@ cudaError_t launch_gemm_dual(kge_handle* h, const DualProb& q0, const DualProb& 
     const int rounds = (total + h->num_sms - 1) / h->num_sms;
     const int grid = (total + rounds - 1) / rounds;
     tc_gemm_dual_kernel<BN><<<grid, 32 * (2 + TC_EPI_WARPS), smem, s>>>(
-        *reinterpret_cast<const CUtensorMap*>(h->tm_g), *reinterpret_cast<const CUtensorMap*>(h->tm_t64),
-        *reinterpret_cast<const CUtensorMap*>(h->tm_g64), *reinterpret_cast<const CUtensorMap*>(h->tm_q64), q0, q1, h->ws.status, h->wait_limit);
+        *reinterpret_cast<const CUtensorMap*>(tmA0), *reinterpret_cast<const CUtensorMap*>(tmB0),
+        *reinterpret_cast<const CUtensorMap*>(tmA1), *reinterpret_cast<const CUtensorMap*>(tmB1), q0, q1, h->ws.status, h->wait_limit);
     return cudaSuccess;
 }
 }  // namespace
@@ -1250,8 +1261,36 @@ int launch_tc_backward(kge_handle* h, cudaStream_t s, cudaStream_t side) {
     const int bn = tc_backward_tile_cols(d);
     const DualProb q0 = dual_prob(B, d, N, h->split_q, w.dQpart, d, bn), q1 = dual_prob(N, d, B, h->split_t, dT_out, d, bn);
     stage_begin(h, ST_ACCUM_Q, s);        // (both contractions: the profile reports them as one stage)
-    KGE_CUDA_CHECK(h, bn == 256 ? launch_gemm_dual<256>(h, q0, q1, s) : launch_gemm_dual<128>(h, q0, q1, s));
+    KGE_CUDA_CHECK(h, bn == 256 ? launch_gemm_dual<256>(h, h->tm_g, h->tm_t64, h->tm_g64, h->tm_q64, q0, q1, s)
+                                : launch_gemm_dual<128>(h, h->tm_g, h->tm_t64, h->tm_g64, h->tm_q64, q0, q1, s));
     stage_end(h, ST_ACCUM_Q, s);
+    KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
+}
+
+// TransH on the fp32 path: the two contractions of the backward whose coefficient is one number per pair,
+//   dW_b += sum_n c_bn t_n      and      dT_n += sum_b c_bn w_b,
+// from bf16 two-term splits x = x1 + x2 of all three operands.  With the splits side by side, [c1 | c2] over K and
+// [x1 | x2] over the output columns, one pass forms c1 x1 + c2 x1 in the left half of a tile and c1 x2 + c2 x2 in
+// the right half: all four products, accumulated in fp32; the halves (and the K splits) land in slabs of their own
+// behind the CUDA-core kernels' slabs and the chain kernel adds them in order.
+int th_contract_slabs(const kge_handle* h) { return h->th_tc ? 2 * h->th_gsplit : 0; }
+
+int launch_th_contract_gemm(kge_handle* h, cudaStream_t s) {
+    const kge_config& c = h->cfg;
+    Workspace& w = h->ws;
+    const int B = c.batch, N = c.num_neg, d = c.dim;
+    const int Np = (N + 63) / 64 * 64, Bp = (B + 63) / 64 * 64;
+    const int bn = tc_backward_tile_cols(2 * d);
+    DualProb q0 = dual_prob(B, 2 * d, 2 * Np, h->th_gsplit, w.dWpart + (size_t)h->split_q * B * d, d, bn);
+    DualProb q1 = dual_prob(N, 2 * d, 2 * Bp, h->th_gsplit, w.dTpart + (size_t)h->split_t * N * d, d, bn);
+    q0.seg_kb = Np / TC_BK; q0.a_seg_x = 0;
+    q1.seg_kb = Bp / TC_BK; q1.a_seg_x = Np;
+    q0.fold = q1.fold = d;
+    q0.fold_stride = (int64_t)B * d; q0.split_stride = 2 * q0.fold_stride;
+    q1.fold_stride = (int64_t)N * d; q1.split_stride = 2 * q1.fold_stride;
+    KGE_CUDA_CHECK(h, bn == 256 ? launch_gemm_dual<256>(h, h->tm_cs, h->tm_ts64, h->tm_cs64, h->tm_ws64, q0, q1, s)
+                                : launch_gemm_dual<128>(h, h->tm_cs, h->tm_ts64, h->tm_cs64, h->tm_ws64, q0, q1, s));
     KGE_LAUNCH_CHECK(h);
     return KGE_OK;
 }

@@ -20,6 +20,7 @@ struct TrainParams {
     const float *ent, *rel, *relw;
     const int32_t *heads, *rels, *tails, *negs;
     int split_q, split_t;
+    int th_slabs;          // TransH: slabs the tensor-core contractions append to dWpart and dTpart
     float* loss_out;    // caller's device scalar for the batch loss, or NULL
     int fused_sample;   // the gather kernel draws the batch itself (ids land in sp.heads ...) instead of reading it
     int slots_per_bucket;
@@ -909,7 +910,7 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
         if (p.kind == KIND_L1) wsum = sum_splits(p.w.Cpart + n, p.N, p.split_t);
         const float creg = p.w.reg_s3 ? reg_coef(p.reg_lambda, p.reg_form, p.w.reg_s3[2 * p.B + n]) : 0.f;
         for (int c = lane; c < d4; c += 32) {
-            float4 s = sum_splits(part + (int64_t)n * d4 + c, (int64_t)p.N * d4, p.split_t);
+            float4 s = sum_splits(part + (int64_t)n * d4 + c, (int64_t)p.N * d4, p.split_t + p.th_slabs);
             if (p.kind == KIND_L1) s = make_float4(2.f * s.x - wsum, 2.f * s.y - wsum, 2.f * s.z - wsum, 2.f * s.w - wsum);
             if (p.tc_l2) {   // dT_n = sum_b C_bn (q_b - t_n) = (C^T Q)_n - (column sum of C) t_n
                 const float cs = p.w.Gcol[n];
@@ -971,7 +972,7 @@ __global__ void __launch_bounds__(256) chain_kernel(TrainParams p) {
             const float4 wraw = in ? wrow[c] : f4zero();
             nrm2 += f4dot(wraw, wraw);
             float4 s = f4zero();
-            if (in) s = sum_splits(reinterpret_cast<const float4*>(p.w.dWpart) + (int64_t)b * d4 + c, (int64_t)p.B * d4, p.split_q);
+            if (in) s = sum_splits(reinterpret_cast<const float4*>(p.w.dWpart) + (int64_t)b * d4 + c, (int64_t)p.B * d4, p.split_q + p.th_slabs);
             dwh[i] = s;
             u += f4dot(wh[i], t[i]); a += f4dot(wh[i], h[i]);
         }
@@ -1148,6 +1149,7 @@ int launch_forward_backward(kge_handle* h, const int32_t* heads, const int32_t* 
     p.ent = h->ent; p.rel = h->rel; p.relw = h->relw;
     p.heads = heads; p.rels = rels; p.tails = tails; p.negs = negs;
     p.split_q = h->split_q; p.split_t = h->split_t;
+    p.th_slabs = th_contract_slabs(h);
     p.loss_out = loss_out;
     p.fused_sample = fused_sample ? 1 : 0;
     p.sp = make_sample_params(h, step);

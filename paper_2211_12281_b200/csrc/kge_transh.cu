@@ -18,14 +18,20 @@
 //             Rows wider than 128 floats are cut into column slabs (blockIdx.z): given the
 //             per-pair numbers every coordinate is independent of the others.
 // Per element: 6 instructions forward (5 without the u sweep), 5 for the query side, 4 for the
-// negatives' side.
+// negatives' side.  Two of the backward's sums, sum_n c_bn t_n and sum_b c_bn w_b with
+// c = -dL/dF . c', are plain contractions with one coefficient per pair: with TCC they leave these
+// kernels (4 and 3 instructions per element) and run on the tensor cores from bf16 two-term splits
+// that the query-side kernel (c) and a small row kernel (t, w) write.
 #include "kge_common.cuh"
+#include <cuda_bf16.h>
 
 namespace kge {
 
 namespace {
 
 __device__ __forceinline__ float4 f4z() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+// acc += w where a > b: a compare into a predicate and a predicated add.  (A float mask, set.gt giving 1.0 or 0.0,
+// times w in a multiply-add is the same count without the predicate registers and was measured 5-16 % slower.)
 __device__ __forceinline__ void add_if_gt(float& acc, float a, float b, float w) {
     asm("{\n .reg .pred p;\n setp.gt.f32 p, %1, %2;\n @p add.f32 %0, %0, %3;\n}\n" : "+f"(acc) : "f"(a), "f"(b), "f"(w));
 }
@@ -199,23 +205,29 @@ struct ThAccArgs {
     const float *G, *U, *Cp;    // [B, N]: dL/dF (divided by the distance for p = 2), w.t, c'
     int own_rows, oth_rows, N, d, split;
     float *out, *out2;          // [split, own_rows, d]; out2: gradient of the unit normal (owner = queries)
+    uint16_t* Csb;              // TCC, owner = queries: bf16 splits of c, [B, 2 ldc2] = [c1 | c2]
+    int ldc2;                   // N rounded up to 64
     int32_t* status;
     int wait_limit;
 };
 
-template <bool OWNER_Q>
+// weight tiles of a chunk: g, u, then c (unless it goes to the tensor cores), then u g (query side)
+__host__ __device__ constexpr int ha_tiles(bool owner_q, bool tcc) { return 2 + (tcc ? 0 : 1) + (owner_q ? 1 : 0); }
+template <bool OWNER_Q, bool TCC>
 inline size_t ha_smem() {
-    return (size_t)2 * HA_CC * HA_SLAB * 4 * (OWNER_Q ? 1 : 2) + (size_t)2 * HA_CC * HA_LDW * 4 * (OWNER_Q ? 4 : 3) + 2 * sizeof(uint64_t);
+    return (size_t)2 * HA_CC * HA_SLAB * 4 * (OWNER_Q ? 1 : 2) + (size_t)2 * HA_CC * HA_LDW * 4 * ha_tiles(OWNER_Q, TCC) + 2 * sizeof(uint64_t);
 }
 
 // OWNER_Q: owner rows are queries (own = Q, oth = Tneg); else negatives (own = Tneg, oth = Q, whose normals come along).
 // The sums run over the other side's rows in ascending order inside a split; the chain kernel adds the splits in order.
 // FULL_SLAB: every column slab is HA_SLAB floats wide (d a multiple of HA_SLAB), so the row stride
 // of the staged rows is a compile-time constant.
-template <bool P1, bool OWNER_Q, bool FULL_SLAB>
+// TCC: the sums with coefficient c are left to the tensor cores; the query side writes c's bf16 splits on its way.
+template <bool P1, bool OWNER_Q, bool FULL_SLAB, bool TCC>
 __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
     extern __shared__ __align__(128) unsigned char smraw[];
-    constexpr int NT = OWNER_Q ? 4 : 3;                      // weight tiles: g, u, c (and u g for the query side)
+    constexpr int NT = ha_tiles(OWNER_Q, TCC);
+    constexpr int TI_C = 2, TI_UG = TCC ? 2 : 3;             // tile indices behind g (0) and u (1)
     const int k0 = blockIdx.z * HA_SLAB, kc = FULL_SLAB ? HA_SLAB : min(HA_SLAB, a.d - k0), d4s = kc >> 2;
     float4* Bs = reinterpret_cast<float4*>(smraw);                                   // [2][32][d4s] rows of the other side
     float4* Ws = Bs + 2 * HA_CC * (HA_SLAB / 4);                                     // [2][32][d4s] their normals (owner = negatives)
@@ -262,23 +274,34 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
             if (OWNER_Q) { cc = idx & 31; rr = idx >> 5; g = (int64_t)(r0 + rr) * a.N + (c0 + cc); }
             else         { rr = idx & 31; cc = idx >> 5; g = (int64_t)(c0 + cc) * a.N + (r0 + rr); }
             const bool in = (r0 + rr) < a.own_rows && (c0 + cc) < c_end;
-            greg[e] = in ? a.G[g] : 0.f; ureg[e] = in ? a.U[g] : 0.f; creg[e] = in ? a.Cp[g] : 0.f;
+            greg[e] = in ? a.G[g] : 0.f; ureg[e] = in ? a.U[g] : 0.f;
+            if (!TCC || OWNER_Q) creg[e] = in ? a.Cp[g] : 0.f;
         }
     };
-    auto store_weights = [&](int buf) {
+    auto store_weights = [&](int chunk, int buf) {
         float* T0 = Tl + (size_t)buf * NT * HA_CC * HA_LDW;
+        const int c0 = c_begin + chunk * HA_CC;
 #pragma unroll
         for (int e = 0; e < HA_WPT; ++e) {
             const int rr = OWNER_Q ? warp + HA_WARPS * e : lane, cc = OWNER_Q ? lane : warp + HA_WARPS * e;
             const int o = cc * HA_LDW + rr;
             T0[o] = greg[e];
             T0[HA_CC * HA_LDW + o] = ureg[e];
-            T0[2 * HA_CC * HA_LDW + o] = -greg[e] * creg[e];                  // c_bn = -dL/dF . c'
-            if (OWNER_Q) T0[3 * HA_CC * HA_LDW + o] = ureg[e] * greg[e];
+            if (!TCC) T0[TI_C * HA_CC * HA_LDW + o] = -greg[e] * creg[e];     // c_bn = -dL/dF . c'
+            if (OWNER_Q) T0[TI_UG * HA_CC * HA_LDW + o] = ureg[e] * greg[e];
+            if (TCC && OWNER_Q && blockIdx.z == 0 && (r0 + rr) < a.own_rows && (c0 + cc) < c_end) {
+                // every pair passes here exactly once (in the first column slab): c = c1 + c2, two bf16 numbers
+                const float c = -greg[e] * creg[e];
+                const __nv_bfloat16 c1 = __float2bfloat16_rn(c), c2 = __float2bfloat16_rn(c - __bfloat162float(c1));
+                uint16_t* dst = a.Csb + (int64_t)(r0 + rr) * (2 * a.ldc2) + (c0 + cc);
+                dst[0] = __bfloat16_as_ushort(c1);
+                dst[a.ldc2] = __bfloat16_as_ushort(c2);
+            }
         }
     };
 
     const bool act = lane < d4s;
+    // accumulators: acc; acc2 = the c sums (without TCC) or, for p = 2 on the query side, -sum u g x; acc3 = P weighted by u g (p = 1, query side)
     float4 A[HA_RPW], Wn[OWNER_Q ? HA_RPW : 1], acc[HA_RPW], acc2[HA_RPW], acc3[OWNER_Q ? HA_RPW : 1];
 #pragma unroll
     for (int i = 0; i < HA_RPW; ++i) {
@@ -295,7 +318,7 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
     if (nchunk > 0) {
         if (warp == 0) issue_rows(0, 0);
         load_weights(0);
-        store_weights(0);
+        store_weights(0, 0);
     }
     __syncthreads();
     for (int chunk = 0; chunk < nchunk; ++chunk) {
@@ -316,8 +339,8 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
         const float4* Wc = Ws + (size_t)cur * HA_CC * d4s;
         const float* Gc = Tl + (size_t)cur * NT * HA_CC * HA_LDW;
         const float* Uc = Gc + HA_CC * HA_LDW;
-        const float* Cc = Uc + HA_CC * HA_LDW;
-        const float* UGc = Cc + HA_CC * HA_LDW;
+        const float* Cc = Gc + TI_C * HA_CC * HA_LDW;       // (not read with TCC)
+        const float* UGc = Gc + TI_UG * HA_CC * HA_LDW;
         if (P1) {   // lane l adds the weights of the chunk's row l (rows beyond the chunk hold zeros)
             const float4 g4 = *reinterpret_cast<const float4*>(&Gc[lane * HA_LDW + warp * HA_RPW]);
             sg[0] += g4.x; sg[1] += g4.y; sg[2] += g4.z; sg[3] += g4.w;
@@ -335,7 +358,7 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
                 static_assert(HA_RPW == 4, "one float4 of each weight tile per warp");
                 const float4 g4 = *reinterpret_cast<const float4*>(&Gc[cc * HA_LDW + warp * HA_RPW]);
                 const float4 u4 = *reinterpret_cast<const float4*>(&Uc[cc * HA_LDW + warp * HA_RPW]);
-                const float4 c4 = *reinterpret_cast<const float4*>(&Cc[cc * HA_LDW + warp * HA_RPW]);
+                const float4 c4 = TCC ? f4z() : *reinterpret_cast<const float4*>(&Cc[cc * HA_LDW + warp * HA_RPW]);
                 const float gw[4] = {g4.x, g4.y, g4.z, g4.w}, uw[4] = {u4.x, u4.y, u4.z, u4.w}, cw[4] = {c4.x, c4.y, c4.z, c4.w};
                 const float4 bv = Bc[cc * d4s + lane];
                 if (OWNER_Q) {       // own = q_b (A) with normal Wn; other = t_n (bv)
@@ -348,14 +371,21 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
                         if (P1) {    // acc = P (weights g), acc3 = P (weights u g), acc2 = sum of c t
                             add2_if_gt(acc[i].x, acc3[i].x, thr.x, bv.x, gw[i], ugw[i]); add2_if_gt(acc[i].y, acc3[i].y, thr.y, bv.y, gw[i], ugw[i]);
                             add2_if_gt(acc[i].z, acc3[i].z, thr.z, bv.z, gw[i], ugw[i]); add2_if_gt(acc[i].w, acc3[i].w, thr.w, bv.w, gw[i], ugw[i]);
-                            acc2[i].x = fmaf(cw[i], bv.x, acc2[i].x); acc2[i].y = fmaf(cw[i], bv.y, acc2[i].y);
-                            acc2[i].z = fmaf(cw[i], bv.z, acc2[i].z); acc2[i].w = fmaf(cw[i], bv.w, acc2[i].w);
+                            if (!TCC) {
+                                acc2[i].x = fmaf(cw[i], bv.x, acc2[i].x); acc2[i].y = fmaf(cw[i], bv.y, acc2[i].y);
+                                acc2[i].z = fmaf(cw[i], bv.z, acc2[i].z); acc2[i].w = fmaf(cw[i], bv.w, acc2[i].w);
+                            }
                         } else {     // acc = -sum g x, acc2 = sum (c t - u g x)
                             const float4 x = make_float4(thr.x - bv.x, thr.y - bv.y, thr.z - bv.z, thr.w - bv.w);
                             acc[i].x = fmaf(-gw[i], x.x, acc[i].x); acc[i].y = fmaf(-gw[i], x.y, acc[i].y);
                             acc[i].z = fmaf(-gw[i], x.z, acc[i].z); acc[i].w = fmaf(-gw[i], x.w, acc[i].w);
-                            acc2[i].x = fmaf(cw[i], bv.x, fmaf(-ugw[i], x.x, acc2[i].x)); acc2[i].y = fmaf(cw[i], bv.y, fmaf(-ugw[i], x.y, acc2[i].y));
-                            acc2[i].z = fmaf(cw[i], bv.z, fmaf(-ugw[i], x.z, acc2[i].z)); acc2[i].w = fmaf(cw[i], bv.w, fmaf(-ugw[i], x.w, acc2[i].w));
+                            if (TCC) {
+                                acc2[i].x = fmaf(-ugw[i], x.x, acc2[i].x); acc2[i].y = fmaf(-ugw[i], x.y, acc2[i].y);
+                                acc2[i].z = fmaf(-ugw[i], x.z, acc2[i].z); acc2[i].w = fmaf(-ugw[i], x.w, acc2[i].w);
+                            } else {
+                                acc2[i].x = fmaf(cw[i], bv.x, fmaf(-ugw[i], x.x, acc2[i].x)); acc2[i].y = fmaf(cw[i], bv.y, fmaf(-ugw[i], x.y, acc2[i].y));
+                                acc2[i].z = fmaf(cw[i], bv.z, fmaf(-ugw[i], x.z, acc2[i].z)); acc2[i].w = fmaf(cw[i], bv.w, fmaf(-ugw[i], x.w, acc2[i].w));
+                            }
                         }
                     }
                 } else {             // own = t_n (A); other = q_b (bv) with its normal wv
@@ -366,8 +396,13 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
                         if (P1) {    // acc = P (weights g), acc2 = sum of c w
                             add_if_gt(acc[i].x, thr.x, A[i].x, gw[i]); add_if_gt(acc[i].y, thr.y, A[i].y, gw[i]);
                             add_if_gt(acc[i].z, thr.z, A[i].z, gw[i]); add_if_gt(acc[i].w, thr.w, A[i].w, gw[i]);
-                            acc2[i].x = fmaf(cw[i], wv.x, acc2[i].x); acc2[i].y = fmaf(cw[i], wv.y, acc2[i].y);
-                            acc2[i].z = fmaf(cw[i], wv.z, acc2[i].z); acc2[i].w = fmaf(cw[i], wv.w, acc2[i].w);
+                            if (!TCC) {
+                                acc2[i].x = fmaf(cw[i], wv.x, acc2[i].x); acc2[i].y = fmaf(cw[i], wv.y, acc2[i].y);
+                                acc2[i].z = fmaf(cw[i], wv.z, acc2[i].z); acc2[i].w = fmaf(cw[i], wv.w, acc2[i].w);
+                            }
+                        } else if (TCC) {   // acc = sum g x
+                            acc[i].x = fmaf(gw[i], thr.x - A[i].x, acc[i].x); acc[i].y = fmaf(gw[i], thr.y - A[i].y, acc[i].y);
+                            acc[i].z = fmaf(gw[i], thr.z - A[i].z, acc[i].z); acc[i].w = fmaf(gw[i], thr.w - A[i].w, acc[i].w);
                         } else {     // acc = sum (g x + c w)
                             acc[i].x = fmaf(cw[i], wv.x, fmaf(gw[i], thr.x - A[i].x, acc[i].x)); acc[i].y = fmaf(cw[i], wv.y, fmaf(gw[i], thr.y - A[i].y, acc[i].y));
                             acc[i].z = fmaf(cw[i], wv.z, fmaf(gw[i], thr.z - A[i].z, acc[i].z)); acc[i].w = fmaf(cw[i], wv.w, fmaf(gw[i], thr.w - A[i].w, acc[i].w));
@@ -376,7 +411,7 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
                 }
             }
         }
-        if (more) store_weights(cur ^ 1);
+        if (more) store_weights(chunk + 1, cur ^ 1);
         __syncthreads();
     }
     if (P1) {
@@ -417,18 +452,39 @@ cudaError_t launch_fwd(const ThFwdParams& p, cudaStream_t s) {
     return launch_dependent(th_block_kernel<P1, 0>, grid, dim3(HB_THREADS), hb_smem(p.d), s, p);
 }
 
-template <bool P1, bool OWNER_Q>
+template <bool P1, bool OWNER_Q, bool TCC>
 cudaError_t launch_acc(const ThAccArgs& a, cudaStream_t s) {
     static DeviceOnce configured;
     const cudaError_t e = once_per_device(configured, [] {
-        const cudaError_t e0 = cudaFuncSetAttribute(th_accum_kernel<P1, OWNER_Q, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ha_smem<OWNER_Q>());
-        return e0 != cudaSuccess ? e0 : cudaFuncSetAttribute(th_accum_kernel<P1, OWNER_Q, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ha_smem<OWNER_Q>());
+        const cudaError_t e0 = cudaFuncSetAttribute(th_accum_kernel<P1, OWNER_Q, true, TCC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ha_smem<OWNER_Q, TCC>());
+        return e0 != cudaSuccess ? e0 : cudaFuncSetAttribute(th_accum_kernel<P1, OWNER_Q, false, TCC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ha_smem<OWNER_Q, TCC>());
     });
     if (e != cudaSuccess) return e;
     dim3 grid((a.own_rows + HA_ROWS - 1) / HA_ROWS, a.split, (a.d + HA_SLAB - 1) / HA_SLAB);
-    if (a.d % HA_SLAB == 0) th_accum_kernel<P1, OWNER_Q, true><<<grid, HA_THREADS, ha_smem<OWNER_Q>(), s>>>(a);
-    else th_accum_kernel<P1, OWNER_Q, false><<<grid, HA_THREADS, ha_smem<OWNER_Q>(), s>>>(a);
+    if (a.d % HA_SLAB == 0) th_accum_kernel<P1, OWNER_Q, true, TCC><<<grid, HA_THREADS, ha_smem<OWNER_Q, TCC>(), s>>>(a);
+    else th_accum_kernel<P1, OWNER_Q, false, TCC><<<grid, HA_THREADS, ha_smem<OWNER_Q, TCC>(), s>>>(a);
     return cudaSuccess;
+}
+template <bool OWNER_Q>
+cudaError_t launch_acc_any(bool p1, bool tcc, const ThAccArgs& a, cudaStream_t s) {
+    if (p1) return tcc ? launch_acc<true, OWNER_Q, true>(a, s) : launch_acc<true, OWNER_Q, false>(a, s);
+    return tcc ? launch_acc<false, OWNER_Q, true>(a, s) : launch_acc<false, OWNER_Q, false>(a, s);
+}
+
+// bf16 two-term splits of the negatives and of the unit normals, [rows, 2d] = [x1 | x2]: the tensor-core
+// contractions' second operands.  One thread per four coordinates.
+__global__ void __launch_bounds__(256) th_split_rows_kernel(const float4* T, int N, const float4* W, int B, int d4, uint2* Ts, uint2* Ws) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (int64_t)(N + B) * d4) return;
+    const int row = (int)(i / d4), c = (int)(i - (int64_t)row * d4);
+    const bool neg = row < N;
+    const float4 v = neg ? T[i] : W[i - (int64_t)N * d4];
+    uint2* dst = (neg ? Ts + (int64_t)row * 2 * d4 : Ws + (int64_t)(row - N) * 2 * d4) + c;
+    const __nv_bfloat162 a1 = __floats2bfloat162_rn(v.x, v.y), b1 = __floats2bfloat162_rn(v.z, v.w);
+    const float2 fa = __bfloat1622float2(a1), fb = __bfloat1622float2(b1);
+    const __nv_bfloat162 a2 = __floats2bfloat162_rn(v.x - fa.x, v.y - fa.y), b2 = __floats2bfloat162_rn(v.z - fb.x, v.w - fb.y);
+    dst[0] = make_uint2(*reinterpret_cast<const uint32_t*>(&a1), *reinterpret_cast<const uint32_t*>(&b1));
+    dst[d4] = make_uint2(*reinterpret_cast<const uint32_t*>(&a2), *reinterpret_cast<const uint32_t*>(&b2));
 }
 
 }  // namespace
@@ -448,16 +504,28 @@ int launch_th_backward(kge_handle* h, cudaStream_t sq, cudaStream_t st) {
     const Workspace& w = h->ws;
     const bool p1 = h->kind == KIND_TH_L1;
     ThAccArgs aq{w.Q, w.Tneg, w.What, w.F, w.U, w.Cc, c.batch, c.num_neg, c.num_neg, c.dim, h->split_q, w.dQpart, w.dWpart,
-                 w.status, h->wait_limit};
+                 w.Csb, (c.num_neg + 63) / 64 * 64, w.status, h->wait_limit};
     ThAccArgs at = aq;
     at.own = w.Tneg; at.oth = w.Q; at.own_rows = c.num_neg; at.oth_rows = c.batch; at.split = h->split_t;
     at.out = w.dTpart; at.out2 = nullptr;
-    stage_begin(h, ST_ACCUM_Q, sq);
-    KGE_CUDA_CHECK(h, p1 ? (launch_acc<true, true>(aq, sq)) : (launch_acc<false, true>(aq, sq)));
-    stage_end(h, ST_ACCUM_Q, sq);
+    const bool tcc = h->th_tc;
+    stage_begin(h, ST_ACCUM_Q, sq);       // (with the tensor-core contractions: their operands' splits, the query side, both contractions)
+    if (tcc) {
+        const int64_t n4 = (int64_t)(c.num_neg + c.batch) * (c.dim / 4);
+        th_split_rows_kernel<<<(int)((n4 + 255) / 256), 256, 0, sq>>>(reinterpret_cast<const float4*>(w.Tneg), c.num_neg,
+                                                                     reinterpret_cast<const float4*>(w.What), c.batch, c.dim / 4,
+                                                                     reinterpret_cast<uint2*>(w.Tsb), reinterpret_cast<uint2*>(w.Wsb));
+        KGE_LAUNCH_CHECK(h);
+    }
+    KGE_CUDA_CHECK(h, launch_acc_any<true>(p1, tcc, aq, sq));
     KGE_LAUNCH_CHECK(h);
+    if (tcc) {
+        const int rc = launch_th_contract_gemm(h, sq);
+        if (rc != KGE_OK) return rc;
+    }
+    stage_end(h, ST_ACCUM_Q, sq);
     stage_begin(h, ST_ACCUM_T, st);
-    KGE_CUDA_CHECK(h, p1 ? (launch_acc<true, false>(at, st)) : (launch_acc<false, false>(at, st)));
+    KGE_CUDA_CHECK(h, launch_acc_any<false>(p1, tcc, at, st));
     stage_end(h, ST_ACCUM_T, st);
     KGE_LAUNCH_CHECK(h);
     return KGE_OK;

@@ -28,11 +28,11 @@ class Problem:
 
     def __init__(self, *, E, R, T, d, score, p_norm=1, loss="logsigmoid", opt="sgd", B, N, P,
                  gamma=0.0, adv_temp=0.0, ce_correction=0.0, loss_scale=1.0, lr=0.1, head_part=-1,
-                 sample_mode=0, seed=0, graph_seed=0, relation_zipf=0.0, eps=None, tc=False, reg_lambda=0.0, reg_form=0):
+                 sample_mode=0, seed=0, graph_seed=0, relation_zipf=0.0, eps=None, tc=False, reg_lambda=0.0, reg_form=0, contract=0):
         self.kw = dict(num_entities=E, num_relations=R, dim=d, score=score, p_norm=p_norm, loss=loss, opt=opt,
                        batch=B, num_neg=N, num_parts=P, gamma=gamma, adv_temp=adv_temp,
                        ce_correction=ce_correction, loss_scale=loss_scale, lr=lr, head_part=head_part,
-                       sample_mode=sample_mode, seed=seed, eps=eps, reg_lambda=reg_lambda, reg_form=reg_form)
+                       sample_mode=sample_mode, seed=seed, eps=eps, reg_lambda=reg_lambda, reg_form=reg_form, contract=contract)
         self.E, self.R, self.T, self.d, self.B, self.N, self.P = E, R, T, d, B, N, P
         self.score, self.opt, self.lr = score, opt, lr
         self.tc = tc      # bf16 tensor-core score block on the GPU, bf16-rounded operands in the oracle
@@ -44,7 +44,7 @@ class Problem:
         return self.d // 2 if self.score in ("rotate", "rotate_real_l1") else self.d
 
     def oracle_cfg(self):
-        kw = {k: v for k, v in self.kw.items() if k not in ("feat_dim", "feat_shared")}     # (the oracle's encoder takes them as arguments)
+        kw = {k: v for k, v in self.kw.items() if k not in ("feat_dim", "feat_shared", "contract")}     # (the oracle's encoder takes them as arguments; where a contraction runs is the library's business)
         return oracle_config(**kw, bf16_operands=1 if self.tc else 0)
 
     def state_shapes(self):

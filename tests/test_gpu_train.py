@@ -310,6 +310,18 @@ def test_transh_l1_row_widths(oracle64, d):
     _run(oracle64, prob, steps=1)
 
 
+@pytest.mark.parametrize("p,d,B,N", [(1, 128, 96, 80), (2, 128, 200, 300), (1, 128, 1024, 1024), (1, 256, 132, 200), (2, 96, 64, 130),
+                                     (1, 64, 260, 64)])
+def test_transh_tensor_core_contractions(oracle64, p, d, B, N):
+    """TransH on the fp32 path with the backward's two contractions with per-pair coefficients forced onto the
+    tensor cores (bf16 two-term splits, all four products): the fp32 tolerances hold.  Shapes: a single ragged
+    tile; ragged rows and columns; four K splits; rows of two 128-float slabs (two column tiles); a row width that
+    leaves the tile's last 64 columns outside the operand; 128-column tiles."""
+    prob = Problem(E=3000, R=6, T=30000, d=d, score="transh", p_norm=p, loss="logsigmoid", B=B, N=N, P=2,
+                   gamma=6.0, adv_temp=0.5, lr=0.05, graph_seed=21, relation_zipf=1.0, contract=1)
+    _run(oracle64, prob, steps=2)
+
+
 @pytest.mark.parametrize("score,p", [("distmult", 1), ("complex", 1), ("transe", 2)])
 @pytest.mark.parametrize("d", [64, 192, 256])
 def test_tensor_core_score_block(oracle64, score, p, d):
