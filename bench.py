@@ -118,7 +118,20 @@ STAGE_OPS = {
     "transh1": dict(block=[(2, MIX_FMA), (2, MIX_SUB_ABS), (2, MIX_CMP_ADD)],
                     accum_q=[(2, MIX_FMA), (3, MIX_CMP_ADD)], accum_t=[(2, MIX_FMA), (2, MIX_CMP_ADD)]),
     "transh2": dict(block=[(5, MIX_FMA)], accum_q=[(5, MIX_FMA)], accum_t=[(4, MIX_FMA)]),
+    # TransH with its three dense contractions (u = w.t forward; sum_n c t and sum_b c w backward) on the tensor cores:
+    # one multiply-add per element less in each CUDA-core kernel; the contractions are stages of their own
+    # ("th_u", "th_contract"), counted at their algorithmic 2 B N d flops each against the bf16 peak (the bf16 splits
+    # that give them fp32 accuracy multiply the executed flops by 6 and by 4: implementation cost, not algorithmic work).
+    "transh1_tc": dict(block=[(1, MIX_FMA), (2, MIX_SUB_ABS), (2, MIX_CMP_ADD)],
+                       accum_q=[(1, MIX_FMA), (3, MIX_CMP_ADD)], accum_t=[(1, MIX_FMA), (2, MIX_CMP_ADD)]),
+    "transh2_tc": dict(block=[(4, MIX_FMA)], accum_q=[(4, MIX_FMA)], accum_t=[(3, MIX_FMA)]),
 }
+TH_TC_CONTRACTIONS = {"th_u": 1, "th_contract": 2}
+
+
+def transh_on_tensor_cores(w):
+    """The library's automatic choice (config field `contract` = 0) for TransH with fp32 arithmetic."""
+    return w["score"] == "transh" and not w.get("tc") and w["d"] % 32 == 0 and w["B"] * w["N"] >= 1 << 22
 
 # Special-function instructions per score of the fused tensor-core epilogues (exponential, logarithm, reciprocal, reciprocal
 # square root: one instruction each).
@@ -512,7 +525,7 @@ def bench_training(ctx, name, w, cpu_seconds):
     kge.profile(False)
     uniq = len(kge.debug_export("ENT_UNIQ"))
     per_stage_us = {k: 1e3 * v[0] / v[1] for k, v in stages.items() if v[1] > 0}
-    kind = f"{w['score']}{w['p_norm']}"
+    kind = f"{w['score']}{w['p_norm']}" + ("_tc" if transh_on_tensor_cores(w) else "")
     ops = dict(STAGE_OPS.get(kind, {}))
     if "accum_q" in per_stage_us and "accum_t" not in per_stage_us:     # dQ and dT share one launch
         per_stage_us["accum"] = per_stage_us.pop("accum_q")
@@ -537,6 +550,9 @@ def bench_training(ctx, name, w, cpu_seconds):
             if st in per_stage_us:
                 t, mix = stage_roof_us(o, elements, ctx.alu)
                 roofs[st] = (t, "alu", {"mix": MIX_NAMES[mix], "instructions_per_element": sum(n for n, _ in o)})
+        for st, ncon in TH_TC_CONTRACTIONS.items():
+            if st in per_stage_us:
+                roofs[st] = (ncon * 2.0 * elements / (ctx.peaks["bf16_tflops"] * 1e12) * 1e6, "tensor", {})
     # the two memory-bound sub-steps: random row gathers and the sparse row update
     rel_bytes = B * 4 * kw_rel * (2 if w["score"] == "transh" else 1)
     build_bytes = (2 * B + N) * 4 * d + rel_bytes + (B + N) * 4 * d + ((B + N) * 2 * d if w.get("tc") else 0)

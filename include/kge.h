@@ -377,9 +377,12 @@ int64_t kge_launch_count(const kge_handle* h);
  * ([host] arrays), stages in the order of kge_stage_t; reset != 0 clears them.
  */
 typedef enum {
-    KGE_STAGE_SAMPLE = 0, KGE_STAGE_BUILD, KGE_STAGE_BLOCK, KGE_STAGE_LOSS, KGE_STAGE_TH_CPASS,
+    KGE_STAGE_SAMPLE = 0, KGE_STAGE_BUILD, KGE_STAGE_BLOCK, KGE_STAGE_LOSS,
+    KGE_STAGE_TH_U,          /* TransH with tensor-core contractions: u = w.t (operand splits + contraction) */
     KGE_STAGE_ACCUM_Q, KGE_STAGE_ACCUM_T, KGE_STAGE_CHAIN, KGE_STAGE_RANK, KGE_STAGE_SEGMENT,
-    KGE_STAGE_UPDATE, KGE_NUM_STAGES
+    KGE_STAGE_UPDATE,
+    KGE_STAGE_TH_CONTRACT,   /* the same: sum_n c_bn t_n and sum_b c_bn w_b (operand splits + both contractions) */
+    KGE_NUM_STAGES
 } kge_stage_t;
 int kge_profile(kge_handle* h, int enable);
 int kge_profile_read(kge_handle* h, double* ms /*[host]*/, int64_t* launches /*[host]*/, int reset);

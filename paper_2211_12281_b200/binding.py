@@ -355,8 +355,8 @@ class Kge:
     def launch_count(self) -> int:
         return int(lib().kge_launch_count(self._h))
 
-    STAGES = ("sample", "build", "block", "loss", "th_cpass", "accum_q", "accum_t", "chain", "rank",
-              "segment", "update")
+    STAGES = ("sample", "build", "block", "loss", "th_u", "accum_q", "accum_t", "chain", "rank",
+              "segment", "update", "th_contract")
 
     def profile(self, enable: bool):
         self._check(lib().kge_profile(self._h, int(enable)), "kge_profile")

@@ -1221,9 +1221,11 @@ int launch_tc_gemm_nt(kge_handle* h, const unsigned char* tmA, const unsigned ch
     p.kb_per_split = (K + TC_BK - 1) / TC_BK;
     p.C = C; p.ldc = ldc; p.split_stride = 0;
     p.status = h->ws.status; p.wait_limit = h->wait_limit;
-    p.bn = TC_BN;
+    // 256-column tiles halve the operand bytes fetched per output once there are enough of them for every SM
+    p.bn = (N >= 1024 && (int64_t)((M + TC_BM - 1) / TC_BM) * ((N + 255) / 256) >= h->num_sms) ? 256 : TC_BN;
     p.tiles_m = (M + TC_BM - 1) / TC_BM; p.tiles_n = (N + p.bn - 1) / p.bn; p.items = p.tiles_m * p.tiles_n;
-    KGE_CUDA_CHECK(h, (launch_gemm_inst<EPI_STORE, 128>(tmA, tmB, p, h->num_sms, s)));
+    if (p.bn == 256) KGE_CUDA_CHECK(h, (launch_gemm_inst<EPI_STORE, 256>(tmA, tmB, p, h->num_sms, s)));
+    else KGE_CUDA_CHECK(h, (launch_gemm_inst<EPI_STORE, 128>(tmA, tmB, p, h->num_sms, s)));
     KGE_LAUNCH_CHECK(h);
     return KGE_OK;
 }

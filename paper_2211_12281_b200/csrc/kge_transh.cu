@@ -61,12 +61,14 @@ inline size_t hb_smem(int d) { return (size_t)hb_stages(d) * HB_ROWS * (hb_kc(d)
 // KC: the chunk length when it is known at compile time (rows of at least HB_KC floats), so that
 // every shared-memory address of the inner loops is one base per operand plus a constant; 0: rows
 // shorter than HB_KC, chunk length = row length.
-template <bool P1, int KC>
+// UEXT: u = w.t is already in p.U (a tensor-core contraction wrote it): one sweep instead of two.
+template <bool P1, int KC, bool UEXT>
 __global__ void __launch_bounds__(HB_THREADS, 2) th_block_kernel(ThFwdParams p) {
     extern __shared__ __align__(128) unsigned char smraw[];
     const int kc = KC ? KC : hb_kc(p.d), ld = kc + 4, nstage = hb_stages(p.d);
     const int nchunk = (p.d + kc - 1) / kc;
-    const int nload = nchunk > 1 ? 2 * nchunk : 1;       // both sweeps read every chunk; a single chunk stays where it is
+    constexpr int SWEEP0 = UEXT ? 1 : 0;
+    const int nload = nchunk > 1 ? (2 - SWEEP0) * nchunk : 1;   // every sweep reads every chunk; a single chunk stays where it is
     float* base = reinterpret_cast<float*>(smraw);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smraw + (size_t)nstage * HB_ROWS * ld * sizeof(float));
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
@@ -104,11 +106,17 @@ __global__ void __launch_bounds__(HB_THREADS, 2) th_block_kernel(ThFwdParams p) 
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) { acc[i][j] = 0.f; u[i][j] = 0.f; cw[i][j] = 0.f; }
+        for (int j = 0; j < 4; ++j) {
+            acc[i][j] = 0.f; cw[i][j] = 0.f; u[i][j] = 0.f;
+            if (UEXT) {
+                const int b = b0 + ty + 16 * i, n = n0 + tx + 16 * j;
+                if (b < p.B && n < p.N) u[i][j] = p.U[(int64_t)b * p.N + n];
+            }
+        }
 
-    for (int sweep = 0; sweep < 2; ++sweep) {
+    for (int sweep = SWEEP0; sweep < 2; ++sweep) {
         for (int chunk = 0; chunk < nchunk; ++chunk) {
-            const int load = nchunk > 1 ? sweep * nchunk + chunk : 0;
+            const int load = nchunk > 1 ? (sweep - SWEEP0) * nchunk + chunk : 0;
             const int stage = load % nstage;
             const bool ok = mbar_wait_bounded(&bars[stage], (uint32_t)(load / nstage) & 1u, p.wait_limit);
             if (!__syncthreads_and(ok)) {
@@ -186,7 +194,7 @@ __global__ void __launch_bounds__(HB_THREADS, 2) th_block_kernel(ThFwdParams p) 
             if (n >= p.N) continue;
             const int64_t o = (int64_t)b * p.N + n;
             p.F[o] = P1 ? -acc[i][j] : -sqrtf(acc[i][j]);
-            p.U[o] = u[i][j];
+            if (!UEXT) p.U[o] = u[i][j];
             p.Cp[o] = P1 ? 2.f * cw[i][j] - ws : cw[i][j];     // p = 1: cw holds the normal's coordinates summed where x > 0
         }
     }
@@ -439,17 +447,45 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
     }
 }
 
-template <bool P1>
+template <bool P1, bool UEXT>
 cudaError_t launch_fwd(const ThFwdParams& p, cudaStream_t s) {
     static DeviceOnce configured;
     const cudaError_t e = once_per_device(configured, [] {
-        const cudaError_t e0 = cudaFuncSetAttribute(th_block_kernel<P1, HB_KC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hb_smem(kMaxDim));
-        return e0 != cudaSuccess ? e0 : cudaFuncSetAttribute(th_block_kernel<P1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hb_smem(HB_KC));
+        const cudaError_t e0 = cudaFuncSetAttribute(th_block_kernel<P1, HB_KC, UEXT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hb_smem(kMaxDim));
+        return e0 != cudaSuccess ? e0 : cudaFuncSetAttribute(th_block_kernel<P1, 0, UEXT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hb_smem(HB_KC));
     });
     if (e != cudaSuccess) return e;
     dim3 grid((p.N + HB_T - 1) / HB_T, (p.B + HB_Q - 1) / HB_Q);
-    if (p.d >= HB_KC) return launch_dependent(th_block_kernel<P1, HB_KC>, grid, dim3(HB_THREADS), hb_smem(p.d), s, p);
-    return launch_dependent(th_block_kernel<P1, 0>, grid, dim3(HB_THREADS), hb_smem(p.d), s, p);
+    if (p.d >= HB_KC) return launch_dependent(th_block_kernel<P1, HB_KC, UEXT>, grid, dim3(HB_THREADS), hb_smem(p.d), s, p);
+    return launch_dependent(th_block_kernel<P1, 0, UEXT>, grid, dim3(HB_THREADS), hb_smem(p.d), s, p);
+}
+
+// bf16 three-term splits x = x1 + x2 + x3 (2^-25 relative) of the unit normals and of the negatives, laid out along K
+// so that one K-major contraction forms the six products that matter:
+//   normals   [B, 6d] = [w1 | w1 | w2 | w1 | w3 | w2]
+//   negatives [N, 6d] = [t1 | t2 | t1 | t3 | t1 | t2]
+// One thread per four coordinates.
+__global__ void __launch_bounds__(256) th_split3_kernel(const float4* W, int B, const float4* T, int N, int d4, uint2* W6, uint2* T6) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (int64_t)(B + N) * d4) return;
+    const int row = (int)(i / d4), c = (int)(i - (int64_t)row * d4);
+    const bool nrm = row < B;
+    const float4 v = nrm ? W[i] : T[i - (int64_t)B * d4];
+    const float x[4] = {v.x, v.y, v.z, v.w};
+    uint16_t t1[4], t2[4], t3[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat16 a = __float2bfloat16_rn(x[e]);
+        const float r1 = x[e] - __bfloat162float(a);
+        const __nv_bfloat16 b = __float2bfloat16_rn(r1);
+        const __nv_bfloat16 cc = __float2bfloat16_rn(r1 - __bfloat162float(b));
+        t1[e] = __bfloat16_as_ushort(a); t2[e] = __bfloat16_as_ushort(b); t3[e] = __bfloat16_as_ushort(cc);
+    }
+    auto pack = [](const uint16_t* t) { return make_uint2((uint32_t)t[0] | ((uint32_t)t[1] << 16), (uint32_t)t[2] | ((uint32_t)t[3] << 16)); };
+    const uint2 p1 = pack(t1), p2 = pack(t2), p3 = pack(t3);
+    uint2* dst = (nrm ? W6 + (int64_t)row * 6 * d4 : T6 + (int64_t)(row - B) * 6 * d4) + c;
+    if (nrm) { dst[0] = p1; dst[d4] = p1; dst[2 * d4] = p2; dst[3 * d4] = p1; dst[4 * d4] = p3; dst[5 * d4] = p2; }
+    else     { dst[0] = p1; dst[d4] = p2; dst[2 * d4] = p1; dst[3 * d4] = p3; dst[4 * d4] = p1; dst[5 * d4] = p2; }
 }
 
 template <bool P1, bool OWNER_Q, bool TCC>
@@ -493,7 +529,23 @@ int launch_th_forward(kge_handle* h, cudaStream_t s) {
     const kge_config& c = h->cfg;
     const Workspace& w = h->ws;
     ThFwdParams p{c.batch, c.num_neg, c.dim, w.Q, w.What, w.Tneg, w.wsum, w.F, w.U, w.Cc, w.status, h->wait_limit};
-    KGE_CUDA_CHECK(h, h->kind == KIND_TH_L1 ? launch_fwd<true>(p, s) : launch_fwd<false>(p, s));
+    const bool p1 = h->kind == KIND_TH_L1;
+    if (h->th_tc) {
+        // u = w.t for all pairs as one tensor-core contraction over the operands' three-term splits
+        stage_begin(h, ST_TH_U, s);
+        const int64_t n4 = (int64_t)(c.batch + c.num_neg) * (c.dim / 4);
+        th_split3_kernel<<<(int)((n4 + 255) / 256), 256, 0, s>>>(reinterpret_cast<const float4*>(w.What), c.batch,
+                                                                 reinterpret_cast<const float4*>(w.Tneg), c.num_neg, c.dim / 4,
+                                                                 reinterpret_cast<uint2*>(w.W6b), reinterpret_cast<uint2*>(w.T6b));
+        KGE_LAUNCH_CHECK(h);
+        const int rc = launch_tc_gemm_nt(h, h->tm_w6, h->tm_t6, c.batch, c.num_neg, 6 * c.dim, w.U, c.num_neg, s);
+        if (rc != KGE_OK) return rc;
+        stage_end(h, ST_TH_U, s);
+        stage_begin(h, ST_BLOCK, s);      // (the caller's bracket opened before the contraction: open it again here)
+        KGE_CUDA_CHECK(h, p1 ? (launch_fwd<true, true>(p, s)) : (launch_fwd<false, true>(p, s)));
+    } else {
+        KGE_CUDA_CHECK(h, p1 ? (launch_fwd<true, false>(p, s)) : (launch_fwd<false, false>(p, s)));
+    }
     KGE_LAUNCH_CHECK(h);
     return KGE_OK;
 }
@@ -509,8 +561,8 @@ int launch_th_backward(kge_handle* h, cudaStream_t sq, cudaStream_t st) {
     at.own = w.Tneg; at.oth = w.Q; at.own_rows = c.num_neg; at.oth_rows = c.batch; at.split = h->split_t;
     at.out = w.dTpart; at.out2 = nullptr;
     const bool tcc = h->th_tc;
-    stage_begin(h, ST_ACCUM_Q, sq);       // (with the tensor-core contractions: their operands' splits, the query side, both contractions)
-    if (tcc) {
+    stage_begin(h, ST_ACCUM_Q, sq);
+    if (tcc) {      // second operands of the contractions (a few microseconds, timed with the query side)
         const int64_t n4 = (int64_t)(c.num_neg + c.batch) * (c.dim / 4);
         th_split_rows_kernel<<<(int)((n4 + 255) / 256), 256, 0, sq>>>(reinterpret_cast<const float4*>(w.Tneg), c.num_neg,
                                                                      reinterpret_cast<const float4*>(w.What), c.batch, c.dim / 4,
@@ -518,12 +570,14 @@ int launch_th_backward(kge_handle* h, cudaStream_t sq, cudaStream_t st) {
         KGE_LAUNCH_CHECK(h);
     }
     KGE_CUDA_CHECK(h, launch_acc_any<true>(p1, tcc, aq, sq));
+    stage_end(h, ST_ACCUM_Q, sq);
     KGE_LAUNCH_CHECK(h);
     if (tcc) {
+        stage_begin(h, ST_TH_CONTRACT, sq);
         const int rc = launch_th_contract_gemm(h, sq);
         if (rc != KGE_OK) return rc;
+        stage_end(h, ST_TH_CONTRACT, sq);
     }
-    stage_end(h, ST_ACCUM_Q, sq);
     stage_begin(h, ST_ACCUM_T, st);
     KGE_CUDA_CHECK(h, launch_acc_any<false>(p1, tcc, at, st));
     stage_end(h, ST_ACCUM_T, st);

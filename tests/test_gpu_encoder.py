@@ -35,7 +35,7 @@ def test_encoder_step_against_oracle(oracle64, score, p, opt, shared, F, d):
     MT_s = MH_s if shared else (None if st_shape is None else torch.zeros(st_shape, dtype=torch.float32, device=dev))
     gpu.kge.bind_features(feat_d, MH_d, MT_d, MH_s, MT_s)
     orc = OracleSide(prob, oracle64)
-    okw = {k: v for k, v in prob.kw.items() if k not in ("feat_dim", "feat_shared")}
+    okw = {k: v for k, v in prob.kw.items() if k not in ("feat_dim", "feat_shared", "contract")}
     from oracle.kge_oracle import make_config
     cfg = make_config(**okw, bf16_projection=1)
     feat64 = feat.float().numpy().astype(np.float64)
