@@ -18,10 +18,16 @@
 //             Rows wider than 128 floats are cut into column slabs (blockIdx.z): given the
 //             per-pair numbers every coordinate is independent of the others.
 // Per element: 6 instructions forward (5 without the u sweep), 5 for the query side, 4 for the
-// negatives' side.  Two of the backward's sums, sum_n c_bn t_n and sum_b c_bn w_b with
-// c = -dL/dF . c', are plain contractions with one coefficient per pair: with TCC they leave these
-// kernels (4 and 3 instructions per element) and run on the tensor cores from bf16 two-term splits
-// that the query-side kernel (c) and a small row kernel (t, w) write.
+// negatives' side.
+//
+// Three pieces of this are dense contractions and run on the tensor cores when the block is
+// large enough (kge_handle::th_tc): u = W T^T forward, and in the backward the two sums whose
+// coefficient is one number per pair, sum_n c_bn t_n and sum_b c_bn w_b with c = -dL/dF . c'.
+// The operands are fp32, so each is split into bf16 terms (x = x1 + x2 + x3 for u, whose error
+// moves the signs of the residuals; two terms for the backward sums) and the products that
+// matter are accumulated in fp32: six for u (2^-25 relative per term), four for the others
+// (2^-17).  The CUDA-core kernels then do 5, 4 and 3 instructions per element: the forward
+// reads u instead of forming it, the query side writes c's split on its way.
 #include "kge_common.cuh"
 #include <cuda_bf16.h>
 
@@ -358,19 +364,23 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
             }
         }
         if (act) {
-            // not unrolled: with two or more iterations in flight the compiler keeps the next
-            // iteration's 20 loaded values in a second register set and copies them over (about
-            // 18 register moves per 80 arithmetic instructions, measured)
-#pragma unroll 1
-            for (int cc = 0; cc < ccmax; ++cc) {
-                static_assert(HA_RPW == 4, "one float4 of each weight tile per warp");
-                const float4 g4 = *reinterpret_cast<const float4*>(&Gc[cc * HA_LDW + warp * HA_RPW]);
-                const float4 u4 = *reinterpret_cast<const float4*>(&Uc[cc * HA_LDW + warp * HA_RPW]);
-                const float4 c4 = TCC ? f4z() : *reinterpret_cast<const float4*>(&Cc[cc * HA_LDW + warp * HA_RPW]);
+            static_assert(HA_RPW == 4, "one float4 of each weight tile per warp");
+            struct Operands { float4 g4, u4, c4, q4, bv, wv; };      // what one row of the other side brings
+            auto fetch = [&](int cc) {
+                Operands v;
+                v.g4 = *reinterpret_cast<const float4*>(&Gc[cc * HA_LDW + warp * HA_RPW]);
+                v.u4 = *reinterpret_cast<const float4*>(&Uc[cc * HA_LDW + warp * HA_RPW]);
+                v.c4 = TCC ? f4z() : *reinterpret_cast<const float4*>(&Cc[cc * HA_LDW + warp * HA_RPW]);
+                v.q4 = OWNER_Q ? *reinterpret_cast<const float4*>(&UGc[cc * HA_LDW + warp * HA_RPW]) : f4z();
+                v.bv = Bc[cc * d4s + lane];
+                v.wv = OWNER_Q ? f4z() : Wc[cc * d4s + lane];
+                return v;
+            };
+            auto accumulate = [&](const Operands& v) {
+                const float4 g4 = v.g4, u4 = v.u4, c4 = v.c4, bv = v.bv;
                 const float gw[4] = {g4.x, g4.y, g4.z, g4.w}, uw[4] = {u4.x, u4.y, u4.z, u4.w}, cw[4] = {c4.x, c4.y, c4.z, c4.w};
-                const float4 bv = Bc[cc * d4s + lane];
                 if (OWNER_Q) {       // own = q_b (A) with normal Wn; other = t_n (bv)
-                    const float4 q4 = *reinterpret_cast<const float4*>(&UGc[cc * HA_LDW + warp * HA_RPW]);
+                    const float4 q4 = v.q4;
                     const float ugw[4] = {q4.x, q4.y, q4.z, q4.w};
 #pragma unroll
                     for (int i = 0; i < HA_RPW; ++i) {
@@ -397,7 +407,7 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
                         }
                     }
                 } else {             // own = t_n (A); other = q_b (bv) with its normal wv
-                    const float4 wv = Wc[cc * d4s + lane];
+                    const float4 wv = v.wv;
 #pragma unroll
                     for (int i = 0; i < HA_RPW; ++i) {
                         const float4 thr = make_float4(fmaf(uw[i], wv.x, bv.x), fmaf(uw[i], wv.y, bv.y), fmaf(uw[i], wv.z, bv.z), fmaf(uw[i], wv.w, bv.w));
@@ -417,7 +427,13 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
                         }
                     }
                 }
-            }
+            };
+            // not unrolled: with two or more iterations in flight the compiler keeps the next
+            // iteration's loaded values in a second register set and copies them over (about 18
+            // register moves per 80 arithmetic instructions, measured); two named operand sets
+            // that take turns, reloaded in place, avoid the copies and were still 3-5 % slower
+#pragma unroll 1
+            for (int cc = 0; cc < ccmax; ++cc) accumulate(fetch(cc));
         }
         if (more) store_weights(chunk + 1, cur ^ 1);
         __syncthreads();
