@@ -35,6 +35,7 @@ constexpr int TC_EPI_WARPS = 8;                           // epilogue warps of t
 constexpr int TC_EPI_WARPS_TOPK = 16;                     // the filter epilogue of full-entity scoring profits from more
 constexpr int TC_EPI_GROUPS = TC_EPI_WARPS / 4;
 constexpr int TC_GRAD_STAGE_BYTES = 2048;                 // per epilogue warp: 32 rows x 32 bf16 columns on their way to memory
+constexpr int TC_STORE_STAGE_BYTES = 4096;                // the same for EPI_STORE's 32 rows x 32 fp32 columns
 constexpr int TC_PIECE = TC_BN / TC_EPI_GROUPS;           // columns of a 128-wide tile per piece of loss statistics
 // The fused loss epilogues on 256-column tiles run on sixteen warps as well (64 columns = one piece of statistics per warp):
 // measured against eight, C3 passes 41.5 / 58.0 -> 39.4 / 53.8 us, the special-function-bound C4 passes 98.7 / 154.7 -> 98.9 / 135.8 us,
@@ -514,18 +515,29 @@ __device__ __forceinline__ void tc_epilogue(const TcGemmParams& p, const TcItem&
     for (int c0 = col_off; c0 < col_off + WIDTH; c0 += 32) {
         float v[32];
         tmem_ld32(taddr + (uint32_t)(c0 - col_off), v);
-        if (row >= p.M) continue;
         const int ncol = it.n0 + c0;
         if (EPI & EPI_L2) {   // the debug tap of the score block: the distance score of the norm expansion, as the fused epilogues form it
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = ncol + i < p.N ? tc_score<true>(p, v[i], rn, ncol + i) : 0.f;
         }
-        float* dst = Cout + (int64_t)row * p.ldc + ncol;
         if (ncol + 32 <= p.N && (p.ldc & 3) == 0) {
+            // (warp-uniform) a lane holds 32 columns of its own row: stored as they are, every instruction would touch
+            // 32 rows with 16 bytes each.  Through shared memory (128-byte rows, 16-byte pieces XOR-swizzled by row) an
+            // instruction writes four rows' whole 128 bytes.
+            float4* st = reinterpret_cast<float4*>(beat_sm);
+            const int lane = threadIdx.x & 31, sw = lane & 7, row0 = row - lane;
 #pragma unroll
-            for (int i = 0; i < 32; i += 4)
-                *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-        } else {
+            for (int i = 0; i < 8; ++i) st[lane * 8 + (i ^ sw)] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int r = j * 4 + (lane >> 3), c = lane & 7;
+                const float4 val = st[r * 8 + (c ^ (r & 7))];
+                if (row0 + r < p.M) *reinterpret_cast<float4*>(Cout + (int64_t)(row0 + r) * p.ldc + ncol + 4 * c) = val;
+            }
+            __syncwarp();
+        } else if (row < p.M) {
+            float* dst = Cout + (int64_t)row * p.ldc + ncol;
 #pragma unroll
             for (int i = 0; i < 32; ++i) if (ncol + i < p.N) dst[i] = v[i];
         }
@@ -766,8 +778,9 @@ __global__ void __launch_bounds__(tc_threads(EPI, BN), 1) tc_gemm_kernel(const _
             tc_fence_after();
             if (!ok || *stop) { if (lane == 0) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); } break; }
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cgrp * GCOLS);
-            // scratch after the barriers: the rank counts of EPI_TOPK, or 2 KB per epilogue warp for EPI_GRAD's stores
-            int32_t* scratch = (EPI & 3) == EPI_GRAD ? beat_sm + (warp - 2) * (TC_GRAD_STAGE_BYTES / 4) : beat_sm;
+            // scratch after the barriers: the rank counts of EPI_TOPK, or 2 / 4 KB per epilogue warp for EPI_GRAD's / EPI_STORE's stores
+            int32_t* scratch = (EPI & 3) == EPI_GRAD ? beat_sm + (warp - 2) * (TC_GRAD_STAGE_BYTES / 4)
+                             : ((EPI & 3) == EPI_STORE ? beat_sm + (warp - 2) * (TC_STORE_STAGE_BYTES / 4) : beat_sm);
             tc_epilogue<EPI, GCOLS>(p, it, it.m0 + quarter * 32 + lane, rs, cgrp * GCOLS, taddr, scratch);
             tc_fence_before();
             __syncwarp();
@@ -1069,8 +1082,9 @@ cudaError_t launch_gemm_inst(const unsigned char* tmA, const unsigned char* tmB,
                              size_t extra_smem = 0) {
     constexpr size_t smem = tc_smem_bytes(BN);
     constexpr size_t extra_max = (EPI & 3) == EPI_TOPK ? (size_t)TC_BEAT_ROWS_MAX * 4
-                               : ((EPI & 3) == EPI_GRAD ? (size_t)tc_epi_warps(EPI, BN) * TC_GRAD_STAGE_BYTES : 0);
-    if ((EPI & 3) == EPI_GRAD) extra_smem = extra_max;
+                               : ((EPI & 3) == EPI_GRAD ? (size_t)tc_epi_warps(EPI, BN) * TC_GRAD_STAGE_BYTES
+                               : ((EPI & 3) == EPI_STORE ? (size_t)tc_epi_warps(EPI, BN) * TC_STORE_STAGE_BYTES : 0));
+    if ((EPI & 3) == EPI_GRAD || (EPI & 3) == EPI_STORE) extra_smem = extra_max;
     static DeviceOnce configured;
     const cudaError_t e = once_per_device(configured, [] {
         return cudaFuncSetAttribute(tc_gemm_kernel<EPI, BN, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(smem + extra_max));
