@@ -35,12 +35,12 @@ int pick_split(int rows, int cols, int num_sms) {
 }
 
 // The same choice for launches of many more CTAs than the GPU holds at once (TransH at large batches).
-int pick_split_waves(int rows, int cols, int num_sms, int ctas_per_sm) {
-    // One CTA covers 32 owner rows and walks its share of the reduced dimension in chunks of 32.  The CTAs of a launch
+int pick_split_waves(int rows, int cols, int num_sms, int ctas_per_sm, int rows_per_cta = 32) {
+    // One CTA covers 32 (or 64) owner rows and walks its share of the reduced dimension in chunks of 32.  The CTAs of a launch
     // run in waves of num_sms * ctas_per_sm; the number of column splits (at most 16, none empty) is the one that
     // leaves the last wave fullest, with at least about two waves so that the CTAs' start-up overlaps other CTAs'
     // work, and the fewer splits among equals (every split adds a partial slab for the chain kernel to sum).
-    const int row_ctas = (rows + 31) / 32;
+    const int row_ctas = (rows + rows_per_cta - 1) / rows_per_cta;
     const int slots = num_sms * ctas_per_sm;
     const int max_split = std::max(1, std::min(16, (cols + 31) / 32));
     int best = 1;
@@ -263,10 +263,16 @@ int kge_create(const kge_config* cfg, kge_handle** out) {
         h->num_sms = sms;
     else
         (void)cudaGetLastError();
-    // resident CTAs per SM of the TransH accumulation kernels: two (128 registers x 256 threads, 70-90 KB of shared memory)
+    // TransH, fp32: its three dense contractions (u = w.t; the backward's two sums with one coefficient per pair) go
+    // to the tensor cores as bf16 splits once a block has enough pairs to pay for the extra launches (`contract`:
+    // 0 automatic, 1 always where the shapes allow, 2 never)
+    h->th_tc = c.score == KGE_TRANSH && c.prec == KGE_PREC_FP32 && c.dim % 32 == 0 && c.contract != 2 &&
+               (c.contract == 1 || (int64_t)c.batch * c.num_neg >= ((int64_t)1 << 22));
+    // resident CTAs per SM of the TransH accumulation kernels: two (128 registers x 256 threads, 70-90 KB of shared memory);
+    // with the c sums on the tensor cores a CTA of the negatives' side owns 64 rows
     if (c.score == KGE_TRANSH) {
         h->split_q = pick_split_waves(c.batch, c.num_neg, h->num_sms, 2);
-        h->split_t = pick_split_waves(c.num_neg, c.batch, h->num_sms, 2);
+        h->split_t = pick_split_waves(c.num_neg, c.batch, h->num_sms, 2, h->th_tc ? 64 : 32);
     } else {
         h->split_q = pick_split(c.batch, c.num_neg, h->num_sms);
         h->split_t = pick_split(c.num_neg, c.batch, h->num_sms);
@@ -275,11 +281,6 @@ int kge_create(const kge_config* cfg, kge_handle** out) {
         h->split_q = pick_split_tc(c.batch, c.dim, c.num_neg, h->num_sms);
         h->split_t = pick_split_tc(c.num_neg, c.dim, c.batch, h->num_sms);
     }
-    // TransH, fp32: the backward's two contractions with per-pair coefficients go to the tensor cores as bf16
-    // two-term splits once a block has enough pairs to pay for the extra launch (`contract`: 0 automatic, 1 always
-    // where the shapes allow, 2 never)
-    h->th_tc = c.score == KGE_TRANSH && c.prec == KGE_PREC_FP32 && c.dim % 32 == 0 && c.contract != 2 &&
-               (c.contract == 1 || (int64_t)c.batch * c.num_neg >= ((int64_t)1 << 22));
     h->th_gsplit = 1;
     if (h->th_tc) {   // K splits: as many as still give every SM at most one tile, each at least eight 64-wide slices deep, at most 4
         const int bn = 2 * c.dim > 128 ? 256 : 128;

@@ -209,9 +209,11 @@ __global__ void __launch_bounds__(HB_THREADS, 2) th_block_kernel(ThFwdParams p) 
 // ------------------------------------------------------------------------------------------
 // backward
 // ------------------------------------------------------------------------------------------
-constexpr int HA_ROWS = 32, HA_CC = 32, HA_LDW = 36, HA_WARPS = 8, HA_THREADS = 32 * HA_WARPS, HA_RPW = HA_ROWS / HA_WARPS;
+constexpr int HA_CC = 32, HA_WARPS = 8, HA_THREADS = 32 * HA_WARPS;
+// Owner rows per warp: four, or eight on the negatives' side once the c sums have left the kernel (one accumulator
+// per row instead of two: the registers allow it, and an iteration's loads and loop instructions serve twice the arithmetic).
+__host__ __device__ constexpr int ha_rpw(bool owner_q, bool tcc) { return (!owner_q && tcc) ? 8 : 4; }
 constexpr int HA_SLAB = 128;                  // floats of a row handled by one thread block
-constexpr int HA_WPT = HA_ROWS * HA_CC / HA_THREADS;
 
 struct ThAccArgs {
     const float *own, *oth;     // [own_rows, d], [oth_rows, d]
@@ -229,7 +231,8 @@ struct ThAccArgs {
 __host__ __device__ constexpr int ha_tiles(bool owner_q, bool tcc) { return 2 + (tcc ? 0 : 1) + (owner_q ? 1 : 0); }
 template <bool OWNER_Q, bool TCC>
 inline size_t ha_smem() {
-    return (size_t)2 * HA_CC * HA_SLAB * 4 * (OWNER_Q ? 1 : 2) + (size_t)2 * HA_CC * HA_LDW * 4 * ha_tiles(OWNER_Q, TCC) + 2 * sizeof(uint64_t);
+    constexpr int LDW = ha_rpw(OWNER_Q, TCC) * HA_WARPS + 4;
+    return (size_t)2 * HA_CC * HA_SLAB * 4 * (OWNER_Q ? 1 : 2) + (size_t)2 * HA_CC * LDW * 4 * ha_tiles(OWNER_Q, TCC) + 2 * sizeof(uint64_t);
 }
 
 // OWNER_Q: owner rows are queries (own = Q, oth = Tneg); else negatives (own = Tneg, oth = Q, whose normals come along).
@@ -241,6 +244,8 @@ template <bool P1, bool OWNER_Q, bool FULL_SLAB, bool TCC>
 __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
     extern __shared__ __align__(128) unsigned char smraw[];
     constexpr int NT = ha_tiles(OWNER_Q, TCC);
+    constexpr int HA_RPW = ha_rpw(OWNER_Q, TCC), HA_ROWS = HA_RPW * HA_WARPS, HA_LDW = HA_ROWS + 4;   // rows per warp / per block; tile row stride
+    constexpr int HA_WPT = HA_ROWS * HA_CC / HA_THREADS, R4 = HA_RPW / 4;
     constexpr int TI_C = 2, TI_UG = TCC ? 2 : 3;             // tile indices behind g (0) and u (1)
     const int k0 = blockIdx.z * HA_SLAB, kc = FULL_SLAB ? HA_SLAB : min(HA_SLAB, a.d - k0), d4s = kc >> 2;
     float4* Bs = reinterpret_cast<float4*>(smraw);                                   // [2][32][d4s] rows of the other side
@@ -286,7 +291,7 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
             const int idx = tid + HA_THREADS * e;
             int rr, cc; int64_t g;
             if (OWNER_Q) { cc = idx & 31; rr = idx >> 5; g = (int64_t)(r0 + rr) * a.N + (c0 + cc); }
-            else         { rr = idx & 31; cc = idx >> 5; g = (int64_t)(c0 + cc) * a.N + (r0 + rr); }
+            else         { rr = idx & (HA_ROWS - 1); cc = idx / HA_ROWS; g = (int64_t)(c0 + cc) * a.N + (r0 + rr); }
             const bool in = (r0 + rr) < a.own_rows && (c0 + cc) < c_end;
             greg[e] = in ? a.G[g] : 0.f; ureg[e] = in ? a.U[g] : 0.f;
             if (!TCC || OWNER_Q) creg[e] = in ? a.Cp[g] : 0.f;
@@ -297,7 +302,8 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
         const int c0 = c_begin + chunk * HA_CC;
 #pragma unroll
         for (int e = 0; e < HA_WPT; ++e) {
-            const int rr = OWNER_Q ? warp + HA_WARPS * e : lane, cc = OWNER_Q ? lane : warp + HA_WARPS * e;
+            const int idx = tid + HA_THREADS * e;       // the element load_weights fetched
+            const int rr = OWNER_Q ? idx >> 5 : idx & (HA_ROWS - 1), cc = OWNER_Q ? idx & 31 : idx / HA_ROWS;
             const int o = cc * HA_LDW + rr;
             T0[o] = greg[e];
             T0[HA_CC * HA_LDW + o] = ureg[e];
@@ -356,32 +362,43 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
         const float* Cc = Gc + TI_C * HA_CC * HA_LDW;       // (not read with TCC)
         const float* UGc = Gc + TI_UG * HA_CC * HA_LDW;
         if (P1) {   // lane l adds the weights of the chunk's row l (rows beyond the chunk hold zeros)
-            const float4 g4 = *reinterpret_cast<const float4*>(&Gc[lane * HA_LDW + warp * HA_RPW]);
-            sg[0] += g4.x; sg[1] += g4.y; sg[2] += g4.z; sg[3] += g4.w;
-            if (OWNER_Q) {
-                const float4 q4 = *reinterpret_cast<const float4*>(&UGc[lane * HA_LDW + warp * HA_RPW]);
-                sug[0] += q4.x; sug[1] += q4.y; sug[2] += q4.z; sug[3] += q4.w;
+#pragma unroll
+            for (int h4 = 0; h4 < R4; ++h4) {
+                const float4 g4 = *reinterpret_cast<const float4*>(&Gc[lane * HA_LDW + warp * HA_RPW + 4 * h4]);
+                sg[4 * h4] += g4.x; sg[4 * h4 + 1] += g4.y; sg[4 * h4 + 2] += g4.z; sg[4 * h4 + 3] += g4.w;
+                if (OWNER_Q) {
+                    const float4 q4 = *reinterpret_cast<const float4*>(&UGc[lane * HA_LDW + warp * HA_RPW + 4 * h4]);
+                    sug[4 * h4] += q4.x; sug[4 * h4 + 1] += q4.y; sug[4 * h4 + 2] += q4.z; sug[4 * h4 + 3] += q4.w;
+                }
             }
         }
         if (act) {
-            static_assert(HA_RPW == 4, "one float4 of each weight tile per warp");
-            struct Operands { float4 g4, u4, c4, q4, bv, wv; };      // what one row of the other side brings
+            struct Operands { float4 g4[R4], u4[R4], c4[R4], q4[R4], bv, wv; };      // what one row of the other side brings
             auto fetch = [&](int cc) {
                 Operands v;
-                v.g4 = *reinterpret_cast<const float4*>(&Gc[cc * HA_LDW + warp * HA_RPW]);
-                v.u4 = *reinterpret_cast<const float4*>(&Uc[cc * HA_LDW + warp * HA_RPW]);
-                v.c4 = TCC ? f4z() : *reinterpret_cast<const float4*>(&Cc[cc * HA_LDW + warp * HA_RPW]);
-                v.q4 = OWNER_Q ? *reinterpret_cast<const float4*>(&UGc[cc * HA_LDW + warp * HA_RPW]) : f4z();
+#pragma unroll
+                for (int h4 = 0; h4 < R4; ++h4) {
+                    const int o = cc * HA_LDW + warp * HA_RPW + 4 * h4;
+                    v.g4[h4] = *reinterpret_cast<const float4*>(&Gc[o]);
+                    v.u4[h4] = *reinterpret_cast<const float4*>(&Uc[o]);
+                    v.c4[h4] = TCC ? f4z() : *reinterpret_cast<const float4*>(&Cc[o]);
+                    v.q4[h4] = OWNER_Q ? *reinterpret_cast<const float4*>(&UGc[o]) : f4z();
+                }
                 v.bv = Bc[cc * d4s + lane];
                 v.wv = OWNER_Q ? f4z() : Wc[cc * d4s + lane];
                 return v;
             };
             auto accumulate = [&](const Operands& v) {
-                const float4 g4 = v.g4, u4 = v.u4, c4 = v.c4, bv = v.bv;
-                const float gw[4] = {g4.x, g4.y, g4.z, g4.w}, uw[4] = {u4.x, u4.y, u4.z, u4.w}, cw[4] = {c4.x, c4.y, c4.z, c4.w};
+                const float4 bv = v.bv;
+                float gw[HA_RPW], uw[HA_RPW], cw[HA_RPW], ugw[HA_RPW];
+#pragma unroll
+                for (int h4 = 0; h4 < R4; ++h4) {
+                    gw[4 * h4] = v.g4[h4].x; gw[4 * h4 + 1] = v.g4[h4].y; gw[4 * h4 + 2] = v.g4[h4].z; gw[4 * h4 + 3] = v.g4[h4].w;
+                    uw[4 * h4] = v.u4[h4].x; uw[4 * h4 + 1] = v.u4[h4].y; uw[4 * h4 + 2] = v.u4[h4].z; uw[4 * h4 + 3] = v.u4[h4].w;
+                    cw[4 * h4] = v.c4[h4].x; cw[4 * h4 + 1] = v.c4[h4].y; cw[4 * h4 + 2] = v.c4[h4].z; cw[4 * h4 + 3] = v.c4[h4].w;
+                    ugw[4 * h4] = v.q4[h4].x; ugw[4 * h4 + 1] = v.q4[h4].y; ugw[4 * h4 + 2] = v.q4[h4].z; ugw[4 * h4 + 3] = v.q4[h4].w;
+                }
                 if (OWNER_Q) {       // own = q_b (A) with normal Wn; other = t_n (bv)
-                    const float4 q4 = v.q4;
-                    const float ugw[4] = {q4.x, q4.y, q4.z, q4.w};
 #pragma unroll
                     for (int i = 0; i < HA_RPW; ++i) {
                         const float4 thr = make_float4(fmaf(uw[i], Wn[i].x, A[i].x), fmaf(uw[i], Wn[i].y, A[i].y),
@@ -512,7 +529,8 @@ cudaError_t launch_acc(const ThAccArgs& a, cudaStream_t s) {
         return e0 != cudaSuccess ? e0 : cudaFuncSetAttribute(th_accum_kernel<P1, OWNER_Q, false, TCC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ha_smem<OWNER_Q, TCC>());
     });
     if (e != cudaSuccess) return e;
-    dim3 grid((a.own_rows + HA_ROWS - 1) / HA_ROWS, a.split, (a.d + HA_SLAB - 1) / HA_SLAB);
+    constexpr int rows = ha_rpw(OWNER_Q, TCC) * HA_WARPS;
+    dim3 grid((a.own_rows + rows - 1) / rows, a.split, (a.d + HA_SLAB - 1) / HA_SLAB);
     if (a.d % HA_SLAB == 0) th_accum_kernel<P1, OWNER_Q, true, TCC><<<grid, HA_THREADS, ha_smem<OWNER_Q, TCC>(), s>>>(a);
     else th_accum_kernel<P1, OWNER_Q, false, TCC><<<grid, HA_THREADS, ha_smem<OWNER_Q, TCC>(), s>>>(a);
     return cudaSuccess;

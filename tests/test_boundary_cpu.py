@@ -44,10 +44,17 @@ def _create(K, **over):
 def test_create_validates_arguments_on_the_host(K):
     h = _create(K)
     assert h.workspace_bytes(20000, 100, 10) > h.workspace_bytes(20000, 0, 0) > h.workspace_bytes(0, 0, 0) > 0
+    # TransH with its contractions on the tensor cores keeps the operands' bf16 splits and extra partial slabs;
+    # a row width that is no multiple of 32 stays on the CUDA cores whatever is asked for
+    th = {c: _create(K, score="transh", contract=c).workspace_bytes(0, 0, 0) for c in (0, 1, 2)}
+    assert th[1] > th[2] == th[0]                     # 64 x 128 pairs: the automatic choice is the CUDA cores
+    th36 = {c: _create(K, score="transh", dim=36, contract=c).workspace_bytes(0, 0, 0) for c in (1, 2)}
+    assert th36[1] == th36[2]
     for bad, code in ((dict(dim=30), -1), (dict(dim=1024), -1), (dict(p_norm=3), -1), (dict(score=7), -1),
                       (dict(batch=66), -2), (dict(num_neg=127), -2), (dict(batch=66, head_part=0), None),
                       (dict(head_part=2), -1), (dict(adv_temp=-1.0), -1), (dict(num_entities=0), -1),
-                      (dict(num_entities=9, num_parts=4, batch=16, num_neg=4), -3)):
+                      (dict(num_entities=9, num_parts=4, batch=16, num_neg=4), -3),
+                      (dict(score="transh", contract=3), -1), (dict(contract=-1), -1)):
         if code is None:
             _create(K, **bad)           # B % P suffices when the head partition is fixed
             continue
