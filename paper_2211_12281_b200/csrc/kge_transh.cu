@@ -445,12 +445,19 @@ __global__ void __launch_bounds__(HA_THREADS, 2) th_accum_kernel(ThAccArgs a) {
                     }
                 }
             };
-            // not unrolled: with two or more iterations in flight the compiler keeps the next
-            // iteration's loaded values in a second register set and copies them over (about 18
-            // register moves per 80 arithmetic instructions, measured); two named operand sets
-            // that take turns, reloaded in place, avoid the copies and were still 3-5 % slower
+            // Rolled, or unrolled completely; nothing in between.  With a loop left around two or more iterations the
+            // compiler keeps the next iteration's loaded values in a second register set and copies them over (about 18
+            // register moves per 80 arithmetic instructions, measured; unrolling by 2, 4, 8 or 16 was 1-10 % slower than
+            // the rolled loop, two named operand sets taking turns 3-5 %).  Without any back edge there is nothing to
+            // rotate: the query side with the c sums gone runs a full chunk's 32 iterations straight, 1.59 -> 1.48 ms at
+            // B = N = 8192 (the negatives' side with eight rows per warp was 1 % slower that way and stays rolled).
+            if (TCC && OWNER_Q && ccmax == HA_CC) {
+#pragma unroll
+                for (int cc = 0; cc < HA_CC; ++cc) accumulate(fetch(cc));
+            } else {
 #pragma unroll 1
-            for (int cc = 0; cc < ccmax; ++cc) accumulate(fetch(cc));
+                for (int cc = 0; cc < ccmax; ++cc) accumulate(fetch(cc));
+            }
         }
         if (more) store_weights(chunk + 1, cur ^ 1);
         __syncthreads();
