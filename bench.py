@@ -603,6 +603,10 @@ def bench_training(ctx, name, w, cpu_seconds):
             "stage_us": per_stage_us, "stage_frac": stage_frac, "step_frac": step_roof_us / (ms_per_step * 1e3),
             "hbm_substeps": hbm_substeps, "unique_rows": uniq, "graph_load_s": graph_load_s, "setup_s": setup_s,
             "loss": loss.item()}
+    if transh_on_tensor_cores(w):
+        line["stage_frac_note"] = ("block / accum_q / accum_t: CUDA-core kernels at 5 / 4 / 3 instructions per element; th_u and th_contract: "
+                                   "the three dense contractions on the tensor cores, counted at their algorithmic 2 B N d flops each against "
+                                   "the bf16 peak (the bf16 splits that give fp32 accuracy execute 6 x and 4 x that)")
     if ctx.rank == 0 and ctx.world == 1 and cpu_seconds > 0:
         v, t_step, b_cpu, cores, sample = oracle_train_sample(w, cpu_seconds, 2, 1)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
