@@ -324,6 +324,22 @@ def test_transh_tensor_core_contractions(oracle64, p, d, B, N):
     _run(oracle64, prob, steps=2)
 
 
+def test_transh_tensor_core_contractions_run_twice_bit_identical():
+    """Three free-running steps of TransH with its contractions on the tensor cores (split-K slabs and the two
+    halves of a folded tile are added in a fixed order), twice from the same tables: the same bits."""
+    prob = Problem(E=5000, R=6, T=40000, d=128, score="transh", p_norm=1, loss="logsigmoid", opt="adagrad", B=1024, N=768, P=2,
+                   gamma=6.0, adv_temp=1.0, lr=0.05, graph_seed=22, relation_zipf=1.0, contract=1)
+    tables = []
+    for _ in range(2):
+        gpu = GpuSide(prob)
+        for step in range(3):
+            gpu.kge.train_step(step, prob.lr)
+        assert gpu.kge.get_status() == 0
+        tables.append(gpu.tables())
+    for a, b in zip(*tables):
+        assert (a == b).all()
+
+
 @pytest.mark.parametrize("score,p", [("distmult", 1), ("complex", 1), ("transe", 2)])
 @pytest.mark.parametrize("d", [64, 192, 256])
 def test_tensor_core_score_block(oracle64, score, p, d):
