@@ -324,6 +324,15 @@ def test_transh_tensor_core_contractions(oracle64, p, d, B, N):
     _run(oracle64, prob, steps=2)
 
 
+@pytest.mark.parametrize("opt,reg", [("adam", 0.0), ("adagrad", 1e-3), ("sgd", 1e-3)])
+def test_transh_tensor_core_contractions_with_optimisers_and_regulariser(oracle64, opt, reg):
+    """The tensor-core route of TransH under the stateful optimisers and with the L3 regulariser's gradient joining
+    the same rows in the chain kernel (softmax loss here; the other tests of this route use the log-sigmoid)."""
+    prob = Problem(E=3000, R=6, T=30000, d=64, score="transh", p_norm=1, loss="softmax", opt=opt, B=132, N=200, P=2,
+                   ce_correction=0.2, lr=0.02, graph_seed=23, relation_zipf=1.0, contract=1, reg_lambda=reg)
+    _run(oracle64, prob, steps=2)
+
+
 def test_transh_tensor_core_contractions_run_twice_bit_identical():
     """Three free-running steps of TransH with its contractions on the tensor cores (split-K slabs and the two
     halves of a folded tile are added in a fixed order), twice from the same tables: the same bits."""
