@@ -817,19 +817,25 @@ struct DualProb {
     int fold; int64_t fold_stride;
 };
 
-template <int BN>
+// PAIR: the A operand has two K segments that meet the same slices of the B operand (two-term splits of dL/dF-like
+// coefficients against one [x1 | x2] operand).  A stage then holds both segments' A tiles beside the one B tile and both
+// are multiplied into the accumulator, so a B slice is fetched once instead of once per segment (a third fewer operand
+// bytes per flop); K runs over one segment's slices.  Three stages instead of four fit.
+template <int BN, bool PAIR = false>
 __global__ void __launch_bounds__(32 * (2 + TC_EPI_WARPS), 1) tc_gemm_dual_kernel(const __grid_constant__ CUtensorMap tmA0,
                                                                                     const __grid_constant__ CUtensorMap tmB0,
                                                                                     const __grid_constant__ CUtensorMap tmA1,
                                                                                     const __grid_constant__ CUtensorMap tmB1,
                                                                                     DualProb q0, DualProb q1, int32_t* status, int wait_limit) {
-    constexpr uint32_t STAGE_BYTES = tc_stage_bytes(BN);
+    constexpr uint32_t A_BYTES = PAIR ? 2 * TC_A_BYTES : TC_A_BYTES;      // A tile(s) of a stage; the B tile follows
+    constexpr uint32_t STAGE_BYTES = tc_stage_bytes(BN) + (PAIR ? TC_A_BYTES : 0u);
+    constexpr int STAGES = PAIR ? 3 : TC_STAGES;
     constexpr int NACC = 512 / BN;
     constexpr uint32_t TMEM_COLS = NACC * BN;
     constexpr int EW = TC_EPI_WARPS, EG = EW / 4;
     extern __shared__ unsigned char tc_smem_raw[];
     unsigned char* base = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
-    uint64_t* full = reinterpret_cast<uint64_t*>(base + (size_t)TC_STAGES * STAGE_BYTES);
+    uint64_t* full = reinterpret_cast<uint64_t*>(base + (size_t)STAGES * STAGE_BYTES);
     uint64_t* empty = full + TC_RING_MAX;
     uint64_t* acc_full = empty + TC_RING_MAX;
     uint64_t* acc_empty = acc_full + NACC;
@@ -846,7 +852,7 @@ __global__ void __launch_bounds__(32 * (2 + TC_EPI_WARPS), 1) tc_gemm_dual_kerne
     };
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         for (int b = 0; b < NACC; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EW); }
         *stop = 0;
         mbar_init_fence();
@@ -871,21 +877,25 @@ __global__ void __launch_bounds__(32 * (2 + TC_EPI_WARPS), 1) tc_gemm_dual_kerne
                 const CUtensorMap* tb = which ? &tmB1 : &tmB0;
                 const int kb0 = it.z * q.kb_per_split, nkb = min(q.kb_per_split, q.kb_total - kb0);
                 for (int kb = 0; kb < nkb; ++kb, ++ring) {
-                    const int s = ring % TC_STAGES;
-                    if (!mbar_wait_idle(&empty[s], ((ring / TC_STAGES) & 1) ^ 1, wait_limit)) { *stop = 1; set_status(status, KGE_ERR_TIMEOUT); break; }
+                    const int s = ring % STAGES;
+                    if (!mbar_wait_idle(&empty[s], ((ring / STAGES) & 1) ^ 1, wait_limit)) { *stop = 1; set_status(status, KGE_ERR_TIMEOUT); break; }
                     unsigned char* sa = base + (size_t)s * STAGE_BYTES;
                     mbar_arrive_expect_tx(&full[s], STAGE_BYTES);
-                    const int kblk = kb0 + kb, seg = kblk / q.seg_kb;
+                    const int kblk = kb0 + kb, seg = PAIR ? 0 : kblk / q.seg_kb;
                     const int k0 = kblk * TC_BK, kseg = (kblk - seg * q.seg_kb) * TC_BK;
-                    if (which) {      // dL/dF with the contraction index as rows: two boxes of 64 output rows
 #pragma unroll
-                        for (int g = 0; g < TC_BM / 64; ++g)
-                            tma_load_2d(sa + g * TC_MN_GROUP_BYTES, ta, it.m0 + 64 * g + seg * q.a_seg_x, kseg, &full[s]);
-                    } else {
-                        tma_load_2d(sa, ta, k0, it.m0, &full[s]);
+                    for (int half = 0; half < (PAIR ? 2 : 1); ++half) {       // PAIR: both segments' A tiles of this slice
+                        unsigned char* da = sa + half * TC_A_BYTES;
+                        if (which) {      // dL/dF with the contraction index as rows: two boxes of 64 output rows
+#pragma unroll
+                            for (int g = 0; g < TC_BM / 64; ++g)
+                                tma_load_2d(da + g * TC_MN_GROUP_BYTES, ta, it.m0 + 64 * g + (PAIR ? half : seg) * q.a_seg_x, kseg, &full[s]);
+                        } else {
+                            tma_load_2d(da, ta, k0 + half * q.seg_kb * TC_BK, it.m0, &full[s]);
+                        }
                     }
 #pragma unroll
-                    for (int g = 0; g < BN / 64; ++g) tma_load_2d(sa + TC_A_BYTES + g * TC_MN_GROUP_BYTES, tb, it.n0 + 64 * g, kseg, &full[s]);
+                    for (int g = 0; g < BN / 64; ++g) tma_load_2d(sa + A_BYTES + g * TC_MN_GROUP_BYTES, tb, it.n0 + 64 * g, kseg, &full[s]);
                 }
             }
         }
@@ -904,15 +914,19 @@ __global__ void __launch_bounds__(32 * (2 + TC_EPI_WARPS), 1) tc_gemm_dual_kerne
                 tc_fence_after();
                 const uint32_t tmem_acc = tmem_base + (uint32_t)buf * BN;
                 for (int kb = 0; kb < nkb; ++kb, ++ring) {
-                    const int s = ring % TC_STAGES;
-                    if (!mbar_wait_idle(&full[s], (ring / TC_STAGES) & 1, wait_limit)) { ok = false; break; }
+                    const int s = ring % STAGES;
+                    if (!mbar_wait_idle(&full[s], (ring / STAGES) & 1, wait_limit)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = smem_u32(base + (size_t)s * STAGE_BYTES);
 #pragma unroll
-                    for (int k = 0; k < TC_BK / 16; ++k) {
-                        const uint64_t ad = which ? umma_desc_mn_sw128(sa + k * 2048) : umma_desc_k_sw128(sa + k * 32);
-                        const uint64_t bd = umma_desc_mn_sw128(sa + TC_A_BYTES + k * 2048);
-                        umma_bf16(tmem_acc, ad, bd, which ? idesc_mn : idesc_k, (kb | k) != 0);
+                    for (int half = 0; half < (PAIR ? 2 : 1); ++half) {
+#pragma unroll
+                        for (int k = 0; k < TC_BK / 16; ++k) {
+                            const uint32_t aa = sa + half * TC_A_BYTES;
+                            const uint64_t ad = which ? umma_desc_mn_sw128(aa + k * 2048) : umma_desc_k_sw128(aa + k * 32);
+                            const uint64_t bd = umma_desc_mn_sw128(sa + A_BYTES + k * 2048);
+                            umma_bf16(tmem_acc, ad, bd, which ? idesc_mn : idesc_k, (kb | k | half) != 0);
+                        }
                     }
                     umma_commit(&empty[s]);
                 }
@@ -1206,20 +1220,20 @@ DualProb dual_prob(int M, int N, int K, int split, float* C, int64_t ldc, int bn
     q.seg_kb = q.kb_total; q.a_seg_x = 0; q.fold = 0; q.fold_stride = 0;
     return q;
 }
-template <int BN>
+template <int BN, bool PAIR = false>
 cudaError_t launch_gemm_dual(kge_handle* h, const unsigned char* tmA0, const unsigned char* tmB0, const unsigned char* tmA1,
                              const unsigned char* tmB1, const DualProb& q0, const DualProb& q1, cudaStream_t s) {
-    constexpr size_t smem = tc_smem_bytes(BN);
+    constexpr size_t smem = PAIR ? 1024 + (size_t)3 * (tc_stage_bytes(BN) + TC_A_BYTES) + 256 : tc_smem_bytes(BN);
     static DeviceOnce configured;
     const cudaError_t e = once_per_device(configured, [] {
-        return cudaFuncSetAttribute(tc_gemm_dual_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        return cudaFuncSetAttribute(tc_gemm_dual_kernel<BN, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     });
     if (e != cudaSuccess) return e;
     // as few CTAs as give the same number of rounds: SMs left over serve the id sort that runs beside this launch
     const int total = q0.items + q1.items;
     const int rounds = (total + h->num_sms - 1) / h->num_sms;
     const int grid = (total + rounds - 1) / rounds;
-    tc_gemm_dual_kernel<BN><<<grid, 32 * (2 + TC_EPI_WARPS), smem, s>>>(
+    tc_gemm_dual_kernel<BN, PAIR><<<grid, 32 * (2 + TC_EPI_WARPS), smem, s>>>(
         *reinterpret_cast<const CUtensorMap*>(tmA0), *reinterpret_cast<const CUtensorMap*>(tmB0),
         *reinterpret_cast<const CUtensorMap*>(tmA1), *reinterpret_cast<const CUtensorMap*>(tmB1), q0, q1, h->ws.status, h->wait_limit);
     return cudaSuccess;
@@ -1298,15 +1312,16 @@ int launch_th_contract_gemm(kge_handle* h, cudaStream_t s) {
     const int B = c.batch, N = c.num_neg, d = c.dim;
     const int Np = (N + 63) / 64 * 64, Bp = (B + 63) / 64 * 64;
     const int bn = tc_backward_tile_cols(2 * d);
-    DualProb q0 = dual_prob(B, 2 * d, 2 * Np, h->th_gsplit, w.dWpart + (size_t)h->split_q * B * d, d, bn);
-    DualProb q1 = dual_prob(N, 2 * d, 2 * Bp, h->th_gsplit, w.dTpart + (size_t)h->split_t * N * d, d, bn);
+    // (K runs over one segment: both segments' tiles of c travel in one stage, see tc_gemm_dual_kernel<BN, PAIR>)
+    DualProb q0 = dual_prob(B, 2 * d, Np, h->th_gsplit, w.dWpart + (size_t)h->split_q * B * d, d, bn);
+    DualProb q1 = dual_prob(N, 2 * d, Bp, h->th_gsplit, w.dTpart + (size_t)h->split_t * N * d, d, bn);
     q0.seg_kb = Np / TC_BK; q0.a_seg_x = 0;
     q1.seg_kb = Bp / TC_BK; q1.a_seg_x = Np;
     q0.fold = q1.fold = d;
     q0.fold_stride = (int64_t)B * d; q0.split_stride = 2 * q0.fold_stride;
     q1.fold_stride = (int64_t)N * d; q1.split_stride = 2 * q1.fold_stride;
-    KGE_CUDA_CHECK(h, bn == 256 ? launch_gemm_dual<256>(h, h->tm_cs, h->tm_ts64, h->tm_cs64, h->tm_ws64, q0, q1, s)
-                                : launch_gemm_dual<128>(h, h->tm_cs, h->tm_ts64, h->tm_cs64, h->tm_ws64, q0, q1, s));
+    KGE_CUDA_CHECK(h, bn == 256 ? (launch_gemm_dual<256, true>(h, h->tm_cs, h->tm_ts64, h->tm_cs64, h->tm_ws64, q0, q1, s))
+                                : (launch_gemm_dual<128, true>(h, h->tm_cs, h->tm_ts64, h->tm_cs64, h->tm_ws64, q0, q1, s)));
     KGE_LAUNCH_CHECK(h);
     return KGE_OK;
 }
