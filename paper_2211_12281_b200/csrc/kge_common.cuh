@@ -72,7 +72,7 @@ struct Workspace {
     // (x = x1 + x2 up to 2^-17 relative) of c = -dL/dF c' as [B, 2 Np] = [c1 | c2] (Np = N rounded up to 64,
     // padding kept zero), of the negatives as [N, 2d] = [t1 | t2] and of the unit normals as [B, 2d]
     uint16_t *Csb, *Tsb, *Wsb;
-    uint16_t *W6b, *T6b;                   // [B, 6d], [N, 6d] bf16 three-term splits of normals and negatives, laid out for u = w.t
+    uint16_t *W6b, *T6b;                   // [B, 3 dp], [N, 3 dp] bf16 three-term splits [x1 | x2 | x3] of normals and negatives (dp = d rounded up to 64, padding zero): operands of u = w.t
     float *dQpart, *dWpart, *dTpart;       // [Sq,B,d], [Sq,B,d] (TransH), [St,N,d]
     float *grad_ent, *grad_rel, *grad_relw;  // [2B+N,d], [B,kw], [B,d]
     // dedup
@@ -231,6 +231,8 @@ int launch_th_backward(kge_handle* h, cudaStream_t sq, cudaStream_t st);
 int th_contract_slabs(const kge_handle* h);          // partial slabs the tensor-core contractions add per side (0 when off)
 int launch_th_contract_gemm(kge_handle* h, cudaStream_t s);
 int launch_tc_forward(kge_handle* h, cudaStream_t s);
+int launch_tc_gemm_terms(kge_handle* h, const unsigned char* tmA, const unsigned char* tmB, int M, int N, int tstride, float* C,
+                         int64_t ldc, cudaStream_t s);
 int launch_tc_gemm_nt(kge_handle* h, const unsigned char* tmA, const unsigned char* tmB, int M, int N, int K, float* C, int64_t ldc,
                       cudaStream_t s);
 int launch_tc_gemm_tn(kge_handle* h, const unsigned char* tmA64, const unsigned char* tmB64, int M, int N, int K, int split, float* C,

@@ -976,6 +976,155 @@ __global__ void __launch_bounds__(32 * (2 + TC_EPI_WARPS), 1) tc_gemm_dual_kerne
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
 }
 
+// ------------------------------------------------------------------------------------------
+// C[M, N] = A . B^T in fp32 accuracy from bf16 operands: both operands arrive as three-term splits x = x1 + x2 + x3 laid
+// out side by side, [x1 | x2 | x3] with `tstride` columns per term (K rounded up to 64, padding zero), and the six
+// products a_i b_j with i + j <= 4 are accumulated in fp32 (what is left out is below 2^-25 relative).  A stage holds
+// one 64-wide K slice of all three terms of both operands (6 x 16 KB), so every slice is fetched once for the up to
+// three products it takes part in: half the operand bytes of the same products run as one long K (each term's slice would
+// be fetched once per product).  128 x 128 tiles, two stages, four accumulators in turn; warp roles, barriers and bounded
+// waits as in tc_gemm_kernel; fp32 tiles leave through shared memory (see tc_epilogue).
+// ------------------------------------------------------------------------------------------
+struct TermsParams {
+    int M, N, kslices, tstride;     // kslices = tstride / 64
+    int tiles_m, tiles_n, items;    // column tile fastest
+    float* C; int64_t ldc;
+    int32_t* status; int wait_limit;
+};
+constexpr uint32_t TT_TERM_BYTES = 128 * TC_BK * 2;           // one term's 128 x 64 bf16 tile
+constexpr uint32_t TT_STAGE_BYTES = 6 * TT_TERM_BYTES;
+constexpr int TT_STAGES = 2;
+constexpr size_t TT_SMEM = 1024 + (size_t)TT_STAGES * TT_STAGE_BYTES + 256 + (size_t)TC_EPI_WARPS * TC_STORE_STAGE_BYTES;
+
+__global__ void __launch_bounds__(32 * (2 + TC_EPI_WARPS), 1) tc_gemm_terms_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                                                     const __grid_constant__ CUtensorMap tmB, TermsParams p) {
+    constexpr int BN = 128, NACC = 512 / BN;
+    constexpr uint32_t TMEM_COLS = 512;
+    extern __shared__ unsigned char tc_smem_raw[];
+    unsigned char* base = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
+    uint64_t* full = reinterpret_cast<uint64_t*>(base + (size_t)TT_STAGES * TT_STAGE_BYTES);
+    uint64_t* empty = full + TT_STAGES;
+    uint64_t* acc_full = empty + TT_STAGES;
+    uint64_t* acc_empty = acc_full + NACC;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + NACC);
+    volatile uint32_t* stop = tmem_slot + 1;
+    float4* store_stage = reinterpret_cast<float4*>(base + (size_t)TT_STAGES * TT_STAGE_BYTES + 256);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < TT_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int b = 0; b < NACC; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], TC_EPI_WARPS); }
+        *stop = 0;
+        mbar_init_fence();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int ring = 0;
+            for (int item = blockIdx.x; item < p.items && !*stop; item += gridDim.x) {
+                const int m0 = (item / p.tiles_n) * TC_BM, n0 = (item % p.tiles_n) * BN;
+                for (int ks = 0; ks < p.kslices; ++ks, ++ring) {
+                    const int s = ring % TT_STAGES;
+                    if (!mbar_wait_idle(&empty[s], ((ring / TT_STAGES) & 1) ^ 1, p.wait_limit)) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); break; }
+                    unsigned char* sa = base + (size_t)s * TT_STAGE_BYTES;
+                    mbar_arrive_expect_tx(&full[s], TT_STAGE_BYTES);
+#pragma unroll
+                    for (int t = 0; t < 3; ++t) {
+                        tma_load_2d(sa + t * TT_TERM_BYTES, &tmA, t * p.tstride + ks * TC_BK, m0, &full[s]);
+                        tma_load_2d(sa + (3 + t) * TT_TERM_BYTES, &tmB, t * p.tstride + ks * TC_BK, n0, &full[s]);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(TC_BM, BN, false, false);
+            int ring = 0;
+            bool ok = true;
+            for (int item = blockIdx.x, local = 0; item < p.items && ok && !*stop; item += gridDim.x, ++local) {
+                const int buf = local % NACC;
+                if (!mbar_wait_idle(&acc_empty[buf], ((local / NACC) & 1) ^ 1, p.wait_limit)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tmem_acc = tmem_base + (uint32_t)buf * BN;
+                for (int ks = 0; ks < p.kslices; ++ks, ++ring) {
+                    const int s = ring % TT_STAGES;
+                    if (!mbar_wait_idle(&full[s], (ring / TT_STAGES) & 1, p.wait_limit)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(base + (size_t)s * TT_STAGE_BYTES);
+#pragma unroll
+                    for (int ta = 0; ta < 3; ++ta) {
+#pragma unroll
+                        for (int tb = 0; tb < 3; ++tb) {
+                            if (ta + tb > 2) continue;          // the six products that matter (terms counted from 0)
+#pragma unroll
+                            for (int k = 0; k < TC_BK / 16; ++k) {
+                                const uint64_t ad = umma_desc_k_sw128(sa + ta * TT_TERM_BYTES + k * 32);
+                                const uint64_t bd = umma_desc_k_sw128(sa + (3 + tb) * TT_TERM_BYTES + k * 32);
+                                umma_bf16(tmem_acc, ad, bd, idesc, (ks | ta | tb | k) != 0);
+                            }
+                        }
+                    }
+                    umma_commit(&empty[s]);
+                }
+                umma_commit(&acc_full[buf]);           // also after a failed wait, so the epilogue warps wake up
+            }
+            if (!ok) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); }
+        }
+    } else {
+        const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
+        const int cgrp = (warp - 2) >> 2;              // which half of the tile's columns
+        constexpr int COLS = BN / (TC_EPI_WARPS / 4);
+        float4* st = store_stage + (size_t)(warp - 2) * (TC_STORE_STAGE_BYTES / 16);
+        for (int item = blockIdx.x, local = 0; item < p.items; item += gridDim.x, ++local) {
+            const int buf = local % NACC;
+            const bool ok = mbar_wait_bounded(&acc_full[buf], (local / NACC) & 1, p.wait_limit);
+            tc_fence_after();
+            if (!ok || *stop) { if (lane == 0) { *stop = 1; set_status(p.status, KGE_ERR_TIMEOUT); } break; }
+            const int m0 = (item / p.tiles_n) * TC_BM, n0 = (item % p.tiles_n) * BN;
+            const int row0 = m0 + quarter * 32, row = row0 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cgrp * COLS);
+#pragma unroll 1
+            for (int c0 = cgrp * COLS; c0 < (cgrp + 1) * COLS; c0 += 32) {
+                float v[32];
+                tmem_ld32(taddr + (uint32_t)(c0 - cgrp * COLS), v);
+                const int ncol = n0 + c0;
+                if (ncol + 32 <= p.N && (p.ldc & 3) == 0) {      // (warp-uniform) four rows' whole 128 bytes per store instruction
+                    const int sw = lane & 7;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) st[lane * 8 + (i ^ sw)] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int r = j * 4 + (lane >> 3), c = lane & 7;
+                        const float4 val = st[r * 8 + (c ^ (r & 7))];
+                        if (row0 + r < p.M) *reinterpret_cast<float4*>(p.C + (int64_t)(row0 + r) * p.ldc + ncol + 4 * c) = val;
+                    }
+                    __syncwarp();
+                } else if (row < p.M) {
+                    float* dst = p.C + (int64_t)row * p.ldc + ncol;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) if (ncol + i < p.N) dst[i] = v[i];
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -1254,6 +1403,23 @@ int launch_tc_gemm_nt(kge_handle* h, const unsigned char* tmA, const unsigned ch
     p.tiles_m = (M + TC_BM - 1) / TC_BM; p.tiles_n = (N + p.bn - 1) / p.bn; p.items = p.tiles_m * p.tiles_n;
     if (p.bn == 256) KGE_CUDA_CHECK(h, (launch_gemm_inst<EPI_STORE, 256>(tmA, tmB, p, h->num_sms, s)));
     else KGE_CUDA_CHECK(h, (launch_gemm_inst<EPI_STORE, 128>(tmA, tmB, p, h->num_sms, s)));
+    KGE_LAUNCH_CHECK(h);
+    return KGE_OK;
+}
+//   C[M, N] = A . B^T with fp32 accuracy from three-term bf16 splits [x1 | x2 | x3] of both operands (`tstride` columns per
+//   term, a multiple of 64 with zero padding; tensor maps with 128-row boxes over [rows, 3 tstride])
+int launch_tc_gemm_terms(kge_handle* h, const unsigned char* tmA, const unsigned char* tmB, int M, int N, int tstride, float* C,
+                         int64_t ldc, cudaStream_t s) {
+    TermsParams p{};
+    p.M = M; p.N = N; p.tstride = tstride; p.kslices = tstride / TC_BK;
+    p.tiles_m = (M + TC_BM - 1) / TC_BM; p.tiles_n = (N + 127) / 128; p.items = p.tiles_m * p.tiles_n;
+    p.C = C; p.ldc = ldc; p.status = h->ws.status; p.wait_limit = h->wait_limit;
+    static DeviceOnce configured;
+    KGE_CUDA_CHECK(h, once_per_device(configured, [] {
+        return cudaFuncSetAttribute(tc_gemm_terms_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TT_SMEM);
+    }));
+    tc_gemm_terms_kernel<<<std::min(p.items, h->num_sms), 32 * (2 + TC_EPI_WARPS), TT_SMEM, s>>>(
+        *reinterpret_cast<const CUtensorMap*>(tmA), *reinterpret_cast<const CUtensorMap*>(tmB), p);
     KGE_LAUNCH_CHECK(h);
     return KGE_OK;
 }

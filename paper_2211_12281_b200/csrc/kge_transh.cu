@@ -501,12 +501,10 @@ cudaError_t launch_fwd(const ThFwdParams& p, cudaStream_t s) {
     return launch_dependent(th_block_kernel<P1, 0, UEXT>, grid, dim3(HB_THREADS), hb_smem(p.d), s, p);
 }
 
-// bf16 three-term splits x = x1 + x2 + x3 (2^-25 relative) of the unit normals and of the negatives, laid out along K
-// so that one K-major contraction forms the six products that matter:
-//   normals   [B, 6d] = [w1 | w1 | w2 | w1 | w3 | w2]
-//   negatives [N, 6d] = [t1 | t2 | t1 | t3 | t1 | t2]
+// bf16 three-term splits x = x1 + x2 + x3 (2^-25 relative) of the unit normals and of the negatives, side by side:
+// [rows, 3 dp] = [x1 | x2 | x3] with dp = d rounded up to 64 (the padding is zeroed once when the workspace is bound).
 // One thread per four coordinates.
-__global__ void __launch_bounds__(256) th_split3_kernel(const float4* W, int B, const float4* T, int N, int d4, uint2* W6, uint2* T6) {
+__global__ void __launch_bounds__(256) th_split3_kernel(const float4* W, int B, const float4* T, int N, int d4, int dp4, uint2* W3, uint2* T3) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (int64_t)(B + N) * d4) return;
     const int row = (int)(i / d4), c = (int)(i - (int64_t)row * d4);
@@ -523,10 +521,8 @@ __global__ void __launch_bounds__(256) th_split3_kernel(const float4* W, int B, 
         t1[e] = __bfloat16_as_ushort(a); t2[e] = __bfloat16_as_ushort(b); t3[e] = __bfloat16_as_ushort(cc);
     }
     auto pack = [](const uint16_t* t) { return make_uint2((uint32_t)t[0] | ((uint32_t)t[1] << 16), (uint32_t)t[2] | ((uint32_t)t[3] << 16)); };
-    const uint2 p1 = pack(t1), p2 = pack(t2), p3 = pack(t3);
-    uint2* dst = (nrm ? W6 + (int64_t)row * 6 * d4 : T6 + (int64_t)(row - B) * 6 * d4) + c;
-    if (nrm) { dst[0] = p1; dst[d4] = p1; dst[2 * d4] = p2; dst[3 * d4] = p1; dst[4 * d4] = p3; dst[5 * d4] = p2; }
-    else     { dst[0] = p1; dst[d4] = p2; dst[2 * d4] = p1; dst[3 * d4] = p3; dst[4 * d4] = p1; dst[5 * d4] = p2; }
+    uint2* dst = (nrm ? W3 + (int64_t)row * 3 * dp4 : T3 + (int64_t)(row - B) * 3 * dp4) + c;
+    dst[0] = pack(t1); dst[dp4] = pack(t2); dst[2 * dp4] = pack(t3);
 }
 
 template <bool P1, bool OWNER_Q, bool TCC>
@@ -573,14 +569,15 @@ int launch_th_forward(kge_handle* h, cudaStream_t s) {
     ThFwdParams p{c.batch, c.num_neg, c.dim, w.Q, w.What, w.Tneg, w.wsum, w.F, w.U, w.Cc, w.status, h->wait_limit};
     const bool p1 = h->kind == KIND_TH_L1;
     if (h->th_tc) {
-        // u = w.t for all pairs as one tensor-core contraction over the operands' three-term splits
+        // u = w.t for all pairs as one tensor-core contraction over the operands' three-term splits (six products per K slice)
         stage_begin(h, ST_TH_U, s);
         const int64_t n4 = (int64_t)(c.batch + c.num_neg) * (c.dim / 4);
+        const int dp = (c.dim + 63) / 64 * 64;
         th_split3_kernel<<<(int)((n4 + 255) / 256), 256, 0, s>>>(reinterpret_cast<const float4*>(w.What), c.batch,
-                                                                 reinterpret_cast<const float4*>(w.Tneg), c.num_neg, c.dim / 4,
+                                                                 reinterpret_cast<const float4*>(w.Tneg), c.num_neg, c.dim / 4, dp / 4,
                                                                  reinterpret_cast<uint2*>(w.W6b), reinterpret_cast<uint2*>(w.T6b));
         KGE_LAUNCH_CHECK(h);
-        const int rc = launch_tc_gemm_nt(h, h->tm_w6, h->tm_t6, c.batch, c.num_neg, 6 * c.dim, w.U, c.num_neg, s);
+        const int rc = launch_tc_gemm_terms(h, h->tm_w6, h->tm_t6, c.batch, c.num_neg, dp, w.U, c.num_neg, s);
         if (rc != KGE_OK) return rc;
         stage_end(h, ST_TH_U, s);
         stage_begin(h, ST_BLOCK, s);      // (the caller's bracket opened before the contraction: open it again here)
