@@ -126,8 +126,8 @@ size_t layout(const kge_handle* h, char* base, int64_t T, int32_t maxq, int32_t 
     w.Tsb = h->th_tc ? cv.take<uint16_t>(N * 2 * d) : nullptr;
     w.Wsb = h->th_tc ? cv.take<uint16_t>(B * 2 * d) : nullptr;
     const size_t dp = (d + 63) / 64 * 64;
-    w.W6b = h->th_tc ? cv.take<uint16_t>(B * 3 * dp) : nullptr;
-    w.T6b = h->th_tc ? cv.take<uint16_t>(N * 3 * dp) : nullptr;
+    w.W3b = h->th_tc ? cv.take<uint16_t>(B * 3 * dp) : nullptr;
+    w.T3b = h->th_tc ? cv.take<uint16_t>(N * 3 * dp) : nullptr;
     const size_t xs = (size_t)th_contract_slabs(h);      // slabs the tensor-core contractions add behind the splits' own
     w.dQpart = cv.take<float>((size_t)h->split_q * B * d);
     w.dWpart = th ? cv.take<float>(((size_t)h->split_q + xs) * B * d) : nullptr;
@@ -381,10 +381,10 @@ int kge_bind(kge_handle* h, float* ent, float* rel, float* relw, float* ent_stat
         if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_ts64, h->ws.Tsb, N, 2 * d, 2 * d, 64);
         if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_ws64, h->ws.Wsb, B, 2 * d, 2 * d, 64);
         const int64_t dp = (d + 63) / 64 * 64;
-        KGE_CUDA_CHECK(h, cudaMemsetAsync(h->ws.W6b, 0, (size_t)B * 3 * dp * 2, static_cast<cudaStream_t>(stream)));
-        KGE_CUDA_CHECK(h, cudaMemsetAsync(h->ws.T6b, 0, (size_t)N * 3 * dp * 2, static_cast<cudaStream_t>(stream)));
-        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_w6, h->ws.W6b, B, 3 * dp, 3 * dp, 128);
-        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_t6, h->ws.T6b, N, 3 * dp, 3 * dp, 128);
+        KGE_CUDA_CHECK(h, cudaMemsetAsync(h->ws.W3b, 0, (size_t)B * 3 * dp * 2, static_cast<cudaStream_t>(stream)));
+        KGE_CUDA_CHECK(h, cudaMemsetAsync(h->ws.T3b, 0, (size_t)N * 3 * dp * 2, static_cast<cudaStream_t>(stream)));
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_w3, h->ws.W3b, B, 3 * dp, 3 * dp, 128);
+        if (rc == KGE_OK) rc = tc_make_operand_map(h, h->tm_t3, h->ws.T3b, N, 3 * dp, 3 * dp, 128);
         if (rc != KGE_OK) return rc;
     }
     if (!h->streams_ready) {

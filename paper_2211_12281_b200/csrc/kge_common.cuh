@@ -72,7 +72,7 @@ struct Workspace {
     // (x = x1 + x2 up to 2^-17 relative) of c = -dL/dF c' as [B, 2 Np] = [c1 | c2] (Np = N rounded up to 64,
     // padding kept zero), of the negatives as [N, 2d] = [t1 | t2] and of the unit normals as [B, 2d]
     uint16_t *Csb, *Tsb, *Wsb;
-    uint16_t *W6b, *T6b;                   // [B, 3 dp], [N, 3 dp] bf16 three-term splits [x1 | x2 | x3] of normals and negatives (dp = d rounded up to 64, padding zero): operands of u = w.t
+    uint16_t *W3b, *T3b;                   // [B, 3 dp], [N, 3 dp] bf16 three-term splits [x1 | x2 | x3] of normals and negatives (dp = d rounded up to 64, padding zero): operands of u = w.t
     float *dQpart, *dWpart, *dTpart;       // [Sq,B,d], [Sq,B,d] (TransH), [St,N,d]
     float *grad_ent, *grad_rel, *grad_relw;  // [2B+N,d], [B,kw], [B,d]
     // dedup
@@ -134,7 +134,7 @@ struct kge_handle {
     // TMA tensor maps (tensor-core path): Qb, Tb (128-row boxes) for the scores; Gb (128-row boxes) and Tb (64-row boxes,
     // read MN-major) for dQ; Gb and Qb (64-row boxes, read MN-major) for dT
     alignas(64) unsigned char tm_q[128], tm_t[128], tm_g[128], tm_g64[128], tm_t64[128], tm_q64[128];
-    alignas(64) unsigned char tm_cs[128], tm_cs64[128], tm_ts64[128], tm_ws64[128], tm_w6[128], tm_t6[128];   // TransH splits: Csb K-major / MN-major, Tsb, Wsb
+    alignas(64) unsigned char tm_cs[128], tm_cs64[128], tm_ts64[128], tm_ws64[128], tm_w3[128], tm_t3[128];   // TransH splits: Csb K-major / MN-major, Tsb, Wsb
     alignas(64) unsigned char tm_iq[128], tm_eb[128];   // inference: bf16 query vectors and bf16 entity table
     alignas(64) unsigned char tm_iq32[128], tm_ent32[128];   // inference on CUDA cores: fp32 query vectors and entity table in 64-row x 32-float boxes
     bool tiles32_ready;

@@ -575,9 +575,9 @@ int launch_th_forward(kge_handle* h, cudaStream_t s) {
         const int dp = (c.dim + 63) / 64 * 64;
         th_split3_kernel<<<(int)((n4 + 255) / 256), 256, 0, s>>>(reinterpret_cast<const float4*>(w.What), c.batch,
                                                                  reinterpret_cast<const float4*>(w.Tneg), c.num_neg, c.dim / 4, dp / 4,
-                                                                 reinterpret_cast<uint2*>(w.W6b), reinterpret_cast<uint2*>(w.T6b));
+                                                                 reinterpret_cast<uint2*>(w.W3b), reinterpret_cast<uint2*>(w.T3b));
         KGE_LAUNCH_CHECK(h);
-        const int rc = launch_tc_gemm_terms(h, h->tm_w6, h->tm_t6, c.batch, c.num_neg, dp, w.U, c.num_neg, s);
+        const int rc = launch_tc_gemm_terms(h, h->tm_w3, h->tm_t3, c.batch, c.num_neg, dp, w.U, c.num_neg, s);
         if (rc != KGE_OK) return rc;
         stage_end(h, ST_TH_U, s);
         stage_begin(h, ST_BLOCK, s);      // (the caller's bracket opened before the contraction: open it again here)
