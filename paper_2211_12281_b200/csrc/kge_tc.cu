@@ -938,6 +938,7 @@ __global__ void __launch_bounds__(32 * (2 + TC_EPI_WARPS), 1) tc_gemm_dual_kerne
         const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
         const int cgrp = (warp - 2) >> 2;              // which half of the tile's columns
         constexpr int COLS = BN / EG;
+        float4* st = reinterpret_cast<float4*>(base + (size_t)STAGES * STAGE_BYTES + 256) + (size_t)(warp - 2) * (TC_STORE_STAGE_BYTES / 16);
         for (int item = blockIdx.x, local = 0; item < total; item += gridDim.x, ++local) {
             const int buf = local % NACC;
             const bool ok = mbar_wait_bounded(&acc_full[buf], (local / NACC) & 1, wait_limit);
@@ -953,14 +954,23 @@ __global__ void __launch_bounds__(32 * (2 + TC_EPI_WARPS), 1) tc_gemm_dual_kerne
             for (int c0 = cgrp * COLS; c0 < (cgrp + 1) * COLS; c0 += 32) {
                 float v[32];
                 tmem_ld32(taddr + (uint32_t)(c0 - cgrp * COLS), v);
-                if (row >= q.M) continue;
                 const int ncol = it.n0 + c0;
-                float* dst = Cout + (int64_t)row * q.ldc + ncol;
-                if (q.fold > 0) dst += (int64_t)(ncol / q.fold) * (q.fold_stride - q.fold);     // (32-column pieces never straddle a fold)
-                if (ncol + 32 <= q.N && (q.ldc & 3) == 0) {
+                float* piece = Cout + ncol;                    // column ncol of row 0 of this item's slab
+                if (q.fold > 0) piece += (int64_t)(ncol / q.fold) * (q.fold_stride - q.fold);   // (32-column pieces never straddle a fold)
+                if (ncol + 32 <= q.N && (q.ldc & 3) == 0) {    // (warp-uniform) through shared memory: four rows' whole 128 bytes per store instruction
+                    const int sw = lane & 7, row0 = row - lane;
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-                } else {
+                    for (int i = 0; i < 8; ++i) st[lane * 8 + (i ^ sw)] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int r = j * 4 + (lane >> 3), c = lane & 7;
+                        const float4 val = st[r * 8 + (c ^ (r & 7))];
+                        if (row0 + r < q.M) *reinterpret_cast<float4*>(piece + (int64_t)(row0 + r) * q.ldc + 4 * c) = val;
+                    }
+                    __syncwarp();
+                } else if (row < q.M) {
+                    float* dst = piece + (int64_t)row * q.ldc;
 #pragma unroll
                     for (int i = 0; i < 32; ++i) if (ncol + i < q.N) dst[i] = v[i];
                 }
@@ -1372,7 +1382,8 @@ DualProb dual_prob(int M, int N, int K, int split, float* C, int64_t ldc, int bn
 template <int BN, bool PAIR = false>
 cudaError_t launch_gemm_dual(kge_handle* h, const unsigned char* tmA0, const unsigned char* tmB0, const unsigned char* tmA1,
                              const unsigned char* tmB1, const DualProb& q0, const DualProb& q1, cudaStream_t s) {
-    constexpr size_t smem = PAIR ? 1024 + (size_t)3 * (tc_stage_bytes(BN) + TC_A_BYTES) + 256 : tc_smem_bytes(BN);
+    constexpr size_t smem = (PAIR ? 1024 + (size_t)3 * (tc_stage_bytes(BN) + TC_A_BYTES) + 256 : tc_smem_bytes(BN)) +
+                            (size_t)TC_EPI_WARPS * TC_STORE_STAGE_BYTES;      // + the epilogue warps' store staging
     static DeviceOnce configured;
     const cudaError_t e = once_per_device(configured, [] {
         return cudaFuncSetAttribute(tc_gemm_dual_kernel<BN, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
