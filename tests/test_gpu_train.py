@@ -311,14 +311,15 @@ def test_transh_l1_row_widths(oracle64, d):
 
 
 @pytest.mark.parametrize("p,d,B,N", [(1, 128, 96, 80), (2, 128, 200, 300), (1, 128, 1024, 1024), (1, 256, 132, 200), (2, 96, 64, 130),
-                                     (1, 64, 260, 64), (1, 160, 36, 40), (2, 32, 8, 16)])
+                                     (1, 64, 260, 64), (1, 160, 36, 40), (2, 32, 8, 16), (1, 512, 68, 72), (2, 384, 36, 136)])
 def test_transh_tensor_core_contractions(oracle64, p, d, B, N):
     """TransH on the fp32 path with its three dense contractions forced onto the tensor cores (u = w.t from
     three-term bf16 splits, six products; the backward's two sums with per-pair coefficients from two-term
     splits, four products): the fp32 tolerances hold.  Shapes: a single ragged
     tile; ragged rows and columns; four K splits; rows of two 128-float slabs (two column tiles); a row width that
     leaves the tile's last 64 columns outside the operand; 128-column tiles; a fold of the output columns that is no
-    multiple of 64; a block smaller than one slice of the contraction index."""
+    multiple of 64; a block smaller than one slice of the contraction index; the widest rows (four column tiles of
+    the folded output, four column slabs in the CUDA-core kernels); three column tiles."""
     prob = Problem(E=3000, R=6, T=30000, d=d, score="transh", p_norm=p, loss="logsigmoid", B=B, N=N, P=2,
                    gamma=6.0, adv_temp=0.5, lr=0.05, graph_seed=21, relation_zipf=1.0, contract=1)
     _run(oracle64, prob, steps=2)
