@@ -466,9 +466,12 @@ struct GroupReduce {
 // dL/dF written back with put(i, g).
 struct StridedRow {    // scores in shared or global memory, covered as t0, t0 + stride, ...
     const float* row; float* out; int t0, stride, n;
+    float* scratch;        // the staged copy of the row when it may be overwritten (shared memory), else NULL
     __device__ __forceinline__ int count() const { return n > t0 ? (n - t0 + stride - 1) / stride : 0; }
     __device__ __forceinline__ float get(int i) const { return row[t0 + i * stride]; }
     __device__ __forceinline__ void put(int i, float g) { out[t0 + i * stride] = g; }
+    __device__ __forceinline__ bool can_keep() const { return scratch != nullptr; }
+    __device__ __forceinline__ void keep(int i, float v) { scratch[t0 + i * stride] = v; }
 };
 template <int V4>      // scores in registers: V4 float4 per lane, the row is 128 * V4 long
 struct RegisterRow {
@@ -476,6 +479,8 @@ struct RegisterRow {
     __device__ __forceinline__ constexpr int count() const { return 4 * V4; }
     __device__ __forceinline__ float get(int i) const { return reinterpret_cast<const float*>(&f[i >> 2])[i & 3]; }
     __device__ __forceinline__ void put(int i, float v) { reinterpret_cast<float*>(&g[i >> 2])[i & 3] = v; }
+    __device__ __forceinline__ constexpr bool can_keep() const { return false; }
+    __device__ __forceinline__ void keep(int, float) {}
 };
 
 // Loss and dL/dF of positive b over the calling threads' shares of the row; `lead` marks the
@@ -491,18 +496,39 @@ __device__ __forceinline__ void loss_row(const TrainParams& p, int b, Row& row, 
     if (p.loss == KGE_LOSS_LOGSIGMOID) {
         const float a = p.adv_temp, gamma = p.gamma;
         float m = 0.f, z = (float)N;
+        // Temperature exactly 1, a staged row and exp(gamma + m) finite: the weight's exponential e = exp(f - m) is kept in
+        // the row's place, and exp(gamma + f) = K e with K = exp(gamma + m) gives the loss term and its derivative from it:
+        // log(1 + K e) and K e / (1 + K e), three special-function instructions per score instead of five.
+        bool shared_exp = false;
         if (a > 0.f) {
             float lm = -INFINITY;
 #pragma unroll
             for (int i = 0; i < cnt; ++i) lm = fmaxf(lm, a * row.get(i));
             m = red.max(lm);
+            shared_exp = a == 1.f && !l2 && row.can_keep() && gamma + m <= 80.f;      // (the same for every thread of the row)
             float lz = 0.f;
+            if (shared_exp) {
+                for (int i = 0; i < cnt; ++i) { const float e = __expf(row.get(i) - m); row.keep(i, e); lz += e; }
+            } else {
 #pragma unroll
-            for (int i = 0; i < cnt; ++i) lz += __expf(a * row.get(i) - m);
+                for (int i = 0; i < cnt; ++i) lz += __expf(a * row.get(i) - m);
+            }
             z = red.sum(lz);
         }
         const float invz = 1.f / z;
         float lacc = 0.f;
+        if (shared_exp) {
+            const float K = __expf(gamma + m);
+            for (int i = 0; i < cnt; ++i) {
+                const float e = row.get(i);                 // each thread reads back what it stored itself
+                const float t = K * e, r = __frcp_rn(1.f + t);
+                const float w = e * invz;
+                lacc += w * __logf(1.f + t);
+                const float g = ls * w * (t * r);
+                row.put(i, g);
+                gsum += g;
+            }
+        } else
 #pragma unroll
         for (int i = 0; i < cnt; ++i) {
             const float f = row.get(i);
@@ -573,7 +599,7 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_kernel(TrainParams p) {
         __syncthreads();
         row = rowbuf;
     }
-    StridedRow sr{row, Frow, tid, LOSS_THREADS, p.N};
+    StridedRow sr{row, Frow, tid, LOSS_THREADS, p.N, p.N <= LOSS_SMEM_FLOATS ? rowbuf : nullptr};
     loss_row(p, b, sr, tid == 0, BlockReduce{sm});
 }
 
@@ -590,7 +616,7 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_warp_kernel(TrainParams p) 
     float* row = rowbuf + (size_t)warp * p.N;
     stage_row(row, Frow, p.N, lane, 32);
     __syncwarp();
-    StridedRow sr{row, Frow, lane, 32, p.N};
+    StridedRow sr{row, Frow, lane, 32, p.N, row};
     loss_row(p, b, sr, lane == 0, WarpReduce{});
 }
 
