@@ -587,7 +587,7 @@ __device__ __forceinline__ void stage_row(float* dst, const float* src, int N, i
 
 // One CTA per positive: long rows.
 __global__ void __launch_bounds__(LOSS_THREADS) loss_kernel(TrainParams p) {
-    extern __shared__ __align__(16) float rowbuf[];
+    extern __shared__ __align__(128) float rowbuf[];
     __shared__ float sm[LOSS_THREADS / 32];
     const int b = blockIdx.x, tid = threadIdx.x;
     grid_dependency_wait();
@@ -595,8 +595,25 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_kernel(TrainParams p) {
     float* Frow = p.w.F + (int64_t)b * p.N;
     const float* row = Frow;
     if (p.N <= LOSS_SMEM_FLOATS) {
-        stage_row(rowbuf, Frow, p.N, tid, LOSS_THREADS);
-        __syncthreads();
+        if ((p.N & 3) == 0) {
+            // the whole row as one bulk copy (a loop of load-then-store pays one trip to memory per 4 KB)
+            __shared__ __align__(8) uint64_t bar;
+            if (tid == 0) {
+                mbar_init(&bar, 1);
+                mbar_init_fence();
+                mbar_arrive_expect_tx(&bar, (uint32_t)p.N * 4u);
+                bulk_g2s(rowbuf, Frow, (uint32_t)p.N * 4u, &bar);
+            }
+            __syncthreads();                 // the barrier is initialised before anyone tests it
+            const bool ok = mbar_wait_bounded(&bar, 0u, p.wait_limit);
+            if (!__syncthreads_and(ok)) {
+                if (tid == 0) { set_status(p.w.status, KGE_ERR_TIMEOUT); (void)mbar_wait_bounded(&bar, 0u, p.wait_limit); }
+                return;
+            }
+        } else {
+            stage_row(rowbuf, Frow, p.N, tid, LOSS_THREADS);
+            __syncthreads();
+        }
         row = rowbuf;
     }
     StridedRow sr{row, Frow, tid, LOSS_THREADS, p.N, p.N <= LOSS_SMEM_FLOATS ? rowbuf : nullptr};
