@@ -472,6 +472,12 @@ struct StridedRow {    // scores in shared or global memory, covered as t0, t0 +
     __device__ __forceinline__ void put(int i, float g) { out[t0 + i * stride] = g; }
     __device__ __forceinline__ bool can_keep() const { return scratch != nullptr; }
     __device__ __forceinline__ void keep(int i, float v) { scratch[t0 + i * stride] = v; }
+    // the same row four scores at a time (a staged row of n % 4 == 0 scores, 16-byte aligned on both sides)
+    __device__ __forceinline__ bool vec4() const { return scratch != nullptr && (n & 3) == 0; }
+    __device__ __forceinline__ int count4() const { const int n4 = n >> 2; return n4 > t0 ? (n4 - t0 + stride - 1) / stride : 0; }
+    __device__ __forceinline__ float4 get4(int i) const { return reinterpret_cast<const float4*>(row)[t0 + i * stride]; }
+    __device__ __forceinline__ void keep4(int i, float4 v) { reinterpret_cast<float4*>(scratch)[t0 + i * stride] = v; }
+    __device__ __forceinline__ void put4(int i, float4 g) { reinterpret_cast<float4*>(out)[t0 + i * stride] = g; }
 };
 template <int V4>      // scores in registers: V4 float4 per lane, the row is 128 * V4 long
 struct RegisterRow {
@@ -481,6 +487,11 @@ struct RegisterRow {
     __device__ __forceinline__ void put(int i, float v) { reinterpret_cast<float*>(&g[i >> 2])[i & 3] = v; }
     __device__ __forceinline__ constexpr bool can_keep() const { return false; }
     __device__ __forceinline__ void keep(int, float) {}
+    __device__ __forceinline__ constexpr bool vec4() const { return false; }
+    __device__ __forceinline__ constexpr int count4() const { return 0; }
+    __device__ __forceinline__ float4 get4(int) const { return make_float4(0.f, 0.f, 0.f, 0.f); }
+    __device__ __forceinline__ void keep4(int, float4) {}
+    __device__ __forceinline__ void put4(int, float4) {}
 };
 
 // Loss and dL/dF of positive b over the calling threads' shares of the row; `lead` marks the
@@ -501,13 +512,26 @@ __device__ __forceinline__ void loss_row(const TrainParams& p, int b, Row& row, 
         // log(1 + K e) and K e / (1 + K e), three special-function instructions per score instead of five.
         bool shared_exp = false;
         if (a > 0.f) {
+            const bool v4 = row.vec4();
+            const int cnt4 = row.count4();
             float lm = -INFINITY;
+            if (v4) {
+                for (int i = 0; i < cnt4; ++i) { const float4 f = row.get4(i); lm = fmaxf(fmaxf(lm, a * f.x), fmaxf(fmaxf(a * f.y, a * f.z), a * f.w)); }
+            } else {
 #pragma unroll
-            for (int i = 0; i < cnt; ++i) lm = fmaxf(lm, a * row.get(i));
+                for (int i = 0; i < cnt; ++i) lm = fmaxf(lm, a * row.get(i));
+            }
             m = red.max(lm);
             shared_exp = a == 1.f && !l2 && row.can_keep() && gamma + m <= 80.f;      // (the same for every thread of the row)
             float lz = 0.f;
-            if (shared_exp) {
+            if (shared_exp && v4) {
+                for (int i = 0; i < cnt4; ++i) {
+                    const float4 f = row.get4(i);
+                    const float4 e = make_float4(__expf(f.x - m), __expf(f.y - m), __expf(f.z - m), __expf(f.w - m));
+                    row.keep4(i, e);
+                    lz += (e.x + e.y) + (e.z + e.w);
+                }
+            } else if (shared_exp) {
                 for (int i = 0; i < cnt; ++i) { const float e = __expf(row.get(i) - m); row.keep(i, e); lz += e; }
             } else {
 #pragma unroll
@@ -517,14 +541,31 @@ __device__ __forceinline__ void loss_row(const TrainParams& p, int b, Row& row, 
         }
         const float invz = 1.f / z;
         float lacc = 0.f;
-        if (shared_exp) {
+        if (shared_exp && row.vec4()) {
+            const float K = __expf(gamma + m);
+            const int cnt4 = row.count4();
+            for (int i = 0; i < cnt4; ++i) {
+                const float4 e4 = row.get4(i);              // each thread reads back what it stored itself
+                const float ev[4] = {e4.x, e4.y, e4.z, e4.w};
+                float gv[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const float t = K * ev[c], t1 = 1.f + t;
+                    const float w = ev[c] * invz;
+                    lacc += w * __logf(t1);
+                    gv[c] = ls * w * __fdividef(t, t1);
+                    gsum += gv[c];
+                }
+                row.put4(i, make_float4(gv[0], gv[1], gv[2], gv[3]));
+            }
+        } else if (shared_exp) {
             const float K = __expf(gamma + m);
             for (int i = 0; i < cnt; ++i) {
                 const float e = row.get(i);                 // each thread reads back what it stored itself
-                const float t = K * e, r = __frcp_rn(1.f + t);
+                const float t = K * e, t1 = 1.f + t;
                 const float w = e * invz;
-                lacc += w * __logf(1.f + t);
-                const float g = ls * w * (t * r);
+                lacc += w * __logf(t1);
+                const float g = ls * w * __fdividef(t, t1);       // (approximate reciprocal: 1 ulp, as in the tensor-core epilogues)
                 row.put(i, g);
                 gsum += g;
             }
