@@ -620,7 +620,15 @@ __device__ __forceinline__ void loss_row(const TrainParams& p, int b, Row& row, 
 
 __device__ __forceinline__ void stage_row(float* dst, const float* src, int N, int t0, int stride) {
     if ((N & 3) == 0) {
-        for (int n = t0; n < (N >> 2); n += stride) reinterpret_cast<float4*>(dst)[n] = reinterpret_cast<const float4*>(src)[n];
+        // eight loads in flight before the first store (load-then-store one at a time pays a trip to memory per element)
+        const int n4 = N >> 2;
+        for (int n = t0; n < n4; n += 8 * stride) {
+            float4 v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { const int idx = n + i * stride; v[i] = idx < n4 ? reinterpret_cast<const float4*>(src)[idx] : make_float4(0.f, 0.f, 0.f, 0.f); }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { const int idx = n + i * stride; if (idx < n4) reinterpret_cast<float4*>(dst)[idx] = v[i]; }
+        }
     } else {
         for (int n = t0; n < N; n += stride) dst[n] = src[n];
     }
