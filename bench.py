@@ -553,14 +553,18 @@ def bench_training(ctx, name, w, cpu_seconds):
         for st, ncon in TH_TC_CONTRACTIONS.items():
             if st in per_stage_us:
                 roofs[st] = (ncon * 2.0 * elements / (ctx.peaks["bf16_tflops"] * 1e12) * 1e6, "tensor", {})
-    # the two memory-bound sub-steps: random row gathers and the sparse row update
+    # the memory-bound sub-steps: random row gathers, the loss pass over the stored score block, the sparse row update
     rel_bytes = B * 4 * kw_rel * (2 if w["score"] == "transh" else 1)
     build_bytes = (2 * B + N) * 4 * d + rel_bytes + (B + N) * 4 * d + ((B + N) * 2 * d if w.get("tc") else 0)
     state_per_row = {"sgd": 8 * d, "adagrad": 8 * d + 8, "adam": 24 * d}[w["opt"]]
     update_bytes = uniq * state_per_row + (2 * B + N) * 4 * d
     hbm = ctx.peaks["hbm_gbs"] * 1e9
     hbm_substeps = {}
-    for st, nbytes in (("build", build_bytes), ("update", update_bytes)):
+    # (CUDA-core paths keep the score block in memory: the loss kernel reads B N scores and writes B N derivatives)
+    loss_bytes = 0 if w.get("tc") else 8 * B * N
+    for st, nbytes in (("build", build_bytes), ("loss", loss_bytes), ("update", update_bytes)):
+        if nbytes <= 0:
+            continue
         if st in per_stage_us:
             gbs = nbytes / (per_stage_us[st] * 1e-6) / 1e9
             hbm_substeps[st] = {"bytes": int(nbytes), "us": per_stage_us[st], "gbs": gbs, "frac": gbs * 1e9 / hbm}
